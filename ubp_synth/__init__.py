@@ -1,0 +1,191 @@
+"""Seeded synthetic inputs for unaligned block-wise pruned (UBP) layers.
+
+This module only draws random data: masks whose ones form non-overlapping
+vertical runs of ``Nb`` output channels inside one input-channel column
+(the 1xN block of Section 3.1), dense weights, activations and biases.
+It performs none of the method's arithmetic (no packing, no products), so
+both the CPU oracle's tests and the CUDA path's tests can take their
+inputs from here without sharing any code of the method itself.
+
+Everything is a pure function of the integer seed (numpy PCG64).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional, Tuple
+
+import numpy as np
+
+__all__ = [
+    "block_budget", "random_block_starts", "mask_from_starts", "random_mask",
+    "Layer", "make_layer", "CONFIGS", "MBV1_CHAIN", "config_layers",
+]
+
+
+def block_budget(M: int, C: int, sparsity_pct: int, Nb: int) -> int:
+    """Number of kept blocks m = floor(M*C*(1-p)/Nb) (Section 3.1), with the
+    pruning rate given as an integer percentage so the floor is exact."""
+    return (M * C * (100 - sparsity_pct)) // (100 * Nb)
+
+
+def random_block_starts(M: int, C: int, Nb: int, m: int,
+                        rng: np.random.Generator,
+                        aligned: bool = False) -> List[np.ndarray]:
+    """Draw ``m`` block start rows spread over the ``C`` columns.
+
+    Column loads: ``m`` balls thrown uniformly at the columns, a ball that
+    lands on a column already holding floor(M/Nb) blocks is thrown again.
+    Inside a column holding ``c`` blocks the placement is uniform over all
+    non-overlapping placements: draw ``c`` distinct integers q_0<...<q_{c-1}
+    from [0, M - c*(Nb-1)) and start block t at q_t + t*(Nb-1).
+    With ``aligned`` the starts are instead distinct multiples of ``Nb``
+    (the aligned pattern the paper calls ABP).
+    Returns one sorted int64 array of start rows per column.
+    """
+    cap = M // Nb
+    if m > cap * C:
+        raise ValueError("more blocks requested than fit")
+    cnt = np.zeros(C, dtype=np.int64)
+    left = m
+    while left > 0:
+        js = rng.integers(0, C, size=left)
+        for j in js:
+            if cnt[j] < cap:
+                cnt[j] += 1
+                left -= 1
+    starts = []
+    for j in range(C):
+        c = int(cnt[j])
+        if aligned:
+            q = np.sort(rng.choice(cap, size=c, replace=False)).astype(np.int64)
+            starts.append(q * Nb)
+        else:
+            q = np.sort(rng.choice(M - c * (Nb - 1), size=c, replace=False)).astype(np.int64)
+            starts.append(q + np.arange(c, dtype=np.int64) * (Nb - 1))
+    return starts
+
+
+def mask_from_starts(M: int, C: int, Nb: int, starts: List[np.ndarray]) -> np.ndarray:
+    """0/1 mask [M][C] (uint8) with ones on rows i..i+Nb-1 of column j for
+    every start row i listed for column j."""
+    mask = np.zeros((M, C), dtype=np.uint8)
+    for j, s in enumerate(starts):
+        for i in s:
+            mask[int(i):int(i) + Nb, j] = 1
+    return mask
+
+
+def random_mask(M: int, C: int, Nb: int, sparsity_pct: int, seed: int,
+                aligned: bool = False) -> Tuple[np.ndarray, List[np.ndarray]]:
+    rng = np.random.Generator(np.random.PCG64(seed))
+    m = block_budget(M, C, sparsity_pct, Nb)
+    starts = random_block_starts(M, C, Nb, m, rng, aligned=aligned)
+    return mask_from_starts(M, C, Nb, starts), starts
+
+
+@dataclass
+class Layer:
+    """One synthetic UBP layer. ``W`` is [M][C][R] (R = taps: 1 or 9),
+    ``mask`` is [M][C]; ``X`` is [C][Nc] for R == 1 and [C][B][H][Wd] for the
+    3x3 case (channel-major activations, columns n = (b, y, x))."""
+    name: str
+    M: int
+    C: int
+    R: int
+    Nb: int
+    sparsity_pct: int
+    m: int
+    W: np.ndarray
+    mask: np.ndarray
+    X: np.ndarray
+    bias: Optional[np.ndarray]
+    relu: bool
+    B: int = 1
+    H: int = 1
+    Wd: int = 1
+    starts: List[np.ndarray] = field(default_factory=list, repr=False)
+
+    @property
+    def Nc(self) -> int:
+        return int(self.X.size // self.C)
+
+    @property
+    def surviving_macs(self) -> int:
+        return self.m * self.Nb * self.R * self.Nc
+
+
+def make_layer(name: str, M: int, C: int, Nb: int, sparsity_pct: int, seed: int, *,
+               Nc: Optional[int] = None, B: int = 1, H: int = 1, Wd: int = 1,
+               R: int = 1, w_dist: str = "normal", w_scale: float = 0.05,
+               x_dist: str = "absnormal", bias: bool = True, relu: bool = True,
+               aligned: bool = False, make_x: bool = True) -> Layer:
+    """Build one seeded layer. ``w_dist``: 'uniform' -> U[-w_scale, w_scale],
+    'normal' -> N(0, w_scale). ``x_dist``: 'normal' -> N(0,1),
+    'absnormal' -> |N(0,1)| (post-ReLU-like). Bias ~ N(0, 0.1)."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    m = block_budget(M, C, sparsity_pct, Nb)
+    starts = random_block_starts(M, C, Nb, m, rng, aligned=aligned)
+    mask = mask_from_starts(M, C, Nb, starts)
+    if w_dist == "uniform":
+        W = rng.uniform(-w_scale, w_scale, size=(M, C, R)).astype(np.float32)
+    else:
+        W = (rng.standard_normal(size=(M, C, R), dtype=np.float32) * np.float32(w_scale)).astype(np.float32)
+    if R == 1:
+        ncols = Nc if Nc is not None else B * H * Wd
+        xshape = (C, ncols)
+    else:
+        xshape = (C, B, H, Wd)
+    if make_x:
+        X = rng.standard_normal(size=xshape, dtype=np.float32)
+        if x_dist == "absnormal":
+            np.abs(X, out=X)
+    else:
+        X = np.zeros((C, 0), dtype=np.float32)
+    b = (rng.standard_normal(size=(M,), dtype=np.float32) * np.float32(0.1)).astype(np.float32) if bias else None
+    return Layer(name, M, C, R, Nb, sparsity_pct, m, W, mask, X, b, relu, B, H, Wd, starts)
+
+
+# (C_in, C_out, spatial) of the 13 pointwise layers of a MobileNetV1-shaped
+# network at 224x224 input.
+MBV1_CHAIN = [(32, 64, 112), (64, 128, 56), (128, 128, 56), (128, 256, 28),
+              (256, 256, 28), (256, 512, 14)] + [(512, 512, 14)] * 5 + \
+             [(512, 1024, 7), (1024, 1024, 7)]
+
+CONFIGS = {
+    "fc64": "FC 64x64, 1x4 blocks, 50 % sparsity, X 64x256 ~ N(0,1), bias, no ReLU",
+    "mbv1_pw512": "pointwise 512->512 at 14x14, batch 32 (M=K=512, Nc=6272), 1x4, 70 %, bias+ReLU",
+    "r50_3x3": "3x3 conv 256->256 at 14x14, batch 64, pad 1, blocks 8x1x3x3, 80 %",
+    "sweep": "M=K=2048, Nc=8192; Nb in {2,4,8,16} x sparsity in {50,70,80,90}",
+    "mbv1_chain": "13 pointwise layers of MobileNetV1, batch 64, 1x4, 80 %, bias+ReLU",
+}
+
+
+def config_layers(cfg: str, *, batch: Optional[int] = None, Nb: Optional[int] = None,
+                  sparsity_pct: Optional[int] = None, index: int = 0,
+                  make_x: bool = True) -> List[Layer]:
+    """Layers of one named configuration; seed = 1000*config_number + index."""
+    if cfg == "fc64":
+        return [make_layer("fc64", 64, 64, 4, 50, 1000 + index, Nc=256, w_dist="uniform",
+                           w_scale=1.0, x_dist="normal", bias=True, relu=False, make_x=make_x)]
+    if cfg == "mbv1_pw512":
+        b = 32 if batch is None else batch
+        return [make_layer("mbv1_pw512", 512, 512, 4, 70, 2000 + index, B=b, H=14, Wd=14,
+                           w_scale=0.05, bias=True, relu=True, make_x=make_x)]
+    if cfg == "r50_3x3":
+        b = 64 if batch is None else batch
+        return [make_layer("r50_3x3", 256, 256, 8, 80, 3000 + index, B=b, H=14, Wd=14, R=9,
+                           w_scale=0.02, bias=True, relu=True, make_x=make_x)]
+    if cfg == "sweep":
+        nb = 4 if Nb is None else Nb
+        sp = 70 if sparsity_pct is None else sparsity_pct
+        idx = [2, 4, 8, 16].index(nb) * 4 + [50, 70, 80, 90].index(sp)
+        return [make_layer(f"sweep_nb{nb}_p{sp}", 2048, 2048, nb, sp, 4000 + idx, Nc=8192,
+                           w_scale=0.02, x_dist="normal", bias=False, relu=False, make_x=make_x)]
+    if cfg == "mbv1_chain":
+        b = 64 if batch is None else batch
+        out = []
+        for li, (ci, co, hw) in enumerate(MBV1_CHAIN):
+            out.append(make_layer(f"mbv1_L{li + 1}", co, ci, 4, 80, 5000 + li, B=b, H=hw, Wd=hw,
+                                  w_scale=0.05, bias=True, relu=True, make_x=make_x))
+        return out
+    raise KeyError(cfg)
