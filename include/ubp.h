@@ -1,0 +1,175 @@
+/*
+ * ubp.h -- C ABI of the B200 library for unaligned block-wise pruned (UBP) layers.
+ *
+ * The layer (Section 3.1 of the paper): a weight W[M][C][R] (M output channels,
+ * C input channels, R = kh*kw taps) keeps only "blocks": Nb consecutive output
+ * channels i..i+Nb-1 at one input channel j, all R taps, starting at ANY row
+ * i <= M-Nb, blocks of one input channel never overlapping (Eq. 1, Eq. 2).
+ * Inference computes Y = act(Wm * X + bias) with Wm the masked weight.
+ *
+ * Conventions for every entry point
+ *   - returns 0 (UBP_OK) or a negative ubp_status; never throws, aborts, prints
+ *     or synchronises the device (exceptions are named below);
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA device
+ *     memory of the current device; the caller owns every buffer it passes;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream); device
+ *     work is enqueued on it and the call returns without waiting;
+ *   - inputs are assumed finite; input and output buffers must not overlap.
+ */
+#ifndef UBP_H_
+#define UBP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    UBP_OK = 0,
+    UBP_E_ARG = -1,       /* null pointer, non-positive size, Nb > M, bad stride ...        */
+    UBP_E_RAGGED = -2,    /* a run of ones in a mask column is not a whole number of blocks */
+    UBP_E_SPACE = -3,     /* caller buffer too small / host allocation failed               */
+    UBP_E_FORMAT = -4,    /* blob or plan is not what it claims to be                       */
+    UBP_E_CUDA = -5,      /* a CUDA runtime/driver call failed (see ubp_last_cuda_error)    */
+    UBP_E_UNSUPPORTED = -6,
+    UBP_E_DEVICE = -7     /* a kernel reported a bounded wait that ran out                  */
+} ubp_status;
+
+const char *ubp_strerror(int status);
+/* last cudaError_t seen by this thread inside the library (0 if none) */
+int ubp_last_cuda_error(void);
+
+/* ------------------------------------------------------------------ format
+ * Canonical packed form of a UBP weight (Section 4.2: "sparse weight format
+ * for WROS"): blocks are grouped by the output row they START at --
+ *   indptr [M+1]  blocks starting at row i are indptr[i] .. indptr[i+1]-1
+ *   indices[m]    input channel j of each block, ascending inside a start row
+ *   values [m][Nb][R]  the block's weights, ROTATED: the weight of output row
+ *                 rho sits in slot rho mod Nb (so a kernel that keeps Nb
+ *                 stationary accumulators never shuffles them); taps in OIHW
+ *                 order (tap = 3*r + s for a 3x3 kernel)
+ * Blob = 64-byte little-endian header {"UBP1", u32 version=1, i32 M, C, R, Nb, m,
+ * u32 flags(bit0 = rotated)} followed by the three arrays, each starting on a
+ * 64-byte boundary, padding bytes zero. The blob is a pure function of
+ * (W, mask, Nb); weights are copied bit for bit.
+ */
+
+/* ubp_pack (host): mask[M][C] of 0/1 + W[M][C][R] -> blob.
+ * The mask is decoded by cutting every run of ones in a column into Nb-row
+ * blocks from the run's first row (the block-division step, Algorithm 2).
+ * blob == NULL: only *blob_len is written (size query).
+ * Errors: UBP_E_ARG (null, sizes, Nb > M, mask value > 1), UBP_E_RAGGED,
+ * UBP_E_SPACE (blob_cap < needed; *blob_len still holds the needed size). */
+int ubp_pack(const float *W, const uint8_t *mask, int M, int C, int R, int Nb,
+             void *blob, size_t blob_cap, size_t *blob_len);
+
+/* ubp_unpack (host): blob -> W_out[M][C][R] (zero where pruned) and
+ * mask_out[M][C]; either output may be NULL. UBP_E_FORMAT on a bad blob. */
+int ubp_unpack(const void *blob, size_t len, float *W_out, uint8_t *mask_out);
+
+typedef struct {
+    int32_t M, C, R, Nb, m;
+    const int32_t *indptr;   /* point into the blob */
+    const int32_t *indices;
+    const float *values;
+} ubp_view_t;
+
+/* ubp_blob_view (host): validate a blob and expose its arrays (no copy). */
+int ubp_blob_view(const void *blob, size_t len, ubp_view_t *view);
+
+/* ------------------------------------------------------------------ plan
+ * The kernels do not walk the canonical arrays directly: a plan is the same
+ * blocks re-bucketed for the GPU (by row panel, input-channel tile and start
+ * offset inside the panel; a block that crosses a panel boundary is listed in
+ * both panels, each taking its own rows -- the GPU answer to the "overlapped
+ * output tiles" of Section 3.3). The plan lives in a device buffer the CALLER
+ * allocates; the library owns only the small host handle.
+ *
+ * variant: 0 = choose from the layer shape; > 0 = a specific kernel
+ * configuration (ubp_variant_count / ubp_variant_describe list them), meant
+ * for measuring configurations against each other.
+ */
+typedef struct ubp_plan ubp_plan_t;
+
+int ubp_variant_count(void);
+/* text description of variant id (1-based) into buf; UBP_E_ARG if out of range */
+int ubp_variant_describe(int variant, char *buf, size_t cap);
+
+/* bytes of device memory a plan of this blob needs (host; no CUDA call) */
+int ubp_plan_size(const void *blob, size_t len, int variant, size_t *dev_bytes);
+
+/* ubp_plan_image (host; no CUDA call): write the exact bytes that
+ * ubp_plan_build would upload into host_buf (>= ubp_plan_size bytes). Meant for
+ * inspection and for checking the plan builder without a GPU. Image layout:
+ *   [0,256) header, int32 status word at byte 0;
+ *   [256,..) uint32 group_off[nkt*NG + 1] in 16-byte units, groups in (tile, row group) order;
+ *   group: uint32 poff[WR+1] (padded to 16), then per panel
+ *          uint16 fo[F+1] (F = panel_rows + nbk - 1 start offsets, padded to 16),
+ *          uint16 jl[n] (input channel inside the tile, padded to 16),
+ *          float  w[n][nbk][R] (weights in row order, i.e. with the rotation undone).
+ * geom receives {nbk, panel_rows, k_tile, WR, dupw, nkt, NP, NG}. */
+int ubp_plan_image(const void *blob, size_t len, int variant, void *host_buf, size_t cap, int32_t geom[8]);
+
+/* Build the plan on the host, copy it into dev_buf (device, >= ubp_plan_size
+ * bytes, 256-byte aligned) with one cudaMemcpyAsync on `stream`, return the
+ * handle. The handle keeps its host copy until ubp_plan_free, so the copy may
+ * still be in flight when this returns. */
+int ubp_plan_build(const void *blob, size_t len, int variant, void *dev_buf, size_t dev_bytes,
+                   void *stream, ubp_plan_t **plan);
+void ubp_plan_free(ubp_plan_t *plan);
+
+typedef struct {
+    int32_t M, C, R, Nb, m;      /* layer                                         */
+    int32_t variant;             /* configuration actually chosen                 */
+    int32_t panel_rows, k_tile;  /* plan geometry                                 */
+    int64_t entries;             /* block entries in the plan (incl. duplicates)  */
+    int64_t dev_bytes;
+} ubp_plan_info_t;
+int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info);
+
+/* Read the plan's device status word: blocks until `stream` has finished
+ * (cudaStreamSynchronize), then returns UBP_OK or UBP_E_DEVICE if a kernel
+ * launched with this plan gave up on a bounded wait. */
+int ubp_plan_check(const ubp_plan_t *plan, void *stream);
+
+/* ------------------------------------------------------------------ compute
+ * ubp_spmm: Y[M][Nc] = act(Wm[M][C] * X[C][Nc] + bias), the 1x1 / fully
+ * connected case (R == 1), the weight-rotating output-stationary product of
+ * Section 4.2 re-organised for the GPU: accumulators stay in registers for
+ * the whole reduction and each output is written once.
+ *   X    device, row c at X + c*ldx, Nc contiguous floats (ldx >= Nc)
+ *   bias device [M] or NULL;  relu != 0 applies max(.,0)
+ *   Y    device, row o at Y + o*ldy (ldy >= Nc)
+ * Fast path needs X, Y 16-byte aligned and ldx, ldy multiples of 4; otherwise a
+ * slower kernel is used (same result). Nc == 0 is a no-op.
+ * fp32 multiply-add, fp32 accumulation, fixed summation order (bitwise
+ * reproducible run to run). */
+int ubp_spmm(const ubp_plan_t *plan, const float *X, int64_t ldx, int64_t Nc,
+             const float *bias, int relu, float *Y, int64_t ldy, void *stream);
+
+/* ubp_conv1x1: 1x1 stride-1 convolution = ubp_spmm over columns n = (b, y, x).
+ * Element strides: in[b][c][y][x] at in + b*in_stride_b + c*in_stride_c + y*Wd + x
+ * (NCHW: (C*H*W, H*W); channel-major "CNHW": (H*W, B*H*W)); same for out.
+ * If both batch strides equal H*W all images form one product with
+ * Nc = B*H*W; otherwise one product per image. */
+int ubp_conv1x1(const ubp_plan_t *plan, const float *in, int B, int H, int Wd,
+                int64_t in_stride_b, int64_t in_stride_c,
+                const float *bias, int relu,
+                float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);
+
+/* ubp_conv3x3_implicit: 3x3, stride 1, zero padding 1, cross-correlation; the
+ * plan must come from a blob with R == 9 (a block = Nb output channels x one
+ * input channel x all nine taps, Section 3.1). The K = 9*C lowered matrix is
+ * never formed: input planes are staged once with their halo and every tap
+ * reads them in place. Same strides as ubp_conv1x1. */
+int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, int Wd,
+                         int64_t in_stride_b, int64_t in_stride_c,
+                         const float *bias, int relu,
+                         float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UBP_H_ */

@@ -1,0 +1,209 @@
+// extern "C" surface of the library (declared in include/ubp.h): argument
+// checks, plan life cycle, and dispatch to the launchers. No device
+// synchronisation except in ubp_plan_check.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "ubp_internal.h"
+
+namespace ubp {
+static thread_local int g_last_cuda = 0;
+void set_last_cuda_error(int e) { g_last_cuda = e; }
+}  // namespace ubp
+
+static const uint32_t kPlanMagic = 0x50504255u;   // "UBPP"
+
+extern "C" {
+
+const char *ubp_strerror(int status)
+{
+    switch (status) {
+        case UBP_OK: return "ok";
+        case UBP_E_ARG: return "invalid argument";
+        case UBP_E_RAGGED: return "mask has a run of ones that is not a whole number of blocks";
+        case UBP_E_SPACE: return "buffer too small or out of host memory";
+        case UBP_E_FORMAT: return "malformed blob or plan";
+        case UBP_E_CUDA: return "CUDA call failed";
+        case UBP_E_UNSUPPORTED: return "unsupported configuration";
+        case UBP_E_DEVICE: return "a kernel gave up on a bounded wait";
+        default: return "unknown status";
+    }
+}
+
+int ubp_last_cuda_error(void) { return ubp::g_last_cuda; }
+
+int ubp_pack(const float *W, const uint8_t *mask, int M, int C, int R, int Nb,
+             void *blob, size_t blob_cap, size_t *blob_len)
+{
+    try { return ubp::pack(W, mask, M, C, R, Nb, blob, blob_cap, blob_len); }
+    catch (const std::bad_alloc &) { return UBP_E_SPACE; }
+}
+
+int ubp_unpack(const void *blob, size_t len, float *W_out, uint8_t *mask_out)
+{
+    try { return ubp::unpack(blob, len, W_out, mask_out); }
+    catch (const std::bad_alloc &) { return UBP_E_SPACE; }
+}
+
+int ubp_blob_view(const void *blob, size_t len, ubp_view_t *view) { return ubp::blob_view(blob, len, view); }
+
+int ubp_variant_count(void) { return (int)ubp::kernel_cfgs().size(); }
+
+int ubp_variant_describe(int variant, char *buf, size_t cap)
+{
+    const ubp::KernelCfg *c = ubp::find_cfg(variant);
+    if (!c || !buf || cap == 0) return UBP_E_ARG;
+    std::snprintf(buf, cap, "%s nbk=%d panel=%d cols/warp=%d warps=%dx%d ktile=%d%s",
+                  c->kind == 0 ? "spmm" : "conv3x3", c->nbk, c->P, 128 * c->V, c->WR, c->WC, c->KT,
+                  c->dupw ? " dupw" : "");
+    return UBP_OK;
+}
+
+static int resolve_cfg(const ubp_view_t &v, int variant, const ubp::KernelCfg **cfg)
+{
+    const ubp::KernelCfg *c = variant == 0 ? ubp::auto_cfg(v.M, v.C, v.R, v.Nb, v.m) : ubp::find_cfg(variant);
+    if (!c) return variant == 0 ? UBP_E_UNSUPPORTED : UBP_E_ARG;
+    *cfg = c;
+    return UBP_OK;
+}
+
+int ubp_plan_size(const void *blob, size_t len, int variant, size_t *dev_bytes)
+{
+    if (!dev_bytes) return UBP_E_ARG;
+    ubp_view_t v;
+    int rc = ubp::blob_view(blob, len, &v);
+    if (rc) return rc;
+    const ubp::KernelCfg *cfg;
+    if ((rc = resolve_cfg(v, variant, &cfg))) return rc;
+    try {
+        ubp::PlanImage img;
+        return ubp::build_plan_image(v, *cfg, true, img, dev_bytes);
+    } catch (const std::bad_alloc &) { return UBP_E_SPACE; }
+}
+
+int ubp_plan_image(const void *blob, size_t len, int variant, void *host_buf, size_t cap, int32_t geom[8])
+{
+    if (!host_buf || !geom) return UBP_E_ARG;
+    ubp_view_t v;
+    int rc = ubp::blob_view(blob, len, &v);
+    if (rc) return rc;
+    const ubp::KernelCfg *cfg;
+    if ((rc = resolve_cfg(v, variant, &cfg))) return rc;
+    try {
+        ubp::PlanImage img;
+        size_t need = 0;
+        if ((rc = ubp::build_plan_image(v, *cfg, false, img, &need))) return rc;
+        if (cap < need) return UBP_E_SPACE;
+        std::memcpy(host_buf, img.bytes.data(), need);
+        geom[0] = cfg->nbk; geom[1] = cfg->P; geom[2] = cfg->KT; geom[3] = cfg->WR; geom[4] = cfg->dupw;
+        geom[5] = img.nkt; geom[6] = img.NP; geom[7] = img.NG;
+    } catch (const std::bad_alloc &) { return UBP_E_SPACE; }
+    return UBP_OK;
+}
+
+int ubp_plan_build(const void *blob, size_t len, int variant, void *dev_buf, size_t dev_bytes,
+                   void *stream, ubp_plan_t **plan)
+{
+    if (!plan || !dev_buf || (reinterpret_cast<uintptr_t>(dev_buf) & 255)) return UBP_E_ARG;
+    *plan = nullptr;
+    ubp_view_t v;
+    int rc = ubp::blob_view(blob, len, &v);
+    if (rc) return rc;
+    const ubp::KernelCfg *cfg;
+    if ((rc = resolve_cfg(v, variant, &cfg))) return rc;
+    ubp_plan *p = nullptr;
+    try {
+        p = new ubp_plan();
+        p->magic = kPlanMagic;
+        p->dims = v; p->dims.indptr = nullptr; p->dims.indices = nullptr; p->dims.values = nullptr;
+        p->cfg = *cfg;
+        size_t need = 0;
+        rc = ubp::build_plan_image(v, *cfg, false, p->img, &need);
+        if (!rc && dev_bytes < need) rc = UBP_E_SPACE;
+        if (rc) { delete p; return rc; }
+        p->dev = dev_buf; p->dev_bytes = need;
+    } catch (const std::bad_alloc &) { delete p; return UBP_E_SPACE; }
+    cudaError_t e = cudaMemcpyAsync(dev_buf, p->img.bytes.data(), p->img.bytes.size(), cudaMemcpyHostToDevice,
+                                    static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { ubp::set_last_cuda_error((int)e); delete p; return UBP_E_CUDA; }
+    *plan = p;
+    return UBP_OK;
+}
+
+void ubp_plan_free(ubp_plan_t *plan)
+{
+    if (plan && plan->magic == kPlanMagic) { plan->magic = 0; delete plan; }
+}
+
+int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info)
+{
+    if (!plan || plan->magic != kPlanMagic || !info) return UBP_E_ARG;
+    info->M = plan->dims.M; info->C = plan->dims.C; info->R = plan->dims.R; info->Nb = plan->dims.Nb; info->m = plan->dims.m;
+    info->variant = plan->cfg.id; info->panel_rows = plan->cfg.P; info->k_tile = plan->cfg.KT;
+    info->entries = plan->img.entries; info->dev_bytes = (int64_t)plan->dev_bytes;
+    return UBP_OK;
+}
+
+int ubp_plan_check(const ubp_plan_t *plan, void *stream)
+{
+    if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
+    int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, plan->dev, sizeof word, cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { ubp::set_last_cuda_error((int)e); return UBP_E_CUDA; }
+    return word == 0 ? UBP_OK : UBP_E_DEVICE;
+}
+
+int ubp_spmm(const ubp_plan_t *plan, const float *X, int64_t ldx, int64_t Nc,
+             const float *bias, int relu, float *Y, int64_t ldy, void *stream)
+{
+    if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
+    if (plan->dims.R != 1 || plan->cfg.kind != 0) return UBP_E_ARG;
+    if (Nc < 0) return UBP_E_ARG;
+    if (Nc == 0) return UBP_OK;
+    if (!X || !Y || ldx < Nc || ldy < Nc) return UBP_E_ARG;
+    return ubp::launch_spmm(plan, X, ldx, Nc, bias, relu, Y, ldy, stream);
+}
+
+int ubp_conv1x1(const ubp_plan_t *plan, const float *in, int B, int H, int Wd,
+                int64_t in_stride_b, int64_t in_stride_c, const float *bias, int relu,
+                float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream)
+{
+    if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
+    if (plan->dims.R != 1 || plan->cfg.kind != 0) return UBP_E_ARG;
+    if (B < 0 || H <= 0 || Wd <= 0) return UBP_E_ARG;
+    if (B == 0) return UBP_OK;
+    if (!in || !out) return UBP_E_ARG;
+    const int64_t hw = (int64_t)H * Wd;
+    if (in_stride_b == hw && out_stride_b == hw) {          // channel-major: one product over all images
+        if (in_stride_c < hw * B || out_stride_c < hw * B) return UBP_E_ARG;
+        return ubp::launch_spmm(plan, in, in_stride_c, hw * B, bias, relu, out, out_stride_c, stream);
+    }
+    if (in_stride_c < hw || out_stride_c < hw || in_stride_b < 0 || out_stride_b < 0) return UBP_E_ARG;
+    for (int b = 0; b < B; ++b) {                            // one product per image
+        int rc = ubp::launch_spmm(plan, in + (size_t)b * in_stride_b, in_stride_c, hw, bias, relu,
+                                  out + (size_t)b * out_stride_b, out_stride_c, stream);
+        if (rc) return rc;
+    }
+    return UBP_OK;
+}
+
+int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, int Wd,
+                         int64_t in_stride_b, int64_t in_stride_c, const float *bias, int relu,
+                         float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream)
+{
+    if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
+    if (plan->dims.R != 9 || plan->cfg.kind != 1) return UBP_E_ARG;
+    if (B < 0 || H <= 0 || Wd <= 0) return UBP_E_ARG;
+    if (B == 0) return UBP_OK;
+    if (!in || !out) return UBP_E_ARG;
+    const int64_t hw = (int64_t)H * Wd;
+    if (in_stride_c < hw || out_stride_c < hw || in_stride_b < 0 || out_stride_b < 0) return UBP_E_ARG;
+    return ubp::launch_conv3x3(plan, in, B, H, Wd, in_stride_b, in_stride_c, bias, relu, out, out_stride_b,
+                               out_stride_c, stream);
+}
+
+}  // extern "C"

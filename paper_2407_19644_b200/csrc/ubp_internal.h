@@ -1,0 +1,74 @@
+// Internal declarations shared by the library's translation units.
+#ifndef UBP_INTERNAL_H_
+#define UBP_INTERNAL_H_
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "ubp.h"
+
+namespace ubp {
+
+// ---- format (ubp_format.cpp)
+int pack(const float *W, const uint8_t *mask, int M, int C, int R, int Nb,
+         void *blob, size_t blob_cap, size_t *blob_len);
+int unpack(const void *blob, size_t len, float *W_out, uint8_t *mask_out);
+int blob_view(const void *blob, size_t len, ubp_view_t *v);
+
+// ---- kernel configurations (ubp_plan.cpp)
+// A configuration fixes how blocks are bucketed (plan geometry) and which
+// kernel instantiation consumes them.
+struct KernelCfg {
+    int id;        // 1-based variant id
+    int kind;      // 0 = 1x1 product (R == 1), 1 = implicit 3x3 (R == 9)
+    int nbk;       // rows per plan entry; divides the layer's Nb
+    int P;         // rows per panel (one warp's output rows)
+    int V;         // float4 column groups per lane (a warp covers 128*V columns)
+    int WR, WC;    // warps per CTA along rows / columns
+    int KT;        // input channels per staged tile
+    int dupw;      // weights stored twice (w, w) for packed f32x2 multiply-add
+};
+const std::vector<KernelCfg> &kernel_cfgs();
+const KernelCfg *find_cfg(int id);
+// pick a configuration for a layer (variant == 0)
+const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m);
+
+// ---- plan (ubp_plan.cpp)
+// Device image layout (all offsets from the image base, which is 256-byte aligned):
+//   [0, 256)            header; int32 status word at byte 0 (0 = fine)
+//   [256, ...)          uint32 group_off[nkt * NG + 1], in 16-byte units from the base
+//   groups in (kt, g) order, each 16-byte aligned:
+//       uint32 poff[WR + 1]            byte offsets of the panel sub-segments from the group start
+//       per panel: uint16 fo[F + 1]    entry offsets per fragment (F = P + nbk - 1), padded to 16
+//                  uint16 jl[n]        input channel inside the tile, padded to 16
+//                  float  w[n][nbk][R][dup]   un-rotated weights of the entry, padded to 16
+struct PlanImage {
+    std::vector<uint8_t> bytes;
+    int nkt = 0, NP = 0, NG = 0, F = 0;
+    int64_t entries = 0;
+    uint32_t max_group_bytes = 0;
+};
+int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only, PlanImage &img, size_t *bytes);
+
+}  // namespace ubp
+
+struct ubp_plan {
+    uint32_t magic;                 // 'UBPP'
+    ubp_view_t dims;                // M, C, R, Nb, m (pointers unused)
+    ubp::KernelCfg cfg;
+    ubp::PlanImage img;             // host copy (kept until free)
+    void *dev;                      // caller's device buffer
+    size_t dev_bytes;
+};
+
+// ---- launches (ubp_kernels.cu)
+namespace ubp {
+int launch_spmm(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                float *Y, int64_t ldy, void *stream);
+int launch_conv3x3(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
+                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream);
+void set_last_cuda_error(int e);
+}
+
+#endif

@@ -1,0 +1,577 @@
+// CUDA kernels (sm_100a) for Y = act(Wm X + bias) on unaligned block-wise
+// pruned weights, and their launchers.
+//
+// Dataflow (the output-stationary idea of Section 4.2, re-organised for SIMT):
+// a warp owns a panel of P output rows x (32 lanes x 4V columns) and keeps it in
+// registers for the whole reduction over input channels; the CTA's warps share
+// one staged activation tile X[k0:k0+KT, strip] per pipeline stage. Blocks are
+// consumed from the plan, bucketed by start offset inside the panel, and the
+// kernel is statically unrolled over that offset, so every accumulator index is
+// a compile-time constant (registers cannot be indexed at run time; this plays
+// the role the weight rotation plays on the paper's SIMD register file).
+//
+// Staging: one producer warp issues, per stage, a TMA tensor copy of the X tile
+// and a bulk copy of the plan group into shared memory, completing on an
+// mbarrier; consumer warps wait on it, compute, and release the stage through a
+// second mbarrier. All waits are bounded; a wait that runs out sets the plan's
+// status word and the CTA drains and exits.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstdio>
+#include <mutex>
+
+#include "ubp_internal.h"
+
+namespace ubp {
+
+// ------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait. Returns false if the wait ran out or another thread of the CTA
+// already gave up (abort flag in shared memory).
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    constexpr uint64_t kLimitNs = 1000ull * 1000ull * 1000ull;   // one second, then give up
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kLimitNs) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+
+template <int N>
+__device__ __forceinline__ void load_floats(float (&w)[N], const float *p)
+{
+    if constexpr (N == 1) {
+        w[0] = p[0];
+    } else if constexpr (N == 2) {
+        const float2 t = *reinterpret_cast<const float2 *>(p);
+        w[0] = t.x; w[1] = t.y;
+    } else {
+        static_assert(N % 4 == 0, "entry weights are loaded as float4");
+#pragma unroll
+        for (int q = 0; q < N / 4; ++q) {
+            const float4 t = *reinterpret_cast<const float4 *>(p + 4 * q);
+            w[4 * q] = t.x; w[4 * q + 1] = t.y; w[4 * q + 2] = t.z; w[4 * q + 3] = t.w;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ main 1x1 kernel
+// One fragment = all entries of this (panel, tile) whose first row sits at
+// offset S inside the panel (S may be negative for an entry that started in the
+// panel above). Rows outside [0, P) are clipped at compile time.
+template <int NBK, int P, int V, int S, bool DUPW, int XROW_BYTES>
+__device__ __forceinline__ void run_fragment(float2 (&acc)[P][2 * V], const uint8_t *xs_lane,
+                                             const uint16_t *jl, const float *wv, int e0, int e1)
+{
+    constexpr int R_LO = (S < 0) ? -S : 0;
+    constexpr int R_HI = (S + NBK > P) ? (P - S) : NBK;
+    constexpr int WF = NBK * (DUPW ? 2 : 1);
+    for (int e = e0; e < e1; ++e) {
+        const uint32_t j = jl[e];
+        const uint8_t *xp = xs_lane + j * (uint32_t)XROW_BYTES;
+        float4 x[V];
+#pragma unroll
+        for (int v = 0; v < V; ++v) x[v] = *reinterpret_cast<const float4 *>(xp + v * 512);
+        float w[WF];
+        load_floats<WF>(w, wv + (size_t)e * WF);
+#pragma unroll
+        for (int r = R_LO; r < R_HI; ++r) {
+            const float2 w2 = DUPW ? make_float2(w[2 * r], w[2 * r + 1]) : make_float2(w[r], w[r]);
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                acc[S + r][2 * v] = fma2(w2, make_float2(x[v].x, x[v].y), acc[S + r][2 * v]);
+                acc[S + r][2 * v + 1] = fma2(w2, make_float2(x[v].z, x[v].w), acc[S + r][2 * v + 1]);
+            }
+        }
+    }
+}
+
+template <int NBK, int P, int V, bool DUPW, int XROW_BYTES, int F0, int F1>
+struct FragmentLoop {
+    __device__ __forceinline__ static void run(float2 (&acc)[P][2 * V], const uint8_t *xs_lane,
+                                               const uint16_t *fo, const uint16_t *jl, const float *wv, int e0)
+    {
+        if constexpr (F0 < F1) {
+            const int e1 = fo[F0 + 1];
+            run_fragment<NBK, P, V, F0 - (NBK - 1), DUPW, XROW_BYTES>(acc, xs_lane, jl, wv, e0, e1);
+            FragmentLoop<NBK, P, V, DUPW, XROW_BYTES, F0 + 1, F1>::run(acc, xs_lane, fo, jl, wv, e1);
+        }
+    }
+};
+
+struct SpmmArgs {
+    const uint8_t *plan;     // device plan image
+    const float *bias;       // [M] or null
+    float *Y;
+    int64_t ldy;
+    int64_t Nc;
+    int M;
+    int nkt, NG;
+    int stages;
+    uint32_t stage_bytes;    // X tile + largest plan group, 128-byte multiple
+    int relu;
+};
+
+template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW>
+__global__ void __launch_bounds__((WR * WC + 1) * 32, 1)
+ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
+{
+    constexpr int CS = WC * 128 * V;               // columns per CTA
+    constexpr int XT_BYTES = KT * CS * 4;
+    constexpr int F = P + NBK - 1;
+    constexpr int NCW = WR * WC;                   // consumer warps
+    constexpr int FO_BYTES = ((F + 1) * 2 + 15) & ~15;
+    constexpr int WF = NBK * (DUPW ? 2 : 1);
+    constexpr int MAX_STAGES = 8;
+
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ __align__(8) uint64_t bar_full[MAX_STAGES];
+    __shared__ __align__(8) uint64_t bar_empty[MAX_STAGES];
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = blockIdx.x;                      // row group
+    const int strip = blockIdx.y;                  // column strip
+    const int S = a.stages;
+    const uint32_t *gtab = reinterpret_cast<const uint32_t *>(a.plan + 256);
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), NCW);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == NCW) {
+        // ---------------- producer warp
+        if (lane == 0) {
+            int issued = 0;
+            bool ok = true;
+            for (int kt = 0; kt < a.nkt && ok; ++kt) {
+                const int st = kt % S;
+                if (kt >= S) ok = mbar_wait(smem_u32(&bar_empty[st]), ((kt / S) - 1) & 1, &abort_flag);
+                if (!ok) break;
+                const uint32_t o0 = gtab[(size_t)kt * a.NG + g], o1 = gtab[(size_t)kt * a.NG + g + 1];
+                const uint32_t gbytes = (o1 - o0) * 16u;
+                const uint32_t bar = smem_u32(&bar_full[st]);
+                uint8_t *stage = smem + (size_t)st * a.stage_bytes;
+                mbar_expect_tx(bar, (uint32_t)XT_BYTES + gbytes);
+                tma_load_2d(smem_u32(stage), &tmX, strip * CS, kt * KT, bar);
+                bulk_load(smem_u32(stage + XT_BYTES), a.plan + (size_t)o0 * 16u, gbytes, bar);
+                ++issued;
+            }
+            if (!ok) {
+                // drain: give copies already in flight a bounded chance to land before the CTA exits
+                const int first = issued > S ? issued - S : 0;
+                for (int kt = first; kt < issued; ++kt)
+                    for (uint32_t it = 0; it < (1u << 16); ++it)
+                        if (mbar_try_wait(smem_u32(&bar_full[kt % S]), (kt / S) & 1)) break;
+                atomicExch(reinterpret_cast<int *>(const_cast<uint8_t *>(a.plan)), 1);
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumer warps
+    const int wr = warp / WC, wc = warp % WC;
+    const int panel = g * WR + wr;
+    float2 acc[P][2 * V];
+#pragma unroll
+    for (int r = 0; r < P; ++r)
+#pragma unroll
+        for (int q = 0; q < 2 * V; ++q) acc[r][q] = make_float2(0.f, 0.f);
+
+    bool ok = true;
+    for (int kt = 0; kt < a.nkt; ++kt) {
+        const int st = kt % S;
+        ok = mbar_wait(smem_u32(&bar_full[st]), (kt / S) & 1, &abort_flag);
+        if (!ok) break;
+        const uint8_t *stage = smem + (size_t)st * a.stage_bytes;
+        const uint8_t *grp = stage + XT_BYTES;
+        const uint32_t po = reinterpret_cast<const uint32_t *>(grp)[wr];
+        const uint32_t pn = reinterpret_cast<const uint32_t *>(grp)[wr + 1];
+        if (pn > po) {                               // panel exists in this group
+            const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
+            const int n = fo[F];
+            const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
+            const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * n + 15) & ~15));
+            const uint8_t *xs_lane = stage + (wc * 128 * V + lane * 4) * 4;
+            FragmentLoop<NBK, P, V, DUPW, CS * 4, 0, F>::run(acc, xs_lane, fo, jl, wv, 0);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bar_empty[st]));
+    }
+    if (!ok) {                                       // report through the plan's status word, store nothing
+        if (lane == 0) atomicExch(reinterpret_cast<int *>(const_cast<uint8_t *>(a.plan)), 1);
+        return;
+    }
+    (void)WF;
+
+    // ---------------- epilogue: bias, activation, one 128-bit store per lane and column group
+    const int64_t col0 = (int64_t)strip * CS + wc * 128 * V + lane * 4;
+#pragma unroll
+    for (int r = 0; r < P; ++r) {
+        const int row = panel * P + r;
+        if (row >= a.M) break;
+        const float b = a.bias ? __ldg(a.bias + row) : 0.f;
+        float *yrow = a.Y + (size_t)row * a.ldy;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const int64_t col = col0 + v * 128;
+            float4 o = make_float4(acc[r][2 * v].x + b, acc[r][2 * v].y + b,
+                                   acc[r][2 * v + 1].x + b, acc[r][2 * v + 1].y + b);
+            if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+            if (col + 3 < a.Nc) {
+                *reinterpret_cast<float4 *>(yrow + col) = o;
+            } else {
+                if (col < a.Nc) yrow[col] = o.x;
+                if (col + 1 < a.Nc) yrow[col + 1] = o.y;
+                if (col + 2 < a.Nc) yrow[col + 2] = o.z;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ fallback 1x1 kernel
+// Any alignment, any leading dimension: one lane per output column, plan and
+// activations read straight from global memory. Same plan, same summation
+// order per output as the main kernel.
+template <int NBK, int P, int S>
+__device__ __forceinline__ void simple_fragment(float (&acc)[P], const float *xcol, int64_t ldx, bool live,
+                                                const uint16_t *jl, const float *wv, int wstride, int wdup,
+                                                int e0, int e1)
+{
+    constexpr int R_LO = (S < 0) ? -S : 0;
+    constexpr int R_HI = (S + NBK > P) ? (P - S) : NBK;
+    for (int e = e0; e < e1; ++e) {
+        const float x = live ? xcol[(size_t)jl[e] * ldx] : 0.f;
+#pragma unroll
+        for (int r = R_LO; r < R_HI; ++r) acc[S + r] = fmaf(wv[(size_t)e * wstride + r * wdup], x, acc[S + r]);
+    }
+}
+template <int NBK, int P, int F0, int F1>
+struct SimpleLoop {
+    __device__ __forceinline__ static void run(float (&acc)[P], const float *xcol, int64_t ldx, bool live,
+                                               const uint16_t *fo, const uint16_t *jl, const float *wv,
+                                               int wstride, int wdup, int e0)
+    {
+        if constexpr (F0 < F1) {
+            const int e1 = fo[F0 + 1];
+            simple_fragment<NBK, P, F0 - (NBK - 1)>(acc, xcol, ldx, live, jl, wv, wstride, wdup, e0, e1);
+            SimpleLoop<NBK, P, F0 + 1, F1>::run(acc, xcol, ldx, live, fo, jl, wv, wstride, wdup, e1);
+        }
+    }
+};
+
+template <int NBK, int P>
+__global__ void __launch_bounds__(128)
+ubp_spmm_simple_kernel(const uint8_t *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                       float *Y, int64_t ldy, int M, int NP, int nkt, int NG, int WR, int KT, int dupw)
+{
+    constexpr int F = P + NBK - 1;
+    constexpr int FO_BYTES = ((F + 1) * 2 + 15) & ~15;
+    const int panel = blockIdx.y;
+    const int64_t col = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool live = col < Nc;
+    if (panel >= NP) return;
+    const int g = panel / WR, wr = panel % WR;
+    const uint32_t *gtab = reinterpret_cast<const uint32_t *>(plan + 256);
+    float acc[P];
+#pragma unroll
+    for (int r = 0; r < P; ++r) acc[r] = 0.f;
+    const int wdup = dupw ? 2 : 1;
+    for (int kt = 0; kt < nkt; ++kt) {
+        const uint8_t *grp = plan + (size_t)gtab[(size_t)kt * NG + g] * 16u;
+        const uint32_t po = reinterpret_cast<const uint32_t *>(grp)[wr];
+        const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
+        const int n = fo[F];
+        const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
+        const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * n + 15) & ~15));
+        const float *xcol = X + (size_t)kt * KT * ldx + (live ? col : 0);
+        SimpleLoop<NBK, P, 0, F>::run(acc, xcol, ldx, live, fo, jl, wv, NBK * wdup, wdup, 0);
+    }
+    if (!live) return;
+#pragma unroll
+    for (int r = 0; r < P; ++r) {
+        const int row = panel * P + r;
+        if (row < M) {
+            float o = acc[r] + (bias ? bias[row] : 0.f);
+            if (relu) o = fmaxf(o, 0.f);
+            Y[(size_t)row * ldy + col] = o;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ 3x3 implicit kernel (first version)
+// One lane per output pixel n = (b, y, x); the nine taps of an entry read the
+// input plane in place (zero outside the image), so the lowered K = 9*C matrix
+// never exists. Entry weights are [nbk][9].
+template <int NBK, int P, int S>
+__device__ __forceinline__ void conv_fragment(float (&acc)[P], const float *inb, int64_t isc, int y, int x, int H, int Wd,
+                                              bool live, const uint16_t *jl, const float *wv, int kt_base, int e0, int e1)
+{
+    constexpr int R_LO = (S < 0) ? -S : 0;
+    constexpr int R_HI = (S + NBK > P) ? (P - S) : NBK;
+    for (int e = e0; e < e1; ++e) {
+        const float *plane = inb + (size_t)(kt_base + jl[e]) * isc;
+        const float *w = wv + (size_t)e * NBK * 9;
+#pragma unroll
+        for (int dy = 0; dy < 3; ++dy)
+#pragma unroll
+            for (int dx = 0; dx < 3; ++dx) {
+                const int yy = y + dy - 1, xx = x + dx - 1;
+                const bool in = live && yy >= 0 && yy < H && xx >= 0 && xx < Wd;
+                const float xv = in ? __ldg(plane + (size_t)yy * Wd + xx) : 0.f;
+#pragma unroll
+                for (int r = R_LO; r < R_HI; ++r) acc[S + r] = fmaf(w[r * 9 + dy * 3 + dx], xv, acc[S + r]);
+            }
+    }
+}
+template <int NBK, int P, int F0, int F1>
+struct ConvLoop {
+    __device__ __forceinline__ static void run(float (&acc)[P], const float *inb, int64_t isc, int y, int x, int H, int Wd,
+                                               bool live, const uint16_t *fo, const uint16_t *jl, const float *wv,
+                                               int kt_base, int e0)
+    {
+        if constexpr (F0 < F1) {
+            const int e1 = fo[F0 + 1];
+            conv_fragment<NBK, P, F0 - (NBK - 1)>(acc, inb, isc, y, x, H, Wd, live, jl, wv, kt_base, e0, e1);
+            ConvLoop<NBK, P, F0 + 1, F1>::run(acc, inb, isc, y, x, H, Wd, live, fo, jl, wv, kt_base, e1);
+        }
+    }
+};
+
+template <int NBK, int P>
+__global__ void __launch_bounds__(128)
+ubp_conv3x3_simple_kernel(const uint8_t *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
+                          const float *bias, int relu, float *out, int64_t osb, int64_t osc,
+                          int M, int NP, int nkt, int NG, int WR, int KT)
+{
+    constexpr int F = P + NBK - 1;
+    constexpr int FO_BYTES = ((F + 1) * 2 + 15) & ~15;
+    const int panel = blockIdx.y;
+    const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t total = (int64_t)B * H * Wd;
+    const bool live = n < total;
+    const int64_t nn = live ? n : 0;
+    const int b = (int)(nn / (H * Wd));
+    const int pix = (int)(nn % (H * Wd));
+    const int y = pix / Wd, x = pix % Wd;
+    const int g = panel / WR, wr = panel % WR;
+    const uint32_t *gtab = reinterpret_cast<const uint32_t *>(plan + 256);
+    const float *inb = in + (size_t)b * isb;
+    float acc[P];
+#pragma unroll
+    for (int r = 0; r < P; ++r) acc[r] = 0.f;
+    for (int kt = 0; kt < nkt; ++kt) {
+        const uint8_t *grp = plan + (size_t)gtab[(size_t)kt * NG + g] * 16u;
+        const uint32_t po = reinterpret_cast<const uint32_t *>(grp)[wr];
+        const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
+        const int cnt = fo[F];
+        const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
+        const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * cnt + 15) & ~15));
+        ConvLoop<NBK, P, 0, F>::run(acc, inb, isc, y, x, H, Wd, live, fo, jl, wv, kt * KT, 0);
+    }
+    if (!live) return;
+#pragma unroll
+    for (int r = 0; r < P; ++r) {
+        const int row = panel * P + r;
+        if (row < M) {
+            float o = acc[r] + (bias ? bias[row] : 0.f);
+            if (relu) o = fmaxf(o, 0.f);
+            out[(size_t)b * osb + (size_t)row * osc + pix] = o;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+static int check(cudaError_t e)
+{
+    if (e == cudaSuccess) return UBP_OK;
+    set_last_cuda_error((int)e);
+    return UBP_E_CUDA;
+}
+
+constexpr size_t kSmemBudget = 227 * 1024 - 1024;   // dynamic shared memory we allow ourselves per CTA
+
+template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW>
+static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                       float *Y, int64_t ldy, cudaStream_t stream)
+{
+    constexpr int CS = WC * 128 * V;
+    constexpr size_t XT = (size_t)KT * CS * 4;
+    const size_t stage_bytes = (XT + pl->img.max_group_bytes + 127) & ~(size_t)127;
+    int stages = (int)(kSmemBudget / stage_bytes);
+    if (stages < 2) return UBP_E_UNSUPPORTED;
+    if (stages > 4) stages = 4;
+    if (stages > pl->img.nkt) stages = pl->img.nkt < 1 ? 1 : pl->img.nkt;
+
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return UBP_E_CUDA;
+    CUtensorMap tm;
+    const cuuint64_t dims[2] = {(cuuint64_t)Nc, (cuuint64_t)pl->dims.C};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)CS, (cuuint32_t)KT};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult cr = enc(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(X), dims, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) { set_last_cuda_error(-(int)cr); return UBP_E_CUDA; }
+
+    auto kern = ubp_spmm_kernel<NBK, P, V, WR, WC, KT, DUPW>;
+    const size_t smem = stage_bytes * stages;
+    static bool attr_done[64] = {};                  // per device: opt in to large dynamic shared memory once
+    int dev = 0;
+    if (int rc = check(cudaGetDevice(&dev))) return rc;
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        if (int rc = check(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget)))
+            return rc;
+        if (dev >= 0 && dev < 64) attr_done[dev] = true;
+    }
+
+    SpmmArgs a;
+    a.plan = static_cast<const uint8_t *>(pl->dev);
+    a.bias = bias; a.Y = Y; a.ldy = ldy; a.Nc = Nc; a.M = pl->dims.M;
+    a.nkt = pl->img.nkt; a.NG = pl->img.NG; a.stages = stages; a.stage_bytes = (uint32_t)stage_bytes; a.relu = relu;
+    dim3 grid((unsigned)pl->img.NG, (unsigned)((Nc + CS - 1) / CS));
+    kern<<<grid, (WR * WC + 1) * 32, smem, stream>>>(tm, a);
+    return check(cudaGetLastError());
+}
+
+template <int NBK, int P>
+static int launch_simple(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                         float *Y, int64_t ldy, cudaStream_t stream)
+{
+    dim3 grid((unsigned)((Nc + 127) / 128), (unsigned)pl->img.NP);
+    ubp_spmm_simple_kernel<NBK, P><<<grid, 128, 0, stream>>>(
+        static_cast<const uint8_t *>(pl->dev), X, ldx, Nc, bias, relu, Y, ldy, pl->dims.M, pl->img.NP, pl->img.nkt,
+        pl->img.NG, pl->cfg.WR, pl->cfg.KT, pl->cfg.dupw);
+    return check(cudaGetLastError());
+}
+
+int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                float *Y, int64_t ldy, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const KernelCfg &c = pl->cfg;
+    const bool fast = ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(Y)) & 15) == 0 &&
+                      (ldx % 4 == 0) && (ldy % 4 == 0) && (int64_t)ldx * 4 < (1ll << 40) &&
+                      pl->dims.C < (1 << 30) && Nc < (1ll << 31);
+    int rc = UBP_E_UNSUPPORTED;
+#define UBP_MAIN(ID, NBK, P, V, WR, WC, KT, DUP)                                                             \
+    if (fast && c.id == ID) rc = launch_main<NBK, P, V, WR, WC, KT, DUP>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
+    UBP_MAIN(1, 4, 16, 2, 8, 1, 32, false)
+    UBP_MAIN(2, 4, 16, 2, 8, 1, 32, true)
+    UBP_MAIN(3, 4, 16, 1, 8, 2, 32, false)
+    UBP_MAIN(4, 4, 16, 1, 16, 1, 64, false)
+    UBP_MAIN(5, 2, 16, 2, 8, 1, 32, false)
+    UBP_MAIN(6, 8, 16, 2, 8, 1, 32, false)
+    UBP_MAIN(7, 16, 16, 2, 8, 1, 32, false)
+    UBP_MAIN(8, 1, 16, 2, 8, 1, 32, false)
+    UBP_MAIN(9, 8, 8, 2, 16, 1, 32, false)
+#undef UBP_MAIN
+    if (rc != UBP_E_UNSUPPORTED) return rc;
+    // slower kernel: unaligned operands, or a plan group too large to stage
+#define UBP_SIMPLE(NBK_, P_) \
+    if (c.nbk == NBK_ && c.P == P_) return launch_simple<NBK_, P_>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
+    UBP_SIMPLE(1, 16) UBP_SIMPLE(2, 16) UBP_SIMPLE(4, 16) UBP_SIMPLE(8, 16) UBP_SIMPLE(16, 16) UBP_SIMPLE(8, 8)
+#undef UBP_SIMPLE
+    return UBP_E_UNSUPPORTED;
+}
+
+int launch_conv3x3(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
+                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const KernelCfg &c = pl->cfg;
+    const int64_t total = (int64_t)B * H * Wd;
+    dim3 grid((unsigned)((total + 127) / 128), (unsigned)pl->img.NP);
+#define UBP_CONV(NBK_, P_)                                                                                      \
+    if (c.nbk == NBK_ && c.P == P_) {                                                                           \
+        ubp_conv3x3_simple_kernel<NBK_, P_><<<grid, 128, 0, stream>>>(                                          \
+            static_cast<const uint8_t *>(pl->dev), in, B, H, Wd, isb, isc, bias, relu, out, osb, osc, pl->dims.M, \
+            pl->img.NP, pl->img.nkt, pl->img.NG, c.WR, c.KT);                                                   \
+        return check(cudaGetLastError());                                                                       \
+    }
+    UBP_CONV(8, 8) UBP_CONV(4, 8) UBP_CONV(2, 8) UBP_CONV(1, 8)
+#undef UBP_CONV
+    return UBP_E_UNSUPPORTED;
+}
+
+}  // namespace ubp

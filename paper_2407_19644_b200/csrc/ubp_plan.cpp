@@ -1,0 +1,204 @@
+// Plan builder: re-buckets the canonical blocks (start row, input channel,
+// rotated values; Section 4.2) for the GPU kernels. Host code only.
+//
+// Each canonical block is un-rotated, cut into entries of `nbk` rows and
+// filed under (input-channel tile, row panel, start offset inside the panel).
+// An entry whose rows cross a panel boundary is filed in both panels (with a
+// negative start offset in the lower one); each panel's kernel code touches
+// only its own rows, so every output element has exactly one writer and a
+// fixed summation order -- the GPU counterpart of the paper's fix for
+// overlapping output tiles (Section 3.3).
+#include "ubp_internal.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+
+namespace ubp {
+
+const std::vector<KernelCfg> &kernel_cfgs()
+{
+    //                 id kind nbk  P  V WR WC  KT dup
+    static const std::vector<KernelCfg> cfgs = {
+        {1, 0, 4, 16, 2, 8, 1, 32, 0},
+        {2, 0, 4, 16, 2, 8, 1, 32, 1},
+        {3, 0, 4, 16, 1, 8, 2, 32, 0},
+        {4, 0, 4, 16, 1, 16, 1, 64, 0},
+        {5, 0, 2, 16, 2, 8, 1, 32, 0},
+        {6, 0, 8, 16, 2, 8, 1, 32, 0},
+        {7, 0, 16, 16, 2, 8, 1, 32, 0},
+        {8, 0, 1, 16, 2, 8, 1, 32, 0},
+        {9, 0, 8, 8, 2, 16, 1, 32, 0},
+        {10, 1, 8, 8, 1, 4, 1, 16, 0},
+        {11, 1, 4, 8, 1, 4, 1, 16, 0},
+        {12, 1, 2, 8, 1, 4, 1, 16, 0},
+        {13, 1, 1, 8, 1, 4, 1, 16, 0},
+    };
+    return cfgs;
+}
+
+const KernelCfg *find_cfg(int id)
+{
+    for (const auto &c : kernel_cfgs())
+        if (c.id == id) return &c;
+    return nullptr;
+}
+
+static int largest_pow2_divisor_le16(int Nb)
+{
+    int k = 1;
+    while (k < 16 && Nb % (k * 2) == 0) k *= 2;
+    return k;
+}
+
+const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
+{
+    (void)M; (void)C; (void)m;
+    const int nbk = largest_pow2_divisor_le16(Nb);
+    if (R == 9) {
+        switch (nbk) {
+            case 16: case 8: return find_cfg(10);
+            case 4: return find_cfg(11);
+            case 2: return find_cfg(12);
+            default: return find_cfg(13);
+        }
+    }
+    if (R != 1) return nullptr;
+    switch (nbk) {
+        case 16: return find_cfg(7);
+        case 8: return find_cfg(6);
+        case 4: return find_cfg(1);
+        case 2: return find_cfg(5);
+        default: return find_cfg(8);
+    }
+}
+
+static inline size_t pad16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only, PlanImage &img, size_t *bytes)
+{
+    const int M = v.M, C = v.C, R = v.R, Nb = v.Nb;
+    const int nbk = cfg.nbk, P = cfg.P, KT = cfg.KT, WR = cfg.WR;
+    if (Nb % nbk != 0) return UBP_E_UNSUPPORTED;
+    if ((cfg.kind == 0 && R != 1) || (cfg.kind == 1 && R != 9)) return UBP_E_UNSUPPORTED;
+    const int nkt = (C + KT - 1) / KT;
+    const int NP = (M + P - 1) / P;
+    const int NG = (NP + WR - 1) / WR;
+    const int F = P + nbk - 1;
+    const int sub = Nb / nbk;
+    const size_t wfloats = (size_t)nbk * R * (cfg.dupw ? 2 : 1);   // floats per entry
+
+    // pass 1: entries per (kt, panel, fragment)
+    std::vector<uint32_t> cnt((size_t)nkt * NP * F, 0);
+    auto bucket = [&](int kt, int p, int f) -> size_t { return ((size_t)kt * NP + p) * F + f; };
+    int64_t entries = 0;
+    for (int i = 0; i < M; ++i)
+        for (int32_t b = v.indptr[i]; b < v.indptr[i + 1]; ++b) {
+            const int kt = v.indices[b] / KT;
+            for (int u = 0; u < sub; ++u) {
+                const int r0 = i + u * nbk;
+                const int p = r0 / P, s = r0 % P;
+                cnt[bucket(kt, p, s + nbk - 1)]++;
+                ++entries;
+                if (s + nbk > P) {           // crosses into the next panel
+                    cnt[bucket(kt, p + 1, s - P + nbk - 1)]++;
+                    ++entries;
+                }
+            }
+        }
+
+    // layout
+    const size_t tab_off = 256;
+    const size_t tab_bytes = pad16(sizeof(uint32_t) * ((size_t)nkt * NG + 1));
+    const size_t poff_bytes = pad16(sizeof(uint32_t) * (size_t)(WR + 1));
+    const size_t fo_bytes = pad16(sizeof(uint16_t) * (size_t)(F + 1));
+    std::vector<size_t> seg_off((size_t)nkt * NP, 0);        // absolute offset of each panel sub-segment
+    std::vector<size_t> grp_off((size_t)nkt * NG + 1, 0);
+    size_t cur = pad16(tab_off + tab_bytes);
+    uint32_t max_group = 0;
+    for (int kt = 0; kt < nkt; ++kt)
+        for (int g = 0; g < NG; ++g) {
+            grp_off[(size_t)kt * NG + g] = cur;
+            const size_t g0 = cur;
+            cur += poff_bytes;
+            for (int p = g * WR; p < std::min(NP, (g + 1) * WR); ++p) {
+                size_t n = 0;
+                for (int f = 0; f < F; ++f) n += cnt[bucket(kt, p, f)];
+                if (n > 65535) return UBP_E_UNSUPPORTED;
+                seg_off[(size_t)kt * NP + p] = cur;
+                cur += fo_bytes + pad16(2 * n) + pad16(4 * n * wfloats);
+            }
+            if (cur - g0 > max_group) max_group = (uint32_t)(cur - g0);
+        }
+    grp_off[(size_t)nkt * NG] = cur;
+    const size_t total = (cur + 255) & ~(size_t)255;
+    if (total / 16 > 0xffffffffull) return UBP_E_UNSUPPORTED;
+    if (bytes) *bytes = total;
+    img.nkt = nkt; img.NP = NP; img.NG = NG; img.F = F; img.entries = entries; img.max_group_bytes = max_group;
+    if (count_only) return UBP_OK;
+
+    img.bytes.assign(total, 0);
+    uint8_t *base = img.bytes.data();
+    uint32_t *tab = reinterpret_cast<uint32_t *>(base + tab_off);
+    for (size_t q = 0; q < grp_off.size(); ++q) tab[q] = (uint32_t)(grp_off[q] / 16);
+    // group headers, fragment offsets; cursors start at the fragment offsets
+    std::vector<uint32_t> cursor(cnt.size(), 0);
+    for (int kt = 0; kt < nkt; ++kt)
+        for (int g = 0; g < NG; ++g) {
+            const size_t g0 = grp_off[(size_t)kt * NG + g];
+            uint32_t *poff = reinterpret_cast<uint32_t *>(base + g0);
+            size_t end = g0 + poff_bytes;
+            for (int w = 0; w <= WR; ++w) {
+                const int p = g * WR + w;
+                if (w < WR && p < NP) {
+                    const size_t so = seg_off[(size_t)kt * NP + p];
+                    poff[w] = (uint32_t)(so - g0);
+                    uint16_t *fo = reinterpret_cast<uint16_t *>(base + so);
+                    uint32_t acc = 0;
+                    for (int f = 0; f < F; ++f) {
+                        fo[f] = (uint16_t)acc;
+                        cursor[bucket(kt, p, f)] = acc;
+                        acc += cnt[bucket(kt, p, f)];
+                    }
+                    fo[F] = (uint16_t)acc;
+                    end = so + fo_bytes + pad16(2 * (size_t)acc) + pad16(4 * (size_t)acc * wfloats);
+                } else {
+                    poff[w] = (uint32_t)(end - g0);
+                }
+            }
+        }
+    // pass 2: file the entries (start rows ascending, then input channel ascending)
+    auto put = [&](int kt, int p, int f, int jl, const float *wsrc /* [nbk][R] */) {
+        const size_t so = seg_off[(size_t)kt * NP + p];
+        const uint16_t *fo = reinterpret_cast<const uint16_t *>(base + so);
+        const size_t n = fo[F];
+        const uint32_t e = cursor[bucket(kt, p, f)]++;
+        uint16_t *jl_arr = reinterpret_cast<uint16_t *>(base + so + fo_bytes);
+        float *w_arr = reinterpret_cast<float *>(base + so + fo_bytes + pad16(2 * n));
+        jl_arr[e] = (uint16_t)jl;
+        float *dst = w_arr + (size_t)e * wfloats;
+        if (cfg.dupw) {
+            for (size_t q = 0; q < (size_t)nbk * R; ++q) { dst[2 * q] = wsrc[q]; dst[2 * q + 1] = wsrc[q]; }
+        } else {
+            std::memcpy(dst, wsrc, sizeof(float) * (size_t)nbk * R);
+        }
+    };
+    std::vector<float> wblk((size_t)Nb * R);
+    for (int i = 0; i < M; ++i)
+        for (int32_t b = v.indptr[i]; b < v.indptr[i + 1]; ++b) {
+            const int j = v.indices[b];
+            const int kt = j / KT, jl = j % KT;
+            const float *val = v.values + (size_t)b * Nb * R;
+            for (int t = 0; t < Nb; ++t)       // undo the rotation: row i+t lives in slot (i+t) mod Nb
+                std::memcpy(&wblk[(size_t)t * R], val + (size_t)((i + t) % Nb) * R, sizeof(float) * (size_t)R);
+            for (int u = 0; u < sub; ++u) {
+                const int r0 = i + u * nbk;
+                const int p = r0 / P, s = r0 % P;
+                put(kt, p, s + nbk - 1, jl, &wblk[(size_t)u * nbk * R]);
+                if (s + nbk > P) put(kt, p + 1, s - P + nbk - 1, jl, &wblk[(size_t)u * nbk * R]);
+            }
+        }
+    return UBP_OK;
+}
+
+}  // namespace ubp

@@ -1,0 +1,154 @@
+"""CPU tests of the library's host code: the C ABI surface, the packer against
+the oracle's independent packer (bit-exact), error paths, and the plan builder."""
+import ctypes
+import os
+import re
+import struct
+
+import numpy as np
+import pytest
+
+import oracle
+import ubp_synth
+import paper_2407_19644_b200 as ubp
+from helpers import plan_to_dense
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "ubp.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    names = set(re.findall(r"\b(ubp_[a-z0-9_]+)\s*\(", hdr))
+    assert {"ubp_pack", "ubp_unpack", "ubp_spmm", "ubp_conv1x1", "ubp_conv3x3_implicit",
+            "ubp_plan_build", "ubp_plan_size"} <= names
+    L = ctypes.CDLL(ubp.lib_path())
+    for n in sorted(names):
+        assert hasattr(L, n), n
+
+
+def test_strerror_and_variants():
+    L = ubp.load()
+    assert L.ubp_strerror(0) == b"ok"
+    assert b"whole number of blocks" in L.ubp_strerror(-2)
+    v = ubp.variants()
+    assert len(v) >= 8 and all(isinstance(s, str) and s for s in v.values())
+
+
+CASES = [(64, 64, 4, 50, 1), (37, 11, 3, 40, 1), (40, 16, 8, 80, 9), (33, 5, 16, 50, 1), (16, 16, 2, 90, 9),
+         (5, 3, 1, 30, 1), (128, 96, 4, 70, 1), (20, 7, 5, 0, 1), (48, 48, 16, 50, 1)]
+
+
+@pytest.mark.parametrize("M,C,Nb,p,R", CASES)
+def test_pack_bit_exact_vs_oracle_and_round_trip(M, C, Nb, p, R):
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 900 + M, Nc=4 if R == 1 else None, R=R, B=1, H=2, Wd=2)
+    blob = ubp.ubp_pack(L.W, L.mask, Nb)
+    assert blob == oracle.pack(L.W, L.mask, Nb)                       # bit-exact format
+    W2, m2 = ubp.ubp_unpack(blob)
+    Wo, mo = oracle.unpack(blob)
+    assert np.array_equal(m2, L.mask) and np.array_equal(mo, m2)
+    assert np.array_equal(W2.view(np.uint32), Wo.view(np.uint32))
+    keep = L.mask.astype(bool)
+    assert np.array_equal(W2[keep].view(np.uint32), L.W[keep].view(np.uint32)) and (W2[~keep].view(np.uint32) == 0).all()
+    d = ubp.blob_view(blob)
+    assert (d["M"], d["C"], d["R"], d["Nb"], d["m"]) == (M, C, R, Nb, L.m)
+    assert d["m"] == oracle.block_budget(M, C, p, Nb)
+
+
+def test_pack_special_values_and_aligned_pattern():
+    M, C, Nb = 12, 3, 4
+    mask, _ = ubp_synth.random_mask(M, C, Nb, 34, seed=2, aligned=True)
+    W = np.random.default_rng(0).standard_normal((M, C, 1)).astype(np.float32)
+    W[mask.astype(bool)][:1] = -0.0
+    W[0, 0, 0] = np.float32(-0.0); W[1, 0, 0] = np.float32(1e-42)
+    assert ubp.ubp_pack(W, mask, Nb) == oracle.pack(W, mask, Nb)
+
+
+@pytest.mark.parametrize("kind", ["ragged", "edge", "value", "nb_gt_m", "nb_zero"])
+def test_pack_rejects_bad_input(kind):
+    M, C, Nb = 8, 2, 3
+    mask = np.zeros((M, C), np.uint8)
+    W = np.ones((M, C), np.float32)
+    want = -2
+    if kind == "ragged":
+        mask[1:5, 0] = 1
+    elif kind == "edge":
+        mask[6:8, 1] = 1
+    elif kind == "value":
+        mask[0:3, 0] = 1; mask[2, 0] = 3; want = -1
+    elif kind == "nb_gt_m":
+        Nb = 9; want = -1
+    else:
+        Nb = 0; want = -1
+    with pytest.raises(ubp.UbpError) as e:
+        ubp.ubp_pack(W, mask, Nb)
+    assert e.value.code == want
+    if kind in ("ragged", "edge", "value"):
+        with pytest.raises(oracle.OracleError):
+            oracle.pack(W, mask, Nb)
+
+
+def test_pack_null_and_small_buffer():
+    L = ubp.load()
+    n = ctypes.c_size_t(0)
+    assert L.ubp_pack(None, None, 4, 4, 1, 2, None, 0, ctypes.byref(n)) == -1
+    W = np.ones((4, 4), np.float32); mask = np.zeros((4, 4), np.uint8); mask[0:2, 1] = 1
+    p = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    assert L.ubp_pack(p(W), p(mask), 4, 4, 1, 2, None, 0, ctypes.byref(n)) == 0 and n.value > 64
+    small = np.zeros(32, np.uint8)
+    assert L.ubp_pack(p(W), p(mask), 4, 4, 1, 2, p(small), 32, ctypes.byref(n)) == -3
+
+
+def test_blob_view_rejects_corruption():
+    L = ubp_synth.make_layer("t", 16, 8, 4, 50, 3, Nc=4)
+    blob = bytearray(ubp.ubp_pack(L.W, L.mask, 4))
+    for mutate in ("magic", "trunc", "indptr", "index"):
+        b = bytearray(blob)
+        if mutate == "magic":
+            b[0] = ord("X")
+        elif mutate == "trunc":
+            b = b[:len(b) - 64]
+        elif mutate == "indptr":
+            struct.pack_into("<i", b, 64 + 4, 9999)
+        else:
+            off = 64 + (4 * 17 + 63) // 64 * 64
+            struct.pack_into("<i", b, off, 1000)
+        with pytest.raises(ubp.UbpError) as e:
+            ubp.blob_view(bytes(b))
+        assert e.value.code == -4
+
+
+@pytest.mark.parametrize("M,C,Nb,p,R,variant", [
+    (64, 64, 4, 50, 1, 0), (100, 70, 4, 60, 1, 1), (100, 70, 4, 60, 1, 2), (100, 70, 4, 60, 1, 4),
+    (37, 45, 3, 40, 1, 0), (50, 33, 2, 50, 1, 0), (72, 40, 8, 50, 1, 0), (72, 40, 8, 50, 1, 9),
+    (80, 40, 16, 50, 1, 0), (60, 20, 12, 40, 1, 0), (45, 17, 1, 70, 1, 0), (40, 20, 8, 50, 9, 0),
+    (24, 18, 4, 50, 9, 0), (30, 10, 6, 40, 9, 0),
+])
+def test_plan_image_replays_to_masked_weight(M, C, Nb, p, R, variant):
+    """Every kept weight appears exactly once among the rows the panels own, with
+    its value; nothing else appears. Entries crossing a panel boundary are listed twice."""
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 70 + M, Nc=4 if R == 1 else None, R=R, B=1, H=2, Wd=2)
+    blob = ubp.ubp_pack(L.W, L.mask, Nb)
+    img, geom = ubp.plan_image(blob, variant)
+    assert len(img) == ubp.plan_size(blob, variant) and len(img) % 256 == 0
+    Wd, hits, n_entries = plan_to_dense(img, geom, M, C, R)
+    assert np.array_equal(hits, L.mask.astype(np.int32))
+    assert np.array_equal(Wd.view(np.uint32), (L.W * L.mask[:, :, None]).view(np.uint32) * L.mask[:, :, None])
+    nbk, P = geom["nbk"], geom["panel_rows"]
+    assert Nb % nbk == 0
+    bi, bj = oracle.decode_mask(L.mask, Nb)
+    sub = np.concatenate([bi + u * nbk for u in range(Nb // nbk)])
+    crossing = int(((sub % P) + nbk > P).sum())
+    assert n_entries == len(sub) + crossing
+
+
+def test_plan_rejects_wrong_kind():
+    L = ubp_synth.make_layer("t", 16, 8, 4, 50, 3, Nc=4)
+    blob = ubp.ubp_pack(L.W, L.mask, 4)
+    with pytest.raises(ubp.UbpError):
+        ubp.plan_size(blob, 10)         # a 3x3 configuration for an R = 1 blob
+    with pytest.raises(ubp.UbpError):
+        ubp.plan_size(blob, 6)          # 8 rows per entry do not divide a block of 4
+    with pytest.raises(ubp.UbpError):
+        ubp.plan_size(blob, 999)
+    assert ubp.plan_size(blob, 5) > 0   # 2 rows per entry: each block becomes two entries

@@ -1,0 +1,247 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the
+same seeded inputs. Gate: max |Y - Yref| / (|Wm||X| + |bias|) <= 1e-4 (fp32
+multiply-add, fp32 accumulation against a double reference); the tighter
+summation bound (L + 2) * 2^-24, L = kept terms per output, is asserted too."""
+import numpy as np
+import pytest
+
+import oracle
+import ubp_synth
+from helpers import scaled_error
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    import paper_2407_19644_b200 as ubp
+    assert torch.cuda.is_available()
+    ubp.load()
+    return torch, ubp
+
+
+def terms_per_output(L):
+    return int(L.mask.sum(axis=1).max()) * L.R
+
+
+def run_spmm(env, L, variant=0, pad=0, misalign=0, relu=None, use_bias=True):
+    torch, ubp = env
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    assert blob == oracle.pack(L.W, L.mask, L.Nb)
+    plan = ubp.Plan(blob, variant)
+    Nc = L.X.shape[1]
+    ld = Nc + pad
+    xbuf = torch.zeros(L.C * ld + 8, dtype=torch.float32, device="cuda")
+    X = xbuf[misalign:misalign + L.C * ld].view(L.C, ld)[:, :Nc]
+    X.copy_(torch.from_numpy(L.X))
+    ybuf = torch.full((L.M * ld + 8,), float("nan"), dtype=torch.float32, device="cuda")
+    Y = ybuf[misalign:misalign + L.M * ld].view(L.M, ld)[:, :Nc]
+    bias = torch.from_numpy(L.bias).cuda() if (use_bias and L.bias is not None) else None
+    r = L.relu if relu is None else relu
+    ubp.ubp_spmm(plan, X, bias, r, out=Y)
+    plan.check()
+    Yh = Y.cpu().numpy()
+    if pad:
+        assert torch.isnan(ybuf[misalign:misalign + L.M * ld].view(L.M, ld)[:, Nc:]).all()   # padding untouched
+    Yref, A = oracle.masked_matmul(L.W, L.mask, L.X, L.bias if bias is not None else None, relu=r)
+    return Yh, Yref, A, plan
+
+
+def check(Yh, Yref, A, L):
+    assert np.isfinite(Yh).all()
+    err = scaled_error(Yh, Yref, A)
+    assert err <= TOL, err
+    assert err <= (terms_per_output(L) + 2) * 2.0 ** -24, err
+    return err
+
+
+SMALL = [
+    # M, C, Nb, p, Nc, variant
+    (64, 64, 4, 50, 256, 0), (100, 70, 4, 60, 300, 1), (100, 70, 4, 60, 300, 2), (100, 70, 4, 60, 520, 3),
+    (300, 150, 4, 70, 260, 4), (37, 45, 3, 40, 132, 0), (50, 33, 2, 50, 388, 0), (72, 40, 8, 50, 264, 0),
+    (200, 40, 8, 50, 264, 9), (80, 40, 16, 50, 260, 0), (60, 20, 12, 40, 128, 0), (45, 17, 1, 70, 256, 0),
+    (16, 8, 4, 50, 4, 0), (130, 257, 4, 80, 1028, 0), (64, 64, 4, 0, 256, 0),
+]
+
+
+@pytest.mark.parametrize("M,C,Nb,p,Nc,variant", SMALL)
+def test_spmm_small(env, M, C, Nb, p, Nc, variant):
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 10 * M + C, Nc=Nc, x_dist="normal", relu=(M % 2 == 0))
+    Yh, Yref, A, _ = run_spmm(env, L, variant)
+    check(Yh, Yref, A, L)
+
+
+@pytest.mark.parametrize("Nc,pad,misalign", [(130, 2, 0), (131, 1, 0), (1, 3, 0), (3, 1, 0), (257, 3, 0),
+                                              (130, 0, 0), (255, 0, 0), (256, 0, 1), (64, 0, 3)])
+def test_spmm_ragged_and_unaligned(env, Nc, pad, misalign):
+    """pad > 0 with (Nc + pad) % 4 == 0 keeps the fast path with a ragged last strip; pad == 0 with odd Nc or a
+    misaligned base pointer takes the slower kernel."""
+    L = ubp_synth.make_layer("t", 70, 50, 4, 60, 4242 + Nc, Nc=Nc, x_dist="normal")
+    Yh, Yref, A, _ = run_spmm(env, L, 0, pad=pad, misalign=misalign)
+    check(Yh, Yref, A, L)
+
+
+def test_spmm_empty_and_degenerate(env):
+    torch, ubp = env
+    L = ubp_synth.make_layer("t", 32, 16, 4, 100, 5, Nc=64)           # no block kept at all
+    assert L.m == 0
+    Yh, Yref, A, plan = run_spmm(env, L, relu=False)
+    assert np.array_equal(Yh, np.broadcast_to(L.bias[:, None], Yh.shape))
+    # zero columns: no launch, no error
+    out = ubp.ubp_spmm(plan, torch.zeros((16, 0), device="cuda"))
+    assert out.shape == (32, 0)
+    # no bias, no relu
+    L2 = ubp_synth.make_layer("t", 48, 24, 4, 50, 6, Nc=128, bias=False, relu=False)
+    check(*run_spmm(env, L2)[:3], L2)
+    # Nb == M: one possible start row
+    L3 = ubp_synth.make_layer("t", 8, 40, 8, 50, 7, Nc=128)
+    check(*run_spmm(env, L3)[:3], L3)
+
+
+def test_spmm_bad_arguments(env):
+    torch, ubp = env
+    L = ubp_synth.make_layer("t", 32, 16, 4, 50, 5, Nc=64)
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, 4))
+    lib = ubp.load()
+    import ctypes as C
+    X = torch.zeros((16, 64), device="cuda"); Y = torch.zeros((32, 64), device="cuda")
+    vp = lambda t: C.c_void_p(t.data_ptr())
+    assert lib.ubp_spmm(plan.handle, None, 64, 64, None, 0, vp(Y), 64, None) == -1
+    assert lib.ubp_spmm(plan.handle, vp(X), 32, 64, None, 0, vp(Y), 64, None) == -1      # ldx < Nc
+    assert lib.ubp_spmm(plan.handle, vp(X), 64, -1, None, 0, vp(Y), 64, None) == -1
+    assert lib.ubp_spmm(None, vp(X), 64, 64, None, 0, vp(Y), 64, None) == -1
+    assert lib.ubp_conv3x3_implicit(plan.handle, vp(X), 1, 8, 8, 64, 64, None, 0, vp(Y), 64, 64, None) == -1  # R != 9
+    torch.cuda.synchronize()
+
+
+def test_spmm_is_bitwise_reproducible(env):
+    torch, ubp = env
+    L = ubp_synth.make_layer("t", 256, 256, 4, 70, 99, Nc=1024)
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, 4))
+    X = torch.from_numpy(L.X).cuda(); b = torch.from_numpy(L.bias).cuda()
+    Y1 = ubp.ubp_spmm(plan, X, b, True).clone()
+    Y2 = ubp.ubp_spmm(plan, X, b, True)
+    assert torch.equal(Y1, Y2)
+    # the slower kernel sums in the same order: identical bits
+    xb = torch.zeros(256 * 1024 + 1, device="cuda")
+    Xm = xb[1:].view(256, 1024); Xm.copy_(X)
+    Y3 = ubp.ubp_spmm(plan, Xm, b, True)
+    assert torch.equal(Y1, Y3)
+
+
+def test_fc64_config(env):
+    L = ubp_synth.config_layers("fc64")[0]
+    Yh, Yref, A, _ = run_spmm(env, L)
+    check(Yh, Yref, A, L)
+
+
+def test_mbv1_pw512_config_full(env):
+    """The benchmark workload at full size, every output compared."""
+    L = ubp_synth.config_layers("mbv1_pw512")[0]
+    assert (L.M, L.C, L.Nc, L.m) == (512, 512, 6272, 19660)
+    torch, ubp = env
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    assert blob == oracle.pack(L.W, L.mask, L.Nb)
+    plan = ubp.Plan(blob)
+    X = torch.from_numpy(L.X).cuda()                       # [C][B][H][W], channel-major
+    Y = ubp.ubp_conv1x1(plan, X, torch.from_numpy(L.bias).cuda(), True, layout="CNHW")
+    plan.check()
+    Yref, A = oracle.masked_matmul(L.W, L.mask, L.X.reshape(L.C, -1), L.bias, relu=True)
+    check(Y.cpu().numpy().reshape(L.M, -1), Yref, A, L)
+
+
+def test_conv1x1_nchw_matches_cnhw(env):
+    torch, ubp = env
+    L = ubp_synth.make_layer("t", 96, 64, 4, 70, 31, B=3, H=14, Wd=14)
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, 4))
+    b = torch.from_numpy(L.bias).cuda()
+    Xc = torch.from_numpy(L.X).cuda()
+    Yc = ubp.ubp_conv1x1(plan, Xc, b, True, layout="CNHW")
+    Xn = Xc.permute(1, 0, 2, 3).contiguous()
+    Yn = ubp.ubp_conv1x1(plan, Xn, b, True, layout="NCHW")
+    assert torch.equal(Yn.permute(1, 0, 2, 3), Yc)
+    Yref, A = oracle.masked_matmul(L.W, L.mask, L.X.reshape(L.C, -1), L.bias, relu=True)
+    check(Yc.cpu().numpy().reshape(L.M, -1), Yref, A, L)
+    # 7x7 planes: 196-byte rows, not 16-byte aligned per image -> slower kernel, same answer
+    L7 = ubp_synth.make_layer("t", 64, 32, 4, 70, 32, B=2, H=7, Wd=7)
+    p7 = ubp.Plan(ubp.ubp_pack(L7.W, L7.mask, 4))
+    X7 = torch.from_numpy(L7.X).cuda().permute(1, 0, 2, 3).contiguous()
+    Y7 = ubp.ubp_conv1x1(p7, X7, None, False, layout="NCHW").permute(1, 0, 2, 3).contiguous()
+    Yref, A = oracle.masked_matmul(L7.W, L7.mask, L7.X.reshape(L7.C, -1), None, relu=False)
+    check(Y7.cpu().numpy().reshape(L7.M, -1), Yref, A, L7)
+
+
+@pytest.mark.parametrize("nb,sp", [(2, 50), (4, 70), (8, 80), (16, 90)])
+def test_sweep_config_sampled(env, nb, sp):
+    """Full-size sweep point (M = K = 2048, Nc = 8192): sampled outputs against the oracle one by one."""
+    torch, ubp = env
+    L = ubp_synth.config_layers("sweep", Nb=nb, sparsity_pct=sp)[0]
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    assert blob == oracle.pack(L.W, L.mask, L.Nb)
+    plan = ubp.Plan(blob)
+    Y = ubp.ubp_spmm(plan, torch.from_numpy(L.X).cuda()).cpu().numpy()
+    plan.check()
+    rng = np.random.default_rng(nb * 100 + sp)
+    so = np.concatenate([rng.integers(0, L.M, 4000), [0, L.M - 1, 0, L.M - 1]])
+    sn = np.concatenate([rng.integers(0, L.Nc, 4000), [0, 0, L.Nc - 1, L.Nc - 1]])
+    ys, as_ = oracle.masked_matmul_samples(L.W, L.mask, L.X, so, sn)
+    err = scaled_error(Y[so, sn], ys, as_)
+    assert err <= TOL and err <= (terms_per_output(L) + 2) * 2.0 ** -24
+    # whole rows too (a panel's first / last row and one in the middle)
+    for o in (0, 15, 16, 1000, L.M - 1):
+        sn2 = np.arange(L.Nc)
+        ys, as_ = oracle.masked_matmul_samples(L.W, L.mask, L.X, np.full(L.Nc, o), sn2)
+        assert scaled_error(Y[o], ys, as_) <= TOL
+
+
+@pytest.mark.parametrize("li", [0, 1, 3, 5, 11, 12])
+def test_mbv1_chain_layers_sampled(env, li):
+    torch, ubp = env
+    L = ubp_synth.config_layers("mbv1_chain", batch=8 if li < 2 else 64)[li]
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb))
+    Y = ubp.ubp_conv1x1(plan, torch.from_numpy(L.X).cuda(), torch.from_numpy(L.bias).cuda(), True)
+    plan.check()
+    Y = Y.cpu().numpy().reshape(L.M, -1)
+    X2 = L.X.reshape(L.C, -1)
+    rng = np.random.default_rng(li)
+    so = rng.integers(0, L.M, 5000); sn = rng.integers(0, X2.shape[1], 5000)
+    sn[:4] = [0, X2.shape[1] - 1, X2.shape[1] - 2, 1]
+    ys, as_ = oracle.masked_matmul_samples(L.W, L.mask, X2, so, sn, L.bias, relu=True)
+    assert scaled_error(Y[so, sn], ys, as_) <= TOL
+
+
+# ------------------------------------------------------------------ 3x3
+@pytest.mark.parametrize("M,C,Nb,p,B,H,Wd", [(16, 8, 4, 50, 2, 6, 5), (40, 20, 8, 60, 3, 14, 14), (24, 18, 2, 50, 1, 7, 9),
+                                              (30, 10, 6, 40, 2, 4, 4), (17, 9, 1, 60, 2, 3, 5), (32, 40, 16, 50, 1, 8, 8)])
+def test_conv3x3_small(env, M, C, Nb, p, B, H, Wd):
+    torch, ubp = env
+    L = ubp_synth.make_layer("c", M, C, Nb, p, 7 * M + C, B=B, H=H, Wd=Wd, R=9, x_dist="normal")
+    blob = ubp.ubp_pack(L.W, L.mask, Nb)
+    assert blob == oracle.pack(L.W, L.mask, Nb)
+    plan = ubp.Plan(blob)
+    b = torch.from_numpy(L.bias).cuda()
+    Y = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda(), b, True, layout="CNHW")
+    Yref, A = oracle.masked_conv3x3(L.W, L.mask, L.X, L.bias, relu=True)
+    check(Y.cpu().numpy(), Yref, A, L)
+    Yn = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda().permute(1, 0, 2, 3).contiguous(), b, True, layout="NCHW")
+    assert torch.equal(Yn.permute(1, 0, 2, 3), Y)
+
+
+def test_r50_3x3_config_sampled(env):
+    torch, ubp = env
+    L = ubp_synth.config_layers("r50_3x3")[0]
+    assert (L.M, L.C, L.m, L.B) == (256, 256, 1638, 64)
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    assert blob == oracle.pack(L.W, L.mask, L.Nb)
+    plan = ubp.Plan(blob)
+    Y = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda(), torch.from_numpy(L.bias).cuda(), True).cpu().numpy()
+    rng = np.random.default_rng(3)
+    n = 6000
+    sb = rng.integers(0, L.B, n); so = rng.integers(0, L.M, n); sy = rng.integers(0, 14, n); sx = rng.integers(0, 14, n)
+    sy[:8] = [0, 0, 13, 13, 0, 13, 7, 7]; sx[:8] = [0, 13, 0, 13, 7, 7, 0, 13]          # corners and edges
+    ys, as_ = oracle.masked_conv3x3_samples(L.W, L.mask, L.X, sb, so, sy, sx, L.bias, relu=True)
+    err = scaled_error(Y[so, sb, sy, sx], ys, as_)
+    assert err <= TOL and err <= (terms_per_output(L) + 2) * 2.0 ** -24

@@ -86,8 +86,9 @@ def random_mask(M: int, C: int, Nb: int, sparsity_pct: int, seed: int,
 @dataclass
 class Layer:
     """One synthetic UBP layer. ``W`` is [M][C][R] (R = taps: 1 or 9),
-    ``mask`` is [M][C]; ``X`` is [C][Nc] for R == 1 and [C][B][H][Wd] for the
-    3x3 case (channel-major activations, columns n = (b, y, x))."""
+    ``mask`` is [M][C]; ``X`` is [C][Nc] when the layer was made with an explicit
+    column count and [C][B][H][Wd] otherwise (channel-major activations,
+    columns n = (b, y, x))."""
     name: str
     M: int
     C: int
@@ -130,9 +131,8 @@ def make_layer(name: str, M: int, C: int, Nb: int, sparsity_pct: int, seed: int,
         W = rng.uniform(-w_scale, w_scale, size=(M, C, R)).astype(np.float32)
     else:
         W = (rng.standard_normal(size=(M, C, R), dtype=np.float32) * np.float32(w_scale)).astype(np.float32)
-    if R == 1:
-        ncols = Nc if Nc is not None else B * H * Wd
-        xshape = (C, ncols)
+    if Nc is not None:
+        xshape = (C, Nc)
     else:
         xshape = (C, B, H, Wd)
     if make_x:
