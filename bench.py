@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the UBP inference path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+                    [--variant V] [--table FILE]
+
+One "step" = one pass of the inference hot path over one batch of synthetic
+activations already resident in HBM: a single launch of the layer's kernel
+(packing and plan building are the offline model-conversion steps; their
+host time is reported separately as pack_ms / plan_ms). The default workload
+is the MobileNetV1-shaped pointwise layer 512->512 at 14x14, batch 32, 1x4
+blocks, 70 % sparsity, fused bias+ReLU. L2 is flushed between steps (the
+26 MB working set would otherwise stay cached).
+
+Prints ONE JSON line (rank 0). With N > 1 (torchrun) every rank runs the
+same layer on its own batch (columns are independent: no collective on the
+path), value = total work / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import ubp_synth  # noqa: E402
+
+SM_COUNT, FP32_LANES, SM_MAX_GHZ = 148, 128, 1.965
+FP32_PEAK_TFLOPS = SM_COUNT * FP32_LANES * 2 * SM_MAX_GHZ / 1e3     # 74.45: plain FP32 FMA pipes at max clock
+
+WORKLOADS = {
+    "mbv1_pw512": dict(cfg="mbv1_pw512", kw={}),
+    "fc64": dict(cfg="fc64", kw={}),
+    "r50_3x3": dict(cfg="r50_3x3", kw={}),
+}
+for _nb in (2, 4, 8, 16):
+    for _sp in (50, 70, 80, 90):
+        WORKLOADS[f"sweep_nb{_nb}_p{_sp}"] = dict(cfg="sweep", kw=dict(Nb=_nb, sparsity_pct=_sp))
+for _li in range(13):
+    WORKLOADS[f"mbv1_L{_li + 1}"] = dict(cfg="mbv1_chain", kw={}, index=_li)
+
+
+def get_layer(name: str, seed_index: int = 0):
+    w = WORKLOADS[name]
+    layers = ubp_synth.config_layers(w["cfg"], index=seed_index, **w["kw"])
+    return layers[w.get("index", 0)]
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def compulsory_bytes(L) -> int:
+    """Activations read once + outputs written once + packed weights/indices + bias."""
+    x = L.X.size * 4
+    y = L.M * L.Nc * 4
+    w = L.m * L.Nb * L.R * 4 + L.m * 4 + (L.M + 1) * 4 + (L.M * 4 if L.bias is not None else 0)
+    return x + y + w
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason sampling during the timed region."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx = float(f[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def build_runner(ubp, torch, L, variant):
+    """Returns (plan, run(stream-less call), pack_ms, plan_ms, device tensors)."""
+    t0 = time.perf_counter()
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    t1 = time.perf_counter()
+    plan = ubp.Plan(blob, variant)
+    torch.cuda.synchronize()
+    t2 = time.perf_counter()
+    X = torch.from_numpy(L.X).cuda()
+    bias = torch.from_numpy(L.bias).cuda() if L.bias is not None else None
+    if L.R == 9:
+        Y = torch.empty((L.M, L.B, L.H, L.Wd), dtype=torch.float32, device="cuda")
+        run = lambda: ubp.ubp_conv3x3_implicit(plan, X, bias, L.relu, out=Y)
+    elif L.X.ndim == 4:
+        Y = torch.empty((L.M, L.B, L.H, L.Wd), dtype=torch.float32, device="cuda")
+        run = lambda: ubp.ubp_conv1x1(plan, X, bias, L.relu, out=Y)
+    else:
+        Y = torch.empty((L.M, L.Nc), dtype=torch.float32, device="cuda")
+        run = lambda: ubp.ubp_spmm(plan, X, bias, L.relu, out=Y)
+    return plan, run, (t1 - t0) * 1e3, (t2 - t1) * 1e3, X, Y, bias
+
+
+def time_steps(torch, run, steps, warmup, flush_buf):
+    """Per-step device times (ms) with CUDA events on the current stream; L2 flushed before every step."""
+    for _ in range(warmup):
+        if flush_buf is not None:
+            flush_buf.zero_()
+        run()
+    torch.cuda.synchronize()
+    evs = []
+    for _ in range(steps):
+        if flush_buf is not None:
+            flush_buf.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); run(); b.record()
+        evs.append((a, b))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in evs]
+
+
+def time_e2e(torch, ubp, plan, L, steps, warmup):
+    """Same step through the public call with HOST buffers: pinned X -> device, kernel, Y -> pinned host."""
+    Xh = torch.from_numpy(L.X).pin_memory()
+    Xd = torch.empty_like(Xh, device="cuda")
+    bias = torch.from_numpy(L.bias).cuda() if L.bias is not None else None
+    shape = (L.M, L.B, L.H, L.Wd) if L.X.ndim == 4 else (L.M, L.Nc)
+    Yd = torch.empty(shape, dtype=torch.float32, device="cuda")
+    Yh = torch.empty(shape, dtype=torch.float32).pin_memory()
+
+    def step():
+        Xd.copy_(Xh, non_blocking=True)
+        if L.R == 9:
+            ubp.ubp_conv3x3_implicit(plan, Xd, bias, L.relu, out=Yd)
+        elif L.X.ndim == 4:
+            ubp.ubp_conv1x1(plan, Xd, bias, L.relu, out=Yd)
+        else:
+            ubp.ubp_spmm(plan, Xd, bias, L.relu, out=Yd)
+        Yh.copy_(Yd, non_blocking=True)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / steps, Xh.numel() * 4, Yh.numel() * 4
+
+
+def cpu_oracle_time(L, budget_s=20.0):
+    """The oracle as it stands on the host cores, on a bounded sample of the workload's columns."""
+    import oracle
+    dense_macs_per_col = L.M * L.C * L.R
+    # aim at ~1 GMAC per timed call, at least 64 columns (3x3: whole images)
+    if L.R == 9:
+        nb = max(1, min(L.B, int(1.0e9 // (dense_macs_per_col * L.H * L.Wd * 0.2 + 1))))
+        Xs = np.ascontiguousarray(L.X[:, :nb])
+        cols = nb * L.H * L.Wd
+        fn = lambda: oracle.masked_conv3x3(L.W, L.mask, Xs, L.bias, relu=L.relu)
+        sample = f"first {nb} of {L.B} images"
+    else:
+        X2 = L.X.reshape(L.C, -1)
+        cols = int(max(64, min(X2.shape[1], 1.5e9 // dense_macs_per_col)))
+        Xs = np.ascontiguousarray(X2[:, :cols])
+        fn = lambda: oracle.masked_matmul(L.W, L.mask, Xs, L.bias, relu=L.relu)
+        sample = f"first {cols} of {X2.shape[1]} columns"
+    fn()
+    ts = []
+    t_start = time.perf_counter()
+    while len(ts) < 3 and time.perf_counter() - t_start < budget_s:
+        t0 = time.perf_counter(); fn(); ts.append(time.perf_counter() - t0)
+    t = float(np.median(ts))
+    flops = 2.0 * L.m * L.Nb * L.R * cols
+    return flops / t / 1e9, oracle.num_threads(), sample, t
+
+
+def run_reference(args, L, name):
+    """--impl reference: the CPU oracle timed on this machine's host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    vals = []
+    sample = ""
+    for i in range(args.warmup + args.steps):
+        g, cores, sample, t = cpu_oracle_time(L, budget_s=1.0)
+        if i >= args.warmup:
+            vals.append((g, t))
+        if i >= args.warmup + 2 and sum(t for _, t in vals) > 90:
+            break
+    g = float(np.median([v for v, _ in vals]))
+    t = float(np.median([t for _, t in vals]))
+    line = {"metric": "effective GFLOP/s (2 x surviving MACs / time) of one UBP layer", "value": g, "unit": "GFLOP/s",
+            "impl": "reference", "n_gpus": args.gpus, "steps": len(vals), "warmup": args.warmup,
+            "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": name, "sample": sample},
+            "cpu_baseline": {"value": g, "unit": "GFLOP/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": g, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--workload", default="mbv1_pw512")
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    ap.add_argument("--no-flush", action="store_true", help="do not flush L2 between steps (warm-L2 figure)")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    name = args.workload
+    L = get_layer(name, seed_index=rank)
+
+    if args.impl == "reference":
+        run_reference(args, L, name)
+        return
+
+    import torch
+    import paper_2407_19644_b200 as ubp
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    ubp.load()
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    plan, run, pack_ms, plan_ms, X, Y, bias = build_runner(ubp, torch, L, args.variant)
+    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+
+    sampler = ClockSampler(local_rank)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    times = time_steps(torch, run, args.steps, args.warmup, flush)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    plan.check()
+    step_ms = float(np.mean(times))
+    if dist is not None:
+        t = torch.tensor([step_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_ms = float(t.item())
+    e2e_ms, h2d, d2h = time_e2e(torch, ubp, plan, L, max(5, min(args.steps, 30)), 3)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    flops = 2.0 * L.surviving_macs
+    gflops = world * flops / (step_ms * 1e-3) / 1e9
+    hbm_gbs, peak_src = measured_peaks()
+    t_alu = flops / (FP32_PEAK_TFLOPS * 1e12)
+    t_hbm = compulsory_bytes(L) / (hbm_gbs * 1e9)
+    per_gpu_tflops = flops / (step_ms * 1e-3) / 1e12
+    if t_alu >= t_hbm:
+        roof = {"bound": "alu", "achieved": per_gpu_tflops, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s",
+                "frac": per_gpu_tflops / FP32_PEAK_TFLOPS, "traffic": None,
+                "peak_source": "148 SMs x 128 FP32 lanes x 2 x 1.965 GHz (derived)"}
+    else:
+        ach = compulsory_bytes(L) / (step_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s", "frac": ach / hbm_gbs,
+                "traffic": None, "peak_source": f"{peak_src} copy bandwidth"}
+    roof["roofline_us"] = max(t_alu, t_hbm) * 1e6
+    roof["frac_of_roofline_time"] = max(t_alu, t_hbm) / (step_ms * 1e-3)
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        with open(prof) as f:
+            roof["traffic"] = json.load(f).get(name)
+
+    line = {
+        "metric": "effective GFLOP/s (2 x surviving MACs / time) of one UBP layer", "value": gflops, "unit": "GFLOP/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
+        "us_per_layer": step_ms * 1e3, "us_min": float(np.min(times)) * 1e3, "us_median": float(np.median(times)) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": name, "M": L.M, "K": L.C * L.R, "Nc": L.Nc, "block": f"{L.Nb}x1x{L.R}",
+                   "sparsity_pct": L.sparsity_pct, "blocks": L.m, "bias": L.bias is not None, "relu": bool(L.relu),
+                   "variant": plan.variant, "l2": "warm" if args.no_flush else "flushed between steps (256 MiB write)",
+                   "parallelism": f"replicated weights, columns sharded x{world}"},
+        "roofline": roof, "clocks": clocks, "gpu_launches": args.steps,
+        "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e9, "unit": "GFLOP/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "offline": {"pack_ms": pack_ms, "plan_ms": plan_ms, "plan_bytes": plan.dev_bytes},
+    }
+    if rank == 0 and not args.no_cpu:
+        g, cores, sample, _ = cpu_oracle_time(L)
+        line["cpu_baseline"] = {"value": g, "unit": "GFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()
