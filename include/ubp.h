@@ -107,8 +107,8 @@ int ubp_plan_size(const void *blob, size_t len, int variant, size_t *dev_bytes);
  *   [256,..) uint32 group_off[nkt*NG + 1] in 16-byte units, groups in (tile, row group) order;
  *   group: uint32 poff[WR+1] (padded to 16), then per panel
  *          uint16 fo[F+1] (F = panel_rows + nbk - 1 start offsets, padded to 16),
- *          uint16 jl[n] (input channel inside the tile, padded to 16),
- *          float  w[n][nbk][R] (weights in row order, i.e. with the rotation undone).
+ *          uint16 jl[n+4] (input channel inside the tile; 4 trailing zeros so a kernel may read ahead; padded to 16),
+ *          float  w[n+2][nbk][R] (weights in row order, i.e. with the rotation undone; 2 trailing zero entries).
  * geom receives {nbk, panel_rows, k_tile, WR, dupw, nkt, NP, NG}. */
 int ubp_plan_image(const void *blob, size_t len, int variant, void *host_buf, size_t cap, int32_t geom[8]);
 

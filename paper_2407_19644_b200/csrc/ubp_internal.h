@@ -41,8 +41,8 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m);
 //   groups in (kt, g) order, each 16-byte aligned:
 //       uint32 poff[WR + 1]            byte offsets of the panel sub-segments from the group start
 //       per panel: uint16 fo[F + 1]    entry offsets per fragment (F = P + nbk - 1), padded to 16
-//                  uint16 jl[n]        input channel inside the tile, padded to 16
-//                  float  w[n][nbk][R][dup]   un-rotated weights of the entry, padded to 16
+//                  uint16 jl[n + 4]    input channel inside the tile (4 zero entries of read-ahead slack), padded to 16
+//                  float  w[n + 2][nbk][R][dup]   un-rotated weights of the entry (2 zero entries of slack), padded to 16
 struct PlanImage {
     std::vector<uint8_t> bytes;
     int nkt = 0, NP = 0, NG = 0, F = 0;

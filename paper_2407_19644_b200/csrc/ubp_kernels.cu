@@ -113,42 +113,78 @@ __device__ __forceinline__ void load_floats(float (&w)[N], const float *p)
 // One fragment = all entries of this (panel, tile) whose first row sits at
 // offset S inside the panel (S may be negative for an entry that started in the
 // panel above). Rows outside [0, P) are clipped at compile time.
-template <int NBK, int P, int V, int S, bool DUPW, int XROW_BYTES>
-__device__ __forceinline__ void run_fragment(float2 (&acc)[P][2 * V], const uint8_t *xs_lane,
-                                             const uint16_t *jl, const float *wv, int e0, int e1)
+//
+// The entry stream of a panel is contiguous across fragments, so the loads of
+// entry e+1 (activation row, weights) and the channel index of entry e+2 are
+// issued before the multiply-adds of entry e: a two-deep software pipeline
+// that runs straight through fragment boundaries.
+template <int V, int WF>
+struct EntryRegs {
+    float4 x[V];
+    float w[WF];
+};
+
+template <int V, int WF, int XROW_BYTES>
+__device__ __forceinline__ void fetch_entry(EntryRegs<V, WF> &r, const uint8_t *xs_lane, uint32_t j,
+                                            const float *wv, int e)
+{
+    const uint8_t *xp = xs_lane + j * (uint32_t)XROW_BYTES;
+#pragma unroll
+    for (int v = 0; v < V; ++v) r.x[v] = *reinterpret_cast<const float4 *>(xp + v * 512);
+    load_floats<WF>(r.w, wv + (size_t)e * WF);
+}
+
+template <int NBK, int P, int V, int S, bool DUPW>
+__device__ __forceinline__ void fma_entry(float2 (&acc)[P][2 * V], const EntryRegs<V, NBK * (DUPW ? 2 : 1)> &r)
 {
     constexpr int R_LO = (S < 0) ? -S : 0;
     constexpr int R_HI = (S + NBK > P) ? (P - S) : NBK;
-    constexpr int WF = NBK * (DUPW ? 2 : 1);
-    for (int e = e0; e < e1; ++e) {
-        const uint32_t j = jl[e];
-        const uint8_t *xp = xs_lane + j * (uint32_t)XROW_BYTES;
-        float4 x[V];
 #pragma unroll
-        for (int v = 0; v < V; ++v) x[v] = *reinterpret_cast<const float4 *>(xp + v * 512);
-        float w[WF];
-        load_floats<WF>(w, wv + (size_t)e * WF);
+    for (int q = R_LO; q < R_HI; ++q) {
+        const float2 w2 = DUPW ? make_float2(r.w[2 * q], r.w[2 * q + 1]) : make_float2(r.w[q], r.w[q]);
 #pragma unroll
-        for (int r = R_LO; r < R_HI; ++r) {
-            const float2 w2 = DUPW ? make_float2(w[2 * r], w[2 * r + 1]) : make_float2(w[r], w[r]);
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                acc[S + r][2 * v] = fma2(w2, make_float2(x[v].x, x[v].y), acc[S + r][2 * v]);
-                acc[S + r][2 * v + 1] = fma2(w2, make_float2(x[v].z, x[v].w), acc[S + r][2 * v + 1]);
-            }
+        for (int v = 0; v < V; ++v) {
+            acc[S + q][2 * v] = fma2(w2, make_float2(r.x[v].x, r.x[v].y), acc[S + q][2 * v]);
+            acc[S + q][2 * v + 1] = fma2(w2, make_float2(r.x[v].z, r.x[v].w), acc[S + q][2 * v + 1]);
         }
     }
 }
 
+// Pipeline state carried across fragments: `cur` holds entry e, jn = channel of entry e+1.
+template <int V, int WF>
+struct PipeState {
+    EntryRegs<V, WF> cur;
+    uint32_t jn;
+    int e;
+};
+
 template <int NBK, int P, int V, bool DUPW, int XROW_BYTES, int F0, int F1>
 struct FragmentLoop {
-    __device__ __forceinline__ static void run(float2 (&acc)[P][2 * V], const uint8_t *xs_lane,
-                                               const uint16_t *fo, const uint16_t *jl, const float *wv, int e0)
+    static constexpr int WF = NBK * (DUPW ? 2 : 1);
+    __device__ __forceinline__ static void run(float2 (&acc)[P][2 * V], PipeState<V, WF> &ps, const uint8_t *xs_lane,
+                                               const uint16_t *fo, const uint16_t *jl, const float *wv)
     {
         if constexpr (F0 < F1) {
+            constexpr int S = F0 - (NBK - 1);
             const int e1 = fo[F0 + 1];
-            run_fragment<NBK, P, V, F0 - (NBK - 1), DUPW, XROW_BYTES>(acc, xs_lane, jl, wv, e0, e1);
-            FragmentLoop<NBK, P, V, DUPW, XROW_BYTES, F0 + 1, F1>::run(acc, xs_lane, fo, jl, wv, e1);
+            EntryRegs<V, WF> nxt;
+            while (ps.e + 2 <= e1) {
+                fetch_entry<V, WF, XROW_BYTES>(nxt, xs_lane, ps.jn, wv, ps.e + 1);
+                const uint32_t j2 = jl[ps.e + 2];
+                fma_entry<NBK, P, V, S, DUPW>(acc, ps.cur);
+                fetch_entry<V, WF, XROW_BYTES>(ps.cur, xs_lane, j2, wv, ps.e + 2);
+                ps.jn = jl[ps.e + 3];
+                fma_entry<NBK, P, V, S, DUPW>(acc, nxt);
+                ps.e += 2;
+            }
+            if (ps.e < e1) {
+                fetch_entry<V, WF, XROW_BYTES>(nxt, xs_lane, ps.jn, wv, ps.e + 1);
+                ps.jn = jl[ps.e + 2];
+                fma_entry<NBK, P, V, S, DUPW>(acc, ps.cur);
+                ps.cur = nxt;
+                ps.e += 1;
+            }
+            FragmentLoop<NBK, P, V, DUPW, XROW_BYTES, F0 + 1, F1>::run(acc, ps, xs_lane, fo, jl, wv);
         }
     }
 };
@@ -252,9 +288,14 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
             const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
             const int n = fo[F];
             const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
-            const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * n + 15) & ~15));
+            const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * (n + 4) + 15) & ~15));
             const uint8_t *xs_lane = stage + (wc * 128 * V + lane * 4) * 4;
-            FragmentLoop<NBK, P, V, DUPW, CS * 4, 0, F>::run(acc, xs_lane, fo, jl, wv, 0);
+            // the plan pads jl with 4 zero entries and w with 2 zero entries, so the pipeline may read ahead
+            PipeState<V, WF> ps;
+            ps.e = 0;
+            fetch_entry<V, WF, CS * 4>(ps.cur, xs_lane, jl[0], wv, 0);
+            ps.jn = jl[1];
+            FragmentLoop<NBK, P, V, DUPW, CS * 4, 0, F>::run(acc, ps, xs_lane, fo, jl, wv);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bar_empty[st]));
@@ -344,7 +385,7 @@ ubp_spmm_simple_kernel(const uint8_t *plan, const float *X, int64_t ldx, int64_t
         const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
         const int n = fo[F];
         const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
-        const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * n + 15) & ~15));
+        const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * (n + 4) + 15) & ~15));
         const float *xcol = X + (size_t)kt * KT * ldx + (live ? col : 0);
         SimpleLoop<NBK, P, 0, F>::run(acc, xcol, ldx, live, fo, jl, wv, NBK * wdup, wdup, 0);
     }
@@ -427,7 +468,7 @@ ubp_conv3x3_simple_kernel(const uint8_t *plan, const float *in, int B, int H, in
         const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
         const int cnt = fo[F];
         const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
-        const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * cnt + 15) & ~15));
+        const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * (cnt + 4) + 15) & ~15));
         ConvLoop<NBK, P, 0, F>::run(acc, inb, isc, y, x, H, Wd, live, fo, jl, wv, kt * KT, 0);
     }
     if (!live) return;

@@ -126,7 +126,7 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
                 for (int f = 0; f < F; ++f) n += cnt[bucket(kt, p, f)];
                 if (n > 65535) return UBP_E_UNSUPPORTED;
                 seg_off[(size_t)kt * NP + p] = cur;
-                cur += fo_bytes + pad16(2 * n) + pad16(4 * n * wfloats);
+                cur += fo_bytes + pad16(2 * (n + 4)) + pad16(4 * (n + 2) * wfloats);
             }
             if (cur - g0 > max_group) max_group = (uint32_t)(cur - g0);
         }
@@ -161,7 +161,7 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
                         acc += cnt[bucket(kt, p, f)];
                     }
                     fo[F] = (uint16_t)acc;
-                    end = so + fo_bytes + pad16(2 * (size_t)acc) + pad16(4 * (size_t)acc * wfloats);
+                    end = so + fo_bytes + pad16(2 * ((size_t)acc + 4)) + pad16(4 * ((size_t)acc + 2) * wfloats);
                 } else {
                     poff[w] = (uint32_t)(end - g0);
                 }
@@ -174,7 +174,7 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         const size_t n = fo[F];
         const uint32_t e = cursor[bucket(kt, p, f)]++;
         uint16_t *jl_arr = reinterpret_cast<uint16_t *>(base + so + fo_bytes);
-        float *w_arr = reinterpret_cast<float *>(base + so + fo_bytes + pad16(2 * n));
+        float *w_arr = reinterpret_cast<float *>(base + so + fo_bytes + pad16(2 * (n + 4)));
         jl_arr[e] = (uint16_t)jl;
         float *dst = w_arr + (size_t)e * wfloats;
         if (cfg.dupw) {

@@ -31,8 +31,9 @@ def plan_to_dense(img: np.ndarray, geom: dict, M: int, C: int, R: int):
                 n = int(fo[F])
                 assert (np.diff(fo.astype(np.int64)) >= 0).all() and fo[0] == 0
                 jl = np.frombuffer(img, "<u2", n, so + fo_bytes)
-                w = np.frombuffer(img, "<f4", n * nbk * R * dup, so + fo_bytes + pad16(2 * n)).reshape(n, nbk, R, dup)
-                assert so + fo_bytes + pad16(2 * n) + pad16(4 * n * nbk * R * dup) == g0 + int(poff[wr + 1])
+                w = np.frombuffer(img, "<f4", n * nbk * R * dup, so + fo_bytes + pad16(2 * (n + 4))).reshape(n, nbk, R, dup)
+                assert so + fo_bytes + pad16(2 * (n + 4)) + pad16(4 * (n + 2) * nbk * R * dup) == g0 + int(poff[wr + 1])
+                assert not np.frombuffer(img, "<u2", 4, so + fo_bytes + 2 * n).any()      # read-ahead slack is zero
                 n_entries += n
                 for f in range(F):
                     s = f - (nbk - 1)
