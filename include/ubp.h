@@ -34,7 +34,8 @@ typedef enum {
     UBP_E_FORMAT = -4,    /* blob or plan is not what it claims to be                       */
     UBP_E_CUDA = -5,      /* a CUDA runtime/driver call failed (see ubp_last_cuda_error)    */
     UBP_E_UNSUPPORTED = -6,
-    UBP_E_DEVICE = -7     /* a kernel reported a bounded wait that ran out                  */
+    UBP_E_DEVICE = -7,    /* a kernel reported a bounded wait that ran out                  */
+    UBP_E_STATIC_LIMIT = -8 /* layer too large for the fixed scratch of ubp_spmm_static      */
 } ubp_status;
 
 const char *ubp_strerror(int status);
@@ -168,6 +169,39 @@ int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, 
                          int64_t in_stride_b, int64_t in_stride_c,
                          const float *bias, int relu,
                          float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);
+
+/* ubp_spmm_static: same result as ubp_spmm, for callers that cannot allocate.
+ * (The paper has no counterpart; this is a deployment convenience.)
+ *
+ * Who needs it: code that has to run a UBP layer but may not obtain device
+ * memory at that point -- a plug-in living inside another engine that owns the
+ * whole device heap, a service whose memory budget was fixed at start-up, a
+ * caller on a path where an allocation (and the implicit synchronisation and
+ * possible failure that come with it) is not acceptable. ubp_spmm needs a
+ * device buffer for the plan; here the plan goes into a fixed array of
+ * ubp_static_plan_capacity() bytes (2 MiB) that is part of the library's
+ * device image, so every GPU that loads the library holds those 2 MiB until
+ * the process ends, whether or not this function is ever called.
+ *
+ *   blob/len   host: canonical packed layer (R == 1), as made by ubp_pack
+ *   X, bias, Y device, same meaning and alignment rules as ubp_spmm
+ * The plan is rebuilt on the host from the blob on EVERY call (host time of the
+ * order of a millisecond for a 512x512 layer) and uploaded with one
+ * cudaMemcpyAsync from pageable memory -- which may wait for earlier work on
+ * `stream` -- then the same kernel as ubp_spmm is launched. The function calls
+ * no cudaMalloc / cudaFree and no other device-allocating routine.
+ * First call on a device: resolves the array's device address
+ * (cudaGetSymbolAddress) with that device current; make that first call
+ * outside any stream capture.
+ * All calls on a device share the one array: two calls whose GPU work overlaps
+ * (different streams, or threads) race on it -- serialise them. The array
+ * keeps the previous call's plan until the next upload overwrites it; the
+ * upload rewrites the status word, so nothing has to be cleared by the caller.
+ * Errors: as ubp_spmm, plus UBP_E_FORMAT (bad blob) and UBP_E_STATIC_LIMIT when
+ * the layer's plan does not fit the array (use ubp_plan_build / ubp_spmm then). */
+size_t ubp_static_plan_capacity(void);
+int ubp_spmm_static(const void *blob, size_t len, const float *X, int64_t ldx, int64_t Nc,
+                    const float *bias, int relu, float *Y, int64_t ldy, void *stream);
 
 #ifdef __cplusplus
 }

@@ -7,7 +7,9 @@ device memory and streams. There is no CPU fallback: if the shared library
 is missing or a call fails, an exception is raised.
 """
 from .binding import (UbpError, Plan, pack_ubp, unpack_ubp, blob_view, plan_size, plan_image, variants,
-                      ubp_pack, ubp_unpack, ubp_spmm, ubp_conv1x1, ubp_conv3x3_implicit, lib_path, load)
+                      ubp_pack, ubp_unpack, ubp_spmm, ubp_conv1x1, ubp_conv3x3_implicit, ubp_spmm_static,
+                      static_plan_capacity, lib_path, load)
 
 __all__ = ["UbpError", "Plan", "pack_ubp", "unpack_ubp", "blob_view", "plan_size", "plan_image", "variants",
-           "ubp_pack", "ubp_unpack", "ubp_spmm", "ubp_conv1x1", "ubp_conv3x3_implicit", "lib_path", "load"]
+           "ubp_pack", "ubp_unpack", "ubp_spmm", "ubp_conv1x1", "ubp_conv3x3_implicit", "ubp_spmm_static",
+           "static_plan_capacity", "lib_path", "load"]

@@ -61,6 +61,8 @@ def load():
     L.ubp_spmm.argtypes = [vp, vp, i64, i64, vp, i32, vp, i64, vp]
     L.ubp_conv1x1.argtypes = [vp, vp, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
     L.ubp_conv3x3_implicit.argtypes = [vp, vp, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
+    L.ubp_static_plan_capacity.restype = sz
+    L.ubp_spmm_static.argtypes = [vp, sz, vp, i64, i64, vp, i32, vp, i64, vp]
     _lib = L
     return L
 
@@ -277,3 +279,32 @@ def ubp_conv3x3_implicit(plan: Plan, x, bias=None, relu: bool = False, out=None,
                                             _dev_ptr(bias, "bias", True), int(bool(relu)), _dev_ptr(out, "out"),
                                             osb, osc, _stream_ptr(stream)), "ubp_conv3x3_implicit")
     return out
+
+
+def ubp_spmm_static(blob: bytes, X, bias=None, relu: bool = False, out=None, stream=None):
+    """ubp_spmm without a Plan object: for callers that must not allocate device memory.
+
+    The plan is rebuilt from `blob` on the host and uploaded into the library's fixed 2 MiB device
+    array on every call, so pass `out` (preallocated [M][Nc]) -- then nothing in this call allocates on the
+    device. Calls whose GPU work could overlap share that array and must be serialised by the caller.
+    Raises UbpError(-8) when the layer's plan does not fit the array."""
+    import torch
+    L = load()
+    b = np.frombuffer(blob, np.uint8)
+    d = blob_view(blob)
+    if X.dim() != 2 or X.shape[0] != d["C"] or (X.stride(1) != 1 and X.shape[1] > 1):
+        raise ValueError("X must be [C][Nc] with unit column stride")
+    Nc = X.shape[1]
+    if out is None:
+        out = torch.empty((d["M"], Nc), dtype=torch.float32, device=X.device)
+    if tuple(out.shape) != (d["M"], Nc) or (out.stride(1) != 1 and Nc > 1):
+        raise ValueError("out must be [M][Nc] with unit column stride")
+    with torch.cuda.device(X.device):
+        _chk(L.ubp_spmm_static(_np_ptr(b), b.size, _dev_ptr(X, "X"), X.stride(0), Nc, _dev_ptr(bias, "bias", True),
+                               int(bool(relu)), _dev_ptr(out, "out"), out.stride(0), _stream_ptr(stream)),
+             "ubp_spmm_static")
+    return out
+
+
+def static_plan_capacity() -> int:
+    return int(load().ubp_static_plan_capacity())

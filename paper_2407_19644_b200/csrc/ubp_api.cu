@@ -29,6 +29,7 @@ const char *ubp_strerror(int status)
         case UBP_E_CUDA: return "CUDA call failed";
         case UBP_E_UNSUPPORTED: return "unsupported configuration";
         case UBP_E_DEVICE: return "a kernel gave up on a bounded wait";
+        case UBP_E_STATIC_LIMIT: return "layer's plan exceeds the fixed device scratch of ubp_spmm_static";
         default: return "unknown status";
     }
 }

@@ -1,0 +1,49 @@
+"""ubp_spmm_static: the entry point for callers that cannot allocate device memory (its plan lives in a fixed
+array inside the library). Checked against ubp_spmm on two calls in a row -- the second call finds the
+first call's plan still in the array and must replace it. Collected last on purpose."""
+import numpy as np
+import pytest
+
+import ubp_synth
+
+pytestmark = pytest.mark.gpu
+
+
+def test_static_entry_matches_planned_entry_twice():
+    import torch
+    import paper_2407_19644_b200 as ubp
+    assert ubp.static_plan_capacity() == 2 * 1024 * 1024
+    layers = [ubp_synth.make_layer("a", 200, 150, 4, 70, 501, Nc=520, x_dist="normal"),
+              ubp_synth.make_layer("b", 96, 260, 8, 60, 502, Nc=300, x_dist="normal", relu=False)]
+    for L in layers:                                   # two calls in a row, different layers
+        blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+        X = torch.from_numpy(L.X).cuda()
+        bias = torch.from_numpy(L.bias).cuda()
+        want = ubp.ubp_spmm(ubp.Plan(blob), X, bias, L.relu)
+        out = torch.full((L.M, L.Nc), float("nan"), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        got = ubp.ubp_spmm_static(blob, X, bias, L.relu, out=out)
+        torch.cuda.synchronize()
+        # same kernel, same plan bytes, same summation order: within the suite's 1e-4 scaled tolerance
+        # (in fact identical)
+        scale = (np.abs(L.W[:, :, 0] * L.mask) @ np.abs(L.X) + np.abs(L.bias)[:, None]).astype(np.float64)
+        err = np.max(np.abs(got.cpu().numpy().astype(np.float64) - want.cpu().numpy()) / scale)
+        assert err <= 1e-4
+        assert torch.equal(got, want)
+    # and the first layer again: the array now holds layer b's plan
+    L = layers[0]
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    X = torch.from_numpy(L.X).cuda(); bias = torch.from_numpy(L.bias).cuda()
+    assert torch.equal(ubp.ubp_spmm_static(blob, X, bias, L.relu), ubp.ubp_spmm(ubp.Plan(blob), X, bias, L.relu))
+
+
+def test_static_entry_rejects_oversized_layer():
+    import torch
+    import paper_2407_19644_b200 as ubp
+    L = ubp_synth.make_layer("big", 2048, 2048, 4, 50, 503, Nc=4, make_x=False)
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    assert ubp.plan_size(blob) > ubp.static_plan_capacity()
+    X = torch.zeros((2048, 4), device="cuda")
+    with pytest.raises(ubp.UbpError) as e:
+        ubp.ubp_spmm_static(blob, X)
+    assert e.value.code == -8 and "fixed device scratch" in str(e.value)
