@@ -95,7 +95,10 @@ int ubp_blob_view(const void *blob, size_t len, ubp_view_t *view);
 typedef struct ubp_plan ubp_plan_t;
 
 int ubp_variant_count(void);
-/* text description of variant id (1-based) into buf; UBP_E_ARG if out of range */
+/* id of the index-th configuration (0 <= index < ubp_variant_count()), or UBP_E_ARG; ids are positive
+ * but not contiguous */
+int ubp_variant_at(int index);
+/* text description of the configuration with this id into buf; UBP_E_ARG if there is none */
 int ubp_variant_describe(int variant, char *buf, size_t cap);
 
 /* bytes of device memory a plan of this blob needs (host; no CUDA call) */

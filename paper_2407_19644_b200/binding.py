@@ -50,6 +50,8 @@ def load():
     L.ubp_unpack.argtypes = [vp, sz, vp, vp]
     L.ubp_blob_view.argtypes = [vp, sz, C.POINTER(_View)]
     L.ubp_variant_count.restype = i32
+    L.ubp_variant_at.argtypes = [i32]
+    L.ubp_variant_at.restype = i32
     L.ubp_variant_describe.argtypes = [i32, C.c_char_p, sz]
     L.ubp_plan_size.argtypes = [vp, sz, i32, C.POINTER(sz)]
     L.ubp_plan_image.argtypes = [vp, sz, i32, vp, sz, C.POINTER(C.c_int32)]
@@ -131,7 +133,8 @@ def variants():
     L = load()
     out = {}
     buf = C.create_string_buffer(256)
-    for i in range(1, L.ubp_variant_count() + 1):
+    for k in range(L.ubp_variant_count()):
+        i = L.ubp_variant_at(k)
         _chk(L.ubp_variant_describe(i, buf, 256), "ubp_variant_describe")
         out[i] = buf.value.decode()
     return out

@@ -53,6 +53,13 @@ int ubp_blob_view(const void *blob, size_t len, ubp_view_t *view) { return ubp::
 
 int ubp_variant_count(void) { return (int)ubp::kernel_cfgs().size(); }
 
+int ubp_variant_at(int index)
+{
+    const auto &c = ubp::kernel_cfgs();
+    if (index < 0 || index >= (int)c.size()) return UBP_E_ARG;
+    return c[(size_t)index].id;
+}
+
 int ubp_variant_describe(int variant, char *buf, size_t cap)
 {
     const ubp::KernelCfg *c = ubp::find_cfg(variant);

@@ -10,9 +10,9 @@
 // a compile-time constant (registers cannot be indexed at run time; this plays
 // the role the weight rotation plays on the paper's SIMD register file).
 //
-// Staging: one producer warp issues, per stage, a TMA tensor copy of the X tile
+// Staging: per pipeline stage one thread issues a TMA tensor copy of the X tile
 // and a bulk copy of the plan group into shared memory, completing on an
-// mbarrier; consumer warps wait on it, compute, and release the stage through a
+// mbarrier; the warps wait on it, compute, and release the stage through a
 // second mbarrier. All waits are bounded; a wait that runs out sets the plan's
 // status word and the CTA drains and exits.
 #include <cuda.h>
@@ -150,41 +150,55 @@ __device__ __forceinline__ void fma_entry(float2 (&acc)[P][2 * V], const EntryRe
     }
 }
 
-// Pipeline state carried across fragments: `cur` holds entry e, jn = channel of entry e+1.
+// Pipeline state carried across fragments: `cur` holds the next entry to be
+// consumed (already loaded), jn the channel of the entry after it; wp / jp point
+// at the weights / channel index of the entry in `cur`.
 template <int V, int WF>
 struct PipeState {
     EntryRegs<V, WF> cur;
     uint32_t jn;
-    int e;
+    const float *wp;
+    const uint16_t *jp;
 };
 
-template <int NBK, int P, int V, bool DUPW, int XROW_BYTES, int F0, int F1>
+// fragment offsets are held in registers as packed 16-bit pairs
+template <int FOW>
+__device__ __forceinline__ int fo_at(const uint32_t (&fw)[FOW], int f)
+{
+    return (f & 1) ? (int)(fw[f >> 1] >> 16) : (int)(fw[f >> 1] & 0xffffu);
+}
+
+template <int NBK, int P, int V, bool DUPW, int XROW_BYTES, int FOW, int F0, int F1>
 struct FragmentLoop {
     static constexpr int WF = NBK * (DUPW ? 2 : 1);
     __device__ __forceinline__ static void run(float2 (&acc)[P][2 * V], PipeState<V, WF> &ps, const uint8_t *xs_lane,
-                                               const uint16_t *fo, const uint16_t *jl, const float *wv)
+                                               const uint32_t (&fw)[FOW])
     {
         if constexpr (F0 < F1) {
             constexpr int S = F0 - (NBK - 1);
-            const int e1 = fo[F0 + 1];
+            int cnt = fo_at<FOW>(fw, F0 + 1) - fo_at<FOW>(fw, F0);
             EntryRegs<V, WF> nxt;
-            while (ps.e + 2 <= e1) {
-                fetch_entry<V, WF, XROW_BYTES>(nxt, xs_lane, ps.jn, wv, ps.e + 1);
-                const uint32_t j2 = jl[ps.e + 2];
+            while (cnt >= 2) {
+                fetch_entry<V, WF, XROW_BYTES>(nxt, xs_lane, ps.jn, ps.wp, 1);
+                const uint32_t j2 = ps.jp[2];
                 fma_entry<NBK, P, V, S, DUPW>(acc, ps.cur);
-                fetch_entry<V, WF, XROW_BYTES>(ps.cur, xs_lane, j2, wv, ps.e + 2);
-                ps.jn = jl[ps.e + 3];
+                fetch_entry<V, WF, XROW_BYTES>(ps.cur, xs_lane, j2, ps.wp, 2);
+                ps.jn = ps.jp[3];
                 fma_entry<NBK, P, V, S, DUPW>(acc, nxt);
-                ps.e += 2;
+                ps.wp += 2 * WF;
+                ps.jp += 2;
+                cnt -= 2;
             }
-            if (ps.e < e1) {
-                fetch_entry<V, WF, XROW_BYTES>(nxt, xs_lane, ps.jn, wv, ps.e + 1);
-                ps.jn = jl[ps.e + 2];
+            if (cnt) {
+                // odd tail: consume `cur`, then refill it in place (no register copies)
+                const uint32_t j2 = ps.jp[2];
                 fma_entry<NBK, P, V, S, DUPW>(acc, ps.cur);
-                ps.cur = nxt;
-                ps.e += 1;
+                fetch_entry<V, WF, XROW_BYTES>(ps.cur, xs_lane, ps.jn, ps.wp, 1);
+                ps.jn = j2;
+                ps.wp += WF;
+                ps.jp += 1;
             }
-            FragmentLoop<NBK, P, V, DUPW, XROW_BYTES, F0 + 1, F1>::run(acc, ps, xs_lane, fo, jl, wv);
+            FragmentLoop<NBK, P, V, DUPW, XROW_BYTES, FOW, F0 + 1, F1>::run(acc, ps, xs_lane, fw);
         }
     }
 };
@@ -202,14 +216,18 @@ struct SpmmArgs {
     int relu;
 };
 
+// All warps of the CTA compute; thread 0 also feeds the pipeline: before it starts on tile kt it issues the
+// copies for tile kt + D (D = stages - 2) into the stage that every warp released two tiles ago, so that wait
+// almost never blocks. Each stage has a "full" mbarrier (completed by the copies' byte count) and an "empty"
+// one (one arrival per warp).
 template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW>
-__global__ void __launch_bounds__((WR * WC + 1) * 32, 1)
+__global__ void __launch_bounds__(WR * WC * 32, 1)
 ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
 {
     constexpr int CS = WC * 128 * V;               // columns per CTA
     constexpr int XT_BYTES = KT * CS * 4;
     constexpr int F = P + NBK - 1;
-    constexpr int NCW = WR * WC;                   // consumer warps
+    constexpr int NCW = WR * WC;                   // warps
     constexpr int FO_BYTES = ((F + 1) * 2 + 15) & ~15;
     constexpr int WF = NBK * (DUPW ? 2 : 1);
     constexpr int MAX_STAGES = 8;
@@ -223,6 +241,7 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
     const int g = blockIdx.x;                      // row group
     const int strip = blockIdx.y;                  // column strip
     const int S = a.stages;
+    const int D = S > 2 ? S - 2 : 1;               // tiles in flight ahead of the one being computed
     const uint32_t *gtab = reinterpret_cast<const uint32_t *>(a.plan + 256);
 
     if (threadIdx.x == 0) {
@@ -236,37 +255,23 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
     }
     __syncthreads();
 
-    if (warp == NCW) {
-        // ---------------- producer warp
-        if (lane == 0) {
-            int issued = 0;
-            bool ok = true;
-            for (int kt = 0; kt < a.nkt && ok; ++kt) {
-                const int st = kt % S;
-                if (kt >= S) ok = mbar_wait(smem_u32(&bar_empty[st]), ((kt / S) - 1) & 1, &abort_flag);
-                if (!ok) break;
-                const uint32_t o0 = gtab[(size_t)kt * a.NG + g], o1 = gtab[(size_t)kt * a.NG + g + 1];
-                const uint32_t gbytes = (o1 - o0) * 16u;
-                const uint32_t bar = smem_u32(&bar_full[st]);
-                uint8_t *stage = smem + (size_t)st * a.stage_bytes;
-                mbar_expect_tx(bar, (uint32_t)XT_BYTES + gbytes);
-                tma_load_2d(smem_u32(stage), &tmX, strip * CS, kt * KT, bar);
-                bulk_load(smem_u32(stage + XT_BYTES), a.plan + (size_t)o0 * 16u, gbytes, bar);
-                ++issued;
-            }
-            if (!ok) {
-                // drain: give copies already in flight a bounded chance to land before the CTA exits
-                const int first = issued > S ? issued - S : 0;
-                for (int kt = first; kt < issued; ++kt)
-                    for (uint32_t it = 0; it < (1u << 16); ++it)
-                        if (mbar_try_wait(smem_u32(&bar_full[kt % S]), (kt / S) & 1)) break;
-                atomicExch(reinterpret_cast<int *>(const_cast<uint8_t *>(a.plan)), 1);
-            }
-        }
-        return;
-    }
+    int issued = 0;                                // tiles whose copies thread 0 has issued
+    auto issue_tile = [&](int kt) -> bool {        // thread 0 only
+        const int st = kt % S;
+        if (kt >= S && !mbar_wait(smem_u32(&bar_empty[st]), ((kt / S) - 1) & 1, &abort_flag)) return false;
+        const uint32_t o0 = gtab[(size_t)kt * a.NG + g], o1 = gtab[(size_t)kt * a.NG + g + 1];
+        const uint32_t gbytes = (o1 - o0) * 16u;
+        const uint32_t bar = smem_u32(&bar_full[st]);
+        uint8_t *stage = smem + (size_t)st * a.stage_bytes;
+        mbar_expect_tx(bar, (uint32_t)XT_BYTES + gbytes);
+        tma_load_2d(smem_u32(stage), &tmX, strip * CS, kt * KT, bar);
+        bulk_load(smem_u32(stage + XT_BYTES), a.plan + (size_t)o0 * 16u, gbytes, bar);
+        ++issued;
+        return true;
+    };
+    if (threadIdx.x == 0)
+        for (int kt = 0; kt < D && kt < a.nkt; ++kt) issue_tile(kt);
 
-    // ---------------- consumer warps
     const int wr = warp / WC, wc = warp % WC;
     const int panel = g * WR + wr;
     float2 acc[P][2 * V];
@@ -277,34 +282,47 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
 
     bool ok = true;
     for (int kt = 0; kt < a.nkt; ++kt) {
+        if (threadIdx.x == 0 && kt + D < a.nkt) ok = issue_tile(kt + D);
         const int st = kt % S;
-        ok = mbar_wait(smem_u32(&bar_full[st]), (kt / S) & 1, &abort_flag);
+        ok = ok && mbar_wait(smem_u32(&bar_full[st]), (kt / S) & 1, &abort_flag);
         if (!ok) break;
         const uint8_t *stage = smem + (size_t)st * a.stage_bytes;
         const uint8_t *grp = stage + XT_BYTES;
         const uint32_t po = reinterpret_cast<const uint32_t *>(grp)[wr];
         const uint32_t pn = reinterpret_cast<const uint32_t *>(grp)[wr + 1];
         if (pn > po) {                               // panel exists in this group
-            const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
-            const int n = fo[F];
-            const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
-            const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * (n + 4) + 15) & ~15));
+            constexpr int FOW = FO_BYTES / 4;
+            uint32_t fw[FOW];
+#pragma unroll
+            for (int q = 0; q < FOW / 4; ++q) {
+                const uint4 t = *reinterpret_cast<const uint4 *>(grp + po + 16 * q);
+                fw[4 * q] = t.x; fw[4 * q + 1] = t.y; fw[4 * q + 2] = t.z; fw[4 * q + 3] = t.w;
+            }
+            const int n = fo_at<FOW>(fw, F);
             const uint8_t *xs_lane = stage + (wc * 128 * V + lane * 4) * 4;
             // the plan pads jl with 4 zero entries and w with 2 zero entries, so the pipeline may read ahead
             PipeState<V, WF> ps;
-            ps.e = 0;
-            fetch_entry<V, WF, CS * 4>(ps.cur, xs_lane, jl[0], wv, 0);
-            ps.jn = jl[1];
-            FragmentLoop<NBK, P, V, DUPW, CS * 4, 0, F>::run(acc, ps, xs_lane, fo, jl, wv);
+            ps.jp = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
+            ps.wp = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * (n + 4) + 15) & ~15));
+            fetch_entry<V, WF, CS * 4>(ps.cur, xs_lane, ps.jp[0], ps.wp, 0);
+            ps.jn = ps.jp[1];
+            FragmentLoop<NBK, P, V, DUPW, CS * 4, FOW, 0, F>::run(acc, ps, xs_lane, fw);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bar_empty[st]));
     }
-    if (!ok) {                                       // report through the plan's status word, store nothing
+    if (!ok) {
+        // A bounded wait ran out somewhere in this CTA: report through the plan's status word and store
+        // nothing. Thread 0 first gives the copies it has in flight a bounded chance to land.
+        if (threadIdx.x == 0) {
+            const int first = issued > S ? issued - S : 0;
+            for (int kt = first; kt < issued; ++kt)
+                for (uint32_t it = 0; it < (1u << 16); ++it)
+                    if (mbar_try_wait(smem_u32(&bar_full[kt % S]), (kt / S) & 1)) break;
+        }
         if (lane == 0) atomicExch(reinterpret_cast<int *>(const_cast<uint8_t *>(a.plan)), 1);
         return;
     }
-    (void)WF;
 
     // ---------------- epilogue: bias, activation, one 128-bit store per lane and column group
     const int64_t col0 = (int64_t)strip * CS + wc * 128 * V + lane * 4;
@@ -520,7 +538,7 @@ static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t 
     const size_t stage_bytes = (XT + pl->img.max_group_bytes + 127) & ~(size_t)127;
     int stages = (int)(kSmemBudget / stage_bytes);
     if (stages < 2) return UBP_E_UNSUPPORTED;
-    if (stages > 4) stages = 4;
+    if (stages > 5) stages = 5;
     if (stages > pl->img.nkt) stages = pl->img.nkt < 1 ? 1 : pl->img.nkt;
 
     EncodeTiledFn enc = encode_fn();
@@ -551,7 +569,7 @@ static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t 
     a.bias = bias; a.Y = Y; a.ldy = ldy; a.Nc = Nc; a.M = pl->dims.M;
     a.nkt = pl->img.nkt; a.NG = pl->img.NG; a.stages = stages; a.stage_bytes = (uint32_t)stage_bytes; a.relu = relu;
     dim3 grid((unsigned)pl->img.NG, (unsigned)((Nc + CS - 1) / CS));
-    kern<<<grid, (WR * WC + 1) * 32, smem, stream>>>(tm, a);
+    kern<<<grid, WR * WC * 32, smem, stream>>>(tm, a);
     return check(cudaGetLastError());
 }
 
@@ -575,24 +593,19 @@ int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, con
                       (ldx % 4 == 0) && (ldy % 4 == 0) && (int64_t)ldx * 4 < (1ll << 40) &&
                       pl->dims.C < (1 << 30) && Nc < (1ll << 31);
     int rc = UBP_E_UNSUPPORTED;
-#define UBP_MAIN(ID, NBK, P, V, WR, WC, KT, DUP)                                                             \
-    if (fast && c.id == ID) rc = launch_main<NBK, P, V, WR, WC, KT, DUP>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
-    UBP_MAIN(1, 4, 16, 2, 8, 1, 32, false)
-    UBP_MAIN(2, 4, 16, 2, 8, 1, 32, true)
-    UBP_MAIN(3, 4, 16, 1, 8, 2, 32, false)
-    UBP_MAIN(4, 4, 16, 1, 16, 1, 64, false)
-    UBP_MAIN(5, 2, 16, 2, 8, 1, 32, false)
-    UBP_MAIN(6, 8, 16, 2, 8, 1, 32, false)
-    UBP_MAIN(7, 16, 16, 2, 8, 1, 32, false)
-    UBP_MAIN(8, 1, 16, 2, 8, 1, 32, false)
-    UBP_MAIN(9, 8, 8, 2, 16, 1, 32, false)
-#undef UBP_MAIN
+#define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP)                                                     \
+    if constexpr (KIND == 0)                                                                                   \
+        if (fast && c.id == ID)                                                                                \
+            rc = launch_main<NBK, P_, V_, WR_, WC_, KT_, (DUP != 0)>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
+#include "ubp_cfgs.inc"
+#undef UBP_CFG
     if (rc != UBP_E_UNSUPPORTED) return rc;
     // slower kernel: unaligned operands, or a plan group too large to stage
-#define UBP_SIMPLE(NBK_, P_) \
-    if (c.nbk == NBK_ && c.P == P_) return launch_simple<NBK_, P_>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
-    UBP_SIMPLE(1, 16) UBP_SIMPLE(2, 16) UBP_SIMPLE(4, 16) UBP_SIMPLE(8, 16) UBP_SIMPLE(16, 16) UBP_SIMPLE(8, 8)
-#undef UBP_SIMPLE
+#define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP) \
+    if constexpr (KIND == 0)                               \
+        if (c.id == ID) return launch_simple<NBK, P_>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
+#include "ubp_cfgs.inc"
+#undef UBP_CFG
     return UBP_E_UNSUPPORTED;
 }
 
@@ -603,15 +616,16 @@ int launch_conv3x3(const ubp_plan *pl, const float *in, int B, int H, int Wd, in
     const KernelCfg &c = pl->cfg;
     const int64_t total = (int64_t)B * H * Wd;
     dim3 grid((unsigned)((total + 127) / 128), (unsigned)pl->img.NP);
-#define UBP_CONV(NBK_, P_)                                                                                      \
-    if (c.nbk == NBK_ && c.P == P_) {                                                                           \
-        ubp_conv3x3_simple_kernel<NBK_, P_><<<grid, 128, 0, stream>>>(                                          \
-            static_cast<const uint8_t *>(pl->dev), in, B, H, Wd, isb, isc, bias, relu, out, osb, osc, pl->dims.M, \
-            pl->img.NP, pl->img.nkt, pl->img.NG, c.WR, c.KT);                                                   \
-        return check(cudaGetLastError());                                                                       \
-    }
-    UBP_CONV(8, 8) UBP_CONV(4, 8) UBP_CONV(2, 8) UBP_CONV(1, 8)
-#undef UBP_CONV
+#define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP)                                                       \
+    if constexpr (KIND == 1)                                                                                     \
+        if (c.id == ID) {                                                                                        \
+            ubp_conv3x3_simple_kernel<NBK, P_><<<grid, 128, 0, stream>>>(                                        \
+                static_cast<const uint8_t *>(pl->dev), in, B, H, Wd, isb, isc, bias, relu, out, osb, osc,        \
+                pl->dims.M, pl->img.NP, pl->img.nkt, pl->img.NG, c.WR, c.KT);                                    \
+            return check(cudaGetLastError());                                                                    \
+        }
+#include "ubp_cfgs.inc"
+#undef UBP_CFG
     return UBP_E_UNSUPPORTED;
 }
 

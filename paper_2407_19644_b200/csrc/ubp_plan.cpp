@@ -18,21 +18,10 @@ namespace ubp {
 
 const std::vector<KernelCfg> &kernel_cfgs()
 {
-    //                 id kind nbk  P  V WR WC  KT dup
     static const std::vector<KernelCfg> cfgs = {
-        {1, 0, 4, 16, 2, 8, 1, 32, 0},
-        {2, 0, 4, 16, 2, 8, 1, 32, 1},
-        {3, 0, 4, 16, 1, 8, 2, 32, 0},
-        {4, 0, 4, 16, 1, 16, 1, 64, 0},
-        {5, 0, 2, 16, 2, 8, 1, 32, 0},
-        {6, 0, 8, 16, 2, 8, 1, 32, 0},
-        {7, 0, 16, 16, 2, 8, 1, 32, 0},
-        {8, 0, 1, 16, 2, 8, 1, 32, 0},
-        {9, 0, 8, 8, 2, 16, 1, 32, 0},
-        {10, 1, 8, 8, 1, 4, 1, 16, 0},
-        {11, 1, 4, 8, 1, 4, 1, 16, 0},
-        {12, 1, 2, 8, 1, 4, 1, 16, 0},
-        {13, 1, 1, 8, 1, 4, 1, 16, 0},
+#define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP) {ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP},
+#include "ubp_cfgs.inc"
+#undef UBP_CFG
     };
     return cfgs;
 }
@@ -57,19 +46,19 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     const int nbk = largest_pow2_divisor_le16(Nb);
     if (R == 9) {
         switch (nbk) {
-            case 16: case 8: return find_cfg(10);
-            case 4: return find_cfg(11);
-            case 2: return find_cfg(12);
-            default: return find_cfg(13);
+            case 16: case 8: return find_cfg(20);
+            case 4: return find_cfg(21);
+            case 2: return find_cfg(22);
+            default: return find_cfg(23);
         }
     }
     if (R != 1) return nullptr;
+    // measured on B200 (2048 x 2048 x 8192 sweep): 8-row panels, 256 columns per warp, 16 warps, 64-channel tiles
     switch (nbk) {
-        case 16: return find_cfg(7);
-        case 8: return find_cfg(6);
-        case 4: return find_cfg(1);
-        case 2: return find_cfg(5);
-        default: return find_cfg(8);
+        case 16: case 8: return find_cfg(16);     // 16-row blocks run as two 8-row entries
+        case 4: return find_cfg(14);
+        case 2: return find_cfg(15);
+        default: return find_cfg(17);
     }
 }
 

@@ -119,7 +119,7 @@ def test_blob_view_rejects_corruption():
 
 
 @pytest.mark.parametrize("M,C,Nb,p,R,variant", [
-    (64, 64, 4, 50, 1, 0), (100, 70, 4, 60, 1, 1), (100, 70, 4, 60, 1, 2), (100, 70, 4, 60, 1, 4),
+    (64, 64, 4, 50, 1, 0), (100, 70, 4, 60, 1, 1), (100, 70, 4, 60, 1, 3), (100, 70, 4, 60, 1, 4), (100, 70, 4, 60, 1, 5), (100, 70, 4, 60, 1, 7),
     (37, 45, 3, 40, 1, 0), (50, 33, 2, 50, 1, 0), (72, 40, 8, 50, 1, 0), (72, 40, 8, 50, 1, 9),
     (80, 40, 16, 50, 1, 0), (60, 20, 12, 40, 1, 0), (45, 17, 1, 70, 1, 0), (40, 20, 8, 50, 9, 0),
     (24, 18, 4, 50, 9, 0), (30, 10, 6, 40, 9, 0),
@@ -146,9 +146,9 @@ def test_plan_rejects_wrong_kind():
     L = ubp_synth.make_layer("t", 16, 8, 4, 50, 3, Nc=4)
     blob = ubp.ubp_pack(L.W, L.mask, 4)
     with pytest.raises(ubp.UbpError):
-        ubp.plan_size(blob, 10)         # a 3x3 configuration for an R = 1 blob
+        ubp.plan_size(blob, 20)         # a 3x3 configuration for an R = 1 blob
     with pytest.raises(ubp.UbpError):
-        ubp.plan_size(blob, 6)          # 8 rows per entry do not divide a block of 4
+        ubp.plan_size(blob, 8)          # 8 rows per entry do not divide a block of 4
     with pytest.raises(ubp.UbpError):
         ubp.plan_size(blob, 999)
-    assert ubp.plan_size(blob, 5) > 0   # 2 rows per entry: each block becomes two entries
+    assert ubp.plan_size(blob, 7) > 0   # 2 rows per entry: each block becomes two entries

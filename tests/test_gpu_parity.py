@@ -61,7 +61,7 @@ def check(Yh, Yref, A, L):
 SMALL = [
     # M, C, Nb, p, Nc, variant
     (64, 64, 4, 50, 256, 0), (100, 70, 4, 60, 300, 1), (100, 70, 4, 60, 300, 2), (100, 70, 4, 60, 520, 3),
-    (300, 150, 4, 70, 260, 4), (37, 45, 3, 40, 132, 0), (50, 33, 2, 50, 388, 0), (72, 40, 8, 50, 264, 0),
+    (300, 150, 4, 70, 260, 4), (300, 150, 4, 70, 260, 5), (300, 150, 4, 70, 516, 6), (300, 150, 4, 70, 516, 14), (64, 300, 8, 70, 516, 13), (64, 300, 2, 70, 516, 12), (37, 45, 3, 40, 132, 0), (50, 33, 2, 50, 388, 0), (72, 40, 8, 50, 264, 0),
     (200, 40, 8, 50, 264, 9), (80, 40, 16, 50, 260, 0), (60, 20, 12, 40, 128, 0), (45, 17, 1, 70, 256, 0),
     (16, 8, 4, 50, 4, 0), (130, 257, 4, 80, 1028, 0), (64, 64, 4, 0, 256, 0),
 ]
