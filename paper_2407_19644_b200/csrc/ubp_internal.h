@@ -21,7 +21,8 @@ int blob_view(const void *blob, size_t len, ubp_view_t *v);
 // kernel instantiation consumes them.
 struct KernelCfg {
     int id;        // 1-based variant id
-    int kind;      // 0 = 1x1 product (R == 1), 1 = implicit 3x3 (R == 9)
+    int kind;      // 0 = 1x1 product (R == 1), 1 = implicit 3x3 (R == 9), 2 = 1x1 on tensor cores (densified
+                   //     panels, 3 x TF32) with the kind-0 plan of the same geometry embedded as its fallback
     int nbk;       // rows per plan entry; divides the layer's Nb
     int P;         // rows per panel (one warp's output rows)
     int V;         // float4 column groups per lane (a warp covers 128*V columns)
@@ -48,6 +49,9 @@ struct PlanImage {
     int nkt = 0, NP = 0, NG = 0, F = 0;
     int64_t entries = 0;
     uint32_t max_group_bytes = 0;
+    // kind 2 only: byte offset of the dense part (Wh [M][tc_kp] then Wl [M][tc_kp], floats) and its row length
+    size_t tc_off = 0;
+    int tc_kp = 0;
 };
 int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only, PlanImage &img, size_t *bytes);
 
@@ -66,6 +70,8 @@ struct ubp_plan {
 namespace ubp {
 int launch_spmm(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                 float *Y, int64_t ldy, void *stream);
+int launch_spmm_tc(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                   float *Y, int64_t ldy, void *stream);
 int launch_conv3x3(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
                    const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream);
 void set_last_cuda_error(int e);

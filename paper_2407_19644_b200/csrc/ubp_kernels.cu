@@ -593,6 +593,7 @@ int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, con
                       (ldx % 4 == 0) && (ldy % 4 == 0) && (int64_t)ldx * 4 < (1ll << 40) &&
                       pl->dims.C < (1 << 30) && Nc < (1ll << 31);
     int rc = UBP_E_UNSUPPORTED;
+    if (fast && c.kind == 2) return launch_spmm_tc(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
 #define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP)                                                     \
     if constexpr (KIND == 0)                                                                                   \
         if (fast && c.id == ID)                                                                                \
@@ -602,7 +603,7 @@ int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, con
     if (rc != UBP_E_UNSUPPORTED) return rc;
     // slower kernel: unaligned operands, or a plan group too large to stage
 #define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP) \
-    if constexpr (KIND == 0)                               \
+    if constexpr (KIND == 0 || KIND == 2)                  \
         if (c.id == ID) return launch_simple<NBK, P_>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
 #include "ubp_cfgs.inc"
 #undef UBP_CFG

@@ -1,0 +1,439 @@
+// Tensor-core variant of the 1x1 product: the block-row panels are densified
+// (the masked weight as a plain M x K matrix) and the product runs on the
+// tcgen05 tensor cores in TF32 with a three-term split that keeps fp32 accuracy:
+//     W = Wh + Wl,  X = Xh + Xl   (h = top 19 bits, l = remainder)
+//     W X ~= Wh Xh + Wl Xh + Wh Xl          (the dropped Wl Xl term is ~2^-20 |w||x|)
+// all three accumulated in fp32 in tensor memory. It does 3 / density times the
+// multiply-adds of the sparse kernel but on a unit ~15x faster than the FP32
+// pipes, so it wins at low and moderate sparsity; the sparse SIMT kernel wins
+// when few blocks survive. Which one runs is the plan's choice (variant).
+//
+// CTA tile: (128 * MT) output rows x 256 columns; K is walked in chunks of 16.
+// Warp roles: warp 0 issues TMA copies of the Wh / Wl chunks from the plan;
+// warps 2-5 read the X chunk from global memory (one column per thread,
+// coalesced across the warp), split it into Xh and Xl and write both transposed
+// into shared memory (the tensor core wants both operands with the reduction
+// index contiguous); warp 1 issues the MMAs (one thread) and owns tensor memory;
+// then warps 2-5 read the accumulators back (tcgen05.ld), add bias, apply ReLU
+// and store. Operand layouts: W is K-major with the 64-byte swizzle (rows of 16
+// floats, exactly what TMA writes for a 16 x 128 box); X is K-major without
+// swizzle (8-column x 4-channel core matrices of 128 contiguous bytes).
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstring>
+
+#include "ubp_internal.h"
+
+namespace ubp {
+
+namespace {
+
+constexpr int TC_N = 256;          // columns per CTA
+constexpr int TC_KC = 16;          // channels per pipeline stage
+constexpr int TC_SPLIT_WARPS = 8;  // warps 2..9 transpose/split X and run the epilogue
+constexpr int TC_THREADS = (2 + TC_SPLIT_WARPS) * 32;
+constexpr uint32_t A_HALF_BYTES = 128 * TC_KC * 4;          // one 128-row chunk of Wh or Wl: 8 KB
+constexpr uint32_t B_BYTES = TC_KC * TC_N * 4;              // Xh or Xl chunk: 16 KB
+constexpr uint32_t B_LBO = 128;                             // next 4 channels of the same 8 columns
+constexpr uint32_t B_SBO = (TC_KC / 4) * 128;               // next 8 columns: 512 B
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// bounded wait (one second); false if it ran out or another thread of the CTA already gave up
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > 1000000000ull) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+// shared-memory matrix descriptor (tcgen05): start address, leading / stride byte offsets (all >> 4),
+// descriptor version 1, swizzle mode in the top three bits
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle)
+{
+    return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46) | ((uint64_t)swizzle << 61);
+}
+constexpr uint32_t SWZ_NONE = 0, SWZ_64B = 4;
+
+// instruction descriptor: D = f32, A = B = tf32, both K-major, N = 256, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | (0u << 15) | (0u << 16) |
+                            ((uint32_t)(TC_N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(kIdesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+
+struct TcArgs {
+    const float *X;          // [K][ldx]
+    int64_t ldx;
+    const float *bias;
+    float *Y;
+    int64_t ldy;
+    int64_t Nc;
+    int M, K;
+    int relu;
+    int *status;             // plan status word
+};
+
+template <int MT>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ CUtensorMap tmWl, const TcArgs a)
+{
+    constexpr uint32_t A_BYTES = MT * 2 * A_HALF_BYTES;                 // [half][hi, lo]
+    constexpr uint32_t STAGE_BYTES = A_BYTES + 2 * B_BYTES;             // + Xh + Xl
+    constexpr int S = (MT == 2) ? 3 : 4;
+    constexpr uint32_t TMEM_COLS = MT * TC_N;                           // 256 or 512
+
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    // the swizzled operand tiles need 1024-byte aligned bases: round the dynamic window up ourselves
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    __shared__ __align__(8) uint64_t bar_full[S], bar_ready[S], bar_empty[S], bar_acc;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row0 = blockIdx.x * (128 * MT);
+    const int64_t col0 = (int64_t)blockIdx.y * TC_N;
+    const int nchunk = (a.K + TC_KC - 1) / TC_KC;
+#ifdef UBP_TC_DEBUG
+    const long long t_begin = clock64();
+#endif
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_ready[s]), TC_SPLIT_WARPS);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_acc), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {   // tensor memory: the whole warp allocates, the address lands in shared memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+
+    bool ok = true;
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            for (int c = 0; c < nchunk && ok; ++c) {
+                const int st = c % S;
+#ifdef UBP_TC_DEBUG
+                long long t0 = clock64();
+#endif
+                if (c >= S) ok = mbar_wait(smem_u32(&bar_empty[st]), ((c / S) - 1) & 1, &abort_flag);
+#ifdef UBP_TC_DEBUG
+                if (blockIdx.x == 0 && blockIdx.y == 0)
+                    atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 7, (unsigned long long)(clock64() - t0));
+#endif
+                if (!ok) break;
+                uint8_t *stage = smem + (size_t)st * STAGE_BYTES;
+                const uint32_t bar = smem_u32(&bar_full[st]);
+                mbar_expect_tx(bar, A_BYTES);
+#pragma unroll
+                for (int h = 0; h < MT; ++h) {
+                    tma_load_2d(smem_u32(stage + (2 * h) * A_HALF_BYTES), &tmWh, c * TC_KC, row0 + h * 128, bar);
+                    tma_load_2d(smem_u32(stage + (2 * h + 1) * A_HALF_BYTES), &tmWl, c * TC_KC, row0 + h * 128, bar);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (one thread)
+        if (lane == 0) {
+            for (int c = 0; c < nchunk && ok; ++c) {
+                const int st = c % S;
+#ifdef UBP_TC_DEBUG
+                long long t0 = clock64();
+                ok = mbar_wait(smem_u32(&bar_full[st]), (c / S) & 1, &abort_flag);
+                long long t1 = clock64();
+                ok = ok && mbar_wait(smem_u32(&bar_ready[st]), (c / S) & 1, &abort_flag);
+                long long t2 = clock64();
+                if (blockIdx.x == 0 && blockIdx.y == 0) {
+                    atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 2, (unsigned long long)(t1 - t0));
+                    atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 3, (unsigned long long)(t2 - t1));
+                }
+#else
+                ok = mbar_wait(smem_u32(&bar_full[st]), (c / S) & 1, &abort_flag) &&
+                     mbar_wait(smem_u32(&bar_ready[st]), (c / S) & 1, &abort_flag);
+#endif
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sbase = smem_u32(smem + (size_t)st * STAGE_BYTES);
+                const uint32_t xh = sbase + A_BYTES, xl = xh + B_BYTES;
+#pragma unroll
+                for (int h = 0; h < MT; ++h) {
+                    const uint32_t wh = sbase + (2 * h) * A_HALF_BYTES, wl = wh + A_HALF_BYTES;
+                    const uint32_t d = tmem_base + h * TC_N;
+#pragma unroll
+                    for (int ks = 0; ks < TC_KC / 8; ++ks) {
+                        // W: K-major, 64-byte rows, 8-row groups 512 B apart; 8 channels further = +32 B
+                        const uint64_t dWh = make_desc(wh + ks * 32, 16, 512, SWZ_64B);
+                        const uint64_t dWl = make_desc(wl + ks * 32, 16, 512, SWZ_64B);
+                        // X: K-major core matrices (8 columns x 4 channels, 128 B); 8 channels further = +256 B
+                        const uint64_t dXh = make_desc(xh + ks * 256, B_LBO, B_SBO, SWZ_NONE);
+                        const uint64_t dXl = make_desc(xl + ks * 256, B_LBO, B_SBO, SWZ_NONE);
+                        mma_tf32(d, dWh, dXh, (c > 0 || ks > 0) ? 1u : 0u);
+                        mma_tf32(d, dWl, dXh, 1u);
+                        mma_tf32(d, dWh, dXl, 1u);
+                    }
+                }
+                mma_commit(smem_u32(&bar_empty[st]));       // stage may be refilled once these MMAs have read it
+            }
+            if (ok) mma_commit(smem_u32(&bar_acc));          // accumulators complete
+        }
+    } else {
+        // ---------------- warps 2-5: X chunk from global memory -> Xh, Xl transposed into the stage
+        const int t = threadIdx.x - 64;                      // 0..255: this thread owns column col0 + t of the tile
+        constexpr int PD = 3;                                // chunks of X in flight in registers (covers L2 latency)
+        float xr[PD][TC_KC];
+        const bool col_live = col0 + t < a.Nc;
+        const float *xcol = a.X + (col_live ? col0 + t : 0);
+        auto load_chunk = [&](int c, float (&dst)[TC_KC]) {
+            const float *p = xcol + (size_t)c * TC_KC * a.ldx;
+            if (col_live && (c + 1) * TC_KC <= a.K) {
+#pragma unroll
+                for (int k = 0; k < TC_KC; ++k) dst[k] = __ldg(p + (size_t)k * a.ldx);
+            } else {
+#pragma unroll
+                for (int k = 0; k < TC_KC; ++k)
+                    dst[k] = (col_live && c * TC_KC + k < a.K) ? __ldg(p + (size_t)k * a.ldx) : 0.f;
+            }
+        };
+        const uint32_t off = (uint32_t)(t & 7) * 16u + (uint32_t)(t >> 3) * B_SBO;
+        auto split_chunk = [&](int c, const float (&src)[TC_KC]) -> bool {
+            const int st = c % S;
+            if (c >= S && !mbar_wait(smem_u32(&bar_empty[st]), ((c / S) - 1) & 1, &abort_flag)) return false;
+            uint8_t *xh = smem + (size_t)st * STAGE_BYTES + A_BYTES + off;
+            uint8_t *xl = xh + B_BYTES;
+#pragma unroll
+            for (int kc = 0; kc < TC_KC / 4; ++kc) {
+                float4 hi, lo;
+                const float v0 = src[4 * kc], v1 = src[4 * kc + 1], v2 = src[4 * kc + 2], v3 = src[4 * kc + 3];
+                hi.x = __uint_as_float(__float_as_uint(v0) & 0xffffe000u); lo.x = v0 - hi.x;
+                hi.y = __uint_as_float(__float_as_uint(v1) & 0xffffe000u); lo.y = v1 - hi.y;
+                hi.z = __uint_as_float(__float_as_uint(v2) & 0xffffe000u); lo.z = v2 - hi.z;
+                hi.w = __uint_as_float(__float_as_uint(v3) & 0xffffe000u); lo.w = v3 - hi.w;
+                *reinterpret_cast<float4 *>(xh + kc * B_LBO) = hi;
+                *reinterpret_cast<float4 *>(xl + kc * B_LBO) = lo;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the writes visible to the MMA unit
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_ready[st]));
+            return true;
+        };
+#pragma unroll
+        for (int d = 0; d < PD; ++d)
+            if (d < nchunk) load_chunk(d, xr[d]);
+        for (int c0 = 0; c0 < nchunk && ok; c0 += PD) {
+#pragma unroll
+            for (int d = 0; d < PD; ++d) {
+                const int c = c0 + d;
+                if (c < nchunk && ok) {
+                    ok = split_chunk(c, xr[d]);
+                    if (c + PD < nchunk) load_chunk(c + PD, xr[d]);
+                }
+            }
+        }
+        // ---------------- epilogue: accumulators -> registers -> bias, ReLU -> global
+        if (ok) ok = mbar_wait(smem_u32(&bar_acc), 0, &abort_flag);
+        if (ok) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int q = warp & 3;                           // this warp may touch tensor-memory lanes 32q .. 32q+31
+            const int chalf = (warp - 2) >> 2;                // two warps share a lane group and split the columns
+#pragma unroll 1
+            for (int h = 0; h < MT; ++h) {
+                const int row = row0 + h * 128 + q * 32 + lane;
+                const float b = (a.bias && row < a.M) ? __ldg(a.bias + row) : 0.f;
+                float *yrow = a.Y + (size_t)(row < a.M ? row : 0) * a.ldy;
+#pragma unroll 1
+                for (int cc = chalf * (TC_N / 64); cc < (chalf + 1) * (TC_N / 64); ++cc) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * TC_N + cc * 32), r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (row < a.M) {
+                        const int64_t cbase = col0 + cc * 32;
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            float4 o = make_float4(__uint_as_float(r[4 * v]) + b, __uint_as_float(r[4 * v + 1]) + b,
+                                                   __uint_as_float(r[4 * v + 2]) + b, __uint_as_float(r[4 * v + 3]) + b);
+                            if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                            const int64_t col = cbase + 4 * v;
+                            if (col + 3 < a.Nc) {
+                                *reinterpret_cast<float4 *>(yrow + col) = o;
+                            } else {
+                                if (col < a.Nc) yrow[col] = o.x;
+                                if (col + 1 < a.Nc) yrow[col + 1] = o.y;
+                                if (col + 2 < a.Nc) yrow[col + 2] = o.z;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+#ifdef UBP_TC_DEBUG
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 64)
+        atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 8, (unsigned long long)(clock64() - t_begin));
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 32)
+        atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 9, (unsigned long long)(clock64() - t_begin));
+#endif
+    if (!ok && lane == 0) atomicExch(a.status, 1);
+    // every thread comes here; tensor memory is released by the warp that allocated it
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn tc_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+int encode_2d(CUtensorMap *tm, const void *base, uint64_t inner, uint64_t outer, uint64_t row_bytes, uint32_t box_in,
+              uint32_t box_out, CUtensorMapSwizzle swz)
+{
+    EncodeTiledFn enc = tc_encode_fn();
+    if (!enc) return UBP_E_CUDA;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {box_in, box_out};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult cr = enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) { set_last_cuda_error(-(int)cr); return UBP_E_CUDA; }
+    return UBP_OK;
+}
+
+}  // namespace
+
+int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                   float *Y, int64_t ldy, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int M = pl->dims.M, K = pl->dims.C;
+    const uint8_t *dev = static_cast<const uint8_t *>(pl->dev);
+    const float *Wh = reinterpret_cast<const float *>(dev + pl->img.tc_off);
+    const float *Wl = Wh + (size_t)M * pl->img.tc_kp;
+    CUtensorMap tmWh, tmWl;
+    int rc;
+    if ((rc = encode_2d(&tmWh, Wh, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,
+                        CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
+    if ((rc = encode_2d(&tmWl, Wl, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,
+                        CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
+
+    TcArgs a;
+    a.X = X; a.ldx = ldx; a.bias = bias; a.Y = Y; a.ldy = ldy; a.Nc = Nc; a.M = M; a.K = K; a.relu = relu;
+    a.status = reinterpret_cast<int *>(pl->dev);
+    const unsigned ncols = (unsigned)((Nc + TC_N - 1) / TC_N);
+    // two 128-row halves per CTA when that still gives every SM a tile; otherwise one half (more, smaller CTAs)
+    int sms = 148, devid = 0;
+    if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
+    const unsigned tiles2 = (unsigned)((M + 255) / 256) * ncols;
+    const bool use2 = tiles2 >= (unsigned)sms;
+    auto launch = [&](auto kern, int MT, size_t smem) -> int {
+        static bool done[2][64] = {};
+        if (devid < 0 || devid >= 64 || !done[MT - 1][devid]) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+            if (devid >= 0 && devid < 64) done[MT - 1][devid] = true;
+        }
+        dim3 grid((unsigned)((M + 128 * MT - 1) / (128 * MT)), ncols);
+        kern<<<grid, TC_THREADS, smem, stream>>>(tmWh, tmWl, a);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+        return UBP_OK;
+    };
+    if (use2) return launch(ubp_tc_kernel<2>, 2, (size_t)3 * (2 * 2 * A_HALF_BYTES + 2 * B_BYTES) + 1024);
+    return launch(ubp_tc_kernel<1>, 1, (size_t)4 * (1 * 2 * A_HALF_BYTES + 2 * B_BYTES) + 1024);
+}
+
+}  // namespace ubp

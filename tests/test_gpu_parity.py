@@ -50,11 +50,16 @@ def run_spmm(env, L, variant=0, pad=0, misalign=0, relu=None, use_bias=True):
     return Yh, Yref, A, plan
 
 
-def check(Yh, Yref, A, L):
+def check(Yh, Yref, A, L, tensor_core=False):
+    """Gate 1e-4, plus the summation bound of the arithmetic that ran: (L + 2) 2^-24 for the fp32 kernels; the
+    tensor-core variant splits each operand into two TF32 pieces and drops the low x low product and the bits
+    below the low pieces (each <= 2^-20 |w||x|), and its accumulator truncates: 2^-18 + (L + 2) 2^-23."""
     assert np.isfinite(Yh).all()
     err = scaled_error(Yh, Yref, A)
     assert err <= TOL, err
-    assert err <= (terms_per_output(L) + 2) * 2.0 ** -24, err
+    n = terms_per_output(L) + 2
+    bound = 2.0 ** -18 + n * 2.0 ** -23 if tensor_core else n * 2.0 ** -24
+    assert err <= bound, (err, bound)
     return err
 
 
@@ -70,8 +75,45 @@ SMALL = [
 @pytest.mark.parametrize("M,C,Nb,p,Nc,variant", SMALL)
 def test_spmm_small(env, M, C, Nb, p, Nc, variant):
     L = ubp_synth.make_layer("t", M, C, Nb, p, 10 * M + C, Nc=Nc, x_dist="normal", relu=(M % 2 == 0))
-    Yh, Yref, A, _ = run_spmm(env, L, variant)
-    check(Yh, Yref, A, L)
+    Yh, Yref, A, plan = run_spmm(env, L, variant)
+    check(Yh, Yref, A, L, tensor_core=plan.variant >= 30)
+
+
+TC_CASES = [
+    # M, C, Nb, p, Nc, variant  (30..33 = tensor-core variants for 1 / 2 / 4 / 8-row entries)
+    (128, 64, 4, 50, 256, 32), (128, 16, 4, 50, 256, 32), (100, 70, 4, 60, 300, 32), (300, 150, 4, 70, 520, 32),
+    (257, 33, 1, 60, 260, 30), (64, 64, 2, 50, 256, 31), (520, 200, 8, 50, 1028, 33), (260, 40, 16, 50, 516, 33),
+    (130, 257, 4, 80, 1028, 32), (384, 100, 12, 40, 772, 32), (256, 128, 4, 0, 512, 32), (200, 20, 4, 100, 256, 32),
+]
+
+
+@pytest.mark.parametrize("M,C,Nb,p,Nc,variant", TC_CASES)
+def test_spmm_tensor_core_variant(env, M, C, Nb, p, Nc, variant):
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 10 * M + C, Nc=Nc, x_dist="normal", relu=(M % 2 == 0))
+    Yh, Yref, A, plan = run_spmm(env, L, variant)
+    assert plan.variant == variant
+    check(Yh, Yref, A, L, tensor_core=True)
+
+
+def test_tensor_core_variant_ragged_unaligned_and_auto(env):
+    torch, ubp = env
+    # ragged last strip on the fast path, then operands the fast path cannot take (falls back to the embedded
+    # sparse plan: fp32 arithmetic, so the tighter bound holds)
+    L = ubp_synth.make_layer("t", 200, 150, 4, 60, 777, Nc=130, x_dist="normal")
+    check(*run_spmm(env, L, 32, pad=2)[:3], L, tensor_core=True)
+    check(*run_spmm(env, L, 32, pad=0, misalign=1)[:3], L)
+    L2 = ubp_synth.make_layer("t", 200, 150, 4, 60, 778, Nc=131, x_dist="normal")
+    check(*run_spmm(env, L2, 32)[:3], L2)
+    # the automatic choice: dense-enough layers run on tensor cores, very sparse or small ones do not
+    dense = ubp_synth.make_layer("t", 256, 256, 4, 70, 779, Nc=512)
+    sparse = ubp_synth.make_layer("t", 256, 256, 4, 95, 780, Nc=512)
+    small = ubp_synth.make_layer("t", 64, 32, 4, 50, 781, Nc=512)
+    pv = lambda l: ubp.Plan(ubp.ubp_pack(l.W, l.mask, l.Nb)).variant
+    assert pv(dense) == 32 and pv(sparse) == 14 and pv(small) == 14
+    # bitwise reproducible run to run
+    plan = ubp.Plan(ubp.ubp_pack(dense.W, dense.mask, 4))
+    X = torch.from_numpy(dense.X).cuda()
+    assert torch.equal(ubp.ubp_spmm(plan, X).clone(), ubp.ubp_spmm(plan, X))
 
 
 @pytest.mark.parametrize("Nc,pad,misalign", [(130, 2, 0), (131, 1, 0), (1, 3, 0), (3, 1, 0), (257, 3, 0),
@@ -120,7 +162,7 @@ def test_spmm_bad_arguments(env):
 def test_spmm_is_bitwise_reproducible(env):
     torch, ubp = env
     L = ubp_synth.make_layer("t", 256, 256, 4, 70, 99, Nc=1024)
-    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, 4))
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, 4), 14)          # sparse kernel
     X = torch.from_numpy(L.X).cuda(); b = torch.from_numpy(L.bias).cuda()
     Y1 = ubp.ubp_spmm(plan, X, b, True).clone()
     Y2 = ubp.ubp_spmm(plan, X, b, True)
@@ -150,7 +192,12 @@ def test_mbv1_pw512_config_full(env):
     Y = ubp.ubp_conv1x1(plan, X, torch.from_numpy(L.bias).cuda(), True, layout="CNHW")
     plan.check()
     Yref, A = oracle.masked_matmul(L.W, L.mask, L.X.reshape(L.C, -1), L.bias, relu=True)
-    check(Y.cpu().numpy().reshape(L.M, -1), Yref, A, L)
+    check(Y.cpu().numpy().reshape(L.M, -1), Yref, A, L, tensor_core=plan.variant >= 30)
+    # and the sparse kernel on the same layer
+    plan_s = ubp.Plan(blob, 14)
+    Ys = ubp.ubp_conv1x1(plan_s, X, torch.from_numpy(L.bias).cuda(), True, layout="CNHW")
+    plan_s.check()
+    check(Ys.cpu().numpy().reshape(L.M, -1), Yref, A, L)
 
 
 def test_conv1x1_nchw_matches_cnhw(env):
@@ -174,14 +221,16 @@ def test_conv1x1_nchw_matches_cnhw(env):
     check(Y7.cpu().numpy().reshape(L7.M, -1), Yref, A, L7)
 
 
-@pytest.mark.parametrize("nb,sp", [(2, 50), (4, 70), (8, 80), (16, 90)])
-def test_sweep_config_sampled(env, nb, sp):
-    """Full-size sweep point (M = K = 2048, Nc = 8192): sampled outputs against the oracle one by one."""
+@pytest.mark.parametrize("nb,sp,variant", [(2, 50, 0), (4, 70, 0), (8, 80, 0), (16, 90, 0), (4, 70, 14), (2, 50, 15),
+                                           (16, 90, 16)])
+def test_sweep_config_sampled(env, nb, sp, variant):
+    """Full-size sweep point (M = K = 2048, Nc = 8192): sampled outputs against the oracle one by one, for the
+    automatically chosen kernel and for the sparse kernel."""
     torch, ubp = env
     L = ubp_synth.config_layers("sweep", Nb=nb, sparsity_pct=sp)[0]
     blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
     assert blob == oracle.pack(L.W, L.mask, L.Nb)
-    plan = ubp.Plan(blob)
+    plan = ubp.Plan(blob, variant)
     Y = ubp.ubp_spmm(plan, torch.from_numpy(L.X).cuda()).cpu().numpy()
     plan.check()
     rng = np.random.default_rng(nb * 100 + sp)
@@ -189,7 +238,8 @@ def test_sweep_config_sampled(env, nb, sp):
     sn = np.concatenate([rng.integers(0, L.Nc, 4000), [0, 0, L.Nc - 1, L.Nc - 1]])
     ys, as_ = oracle.masked_matmul_samples(L.W, L.mask, L.X, so, sn)
     err = scaled_error(Y[so, sn], ys, as_)
-    assert err <= TOL and err <= (terms_per_output(L) + 2) * 2.0 ** -24
+    n = terms_per_output(L) + 2
+    assert err <= TOL and err <= (2.0 ** -18 + n * 2.0 ** -23 if plan.variant >= 30 else n * 2.0 ** -24)
     # whole rows too (a panel's first / last row and one in the middle)
     for o in (0, 15, 16, 1000, L.M - 1):
         sn2 = np.arange(L.Nc)
