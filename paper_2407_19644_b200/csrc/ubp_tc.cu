@@ -10,11 +10,11 @@
 //
 // CTA tile: (128 * MT) output rows x 256 columns; K is walked in chunks of 16.
 // Warp roles: warp 0 issues TMA copies of the Wh / Wl chunks from the plan;
-// warps 2-5 read the X chunk from global memory (one column per thread,
-// coalesced across the warp), split it into Xh and Xl and write both transposed
+// warps 2-17 read the X chunk from global memory (one column and 8 channels per
+// thread, coalesced across the warp), split it into Xh and Xl and write both transposed
 // into shared memory (the tensor core wants both operands with the reduction
 // index contiguous); warp 1 issues the MMAs (one thread) and owns tensor memory;
-// then warps 2-5 read the accumulators back (tcgen05.ld), add bias, apply ReLU
+// then warps 2-17 read the accumulators back (tcgen05.ld), add bias, apply ReLU
 // and store. Operand layouts: W is K-major with the 64-byte swizzle (rows of 16
 // floats, exactly what TMA writes for a 16 x 128 box); X is K-major without
 // swizzle (8-column x 4-channel core matrices of 128 contiguous bytes).
@@ -32,7 +32,7 @@ namespace {
 
 constexpr int TC_N = 256;          // columns per CTA
 constexpr int TC_KC = 16;          // channels per pipeline stage
-constexpr int TC_SPLIT_WARPS = 8;  // warps 2..9 transpose/split X and run the epilogue
+constexpr int TC_SPLIT_WARPS = 16; // warps 2..17 transpose/split X and run the epilogue
 constexpr int TC_THREADS = (2 + TC_SPLIT_WARPS) * 32;
 constexpr uint32_t A_HALF_BYTES = 128 * TC_KC * 4;          // one 128-row chunk of Wh or Wl: 8 KB
 constexpr uint32_t B_BYTES = TC_KC * TC_N * 4;              // Xh or Xl chunk: 16 KB
@@ -83,6 +83,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     return false;
 }
+// same, for waiters that are not on the critical path: sleep between polls so they do not take issue slots
+// from the thread that feeds the tensor core
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        __nanosleep(40);
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > 1000000000ull) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar)
 {
     asm volatile(
@@ -99,11 +116,15 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 }
 constexpr uint32_t SWZ_NONE = 0, SWZ_64B = 4;
 
-// instruction descriptor: D = f32, A = B = tf32, both K-major, N = 256, M = 128
-constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | (0u << 15) | (0u << 16) |
-                            ((uint32_t)(TC_N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+// instruction descriptor: D = f32, A = B = tf32, both K-major, M = 128, N given at run time (multiple of 16)
+__device__ __forceinline__ uint32_t make_idesc(int n)
+{
+    return (1u << 4) | (2u << 7) | (2u << 10) | (0u << 15) | (0u << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(128 >> 4) << 24);
+}
 
-__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
+__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t kIdesc,
+                                         uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -137,6 +158,7 @@ struct TcArgs {
     int64_t ldy;
     int64_t Nc;
     int M, K;
+    int ntile;               // columns per CTA: multiple of 32, <= 256
     int relu;
     int *status;             // plan status word
 };
@@ -159,12 +181,8 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row0 = blockIdx.x * (128 * MT);
-    const int64_t col0 = (int64_t)blockIdx.y * TC_N;
+    const int64_t col0 = (int64_t)blockIdx.y * a.ntile;
     const int nchunk = (a.K + TC_KC - 1) / TC_KC;
-#ifdef UBP_TC_DEBUG
-    const long long t_begin = clock64();
-#endif
-
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < S; ++s) {
@@ -188,18 +206,11 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
 
     bool ok = true;
     if (warp == 0) {
-        // ---------------- TMA producer
+        // ---------------- TMA producer: Wh / Wl chunks of this row tile
         if (lane == 0) {
             for (int c = 0; c < nchunk && ok; ++c) {
                 const int st = c % S;
-#ifdef UBP_TC_DEBUG
-                long long t0 = clock64();
-#endif
-                if (c >= S) ok = mbar_wait(smem_u32(&bar_empty[st]), ((c / S) - 1) & 1, &abort_flag);
-#ifdef UBP_TC_DEBUG
-                if (blockIdx.x == 0 && blockIdx.y == 0)
-                    atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 7, (unsigned long long)(clock64() - t0));
-#endif
+                if (c >= S) ok = mbar_wait_relaxed(smem_u32(&bar_empty[st]), ((c / S) - 1) & 1, &abort_flag);
                 if (!ok) break;
                 uint8_t *stage = smem + (size_t)st * STAGE_BYTES;
                 const uint32_t bar = smem_u32(&bar_full[st]);
@@ -214,41 +225,33 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
     } else if (warp == 1) {
         // ---------------- MMA issuer (one thread)
         if (lane == 0) {
+            const uint32_t kIdesc = make_idesc(a.ntile);
+            // W: K-major, 64-byte rows, 8-row groups 512 B apart (64-byte swizzle);
+            // X: K-major core matrices of 8 columns x 4 channels (128 B), next 4 channels +128 B, next 8 columns +512 B
+            const uint64_t dWh0 = make_desc(smem_u32(smem), 16, 512, SWZ_64B);
+            const uint64_t dXh0 = make_desc(smem_u32(smem) + A_BYTES, B_LBO, B_SBO, SWZ_NONE);
             for (int c = 0; c < nchunk && ok; ++c) {
                 const int st = c % S;
-#ifdef UBP_TC_DEBUG
-                long long t0 = clock64();
-                ok = mbar_wait(smem_u32(&bar_full[st]), (c / S) & 1, &abort_flag);
-                long long t1 = clock64();
-                ok = ok && mbar_wait(smem_u32(&bar_ready[st]), (c / S) & 1, &abort_flag);
-                long long t2 = clock64();
-                if (blockIdx.x == 0 && blockIdx.y == 0) {
-                    atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 2, (unsigned long long)(t1 - t0));
-                    atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 3, (unsigned long long)(t2 - t1));
-                }
-#else
                 ok = mbar_wait(smem_u32(&bar_full[st]), (c / S) & 1, &abort_flag) &&
                      mbar_wait(smem_u32(&bar_ready[st]), (c / S) & 1, &abort_flag);
-#endif
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t sbase = smem_u32(smem + (size_t)st * STAGE_BYTES);
-                const uint32_t xh = sbase + A_BYTES, xl = xh + B_BYTES;
+                // descriptors of this stage = descriptors of stage 0 + the stage offset in the address field
+                // (16-byte units; shared-memory addresses stay below 2^18, so the 14-bit field never carries)
+                const uint64_t soff = (uint64_t)((uint32_t)st * (STAGE_BYTES >> 4));
 #pragma unroll
                 for (int h = 0; h < MT; ++h) {
-                    const uint32_t wh = sbase + (2 * h) * A_HALF_BYTES, wl = wh + A_HALF_BYTES;
                     const uint32_t d = tmem_base + h * TC_N;
 #pragma unroll
                     for (int ks = 0; ks < TC_KC / 8; ++ks) {
-                        // W: K-major, 64-byte rows, 8-row groups 512 B apart; 8 channels further = +32 B
-                        const uint64_t dWh = make_desc(wh + ks * 32, 16, 512, SWZ_64B);
-                        const uint64_t dWl = make_desc(wl + ks * 32, 16, 512, SWZ_64B);
-                        // X: K-major core matrices (8 columns x 4 channels, 128 B); 8 channels further = +256 B
-                        const uint64_t dXh = make_desc(xh + ks * 256, B_LBO, B_SBO, SWZ_NONE);
-                        const uint64_t dXl = make_desc(xl + ks * 256, B_LBO, B_SBO, SWZ_NONE);
-                        mma_tf32(d, dWh, dXh, (c > 0 || ks > 0) ? 1u : 0u);
-                        mma_tf32(d, dWl, dXh, 1u);
-                        mma_tf32(d, dWh, dXl, 1u);
+                        // W: 8 channels further = +32 B (2 units); X: 8 channels further = +256 B (16 units)
+                        const uint64_t dWh = dWh0 + soff + (uint64_t)(h * (2 * A_HALF_BYTES >> 4) + ks * 2);
+                        const uint64_t dWl = dWh + (A_HALF_BYTES >> 4);
+                        const uint64_t dXh = dXh0 + soff + (uint64_t)(ks * 16);
+                        const uint64_t dXl = dXh + (B_BYTES >> 4);
+                        mma_tf32(d, dWh, dXh, kIdesc, (c > 0 || ks > 0) ? 1u : 0u);
+                        mma_tf32(d, dWl, dXh, kIdesc, 1u);
+                        mma_tf32(d, dWh, dXl, kIdesc, 1u);
                     }
                 }
                 mma_commit(smem_u32(&bar_empty[st]));       // stage may be refilled once these MMAs have read it
@@ -256,31 +259,33 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
             if (ok) mma_commit(smem_u32(&bar_acc));          // accumulators complete
         }
     } else {
-        // ---------------- warps 2-5: X chunk from global memory -> Xh, Xl transposed into the stage
-        const int t = threadIdx.x - 64;                      // 0..255: this thread owns column col0 + t of the tile
+        // ---------------- warps 2-17: X chunk from global memory -> Xh, Xl transposed into the stage
+        const int t = (threadIdx.x - 64) & 255;              // column col0 + t of the tile
+        const int kh = (threadIdx.x - 64) >> 8;              // which 8 of the chunk's 16 channels
+        constexpr int KH = TC_KC / 2;
         constexpr int PD = 3;                                // chunks of X in flight in registers (covers L2 latency)
-        float xr[PD][TC_KC];
-        const bool col_live = col0 + t < a.Nc;
-        const float *xcol = a.X + (col_live ? col0 + t : 0);
-        auto load_chunk = [&](int c, float (&dst)[TC_KC]) {
+        float xr[PD][KH];
+        const bool col_live = t < a.ntile && col0 + t < a.Nc;
+        const float *xcol = a.X + (col_live ? col0 + t : 0) + (size_t)kh * KH * a.ldx;
+        auto load_chunk = [&](int c, float (&dst)[KH]) {
             const float *p = xcol + (size_t)c * TC_KC * a.ldx;
             if (col_live && (c + 1) * TC_KC <= a.K) {
 #pragma unroll
-                for (int k = 0; k < TC_KC; ++k) dst[k] = __ldg(p + (size_t)k * a.ldx);
+                for (int k = 0; k < KH; ++k) dst[k] = __ldg(p + (size_t)k * a.ldx);
             } else {
 #pragma unroll
-                for (int k = 0; k < TC_KC; ++k)
-                    dst[k] = (col_live && c * TC_KC + k < a.K) ? __ldg(p + (size_t)k * a.ldx) : 0.f;
+                for (int k = 0; k < KH; ++k)
+                    dst[k] = (col_live && c * TC_KC + kh * KH + k < a.K) ? __ldg(p + (size_t)k * a.ldx) : 0.f;
             }
         };
-        const uint32_t off = (uint32_t)(t & 7) * 16u + (uint32_t)(t >> 3) * B_SBO;
-        auto split_chunk = [&](int c, const float (&src)[TC_KC]) -> bool {
+        const uint32_t off = (uint32_t)(t & 7) * 16u + (uint32_t)(t >> 3) * B_SBO + (uint32_t)kh * (KH / 4) * B_LBO;
+        auto split_chunk = [&](int c, const float (&src)[KH]) -> bool {
             const int st = c % S;
-            if (c >= S && !mbar_wait(smem_u32(&bar_empty[st]), ((c / S) - 1) & 1, &abort_flag)) return false;
+            if (c >= S && !mbar_wait_relaxed(smem_u32(&bar_empty[st]), ((c / S) - 1) & 1, &abort_flag)) return false;
             uint8_t *xh = smem + (size_t)st * STAGE_BYTES + A_BYTES + off;
             uint8_t *xl = xh + B_BYTES;
 #pragma unroll
-            for (int kc = 0; kc < TC_KC / 4; ++kc) {
+            for (int kc = 0; kc < KH / 4; ++kc) {
                 float4 hi, lo;
                 const float v0 = src[4 * kc], v1 = src[4 * kc + 1], v2 = src[4 * kc + 2], v3 = src[4 * kc + 3];
                 hi.x = __uint_as_float(__float_as_uint(v0) & 0xffffe000u); lo.x = v0 - hi.x;
@@ -309,29 +314,42 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
             }
         }
         // ---------------- epilogue: accumulators -> registers -> bias, ReLU -> global
-        if (ok) ok = mbar_wait(smem_u32(&bar_acc), 0, &abort_flag);
+        if (ok) ok = mbar_wait_relaxed(smem_u32(&bar_acc), 0, &abort_flag);
         if (ok) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int q = warp & 3;                           // this warp may touch tensor-memory lanes 32q .. 32q+31
-            const int chalf = (warp - 2) >> 2;                // two warps share a lane group and split the columns
+            const int cpart = (warp - 2) >> 2;                // four warps share a lane group and split the columns
+            // Each 32 x 32 block goes registers -> shared memory (row per lane, 144-byte pitch) -> registers with
+            // 8 lanes per row, so that every store instruction writes four complete 128-byte row segments.
+            // The pipeline stages are idle by now (all MMAs have completed), so their memory is reused.
+            constexpr int PITCH = 36;                         // floats
+            float *tile = reinterpret_cast<float *>(smem) + (warp - 2) * 32 * PITCH;
+            const int sub_row = lane >> 3, sub_col = (lane & 7) * 4;
 #pragma unroll 1
             for (int h = 0; h < MT; ++h) {
-                const int row = row0 + h * 128 + q * 32 + lane;
-                const float b = (a.bias && row < a.M) ? __ldg(a.bias + row) : 0.f;
-                float *yrow = a.Y + (size_t)(row < a.M ? row : 0) * a.ldy;
+                const int rbase = row0 + h * 128 + q * 32;
 #pragma unroll 1
-                for (int cc = chalf * (TC_N / 64); cc < (chalf + 1) * (TC_N / 64); ++cc) {
+                for (int cc = cpart; cc < a.ntile / 32; cc += TC_SPLIT_WARPS / 4) {
                     uint32_t r[32];
                     tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * TC_N + cc * 32), r);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (row < a.M) {
-                        const int64_t cbase = col0 + cc * 32;
 #pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            float4 o = make_float4(__uint_as_float(r[4 * v]) + b, __uint_as_float(r[4 * v + 1]) + b,
-                                                   __uint_as_float(r[4 * v + 2]) + b, __uint_as_float(r[4 * v + 3]) + b);
+                    for (int v = 0; v < 8; ++v)
+                        *reinterpret_cast<float4 *>(tile + lane * PITCH + 4 * v) =
+                            make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                        __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                    __syncwarp();
+                    const int64_t col = col0 + cc * 32 + sub_col;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int rr = i * 4 + sub_row;
+                        const int row = rbase + rr;
+                        float4 o = *reinterpret_cast<const float4 *>(tile + rr * PITCH + sub_col);
+                        if (row < a.M) {
+                            const float b = a.bias ? __ldg(a.bias + row) : 0.f;
+                            o.x += b; o.y += b; o.z += b; o.w += b;
                             if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
-                            const int64_t col = cbase + 4 * v;
+                            float *yrow = a.Y + (size_t)row * a.ldy;
                             if (col + 3 < a.Nc) {
                                 *reinterpret_cast<float4 *>(yrow + col) = o;
                             } else {
@@ -341,16 +359,11 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
                             }
                         }
                     }
+                    __syncwarp();
                 }
             }
         }
     }
-#ifdef UBP_TC_DEBUG
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 64)
-        atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 8, (unsigned long long)(clock64() - t_begin));
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 32)
-        atomicAdd(reinterpret_cast<unsigned long long *>(a.status) + 9, (unsigned long long)(clock64() - t_begin));
-#endif
     if (!ok && lane == 0) atomicExch(a.status, 1);
     // every thread comes here; tensor memory is released by the warp that allocated it
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -413,12 +426,28 @@ int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, 
     TcArgs a;
     a.X = X; a.ldx = ldx; a.bias = bias; a.Y = Y; a.ldy = ldy; a.Nc = Nc; a.M = M; a.K = K; a.relu = relu;
     a.status = reinterpret_cast<int *>(pl->dev);
-    const unsigned ncols = (unsigned)((Nc + TC_N - 1) / TC_N);
-    // two 128-row halves per CTA when that still gives every SM a tile; otherwise one half (more, smaller CTAs)
+    // Tile choice: 128 or 256 rows, 64..256 columns (multiples of 32). Estimate the time of each candidate as
+    // (waves over the SMs) x (chunks x MMA cycles per chunk + a fixed per-tile cost) and keep the cheapest.
     int sms = 148, devid = 0;
     if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
-    const unsigned tiles2 = (unsigned)((M + 255) / 256) * ncols;
-    const bool use2 = tiles2 >= (unsigned)sms;
+    const int nchunk = (K + TC_KC - 1) / TC_KC;
+    double best = 1e300;
+    int best_mt = 1, best_n = TC_N;
+    for (int mt = 1; mt <= 2; ++mt)
+        for (int n = 64; n <= TC_N; n += 32) {
+            const long long tiles = (long long)((M + 128 * mt - 1) / (128 * mt)) * ((Nc + n - 1) / n);
+            const long long waves = (tiles + sms - 1) / sms;
+            // 6 MMAs per 8 channels and 128-row half, n/2 cycles each; narrow tiles re-read W more often, which
+            // shows as a floor on the cycles per chunk; ~6000 cycles of prologue + epilogue per tile
+            double per_chunk = mt * 6.0 * (TC_KC / 8) * (n / 2.0);
+            const double floor_chunk = mt == 2 ? 1400.0 : 750.0;
+            if (per_chunk < floor_chunk) per_chunk = floor_chunk;
+            const double t = (double)waves * (nchunk * per_chunk + 6000.0 + 40.0 * mt * n);
+            if (t < best) { best = t; best_mt = mt; best_n = n; }
+        }
+    a.ntile = best_n;
+    const bool use2 = best_mt == 2;
+    const unsigned ncols = (unsigned)((Nc + best_n - 1) / best_n);
     auto launch = [&](auto kern, int MT, size_t smem) -> int {
         static bool done[2][64] = {};
         if (devid < 0 || devid >= 64 || !done[MT - 1][devid]) {
