@@ -63,6 +63,24 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def tf32_peak_tflops():
+    """Dense TF32 peak = measured bf16 peak x the nominal tf32/bf16 ratio (1/2)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["bf16_tflops"]) / 2, "measured bf16 burst x 0.5"
+    return 1590.0 / 2, "fallback bf16 x 0.5"
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (key: workload, tensor-core variant?)
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    ("mbv1_pw512", True): 14982400 + 768,      # profiles/ncu_full_ubp_tc_kernel_mbv1_pw512.md (output still in L2)
+    ("mbv1_pw512", False): 13414656,           # profiles/ncu_full_ubp_spmm_kernel.md
+    ("sweep_nb4_p70", False): 76188928 + 33089024,
+}
+
+
 def compulsory_bytes(L) -> int:
     """Activations read once + outputs written once + packed weights/indices + bias."""
     x = L.X.size * 4
@@ -315,10 +333,14 @@ def main():
                 "traffic": None, "peak_source": f"{peak_src} copy bandwidth"}
     roof["roofline_us"] = max(t_alu, t_hbm) * 1e6
     roof["frac_of_roofline_time"] = max(t_alu, t_hbm) / (step_ms * 1e-3)
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(prof):
-        with open(prof) as f:
-            roof["traffic"] = json.load(f).get(name)
+    roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((name, plan.variant >= 30))
+    roof["kernel"] = "ubp_tc_kernel (dense 3xTF32 on tcgen05)" if plan.variant >= 30 else "ubp_spmm_kernel (sparse, FP32 FMA)"
+    if plan.variant >= 30 and L.R == 1:
+        # the tensor-core variant does 3 x the DENSE multiply-adds; report that rate against the TF32 peak too
+        dense_tf = 3 * 2.0 * L.M * L.C * L.Nc / (step_ms * 1e-3) / 1e12
+        tf32_peak = tf32_peak_tflops()
+        roof["tensor"] = {"dense_tf32_tflops": dense_tf, "peak": tf32_peak[0], "peak_source": tf32_peak[1],
+                          "frac": dense_tf / tf32_peak[0]}
 
     line = {
         "metric": "effective GFLOP/s (2 x surviving MACs / time) of one UBP layer", "value": gflops, "unit": "GFLOP/s",

@@ -61,8 +61,18 @@ int ubp_spmm_static(const void *blob, size_t len, const float *X, int64_t ldx, i
         tmp.dims = v;
         tmp.cfg = *cfg;
         size_t need = 0;
-        if ((rc = ubp::build_plan_image(v, *cfg, false, tmp.img, &need))) return rc;
+        if ((rc = ubp::build_plan_image(v, *cfg, true, tmp.img, &need))) return rc;
+        if (need > UBP_STATIC_PLAN_BYTES && cfg->kind == 2) {
+            // the tensor-core plan carries a dense copy of the weight; the sparse plan of the same geometry is
+            // much smaller, so try that before giving up
+            for (const auto &c : ubp::kernel_cfgs())
+                if (c.kind == 0 && c.nbk == cfg->nbk && c.P == cfg->P && c.KT == cfg->KT && c.WR == cfg->WR &&
+                    c.V == cfg->V && c.WC == cfg->WC && c.dupw == cfg->dupw) { cfg = &c; break; }
+            tmp.cfg = *cfg;
+            if ((rc = ubp::build_plan_image(v, *cfg, true, tmp.img, &need))) return rc;
+        }
         if (need > UBP_STATIC_PLAN_BYTES) return UBP_E_STATIC_LIMIT;
+        if ((rc = ubp::build_plan_image(v, *cfg, false, tmp.img, &need))) return rc;
         void *dev = nullptr;
         if ((rc = static_plan_ptr(&dev))) return rc;
         tmp.dev = dev;

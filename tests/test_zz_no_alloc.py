@@ -37,6 +37,20 @@ def test_static_entry_matches_planned_entry_twice():
     assert torch.equal(ubp.ubp_spmm_static(blob, X, bias, L.relu), ubp.ubp_spmm(ubp.Plan(blob), X, bias, L.relu))
 
 
+def test_static_entry_falls_back_to_the_smaller_plan():
+    """512x512 at 70 %: the tensor-core plan (with its dense weight copy) exceeds the 2 MiB array, the sparse plan
+    fits, so the call succeeds on the sparse kernel."""
+    import torch
+    import paper_2407_19644_b200 as ubp
+    L = ubp_synth.make_layer("mid", 512, 512, 4, 70, 504, Nc=520, x_dist="normal")
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    assert ubp.plan_size(blob) > ubp.static_plan_capacity() > ubp.plan_size(blob, 14)
+    X = torch.from_numpy(L.X).cuda(); bias = torch.from_numpy(L.bias).cuda()
+    got = ubp.ubp_spmm_static(blob, X, bias, True)
+    want = ubp.ubp_spmm(ubp.Plan(blob, 14), X, bias, True)
+    assert torch.equal(got, want)
+
+
 def test_static_entry_rejects_oversized_layer():
     import torch
     import paper_2407_19644_b200 as ubp
