@@ -234,6 +234,20 @@ def cpu_oracle_time(L, budget_s=20.0):
     return flops / t / 1e9, oracle.num_threads(), sample, t
 
 
+def max_over_ranks(ms: float, dist, torch, device) -> float:
+    """A step is as slow as its slowest rank: MAX-reduce the per-rank device time (no-op without a group)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_gflops(flops_per_rank: float, world: int, step_ms: float) -> float:
+    """Whole-job throughput: every rank does the same amount of work on its own columns (weak scaling)."""
+    return world * flops_per_rank / (step_ms * 1e-3) / 1e9
+
+
 def run_reference(args, L, name):
     """--impl reference: the CPU oracle timed on this machine's host cores (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -269,6 +283,8 @@ def main():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     ap.add_argument("--no-flush", action="store_true", help="do not flush L2 between steps (warm-L2 figure)")
+    ap.add_argument("--profile", type=int, default=0, metavar="N",
+                    help="build the plan, launch the layer N times and exit (a small target for ncu captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -295,6 +311,13 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     plan, run, pack_ms, plan_ms, X, Y, bias = build_runner(ubp, torch, L, args.variant)
+    if args.profile > 0:
+        for _ in range(args.profile):
+            run()
+        torch.cuda.synchronize()
+        plan.check()
+        print(json.dumps({"profile_launches": args.profile, "workload": name, "variant": plan.variant}), flush=True)
+        return
     flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
 
     sampler = ClockSampler(local_rank)
@@ -306,19 +329,12 @@ def main():
     torch.cuda.synchronize()
     clocks = sampler.stop()
     plan.check()
-    step_ms = float(np.mean(times))
-    if dist is not None:
-        t = torch.tensor([step_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_ms = float(t.item())
+    step_ms = max_over_ranks(float(np.mean(times)), dist, torch, "cuda")
     e2e_ms, h2d, d2h = time_e2e(torch, ubp, plan, L, max(5, min(args.steps, 30)), 3)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, torch, "cuda")
 
     flops = 2.0 * L.surviving_macs
-    gflops = world * flops / (step_ms * 1e-3) / 1e9
+    gflops = aggregate_gflops(flops, world, step_ms)
     hbm_gbs, peak_src = measured_peaks()
     t_alu = flops / (FP32_PEAK_TFLOPS * 1e12)
     t_hbm = compulsory_bytes(L) / (hbm_gbs * 1e9)
