@@ -65,7 +65,7 @@ int ubp_variant_describe(int variant, char *buf, size_t cap)
     const ubp::KernelCfg *c = ubp::find_cfg(variant);
     if (!c || !buf || cap == 0) return UBP_E_ARG;
     std::snprintf(buf, cap, "%s nbk=%d panel=%d cols/warp=%d warps=%dx%d ktile=%d%s",
-                  c->kind == 0 ? "spmm" : (c->kind == 1 ? "conv3x3" : "spmm-tensorcore(3xTF32) fallback"), c->nbk, c->P, 128 * c->V, c->WR, c->WC, c->KT,
+                  c->kind == 0 ? "spmm" : (c->kind == 1 ? "conv3x3" : (c->kind == 2 ? "spmm-tensorcore(3xTF32) fallback" : "conv3x3-tensorcore(3xTF32) fallback")), c->nbk, c->P, 128 * c->V, c->WR, c->WC, c->KT,
                   c->dupw ? " dupw" : "");
     return UBP_OK;
 }
@@ -169,7 +169,7 @@ int ubp_spmm(const ubp_plan_t *plan, const float *X, int64_t ldx, int64_t Nc,
              const float *bias, int relu, float *Y, int64_t ldy, void *stream)
 {
     if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
-    if (plan->dims.R != 1 || plan->cfg.kind == 1) return UBP_E_ARG;
+    if (plan->dims.R != 1 || plan->cfg.kind == 1 || plan->cfg.kind == 3) return UBP_E_ARG;
     if (Nc < 0) return UBP_E_ARG;
     if (Nc == 0) return UBP_OK;
     if (!X || !Y || ldx < Nc || ldy < Nc) return UBP_E_ARG;
@@ -181,7 +181,7 @@ int ubp_conv1x1(const ubp_plan_t *plan, const float *in, int B, int H, int Wd,
                 float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream)
 {
     if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
-    if (plan->dims.R != 1 || plan->cfg.kind == 1) return UBP_E_ARG;
+    if (plan->dims.R != 1 || plan->cfg.kind == 1 || plan->cfg.kind == 3) return UBP_E_ARG;
     if (B < 0 || H <= 0 || Wd <= 0) return UBP_E_ARG;
     if (B == 0) return UBP_OK;
     if (!in || !out) return UBP_E_ARG;
@@ -204,7 +204,7 @@ int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, 
                          float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream)
 {
     if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
-    if (plan->dims.R != 9 || plan->cfg.kind != 1) return UBP_E_ARG;
+    if (plan->dims.R != 9 || (plan->cfg.kind != 1 && plan->cfg.kind != 3)) return UBP_E_ARG;
     if (B < 0 || H <= 0 || Wd <= 0) return UBP_E_ARG;
     if (B == 0) return UBP_OK;
     if (!in || !out) return UBP_E_ARG;

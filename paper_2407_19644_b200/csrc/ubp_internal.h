@@ -22,7 +22,8 @@ int blob_view(const void *blob, size_t len, ubp_view_t *v);
 struct KernelCfg {
     int id;        // 1-based variant id
     int kind;      // 0 = 1x1 product (R == 1), 1 = implicit 3x3 (R == 9), 2 = 1x1 on tensor cores (densified
-                   //     panels, 3 x TF32) with the kind-0 plan of the same geometry embedded as its fallback
+                   //     panels, 3 x TF32) with the kind-0 plan of the same geometry embedded as its fallback,
+                   // 3 = 3x3 as an implicit GEMM on tensor cores with the kind-1 plan embedded
     int nbk;       // rows per plan entry; divides the layer's Nb
     int P;         // rows per panel (one warp's output rows)
     int V;         // float4 column groups per lane (a warp covers 128*V columns)
@@ -72,6 +73,8 @@ int launch_spmm(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, c
                 float *Y, int64_t ldy, void *stream);
 int launch_spmm_tc(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                    float *Y, int64_t ldy, void *stream);
+int launch_conv3x3_tc(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
+                      const float *bias, int relu, float *out, int64_t out_ld, void *stream);
 int launch_conv3x3(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
                    const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream);
 void set_last_cuda_error(int e);

@@ -616,9 +616,13 @@ int launch_conv3x3(const ubp_plan *pl, const float *in, int B, int H, int Wd, in
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const KernelCfg &c = pl->cfg;
     const int64_t total = (int64_t)B * H * Wd;
+    // tensor-core path: needs the output as one [M][B*H*W] matrix (batch stride = plane size) with 16-byte rows
+    if (c.kind == 3 && osb == (int64_t)H * Wd && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && osc % 4 == 0 &&
+        osc >= total && total < (1ll << 31))
+        return launch_conv3x3_tc(pl, in, B, H, Wd, isb, isc, bias, relu, out, osc, stream_);
     dim3 grid((unsigned)((total + 127) / 128), (unsigned)pl->img.NP);
 #define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP)                                                       \
-    if constexpr (KIND == 1)                                                                                     \
+    if constexpr (KIND == 1 || KIND == 3)                                                                        \
         if (c.id == ID) {                                                                                        \
             ubp_conv3x3_simple_kernel<NBK, P_><<<grid, 128, 0, stream>>>(                                        \
                 static_cast<const uint8_t *>(pl->dev), in, B, H, Wd, isb, isc, bias, relu, out, osb, osc,        \

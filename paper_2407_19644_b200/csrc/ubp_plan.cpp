@@ -44,6 +44,15 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
 {
     (void)M; (void)C; (void)m;
     const int nbk = largest_pow2_divisor_le16(Nb);
+    const double dens = (double)m * Nb / ((double)M * C);
+    if (R == 9 && dens >= 0.08 && M >= 128 && C >= 16) {    // implicit GEMM on tensor cores
+        switch (nbk) {
+            case 16: case 8: return find_cfg(40);
+            case 4: return find_cfg(41);
+            case 2: return find_cfg(42);
+            default: return find_cfg(43);
+        }
+    }
     if (R == 9) {
         switch (nbk) {
             case 16: case 8: return find_cfg(20);
@@ -56,8 +65,7 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     // Dense tensor-core variant when enough of the weight survives: measured on B200 (2048 x 2048 x 8192) it
     // takes the same time at every sparsity and beats the sparse kernel up to ~90 % sparsity; small or very
     // sparse layers stay on the sparse kernel.
-    const double density = (double)m * Nb / ((double)M * C);
-    if (density >= 0.08 && M >= 128 && C >= 128) {
+    if (dens >= 0.08 && M >= 128 && C >= 128) {
         switch (nbk) {
             case 16: case 8: return find_cfg(33);
             case 4: return find_cfg(32);
@@ -81,7 +89,8 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
     const int M = v.M, C = v.C, R = v.R, Nb = v.Nb;
     const int nbk = cfg.nbk, P = cfg.P, KT = cfg.KT, WR = cfg.WR;
     if (Nb % nbk != 0) return UBP_E_UNSUPPORTED;
-    if ((cfg.kind != 1 && R != 1) || (cfg.kind == 1 && R != 9)) return UBP_E_UNSUPPORTED;
+    const bool conv = (cfg.kind == 1 || cfg.kind == 3);
+    if ((!conv && R != 1) || (conv && R != 9)) return UBP_E_UNSUPPORTED;
     const int nkt = (C + KT - 1) / KT;
     const int NP = (M + P - 1) / P;
     const int NG = (NP + WR - 1) / WR;
@@ -135,8 +144,8 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
     size_t total = (cur + 255) & ~(size_t)255;
     if (total / 16 > 0xffffffffull) return UBP_E_UNSUPPORTED;
     img.tc_off = 0; img.tc_kp = 0;
-    if (cfg.kind == 2) {                 // dense part for the tensor-core kernel: Wh, Wl as [M][Kp] floats
-        img.tc_kp = (C + 3) & ~3;
+    if (cfg.kind == 2 || cfg.kind == 3) {   // dense part for the tensor-core kernel: Wh, Wl as [M][Kp] floats,
+        img.tc_kp = (C * R + 3) & ~3;       // reduction index k = channel * R + tap
         img.tc_off = total;
         total += ((size_t)2 * M * img.tc_kp * sizeof(float) + 255) & ~(size_t)255;
     }
@@ -205,7 +214,7 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
                 if (s + nbk > P) put(kt, p + 1, s - P + nbk - 1, jl, &wblk[(size_t)u * nbk * R]);
             }
         }
-    if (cfg.kind == 2) {
+    if (cfg.kind == 2 || cfg.kind == 3) {
         // Densify and split every kept weight into the part a TF32 operand holds exactly (sign, exponent,
         // top 10 mantissa bits) and the remainder, itself cut to TF32; pruned positions stay zero.
         float *Wh = reinterpret_cast<float *>(base + img.tc_off);
@@ -213,9 +222,10 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         for (int i = 0; i < M; ++i)
             for (int32_t b = v.indptr[i]; b < v.indptr[i + 1]; ++b) {
                 const int j = v.indices[b];
-                const float *val = v.values + (size_t)b * Nb;
-                for (int t = 0; t < Nb; ++t) {
-                    const float w = val[(i + t) % Nb];
+                const float *val = v.values + (size_t)b * Nb * R;
+                for (int t = 0; t < Nb; ++t)
+                  for (int r = 0; r < R; ++r) {
+                    const float w = val[(size_t)((i + t) % Nb) * R + r];
                     uint32_t bits;
                     std::memcpy(&bits, &w, 4);
                     bits &= 0xffffe000u;
@@ -225,9 +235,9 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
                     std::memcpy(&bits, &lo, 4);
                     bits &= 0xffffe000u;
                     std::memcpy(&lo, &bits, 4);
-                    Wh[(size_t)(i + t) * img.tc_kp + j] = hi;
-                    Wl[(size_t)(i + t) * img.tc_kp + j] = lo;
-                }
+                    Wh[(size_t)(i + t) * img.tc_kp + (size_t)j * R + r] = hi;
+                    Wl[(size_t)(i + t) * img.tc_kp + (size_t)j * R + r] = lo;
+                  }
             }
     }
     return UBP_OK;

@@ -151,8 +151,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 }
 
 struct TcArgs {
-    const float *X;          // [K][ldx]
+    const float *X;          // 1x1: [K][ldx]; 3x3: input tensor, element (b, c, y, x) at b*isb + c*isc + y*W + x
     int64_t ldx;
+    int conv;                // 0 = 1x1 product, 1 = 3x3 / stride 1 / pad 1 implicit GEMM (k = channel * 9 + tap)
+    int H, W;                // 3x3 only: plane size; column n = b*H*W + y*W + x
+    int64_t isb, isc;        // 3x3 only: input batch / channel strides (elements)
     const float *bias;
     float *Y;
     int64_t ldy;
@@ -267,7 +270,35 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
         float xr[PD][KH];
         const bool col_live = t < a.ntile && col0 + t < a.Nc;
         const float *xcol = a.X + (col_live ? col0 + t : 0) + (size_t)kh * KH * a.ldx;
+        // 3x3: this thread's output pixel and which of its nine taps fall inside the image
+        const float *pix_base = a.X;
+        uint32_t tap_ok = 0;
+        if (a.conv && col_live) {
+            const int64_t n = col0 + t;
+            const int hw = a.H * a.W;
+            const int b = (int)(n / hw), pix = (int)(n - (int64_t)b * hw);
+            const int y = pix / a.W, x = pix - y * a.W;
+            pix_base = a.X + (size_t)b * a.isb + (size_t)y * a.W + x;
+#pragma unroll
+            for (int tp = 0; tp < 9; ++tp) {
+                const int yy = y + tp / 3 - 1, xx = x + tp % 3 - 1;
+                if (yy >= 0 && yy < a.H && xx >= 0 && xx < a.W) tap_ok |= 1u << tp;
+            }
+        }
         auto load_chunk = [&](int c, float (&dst)[KH]) {
+            if (a.conv) {
+                // implicit lowering: reduction index k = channel * 9 + tap reads the input plane in place
+                int k = c * TC_KC + kh * KH;
+                int ch = k / 9, tp = k - 9 * ch;
+#pragma unroll
+                for (int i = 0; i < KH; ++i) {
+                    const bool live = ((tap_ok >> tp) & 1u) && k + i < a.K;
+                    const int doff = (tp / 3 - 1) * a.W + (tp % 3 - 1);
+                    dst[i] = live ? __ldg(pix_base + (size_t)ch * a.isc + doff) : 0.f;
+                    if (++tp == 9) { tp = 0; ++ch; }
+                }
+                return;
+            }
             const float *p = xcol + (size_t)c * TC_KC * a.ldx;
             if (col_live && (c + 1) * TC_KC <= a.K) {
 #pragma unroll
@@ -408,11 +439,10 @@ int encode_2d(CUtensorMap *tm, const void *base, uint64_t inner, uint64_t outer,
 
 }  // namespace
 
-int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
-                   float *Y, int64_t ldy, void *stream_)
+static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
 {
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const int M = pl->dims.M, K = pl->dims.C;
+    const int M = pl->dims.M, K = a.K;
+    const int64_t Nc = a.Nc;
     const uint8_t *dev = static_cast<const uint8_t *>(pl->dev);
     const float *Wh = reinterpret_cast<const float *>(dev + pl->img.tc_off);
     const float *Wl = Wh + (size_t)M * pl->img.tc_kp;
@@ -422,12 +452,10 @@ int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, 
                         CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
     if ((rc = encode_2d(&tmWl, Wl, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,
                         CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
-
-    TcArgs a;
-    a.X = X; a.ldx = ldx; a.bias = bias; a.Y = Y; a.ldy = ldy; a.Nc = Nc; a.M = M; a.K = K; a.relu = relu;
+    a.M = M;
     a.status = reinterpret_cast<int *>(pl->dev);
     // Tile choice: 128 or 256 rows, 64..256 columns (multiples of 32). Estimate the time of each candidate as
-    // (waves over the SMs) x (chunks x MMA cycles per chunk + a fixed per-tile cost) and keep the cheapest.
+    // (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost) and keep the cheapest.
     int sms = 148, devid = 0;
     if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
     const int nchunk = (K + TC_KC - 1) / TC_KC;
@@ -437,11 +465,12 @@ int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, 
         for (int n = 64; n <= TC_N; n += 32) {
             const long long tiles = (long long)((M + 128 * mt - 1) / (128 * mt)) * ((Nc + n - 1) / n);
             const long long waves = (tiles + sms - 1) / sms;
-            // 6 MMAs per 8 channels and 128-row half, n/2 cycles each; narrow tiles re-read W more often, which
-            // shows as a floor on the cycles per chunk; ~6000 cycles of prologue + epilogue per tile
-            double per_chunk = mt * 6.0 * (TC_KC / 8) * (n / 2.0);
-            const double floor_chunk = mt == 2 ? 1400.0 : 750.0;
-            if (per_chunk < floor_chunk) per_chunk = floor_chunk;
+            // 6 MMAs per 8 channels and 128-row half, n/2 cycles each; shared-memory traffic (operand reads of
+            // the MMAs plus the W and X writes, ~128 B/cycle) puts a floor under the cycles per chunk
+            const double mma = mt * 6.0 * (TC_KC / 8) * (n / 2.0);
+            const double smem_bytes = mt * 6.0 * (TC_KC / 8) * (4096.0 + 32.0 * n) + mt * 16384.0 + 128.0 * n;
+            double per_chunk = mma > smem_bytes / 110.0 ? mma : smem_bytes / 110.0;
+            if (per_chunk < 700.0) per_chunk = 700.0;           // the transposing warps need about this long
             const double t = (double)waves * (nchunk * per_chunk + 6000.0 + 40.0 * mt * n);
             if (t < best) { best = t; best_mt = mt; best_n = n; }
         }
@@ -463,6 +492,23 @@ int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, 
     };
     if (use2) return launch(ubp_tc_kernel<2>, 2, (size_t)3 * (2 * 2 * A_HALF_BYTES + 2 * B_BYTES) + 1024);
     return launch(ubp_tc_kernel<1>, 1, (size_t)4 * (1 * 2 * A_HALF_BYTES + 2 * B_BYTES) + 1024);
+}
+
+int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                   float *Y, int64_t ldy, void *stream_)
+{
+    TcArgs a{};
+    a.X = X; a.ldx = ldx; a.conv = 0; a.bias = bias; a.Y = Y; a.ldy = ldy; a.Nc = Nc; a.K = pl->dims.C; a.relu = relu;
+    return launch_tc_common(pl, a, static_cast<cudaStream_t>(stream_));
+}
+
+int launch_conv3x3_tc(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
+                      const float *bias, int relu, float *out, int64_t out_ld, void *stream_)
+{
+    TcArgs a{};
+    a.X = in; a.ldx = 0; a.conv = 1; a.H = H; a.W = Wd; a.isb = isb; a.isc = isc;
+    a.bias = bias; a.Y = out; a.ldy = out_ld; a.Nc = (int64_t)B * H * Wd; a.K = pl->dims.C * 9; a.relu = relu;
+    return launch_tc_common(pl, a, static_cast<cudaStream_t>(stream_));
 }
 
 }  // namespace ubp

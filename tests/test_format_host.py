@@ -152,3 +152,27 @@ def test_plan_rejects_wrong_kind():
     with pytest.raises(ubp.UbpError):
         ubp.plan_size(blob, 999)
     assert ubp.plan_size(blob, 7) > 0   # 2 rows per entry: each block becomes two entries
+
+
+@pytest.mark.parametrize("M,C,Nb,p,R,variant,sparse_variant", [(130, 140, 4, 60, 1, 32, 14), (128, 20, 8, 50, 9, 40, 20)])
+def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
+    """The dense part of a tensor-core plan: Wh + Wl reproduces the masked weight to 2^-21 relative, both pieces are
+    exact TF32 numbers (low 13 mantissa bits clear), pruned positions are zero; k = channel * R + tap."""
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 33 + M, Nc=4 if R == 1 else None, R=R, B=1, H=2, Wd=2)
+    blob = ubp.ubp_pack(L.W, L.mask, Nb)
+    img, geom = ubp.plan_image(blob, variant)
+    tc_off = ubp.plan_size(blob, sparse_variant)             # same geometry without the dense part
+    kp = (C * R + 3) // 4 * 4
+    assert len(img) == tc_off + (2 * M * kp * 4 + 255) // 256 * 256
+    # the embedded sparse plan is byte-identical to the stand-alone one
+    img_s, _ = ubp.plan_image(blob, sparse_variant)
+    assert np.array_equal(img[:tc_off], img_s)
+    Wh = np.frombuffer(img, "<f4", M * kp, tc_off).reshape(M, kp)
+    Wl = np.frombuffer(img, "<f4", M * kp, tc_off + 4 * M * kp).reshape(M, kp)
+    assert not (Wh.view(np.uint32) & 0x1fff).any() and not (Wl.view(np.uint32) & 0x1fff).any()
+    Wm = (L.W * L.mask[:, :, None]).reshape(M, C * R)
+    assert not Wh[:, C * R:].any() and not Wl[:, C * R:].any()
+    got = Wh[:, :C * R].astype(np.float64) + Wl[:, :C * R]
+    assert np.all(np.abs(got - Wm) <= np.abs(Wm) * 2.0 ** -20)
+    assert not got[Wm == 0].any()
+    assert np.array_equal(Wh[:, :C * R], (Wm.view(np.uint32) & 0xffffe000).view(np.float32))

@@ -280,6 +280,25 @@ def test_conv3x3_small(env, M, C, Nb, p, B, H, Wd):
     assert torch.equal(Yn.permute(1, 0, 2, 3), Y)
 
 
+@pytest.mark.parametrize("M,C,Nb,p,B,H,Wd,variant", [(128, 16, 8, 50, 2, 14, 14, 0), (256, 32, 4, 60, 3, 7, 9, 0),
+                                                      (130, 20, 2, 50, 2, 5, 6, 42), (200, 24, 1, 70, 1, 8, 8, 43),
+                                                      (128, 40, 16, 50, 5, 6, 6, 40), (64, 16, 8, 50, 2, 6, 6, 40)])
+def test_conv3x3_tensor_core_variant(env, M, C, Nb, p, B, H, Wd, variant):
+    """3x3 as an implicit GEMM on tensor cores (variants 40..43; chosen automatically for dense-enough layers)."""
+    torch, ubp = env
+    L = ubp_synth.make_layer("c", M, C, Nb, p, 11 * M + C, B=B, H=H, Wd=Wd, R=9, x_dist="normal")
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb), variant)
+    assert plan.variant >= 40
+    b = torch.from_numpy(L.bias).cuda()
+    Y = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda(), b, True, layout="CNHW")
+    plan.check()
+    Yref, A = oracle.masked_conv3x3(L.W, L.mask, L.X, L.bias, relu=True)
+    check(Y.cpu().numpy(), Yref, A, L, tensor_core=True)
+    # NCHW output is not one [M][B*H*W] matrix: served by the plain kernel on the embedded sparse plan
+    Yn = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda().permute(1, 0, 2, 3).contiguous(), b, True, layout="NCHW")
+    check(Yn.permute(1, 0, 2, 3).contiguous().cpu().numpy(), Yref, A, L)
+
+
 def test_r50_3x3_config_sampled(env):
     torch, ubp = env
     L = ubp_synth.config_layers("r50_3x3")[0]
@@ -294,4 +313,9 @@ def test_r50_3x3_config_sampled(env):
     sy[:8] = [0, 0, 13, 13, 0, 13, 7, 7]; sx[:8] = [0, 13, 0, 13, 7, 7, 0, 13]          # corners and edges
     ys, as_ = oracle.masked_conv3x3_samples(L.W, L.mask, L.X, sb, so, sy, sx, L.bias, relu=True)
     err = scaled_error(Y[so, sb, sy, sx], ys, as_)
-    assert err <= TOL and err <= (terms_per_output(L) + 2) * 2.0 ** -24
+    n_terms = terms_per_output(L) + 2
+    assert err <= TOL and err <= (2.0 ** -18 + n_terms * 2.0 ** -23 if plan.variant >= 40 else n_terms * 2.0 ** -24)
+    # the plain 3x3 kernel on the same layer
+    plan_s = ubp.Plan(blob, 20)
+    Ys = ubp.ubp_conv3x3_implicit(plan_s, torch.from_numpy(L.X).cuda(), torch.from_numpy(L.bias).cuda(), True).cpu().numpy()
+    assert scaled_error(Ys[so, sb, sy, sx], ys, as_) <= n_terms * 2.0 ** -24
