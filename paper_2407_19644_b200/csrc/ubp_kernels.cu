@@ -584,6 +584,37 @@ static int launch_simple(const ubp_plan *pl, const float *X, int64_t ldx, int64_
     return check(cudaGetLastError());
 }
 
+// Dispatch helpers: only the kernels a configuration kind can use are instantiated.
+template <int KIND, int NBK, int P, int V, int WR, int WC, int KT, bool DUP>
+struct CfgLaunch {
+    static int main_kernel(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                           float *Y, int64_t ldy, cudaStream_t s)
+    {
+        if constexpr (KIND == 0) return launch_main<NBK, P, V, WR, WC, KT, DUP>(pl, X, ldx, Nc, bias, relu, Y, ldy, s);
+        else return UBP_E_UNSUPPORTED;
+    }
+    static int simple_kernel(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                             float *Y, int64_t ldy, cudaStream_t s)
+    {
+        if constexpr (KIND == 0 || KIND == 2) return launch_simple<NBK, P>(pl, X, ldx, Nc, bias, relu, Y, ldy, s);
+        else return UBP_E_UNSUPPORTED;
+    }
+    static int conv_kernel(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
+                           const float *bias, int relu, float *out, int64_t osb, int64_t osc, cudaStream_t s)
+    {
+        if constexpr (KIND == 1 || KIND == 3) {
+            const int64_t total = (int64_t)B * H * Wd;
+            dim3 grid((unsigned)((total + 127) / 128), (unsigned)pl->img.NP);
+            ubp_conv3x3_simple_kernel<NBK, P><<<grid, 128, 0, s>>>(
+                static_cast<const uint8_t *>(pl->dev), in, B, H, Wd, isb, isc, bias, relu, out, osb, osc, pl->dims.M,
+                pl->img.NP, pl->img.nkt, pl->img.NG, pl->cfg.WR, pl->cfg.KT);
+            return check(cudaGetLastError());
+        } else {
+            return UBP_E_UNSUPPORTED;
+        }
+    }
+};
+
 int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                 float *Y, int64_t ldy, void *stream_)
 {
@@ -594,17 +625,16 @@ int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, con
                       pl->dims.C < (1 << 30) && Nc < (1ll << 31);
     int rc = UBP_E_UNSUPPORTED;
     if (fast && c.kind == 2) return launch_spmm_tc(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
-#define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP)                                                     \
-    if constexpr (KIND == 0)                                                                                   \
-        if (fast && c.id == ID)                                                                                \
-            rc = launch_main<NBK, P_, V_, WR_, WC_, KT_, (DUP != 0)>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
+#define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP)                                                \
+    if (fast && c.id == ID)                                                                               \
+        rc = CfgLaunch<KIND, NBK, P_, V_, WR_, WC_, KT_, (DUP != 0)>::main_kernel(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
 #include "ubp_cfgs.inc"
 #undef UBP_CFG
     if (rc != UBP_E_UNSUPPORTED) return rc;
     // slower kernel: unaligned operands, or a plan group too large to stage
 #define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP) \
-    if constexpr (KIND == 0 || KIND == 2)                  \
-        if (c.id == ID) return launch_simple<NBK, P_>(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
+    if (c.id == ID)                                        \
+        return CfgLaunch<KIND, NBK, P_, V_, WR_, WC_, KT_, (DUP != 0)>::simple_kernel(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
 #include "ubp_cfgs.inc"
 #undef UBP_CFG
     return UBP_E_UNSUPPORTED;
@@ -620,15 +650,9 @@ int launch_conv3x3(const ubp_plan *pl, const float *in, int B, int H, int Wd, in
     if (c.kind == 3 && osb == (int64_t)H * Wd && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && osc % 4 == 0 &&
         osc >= total && total < (1ll << 31))
         return launch_conv3x3_tc(pl, in, B, H, Wd, isb, isc, bias, relu, out, osc, stream_);
-    dim3 grid((unsigned)((total + 127) / 128), (unsigned)pl->img.NP);
-#define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP)                                                       \
-    if constexpr (KIND == 1 || KIND == 3)                                                                        \
-        if (c.id == ID) {                                                                                        \
-            ubp_conv3x3_simple_kernel<NBK, P_><<<grid, 128, 0, stream>>>(                                        \
-                static_cast<const uint8_t *>(pl->dev), in, B, H, Wd, isb, isc, bias, relu, out, osb, osc,        \
-                pl->dims.M, pl->img.NP, pl->img.nkt, pl->img.NG, c.WR, c.KT);                                    \
-            return check(cudaGetLastError());                                                                    \
-        }
+#define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP) \
+    if (c.id == ID)                                        \
+        return CfgLaunch<KIND, NBK, P_, V_, WR_, WC_, KT_, (DUP != 0)>::conv_kernel(pl, in, B, H, Wd, isb, isc, bias, relu, out, osb, osc, stream);
 #include "ubp_cfgs.inc"
 #undef UBP_CFG
     return UBP_E_UNSUPPORTED;

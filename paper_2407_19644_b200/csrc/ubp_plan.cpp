@@ -62,10 +62,10 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
         }
     }
     if (R != 1) return nullptr;
-    // Dense tensor-core variant when enough of the weight survives: measured on B200 (2048 x 2048 x 8192) it
-    // takes the same time at every sparsity and beats the sparse kernel up to ~90 % sparsity; small or very
-    // sparse layers stay on the sparse kernel.
-    if (dens >= 0.08 && M >= 128 && C >= 128) {
+    // Dense tensor-core variant when enough of the weight survives and the layer is large enough to amortise its
+    // per-tile set-up: measured on B200 it takes the same time at every sparsity and beats the sparse kernel up to
+    // ~90 % sparsity on 2048 x 2048 x 8192; with 128 input channels or fewer the sparse kernel is as fast or faster.
+    if (dens >= 0.08 && M >= 128 && C >= 256) {
         switch (nbk) {
             case 16: case 8: return find_cfg(33);
             case 4: return find_cfg(32);
@@ -73,13 +73,18 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
             default: return find_cfg(30);
         }
     }
-    // measured on B200 (2048 x 2048 x 8192 sweep): 8-row panels, 256 columns per warp, 16 warps, 64-channel tiles
+    // Sparse kernel (measured sweep): 8-row panels, 256 columns per warp; 16 warps per CTA, or 8 when the layer has
+    // no more than 64 output rows; 64-channel tiles, or 32 when the layer has no more than 32 input channels.
+    // 16-row blocks run as two 8-row entries.
+    const bool few_rows = M <= 64, few_ch = C <= 32;
+    int id;
     switch (nbk) {
-        case 16: case 8: return find_cfg(16);     // 16-row blocks run as two 8-row entries
-        case 4: return find_cfg(14);
-        case 2: return find_cfg(15);
-        default: return find_cfg(17);
+        case 16: case 8: id = few_rows ? (few_ch ? 54 : 55) : 16; break;
+        case 4: id = few_rows ? (few_ch ? 50 : 51) : 14; break;
+        case 2: id = few_rows ? (few_ch ? 52 : 53) : 15; break;
+        default: id = few_rows ? (few_ch ? 56 : 57) : 17; break;
     }
+    return find_cfg(id);
 }
 
 static inline size_t pad16(size_t x) { return (x + 15) & ~(size_t)15; }

@@ -148,7 +148,7 @@ def test_plan_rejects_wrong_kind():
     with pytest.raises(ubp.UbpError):
         ubp.plan_size(blob, 20)         # a 3x3 configuration for an R = 1 blob
     with pytest.raises(ubp.UbpError):
-        ubp.plan_size(blob, 8)          # 8 rows per entry do not divide a block of 4
+        ubp.plan_size(blob, 9)          # 8 rows per entry do not divide a block of 4
     with pytest.raises(ubp.UbpError):
         ubp.plan_size(blob, 999)
     assert ubp.plan_size(blob, 7) > 0   # 2 rows per entry: each block becomes two entries
