@@ -211,13 +211,14 @@ struct SpmmArgs {
     int64_t Nc;
     int M;
     int nkt, NG;
+    int nstrips;             // column strips of the product (a CTA walks every gridDim.y-th of them)
     int stages;
     uint32_t stage_bytes;    // X tile + largest plan group, 128-byte multiple
     int relu;
 };
 
-// All warps of the CTA compute; thread 0 also feeds the pipeline: before it starts on tile kt it issues the
-// copies for tile kt + D (D = stages - 2) into the stage that every warp released two tiles ago, so that wait
+// All warps of the CTA compute; thread 0 also feeds the pipeline: before it starts on step `it` it issues the
+// copies for step it + D (D = stages - 2) into the stage that every warp released two steps ago, so that wait
 // almost never blocks. Each stage has a "full" mbarrier (completed by the copies' byte count) and an "empty"
 // one (one arrival per warp).
 template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW>
@@ -239,9 +240,12 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = blockIdx.x;                      // row group
-    const int strip = blockIdx.y;                  // column strip
+    // The CTA is persistent over column strips blockIdx.y, blockIdx.y + gridDim.y, ...: the copy pipeline runs
+    // straight across strip boundaries, so the loads of the next strip fly while this one computes and stores.
+    const int my_strips = (a.nstrips - (int)blockIdx.y + (int)gridDim.y - 1) / (int)gridDim.y;
+    const int total = my_strips * a.nkt;           // (strip, channel tile) steps of this CTA
     const int S = a.stages;
-    const int D = S > 2 ? S - 2 : 1;               // tiles in flight ahead of the one being computed
+    const int D = S > 2 ? S - 2 : 1;               // steps in flight ahead of the one being computed
     const uint32_t *gtab = reinterpret_cast<const uint32_t *>(a.plan + 256);
 
     if (threadIdx.x == 0) {
@@ -255,36 +259,41 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
     }
     __syncthreads();
 
-    int issued = 0;                                // tiles whose copies thread 0 has issued
-    auto issue_tile = [&](int kt) -> bool {        // thread 0 only
-        const int st = kt % S;
-        if (kt >= S && !mbar_wait(smem_u32(&bar_empty[st]), ((kt / S) - 1) & 1, &abort_flag)) return false;
-        const uint32_t o0 = gtab[(size_t)kt * a.NG + g], o1 = gtab[(size_t)kt * a.NG + g + 1];
+    int issued = 0;                                // steps whose copies thread 0 has issued
+    int iss_kt = 0, iss_strip = blockIdx.y;        // (channel tile, strip) of the next step to issue
+    auto issue_step = [&]() -> bool {              // thread 0 only
+        const int it = issued, st = it % S;
+        if (it >= S && !mbar_wait(smem_u32(&bar_empty[st]), ((it / S) - 1) & 1, &abort_flag)) return false;
+        const uint32_t o0 = gtab[(size_t)iss_kt * a.NG + g], o1 = gtab[(size_t)iss_kt * a.NG + g + 1];
         const uint32_t gbytes = (o1 - o0) * 16u;
         const uint32_t bar = smem_u32(&bar_full[st]);
         uint8_t *stage = smem + (size_t)st * a.stage_bytes;
         mbar_expect_tx(bar, (uint32_t)XT_BYTES + gbytes);
-        tma_load_2d(smem_u32(stage), &tmX, strip * CS, kt * KT, bar);
+        tma_load_2d(smem_u32(stage), &tmX, iss_strip * CS, iss_kt * KT, bar);
         bulk_load(smem_u32(stage + XT_BYTES), a.plan + (size_t)o0 * 16u, gbytes, bar);
         ++issued;
+        if (++iss_kt == a.nkt) { iss_kt = 0; iss_strip += gridDim.y; }
         return true;
     };
     if (threadIdx.x == 0)
-        for (int kt = 0; kt < D && kt < a.nkt; ++kt) issue_tile(kt);
+        for (int it = 0; it < D && it < total; ++it) issue_step();
 
     const int wr = warp / WC, wc = warp % WC;
     const int panel = g * WR + wr;
     float2 acc[P][2 * V];
-#pragma unroll
-    for (int r = 0; r < P; ++r)
-#pragma unroll
-        for (int q = 0; q < 2 * V; ++q) acc[r][q] = make_float2(0.f, 0.f);
 
     bool ok = true;
-    for (int kt = 0; kt < a.nkt; ++kt) {
-        if (threadIdx.x == 0 && kt + D < a.nkt) ok = issue_tile(kt + D);
-        const int st = kt % S;
-        ok = ok && mbar_wait(smem_u32(&bar_full[st]), (kt / S) & 1, &abort_flag);
+    int kt = 0, strip = blockIdx.y;
+    for (int it = 0; it < total; ++it) {
+        if (threadIdx.x == 0 && it + D < total) ok = issue_step();
+        if (kt == 0) {
+#pragma unroll
+            for (int r = 0; r < P; ++r)
+#pragma unroll
+                for (int q = 0; q < 2 * V; ++q) acc[r][q] = make_float2(0.f, 0.f);
+        }
+        const int st = it % S;
+        ok = ok && mbar_wait(smem_u32(&bar_full[st]), (it / S) & 1, &abort_flag);
         if (!ok) break;
         const uint8_t *stage = smem + (size_t)st * a.stage_bytes;
         const uint8_t *grp = stage + XT_BYTES;
@@ -310,42 +319,45 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bar_empty[st]));
-    }
-    if (!ok) {
-        // A bounded wait ran out somewhere in this CTA: report through the plan's status word and store
-        // nothing. Thread 0 first gives the copies it has in flight a bounded chance to land.
-        if (threadIdx.x == 0) {
-            const int first = issued > S ? issued - S : 0;
-            for (int kt = first; kt < issued; ++kt)
-                for (uint32_t it = 0; it < (1u << 16); ++it)
-                    if (mbar_try_wait(smem_u32(&bar_full[kt % S]), (kt / S) & 1)) break;
-        }
-        if (lane == 0) atomicExch(reinterpret_cast<int *>(const_cast<uint8_t *>(a.plan)), 1);
-        return;
-    }
+        if (++kt < a.nkt) continue;
 
-    // ---------------- epilogue: bias, activation, one 128-bit store per lane and column group
-    const int64_t col0 = (int64_t)strip * CS + wc * 128 * V + lane * 4;
+        // ---------------- strip finished: bias, activation, one 128-bit store per lane and column group
+        const int64_t col0 = (int64_t)strip * CS + wc * 128 * V + lane * 4;
 #pragma unroll
-    for (int r = 0; r < P; ++r) {
-        const int row = panel * P + r;
-        if (row >= a.M) break;
-        const float b = a.bias ? __ldg(a.bias + row) : 0.f;
-        float *yrow = a.Y + (size_t)row * a.ldy;
+        for (int r = 0; r < P; ++r) {
+            const int row = panel * P + r;
+            if (row < a.M) {
+                const float b = a.bias ? __ldg(a.bias + row) : 0.f;
+                float *yrow = a.Y + (size_t)row * a.ldy;
 #pragma unroll
-        for (int v = 0; v < V; ++v) {
-            const int64_t col = col0 + v * 128;
-            float4 o = make_float4(acc[r][2 * v].x + b, acc[r][2 * v].y + b,
-                                   acc[r][2 * v + 1].x + b, acc[r][2 * v + 1].y + b);
-            if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
-            if (col + 3 < a.Nc) {
-                *reinterpret_cast<float4 *>(yrow + col) = o;
-            } else {
-                if (col < a.Nc) yrow[col] = o.x;
-                if (col + 1 < a.Nc) yrow[col + 1] = o.y;
-                if (col + 2 < a.Nc) yrow[col + 2] = o.z;
+                for (int v = 0; v < V; ++v) {
+                    const int64_t col = col0 + v * 128;
+                    float4 o = make_float4(acc[r][2 * v].x + b, acc[r][2 * v].y + b,
+                                           acc[r][2 * v + 1].x + b, acc[r][2 * v + 1].y + b);
+                    if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                    if (col + 3 < a.Nc) {
+                        *reinterpret_cast<float4 *>(yrow + col) = o;
+                    } else {
+                        if (col < a.Nc) yrow[col] = o.x;
+                        if (col + 1 < a.Nc) yrow[col + 1] = o.y;
+                        if (col + 2 < a.Nc) yrow[col + 2] = o.z;
+                    }
+                }
             }
         }
+        kt = 0;
+        strip += gridDim.y;
+    }
+    if (!ok) {
+        // A bounded wait ran out somewhere in this CTA: report through the plan's status word and stop
+        // storing. Thread 0 first gives the copies it has in flight a bounded chance to land.
+        if (threadIdx.x == 0) {
+            const int first = issued > S ? issued - S : 0;
+            for (int it = first; it < issued; ++it)
+                for (uint32_t w = 0; w < (1u << 16); ++w)
+                    if (mbar_try_wait(smem_u32(&bar_full[it % S]), (it / S) & 1)) break;
+        }
+        if (lane == 0) atomicExch(reinterpret_cast<int *>(const_cast<uint8_t *>(a.plan)), 1);
     }
 }
 
@@ -539,7 +551,6 @@ static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t 
     int stages = (int)(kSmemBudget / stage_bytes);
     if (stages < 2) return UBP_E_UNSUPPORTED;
     if (stages > 5) stages = 5;
-    if (stages > pl->img.nkt) stages = pl->img.nkt < 1 ? 1 : pl->img.nkt;
 
     EncodeTiledFn enc = encode_fn();
     if (!enc) return UBP_E_CUDA;
@@ -568,7 +579,18 @@ static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t 
     a.plan = static_cast<const uint8_t *>(pl->dev);
     a.bias = bias; a.Y = Y; a.ldy = ldy; a.Nc = Nc; a.M = pl->dims.M;
     a.nkt = pl->img.nkt; a.NG = pl->img.NG; a.stages = stages; a.stage_bytes = (uint32_t)stage_bytes; a.relu = relu;
-    dim3 grid((unsigned)pl->img.NG, (unsigned)((Nc + CS - 1) / CS));
+    // one CTA per SM is resident (shared memory); give every SM about one CTA and let it walk its strips
+    const int nstrips = (int)((Nc + CS - 1) / CS);
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int gy = sms / pl->img.NG;
+    if (gy < 1) gy = 1;
+    if (gy > nstrips) gy = nstrips;
+    // even out the strips per CTA: with k strips each at most, do not launch more CTAs than needed for that k
+    const int per = (nstrips + gy - 1) / gy;
+    gy = (nstrips + per - 1) / per;
+    a.nstrips = nstrips;
+    dim3 grid((unsigned)pl->img.NG, (unsigned)gy);
     kern<<<grid, WR * WC * 32, smem, stream>>>(tm, a);
     return check(cudaGetLastError());
 }
