@@ -234,6 +234,63 @@ def cpu_oracle_time(L, budget_s=20.0):
     return flops / t / 1e9, oracle.num_threads(), sample, t
 
 
+def roofline_us(L, hbm_gbs):
+    """(time at the FP32 peak, time at the HBM copy bandwidth) of one layer, in microseconds."""
+    return (2.0 * L.surviving_macs / (FP32_PEAK_TFLOPS * 1e12) * 1e6, compulsory_bytes(L) / (hbm_gbs * 1e9) * 1e6)
+
+
+def run_chain(args, torch, ubp, rank, world, dist):
+    """The 13 pointwise layers of the MobileNetV1-shaped chain (batch 64, 1x4 blocks, 80 %, bias+ReLU, independent
+    seeded inputs per layer). One step = the 13 launches replayed from one CUDA graph."""
+    layers = ubp_synth.config_layers("mbv1_chain", index=rank)
+    hbm_gbs, peak_src = measured_peaks()
+    runs, plans, keep = [], [], []
+    for L in layers:
+        plan, run, _, _, X, Y, bias = build_runner(ubp, torch, L, args.variant)
+        plans.append(plan); runs.append(run); keep.append((X, Y, bias))
+    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    for run in runs:            # warm every kernel outside the capture (first-launch attribute set-up)
+        run()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    cap_stream = torch.cuda.Stream()
+    with torch.cuda.graph(graph, stream=cap_stream):
+        for run in runs:
+            run()
+    per_layer = []
+    for L, run in zip(layers, runs):
+        ts = time_steps(torch, run, max(5, args.steps // 5), 3, flush)
+        per_layer.append(float(np.median(ts)) * 1e3)
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    times = time_steps(torch, graph.replay, args.steps, args.warmup, flush)
+    clocks = sampler.stop()
+    for p in plans:
+        p.check()
+    step_ms = max_over_ranks(float(np.mean(times)), dist, torch, "cuda")
+    flops = sum(2.0 * L.surviving_macs for L in layers)
+    roofs = [roofline_us(L, hbm_gbs) for L in layers]
+    roof_total_us = sum(max(r) for r in roofs)
+    line = {
+        "metric": "effective GFLOP/s (2 x surviving MACs / time) of the 13-layer pointwise chain",
+        "value": aggregate_gflops(flops, world, step_ms), "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "mbv1_chain", "layers": 13, "batch": 64, "block": "4x1x1", "sparsity_pct": 80,
+                   "launch": "13 kernels replayed from one CUDA graph",
+                   "l2": "warm" if args.no_flush else "flushed between steps (256 MiB write)"},
+        "roofline": {"bound": "mixed (layers 1-4 hbm, 5-13 alu)", "roofline_us": roof_total_us,
+                     "frac_of_roofline_time": roof_total_us / (step_ms * 1e3),
+                     "peak_source": f"FP32 74.45 TFLOP/s derived; HBM {hbm_gbs} GB/s {peak_src}"},
+        "layers": [{"name": L.name, "M": L.M, "K": L.C, "Nc": L.Nc, "variant": p.variant, "us": us,
+                    "roofline_us": max(r), "bound": "alu" if r[0] >= r[1] else "hbm", "frac": max(r) / us}
+                   for L, p, us, r in zip(layers, plans, per_layer, roofs)],
+        "clocks": clocks, "gpu_launches": 13 * args.steps,
+    }
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
 def max_over_ranks(ms: float, dist, torch, device) -> float:
     """A step is as slow as its slowest rank: MAX-reduce the per-rank device time (no-op without a group)."""
     if dist is None:
@@ -293,6 +350,24 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     name = args.workload
+    if name == "mbv1_chain":
+        if args.impl == "reference":
+            raise SystemExit("--impl reference times single layers; pick a layer workload")
+        import torch
+        import paper_2407_19644_b200 as ubp
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+        ubp.load()
+        torch.cuda.set_device(local_rank)
+        dist = None
+        if world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        run_chain(args, torch, ubp, rank, world, dist)
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     L = get_layer(name, seed_index=rank)
 
     if args.impl == "reference":
