@@ -138,6 +138,16 @@ int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info);
  * launched with this plan gave up on a bounded wait. */
 int ubp_plan_check(const ubp_plan_t *plan, void *stream);
 
+/* ubp_plan_clear_status: reset the plan's device status word to 0 (one 4-byte cudaMemsetAsync on `stream`). */
+int ubp_plan_clear_status(const ubp_plan_t *plan, void *stream);
+
+/* ubp_selftest_bounded_wait: enqueue a one-warp kernel that waits on an mbarrier nobody ever completes, with
+ * the same bounded-wait code the product kernels use but a limit of `limit_us` microseconds (1 .. 1 000 000).
+ * When the limit runs out the kernel sets the plan's status word and returns, so a following ubp_plan_check
+ * reports UBP_E_DEVICE and the context stays usable. Exists so that the "a wait that runs out is reported, not
+ * hung" path can be exercised without any fault; not part of the paper's method. */
+int ubp_selftest_bounded_wait(const ubp_plan_t *plan, unsigned limit_us, void *stream);
+
 /* ------------------------------------------------------------------ compute
  * ubp_spmm: Y[M][Nc] = act(Wm[M][C] * X[C][Nc] + bias), the 1x1 / fully
  * connected case (R == 1), the weight-rotating output-stationary product of

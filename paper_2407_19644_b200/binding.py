@@ -63,6 +63,8 @@ def load():
     L.ubp_spmm.argtypes = [vp, vp, i64, i64, vp, i32, vp, i64, vp]
     L.ubp_conv1x1.argtypes = [vp, vp, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
     L.ubp_conv3x3_implicit.argtypes = [vp, vp, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
+    L.ubp_plan_clear_status.argtypes = [vp, vp]
+    L.ubp_selftest_bounded_wait.argtypes = [vp, C.c_uint, vp]
     L.ubp_static_plan_capacity.restype = sz
     L.ubp_spmm_static.argtypes = [vp, sz, vp, i64, i64, vp, i32, vp, i64, vp]
     _lib = L
@@ -212,6 +214,15 @@ class Plan:
     def check(self, stream=None):
         """Synchronise the stream and raise if a kernel reported a failed bounded wait."""
         _chk(self._lib.ubp_plan_check(self.handle, _stream_ptr(stream)), "ubp_plan_check")
+
+    def clear_status(self, stream=None):
+        _chk(self._lib.ubp_plan_clear_status(self.handle, _stream_ptr(stream)), "ubp_plan_clear_status")
+
+    def selftest_bounded_wait(self, limit_us: int = 20000, stream=None):
+        """Launch the library's wait self test: a kernel whose wait can never complete gives up after `limit_us`
+        and flags the plan; check() then raises UbpError(-7)."""
+        _chk(self._lib.ubp_selftest_bounded_wait(self.handle, int(limit_us), _stream_ptr(stream)),
+             "ubp_selftest_bounded_wait")
 
     def free(self):
         if self._handle is not None:

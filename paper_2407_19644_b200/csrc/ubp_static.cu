@@ -40,7 +40,54 @@ int static_plan_ptr(void **out)
 
 }  // namespace
 
+// ---- bounded-wait self test -------------------------------------------------------------------------------
+namespace {
+__global__ void ubp_wait_selftest_kernel(int *status, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    const unsigned addr = (unsigned)__cvta_generic_to_shared(&bar);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(addr));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        unsigned long long t0, t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+        bool done = false;
+        for (unsigned it = 0; !done; ++it) {          // nobody arrives: only the clock ends this loop
+            unsigned ok;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                         "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(addr), "r"(0u) : "memory");
+            if (ok) break;
+            if ((it & 63u) == 0u) {
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+                if (t - t0 > limit_ns) { atomicExch(status, 1); done = true; }
+            }
+        }
+    }
+}
+}  // namespace
+
 extern "C" {
+
+int ubp_plan_clear_status(const ubp_plan_t *plan, void *stream)
+{
+    if (!plan || !plan->dev) return UBP_E_ARG;
+    cudaError_t e = cudaMemsetAsync(plan->dev, 0, sizeof(int), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { ubp::set_last_cuda_error((int)e); return UBP_E_CUDA; }
+    return UBP_OK;
+}
+
+int ubp_selftest_bounded_wait(const ubp_plan_t *plan, unsigned limit_us, void *stream)
+{
+    if (!plan || !plan->dev || limit_us == 0 || limit_us > 1000000u) return UBP_E_ARG;
+    ubp_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<int *>(plan->dev),
+                                                                             (unsigned long long)limit_us * 1000ull);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { ubp::set_last_cuda_error((int)e); return UBP_E_CUDA; }
+    return UBP_OK;
+}
 
 size_t ubp_static_plan_capacity(void) { return UBP_STATIC_PLAN_BYTES; }
 

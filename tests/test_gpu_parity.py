@@ -320,3 +320,48 @@ def test_r50_3x3_config_sampled(env):
     plan_s = ubp.Plan(blob, 20)
     Ys = ubp.ubp_conv3x3_implicit(plan_s, torch.from_numpy(L.X).cuda(), torch.from_numpy(L.bias).cuda(), True).cpu().numpy()
     assert scaled_error(Ys[so, sb, sy, sx], ys, as_) <= n_terms * 2.0 ** -24
+
+
+def test_bounded_wait_is_reported_not_hung(env):
+    """A wait that can never complete returns after its limit and is reported through the plan's status word; the
+    context stays usable and the next product is correct."""
+    import time
+    torch, ubp = env
+    L = ubp_synth.make_layer("t", 64, 32, 4, 50, 91, Nc=256)
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, 4))
+    plan.check()
+    t0 = time.perf_counter()
+    plan.selftest_bounded_wait(limit_us=20000)
+    with pytest.raises(ubp.UbpError) as e:
+        plan.check()
+    assert e.value.code == -7 and time.perf_counter() - t0 < 5.0
+    plan.clear_status()
+    plan.check()
+    Yh, Yref, A, _ = run_spmm(env, L)
+    check(Yh, Yref, A, L)
+
+
+def test_launches_can_be_captured_in_a_cuda_graph(env):
+    """Two layers chained through a CUDA graph (as the 13-layer benchmark does) give the eager results."""
+    torch, ubp = env
+    L1 = ubp_synth.make_layer("a", 256, 256, 4, 70, 92, Nc=1024)            # tensor-core kernel
+    L2 = ubp_synth.make_layer("b", 64, 256, 4, 90, 93, Nc=1024)             # sparse kernel
+    p1 = ubp.Plan(ubp.ubp_pack(L1.W, L1.mask, 4)); p2 = ubp.Plan(ubp.ubp_pack(L2.W, L2.mask, 4))
+    X = torch.from_numpy(L1.X).cuda()
+    b1 = torch.from_numpy(L1.bias).cuda(); b2 = torch.from_numpy(L2.bias).cuda()
+    Y1 = torch.empty((256, 1024), device="cuda"); Y2 = torch.empty((64, 1024), device="cuda")
+    ubp.ubp_spmm(p1, X, b1, True, out=Y1); ubp.ubp_spmm(p2, Y1, b2, True, out=Y2)   # eager (also first-launch set-up)
+    want = Y2.clone()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=torch.cuda.Stream()):
+        ubp.ubp_spmm(p1, X, b1, True, out=Y1)
+        ubp.ubp_spmm(p2, Y1, b2, True, out=Y2)
+    Y2.zero_()
+    g.replay(); g.replay()
+    torch.cuda.synchronize()
+    p1.check(); p2.check()
+    assert torch.equal(Y2, want)
+    Yref1, _ = oracle.masked_matmul(L1.W, L1.mask, L1.X, L1.bias, relu=True)
+    Yref2, A2 = oracle.masked_matmul(L2.W, L2.mask, Yref1.astype(np.float32), L2.bias, relu=True)
+    assert scaled_error(Y2.cpu().numpy(), Yref2, A2) <= TOL
