@@ -150,7 +150,7 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
     if (total / 16 > 0xffffffffull) return UBP_E_UNSUPPORTED;
     img.tc_off = 0; img.tc_kp = 0;
     if (cfg.kind == 2 || cfg.kind == 3) {   // dense part for the tensor-core kernel: Wh, Wl as [M][Kp] floats,
-        img.tc_kp = (C * R + 3) & ~3;       // reduction index k = channel * R + tap
+        img.tc_kp = (C * R + 3) & ~3;       // reduction index k = tap * C + channel (tap-major)
         img.tc_off = total;
         total += ((size_t)2 * M * img.tc_kp * sizeof(float) + 255) & ~(size_t)255;
     }
@@ -240,8 +240,8 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
                     std::memcpy(&bits, &lo, 4);
                     bits &= 0xffffe000u;
                     std::memcpy(&lo, &bits, 4);
-                    Wh[(size_t)(i + t) * img.tc_kp + (size_t)j * R + r] = hi;
-                    Wl[(size_t)(i + t) * img.tc_kp + (size_t)j * R + r] = lo;
+                    Wh[(size_t)(i + t) * img.tc_kp + (size_t)r * C + j] = hi;
+                    Wl[(size_t)(i + t) * img.tc_kp + (size_t)r * C + j] = lo;
                   }
             }
     }

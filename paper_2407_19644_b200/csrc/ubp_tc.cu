@@ -153,7 +153,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 struct TcArgs {
     const float *X;          // 1x1: [K][ldx]; 3x3: input tensor, element (b, c, y, x) at b*isb + c*isc + y*W + x
     int64_t ldx;
-    int conv;                // 0 = 1x1 product, 1 = 3x3 / stride 1 / pad 1 implicit GEMM (k = channel * 9 + tap)
+    int conv;                // 0 = 1x1 product, 1 = 3x3 / stride 1 / pad 1 implicit GEMM (k = tap * C + channel)
     int H, W;                // 3x3 only: plane size; column n = b*H*W + y*W + x
     int64_t isb, isc;        // 3x3 only: input batch / channel strides (elements)
     const float *bias;
@@ -287,15 +287,24 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
         }
         auto load_chunk = [&](int c, float (&dst)[KH]) {
             if (a.conv) {
-                // implicit lowering: reduction index k = channel * 9 + tap reads the input plane in place
-                int k = c * TC_KC + kh * KH;
-                int ch = k / 9, tp = k - 9 * ch;
+                // implicit lowering: reduction index k = tap * C + channel reads the input plane in place; the
+                // 8 channels of this thread normally share one tap, so tap test and offset are per chunk
+                const int C = a.K / 9;
+                const int k0 = c * TC_KC + kh * KH;
+                int tp = k0 / C, ch = k0 - tp * C;
+                if (ch + KH <= C) {
+                    const bool live = tp < 9 && ((tap_ok >> tp) & 1u);
+                    const float *p = pix_base + (size_t)ch * a.isc + ((tp / 3 - 1) * a.W + (tp % 3 - 1));
 #pragma unroll
-                for (int i = 0; i < KH; ++i) {
-                    const bool live = ((tap_ok >> tp) & 1u) && k + i < a.K;
-                    const int doff = (tp / 3 - 1) * a.W + (tp % 3 - 1);
-                    dst[i] = live ? __ldg(pix_base + (size_t)ch * a.isc + doff) : 0.f;
-                    if (++tp == 9) { tp = 0; ++ch; }
+                    for (int i = 0; i < KH; ++i) dst[i] = live ? __ldg(p + (size_t)i * a.isc) : 0.f;
+                } else {
+#pragma unroll
+                    for (int i = 0; i < KH; ++i) {
+                        const bool live = tp < 9 && ((tap_ok >> tp) & 1u);
+                        const int doff = (tp / 3 - 1) * a.W + (tp % 3 - 1);
+                        dst[i] = live ? __ldg(pix_base + (size_t)ch * a.isc + doff) : 0.f;
+                        if (++ch == C) { ch = 0; ++tp; }
+                    }
                 }
                 return;
             }

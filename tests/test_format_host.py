@@ -157,7 +157,7 @@ def test_plan_rejects_wrong_kind():
 @pytest.mark.parametrize("M,C,Nb,p,R,variant,sparse_variant", [(130, 140, 4, 60, 1, 32, 14), (128, 20, 8, 50, 9, 40, 20)])
 def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     """The dense part of a tensor-core plan: Wh + Wl reproduces the masked weight to 2^-21 relative, both pieces are
-    exact TF32 numbers (low 13 mantissa bits clear), pruned positions are zero; k = channel * R + tap."""
+    exact TF32 numbers (low 13 mantissa bits clear), pruned positions are zero; k = tap * C + channel."""
     L = ubp_synth.make_layer("t", M, C, Nb, p, 33 + M, Nc=4 if R == 1 else None, R=R, B=1, H=2, Wd=2)
     blob = ubp.ubp_pack(L.W, L.mask, Nb)
     img, geom = ubp.plan_image(blob, variant)
@@ -170,7 +170,7 @@ def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     Wh = np.frombuffer(img, "<f4", M * kp, tc_off).reshape(M, kp)
     Wl = np.frombuffer(img, "<f4", M * kp, tc_off + 4 * M * kp).reshape(M, kp)
     assert not (Wh.view(np.uint32) & 0x1fff).any() and not (Wl.view(np.uint32) & 0x1fff).any()
-    Wm = (L.W * L.mask[:, :, None]).reshape(M, C * R)
+    Wm = np.ascontiguousarray((L.W * L.mask[:, :, None]).transpose(0, 2, 1)).reshape(M, R * C)   # k = tap * C + channel
     assert not Wh[:, C * R:].any() and not Wl[:, C * R:].any()
     got = Wh[:, :C * R].astype(np.float64) + Wl[:, :C * R]
     assert np.all(np.abs(got - Wm) <= np.abs(Wm) * 2.0 ** -20)
