@@ -474,12 +474,15 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
         for (int n = 64; n <= TC_N; n += 32) {
             const long long tiles = (long long)((M + 128 * mt - 1) / (128 * mt)) * ((Nc + n - 1) / n);
             const long long waves = (tiles + sms - 1) / sms;
-            // 6 MMAs per 8 channels and 128-row half, n/2 cycles each; shared-memory traffic (operand reads of
-            // the MMAs plus the W and X writes, ~128 B/cycle) puts a floor under the cycles per chunk
-            const double mma = mt * 6.0 * (TC_KC / 8) * (n / 2.0);
-            const double smem_bytes = mt * 6.0 * (TC_KC / 8) * (4096.0 + 32.0 * n) + mt * 16384.0 + 128.0 * n;
-            double per_chunk = mma > smem_bytes / 110.0 ? mma : smem_bytes / 110.0;
-            if (per_chunk < 700.0) per_chunk = 700.0;           // the transposing warps need about this long
+            // Per 16-channel chunk: 6 MMAs per 128-row half, n/2 cycles each; shared memory carries the MMAs'
+            // operand reads (4 KB of W + 32 B per column each) plus the W (TMA) and X (transposing warps) writes at
+            // ~120 B/cycle; the transposing warps themselves need ~1150 cycles per chunk (1500 with two halves:
+            // measured with in-kernel timers). Per tile ~6000 cycles of prologue plus an epilogue ~ its outputs.
+            const double mma = mt * 3.0 * (TC_KC / 8) * (n / 2.0);
+            const double smem_bytes = mt * 3.0 * (TC_KC / 8) * (4096.0 + 32.0 * n) + mt * 16384.0 + 128.0 * n;
+            double per_chunk = mma > smem_bytes / 120.0 ? mma : smem_bytes / 120.0;
+            const double floor_chunk = mt == 1 ? 1150.0 : 1500.0;
+            if (per_chunk < floor_chunk) per_chunk = floor_chunk;
             const double t = (double)waves * (nchunk * per_chunk + 6000.0 + 40.0 * mt * n);
             if (t < best) { best = t; best_mt = mt; best_n = n; }
         }
