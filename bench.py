@@ -75,9 +75,10 @@ def tf32_peak_tflops():
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (key: workload, tensor-core variant?)
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("mbv1_pw512", True): 14982400 + 768,      # profiles/ncu_full_ubp_tc_kernel_mbv1_pw512.md (output still in L2)
-    ("mbv1_pw512", False): 13414656,           # profiles/ncu_full_ubp_spmm_kernel.md
-    ("sweep_nb4_p70", False): 76188928 + 33089024,
+    ("mbv1_pw512", True): 15005696 + 0,          # profiles/ncu_ubp_tc_kernel_mbv1_pw512.md (the output is still in L2)
+    ("sweep_nb4_p70", True): 135086848 + 37817856,   # profiles/ncu_ubp_tc_kernel_sweep_nb4_p70.md
+    ("r50_3x3", True): 17635840 + 0,             # profiles/ncu_ubp_tc_kernel_r50_3x3.md
+    ("sweep_nb4_p90", False): 70554368 + 23536640,   # profiles/ncu_ubp_spmm_kernel_sweep_nb4_p90.md
 }
 
 
@@ -426,9 +427,9 @@ def main():
     roof["frac_of_roofline_time"] = max(t_alu, t_hbm) / (step_ms * 1e-3)
     roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((name, plan.variant >= 30))
     roof["kernel"] = "ubp_tc_kernel (dense 3xTF32 on tcgen05)" if plan.variant >= 30 else "ubp_spmm_kernel (sparse, FP32 FMA)"
-    if plan.variant >= 30 and L.R == 1:
+    if plan.variant >= 30:
         # the tensor-core variant does 3 x the DENSE multiply-adds; report that rate against the TF32 peak too
-        dense_tf = 3 * 2.0 * L.M * L.C * L.Nc / (step_ms * 1e-3) / 1e12
+        dense_tf = 3 * 2.0 * L.M * L.C * L.R * L.Nc / (step_ms * 1e-3) / 1e12
         tf32_peak = tf32_peak_tflops()
         roof["tensor"] = {"dense_tf32_tflops": dense_tf, "peak": tf32_peak[0], "peak_source": tf32_peak[1],
                           "frac": dense_tf / tf32_peak[0]}
