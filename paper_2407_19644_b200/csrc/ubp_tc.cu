@@ -25,13 +25,15 @@
 #include <cstring>
 
 #include "ubp_internal.h"
+#include "ubp_tc_common.cuh"
 
 namespace ubp {
 
 namespace {
 
+using namespace tc;
+
 constexpr int TC_N = 256;          // columns per CTA
-constexpr int TC_KC = 16;          // channels per pipeline stage
 constexpr int TC_SPLIT_WARPS = 16; // warps 2..17 transpose/split X and run the epilogue
 constexpr int TC_THREADS = (2 + TC_SPLIT_WARPS) * 32;
 constexpr uint32_t A_HALF_BYTES = 128 * TC_KC * 4;          // one 128-row chunk of Wh or Wl: 8 KB
@@ -39,132 +41,6 @@ constexpr uint32_t B_BYTES = TC_KC * TC_N * 4;              // Xh or Xl chunk: 1
 constexpr uint32_t B_LBO = 128;                             // next 4 channels of the same 8 columns
 constexpr uint32_t B_SBO = (TC_KC / 4) * 128;               // next 8 columns: 512 B
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// bounded wait (one second); false if it ran out or another thread of the CTA already gave up
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > 1000000000ull) break;
-        }
-    }
-    *abort_flag = 1;
-    return false;
-}
-// same, for waiters that are not on the critical path: sleep between polls so they do not take issue slots
-// from the thread that feeds the tensor core
-__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int *abort_flag)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_ns();
-    for (uint32_t it = 1;; ++it) {
-        __nanosleep(40);
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > 1000000000ull) break;
-        }
-    }
-    *abort_flag = 1;
-    return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-
-// shared-memory matrix descriptor (tcgen05): start address, leading / stride byte offsets (all >> 4),
-// descriptor version 1, swizzle mode in the top three bits
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle)
-{
-    return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
-           ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46) | ((uint64_t)swizzle << 61);
-}
-constexpr uint32_t SWZ_NONE = 0, SWZ_64B = 4;
-
-// instruction descriptor: D = f32, A = B = tf32, both K-major, M = 128, N given at run time (multiple of 16)
-__device__ __forceinline__ uint32_t make_idesc(int n)
-{
-    return (1u << 4) | (2u << 7) | (2u << 10) | (0u << 15) | (0u << 16) | ((uint32_t)(n >> 3) << 17) |
-           ((uint32_t)(128 >> 4) << 24);
-}
-
-__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t kIdesc,
-                                         uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(kIdesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
-        : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-
-struct TcArgs {
-    const float *X;          // 1x1: [K][ldx]; 3x3: input tensor, element (b, c, y, x) at b*isb + c*isc + y*W + x
-    int64_t ldx;
-    int conv;                // 0 = 1x1 product, 1 = 3x3 / stride 1 / pad 1 implicit GEMM (k = tap * C + channel)
-    int H, W;                // 3x3 only: plane size; column n = b*H*W + y*W + x
-    int64_t isb, isc;        // 3x3 only: input batch / channel strides (elements)
-    const float *bias;
-    float *Y;
-    int64_t ldy;
-    int64_t Nc;
-    int M, K;
-    int ntile;               // columns per CTA: multiple of 32, <= 256
-    int relu;
-    int *status;             // plan status word
-};
 
 template <int MT>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -446,7 +322,28 @@ int encode_2d(CUtensorMap *tm, const void *base, uint64_t inner, uint64_t outer,
     return UBP_OK;
 }
 
+int encode_3d(CUtensorMap *tm, const void *base, const uint64_t (&dims)[3], uint64_t stride1_bytes, uint64_t stride2_bytes,
+              const uint32_t (&box)[3], CUtensorMapSwizzle swz)
+{
+    EncodeTiledFn enc = tc_encode_fn();
+    if (!enc) return UBP_E_CUDA;
+    const cuuint64_t d[3] = {dims[0], dims[1], dims[2]};
+    const cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+    const cuuint32_t b[3] = {box[0], box[1], box[2]};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult cr = enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), d, strides, b, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) { set_last_cuda_error(-(int)cr); return UBP_E_CUDA; }
+    return UBP_OK;
+}
+
 }  // namespace
+
+
+// two-CTA kernel (ubp_tc2.cu)
+int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, const void *args, int M, int64_t Nc,
+                   int ntile, void *stream);
 
 static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
 {
@@ -486,6 +383,43 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
             const double t = (double)waves * (nchunk * per_chunk + 6000.0 + 40.0 * mt * n);
             if (t < best) { best = t; best_mt = mt; best_n = n; }
         }
+    // Two-CTA kernel for the 1x1 product (256 rows per CTA pair; X goes from global memory into the operand layout
+    // by TMA, each SM holds and reads only half of the X tile). Its chunk time is the MMA time (6 MMAs of n/2
+    // cycles) or, for narrow tiles, what the issuing thread needs per chunk (~680 cycles measured); per tile
+    // ~9000 cycles of pipeline fill and drain plus an epilogue ~ its outputs.
+    if (M > 128 && !a.conv) {
+        double best2 = 1e300;
+        int best2_n = 256;
+        for (int n = 64; n <= 256; n += 64) {
+            const long long ctas = 2ll * ((M + 255) / 256) * ((Nc + n - 1) / n);
+            const long long waves = (ctas + (sms & ~1) - 1) / (sms & ~1);
+            double per_chunk = 3.0 * (TC_KC / 8) * (n / 2.0);
+            if (per_chunk < 680.0) per_chunk = 680.0;
+            const double t = (double)waves * (nchunk * per_chunk + 9000.0 + 30.0 * n);
+            if (t < best2) { best2 = t; best2_n = n; }
+        }
+        if (best2 < best) {
+            // Wh and Wl as one 3-D tensor (channel, row, part): one copy per chunk brings both
+            CUtensorMap tmW, tmX;
+            const uint64_t wdims[3] = {(uint64_t)pl->img.tc_kp, (uint64_t)M, 2};
+            const uint32_t wbox[3] = {TC_KC, 128, 2};
+            if ((rc = encode_3d(&tmW, Wh, wdims, (uint64_t)pl->img.tc_kp * 4, (uint64_t)M * pl->img.tc_kp * 4, wbox,
+                                CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
+            // X as (column in a group of 32, channel, group): one copy per chunk brings all of a CTA's columns in
+            // the operand layout. Needs whole groups; otherwise one 2-D copy per group.
+            const int x3d = (Nc % 32 == 0) ? 1 : 0;
+            if (x3d) {
+                const uint64_t xdims[3] = {32, (uint64_t)K, (uint64_t)(Nc / 32)};
+                const uint32_t xbox[3] = {32, TC_KC, (uint32_t)(best2_n / 64)};
+                rc = encode_3d(&tmX, a.X, xdims, (uint64_t)a.ldx * 4, 128, xbox, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+            } else {
+                rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)K, (uint64_t)a.ldx * 4, 32, TC_KC,
+                               CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+            }
+            if (rc) return rc;
+            return launch_tc_pair(&tmW, &tmX, x3d, &a, M, Nc, best2_n, stream);
+        }
+    }
     a.ntile = best_n;
     const bool use2 = best_mt == 2;
     const unsigned ncols = (unsigned)((Nc + best_n - 1) / best_n);

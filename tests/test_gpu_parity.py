@@ -85,6 +85,9 @@ TC_CASES = [
     (128, 64, 4, 50, 256, 32), (128, 16, 4, 50, 256, 32), (100, 70, 4, 60, 300, 32), (300, 150, 4, 70, 520, 32),
     (257, 33, 1, 60, 260, 30), (64, 64, 2, 50, 256, 31), (520, 200, 8, 50, 1028, 33), (260, 40, 16, 50, 516, 33),
     (130, 257, 4, 80, 1028, 32), (384, 100, 12, 40, 772, 32), (256, 128, 4, 0, 512, 32), (200, 20, 4, 100, 256, 32),
+    # more than 128 rows: the two-CTA kernel; whole 32-column groups (one 3-D copy of X per chunk) with and without
+    # a ragged last column tile, more chunks than pipeline stages, a ragged last row pair
+    (512, 96, 4, 60, 2048, 32), (300, 150, 4, 70, 544, 32), (256, 256, 4, 70, 4128, 32), (640, 40, 8, 50, 96, 33),
 ]
 
 
@@ -248,7 +251,36 @@ def test_sweep_config_sampled(env, nb, sp, variant):
         assert scaled_error(Y[o], ys, as_) <= TOL
 
 
-@pytest.mark.parametrize("li", [0, 1, 3, 5, 11, 12])
+def test_two_cta_kernel_padded_rows_and_repeated_launches(env):
+    """The two-CTA tensor-core kernel with a leading dimension larger than the column count, and forty launches
+    in a row on a layer with many column tiles and few chunks (several waves of CTA pairs; the copies of different
+    chunks land out of order under load): every launch must finish with a clean status word and the same result."""
+    torch, ubp = env
+    L = ubp_synth.make_layer("t", 256, 64, 4, 60, 4242, Nc=512, x_dist="normal")
+    check(*run_spmm(env, L, 32, pad=4)[:3], L, tensor_core=True)
+    L = ubp_synth.config_layers("mbv1_chain", batch=64)[4]          # 256 -> 256 channels at 28 x 28: 50176 columns
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb), 32)
+    X = torch.from_numpy(L.X).cuda().reshape(L.C, -1)
+    bias = torch.from_numpy(L.bias).cuda()
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device="cuda")
+    Y0 = ubp.ubp_spmm(plan, X, bias, True).clone()
+    plan.check()
+    Y = torch.empty_like(Y0)
+    for i in range(40):
+        if i % 2:
+            flush.zero_()
+        ubp.ubp_spmm(plan, X, bias, True, out=Y)
+    plan.check()
+    assert torch.equal(Y, Y0)
+    Yh = Y.cpu().numpy()
+    X2 = L.X.reshape(L.C, -1)
+    rng = np.random.default_rng(5)
+    so = rng.integers(0, L.M, 5000); sn = rng.integers(0, X2.shape[1], 5000)
+    ys, as_ = oracle.masked_matmul_samples(L.W, L.mask, X2, so, sn, L.bias, relu=True)
+    assert scaled_error(Yh[so, sn], ys, as_) <= TOL
+
+
+@pytest.mark.parametrize("li", [0, 1, 3, 4, 5, 6, 11, 12])
 def test_mbv1_chain_layers_sampled(env, li):
     torch, ubp = env
     L = ubp_synth.config_layers("mbv1_chain", batch=8 if li < 2 else 64)[li]
