@@ -75,7 +75,7 @@ def tf32_peak_tflops():
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (key: workload, tensor-core variant?)
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("mbv1_pw512", True): 15005696 + 0,          # profiles/ncu_ubp_tc_kernel_mbv1_pw512.md (the output is still in L2)
+    ("mbv1_pw512", True): 14976000 + 0,          # profiles/ncu_ubp_tc2_kernel_mbv1_pw512.md (the output is still in L2)
     ("sweep_nb4_p70", True): 135086848 + 37817856,   # profiles/ncu_ubp_tc_kernel_sweep_nb4_p70.md
     ("r50_3x3", True): 17635840 + 0,             # profiles/ncu_ubp_tc_kernel_r50_3x3.md
     ("sweep_nb4_p90", False): 70554368 + 23536640,   # profiles/ncu_ubp_spmm_kernel_sweep_nb4_p90.md
@@ -426,7 +426,10 @@ def main():
     roof["roofline_us"] = max(t_alu, t_hbm) * 1e6
     roof["frac_of_roofline_time"] = max(t_alu, t_hbm) / (step_ms * 1e-3)
     roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((name, plan.variant >= 30))
-    roof["kernel"] = "ubp_tc_kernel (dense 3xTF32 on tcgen05)" if plan.variant >= 30 else "ubp_spmm_kernel (sparse, FP32 FMA)"
+    kern, tile_rows, tile_cols = plan.tile_choice(L.Nc)
+    roof["kernel"] = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF32 on tcgen05, one CTA per tile)",
+                      "ubp_tc2_kernel (dense 3xTF32 on tcgen05, CTA pair per tile)")[kern]
+    roof["tile"] = [tile_rows, tile_cols]
     if plan.variant >= 30:
         # the tensor-core variant does 3 x the DENSE multiply-adds; report that rate against the TF32 peak too
         dense_tf = 3 * 2.0 * L.M * L.C * L.R * L.Nc / (step_ms * 1e-3) / 1e12

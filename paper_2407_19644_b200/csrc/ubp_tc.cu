@@ -345,25 +345,11 @@ int encode_3d(CUtensorMap *tm, const void *base, const uint64_t (&dims)[3], uint
 int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, const void *args, int M, int64_t Nc,
                    int ntile, void *stream);
 
-static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
+// Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
+// Each candidate's time is estimated as (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost)
+// and the cheapest kept.
+void tc_choose(int M, int K, int64_t Nc, int conv, int sms, int *kernel, int *rows, int *cols)
 {
-    const int M = pl->dims.M, K = a.K;
-    const int64_t Nc = a.Nc;
-    const uint8_t *dev = static_cast<const uint8_t *>(pl->dev);
-    const float *Wh = reinterpret_cast<const float *>(dev + pl->img.tc_off);
-    const float *Wl = Wh + (size_t)M * pl->img.tc_kp;
-    CUtensorMap tmWh, tmWl;
-    int rc;
-    if ((rc = encode_2d(&tmWh, Wh, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,
-                        CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
-    if ((rc = encode_2d(&tmWl, Wl, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,
-                        CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
-    a.M = M;
-    a.status = reinterpret_cast<int *>(pl->dev);
-    // Tile choice: 128 or 256 rows, 64..256 columns (multiples of 32). Estimate the time of each candidate as
-    // (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost) and keep the cheapest.
-    int sms = 148, devid = 0;
-    if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
     const int nchunk = (K + TC_KC - 1) / TC_KC;
     double best = 1e300;
     int best_mt = 1, best_n = TC_N;
@@ -383,11 +369,12 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
             const double t = (double)waves * (nchunk * per_chunk + 6000.0 + 40.0 * mt * n);
             if (t < best) { best = t; best_mt = mt; best_n = n; }
         }
+    *kernel = 1; *rows = 128 * best_mt; *cols = best_n;
     // Two-CTA kernel for the 1x1 product (256 rows per CTA pair; X goes from global memory into the operand layout
     // by TMA, each SM holds and reads only half of the X tile). Its chunk time is the MMA time (6 MMAs of n/2
     // cycles) or, for narrow tiles, what the issuing thread needs per chunk (~680 cycles measured); per tile
     // ~9000 cycles of pipeline fill and drain plus an epilogue ~ its outputs.
-    if (M > 128 && !a.conv) {
+    if (M > 128 && !conv) {
         double best2 = 1e300;
         int best2_n = 256;
         for (int n = 64; n <= 256; n += 64) {
@@ -398,30 +385,52 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
             const double t = (double)waves * (nchunk * per_chunk + 9000.0 + 30.0 * n);
             if (t < best2) { best2 = t; best2_n = n; }
         }
-        if (best2 < best) {
-            // Wh and Wl as one 3-D tensor (channel, row, part): one copy per chunk brings both
-            CUtensorMap tmW, tmX;
-            const uint64_t wdims[3] = {(uint64_t)pl->img.tc_kp, (uint64_t)M, 2};
-            const uint32_t wbox[3] = {TC_KC, 128, 2};
-            if ((rc = encode_3d(&tmW, Wh, wdims, (uint64_t)pl->img.tc_kp * 4, (uint64_t)M * pl->img.tc_kp * 4, wbox,
-                                CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
-            // X as (column in a group of 32, channel, group): one copy per chunk brings all of a CTA's columns in
-            // the operand layout. Needs whole groups; otherwise one 2-D copy per group.
-            const int x3d = (Nc % 32 == 0) ? 1 : 0;
-            if (x3d) {
-                const uint64_t xdims[3] = {32, (uint64_t)K, (uint64_t)(Nc / 32)};
-                const uint32_t xbox[3] = {32, TC_KC, (uint32_t)(best2_n / 64)};
-                rc = encode_3d(&tmX, a.X, xdims, (uint64_t)a.ldx * 4, 128, xbox, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
-            } else {
-                rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)K, (uint64_t)a.ldx * 4, 32, TC_KC,
-                               CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
-            }
-            if (rc) return rc;
-            return launch_tc_pair(&tmW, &tmX, x3d, &a, M, Nc, best2_n, stream);
-        }
+        if (best2 < best) { *kernel = 2; *rows = 256; *cols = best2_n; }
     }
+}
+
+static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
+{
+    const int M = pl->dims.M, K = a.K;
+    const int64_t Nc = a.Nc;
+    const uint8_t *dev = static_cast<const uint8_t *>(pl->dev);
+    const float *Wh = reinterpret_cast<const float *>(dev + pl->img.tc_off);
+    const float *Wl = Wh + (size_t)M * pl->img.tc_kp;
+    int rc;
+    a.M = M;
+    a.status = reinterpret_cast<int *>(pl->dev);
+    int sms = 148, devid = 0;
+    if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
+    int kernel, rows, best_n;
+    tc_choose(M, K, Nc, a.conv, sms, &kernel, &rows, &best_n);
+    if (kernel == 2) {
+        // Wh and Wl as one 3-D tensor (channel, row, part): one copy per chunk brings both
+        CUtensorMap tmW, tmX;
+        const uint64_t wdims[3] = {(uint64_t)pl->img.tc_kp, (uint64_t)M, 2};
+        const uint32_t wbox[3] = {TC_KC, 128, 2};
+        if ((rc = encode_3d(&tmW, Wh, wdims, (uint64_t)pl->img.tc_kp * 4, (uint64_t)M * pl->img.tc_kp * 4, wbox,
+                            CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
+        // X as (column in a group of 32, channel, group): one copy per chunk brings all of a CTA's columns in the
+        // operand layout. Needs whole groups; otherwise one 2-D copy per group.
+        const int x3d = (Nc % 32 == 0) ? 1 : 0;
+        if (x3d) {
+            const uint64_t xdims[3] = {32, (uint64_t)K, (uint64_t)(Nc / 32)};
+            const uint32_t xbox[3] = {32, TC_KC, (uint32_t)(best_n / 64)};
+            rc = encode_3d(&tmX, a.X, xdims, (uint64_t)a.ldx * 4, 128, xbox, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+        } else {
+            rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)K, (uint64_t)a.ldx * 4, 32, TC_KC,
+                           CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+        }
+        if (rc) return rc;
+        return launch_tc_pair(&tmW, &tmX, x3d, &a, M, Nc, best_n, stream);
+    }
+    CUtensorMap tmWh, tmWl;
+    if ((rc = encode_2d(&tmWh, Wh, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,
+                        CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
+    if ((rc = encode_2d(&tmWl, Wl, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,
+                        CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
     a.ntile = best_n;
-    const bool use2 = best_mt == 2;
+    const bool use2 = rows == 256;
     const unsigned ncols = (unsigned)((Nc + best_n - 1) / best_n);
     auto launch = [&](auto kern, int MT, size_t smem) -> int {
         static bool done[2][64] = {};

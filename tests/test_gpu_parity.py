@@ -260,6 +260,7 @@ def test_two_cta_kernel_padded_rows_and_repeated_launches(env):
     check(*run_spmm(env, L, 32, pad=4)[:3], L, tensor_core=True)
     L = ubp_synth.config_layers("mbv1_chain", batch=64)[4]          # 256 -> 256 channels at 28 x 28: 50176 columns
     plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb), 32)
+    assert plan.tile_choice(L.Nc)[0] == 2                            # the CTA-pair kernel is what runs here
     X = torch.from_numpy(L.X).cuda().reshape(L.C, -1)
     bias = torch.from_numpy(L.bias).cuda()
     flush = torch.empty(192 << 20, dtype=torch.uint8, device="cuda")
