@@ -22,6 +22,8 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "ubp_internal.h"
@@ -342,8 +344,8 @@ int encode_3d(CUtensorMap *tm, const void *base, const uint64_t (&dims)[3], uint
 
 
 // two-CTA kernel (ubp_tc2.cu)
-int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, const void *args, int M, int64_t Nc,
-                   int ntile, void *stream);
+int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, const CUtensorMap_st *tmY, int x3d,
+                   const void *args, int M, int64_t Nc, int ntile, int sms, void *stream);
 
 // Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
 // Each candidate's time is estimated as (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost)
@@ -371,18 +373,23 @@ void tc_choose(int M, int K, int64_t Nc, int conv, int sms, int *kernel, int *ro
         }
     *kernel = 1; *rows = 128 * best_mt; *cols = best_n;
     // Two-CTA kernel for the 1x1 product (256 rows per CTA pair; X goes from global memory into the operand layout
-    // by TMA, each SM holds and reads only half of the X tile). Its chunk time is the MMA time (6 MMAs of n/2
-    // cycles) or, for narrow tiles, what the issuing thread needs per chunk (~680 cycles measured); per tile
-    // ~9000 cycles of pipeline fill and drain plus an epilogue ~ its outputs.
+    // by TMA, each SM holds and reads only half of the X tile; persistent, the epilogue of a tile runs under the
+    // main loop of the next). Calibrated on forced tile widths: a chunk takes its MMA time (6 MMAs of n/2 cycles,
+    // ~10 % more in practice) or, for narrow tiles, what the copy / Xl / issue chain needs (~500 + n/2 cycles); a
+    // tile takes its chunks or, if longer, its epilogue on eight warps (~45 cycles per column); per launch ~4400
+    // cycles of pipeline fill and ~4500 + 30 per column of drain and last epilogue.
     if (M > 128 && !conv) {
         double best2 = 1e300;
         int best2_n = 256;
         for (int n = 64; n <= 256; n += 64) {
-            const long long ctas = 2ll * ((M + 255) / 256) * ((Nc + n - 1) / n);
-            const long long waves = (ctas + (sms & ~1) - 1) / (sms & ~1);
-            double per_chunk = 3.0 * (TC_KC / 8) * (n / 2.0);
-            if (per_chunk < 680.0) per_chunk = 680.0;
-            const double t = (double)waves * (nchunk * per_chunk + 9000.0 + 30.0 * n);
+            const long long ntiles = (long long)((M + 255) / 256) * ((Nc + n - 1) / n);
+            const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
+            const long long per_pair = (ntiles + pairs - 1) / pairs;
+            double per_chunk = 3.3 * n;
+            if (per_chunk < 500.0 + 0.5 * n) per_chunk = 500.0 + 0.5 * n;
+            double per_tile = nchunk * per_chunk;
+            if (per_tile < 45.0 * n) per_tile = 45.0 * n;
+            const double t = 4400.0 + (double)per_pair * per_tile + 4500.0 + 30.0 * n;
             if (t < best2) { best2 = t; best2_n = n; }
         }
         if (best2 < best) { *kernel = 2; *rows = 256; *cols = best2_n; }
@@ -403,6 +410,9 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
     if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
     int kernel, rows, best_n;
     tc_choose(M, K, Nc, a.conv, sms, &kernel, &rows, &best_n);
+#ifdef UBP_TC_TUNE   // diagnostic builds only: force the kernel and tile width from the environment
+    if (const char *e = getenv("UBP_TC_FORCE")) { int k = 0, n = 0; if (sscanf(e, "%d,%d", &k, &n) == 2) { kernel = k; best_n = n; rows = (k == 2 || k == 12) ? 256 : 128; if (k == 12) kernel = 1; } }
+#endif
     if (kernel == 2) {
         // Wh and Wl as one 3-D tensor (channel, row, part): one copy per chunk brings both
         CUtensorMap tmW, tmX;
@@ -422,7 +432,14 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
                            CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
         }
         if (rc) return rc;
-        return launch_tc_pair(&tmW, &tmX, x3d, &a, M, Nc, best_n, stream);
+        // the output as (column, row): the epilogue stores 32 x 32 boxes and TMA clips the ragged edges, in units of
+        // 16 bytes along a row: the map covers whole groups of four columns (a last ragged group is stored by the
+        // kernel's threads)
+        CUtensorMap tmY;
+        const uint64_t ycols = Nc >= 4 ? (uint64_t)(Nc & ~(int64_t)3) : 4;   // (fewer than 4 columns: ldy >= 4 holds, nothing is stored through the map)
+        if ((rc = encode_2d(&tmY, a.Y, ycols, (uint64_t)M, (uint64_t)a.ldy * 4, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B)))
+            return rc;
+        return launch_tc_pair(&tmW, &tmX, &tmY, x3d, &a, M, Nc, best_n, sms, stream);
     }
     CUtensorMap tmWh, tmWl;
     if ((rc = encode_2d(&tmWh, Wh, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,
