@@ -75,8 +75,8 @@ def tf32_peak_tflops():
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (key: workload, tensor-core variant?)
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("mbv1_pw512", True): 14976000 + 0,          # profiles/ncu_ubp_tc2_kernel_mbv1_pw512.md (the output is still in L2)
-    ("sweep_nb4_p70", True): 135086848 + 37817856,   # profiles/ncu_ubp_tc_kernel_sweep_nb4_p70.md
+    ("mbv1_pw512", True): 14984448 + 256,        # profiles/ncu_ubp_tc2_kernel_mbv1_pw512.md (the output is still in L2)
+    ("sweep_nb4_p70", True): 124626432 + 48126208,   # profiles/ncu_ubp_tc2_kernel_sweep_nb4_p70.md
     ("r50_3x3", True): 17635840 + 0,             # profiles/ncu_ubp_tc_kernel_r50_3x3.md
     ("sweep_nb4_p90", False): 70554368 + 23536640,   # profiles/ncu_ubp_spmm_kernel_sweep_nb4_p90.md
 }

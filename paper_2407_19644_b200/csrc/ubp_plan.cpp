@@ -64,8 +64,10 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     if (R != 1) return nullptr;
     // Dense tensor-core variant when enough of the weight survives and the layer is large enough to amortise its
     // per-tile set-up: measured on B200 it takes the same time at every sparsity and beats the sparse kernel up to
-    // ~90 % sparsity on 2048 x 2048 x 8192; with 128 input channels or fewer the sparse kernel is as fast or faster.
-    if (dens >= 0.08 && M >= 128 && C >= 256) {
+    // ~90 % sparsity on 2048 x 2048 x 8192. With more than 128 rows the CTA-pair kernel runs, which pays from 128
+    // input channels on; with exactly 128 rows (one CTA per tile) from 256 on; below that the sparse kernel is as
+    // fast or faster.
+    if (dens >= 0.08 && ((M > 128 && C >= 128) || (M >= 128 && C >= 256))) {
         switch (nbk) {
             case 16: case 8: return find_cfg(33);
             case 4: return find_cfg(32);

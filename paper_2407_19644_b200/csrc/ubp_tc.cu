@@ -344,8 +344,8 @@ int encode_3d(CUtensorMap *tm, const void *base, const uint64_t (&dims)[3], uint
 
 
 // two-CTA kernel (ubp_tc2.cu)
-int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, const CUtensorMap_st *tmY, int x3d,
-                   const void *args, int M, int64_t Nc, int ntile, int sms, void *stream);
+int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, const void *args, int M, int64_t Nc,
+                   int ntile, int sms, void *stream);
 
 // Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
 // Each candidate's time is estimated as (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost)
@@ -375,9 +375,10 @@ void tc_choose(int M, int K, int64_t Nc, int conv, int sms, int *kernel, int *ro
     // Two-CTA kernel for the 1x1 product (256 rows per CTA pair; X goes from global memory into the operand layout
     // by TMA, each SM holds and reads only half of the X tile; persistent, the epilogue of a tile runs under the
     // main loop of the next). Calibrated on forced tile widths: a chunk takes its MMA time (6 MMAs of n/2 cycles,
-    // ~10 % more in practice) or, for narrow tiles, what the copy / Xl / issue chain needs (~500 + n/2 cycles); a
-    // tile takes its chunks or, if longer, its epilogue on eight warps (~45 cycles per column); per launch ~4400
-    // cycles of pipeline fill and ~4500 + 30 per column of drain and last epilogue.
+    // ~10 % more in practice) or, for narrow tiles, the time shared memory needs for it (MMA operand reads 24 KB of
+    // W + 96 B per column, copies 16 KB + 32 B per column, Xl pass 64 B per column, at ~120 B/cycle: ~500 + n/2
+    // cycles); a tile takes its chunks or, if longer, its epilogue on eight warps (~45 cycles per column); per
+    // launch ~4400 cycles of pipeline fill and ~4500 + 30 per column of drain and last epilogue.
     if (M > 128 && !conv) {
         double best2 = 1e300;
         int best2_n = 256;
@@ -432,14 +433,7 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
                            CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
         }
         if (rc) return rc;
-        // the output as (column, row): the epilogue stores 32 x 32 boxes and TMA clips the ragged edges, in units of
-        // 16 bytes along a row: the map covers whole groups of four columns (a last ragged group is stored by the
-        // kernel's threads)
-        CUtensorMap tmY;
-        const uint64_t ycols = Nc >= 4 ? (uint64_t)(Nc & ~(int64_t)3) : 4;   // (fewer than 4 columns: ldy >= 4 holds, nothing is stored through the map)
-        if ((rc = encode_2d(&tmY, a.Y, ycols, (uint64_t)M, (uint64_t)a.ldy * 4, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B)))
-            return rc;
-        return launch_tc_pair(&tmW, &tmX, &tmY, x3d, &a, M, Nc, best_n, sms, stream);
+        return launch_tc_pair(&tmW, &tmX, x3d, &a, M, Nc, best_n, sms, stream);
     }
     CUtensorMap tmWh, tmWl;
     if ((rc = encode_2d(&tmWh, Wh, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,

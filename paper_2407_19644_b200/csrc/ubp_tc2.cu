@@ -51,9 +51,7 @@ constexpr int T2_THREADS = (2 + T2_XL_WARPS + T2_EPI_WARPS) * 32;
 constexpr int T2_MAX_STAGES = 8;                          // pipeline stages: as many as fit, at most this
 constexpr uint32_t T2_A_HALF = 128 * TC_KC * 4;           // Wh or Wl chunk of this CTA's 128 rows: 8 KB
 constexpr uint32_t T2_XG = 32 * TC_KC * 4;                // one box of X: 16 channels x 32 columns, 2 KB
-constexpr int T2_PITCH = 32;                              // floats per row of an epilogue staging tile (XOR-swizzled)
-constexpr uint32_t T2_STAGING = T2_EPI_WARPS * 32 * T2_PITCH * 4;      // the epilogue warps' staging tiles: 32 KB
-constexpr uint32_t T2_PIPE_BUDGET = 192 * 1024;           // pipeline stages together
+constexpr uint32_t T2_PIPE_BUDGET = 222 * 1024;           // pipeline stages together
 // a stage = Wh + Wl chunk (16 KB) + raw X + Xl of `ngrp` 32-column boxes (2 KB each): 20 .. 32 KB, 8 or 6 stages.
 // The count is a multiple of T2_XL_GROUPS so that a stage always belongs to the same group of Xl warps: a waiter
 // must see every phase of a barrier it waits on (a parity wait cannot tell phase k from phase k + 2).
@@ -137,26 +135,37 @@ __device__ __forceinline__ bool mma2_chunk(uint32_t d_tmem, uint64_t dWh, uint64
     return ready != 0;
 }
 
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+
 // Epilogue of 32 rows (tensor-memory lane quarter q of accumulator `acc`) x the 32-column blocks first, first + step,
-// ... of one CTA's 128 x N part of a tile: tensor memory -> registers (lane = row: bias, ReLU) -> a 32 x 32 staging
-// tile in shared memory (128-byte rows whose 16-byte pieces are XOR-swizzled with the row number: conflict-free to
-// write, and exactly TMA's 128-byte swizzle) -> global memory by a TMA store, which also clips the ragged last
-// rows and columns. The next block's tensor-memory read is in flight while TMA drains the staging tile.
+// ... of one CTA's 128 x N part of a tile, without shared memory (the MMA operands and the copies already use all
+// of its bandwidth). The accumulator is read in the 16 x 256-bit shape: lane t gets, per group j of 8 columns,
+// the column pair 8j + 2(t mod 4) of rows t/4 and t/4 + 8 of a 16-row half. Four lanes therefore hold 32
+// consecutive bytes of an output row, and every 8-byte store instruction of the warp writes eight whole 32-byte
+// sectors; bias and ReLU are applied in registers.
 // `done_bar` != 0: once this warp's last tensor-memory read has completed, lane 0 arrives on that barrier of the
 // leader CTA (the accumulator may be overwritten from then on).
-__device__ __forceinline__ void epilogue_blocks(const TcArgs &a, const CUtensorMap *tmY, uint32_t acc, int q, int first,
-                                                int step, int N, float *tile_s, int row0, int64_t col0, int lane,
-                                                uint32_t done_bar, uint32_t rank, bool &stored)
+__device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, int q, int first, int step, int N,
+                                                int row0, int64_t col0, int lane, uint32_t done_bar, uint32_t rank)
 {
-    const int rbase = row0 + q * 32;
+    const int rbase = row0 + q * 32 + (lane >> 2);          // this lane's rows: rbase + {0, 8, 16, 24}
     const int nblk = N / 32;
-    const int row = rbase + lane;
-    const float bias = (a.bias && row < a.M) ? __ldg(a.bias + row) : 0.f;
-    const uint32_t tile_u = smem_u32(tile_s);
+    float bias[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) bias[i] = (a.bias && rbase + 8 * i < a.M) ? __ldg(a.bias + rbase + 8 * i) : 0.f;
 #pragma unroll 1
     for (int cc = first; cc < nblk; cc += step) {
-        uint32_t r[32];
-        tmem_ld32(acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), r);
+        uint32_t r[2][16];
+        tmem_ld_16x256b_x4(acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), r[0]);
+        tmem_ld_16x256b_x4(acc + ((uint32_t)(q * 32 + 16) << 16) + (uint32_t)(cc * 32), r[1]);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (done_bar && cc + step >= nblk) {
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -165,35 +174,25 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, const CUtensorM
                 else mbar_arrive_remote(done_bar, 0);
             }
         }
-        const int64_t cb = col0 + cc * 32;
-        if (cb >= a.Nc || rbase >= a.M) continue;           // a block entirely outside the output
-        // TMA clips in 16-byte units, so the output map ends at the last whole group of four columns; a ragged
-        // last group is stored from the registers below
-        const bool by_tma = cb < (a.Nc & ~(int64_t)3);
-        if (by_tma && stored) {                             // the previous store must have read the staging tile
-            if (lane == 0) tma_store_wait_read();
-            __syncwarp();
-        }
+        const int64_t cb = col0 + cc * 32 + 2 * (lane & 3);
 #pragma unroll
-        for (int v = 0; v < 8; ++v) {
-            float4 o = make_float4(__uint_as_float(r[4 * v]) + bias, __uint_as_float(r[4 * v + 1]) + bias,
-                                   __uint_as_float(r[4 * v + 2]) + bias, __uint_as_float(r[4 * v + 3]) + bias);
-            if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
-            if (by_tma) *reinterpret_cast<float4 *>(tile_s + lane * T2_PITCH + 4 * (v ^ (lane & 7))) = o;
-            const int64_t colv = cb + 4 * v;
-            if (colv < a.Nc && colv + 4 > a.Nc && row < a.M) {
-                float *y = a.Y + (size_t)row * a.ldy + colv;
-                y[0] = o.x;
-                if (colv + 1 < a.Nc) y[1] = o.y;
-                if (colv + 2 < a.Nc) y[2] = o.z;
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int row = rbase + 16 * half + 8 * h;
+                if (row >= a.M) continue;
+                float *yrow = a.Y + (size_t)row * a.ldy;
+                const float b = bias[2 * half + h];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float2 o = make_float2(__uint_as_float(r[half][4 * j + 2 * h]) + b,
+                                           __uint_as_float(r[half][4 * j + 2 * h + 1]) + b);
+                    if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); }
+                    const int64_t col = cb + 8 * j;
+                    if (col + 1 < a.Nc) *reinterpret_cast<float2 *>(yrow + col) = o;
+                    else if (col < a.Nc) yrow[col] = o.x;
+                }
             }
-        }
-        if (by_tma) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the tile visible to the TMA unit
-            __syncwarp();
-            if (lane == 0) tma_store_2d(tmY, tile_u, (int)cb, rbase);
-            stored = true;
-        }
     }
     // a warp with no block of its own still owes its arrival
     if (done_bar && first >= nblk) {
@@ -205,8 +204,8 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, const CUtensorM
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T2_THREADS, 1)
-ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-               const __grid_constant__ CUtensorMap tmY, const TcArgs a, const int x3d, const int nrp, const int ntiles)
+ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const TcArgs a,
+               const int x3d, const int nrp, const int ntiles)
 {
     constexpr int MAXS = T2_MAX_STAGES;
     constexpr uint32_t TMEM_COLS = 2 * T2_ACC_COLS;
@@ -252,7 +251,6 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (threadIdx.x == 0) {
         prefetch_tensormap(&tmW);
         prefetch_tensormap(&tmX);
-        prefetch_tensormap(&tmY);
         abort_flag = 0;
         for (int s = 0; s < S; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
@@ -376,28 +374,21 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (ok && nmy > 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int i = nmy - 1;
-            // every MMA and every copy of this CTA is done, so the pipeline stages serve as staging tiles
-            float *tile_s = reinterpret_cast<float *>(smem) + (warp - 2) * 32 * T2_PITCH;
-            bool stored = false;
-            epilogue_blocks(a, &tmY, tmem_base + (uint32_t)(i & 1) * T2_ACC_COLS, warp & 3, 2 + ((warp - 2) >> 2), 4, N,
-                            tile_s, tile_row0(i), tile_col0(i), lane, 0u, rank, stored);
-            if (stored && lane == 0) tma_store_wait_all();
+            epilogue_blocks(a, tmem_base + (uint32_t)(i & 1) * T2_ACC_COLS, warp & 3, 2 + ((warp - 2) >> 2), 4, N,
+                            tile_row0(i), tile_col0(i), lane, 0u, rank);
         }
     } else {
         // ---------------- epilogue warps: tile i's accumulator while the main loop works on tile i + 1
-        float *tile_s = reinterpret_cast<float *>(smem + (size_t)S * stage_bytes) + (warp - 2 - T2_XL_WARPS) * 32 * T2_PITCH;
         const int part = (warp - 2 - T2_XL_WARPS) >> 2;       // two warps share a lane quarter and split the columns
-        bool stored = false;
         for (int i = 0; i < nmy && ok; ++i) {
             const int b = i & 1;
             ok = mbar_wait_relaxed(smem_u32(&bar_acc_full[b]), (uint32_t)(i >> 1) & 1u, &abort_flag);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const bool last = i == nmy - 1;
-            epilogue_blocks(a, &tmY, tmem_base + (uint32_t)b * T2_ACC_COLS, warp & 3, part, last ? 4 : 2, N, tile_s,
-                            tile_row0(i), tile_col0(i), lane, last ? 0u : smem_u32(&bar_acc_empty[b]), rank, stored);
+            epilogue_blocks(a, tmem_base + (uint32_t)b * T2_ACC_COLS, warp & 3, part, last ? 4 : 2, N, tile_row0(i),
+                            tile_col0(i), lane, last ? 0u : smem_u32(&bar_acc_empty[b]), rank);
         }
-        if (stored && lane == 0) tma_store_wait_all();     // every store of this warp has reached global memory
     }
     if (!ok && lane == 0) atomicExch(a.status, 1);
     // every thread of both CTAs comes here: neither CTA may free tensor memory or leave while the other could
@@ -418,21 +409,19 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 // tmW: 3-D map over the plan's dense part (channel, row, {Wh, Wl}), box 16 x 128 x 2, 64-byte swizzle.
 // tmX: 128-byte swizzle with 32-byte atoms; x3d != 0: 3-D map (column in group, channel, 32-column group) with box
 // 32 x 16 x ntile/64; x3d == 0: 2-D map (column, channel) with box 32 x 16.
-// tmY: 2-D map over the output (column, row) up to the last whole group of four columns, box 32 x 32, 128-byte
-// swizzle.
-int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, const CUtensorMap_st *tmY, int x3d,
-                   const void *args_, int M, int64_t Nc, int ntile, int sms, void *stream)
+int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, const void *args_, int M, int64_t Nc,
+                   int ntile, int sms, void *stream)
 {
     TcArgs a = *static_cast<const TcArgs *>(args_);
     a.ntile = ntile;
     const int ngrp = ntile / 64;
-    const size_t smem = (size_t)t2_stages(ngrp) * (2 * T2_A_HALF + 2 * (size_t)ngrp * T2_XG) + T2_STAGING + 1024;
+    const size_t smem = (size_t)t2_stages(ngrp) * (2 * T2_A_HALF + 2 * (size_t)ngrp * T2_XG) + 1024;
     static bool done[64] = {};
     int devid = 0;
     if (cudaGetDevice(&devid) != cudaSuccess) devid = -1;
     if (devid < 0 || devid >= 64 || !done[devid]) {
         cudaError_t e = cudaFuncSetAttribute(ubp_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(T2_PIPE_BUDGET + T2_STAGING + 1024));
+                                             (int)(T2_PIPE_BUDGET + 1024));
         if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
         if (devid >= 0 && devid < 64) done[devid] = true;
     }
@@ -442,7 +431,7 @@ int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, const C
     if (ntiles > 0x7fffffffll) return UBP_E_UNSUPPORTED;
     const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
     ubp_tc2_kernel<<<dim3((unsigned)(2 * pairs)), T2_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(
-        *tmW, *tmX, *tmY, a, x3d, nrp, (int)ntiles);
+        *tmW, *tmX, a, x3d, nrp, (int)ntiles);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
     return UBP_OK;
