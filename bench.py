@@ -426,7 +426,7 @@ def main():
     roof["roofline_us"] = max(t_alu, t_hbm) * 1e6
     roof["frac_of_roofline_time"] = max(t_alu, t_hbm) / (step_ms * 1e-3)
     roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((name, plan.variant >= 30))
-    kern, tile_rows, tile_cols = plan.tile_choice(L.Nc)
+    kern, tile_rows, tile_cols = plan.tile_choice(L.Nc, L.Wd if L.R == 9 else 0)
     roof["kernel"] = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF32 on tcgen05, one CTA per tile)",
                       "ubp_tc2_kernel (dense 3xTF32 on tcgen05, CTA pair per tile)")[kern]
     roof["tile"] = [tile_rows, tile_cols]

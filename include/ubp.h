@@ -134,11 +134,13 @@ typedef struct {
 int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info);
 
 /* ubp_plan_tile_choice: which kernel a launch of this plan over `Nc` columns uses on the current device when the
- * operands qualify for the fast path, and its output tile. *kernel: 0 = sparse FP32 kernel (Section 4.2's
- * output-stationary product on the CUDA cores), 1 = tensor-core kernel with one CTA per tile, 2 = tensor-core
- * kernel with a CTA pair per tile (1x1 only). Host only; enqueues nothing. Not part of the paper's method: it
- * exists so that measurements and tests can name what ran. */
-int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int *kernel, int *tile_rows, int *tile_cols);
+ * operands qualify for the fast path (for 3x3: input and output as one [channel][batch, y, x] matrix each), and
+ * its output tile. `image_width` is the width of the input planes for a 3x3 plan (Nc = batch * height * width),
+ * ignored for 1x1. *kernel: 0 = sparse FP32 kernel (Section 4.2's output-stationary product on the CUDA cores),
+ * 1 = tensor-core kernel with one CTA per tile, 2 = tensor-core kernel with a CTA pair per tile. Host only;
+ * enqueues nothing. Not part of the paper's method: it exists so that measurements and tests can name what ran. */
+int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, int *kernel, int *tile_rows,
+                         int *tile_cols);
 
 /* Read the plan's device status word: blocks until `stream` has finished
  * (cudaStreamSynchronize), then returns UBP_OK or UBP_E_DEVICE if a kernel

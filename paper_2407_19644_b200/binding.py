@@ -60,7 +60,7 @@ def load():
     L.ubp_plan_free.restype = None
     L.ubp_plan_info.argtypes = [vp, C.POINTER(_PlanInfo)]
     L.ubp_plan_check.argtypes = [vp, vp]
-    L.ubp_plan_tile_choice.argtypes = [vp, i64, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+    L.ubp_plan_tile_choice.argtypes = [vp, i64, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
     L.ubp_spmm.argtypes = [vp, vp, i64, i64, vp, i32, vp, i64, vp]
     L.ubp_conv1x1.argtypes = [vp, vp, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
     L.ubp_conv3x3_implicit.argtypes = [vp, vp, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
@@ -216,13 +216,14 @@ class Plan:
         """Synchronise the stream and raise if a kernel reported a failed bounded wait."""
         _chk(self._lib.ubp_plan_check(self.handle, _stream_ptr(stream)), "ubp_plan_check")
 
-    def tile_choice(self, Nc: int):
-        """(kernel, tile_rows, tile_cols) of a fast-path launch over Nc columns on the plan's device:
-        kernel 0 = sparse FP32, 1 = tensor core / one CTA per tile, 2 = tensor core / CTA pair per tile."""
+    def tile_choice(self, Nc: int, image_width: int = 0):
+        """(kernel, tile_rows, tile_cols) of a fast-path launch over Nc columns on the plan's device (3x3 plans:
+        Nc = batch * height * width and image_width = width): kernel 0 = sparse FP32, 1 = tensor core / one CTA
+        per tile, 2 = tensor core / CTA pair per tile."""
         k, r, c = C.c_int32(), C.c_int32(), C.c_int32()
         import torch
         with torch.cuda.device(self.buffer.device):
-            _chk(self._lib.ubp_plan_tile_choice(self.handle, int(Nc), C.byref(k), C.byref(r), C.byref(c)),
+            _chk(self._lib.ubp_plan_tile_choice(self.handle, int(Nc), int(image_width), C.byref(k), C.byref(r), C.byref(c)),
                  "ubp_plan_tile_choice")
         return k.value, r.value, c.value
 

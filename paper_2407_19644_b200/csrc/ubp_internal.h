@@ -71,8 +71,9 @@ struct ubp_plan {
 namespace ubp {
 int launch_spmm(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                 float *Y, int64_t ldy, void *stream);
-// tensor-core tile choice for a launch over Nc columns: kernel 1 = one CTA per tile, 2 = CTA pair per tile
-void tc_choose(int M, int K, int64_t Nc, int conv, int sms, int *kernel, int *rows, int *cols);
+// tensor-core tile choice for a launch over Nc columns: kernel 1 = one CTA per tile, 2 = CTA pair per tile;
+// conv_w = 0: 1x1; > 0: 3x3 on images conv_w pixels wide (operands fit the pair kernel); < 0: 3x3, one CTA only
+void tc_choose(int M, int K, int64_t Nc, int conv_w, int sms, int *kernel, int *rows, int *cols);
 int launch_spmm_tc(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                    float *Y, int64_t ldy, void *stream);
 int launch_conv3x3_tc(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,

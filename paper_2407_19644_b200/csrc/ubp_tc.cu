@@ -344,14 +344,18 @@ int encode_3d(CUtensorMap *tm, const void *base, const uint64_t (&dims)[3], uint
 
 
 // two-CTA kernel (ubp_tc2.cu)
-int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, const void *args, int M, int64_t Nc,
-                   int ntile, int sms, void *stream);
+int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, int halo, const void *args, int M,
+                   int64_t Nc, int ntile, int sms, void *stream);
+int tc_pair_stages(int ntile, int halo);
 
 // Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
 // Each candidate's time is estimated as (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost)
 // and the cheapest kept.
-void tc_choose(int M, int K, int64_t Nc, int conv, int sms, int *kernel, int *rows, int *cols)
+// conv_w: 0 = 1x1 product; > 0 = 3x3 on images `conv_w` pixels wide whose operands the pair kernel can take;
+// < 0 = 3x3, one-CTA kernel only.
+void tc_choose(int M, int K, int64_t Nc, int conv_w, int sms, int *kernel, int *rows, int *cols)
 {
+    const int conv = conv_w != 0;
     const int nchunk = (K + TC_KC - 1) / TC_KC;
     double best = 1e300;
     int best_mt = 1, best_n = TC_N;
@@ -379,21 +383,26 @@ void tc_choose(int M, int K, int64_t Nc, int conv, int sms, int *kernel, int *ro
     // W + 96 B per column, copies 16 KB + 32 B per column, Xl pass 64 B per column, at ~120 B/cycle: ~500 + n/2
     // cycles); a tile takes its chunks or, if longer, its epilogue on eight warps (~45 cycles per column); per
     // launch ~4400 cycles of pipeline fill and ~4500 + 30 per column of drain and last epilogue.
-    if (M > 128 && !conv) {
+    // 3x3: the shifted tiles are cut from a raw copy with a halo of image width + 1 columns either side, which
+    // adds shared-memory traffic (~560 + 0.75 n cycles per chunk) and leaves fewer stages.
+    const int halo = conv_w > 0 ? (conv_w + 1 + 3) & ~3 : 0;
+    if (M > 128 && conv_w >= 0 && (!conv || ((K / 9) % TC_KC == 0 && halo <= 64))) {
         double best2 = 1e300;
-        int best2_n = 256;
+        int best2_n = 0;
         for (int n = 64; n <= 256; n += 64) {
+            if (conv && (n / 2 + 2 * halo > 256 || tc_pair_stages(n, halo) < 4)) continue;
             const long long ntiles = (long long)((M + 255) / 256) * ((Nc + n - 1) / n);
             const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
             const long long per_pair = (ntiles + pairs - 1) / pairs;
             double per_chunk = 3.3 * n;
-            if (per_chunk < 500.0 + 0.5 * n) per_chunk = 500.0 + 0.5 * n;
+            const double smem_chunk = conv ? 560.0 + 0.75 * n : 500.0 + 0.5 * n;
+            if (per_chunk < smem_chunk) per_chunk = smem_chunk;
             double per_tile = nchunk * per_chunk;
             if (per_tile < 45.0 * n) per_tile = 45.0 * n;
             const double t = 4400.0 + (double)per_pair * per_tile + 4500.0 + 30.0 * n;
             if (t < best2) { best2 = t; best2_n = n; }
         }
-        if (best2 < best) { *kernel = 2; *rows = 256; *cols = best2_n; }
+        if (best2_n && best2 < best) { *kernel = 2; *rows = 256; *cols = best2_n; }
     }
 }
 
@@ -410,7 +419,10 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
     int sms = 148, devid = 0;
     if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
     int kernel, rows, best_n;
-    tc_choose(M, K, Nc, a.conv, sms, &kernel, &rows, &best_n);
+    // 3x3 on CTA pairs needs the input as one [channel][b, y, x] matrix with 16-byte aligned rows
+    const bool conv_pair_ok = a.conv && a.isb == (int64_t)a.H * a.W && a.isc % 4 == 0 &&
+                              (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && a.isc >= Nc;
+    tc_choose(M, K, Nc, a.conv ? (conv_pair_ok ? a.W : -1) : 0, sms, &kernel, &rows, &best_n);
 #ifdef UBP_TC_TUNE   // diagnostic builds only: force the kernel and tile width from the environment
     if (const char *e = getenv("UBP_TC_FORCE")) { int k = 0, n = 0; if (sscanf(e, "%d,%d", &k, &n) == 2) { kernel = k; best_n = n; rows = (k == 2 || k == 12) ? 256 : 128; if (k == 12) kernel = 1; } }
 #endif
@@ -423,8 +435,12 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
                             CU_TENSOR_MAP_SWIZZLE_64B))) return rc;
         // X as (column in a group of 32, channel, group): one copy per chunk brings all of a CTA's columns in the
         // operand layout. Needs whole groups; otherwise one 2-D copy per group.
-        const int x3d = (Nc % 32 == 0) ? 1 : 0;
-        if (x3d) {
+        const int x3d = (!a.conv && Nc % 32 == 0) ? 1 : 0;
+        const int halo = a.conv ? (a.W + 1 + 3) & ~3 : 0;
+        if (a.conv) {
+            rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)(K / 9), (uint64_t)a.isc * 4, (uint32_t)(best_n / 2 + 2 * halo),
+                           TC_KC, CU_TENSOR_MAP_SWIZZLE_NONE);
+        } else if (x3d) {
             const uint64_t xdims[3] = {32, (uint64_t)K, (uint64_t)(Nc / 32)};
             const uint32_t xbox[3] = {32, TC_KC, (uint32_t)(best_n / 64)};
             rc = encode_3d(&tmX, a.X, xdims, (uint64_t)a.ldx * 4, 128, xbox, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
@@ -433,7 +449,7 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
                            CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
         }
         if (rc) return rc;
-        return launch_tc_pair(&tmW, &tmX, x3d, &a, M, Nc, best_n, sms, stream);
+        return launch_tc_pair(&tmW, &tmX, x3d, halo, &a, M, Nc, best_n, sms, stream);
     }
     CUtensorMap tmWh, tmWl;
     if ((rc = encode_2d(&tmWh, Wh, (uint64_t)pl->img.tc_kp, (uint64_t)M, (uint64_t)pl->img.tc_kp * 4, TC_KC, 128,

@@ -55,9 +55,19 @@ constexpr uint32_t T2_PIPE_BUDGET = 222 * 1024;           // pipeline stages tog
 // a stage = Wh + Wl chunk (16 KB) + raw X + Xl of `ngrp` 32-column boxes (2 KB each): 20 .. 32 KB, 8 or 6 stages.
 // The count is a multiple of T2_XL_GROUPS so that a stage always belongs to the same group of Xl warps: a waiter
 // must see every phase of a barrier it waits on (a parity wait cannot tell phase k from phase k + 2).
-__host__ __device__ constexpr int t2_stages(int ngrp)
+// For 3x3 a stage also holds the raw copy the shifted tiles are cut from: 16 channels x (columns + 2 x halo) floats,
+// halo = image width + 1 rounded up to a multiple of 4 (0 for 1x1), padded to a multiple of 1 KB.
+__host__ __device__ constexpr uint32_t t2_raw_bytes(int ngrp, int halo)
 {
-    const int s = (int)(T2_PIPE_BUDGET / (2 * T2_A_HALF + 2 * (uint32_t)ngrp * T2_XG));
+    return halo ? (((uint32_t)(ngrp * 32 + 2 * halo) * TC_KC * 4 + 1023u) & ~1023u) : 0u;
+}
+__host__ __device__ constexpr uint32_t t2_stage_bytes(int ngrp, int halo)
+{
+    return 2 * T2_A_HALF + 2 * (uint32_t)ngrp * T2_XG + t2_raw_bytes(ngrp, halo);
+}
+__host__ __device__ constexpr int t2_stages(int ngrp, int halo)
+{
+    const int s = (int)(T2_PIPE_BUDGET / t2_stage_bytes(ngrp, halo));
     return (s > T2_MAX_STAGES ? T2_MAX_STAGES : s) / T2_XL_GROUPS * T2_XL_GROUPS;
 }
 constexpr uint32_t SWZ_128B_ATOM32 = 1;                   // descriptor layout type: 128-byte swizzle, 32-byte atoms
@@ -203,9 +213,10 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
     }
 }
 
+template <bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T2_THREADS, 1)
 ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const TcArgs a,
-               const int x3d, const int nrp, const int ntiles)
+               const int xmode, const int nrp, const int ntiles)
 {
     constexpr int MAXS = T2_MAX_STAGES;
     constexpr uint32_t TMEM_COLS = 2 * T2_ACC_COLS;
@@ -222,11 +233,15 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const uint32_t rank = cluster_rank();
     const int N = a.ntile, NH = N / 2;                     // tile columns; columns whose X this CTA holds
     const int ngrp = NH / 32;                              // 32-column boxes per chunk in this CTA
-    const uint32_t x_bytes = (uint32_t)ngrp * T2_XG;       // raw X (and Xl) bytes per stage
-    const uint32_t stage_bytes = 2 * T2_A_HALF + 2 * x_bytes;
-    const int S = t2_stages(ngrp);
+    const uint32_t x_bytes = (uint32_t)ngrp * T2_XG;       // Xh (1x1: the raw X tile) and Xl bytes per stage
+    const int x3d = CONV ? 0 : xmode;                      // 1x1: X copied by one 3-D box per chunk
+    const int halo = CONV ? xmode : 0;                     // 3x3: columns copied beyond either end of the tile
+    const uint32_t stage_bytes = t2_stage_bytes(ngrp, halo);
+    const uint32_t raw_row = (uint32_t)(NH + 2 * halo) * 4;                   // 3x3: the copy the shifted tiles are cut from
+    const int S = t2_stages(ngrp, halo);
     const int nchunk = (a.K + TC_KC - 1) / TC_KC;
-    const uint32_t tx = 2 * T2_A_HALF + x_bytes;
+    const uint32_t tx = 2 * T2_A_HALF + (CONV ? raw_row * TC_KC : x_bytes);
+    const int Cin = CONV ? a.K / 9 : a.K;                  // 3x3: reduction index k = tap * Cin + channel, Cin % 16 == 0
     // this pair's tiles: pair, pair + npairs, ...; tile t = (row pair t % nrp, column tile t / nrp)
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
     const int nmy = pair < ntiles ? (ntiles - pair + npairs - 1) / npairs : 0;
@@ -240,7 +255,12 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const uint32_t bar = smem_u32(&bar_full[st]);
         mbar_expect_tx(bar, tx);
         tma_load_3d(smem_u32(stage), &tmW, c * TC_KC, row0, 0, bar);
-        if (x3d) {
+        if (CONV) {
+            // 16 channels of the chunk's tap, columns xcol - halo .. xcol + NH + halo - 1 of the flattened (b, y, x)
+            // axis: every tap's shift dy * W + dx (at most W + 1 <= halo either way) lies inside
+            const int ch0 = (c * TC_KC) % Cin;
+            tma_load_2d(smem_u32(stage + 2 * T2_A_HALF + 2 * x_bytes), &tmX, xcol - halo, ch0, bar);
+        } else if (x3d) {
             tma_load_3d(smem_u32(stage + 2 * T2_A_HALF), &tmX, 0, c * TC_KC, xcol >> 5, bar);
         } else {
             for (int g = 0; g < ngrp; ++g)
@@ -346,10 +366,67 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int total = nmy * nchunk;
         int st = grp;                                      // the stage count is even: stages grp, grp + 2, ...
         uint32_t ph = 0;
+        const int cg = lane, cw = (gt >> 5);               // 3x3: column group and first channel of this thread
+        unsigned long long tap_ok = 0;                     // 3x3: bit tap * 4 + e: tap inside the image for column 4 cg + e
+        int mask_tile = -1;
         for (int f = grp; f < total && ok; f += T2_XL_GROUPS) {
             ok = mbar_wait_relaxed(smem_u32(&bar_full[st]), ph, &abort_flag);
             if (!ok) break;
             uint8_t *xr = smem + (size_t)st * stage_bytes + 2 * T2_A_HALF;
+            if (CONV) {
+                // 3x3: cut the tap's shifted, border-masked tile out of the raw copy and write Xh and Xl in the
+                // operand layout. Lane cg of a warp owns columns 4 cg .. 4 cg + 3 of the CTA's part of the tile,
+                // warp w of the group the channels w, w + 4, w + 8, w + 12 of the chunk.
+                const int ti = f / nchunk, c = f - ti * nchunk;
+                if (ti != mask_tile) {                     // new tile: which taps of my four columns are inside the image
+                    mask_tile = ti;
+                    const int64_t n0 = tile_col0(ti) + (int64_t)rank * NH + 4 * cg;
+                    const int hw = a.H * a.W;
+                    tap_ok = 0;
+                    for (int e = 0; e < 4; ++e) {
+                        const int64_t n = n0 + e;
+                        if (cg * 4 >= NH || n >= a.Nc) continue;
+                        const int pix = (int)(n % hw), y = pix / a.W, x = pix - y * a.W;
+                        for (int tp = 0; tp < 9; ++tp) {
+                            const int yy = y + tp / 3 - 1, xx = x + tp % 3 - 1;
+                            if (yy >= 0 && yy < a.H && xx >= 0 && xx < a.W) tap_ok |= 1ull << (tp * 4 + e);
+                        }
+                    }
+                }
+                if (cg * 4 < NH) {
+                    const int tp = (c * TC_KC) / Cin;
+                    const int sh = (tp / 3 - 1) * a.W + (tp % 3 - 1) + halo;      // >= 0: offset into the raw rows
+                    const uint32_t ok4 = (uint32_t)(tap_ok >> (tp * 4)) & 15u;
+                    const uint8_t *raw = xr + 2 * x_bytes;
+                    const uint32_t rpitch = raw_row;
+                    const int o = 4 * cg + sh, ob = o & ~3, r = o & 3;          // r is the same for every lane
+                    const uint32_t dst = (uint32_t)(cg >> 3) * T2_XG + (uint32_t)(cg & 1) * 16u;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = cw + 4 * i;
+                        const float4 lo4 = *reinterpret_cast<const float4 *>(raw + k * rpitch + ob * 4);
+                        const float4 hi4 = *reinterpret_cast<const float4 *>(raw + k * rpitch + ob * 4 + 16);
+                        float4 v;
+                        if (r == 0) v = lo4;
+                        else if (r == 1) v = make_float4(lo4.y, lo4.z, lo4.w, hi4.x);
+                        else if (r == 2) v = make_float4(lo4.z, lo4.w, hi4.x, hi4.y);
+                        else v = make_float4(lo4.w, hi4.x, hi4.y, hi4.z);
+                        if (!(ok4 & 1u)) v.x = 0.f;
+                        if (!(ok4 & 2u)) v.y = 0.f;
+                        if (!(ok4 & 4u)) v.z = 0.f;
+                        if (!(ok4 & 8u)) v.w = 0.f;
+                        float4 h, l;
+                        h.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u); l.x = v.x - h.x;
+                        h.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u); l.y = v.y - h.y;
+                        h.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u); l.z = v.z - h.z;
+                        h.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u); l.w = v.w - h.w;
+                        // row k of the 32-column box: 128 bytes whose 32-byte atoms are XOR-swizzled with k mod 4
+                        const uint32_t off = dst + (uint32_t)k * 128u + ((((uint32_t)(cg & 7) >> 1) ^ ((uint32_t)k & 3u)) << 5);
+                        *reinterpret_cast<float4 *>(xr + off) = h;
+                        *reinterpret_cast<float4 *>(xr + x_bytes + off) = l;
+                    }
+                }
+            } else
             for (int i = gt; i < npiece; i += GT) {
                 const float4 v = *reinterpret_cast<const float4 *>(xr + i * 16);
                 float4 lo;
@@ -407,34 +484,45 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 // Launch the pair kernel on tiles of 256 rows x `ntile` columns (a multiple of 64): one persistent CTA pair per SM
 // pair, or fewer if there are fewer tiles.
 // tmW: 3-D map over the plan's dense part (channel, row, {Wh, Wl}), box 16 x 128 x 2, 64-byte swizzle.
-// tmX: 128-byte swizzle with 32-byte atoms; x3d != 0: 3-D map (column in group, channel, 32-column group) with box
-// 32 x 16 x ntile/64; x3d == 0: 2-D map (column, channel) with box 32 x 16.
-int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, const void *args_, int M, int64_t Nc,
-                   int ntile, int sms, void *stream)
+// 1x1 (halo == 0): tmX in the 128-byte swizzle with 32-byte atoms; x3d != 0: 3-D map (column in group, channel,
+// 32-column group) with box 32 x 16 x ntile/64; x3d == 0: 2-D map (column, channel) with box 32 x 16.
+// 3x3 (halo = image width + 1 rounded up to a multiple of 4): tmX is a plain 2-D map (flattened (b, y, x) column,
+// channel) with box (ntile/2 + 2 halo) x 16.
+int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, int halo, const void *args_, int M,
+                   int64_t Nc, int ntile, int sms, void *stream)
 {
     TcArgs a = *static_cast<const TcArgs *>(args_);
     a.ntile = ntile;
     const int ngrp = ntile / 64;
-    const size_t smem = (size_t)t2_stages(ngrp) * (2 * T2_A_HALF + 2 * (size_t)ngrp * T2_XG) + 1024;
-    static bool done[64] = {};
+    const size_t smem = (size_t)t2_stages(ngrp, halo) * t2_stage_bytes(ngrp, halo) + 1024;
+    static bool done[2][64] = {};
     int devid = 0;
     if (cudaGetDevice(&devid) != cudaSuccess) devid = -1;
-    if (devid < 0 || devid >= 64 || !done[devid]) {
-        cudaError_t e = cudaFuncSetAttribute(ubp_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(T2_PIPE_BUDGET + 1024));
+    const int which = halo ? 1 : 0;
+    if (devid < 0 || devid >= 64 || !done[which][devid]) {
+        cudaError_t e = halo ? cudaFuncSetAttribute(ubp_tc2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)(T2_PIPE_BUDGET + 1024))
+                             : cudaFuncSetAttribute(ubp_tc2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)(T2_PIPE_BUDGET + 1024));
         if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
-        if (devid >= 0 && devid < 64) done[devid] = true;
+        if (devid >= 0 && devid < 64) done[which][devid] = true;
     }
     const int nrp = (M + 255) / 256;
     const long long ntiles = (long long)nrp * ((Nc + ntile - 1) / ntile);
     if (ntiles <= 0) return UBP_OK;
     if (ntiles > 0x7fffffffll) return UBP_E_UNSUPPORTED;
     const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
-    ubp_tc2_kernel<<<dim3((unsigned)(2 * pairs)), T2_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(
-        *tmW, *tmX, a, x3d, nrp, (int)ntiles);
+    const dim3 grid((unsigned)(2 * pairs));
+    if (halo)
+        ubp_tc2_kernel<true><<<grid, T2_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(*tmW, *tmX, a, halo, nrp, (int)ntiles);
+    else
+        ubp_tc2_kernel<false><<<grid, T2_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(*tmW, *tmX, a, x3d, nrp, (int)ntiles);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
     return UBP_OK;
 }
+
+// how many pipeline stages the pair kernel gets for a tile width and halo (0 = too few to run)
+int tc_pair_stages(int ntile, int halo) { return t2_stages(ntile / 64, halo); }
 
 }  // namespace ubp

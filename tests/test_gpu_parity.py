@@ -316,7 +316,13 @@ def test_conv3x3_small(env, M, C, Nb, p, B, H, Wd):
 
 @pytest.mark.parametrize("M,C,Nb,p,B,H,Wd,variant", [(128, 16, 8, 50, 2, 14, 14, 0), (256, 32, 4, 60, 3, 7, 9, 0),
                                                       (130, 20, 2, 50, 2, 5, 6, 42), (200, 24, 1, 70, 1, 8, 8, 43),
-                                                      (128, 40, 16, 50, 5, 6, 6, 40), (64, 16, 8, 50, 2, 6, 6, 40)])
+                                                      (128, 40, 16, 50, 5, 6, 6, 40), (64, 16, 8, 50, 2, 6, 6, 40),
+                                                      # more than 128 rows and a multiple of 16 channels: CTA pairs.
+                                                      # Ragged last row pair, column counts that are no multiple
+                                                      # of 32, wide images (larger halo), several tiles per pair
+                                                      (300, 48, 4, 60, 2, 14, 14, 41), (256, 16, 8, 50, 1, 28, 28, 40),
+                                                      (260, 32, 2, 50, 3, 13, 11, 42), (512, 64, 4, 70, 7, 14, 14, 41),
+                                                      (256, 32, 4, 60, 1, 9, 60, 41)])
 def test_conv3x3_tensor_core_variant(env, M, C, Nb, p, B, H, Wd, variant):
     """3x3 as an implicit GEMM on tensor cores (variants 40..43; chosen automatically for dense-enough layers)."""
     torch, ubp = env
@@ -324,6 +330,8 @@ def test_conv3x3_tensor_core_variant(env, M, C, Nb, p, B, H, Wd, variant):
     plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb), variant)
     assert plan.variant >= 40
     b = torch.from_numpy(L.bias).cuda()
+    if M > 128 and C % 16 == 0:
+        assert plan.tile_choice(B * H * Wd, Wd)[0] == 2
     Y = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda(), b, True, layout="CNHW")
     plan.check()
     Yref, A = oracle.masked_conv3x3(L.W, L.mask, L.X, L.bias, relu=True)
