@@ -77,7 +77,7 @@ def tf32_peak_tflops():
 NCU_DRAM_BYTES_PER_LAUNCH = {
     ("mbv1_pw512", True): 14984448 + 256,        # profiles/ncu_ubp_tc2_kernel_mbv1_pw512.md (the output is still in L2)
     ("sweep_nb4_p70", True): 124626432 + 48126208,   # profiles/ncu_ubp_tc2_kernel_sweep_nb4_p70.md
-    ("r50_3x3", True): 17635840 + 0,             # profiles/ncu_ubp_tc_kernel_r50_3x3.md
+    ("r50_3x3", True): 17614080 + 0,             # profiles/ncu_ubp_tc2_kernel_r50_3x3.md
     ("sweep_nb4_p90", False): 70554368 + 23536640,   # profiles/ncu_ubp_spmm_kernel_sweep_nb4_p90.md
 }
 

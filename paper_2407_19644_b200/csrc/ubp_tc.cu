@@ -384,7 +384,8 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int sms, int *kernel, int *
     // cycles); a tile takes its chunks or, if longer, its epilogue on eight warps (~45 cycles per column); per
     // launch ~4400 cycles of pipeline fill and ~4500 + 30 per column of drain and last epilogue.
     // 3x3: the shifted tiles are cut from a raw copy with a halo of image width + 1 columns either side, which
-    // adds shared-memory traffic (~560 + 0.75 n cycles per chunk) and leaves fewer stages.
+    // adds shared-memory traffic (raw copy in, two reads of it, Xh and Xl out: ~560 + n cycles per chunk, measured
+    // ~740 at n = 192) and leaves fewer stages.
     const int halo = conv_w > 0 ? (conv_w + 1 + 3) & ~3 : 0;
     if (M > 128 && conv_w >= 0 && (!conv || ((K / 9) % TC_KC == 0 && halo <= 64))) {
         double best2 = 1e300;
@@ -395,7 +396,7 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int sms, int *kernel, int *
             const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
             const long long per_pair = (ntiles + pairs - 1) / pairs;
             double per_chunk = 3.3 * n;
-            const double smem_chunk = conv ? 560.0 + 0.75 * n : 500.0 + 0.5 * n;
+            const double smem_chunk = conv ? 560.0 + 1.0 * n : 500.0 + 0.5 * n;
             if (per_chunk < smem_chunk) per_chunk = smem_chunk;
             double per_tile = nchunk * per_chunk;
             if (per_tile < 45.0 * n) per_tile = 45.0 * n;
