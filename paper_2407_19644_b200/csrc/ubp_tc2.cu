@@ -1,5 +1,5 @@
-// Two-CTA form of the tensor-core kernel for the 1x1 product (see ubp_tc.cu for the arithmetic: densified panels,
-// three TF32 products per fp32 product, fp32 accumulation in tensor memory).
+// Two-CTA form of the tensor-core kernel, for the 1x1 product and the 3x3 implicit GEMM (see ubp_tc.cu for the
+// arithmetic: densified panels, three TF32 products per fp32 product, fp32 accumulation in tensor memory).
 //
 // A cluster of two CTAs (two SMs) computes tiles of 256 output rows x N columns with tcgen05.mma.cta_group::2:
 // every MMA has M = 256, CTA r supplies rows 128r..128r+127 of W from its own shared memory and columns
@@ -19,11 +19,17 @@
 // memory, so the epilogue of tile t (tensor memory -> bias, ReLU -> global memory) runs under the main loop of
 // tile t + 1.
 //
+// 3x3 (stride 1, padding 1; template parameter CONV): the reduction index is k = tap * C + channel with C a multiple
+// of 16, so a chunk belongs to one tap, i.e. to one shift dy * W + dx of the flattened (b, y, x) column axis. TMA
+// cannot start a row at an odd element, so it copies the chunk's 16 channel rows for the tile's columns plus a halo
+// either side, and the Xl warps cut the shifted tile out of that copy, zero the taps that fall outside the image,
+// and write both Xh and Xl in the operand layout.
+//
 // Per CTA: warp 0 = TMA producer (its Wh / Wl rows and its X columns, one 3-D box each per chunk); warp 1 = in the
-// leader CTA (cluster rank 0) one thread issues all MMAs for the pair and commits stages and accumulators back to
-// BOTH CTAs (tcgen05.commit with a cluster multicast mask); warps 2..9 = Xl pass (two groups taking turns on the
-// chunks); warps 10..17 = epilogue (on a
-// CTA's last tile, when nothing is left to overlap with, the Xl warps take half of the epilogue). The Xl warps of
+// leader CTA (cluster rank 0) issues all MMAs for the pair (the whole warp walks the loop, one elected lane issues)
+// and commits stages and accumulators back to BOTH CTAs (tcgen05.commit with a cluster multicast mask);
+// warps 2..9 = Xl pass (two groups taking turns on the chunks); warps 10..17 = epilogue (on a CTA's last tile,
+// when nothing is left to overlap with, the Xl warps take half of the epilogue). The Xl warps of
 // BOTH CTAs arrive on one barrier per stage in the leader's shared memory (the peer's through a mapa-translated
 // address) once their CTA's copies have landed and its Xl tile is written, so the issuing thread waits once per
 // chunk; the epilogue warps of both CTAs likewise hand an accumulator back to the leader. Every waiter sees every
