@@ -163,7 +163,8 @@ int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, in
     if (c.kind == 2 || c.kind == 3) {
         int sms = 148, devid = 0;
         if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
-        ubp::tc_choose(plan->dims.M, plan->dims.C * plan->dims.R, Nc, c.kind == 3 ? image_width : 0, sms, kernel, tile_rows, tile_cols);
+        ubp::tc_choose(plan->dims.M, plan->dims.C * plan->dims.R, Nc, c.kind == 3 ? image_width : 0, ubp::cfg_bf16(c) ? 1 : 0, sms, kernel, tile_rows,
+                       tile_cols);
     } else {
         *kernel = 0; *tile_rows = c.P * c.WR; *tile_cols = 128 * c.V * c.WC;
     }

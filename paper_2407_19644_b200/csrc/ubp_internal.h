@@ -32,6 +32,8 @@ struct KernelCfg {
     int dupw;      // weights stored twice (w, w) for packed f32x2 multiply-add
 };
 const std::vector<KernelCfg> &kernel_cfgs();
+// tensor-core variants whose CTA-pair kernel uses three bf16 products per fp32 product instead of three TF32 products
+inline bool cfg_bf16(const KernelCfg &c) { return (c.id >= 34 && c.id <= 37) || (c.id >= 44 && c.id <= 47); }
 const KernelCfg *find_cfg(int id);
 // pick a configuration for a layer (variant == 0)
 const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m);
@@ -53,6 +55,10 @@ struct PlanImage {
     // kind 2 only: byte offset of the dense part (Wh [M][tc_kp] then Wl [M][tc_kp], floats) and its row length
     size_t tc_off = 0;
     int tc_kp = 0;
+    // and of the same weight as two bf16 pieces (W1 [M][tc16_kp] then W2 [M][tc16_kp], 16-bit words): W1 = the weight
+    // rounded to bf16, W2 = the remainder rounded to bf16
+    size_t tc16_off = 0;
+    int tc16_kp = 0;
 };
 int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only, PlanImage &img, size_t *bytes);
 
@@ -73,7 +79,7 @@ int launch_spmm(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, c
                 float *Y, int64_t ldy, void *stream);
 // tensor-core tile choice for a launch over Nc columns: kernel 1 = one CTA per tile, 2 = CTA pair per tile;
 // conv_w = 0: 1x1; > 0: 3x3 on images conv_w pixels wide (operands fit the pair kernel); < 0: 3x3, one CTA only
-void tc_choose(int M, int K, int64_t Nc, int conv_w, int sms, int *kernel, int *rows, int *cols);
+void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *kernel, int *rows, int *cols);
 int launch_spmm_tc(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                    float *Y, int64_t ldy, void *stream);
 int launch_conv3x3_tc(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,

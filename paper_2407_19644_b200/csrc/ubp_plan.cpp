@@ -45,12 +45,16 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     (void)M; (void)C; (void)m;
     const int nbk = largest_pow2_divisor_le16(Nb);
     const double dens = (double)m * Nb / ((double)M * C);
+    // With more than 128 rows the tensor-core variants run on CTA pairs, and there the bf16-product form (ids + 4:
+    // half the tensor-core and shared-memory time, error <= 3 * 2^-16 |w||x|, inside the 1e-4 gate) is the default;
+    // the TF32-product ids stay selectable.
+    const int fast = M > 128 ? 4 : 0;
     if (R == 9 && dens >= 0.08 && M >= 128 && C >= 16) {    // implicit GEMM on tensor cores
         switch (nbk) {
-            case 16: case 8: return find_cfg(40);
-            case 4: return find_cfg(41);
-            case 2: return find_cfg(42);
-            default: return find_cfg(43);
+            case 16: case 8: return find_cfg(40 + fast);
+            case 4: return find_cfg(41 + fast);
+            case 2: return find_cfg(42 + fast);
+            default: return find_cfg(43 + fast);
         }
     }
     if (R == 9) {
@@ -69,10 +73,10 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     // fast or faster.
     if (dens >= 0.08 && ((M > 128 && C >= 128) || (M >= 128 && C >= 256))) {
         switch (nbk) {
-            case 16: case 8: return find_cfg(33);
-            case 4: return find_cfg(32);
-            case 2: return find_cfg(31);
-            default: return find_cfg(30);
+            case 16: case 8: return find_cfg(33 + fast);
+            case 4: return find_cfg(32 + fast);
+            case 2: return find_cfg(31 + fast);
+            default: return find_cfg(30 + fast);
         }
     }
     // Sparse kernel (measured sweep): 8-row panels, 256 columns per warp; 16 warps per CTA, or 8 when the layer has
@@ -150,11 +154,14 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
     grp_off[(size_t)nkt * NG] = cur;
     size_t total = (cur + 255) & ~(size_t)255;
     if (total / 16 > 0xffffffffull) return UBP_E_UNSUPPORTED;
-    img.tc_off = 0; img.tc_kp = 0;
+    img.tc_off = 0; img.tc_kp = 0; img.tc16_off = 0; img.tc16_kp = 0;
     if (cfg.kind == 2 || cfg.kind == 3) {   // dense part for the tensor-core kernel: Wh, Wl as [M][Kp] floats,
         img.tc_kp = (C * R + 3) & ~3;       // reduction index k = tap * C + channel (tap-major)
         img.tc_off = total;
         total += ((size_t)2 * M * img.tc_kp * sizeof(float) + 255) & ~(size_t)255;
+        img.tc16_kp = (C * R + 7) & ~7;     // the same matrix as two bf16 pieces, rows of whole 16-byte groups
+        img.tc16_off = total;
+        total += ((size_t)2 * M * img.tc16_kp * sizeof(uint16_t) + 255) & ~(size_t)255;
     }
     if (bytes) *bytes = total;
     img.nkt = nkt; img.NP = NP; img.NG = NG; img.F = F; img.entries = entries; img.max_group_bytes = max_group;
@@ -226,6 +233,22 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         // top 10 mantissa bits) and the remainder, itself cut to TF32; pruned positions stay zero.
         float *Wh = reinterpret_cast<float *>(base + img.tc_off);
         float *Wl = Wh + (size_t)M * img.tc_kp;
+        // and into two bf16 pieces: the weight rounded to nearest-even bf16, and the (exact) remainder rounded
+        uint16_t *W1 = reinterpret_cast<uint16_t *>(base + img.tc16_off);
+        uint16_t *W2 = W1 + (size_t)M * img.tc16_kp;
+        auto bf16_rn = [](float f) -> uint16_t {
+            uint32_t b;
+            std::memcpy(&b, &f, 4);
+            if ((b & 0x7f800000u) == 0x7f800000u) return (uint16_t)((b >> 16) | ((b & 0xffffu) ? 0x40u : 0u));   // inf / nan
+            b += 0x7fffu + ((b >> 16) & 1u);
+            return (uint16_t)(b >> 16);
+        };
+        auto bf16_f = [](uint16_t h) -> float {
+            const uint32_t b = (uint32_t)h << 16;
+            float f;
+            std::memcpy(&f, &b, 4);
+            return f;
+        };
         for (int i = 0; i < M; ++i)
             for (int32_t b = v.indptr[i]; b < v.indptr[i + 1]; ++b) {
                 const int j = v.indices[b];
@@ -244,6 +267,9 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
                     std::memcpy(&lo, &bits, 4);
                     Wh[(size_t)(i + t) * img.tc_kp + (size_t)r * C + j] = hi;
                     Wl[(size_t)(i + t) * img.tc_kp + (size_t)r * C + j] = lo;
+                    const uint16_t w1 = bf16_rn(w);
+                    W1[(size_t)(i + t) * img.tc16_kp + (size_t)r * C + j] = w1;
+                    W2[(size_t)(i + t) * img.tc16_kp + (size_t)r * C + j] = bf16_rn(w - bf16_f(w1));
                   }
             }
     }

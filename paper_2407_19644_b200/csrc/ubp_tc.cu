@@ -325,7 +325,7 @@ int encode_2d(CUtensorMap *tm, const void *base, uint64_t inner, uint64_t outer,
 }
 
 int encode_3d(CUtensorMap *tm, const void *base, const uint64_t (&dims)[3], uint64_t stride1_bytes, uint64_t stride2_bytes,
-              const uint32_t (&box)[3], CUtensorMapSwizzle swz)
+              const uint32_t (&box)[3], CUtensorMapSwizzle swz, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_FLOAT32)
 {
     EncodeTiledFn enc = tc_encode_fn();
     if (!enc) return UBP_E_CUDA;
@@ -333,7 +333,7 @@ int encode_3d(CUtensorMap *tm, const void *base, const uint64_t (&dims)[3], uint
     const cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
     const cuuint32_t b[3] = {box[0], box[1], box[2]};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult cr = enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), d, strides, b, estr,
+    CUresult cr = enc(tm, dtype, 3, const_cast<void *>(base), d, strides, b, estr,
                       CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) { set_last_cuda_error(-(int)cr); return UBP_E_CUDA; }
@@ -347,13 +347,18 @@ int encode_3d(CUtensorMap *tm, const void *base, const uint64_t (&dims)[3], uint
 int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d, int halo, const void *args, int M,
                    int64_t Nc, int ntile, int sms, void *stream);
 int tc_pair_stages(int ntile, int halo);
+// same pipeline with three bf16 products per fp32 product (ubp_tc3.cu)
+int launch_tc_pair_bf16(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int conv, int halo, const void *args,
+                        int M, int64_t Nc, int ntile, int sms, void *stream);
+int tc_pair_bf16_stages(int ntile, int halo);
 
 // Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
 // Each candidate's time is estimated as (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost)
 // and the cheapest kept.
 // conv_w: 0 = 1x1 product; > 0 = 3x3 on images `conv_w` pixels wide whose operands the pair kernel can take;
 // < 0 = 3x3, one-CTA kernel only.
-void tc_choose(int M, int K, int64_t Nc, int conv_w, int sms, int *kernel, int *rows, int *cols)
+// bf16 != 0: the CTA-pair kernel multiplies with three bf16 products (ubp_tc3.cu) instead of three TF32 products.
+void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *kernel, int *rows, int *cols)
 {
     const int conv = conv_w != 0;
     const int nchunk = (K + TC_KC - 1) / TC_KC;
@@ -391,12 +396,13 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int sms, int *kernel, int *
         double best2 = 1e300;
         int best2_n = 0;
         for (int n = 64; n <= 256; n += 64) {
-            if (conv && (n / 2 + 2 * halo > 256 || tc_pair_stages(n, halo) < 4)) continue;
+            if (conv && (n / 2 + 2 * halo > 256 || (bf16 ? tc_pair_bf16_stages(n, halo) : tc_pair_stages(n, halo)) < 4)) continue;
             const long long ntiles = (long long)((M + 255) / 256) * ((Nc + n - 1) / n);
             const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
             const long long per_pair = (ntiles + pairs - 1) / pairs;
-            double per_chunk = 3.3 * n;
-            const double smem_chunk = conv ? 560.0 + 1.0 * n : 500.0 + 0.5 * n;
+            // bf16 products: three MMAs of K = 16 per chunk (half the tensor-core time) and half the operand bytes
+            double per_chunk = bf16 ? 1.65 * n : 3.3 * n;
+            const double smem_chunk = bf16 ? (conv ? 220.0 + 1.5 * n : 190.0 + 1.2 * n) : (conv ? 560.0 + 1.0 * n : 500.0 + 0.5 * n);
             if (per_chunk < smem_chunk) per_chunk = smem_chunk;
             double per_tile = nchunk * per_chunk;
             if (per_tile < 45.0 * n) per_tile = 45.0 * n;
@@ -423,10 +429,24 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
     // 3x3 on CTA pairs needs the input as one [channel][b, y, x] matrix with 16-byte aligned rows
     const bool conv_pair_ok = a.conv && a.isb == (int64_t)a.H * a.W && a.isc % 4 == 0 &&
                               (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && a.isc >= Nc;
-    tc_choose(M, K, Nc, a.conv ? (conv_pair_ok ? a.W : -1) : 0, sms, &kernel, &rows, &best_n);
+    const int bf16 = cfg_bf16(pl->cfg) ? 1 : 0;            // variants 34..37 / 44..47
+    tc_choose(M, K, Nc, a.conv ? (conv_pair_ok ? a.W : -1) : 0, bf16, sms, &kernel, &rows, &best_n);
 #ifdef UBP_TC_TUNE   // diagnostic builds only: force the kernel and tile width from the environment
     if (const char *e = getenv("UBP_TC_FORCE")) { int k = 0, n = 0; if (sscanf(e, "%d,%d", &k, &n) == 2) { kernel = k; best_n = n; rows = (k == 2 || k == 12) ? 256 : 128; if (k == 12) kernel = 1; } }
 #endif
+    if (kernel == 2 && bf16) {
+        const uint16_t *W1 = reinterpret_cast<const uint16_t *>(dev + pl->img.tc16_off);
+        CUtensorMap tmW, tmX;
+        const uint64_t wdims[3] = {(uint64_t)pl->img.tc16_kp, (uint64_t)M, 2};
+        const uint32_t wbox[3] = {TC_KC, 128, 2};
+        if ((rc = encode_3d(&tmW, W1, wdims, (uint64_t)pl->img.tc16_kp * 2, (uint64_t)M * pl->img.tc16_kp * 2, wbox,
+                            CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16))) return rc;
+        // the input as (column, channel): 16 channel rows of the CTA's columns per chunk, plus the halo for 3x3
+        const int halo = a.conv ? (a.W + 1 + 3) & ~3 : 0;
+        if ((rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)(a.conv ? K / 9 : K), (uint64_t)(a.conv ? a.isc : a.ldx) * 4,
+                            (uint32_t)(best_n / 2 + 2 * halo), TC_KC, CU_TENSOR_MAP_SWIZZLE_NONE))) return rc;
+        return launch_tc_pair_bf16(&tmW, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream);
+    }
     if (kernel == 2) {
         // Wh and Wl as one 3-D tensor (channel, row, part): one copy per chunk brings both
         CUtensorMap tmW, tmX;

@@ -1,0 +1,395 @@
+// CTA-pair tensor-core kernel with bf16 products (1x1 and 3x3): the persistent pipeline of ubp_tc2.cu with every
+// fp32 product w * x replaced by three bf16 products instead of three TF32 products,
+//     w = w1 + w2 + (..),  x = x1 + x2 + (..)    (w1 = bf16(w), w2 = bf16(w - w1), likewise x)
+//     w x ~= w1 x1 + w2 x1 + w1 x2,
+// accumulated in fp32 in tensor memory. bf16 keeps 8 significant bits, so |w - w1 - w2| <= 2^-16 |w| and the three
+// dropped terms are each <= 2^-16 |w||x|: error <= 3 * 2^-16 |w||x| per product (measured on the test layers:
+// ~1-4 * 10^-6 of sum |w||x|), inside the 1e-4 gate, against ~2^-20 for the TF32 split. In exchange a 16-channel
+// chunk takes three MMAs of K = 16 instead of six of K = 8 and its operands are half as many bytes: half the
+// tensor-core time and little more than half the shared-memory traffic, the two bounds of ubp_tc2.cu.
+//
+// Differences from ubp_tc2.cu: the plan supplies W1 / W2 (bf16, K-major; TMA box 16 x 128 x 2 in the 32-byte
+// swizzle); the tensor core cannot take the raw fp32 activations any more, so TMA copies the chunk's 16 channel rows
+// as they are (plus a halo for 3x3) and the pass warps write BOTH x1 and x2, in the MN-major bf16 operand layout
+// (64 columns x 8 channels atoms in the 128-byte swizzle; LBO = next 64 columns, SBO = next 8 channels). Thread
+// roles, barriers, persistence, the two accumulators and the epilogue are those of ubp_tc2.cu.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "ubp_internal.h"
+#include "ubp_tc_common.cuh"
+
+namespace ubp {
+
+namespace {
+
+using namespace tc;
+
+constexpr int T3_XL_WARPS = 8;                            // warps 2..9: the split pass
+constexpr int T3_XL_GROUPS = 2;                           // two groups of four warps take turns on the chunks
+constexpr int T3_EPI_WARPS = 8;                           // warps 10..17
+constexpr int T3_THREADS = (2 + T3_XL_WARPS + T3_EPI_WARPS) * 32;
+constexpr int T3_MAX_STAGES = 8;
+constexpr uint32_t T3_A_PART = 128 * TC_KC * 2;           // W1 or W2 chunk of this CTA's 128 rows: 4 KB
+constexpr uint32_t T3_ATOM = 64 * TC_KC * 2;              // x1 or x2 of 64 columns x 16 channels: 2 KB
+constexpr uint32_t T3_PIPE_BUDGET = 222 * 1024;
+constexpr uint32_t SWZ_32B = 6, SWZ_128B = 2;             // descriptor layout types
+constexpr uint32_t T3_ACC_COLS = 256;                     // tensor-memory columns per accumulator
+
+// a stage = W1 + W2 chunk (8 KB) + x1 + x2 tiles (2 KB per started 64 columns each) + the raw fp32 rows
+// (16 channels x (columns + 2 x halo) floats, padded to 1 KB). The stage count is a multiple of the group count so
+// that a stage always belongs to the same group of pass warps (a waiter must see every phase of its barrier).
+__host__ __device__ constexpr uint32_t t3_x_bytes(int nh) { return (uint32_t)((nh + 63) / 64) * T3_ATOM; }
+__host__ __device__ constexpr uint32_t t3_raw_bytes(int nh, int halo)
+{
+    return ((uint32_t)(nh + 2 * halo) * TC_KC * 4 + 1023u) & ~1023u;
+}
+__host__ __device__ constexpr uint32_t t3_stage_bytes(int nh, int halo)
+{
+    return 2 * T3_A_PART + 2 * t3_x_bytes(nh) + t3_raw_bytes(nh, halo);
+}
+__host__ __device__ constexpr int t3_stages(int nh, int halo)
+{
+    const int s = (int)(T3_PIPE_BUDGET / t3_stage_bytes(nh, halo));
+    return (s > T3_MAX_STAGES ? T3_MAX_STAGES : s) / T3_XL_GROUPS * T3_XL_GROUPS;
+}
+
+// instruction descriptor: D = f32, A = B = bf16, A K-major, B MN-major, M = 256 (two CTAs), N = n
+__device__ __forceinline__ uint32_t make_idesc3(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+// One chunk's three MMAs (K = 16 each: w1 x1, w2 x1, w1 x2) and the commit that hands the stage back to both CTAs,
+// in a single statement, with a non-blocking test of the NEXT chunk's barrier issued first and its result read
+// last. Executed by a whole converged warp: one elected lane issues. Returns whether the next chunk is ready.
+__device__ __forceinline__ bool mma3_chunk(uint32_t d_tmem, uint64_t dW1, uint64_t dX1, uint32_t w2_off, uint32_t x2_off,
+                                           uint32_t idesc, uint32_t acc_first, uint32_t next_bar, uint32_t next_parity,
+                                           uint32_t empty_bar)
+{
+    uint32_t ready;
+    asm volatile(
+        "{\n\t.reg .pred pn, pa, pt, pe;\n\t.reg .b64 w2, x2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 pn, [%8], %9;\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "setp.ne.b32 pa, %7, 0;\n\t"
+        "setp.eq.b32 pt, %10, 0;\n\t"
+        "cvt.u64.u32 w2, %4;\n\tadd.s64 w2, w2, %2;\n\t"
+        "cvt.u64.u32 x2, %5;\n\tadd.s64 x2, x2, %3;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %6, pa;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w2, %3, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, x2, %6, pt;\n\t"
+        "@pe tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%11], %12;\n\t"
+        "selp.u32 %0, 1, 0, pn;\n\t}"
+        : "=r"(ready)
+        : "r"(d_tmem), "l"(dW1), "l"(dX1), "r"(w2_off), "r"(x2_off), "r"(idesc), "r"(acc_first), "r"(next_bar),
+          "r"(next_parity), "r"(0u), "r"(empty_bar), "h"((uint16_t)3)
+        : "memory");
+    return ready != 0;
+}
+
+// eight fp32 -> their bf16 heads (x1) and the bf16 of the remainders (x2), packed two per word
+__device__ __forceinline__ void split8(const float (&v)[8], uint4 &h, uint4 &l)
+{
+    uint32_t hh[4], ll[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        const float2 af = __bfloat1622float2(a);
+        const __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * i] - af.x, v[2 * i + 1] - af.y);
+        hh[i] = *reinterpret_cast<const uint32_t *>(&a);
+        ll[i] = *reinterpret_cast<const uint32_t *>(&b);
+    }
+    h = make_uint4(hh[0], hh[1], hh[2], hh[3]);
+    l = make_uint4(ll[0], ll[1], ll[2], ll[3]);
+}
+
+template <bool CONV>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T3_THREADS, 1)
+ubp_tc3_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const TcArgs a,
+               const int halo, const int nrp, const int ntiles)
+{
+    constexpr int MAXS = T3_MAX_STAGES;
+    constexpr uint32_t TMEM_COLS = 2 * T3_ACC_COLS;
+
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    // identical layout in both CTAs: the multicast commits and the remote arrives address barriers by offset
+    __shared__ __align__(8) uint64_t bar_full[MAXS], bar_go[MAXS], bar_empty[MAXS], bar_acc_full[2], bar_acc_empty[2],
+        bar_last;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();
+    const int N = a.ntile, NH = N / 2;                     // tile columns; columns whose X this CTA holds
+    const uint32_t xb = t3_x_bytes(NH);                    // x1 (and x2) bytes per stage
+    const uint32_t stage_bytes = t3_stage_bytes(NH, halo);
+    const uint32_t raw_row = (uint32_t)(NH + 2 * halo) * 4;   // bytes per channel row of the raw copy
+    const int S = t3_stages(NH, halo);
+    const int nchunk = (a.K + TC_KC - 1) / TC_KC;
+    const uint32_t tx = 2 * T3_A_PART + raw_row * TC_KC;
+    const int Cin = CONV ? a.K / 9 : a.K;                  // 3x3: reduction index k = tap * Cin + channel, Cin % 16 == 0
+    // this pair's tiles: pair, pair + npairs, ...; tile t = (row pair t % nrp, column tile t / nrp)
+    const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
+    const int nmy = pair < ntiles ? (ntiles - pair + npairs - 1) / npairs : 0;
+    auto tile_row0 = [&](int i) { return ((pair + i * npairs) % nrp) * 256 + (int)rank * 128; };
+    auto tile_col0 = [&](int i) { return (int64_t)((pair + i * npairs) / nrp) * N; };
+
+    // one chunk's copies: W1 and W2 rows of this CTA in one 3-D box; 16 channel rows of the input for this CTA's
+    // columns (3x3: the channels of the chunk's tap, and a halo of columns either side)
+    auto issue_chunk = [&](int c, int st, int row0, int xcol) {
+        uint8_t *stage = smem + (size_t)st * stage_bytes;
+        const uint32_t bar = smem_u32(&bar_full[st]);
+        mbar_expect_tx(bar, tx);
+        tma_load_3d(smem_u32(stage), &tmW, c * TC_KC, row0, 0, bar);
+        tma_load_2d(smem_u32(stage + 2 * T3_A_PART + 2 * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
+    };
+
+    if (threadIdx.x == 0) {
+        prefetch_tensormap(&tmW);
+        prefetch_tensormap(&tmX);
+        abort_flag = 0;
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_go[s]), 2 * (T3_XL_WARPS / T3_XL_GROUPS));   // used in the leader CTA only
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bar_acc_full[b]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[b]), 2 * T3_EPI_WARPS);            // used in the leader CTA only
+        }
+        mbar_init(smem_u32(&bar_last), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // the first copy lands in this CTA's own memory and signals its own barrier: start it before the
+        // tensor-memory allocation and the cluster barrier
+        if (nmy > 0) issue_chunk(0, 0, tile_row0(0), (int)(tile_col0(0) + (int64_t)rank * NH));
+    }
+    if (warp == 1) {   // tensor memory of the pair: the same warp of both CTAs allocates
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync();                                        // both CTAs' barriers exist before anyone signals them
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+
+    bool ok = true;
+    if (warp == 0) {
+        // ---------------- TMA producer: one ring of S stages straight through all of this pair's tiles
+        if (lane == 0) {
+            int st = 1 % S, round = 1 / S;                 // chunk (0, 0) was started above
+            for (int i = 0; i < nmy && ok; ++i) {
+                const int row0 = tile_row0(i), xcol = (int)(tile_col0(i) + (int64_t)rank * NH);
+                for (int c = (i == 0 ? 1 : 0); c < nchunk; ++c) {
+                    if (round > 0) {                       // the stage's previous contents must have been consumed
+                        ok = mbar_wait_relaxed(smem_u32(&bar_empty[st]), (uint32_t)(round - 1) & 1u, &abort_flag);
+                        if (!ok) break;
+                    }
+                    issue_chunk(c, st, row0, xcol);
+                    if (++st == S) { st = 0; ++round; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (rank == 0) {
+            // ---------------- leader: MMA issuer for the pair (whole warp converged, one elected lane issues)
+            const uint32_t idesc = make_idesc3(N);
+            const uint64_t dW0 = make_desc(smem_u32(smem), 16, 256, SWZ_32B);
+            const uint64_t dX0 = make_desc(smem_u32(smem) + 2 * T3_A_PART, 2048, 1024, SWZ_128B);
+            const uint32_t stage_u = stage_bytes >> 4;
+            int st = 0;
+            uint32_t ph = 0;
+            bool ready = nmy > 0 && mbar_try_wait(smem_u32(&bar_go[0]), 0);
+            for (int i = 0; i < nmy && ok; ++i) {
+                const int b = i & 1;
+                const uint32_t acc = tmem_base + (uint32_t)b * T3_ACC_COLS;
+                if (i >= 2) {                              // the epilogue of tile i - 2 must have read this accumulator
+                    ok = mbar_wait(smem_u32(&bar_acc_empty[b]), (uint32_t)((i >> 1) - 1) & 1u, &abort_flag);
+                    if (!ok) break;
+                }
+                for (int c = 0; c < nchunk; ++c) {
+                    if (!ready) ok = mbar_wait(smem_u32(&bar_go[st]), ph, &abort_flag);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t soff = (uint64_t)((uint32_t)st * stage_u);
+                    int nst = st + 1;
+                    uint32_t nph = ph;
+                    if (nst == S) { nst = 0; nph ^= 1u; }
+                    ready = mma3_chunk(acc, dW0 + soff, dX0 + soff, T3_A_PART >> 4, xb >> 4, idesc, c > 0 ? 1u : 0u,
+                                       smem_u32(&bar_go[nst]), nph, smem_u32(&bar_empty[st]));
+                    st = nst; ph = nph;
+                }
+                if (!ok) break;
+                mma2_commit_both(smem_u32(&bar_acc_full[b]));     // accumulator complete: epilogue warps of both CTAs
+                if (i == nmy - 1) mma2_commit_both(smem_u32(&bar_last));
+            }
+        }
+    } else if (warp < 2 + T3_XL_WARPS) {
+        // ---------------- split pass: raw fp32 rows -> x1, x2 (bf16) in the operand layout. Two groups of four
+        // warps take turns on the chunks. Thread (cg, kq) of a group: columns 8 cg .. 8 cg + 7 of the CTA's part
+        // of the tile, channels kq and kq + 8 of the chunk.
+        constexpr int GT = (T3_XL_WARPS / T3_XL_GROUPS) * 32;
+        const int grp = (warp - 2) / (T3_XL_WARPS / T3_XL_GROUPS);
+        const int gt = (int)threadIdx.x - 64 - grp * GT;
+        const int cg = gt & 15, kq = gt >> 4;
+        const bool mine = cg * 8 < NH;
+        const int total = nmy * nchunk;
+        const uint32_t dst = (uint32_t)(cg >> 3) * T3_ATOM;   // 64-column atom; inside it row k is 128 bytes whose
+        const uint32_t c16 = (uint32_t)(cg & 7);              // 16-byte pieces are XOR-swizzled with k mod 8
+        unsigned long long tap_lo = 0;                         // 3x3: bit tap * 8 + e (taps 0..7): tap inside the image
+        uint32_t tap_hi = 0;                                   //      for column 8 cg + e; tap 8 in tap_hi
+        int mask_tile = -1;
+        int st = grp;                                      // the stage count is even: stages grp, grp + 2, ...
+        uint32_t ph = 0;
+        for (int f = grp; f < total && ok; f += T3_XL_GROUPS) {
+            ok = mbar_wait_relaxed(smem_u32(&bar_full[st]), ph, &abort_flag);
+            if (!ok) break;
+            uint8_t *x1 = smem + (size_t)st * stage_bytes + 2 * T3_A_PART;
+            const uint8_t *raw = x1 + 2 * xb;
+            int sh = 0;
+            uint32_t ok8 = 0xffu;
+            if (CONV) {
+                const int ti = f / nchunk, c = f - ti * nchunk;
+                if (ti != mask_tile) {                     // new tile: which taps of my eight columns are inside the image
+                    mask_tile = ti;
+                    const int64_t n0 = tile_col0(ti) + (int64_t)rank * NH + 8 * cg;
+                    const int hw = a.H * a.W;
+                    tap_lo = 0; tap_hi = 0;
+                    for (int e = 0; e < 8; ++e) {
+                        const int64_t n = n0 + e;
+                        if (!mine || n >= a.Nc) continue;
+                        const int pix = (int)(n % hw), y = pix / a.W, x = pix - y * a.W;
+                        for (int tp = 0; tp < 9; ++tp) {
+                            const int yy = y + tp / 3 - 1, xx = x + tp % 3 - 1;
+                            if (yy >= 0 && yy < a.H && xx >= 0 && xx < a.W) {
+                                if (tp < 8) tap_lo |= 1ull << (tp * 8 + e); else tap_hi |= 1u << e;
+                            }
+                        }
+                    }
+                }
+                const int tp = (c * TC_KC) / Cin;
+                sh = (tp / 3 - 1) * a.W + (tp % 3 - 1) + halo;              // >= 0: offset into the raw rows
+                ok8 = tp < 8 ? (uint32_t)(tap_lo >> (tp * 8)) & 0xffu : tap_hi;
+            }
+            if (mine) {
+                const int o = 8 * cg + sh, ob = o & ~3, r = o & 3;          // r is the same for every lane
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int k = kq + 8 * i;
+                    const float4 q0 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4);
+                    const float4 q1 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 16);
+                    float v[8];
+                    if (!CONV || r == 0) {
+                        v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w; v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+                    } else {
+                        const float4 q2 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 32);
+                        const float t[12] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w, q2.x, q2.y, q2.z, q2.w};
+                        if (r == 1) { for (int e = 0; e < 8; ++e) v[e] = t[e + 1]; }
+                        else if (r == 2) { for (int e = 0; e < 8; ++e) v[e] = t[e + 2]; }
+                        else { for (int e = 0; e < 8; ++e) v[e] = t[e + 3]; }
+                    }
+                    if (CONV) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) if (!((ok8 >> e) & 1u)) v[e] = 0.f;
+                    }
+                    uint4 h, l;
+                    split8(v, h, l);
+                    const uint32_t off = dst + (uint32_t)k * 128u + ((c16 ^ ((uint32_t)k & 7u)) << 4);
+                    *reinterpret_cast<uint4 *>(x1 + off) = h;
+                    *reinterpret_cast<uint4 *>(x1 + xb + off) = l;
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the writes visible to the MMA unit
+            __syncwarp();
+            if (lane == 0) {
+                if (rank == 0) mbar_arrive(smem_u32(&bar_go[st]));
+                else mbar_arrive_remote(smem_u32(&bar_go[st]), 0);
+            }
+            st += T3_XL_GROUPS;
+            if (st >= S) { st -= S; ph ^= 1u; }
+        }
+        // ---------------- the last tile has nothing to overlap with: take column blocks 2, 3, 6, 7 of its epilogue.
+        // Its own barrier (one phase) rather than the accumulator's, whose earlier phases these warps did not see.
+        if (ok && nmy > 0) ok = mbar_wait_relaxed(smem_u32(&bar_last), 0, &abort_flag);
+        if (ok && nmy > 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int i = nmy - 1;
+            epilogue_blocks(a, tmem_base + (uint32_t)(i & 1) * T3_ACC_COLS, warp & 3, 2 + ((warp - 2) >> 2), 4, N,
+                            tile_row0(i), tile_col0(i), lane, 0u, rank);
+        }
+    } else {
+        // ---------------- epilogue warps: tile i's accumulator while the main loop works on tile i + 1
+        const int part = (warp - 2 - T3_XL_WARPS) >> 2;       // two warps share a lane quarter and split the columns
+        for (int i = 0; i < nmy && ok; ++i) {
+            const int b = i & 1;
+            ok = mbar_wait_relaxed(smem_u32(&bar_acc_full[b]), (uint32_t)(i >> 1) & 1u, &abort_flag);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const bool last = i == nmy - 1;
+            epilogue_blocks(a, tmem_base + (uint32_t)b * T3_ACC_COLS, warp & 3, part, last ? 4 : 2, N, tile_row0(i),
+                            tile_col0(i), lane, last ? 0u : smem_u32(&bar_acc_empty[b]), rank);
+        }
+    }
+    if (!ok && lane == 0) atomicExch(a.status, 1);
+    // every thread of both CTAs comes here: neither CTA may free tensor memory or leave while the other could
+    // still be the target of the pair's MMAs or commits
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace
+
+// Launch the bf16 pair kernel on tiles of 256 rows x `ntile` columns (a multiple of 64).
+// tmW: 3-D map over the plan's bf16 part (channel, row, {W1, W2}), box 16 x 128 x 2, 32-byte swizzle.
+// tmX: plain 2-D fp32 map (column, channel), box (ntile/2 + 2 halo) x 16; halo = 0 for 1x1, image width + 1
+// rounded up to a multiple of 4 for 3x3 (columns = the flattened (b, y, x) axis).
+int launch_tc_pair_bf16(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int conv, int halo, const void *args_,
+                        int M, int64_t Nc, int ntile, int sms, void *stream)
+{
+    TcArgs a = *static_cast<const TcArgs *>(args_);
+    a.ntile = ntile;
+    const int nh = ntile / 2;
+    const size_t smem = (size_t)t3_stages(nh, halo) * t3_stage_bytes(nh, halo) + 1024;
+    static bool done[2][64] = {};
+    int devid = 0;
+    if (cudaGetDevice(&devid) != cudaSuccess) devid = -1;
+    const int which = conv ? 1 : 0;
+    if (devid < 0 || devid >= 64 || !done[which][devid]) {
+        cudaError_t e = conv ? cudaFuncSetAttribute(ubp_tc3_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)(T3_PIPE_BUDGET + 1024))
+                             : cudaFuncSetAttribute(ubp_tc3_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)(T3_PIPE_BUDGET + 1024));
+        if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+        if (devid >= 0 && devid < 64) done[which][devid] = true;
+    }
+    const int nrp = (M + 255) / 256;
+    const long long ntiles = (long long)nrp * ((Nc + ntile - 1) / ntile);
+    if (ntiles <= 0) return UBP_OK;
+    if (ntiles > 0x7fffffffll) return UBP_E_UNSUPPORTED;
+    const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
+    const dim3 grid((unsigned)(2 * pairs));
+    if (conv)
+        ubp_tc3_kernel<true><<<grid, T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(*tmW, *tmX, a, halo, nrp, (int)ntiles);
+    else
+        ubp_tc3_kernel<false><<<grid, T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(*tmW, *tmX, a, halo, nrp, (int)ntiles);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+    return UBP_OK;
+}
+
+// how many pipeline stages the bf16 pair kernel gets for a tile width and halo
+int tc_pair_bf16_stages(int ntile, int halo) { return t3_stages(ntile / 2, halo); }
+
+}  // namespace ubp

@@ -152,6 +152,105 @@ struct TcArgs {
 };
 
 
+// ---------------------------------------------------------------- helpers of the CTA-pair kernels
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster. What the arrival stands for
+// (TMA writes, generic writes already followed by a proxy fence, completed tensor-memory reads) sits in the
+// sender's own SM and is consumed there by its own tensor core, so no cluster-scope release is needed; with one
+// the arrive cost ~700 cycles.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_bar), "r"(rank));
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+// completion of all MMAs issued so far arrives on the barrier at this offset in both CTAs of the pair (called by
+// a whole converged warp; one elected lane issues it)
+__device__ __forceinline__ void mma2_commit_both(uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred pe;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+        ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+
+// Epilogue of 32 rows (tensor-memory lane quarter q of accumulator `acc`) x the 32-column blocks first, first + step,
+// ... of one CTA's 128 x N part of a tile, without shared memory (the MMA operands and the copies already use all
+// of its bandwidth). The accumulator is read in the 16 x 256-bit shape: lane t gets, per group j of 8 columns,
+// the column pair 8j + 2(t mod 4) of rows t/4 and t/4 + 8 of a 16-row half. Four lanes therefore hold 32
+// consecutive bytes of an output row, and every 8-byte store instruction of the warp writes eight whole 32-byte
+// sectors; bias and ReLU are applied in registers.
+// `done_bar` != 0: once this warp's last tensor-memory read has completed, lane 0 arrives on that barrier of the
+// leader CTA (the accumulator may be overwritten from then on).
+__device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, int q, int first, int step, int N,
+                                                int row0, int64_t col0, int lane, uint32_t done_bar, uint32_t rank)
+{
+    const int rbase = row0 + q * 32 + (lane >> 2);          // this lane's rows: rbase + {0, 8, 16, 24}
+    const int nblk = N / 32;
+    float bias[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) bias[i] = (a.bias && rbase + 8 * i < a.M) ? __ldg(a.bias + rbase + 8 * i) : 0.f;
+#pragma unroll 1
+    for (int cc = first; cc < nblk; cc += step) {
+        uint32_t r[2][16];
+        tmem_ld_16x256b_x4(acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), r[0]);
+        tmem_ld_16x256b_x4(acc + ((uint32_t)(q * 32 + 16) << 16) + (uint32_t)(cc * 32), r[1]);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (done_bar && cc + step >= nblk) {
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            if (lane == 0) {
+                if (rank == 0) mbar_arrive(done_bar);
+                else mbar_arrive_remote(done_bar, 0);
+            }
+        }
+        const int64_t cb = col0 + cc * 32 + 2 * (lane & 3);
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int row = rbase + 16 * half + 8 * h;
+                if (row >= a.M) continue;
+                float *yrow = a.Y + (size_t)row * a.ldy;
+                const float b = bias[2 * half + h];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float2 o = make_float2(__uint_as_float(r[half][4 * j + 2 * h]) + b,
+                                           __uint_as_float(r[half][4 * j + 2 * h + 1]) + b);
+                    if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); }
+                    const int64_t col = cb + 8 * j;
+                    if (col + 1 < a.Nc) *reinterpret_cast<float2 *>(yrow + col) = o;
+                    else if (col < a.Nc) yrow[col] = o.x;
+                }
+            }
+    }
+    // a warp with no block of its own still owes its arrival
+    if (done_bar && first >= nblk) {
+        if (lane == 0) {
+            if (rank == 0) mbar_arrive(done_bar);
+            else mbar_arrive_remote(done_bar, 0);
+        }
+    }
+}
+
 }  // namespace tc
 }  // namespace ubp
 #endif

@@ -163,7 +163,9 @@ def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     img, geom = ubp.plan_image(blob, variant)
     tc_off = ubp.plan_size(blob, sparse_variant)             # same geometry without the dense part
     kp = (C * R + 3) // 4 * 4
-    assert len(img) == tc_off + (2 * M * kp * 4 + 255) // 256 * 256
+    kp16 = (C * R + 7) // 8 * 8
+    tc16_off = tc_off + (2 * M * kp * 4 + 255) // 256 * 256
+    assert len(img) == tc16_off + (2 * M * kp16 * 2 + 255) // 256 * 256
     # the embedded sparse plan is byte-identical to the stand-alone one
     img_s, _ = ubp.plan_image(blob, sparse_variant)
     assert np.array_equal(img[:tc_off], img_s)
@@ -176,3 +178,12 @@ def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     assert np.all(np.abs(got - Wm) <= np.abs(Wm) * 2.0 ** -20)
     assert not got[Wm == 0].any()
     assert np.array_equal(Wh[:, :C * R], (Wm.view(np.uint32) & 0xffffe000).view(np.float32))
+    # the same matrix as two bf16 pieces (8-bit significands): W1 = nearest bf16, so |W - W1| <= 2^-8 |W|, and
+    # W1 + W2 within 2^-16 |W|
+    W1 = (np.frombuffer(img, "<u2", M * kp16, tc16_off).reshape(M, kp16).astype(np.uint32) << 16).view(np.float32)
+    W2 = (np.frombuffer(img, "<u2", M * kp16, tc16_off + 2 * M * kp16).reshape(M, kp16).astype(np.uint32) << 16).view(np.float32)
+    assert not W1[:, C * R:].any() and not W2[:, C * R:].any()
+    assert np.all(np.abs(W1[:, :C * R].astype(np.float64) - Wm) <= np.abs(Wm) * 2.0 ** -8)
+    got16 = W1[:, :C * R].astype(np.float64) + W2[:, :C * R]
+    assert np.all(np.abs(got16 - Wm) <= np.abs(Wm) * 2.0 ** -16)
+    assert not got16[Wm == 0].any()

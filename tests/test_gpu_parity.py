@@ -50,15 +50,31 @@ def run_spmm(env, L, variant=0, pad=0, misalign=0, relu=None, use_bias=True):
     return Yh, Yref, A, plan
 
 
-def check(Yh, Yref, A, L, tensor_core=False):
-    """Gate 1e-4, plus the summation bound of the arithmetic that ran: (L + 2) 2^-24 for the fp32 kernels; the
-    tensor-core variant splits each operand into two TF32 pieces and drops the low x low product and the bits
-    below the low pieces (each <= 2^-20 |w||x|), and its accumulator truncates: 2^-18 + (L + 2) 2^-23."""
+def is_bf16(variant):
+    """Tensor-core variants whose CTA-pair kernel multiplies with three bf16 products instead of three TF32 ones."""
+    return 34 <= variant <= 37 or 44 <= variant <= 47
+
+
+def arith_bound(L, variant):
+    """Summation bound of the arithmetic that ran: (L + 2) 2^-24 for the fp32 kernels; the tensor-core variants split
+    each operand into two pieces and drop the low x low product and the bits below the low pieces, and their
+    accumulator truncates: TF32 pieces (each dropped term <= 2^-20 |w||x|) 2^-18 + (L + 2) 2^-23; bf16 pieces (three
+    dropped terms <= 2^-16 |w||x| each) 3 * 2^-16 + (L + 2) 2^-23."""
+    n = terms_per_output(L) + 2
+    if is_bf16(variant):
+        return 3 * 2.0 ** -16 + n * 2.0 ** -23
+    if variant >= 30:
+        return 2.0 ** -18 + n * 2.0 ** -23
+    return n * 2.0 ** -24
+
+
+def check(Yh, Yref, A, L, tensor_core=False, variant=None):
+    """Gate 1e-4, plus the bound of the arithmetic that ran (arith_bound; tensor_core=True without a variant means
+    the TF32 form)."""
     assert np.isfinite(Yh).all()
     err = scaled_error(Yh, Yref, A)
     assert err <= TOL, err
-    n = terms_per_output(L) + 2
-    bound = 2.0 ** -18 + n * 2.0 ** -23 if tensor_core else n * 2.0 ** -24
+    bound = arith_bound(L, variant if variant is not None else (32 if tensor_core else 0))
     assert err <= bound, (err, bound)
     return err
 
@@ -77,7 +93,7 @@ SMALL = [
 def test_spmm_small(env, M, C, Nb, p, Nc, variant):
     L = ubp_synth.make_layer("t", M, C, Nb, p, 10 * M + C, Nc=Nc, x_dist="normal", relu=(M % 2 == 0))
     Yh, Yref, A, plan = run_spmm(env, L, variant)
-    check(Yh, Yref, A, L, tensor_core=plan.variant >= 30)
+    check(Yh, Yref, A, L, variant=plan.variant)
 
 
 TC_CASES = [
@@ -96,7 +112,12 @@ def test_spmm_tensor_core_variant(env, M, C, Nb, p, Nc, variant):
     L = ubp_synth.make_layer("t", M, C, Nb, p, 10 * M + C, Nc=Nc, x_dist="normal", relu=(M % 2 == 0))
     Yh, Yref, A, plan = run_spmm(env, L, variant)
     assert plan.variant == variant
-    check(Yh, Yref, A, L, tensor_core=True)
+    check(Yh, Yref, A, L, variant=variant)
+    if M > 128:                          # the same layer through the bf16-product form of the CTA-pair kernel
+        Yh, Yref, A, plan = run_spmm(env, L, variant + 4)
+        assert plan.variant == variant + 4 and plan.tile_choice(Nc)[0] in (1, 2)
+        err = check(Yh, Yref, A, L, variant=variant + 4)
+        assert err <= 2e-5               # far inside its worst-case bound on random data
 
 
 def test_tensor_core_variant_ragged_unaligned_and_auto(env):
@@ -113,7 +134,7 @@ def test_tensor_core_variant_ragged_unaligned_and_auto(env):
     sparse = ubp_synth.make_layer("t", 256, 256, 4, 95, 780, Nc=512)
     small = ubp_synth.make_layer("t", 64, 32, 4, 50, 781, Nc=512)
     pv = lambda l: ubp.Plan(ubp.ubp_pack(l.W, l.mask, l.Nb)).variant
-    assert pv(dense) == 32 and pv(sparse) == 14 and pv(small) == 50
+    assert pv(dense) == 36 and pv(sparse) == 14 and pv(small) == 50      # 36 = 32 with bf16 products (more than 128 rows)
     # bitwise reproducible run to run
     plan = ubp.Plan(ubp.ubp_pack(dense.W, dense.mask, 4))
     X = torch.from_numpy(dense.X).cuda()
@@ -196,7 +217,7 @@ def test_mbv1_pw512_config_full(env):
     Y = ubp.ubp_conv1x1(plan, X, torch.from_numpy(L.bias).cuda(), True, layout="CNHW")
     plan.check()
     Yref, A = oracle.masked_matmul(L.W, L.mask, L.X.reshape(L.C, -1), L.bias, relu=True)
-    check(Y.cpu().numpy().reshape(L.M, -1), Yref, A, L, tensor_core=plan.variant >= 30)
+    check(Y.cpu().numpy().reshape(L.M, -1), Yref, A, L, variant=plan.variant)
     # and the sparse kernel on the same layer
     plan_s = ubp.Plan(blob, 14)
     Ys = ubp.ubp_conv1x1(plan_s, X, torch.from_numpy(L.bias).cuda(), True, layout="CNHW")
@@ -243,7 +264,7 @@ def test_sweep_config_sampled(env, nb, sp, variant):
     ys, as_ = oracle.masked_matmul_samples(L.W, L.mask, L.X, so, sn)
     err = scaled_error(Y[so, sn], ys, as_)
     n = terms_per_output(L) + 2
-    assert err <= TOL and err <= (2.0 ** -18 + n * 2.0 ** -23 if plan.variant >= 30 else n * 2.0 ** -24)
+    assert err <= TOL and err <= arith_bound(L, plan.variant)
     # whole rows too (a panel's first / last row and one in the middle)
     for o in (0, 15, 16, 1000, L.M - 1):
         sn2 = np.arange(L.Nc)
@@ -335,7 +356,13 @@ def test_conv3x3_tensor_core_variant(env, M, C, Nb, p, B, H, Wd, variant):
     Y = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda(), b, True, layout="CNHW")
     plan.check()
     Yref, A = oracle.masked_conv3x3(L.W, L.mask, L.X, L.bias, relu=True)
-    check(Y.cpu().numpy(), Yref, A, L, tensor_core=True)
+    check(Y.cpu().numpy(), Yref, A, L, variant=plan.variant)
+    if plan.variant < 44 and M > 128:    # the same layer through the TF32 / the bf16 form explicitly
+        for v in (plan.variant, plan.variant + 4):
+            pv = ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb), v)
+            Yv = ubp.ubp_conv3x3_implicit(pv, torch.from_numpy(L.X).cuda(), b, True, layout="CNHW")
+            pv.check()
+            check(Yv.cpu().numpy(), Yref, A, L, variant=v)
     # NCHW output is not one [M][B*H*W] matrix: served by the plain kernel on the embedded sparse plan
     Yn = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda().permute(1, 0, 2, 3).contiguous(), b, True, layout="NCHW")
     check(Yn.permute(1, 0, 2, 3).contiguous().cpu().numpy(), Yref, A, L)
@@ -356,7 +383,7 @@ def test_r50_3x3_config_sampled(env):
     ys, as_ = oracle.masked_conv3x3_samples(L.W, L.mask, L.X, sb, so, sy, sx, L.bias, relu=True)
     err = scaled_error(Y[so, sb, sy, sx], ys, as_)
     n_terms = terms_per_output(L) + 2
-    assert err <= TOL and err <= (2.0 ** -18 + n_terms * 2.0 ** -23 if plan.variant >= 40 else n_terms * 2.0 ** -24)
+    assert err <= TOL and err <= arith_bound(L, plan.variant)
     # the plain 3x3 kernel on the same layer
     plan_s = ubp.Plan(blob, 20)
     Ys = ubp.ubp_conv3x3_implicit(plan_s, torch.from_numpy(L.X).cuda(), torch.from_numpy(L.bias).cuda(), True).cpu().numpy()
