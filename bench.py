@@ -438,15 +438,25 @@ def main():
     roof["frac_of_roofline_time"] = max(t_alu, t_hbm) / (step_ms * 1e-3)
     roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((name, plan.variant >= 30))
     kern, tile_rows, tile_cols = plan.tile_choice(L.Nc, L.Wd if L.R == 9 else 0)
+    bf16 = 34 <= plan.variant <= 37 or 44 <= plan.variant <= 47
     roof["kernel"] = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF32 on tcgen05, one CTA per tile)",
+                      "ubp_tc3_kernel (dense 3xBF16 on tcgen05, CTA pair per tile)" if bf16 else
                       "ubp_tc2_kernel (dense 3xTF32 on tcgen05, CTA pair per tile)")[kern]
+    roof["arithmetic"] = ("fp32 FMA, fp32 accumulate", "3 TF32 products per fp32 product, fp32 accumulate (error ~2^-20 |w||x|)",
+                          "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)" if bf16 else
+                          "3 TF32 products per fp32 product, fp32 accumulate (error ~2^-20 |w||x|)")[kern]
     roof["tile"] = [tile_rows, tile_cols]
     if plan.variant >= 30:
-        # the tensor-core variant does 3 x the DENSE multiply-adds; report that rate against the TF32 peak too
+        # the tensor-core variants do 3 x the DENSE multiply-adds; report that rate against the tensor peak of the
+        # operand type too (bf16: the measured cuBLAS figure; TF32: half of it, the nominal ratio)
         dense_tf = 3 * 2.0 * L.M * L.C * L.R * L.Nc / (step_ms * 1e-3) / 1e12
         tf32_peak = tf32_peak_tflops()
-        roof["tensor"] = {"dense_tf32_tflops": dense_tf, "peak": tf32_peak[0], "peak_source": tf32_peak[1],
-                          "frac": dense_tf / tf32_peak[0]}
+        if bf16 and kern == 2:
+            roof["tensor"] = {"dense_bf16_tflops": dense_tf, "peak": tf32_peak[0] * 2,
+                              "peak_source": tf32_peak[1].replace(" x 0.5", ""), "frac": dense_tf / (tf32_peak[0] * 2)}
+        else:
+            roof["tensor"] = {"dense_tf32_tflops": dense_tf, "peak": tf32_peak[0], "peak_source": tf32_peak[1],
+                              "frac": dense_tf / tf32_peak[0]}
 
     line = {
         "metric": "effective GFLOP/s (2 x surviving MACs / time) of one UBP layer", "value": gflops, "unit": "GFLOP/s",

@@ -395,17 +395,25 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
     if (M > 128 && conv_w >= 0 && (!conv || ((K / 9) % TC_KC == 0 && halo <= 64))) {
         double best2 = 1e300;
         int best2_n = 0;
-        for (int n = 64; n <= 256; n += 64) {
+        // tile widths: multiples of 64 for the TF32 kernel (X arrives in 32-column boxes per CTA), of 32 for the bf16
+        // kernel (whose only unit is the 32-column block of the epilogue)
+        for (int n = 64; n <= 256; n += bf16 ? 32 : 64) {
             if (conv && (n / 2 + 2 * halo > 256 || (bf16 ? tc_pair_bf16_stages(n, halo) : tc_pair_stages(n, halo)) < 4)) continue;
             const long long ntiles = (long long)((M + 255) / 256) * ((Nc + n - 1) / n);
             const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
             const long long per_pair = (ntiles + pairs - 1) / pairs;
-            // bf16 products: three MMAs of K = 16 per chunk (half the tensor-core time) and half the operand bytes
+            // bf16 products (calibrated the same way): three MMAs of K = 16 per chunk, n/2 cycles each; below that
+            // a floor of ~470 + n/3 cycles that is nearly flat in n - the copies (W in 32-byte row pieces, the raw
+            // fp32 rows) arrive at ~32 B/cycle/SM, the rate of the L2-to-SM path; 3x3: the shifted-tile pass
+            // (~700 + 0.6 n). A tile costs its chunks or its epilogue (~50 cycles per column) plus ~2500 cycles of
+            // hand-over between tiles.
             double per_chunk = bf16 ? 1.65 * n : 3.3 * n;
-            const double smem_chunk = bf16 ? (conv ? 220.0 + 1.5 * n : 190.0 + 1.2 * n) : (conv ? 560.0 + 1.0 * n : 500.0 + 0.5 * n);
+            const double smem_chunk = bf16 ? (conv ? 700.0 + 0.6 * n : 470.0 + 0.33 * n) : (conv ? 560.0 + 1.0 * n : 500.0 + 0.5 * n);
             if (per_chunk < smem_chunk) per_chunk = smem_chunk;
             double per_tile = nchunk * per_chunk;
-            if (per_tile < 45.0 * n) per_tile = 45.0 * n;
+            const double epi = bf16 ? 50.0 * n : 45.0 * n;
+            if (per_tile < epi) per_tile = epi;
+            if (bf16) per_tile += 2500.0;
             const double t = 4400.0 + (double)per_pair * per_tile + 4500.0 + 30.0 * n;
             if (t < best2) { best2 = t; best2_n = n; }
         }

@@ -32,7 +32,7 @@ constexpr int T3_XL_WARPS = 8;                            // warps 2..9: the spl
 constexpr int T3_XL_GROUPS = 2;                           // two groups of four warps take turns on the chunks
 constexpr int T3_EPI_WARPS = 8;                           // warps 10..17
 constexpr int T3_THREADS = (2 + T3_XL_WARPS + T3_EPI_WARPS) * 32;
-constexpr int T3_MAX_STAGES = 8;
+constexpr int T3_MAX_STAGES = 10;
 constexpr uint32_t T3_A_PART = 128 * TC_KC * 2;           // W1 or W2 chunk of this CTA's 128 rows: 4 KB
 constexpr uint32_t T3_ATOM = 64 * TC_KC * 2;              // x1 or x2 of 64 columns x 16 channels: 2 KB
 constexpr uint32_t T3_PIPE_BUDGET = 222 * 1024;
@@ -246,6 +246,9 @@ ubp_tc3_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         unsigned long long tap_lo = 0;                         // 3x3: bit tap * 8 + e (taps 0..7): tap inside the image
         uint32_t tap_hi = 0;                                   //      for column 8 cg + e; tap 8 in tap_hi
         int mask_tile = -1;
+        // 3x3: tile, chunk in the tile, tap and first channel in the tap of this group's current chunk (chunk grp)
+        int ti = nchunk > 0 ? grp / nchunk : 0, cc = nchunk > 0 ? grp % nchunk : 0;
+        int tp = CONV ? (cc * TC_KC) / Cin : 0, ch = CONV ? (cc * TC_KC) % Cin : 0;
         int st = grp;                                      // the stage count is even: stages grp, grp + 2, ...
         uint32_t ph = 0;
         for (int f = grp; f < total && ok; f += T3_XL_GROUPS) {
@@ -256,7 +259,6 @@ ubp_tc3_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             int sh = 0;
             uint32_t ok8 = 0xffu;
             if (CONV) {
-                const int ti = f / nchunk, c = f - ti * nchunk;
                 if (ti != mask_tile) {                     // new tile: which taps of my eight columns are inside the image
                     mask_tile = ti;
                     const int64_t n0 = tile_col0(ti) + (int64_t)rank * NH + 8 * cg;
@@ -274,9 +276,15 @@ ubp_tc3_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                         }
                     }
                 }
-                const int tp = (c * TC_KC) / Cin;
                 sh = (tp / 3 - 1) * a.W + (tp % 3 - 1) + halo;              // >= 0: offset into the raw rows
                 ok8 = tp < 8 ? (uint32_t)(tap_lo >> (tp * 8)) & 0xffu : tap_hi;
+                // this group's next chunk is two further on: keep (tile, chunk in tile, tap, channel in tap) by
+                // increments instead of divisions
+                for (int u = 0; u < T3_XL_GROUPS; ++u) {
+                    ch += TC_KC;
+                    if (ch >= Cin) { ch = 0; ++tp; }
+                    if (++cc == nchunk) { cc = 0; tp = 0; ch = 0; ++ti; }
+                }
             }
             if (mine) {
                 const int o = 8 * cg + sh, ob = o & ~3, r = o & 3;          // r is the same for every lane
