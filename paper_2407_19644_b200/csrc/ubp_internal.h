@@ -55,8 +55,9 @@ struct PlanImage {
     // kind 2 only: byte offset of the dense part (Wh [M][tc_kp] then Wl [M][tc_kp], floats) and its row length
     size_t tc_off = 0;
     int tc_kp = 0;
-    // and of the same weight as two bf16 pieces (W1 [M][tc16_kp] then W2 [M][tc16_kp], 16-bit words): W1 = the weight
-    // rounded to bf16, W2 = the remainder rounded to bf16
+    // and of the same weight as two bf16 pieces (W1 = the weight rounded to bf16, W2 = the remainder rounded to bf16),
+    // tiled: 8 KB blocks [row tile of 128][chunk of 16 channels] = [piece][128 rows][16 channels] in the 32-byte
+    // swizzle; tc16_kp = reduction length padded to whole chunks
     size_t tc16_off = 0;
     int tc16_kp = 0;
 };

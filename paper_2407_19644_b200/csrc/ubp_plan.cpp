@@ -159,9 +159,13 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         img.tc_kp = (C * R + 3) & ~3;       // reduction index k = tap * C + channel (tap-major)
         img.tc_off = total;
         total += ((size_t)2 * M * img.tc_kp * sizeof(float) + 255) & ~(size_t)255;
-        img.tc16_kp = (C * R + 7) & ~7;     // the same matrix as two bf16 pieces, rows of whole 16-byte groups
+        // The same matrix as two bf16 pieces, tiled for the CTA-pair kernel: one 8 KB block per (128-row tile,
+        // 16-channel chunk) = [piece W1, W2][128 rows][16 channels] exactly as the kernel wants it in shared memory
+        // (rows of 32 bytes whose two 16-byte halves are swapped on rows with bit 2 set: the 32-byte swizzle of a
+        // K-major operand), so that a chunk is ONE contiguous bulk copy instead of 256 row pieces.
+        img.tc16_kp = (C * R + 15) & ~15;   // padded reduction length: whole chunks
         img.tc16_off = total;
-        total += ((size_t)2 * M * img.tc16_kp * sizeof(uint16_t) + 255) & ~(size_t)255;
+        total += (size_t)((M + 255) / 256) * 2 * (img.tc16_kp / 16) * 8192;   // whole pairs of row tiles (zero rows pad)
     }
     if (bytes) *bytes = total;
     img.nkt = nkt; img.NP = NP; img.NG = NG; img.F = F; img.entries = entries; img.max_group_bytes = max_group;
@@ -234,8 +238,14 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         float *Wh = reinterpret_cast<float *>(base + img.tc_off);
         float *Wl = Wh + (size_t)M * img.tc_kp;
         // and into two bf16 pieces: the weight rounded to nearest-even bf16, and the (exact) remainder rounded
-        uint16_t *W1 = reinterpret_cast<uint16_t *>(base + img.tc16_off);
-        uint16_t *W2 = W1 + (size_t)M * img.tc16_kp;
+        uint8_t *W16 = base + img.tc16_off;
+        const size_t nchunk16 = (size_t)img.tc16_kp / 16;
+        auto w16_at = [&](int row, size_t k, int piece) -> uint16_t * {
+            const size_t blk = (size_t)(row / 128) * nchunk16 + k / 16;
+            const int i = row % 128, kk = (int)(k % 16);
+            return reinterpret_cast<uint16_t *>(W16 + blk * 8192 + (size_t)piece * 4096 + (size_t)i * 32 +
+                                                (size_t)(((kk >> 3) ^ ((i >> 2) & 1)) * 16) + (size_t)(kk & 7) * 2);
+        };
         auto bf16_rn = [](float f) -> uint16_t {
             uint32_t b;
             std::memcpy(&b, &f, 4);
@@ -268,8 +278,8 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
                     Wh[(size_t)(i + t) * img.tc_kp + (size_t)r * C + j] = hi;
                     Wl[(size_t)(i + t) * img.tc_kp + (size_t)r * C + j] = lo;
                     const uint16_t w1 = bf16_rn(w);
-                    W1[(size_t)(i + t) * img.tc16_kp + (size_t)r * C + j] = w1;
-                    W2[(size_t)(i + t) * img.tc16_kp + (size_t)r * C + j] = bf16_rn(w - bf16_f(w1));
+                    *w16_at(i + t, (size_t)r * C + j, 0) = w1;
+                    *w16_at(i + t, (size_t)r * C + j, 1) = bf16_rn(w - bf16_f(w1));
                   }
             }
     }

@@ -348,7 +348,7 @@ int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d
                    int64_t Nc, int ntile, int sms, void *stream);
 int tc_pair_stages(int ntile, int halo);
 // same pipeline with three bf16 products per fp32 product (ubp_tc3.cu)
-int launch_tc_pair_bf16(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int conv, int halo, const void *args,
+int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, int halo, const void *args,
                         int M, int64_t Nc, int ntile, int sms, void *stream);
 int tc_pair_bf16_stages(int ntile, int halo);
 
@@ -443,17 +443,12 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
     if (const char *e = getenv("UBP_TC_FORCE")) { int k = 0, n = 0; if (sscanf(e, "%d,%d", &k, &n) == 2) { kernel = k; best_n = n; rows = (k == 2 || k == 12) ? 256 : 128; if (k == 12) kernel = 1; } }
 #endif
     if (kernel == 2 && bf16) {
-        const uint16_t *W1 = reinterpret_cast<const uint16_t *>(dev + pl->img.tc16_off);
-        CUtensorMap tmW, tmX;
-        const uint64_t wdims[3] = {(uint64_t)pl->img.tc16_kp, (uint64_t)M, 2};
-        const uint32_t wbox[3] = {TC_KC, 128, 2};
-        if ((rc = encode_3d(&tmW, W1, wdims, (uint64_t)pl->img.tc16_kp * 2, (uint64_t)M * pl->img.tc16_kp * 2, wbox,
-                            CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16))) return rc;
+        CUtensorMap tmX;
         // the input as (column, channel): 16 channel rows of the CTA's columns per chunk, plus the halo for 3x3
         const int halo = a.conv ? (a.W + 1 + 3) & ~3 : 0;
         if ((rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)(a.conv ? K / 9 : K), (uint64_t)(a.conv ? a.isc : a.ldx) * 4,
                             (uint32_t)(best_n / 2 + 2 * halo), TC_KC, CU_TENSOR_MAP_SWIZZLE_NONE))) return rc;
-        return launch_tc_pair_bf16(&tmW, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream);
+        return launch_tc_pair_bf16(dev + pl->img.tc16_off, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream);
     }
     if (kernel == 2) {
         // Wh and Wl as one 3-D tensor (channel, row, part): one copy per chunk brings both

@@ -8,8 +8,8 @@
 // chunk takes three MMAs of K = 16 instead of six of K = 8 and its operands are half as many bytes: half the
 // tensor-core time and little more than half the shared-memory traffic, the two bounds of ubp_tc2.cu.
 //
-// Differences from ubp_tc2.cu: the plan supplies W1 / W2 (bf16, K-major; TMA box 16 x 128 x 2 in the 32-byte
-// swizzle); the tensor core cannot take the raw fp32 activations any more, so TMA copies the chunk's 16 channel rows
+// Differences from ubp_tc2.cu: the plan supplies W1 / W2 (bf16, K-major, 32-byte swizzle) already tiled into the
+// 8 KB blocks a chunk needs, so a chunk's weights are one contiguous bulk copy; the tensor core cannot take the raw fp32 activations any more, so TMA copies the chunk's 16 channel rows
 // as they are (plus a halo for 3x3) and the pass warps write BOTH x1 and x2, in the MN-major bf16 operand layout
 // (64 columns x 8 channels atoms in the 128-byte swizzle; LBO = next 64 columns, SBO = next 8 channels). Thread
 // roles, barriers, persistence, the two accumulators and the epilogue are those of ubp_tc2.cu.
@@ -109,7 +109,7 @@ __device__ __forceinline__ void split8(const float (&v)[8], uint4 &h, uint4 &l)
 
 template <bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T3_THREADS, 1)
-ubp_tc3_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const TcArgs a,
+ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensorMap tmX, const TcArgs a,
                const int halo, const int nrp, const int ntiles)
 {
     constexpr int MAXS = T3_MAX_STAGES;
@@ -139,18 +139,19 @@ ubp_tc3_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     auto tile_row0 = [&](int i) { return ((pair + i * npairs) % nrp) * 256 + (int)rank * 128; };
     auto tile_col0 = [&](int i) { return (int64_t)((pair + i * npairs) / nrp) * N; };
 
-    // one chunk's copies: W1 and W2 rows of this CTA in one 3-D box; 16 channel rows of the input for this CTA's
-    // columns (3x3: the channels of the chunk's tap, and a halo of columns either side)
+    // one chunk's copies: the W1 / W2 block of this CTA's 128 rows (8 KB, stored in the plan exactly as it must lie in
+    // shared memory: one contiguous bulk copy; as a tensor box it was 256 row pieces, and the ~2 cycles the copy
+    // engine needs per piece were what bounded a chunk); 16 channel rows of the input for this CTA's columns
+    // (3x3: the channels of the chunk's tap, and a halo of columns either side)
     auto issue_chunk = [&](int c, int st, int row0, int xcol) {
         uint8_t *stage = smem + (size_t)st * stage_bytes;
         const uint32_t bar = smem_u32(&bar_full[st]);
         mbar_expect_tx(bar, tx);
-        tma_load_3d(smem_u32(stage), &tmW, c * TC_KC, row0, 0, bar);
+        bulk_load(smem_u32(stage), W16 + ((size_t)(row0 >> 7) * nchunk + c) * (2 * T3_A_PART), 2 * T3_A_PART, bar);
         tma_load_2d(smem_u32(stage + 2 * T3_A_PART + 2 * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
     };
 
     if (threadIdx.x == 0) {
-        prefetch_tensormap(&tmW);
         prefetch_tensormap(&tmX);
         abort_flag = 0;
         for (int s = 0; s < S; ++s) {
@@ -360,10 +361,10 @@ ubp_tc3_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 }  // namespace
 
 // Launch the bf16 pair kernel on tiles of 256 rows x `ntile` columns (a multiple of 64).
-// tmW: 3-D map over the plan's bf16 part (channel, row, {W1, W2}), box 16 x 128 x 2, 32-byte swizzle.
+// W16: the plan's bf16 part: 8 KB blocks [row tile of 128][chunk] = [W1, W2][128 rows][16 channels], pre-swizzled.
 // tmX: plain 2-D fp32 map (column, channel), box (ntile/2 + 2 halo) x 16; halo = 0 for 1x1, image width + 1
 // rounded up to a multiple of 4 for 3x3 (columns = the flattened (b, y, x) axis).
-int launch_tc_pair_bf16(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int conv, int halo, const void *args_,
+int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, int halo, const void *args_,
                         int M, int64_t Nc, int ntile, int sms, void *stream)
 {
     TcArgs a = *static_cast<const TcArgs *>(args_);
@@ -389,9 +390,9 @@ int launch_tc_pair_bf16(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, in
     const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
     const dim3 grid((unsigned)(2 * pairs));
     if (conv)
-        ubp_tc3_kernel<true><<<grid, T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(*tmW, *tmX, a, halo, nrp, (int)ntiles);
+        ubp_tc3_kernel<true><<<grid, T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint8_t *>(W16), *tmX, a, halo, nrp, (int)ntiles);
     else
-        ubp_tc3_kernel<false><<<grid, T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(*tmW, *tmX, a, halo, nrp, (int)ntiles);
+        ubp_tc3_kernel<false><<<grid, T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint8_t *>(W16), *tmX, a, halo, nrp, (int)ntiles);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
     return UBP_OK;

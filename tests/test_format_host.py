@@ -163,9 +163,10 @@ def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     img, geom = ubp.plan_image(blob, variant)
     tc_off = ubp.plan_size(blob, sparse_variant)             # same geometry without the dense part
     kp = (C * R + 3) // 4 * 4
-    kp16 = (C * R + 7) // 8 * 8
+    kp16 = (C * R + 15) // 16 * 16
     tc16_off = tc_off + (2 * M * kp * 4 + 255) // 256 * 256
-    assert len(img) == tc16_off + (2 * M * kp16 * 2 + 255) // 256 * 256
+    nrt, nch = (M + 255) // 256 * 2, kp16 // 16                # whole pairs of 128-row tiles
+    assert len(img) == tc16_off + nrt * nch * 8192
     # the embedded sparse plan is byte-identical to the stand-alone one
     img_s, _ = ubp.plan_image(blob, sparse_variant)
     assert np.array_equal(img[:tc_off], img_s)
@@ -180,8 +181,17 @@ def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     assert np.array_equal(Wh[:, :C * R], (Wm.view(np.uint32) & 0xffffe000).view(np.float32))
     # the same matrix as two bf16 pieces (8-bit significands): W1 = nearest bf16, so |W - W1| <= 2^-8 |W|, and
     # W1 + W2 within 2^-16 |W|
-    W1 = (np.frombuffer(img, "<u2", M * kp16, tc16_off).reshape(M, kp16).astype(np.uint32) << 16).view(np.float32)
-    W2 = (np.frombuffer(img, "<u2", M * kp16, tc16_off + 2 * M * kp16).reshape(M, kp16).astype(np.uint32) << 16).view(np.float32)
+    # tiled: 8 KB blocks [row tile][chunk] = [piece][128 rows][16 channels], rows of 32 bytes whose 16-byte halves
+    # are swapped on rows with bit 2 set
+    blocks = np.frombuffer(img, "<u2", nrt * nch * 4096, tc16_off).reshape(nrt, nch, 2, 128, 2, 8)
+    rows = np.arange(128)
+    swap = ((rows >> 2) & 1).astype(bool)
+    blocks = blocks.copy()
+    blocks[:, :, :, swap] = blocks[:, :, :, swap][..., ::-1, :]
+    W12 = blocks.reshape(nrt, nch, 2, 128, 16).transpose(2, 0, 3, 1, 4).reshape(2, nrt * 128, kp16)
+    assert not W12[:, M:].any()                                # padding rows
+    W1 = (W12[0, :M].astype(np.uint32) << 16).view(np.float32)
+    W2 = (W12[1, :M].astype(np.uint32) << 16).view(np.float32)
     assert not W1[:, C * R:].any() and not W2[:, C * R:].any()
     assert np.all(np.abs(W1[:, :C * R].astype(np.float64) - Wm) <= np.abs(Wm) * 2.0 ** -8)
     got16 = W1[:, :C * R].astype(np.float64) + W2[:, :C * R]
