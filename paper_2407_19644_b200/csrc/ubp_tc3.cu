@@ -32,14 +32,15 @@ constexpr int T3_XL_WARPS = 8;                            // warps 2..9: the spl
 constexpr int T3_XL_GROUPS = 2;                           // two groups of four warps take turns on the chunks
 constexpr int T3_EPI_WARPS = 8;                           // warps 10..17
 constexpr int T3_THREADS = (2 + T3_XL_WARPS + T3_EPI_WARPS) * 32;
-constexpr int T3_MAX_STAGES = 10;
+constexpr int T3_MAX_STAGES = 8;
+constexpr int T3_MAX_SUB = 2;                             // 16-channel chunks per pipeline stage: 1 or 2 (chosen per launch)
 constexpr uint32_t T3_A_PART = 128 * TC_KC * 2;           // W1 or W2 chunk of this CTA's 128 rows: 4 KB
 constexpr uint32_t T3_ATOM = 64 * TC_KC * 2;              // x1 or x2 of 64 columns x 16 channels: 2 KB
 constexpr uint32_t T3_PIPE_BUDGET = 222 * 1024;
 constexpr uint32_t SWZ_32B = 6, SWZ_128B = 2;             // descriptor layout types
 constexpr uint32_t T3_ACC_COLS = 256;                     // tensor-memory columns per accumulator
 
-// a stage = W1 + W2 chunk (8 KB) + x1 + x2 tiles (2 KB per started 64 columns each) + the raw fp32 rows
+// a chunk = W1 + W2 block (8 KB) + x1 + x2 tiles (2 KB per started 64 columns each) + the raw fp32 rows
 // (16 channels x (columns + 2 x halo) floats, padded to 1 KB). The stage count is a multiple of the group count so
 // that a stage always belongs to the same group of pass warps (a waiter must see every phase of its barrier).
 __host__ __device__ constexpr uint32_t t3_x_bytes(int nh) { return (uint32_t)((nh + 63) / 64) * T3_ATOM; }
@@ -47,13 +48,19 @@ __host__ __device__ constexpr uint32_t t3_raw_bytes(int nh, int halo)
 {
     return ((uint32_t)(nh + 2 * halo) * TC_KC * 4 + 1023u) & ~1023u;
 }
-__host__ __device__ constexpr uint32_t t3_stage_bytes(int nh, int halo)
+// one chunk's part of a stage
+__host__ __device__ constexpr uint32_t t3_chunk_bytes(int nh, int halo)
 {
     return 2 * T3_A_PART + 2 * t3_x_bytes(nh) + t3_raw_bytes(nh, halo);
 }
-__host__ __device__ constexpr int t3_stages(int nh, int halo)
+// A stage holds `sub` chunks. With two, every barrier round trip (copies landed -> split pass -> MMA issue -> stage
+// free) serves 32 channels: fewer waits per channel, which pays on long reductions (3x3: 144 chunks; 1024 channels)
+// where the pass or the issue thread is the bound; with one, the pipeline fills and drains in finer steps, which
+// pays on short reductions (512 channels: 32 chunks).
+__host__ __device__ constexpr uint32_t t3_stage_bytes(int nh, int halo, int sub) { return (uint32_t)sub * t3_chunk_bytes(nh, halo); }
+__host__ __device__ constexpr int t3_stages(int nh, int halo, int sub)
 {
-    const int s = (int)(T3_PIPE_BUDGET / t3_stage_bytes(nh, halo));
+    const int s = (int)(T3_PIPE_BUDGET / t3_stage_bytes(nh, halo, sub));
     return (s > T3_MAX_STAGES ? T3_MAX_STAGES : s) / T3_XL_GROUPS * T3_XL_GROUPS;
 }
 
@@ -63,18 +70,21 @@ __device__ __forceinline__ uint32_t make_idesc3(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
-// One chunk's three MMAs (K = 16 each: w1 x1, w2 x1, w1 x2) and the commit that hands the stage back to both CTAs,
-// in a single statement, with a non-blocking test of the NEXT chunk's barrier issued first and its result read
-// last. Executed by a whole converged warp: one elected lane issues. Returns whether the next chunk is ready.
+// One chunk's three MMAs (K = 16 each: w1 x1, w2 x1, w1 x2) and, after a stage's last chunk (`last`), the commit that
+// hands the stage back to both CTAs, in a single statement, with a non-blocking test of the NEXT stage's barrier
+// issued first and its result read last. Executed by a whole converged warp: one elected lane issues. Returns
+// whether the next stage is ready.
 __device__ __forceinline__ bool mma3_chunk(uint32_t d_tmem, uint64_t dW1, uint64_t dX1, uint32_t w2_off, uint32_t x2_off,
                                            uint32_t idesc, uint32_t acc_first, uint32_t next_bar, uint32_t next_parity,
-                                           uint32_t empty_bar)
+                                           uint32_t empty_bar, uint32_t last)
 {
     uint32_t ready;
     asm volatile(
-        "{\n\t.reg .pred pn, pa, pt, pe;\n\t.reg .b64 w2, x2;\n\t"
+        "{\n\t.reg .pred pn, pa, pt, pe, pc;\n\t.reg .b64 w2, x2;\n\t"
         "mbarrier.test_wait.parity.shared::cta.b64 pn, [%8], %9;\n\t"
         "elect.sync _|pe, 0xffffffff;\n\t"
+        "setp.ne.b32 pc, %13, 0;\n\t"
+        "and.pred pc, pc, pe;\n\t"
         "setp.ne.b32 pa, %7, 0;\n\t"
         "setp.eq.b32 pt, %10, 0;\n\t"
         "cvt.u64.u32 w2, %4;\n\tadd.s64 w2, w2, %2;\n\t"
@@ -82,11 +92,11 @@ __device__ __forceinline__ bool mma3_chunk(uint32_t d_tmem, uint64_t dW1, uint64
         "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %6, pa;\n\t"
         "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w2, %3, %6, pt;\n\t"
         "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, x2, %6, pt;\n\t"
-        "@pe tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%11], %12;\n\t"
+        "@pc tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%11], %12;\n\t"
         "selp.u32 %0, 1, 0, pn;\n\t}"
         : "=r"(ready)
         : "r"(d_tmem), "l"(dW1), "l"(dX1), "r"(w2_off), "r"(x2_off), "r"(idesc), "r"(acc_first), "r"(next_bar),
-          "r"(next_parity), "r"(0u), "r"(empty_bar), "h"((uint16_t)3)
+          "r"(next_parity), "r"(0u), "r"(empty_bar), "h"((uint16_t)3), "r"(last)
         : "memory");
     return ready != 0;
 }
@@ -107,7 +117,7 @@ __device__ __forceinline__ void split8(const float (&v)[8], uint4 &h, uint4 &l)
     l = make_uint4(ll[0], ll[1], ll[2], ll[3]);
 }
 
-template <bool CONV>
+template <bool CONV, int SUB>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T3_THREADS, 1)
 ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensorMap tmX, const TcArgs a,
                const int halo, const int nrp, const int ntiles)
@@ -126,12 +136,13 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();
     const int N = a.ntile, NH = N / 2;                     // tile columns; columns whose X this CTA holds
-    const uint32_t xb = t3_x_bytes(NH);                    // x1 (and x2) bytes per stage
-    const uint32_t stage_bytes = t3_stage_bytes(NH, halo);
+    const uint32_t xb = t3_x_bytes(NH);                    // x1 (and x2) bytes per chunk
+    const uint32_t chunk_bytes = t3_chunk_bytes(NH, halo), stage_bytes = (uint32_t)SUB * chunk_bytes;
     const uint32_t raw_row = (uint32_t)(NH + 2 * halo) * 4;   // bytes per channel row of the raw copy
-    const int S = t3_stages(NH, halo);
+    const int S = t3_stages(NH, halo, SUB);
     const int nchunk = (a.K + TC_KC - 1) / TC_KC;
-    const uint32_t tx = 2 * T3_A_PART + raw_row * TC_KC;
+    const int nstage = (nchunk + SUB - 1) / SUB;     // stages per tile; the last one may hold a single chunk
+    const uint32_t tx = 2 * T3_A_PART + raw_row * TC_KC;   // bytes copied per chunk
     const int Cin = CONV ? a.K / 9 : a.K;                  // 3x3: reduction index k = tap * Cin + channel, Cin % 16 == 0
     // this pair's tiles: pair, pair + npairs, ...; tile t = (row pair t % nrp, column tile t / nrp)
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
@@ -139,16 +150,22 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     auto tile_row0 = [&](int i) { return ((pair + i * npairs) % nrp) * 256 + (int)rank * 128; };
     auto tile_col0 = [&](int i) { return (int64_t)((pair + i * npairs) / nrp) * N; };
 
-    // one chunk's copies: the W1 / W2 block of this CTA's 128 rows (8 KB, stored in the plan exactly as it must lie in
-    // shared memory: one contiguous bulk copy; as a tensor box it was 256 row pieces, and the ~2 cycles the copy
-    // engine needs per piece were what bounded a chunk); 16 channel rows of the input for this CTA's columns
-    // (3x3: the channels of the chunk's tap, and a halo of columns either side)
-    auto issue_chunk = [&](int c, int st, int row0, int xcol) {
-        uint8_t *stage = smem + (size_t)st * stage_bytes;
+    // one stage's copies (stage sg of a tile = chunks sg * SUB ...): per chunk the W1 / W2 block of this CTA's 128
+    // rows (8 KB, stored in the plan exactly as it must lie in shared memory: one contiguous bulk copy) and 16
+    // channel rows of the input for this CTA's columns (3x3: the channels of the chunk's tap, and a halo of columns
+    // either side)
+    auto issue_stage = [&](int sg, int st, int row0, int xcol) {
         const uint32_t bar = smem_u32(&bar_full[st]);
-        mbar_expect_tx(bar, tx);
-        bulk_load(smem_u32(stage), W16 + ((size_t)(row0 >> 7) * nchunk + c) * (2 * T3_A_PART), 2 * T3_A_PART, bar);
-        tma_load_2d(smem_u32(stage + 2 * T3_A_PART + 2 * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
+        const int c0 = sg * SUB, nsub = nchunk - c0 < SUB ? nchunk - c0 : SUB;
+        mbar_expect_tx(bar, (uint32_t)nsub * tx);
+#pragma unroll
+        for (int u = 0; u < SUB; ++u) {
+            if (u >= nsub) break;
+            const int c = c0 + u;
+            uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
+            bulk_load(smem_u32(chunk), W16 + ((size_t)(row0 >> 7) * nchunk + c) * (2 * T3_A_PART), 2 * T3_A_PART, bar);
+            tma_load_2d(smem_u32(chunk + 2 * T3_A_PART + 2 * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
+        }
     };
 
     if (threadIdx.x == 0) {
@@ -168,7 +185,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         // the first copy lands in this CTA's own memory and signals its own barrier: start it before the
         // tensor-memory allocation and the cluster barrier
-        if (nmy > 0) issue_chunk(0, 0, tile_row0(0), (int)(tile_col0(0) + (int64_t)rank * NH));
+        if (nmy > 0) issue_stage(0, 0, tile_row0(0), (int)(tile_col0(0) + (int64_t)rank * NH));
     }
     if (warp == 1) {   // tensor memory of the pair: the same warp of both CTAs allocates
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -185,15 +202,15 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     if (warp == 0) {
         // ---------------- TMA producer: one ring of S stages straight through all of this pair's tiles
         if (lane == 0) {
-            int st = 1 % S, round = 1 / S;                 // chunk (0, 0) was started above
+            int st = 1 % S, round = 1 / S;                 // stage 0 of the first tile was started above
             for (int i = 0; i < nmy && ok; ++i) {
                 const int row0 = tile_row0(i), xcol = (int)(tile_col0(i) + (int64_t)rank * NH);
-                for (int c = (i == 0 ? 1 : 0); c < nchunk; ++c) {
+                for (int sg = (i == 0 ? 1 : 0); sg < nstage; ++sg) {
                     if (round > 0) {                       // the stage's previous contents must have been consumed
                         ok = mbar_wait_relaxed(smem_u32(&bar_empty[st]), (uint32_t)(round - 1) & 1u, &abort_flag);
                         if (!ok) break;
                     }
-                    issue_chunk(c, st, row0, xcol);
+                    issue_stage(sg, st, row0, xcol);
                     if (++st == S) { st = 0; ++round; }
                 }
             }
@@ -204,7 +221,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             const uint32_t idesc = make_idesc3(N);
             const uint64_t dW0 = make_desc(smem_u32(smem), 16, 256, SWZ_32B);
             const uint64_t dX0 = make_desc(smem_u32(smem) + 2 * T3_A_PART, 2048, 1024, SWZ_128B);
-            const uint32_t stage_u = stage_bytes >> 4;
+            const uint32_t stage_u = stage_bytes >> 4, chunk_u = chunk_bytes >> 4;
             int st = 0;
             uint32_t ph = 0;
             bool ready = nmy > 0 && mbar_try_wait(smem_u32(&bar_go[0]), 0);
@@ -215,7 +232,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                     ok = mbar_wait(smem_u32(&bar_acc_empty[b]), (uint32_t)((i >> 1) - 1) & 1u, &abort_flag);
                     if (!ok) break;
                 }
-                for (int c = 0; c < nchunk; ++c) {
+                for (int sg = 0; sg < nstage; ++sg) {
                     if (!ready) ok = mbar_wait(smem_u32(&bar_go[st]), ph, &abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -223,8 +240,12 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                     int nst = st + 1;
                     uint32_t nph = ph;
                     if (nst == S) { nst = 0; nph ^= 1u; }
-                    ready = mma3_chunk(acc, dW0 + soff, dX0 + soff, T3_A_PART >> 4, xb >> 4, idesc, c > 0 ? 1u : 0u,
-                                       smem_u32(&bar_go[nst]), nph, smem_u32(&bar_empty[st]));
+                    const int nsub = nchunk - sg * SUB < SUB ? nchunk - sg * SUB : SUB;
+#pragma unroll
+                    for (int u = 0; u < SUB; ++u)
+                        if (u < nsub) ready = mma3_chunk(acc, dW0 + soff + (uint64_t)(u * chunk_u), dX0 + soff + (uint64_t)(u * chunk_u),
+                                           T3_A_PART >> 4, xb >> 4, idesc, (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
+                                           smem_u32(&bar_empty[st]), u == nsub - 1 ? 1u : 0u);
                     st = nst; ph = nph;
                 }
                 if (!ok) break;
@@ -241,78 +262,87 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         const int gt = (int)threadIdx.x - 64 - grp * GT;
         const int cg = gt & 15, kq = gt >> 4;
         const bool mine = cg * 8 < NH;
-        const int total = nmy * nchunk;
+        const int total = nmy * nstage;
         const uint32_t dst = (uint32_t)(cg >> 3) * T3_ATOM;   // 64-column atom; inside it row k is 128 bytes whose
         const uint32_t c16 = (uint32_t)(cg & 7);              // 16-byte pieces are XOR-swizzled with k mod 8
         unsigned long long tap_lo = 0;                         // 3x3: bit tap * 8 + e (taps 0..7): tap inside the image
         uint32_t tap_hi = 0;                                   //      for column 8 cg + e; tap 8 in tap_hi
         int mask_tile = -1;
-        // 3x3: tile, chunk in the tile, tap and first channel in the tap of this group's current chunk (chunk grp)
-        int ti = nchunk > 0 ? grp / nchunk : 0, cc = nchunk > 0 ? grp % nchunk : 0;
-        int tp = CONV ? (cc * TC_KC) / Cin : 0, ch = CONV ? (cc * TC_KC) % Cin : 0;
+        // tile and stage in the tile of this group's current stage; 3x3: tap and first channel of its first chunk,
+        // kept by increments (a division per chunk is what the pass cannot afford)
+        int ti = grp / nstage, sg = grp % nstage;
+        int tp = CONV ? (sg * SUB * TC_KC) / Cin : 0, ch = CONV ? (sg * SUB * TC_KC) % Cin : 0;
         int st = grp;                                      // the stage count is even: stages grp, grp + 2, ...
         uint32_t ph = 0;
         for (int f = grp; f < total && ok; f += T3_XL_GROUPS) {
             ok = mbar_wait_relaxed(smem_u32(&bar_full[st]), ph, &abort_flag);
             if (!ok) break;
-            uint8_t *x1 = smem + (size_t)st * stage_bytes + 2 * T3_A_PART;
-            const uint8_t *raw = x1 + 2 * xb;
-            int sh = 0;
-            uint32_t ok8 = 0xffu;
-            if (CONV) {
-                if (ti != mask_tile) {                     // new tile: which taps of my eight columns are inside the image
-                    mask_tile = ti;
-                    const int64_t n0 = tile_col0(ti) + (int64_t)rank * NH + 8 * cg;
-                    const int hw = a.H * a.W;
-                    tap_lo = 0; tap_hi = 0;
-                    for (int e = 0; e < 8; ++e) {
-                        const int64_t n = n0 + e;
-                        if (!mine || n >= a.Nc) continue;
-                        const int pix = (int)(n % hw), y = pix / a.W, x = pix - y * a.W;
-                        for (int tp = 0; tp < 9; ++tp) {
-                            const int yy = y + tp / 3 - 1, xx = x + tp % 3 - 1;
-                            if (yy >= 0 && yy < a.H && xx >= 0 && xx < a.W) {
-                                if (tp < 8) tap_lo |= 1ull << (tp * 8 + e); else tap_hi |= 1u << e;
-                            }
+            if (CONV && ti != mask_tile) {                 // new tile: which taps of my eight columns are inside the image
+                mask_tile = ti;
+                const int64_t n0 = tile_col0(ti) + (int64_t)rank * NH + 8 * cg;
+                const int hw = a.H * a.W;
+                tap_lo = 0; tap_hi = 0;
+                for (int e = 0; e < 8; ++e) {
+                    const int64_t n = n0 + e;
+                    if (!mine || n >= a.Nc) continue;
+                    const int pix = (int)(n % hw), y = pix / a.W, x = pix - y * a.W;
+                    for (int t9 = 0; t9 < 9; ++t9) {
+                        const int yy = y + t9 / 3 - 1, xx = x + t9 % 3 - 1;
+                        if (yy >= 0 && yy < a.H && xx >= 0 && xx < a.W) {
+                            if (t9 < 8) tap_lo |= 1ull << (t9 * 8 + e); else tap_hi |= 1u << e;
                         }
                     }
                 }
-                sh = (tp / 3 - 1) * a.W + (tp % 3 - 1) + halo;              // >= 0: offset into the raw rows
-                ok8 = tp < 8 ? (uint32_t)(tap_lo >> (tp * 8)) & 0xffu : tap_hi;
-                // this group's next chunk is two further on: keep (tile, chunk in tile, tap, channel in tap) by
-                // increments instead of divisions
-                for (int u = 0; u < T3_XL_GROUPS; ++u) {
-                    ch += TC_KC;
-                    if (ch >= Cin) { ch = 0; ++tp; }
-                    if (++cc == nchunk) { cc = 0; tp = 0; ch = 0; ++ti; }
+            }
+            const int nsub = nchunk - sg * SUB < SUB ? nchunk - sg * SUB : SUB;
+            int tpu = tp, chu = ch;                        // 3x3: tap / channel of chunk u of the stage
+#pragma unroll
+            for (int u = 0; u < SUB; ++u) {
+                if (u >= nsub) break;
+                uint8_t *x1 = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes + 2 * T3_A_PART;
+                const uint8_t *raw = x1 + 2 * xb;
+                int sh = 0;
+                uint32_t ok8 = 0xffu;
+                if (CONV) {
+                    sh = (tpu / 3 - 1) * a.W + (tpu % 3 - 1) + halo;        // >= 0: offset into the raw rows
+                    ok8 = tpu < 8 ? (uint32_t)(tap_lo >> (tpu * 8)) & 0xffu : tap_hi;
+                    chu += TC_KC;
+                    if (chu >= Cin) { chu = 0; ++tpu; }
+                }
+                if (mine) {
+                    const int o = 8 * cg + sh, ob = o & ~3, r = o & 3;      // r is the same for every lane
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const int k = kq + 8 * i;
+                        const float4 q0 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4);
+                        const float4 q1 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 16);
+                        float v[8];
+                        if (!CONV || r == 0) {
+                            v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w; v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+                        } else {
+                            const float4 q2 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 32);
+                            const float t[12] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w, q2.x, q2.y, q2.z, q2.w};
+                            if (r == 1) { for (int e = 0; e < 8; ++e) v[e] = t[e + 1]; }
+                            else if (r == 2) { for (int e = 0; e < 8; ++e) v[e] = t[e + 2]; }
+                            else { for (int e = 0; e < 8; ++e) v[e] = t[e + 3]; }
+                        }
+                        if (CONV) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) if (!((ok8 >> e) & 1u)) v[e] = 0.f;
+                        }
+                        uint4 h, l;
+                        split8(v, h, l);
+                        const uint32_t off = dst + (uint32_t)k * 128u + ((c16 ^ ((uint32_t)k & 7u)) << 4);
+                        *reinterpret_cast<uint4 *>(x1 + off) = h;
+                        *reinterpret_cast<uint4 *>(x1 + xb + off) = l;
+                    }
                 }
             }
-            if (mine) {
-                const int o = 8 * cg + sh, ob = o & ~3, r = o & 3;          // r is the same for every lane
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const int k = kq + 8 * i;
-                    const float4 q0 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4);
-                    const float4 q1 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 16);
-                    float v[8];
-                    if (!CONV || r == 0) {
-                        v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w; v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
-                    } else {
-                        const float4 q2 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 32);
-                        const float t[12] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w, q2.x, q2.y, q2.z, q2.w};
-                        if (r == 1) { for (int e = 0; e < 8; ++e) v[e] = t[e + 1]; }
-                        else if (r == 2) { for (int e = 0; e < 8; ++e) v[e] = t[e + 2]; }
-                        else { for (int e = 0; e < 8; ++e) v[e] = t[e + 3]; }
-                    }
-                    if (CONV) {
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) if (!((ok8 >> e) & 1u)) v[e] = 0.f;
-                    }
-                    uint4 h, l;
-                    split8(v, h, l);
-                    const uint32_t off = dst + (uint32_t)k * 128u + ((c16 ^ ((uint32_t)k & 7u)) << 4);
-                    *reinterpret_cast<uint4 *>(x1 + off) = h;
-                    *reinterpret_cast<uint4 *>(x1 + xb + off) = l;
+            // this group's next stage is T3_XL_GROUPS stages on
+            for (int g = 0; g < T3_XL_GROUPS; ++g) {
+                if (++sg == nstage) { sg = 0; ++ti; tp = 0; ch = 0; }
+                else if (CONV) {
+                    for (int u = 0; u < SUB; ++u) { ch += TC_KC; if (ch >= Cin) { ch = 0; ++tp; } }
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the writes visible to the MMA unit
@@ -370,16 +400,18 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     TcArgs a = *static_cast<const TcArgs *>(args_);
     a.ntile = ntile;
     const int nh = ntile / 2;
-    const size_t smem = (size_t)t3_stages(nh, halo) * t3_stage_bytes(nh, halo) + 1024;
-    static bool done[2][64] = {};
+    // chunks per stage: two on long reductions (48 chunks and more), else one
+    const int sub = (a.K + TC_KC - 1) / TC_KC >= 48 && t3_stages(nh, halo, 2) >= 4 ? 2 : 1;
+    const size_t smem = (size_t)t3_stages(nh, halo, sub) * t3_stage_bytes(nh, halo, sub) + 1024;
+    static bool done[4][64] = {};
     int devid = 0;
     if (cudaGetDevice(&devid) != cudaSuccess) devid = -1;
-    const int which = conv ? 1 : 0;
+    const int which = (conv ? 2 : 0) + (sub == 2 ? 1 : 0);
+    using KernelFn = void (*)(const uint8_t *, const CUtensorMap, const TcArgs, const int, const int, const int);
+    const KernelFn kernels[4] = {ubp_tc3_kernel<false, 1>, ubp_tc3_kernel<false, 2>, ubp_tc3_kernel<true, 1>, ubp_tc3_kernel<true, 2>};
+    const KernelFn kern = kernels[which];
     if (devid < 0 || devid >= 64 || !done[which][devid]) {
-        cudaError_t e = conv ? cudaFuncSetAttribute(ubp_tc3_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                    (int)(T3_PIPE_BUDGET + 1024))
-                             : cudaFuncSetAttribute(ubp_tc3_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                    (int)(T3_PIPE_BUDGET + 1024));
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(T3_PIPE_BUDGET + 1024));
         if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
         if (devid >= 0 && devid < 64) done[which][devid] = true;
     }
@@ -388,17 +420,14 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     if (ntiles <= 0) return UBP_OK;
     if (ntiles > 0x7fffffffll) return UBP_E_UNSUPPORTED;
     const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
-    const dim3 grid((unsigned)(2 * pairs));
-    if (conv)
-        ubp_tc3_kernel<true><<<grid, T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint8_t *>(W16), *tmX, a, halo, nrp, (int)ntiles);
-    else
-        ubp_tc3_kernel<false><<<grid, T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint8_t *>(W16), *tmX, a, halo, nrp, (int)ntiles);
+    kern<<<dim3((unsigned)(2 * pairs)), T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint8_t *>(W16), *tmX, a, halo, nrp, (int)ntiles);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
     return UBP_OK;
 }
 
 // how many pipeline stages the bf16 pair kernel gets for a tile width and halo
-int tc_pair_bf16_stages(int ntile, int halo) { return t3_stages(ntile / 2, halo); }
+int tc_pair_bf16_stages(int ntile, int halo) { return t3_stages(ntile / 2, halo, 1); }
 
 }  // namespace ubp
