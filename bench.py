@@ -73,12 +73,15 @@ def tf32_peak_tflops():
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (key: workload, tensor-core variant?)
+# summarised under profiles/ (key: workload, plan variant)
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("mbv1_pw512", True): 14984448 + 256,        # profiles/ncu_ubp_tc2_kernel_mbv1_pw512.md (the output is still in L2)
-    ("sweep_nb4_p70", True): 124626432 + 48126208,   # profiles/ncu_ubp_tc2_kernel_sweep_nb4_p70.md
-    ("r50_3x3", True): 17614080 + 0,             # profiles/ncu_ubp_tc2_kernel_r50_3x3.md
-    ("sweep_nb4_p90", False): 70554368 + 23536640,   # profiles/ncu_ubp_spmm_kernel_sweep_nb4_p90.md
+    ("mbv1_pw512", 36): 13933568 + 512,          # profiles/ncu_ubp_tc3_kernel_mbv1_pw512.md (the output is still in L2)
+    ("sweep_nb4_p70", 36): 84903936 + 40135680,  # profiles/ncu_ubp_tc3_kernel_sweep_nb4_p70.md
+    ("r50_3x3", 44): 15257344 + 1280,            # profiles/ncu_ubp_tc3_kernel_r50_3x3.md
+    ("mbv1_pw512", 32): 14984448 + 256,          # profiles/ncu_ubp_tc2_kernel_mbv1_pw512.md
+    ("sweep_nb4_p70", 32): 124626432 + 48126208, # profiles/ncu_ubp_tc2_kernel_sweep_nb4_p70.md
+    ("r50_3x3", 40): 17614080 + 0,               # profiles/ncu_ubp_tc2_kernel_r50_3x3.md
+    ("sweep_nb4_p90", 14): 70554368 + 23536640,  # profiles/ncu_ubp_spmm_kernel_sweep_nb4_p90.md
 }
 
 
@@ -436,7 +439,7 @@ def main():
                 "traffic": None, "peak_source": f"{peak_src} copy bandwidth"}
     roof["roofline_us"] = max(t_alu, t_hbm) * 1e6
     roof["frac_of_roofline_time"] = max(t_alu, t_hbm) / (step_ms * 1e-3)
-    roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((name, plan.variant >= 30))
+    roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((name, plan.variant))
     kern, tile_rows, tile_cols = plan.tile_choice(L.Nc, L.Wd if L.R == 9 else 0)
     bf16 = 34 <= plan.variant <= 37 or 44 <= plan.variant <= 47
     roof["kernel"] = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF32 on tcgen05, one CTA per tile)",
