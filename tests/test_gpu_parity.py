@@ -126,7 +126,9 @@ def test_tensor_core_variant_ragged_unaligned_and_auto(env):
     # sparse plan: fp32 arithmetic, so the tighter bound holds)
     L = ubp_synth.make_layer("t", 200, 150, 4, 60, 777, Nc=130, x_dist="normal")
     check(*run_spmm(env, L, 32, pad=2)[:3], L, tensor_core=True)
+    check(*run_spmm(env, L, 36, pad=2)[:3], L, variant=36)          # the same through the bf16-product kernel
     check(*run_spmm(env, L, 32, pad=0, misalign=1)[:3], L)
+    check(*run_spmm(env, L, 36, pad=0, misalign=1)[:3], L)
     L2 = ubp_synth.make_layer("t", 200, 150, 4, 60, 778, Nc=131, x_dist="normal")
     check(*run_spmm(env, L2, 32)[:3], L2)
     # the automatic choice: dense-enough layers run on tensor cores, very sparse or small ones do not
@@ -279,8 +281,17 @@ def test_two_cta_kernel_padded_rows_and_repeated_launches(env):
     torch, ubp = env
     L = ubp_synth.make_layer("t", 256, 64, 4, 60, 4242, Nc=512, x_dist="normal")
     check(*run_spmm(env, L, 32, pad=4)[:3], L, tensor_core=True)
+    check(*run_spmm(env, L, 36, pad=4)[:3], L, variant=36)
+    L = ubp_synth.make_layer("t", 384, 1040, 4, 70, 4243, Nc=260, x_dist="normal")   # 65 chunks: two per stage, odd count
+    check(*run_spmm(env, L, 36, pad=0)[:3], L, variant=36)
     L = ubp_synth.config_layers("mbv1_chain", batch=64)[4]          # 256 -> 256 channels at 28 x 28: 50176 columns
-    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb), 32)
+    for variant in (32, 36):
+        _repeated_launches(env, L, variant)
+
+
+def _repeated_launches(env, L, variant):
+    torch, ubp = env
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb), variant)
     assert plan.tile_choice(L.Nc)[0] == 2                            # the CTA-pair kernel is what runs here
     X = torch.from_numpy(L.X).cuda().reshape(L.C, -1)
     bias = torch.from_numpy(L.bias).cuda()
