@@ -9,10 +9,12 @@
 // tensor-core time and little more than half the shared-memory traffic, the two bounds of ubp_tc2.cu.
 //
 // Differences from ubp_tc2.cu: the plan supplies W1 / W2 (bf16, K-major, 32-byte swizzle) already tiled into the
-// 8 KB blocks a chunk needs, so a chunk's weights are one contiguous bulk copy; the tensor core cannot take the raw fp32 activations any more, so TMA copies the chunk's 16 channel rows
-// as they are (plus a halo for 3x3) and the pass warps write BOTH x1 and x2, in the MN-major bf16 operand layout
-// (64 columns x 8 channels atoms in the 128-byte swizzle; LBO = next 64 columns, SBO = next 8 channels). Thread
-// roles, barriers, persistence, the two accumulators and the epilogue are those of ubp_tc2.cu.
+// 8 KB blocks a chunk needs, so a chunk's weights are one contiguous bulk copy; the tensor core cannot take the raw
+// fp32 activations any more, so TMA copies the chunk's 16 channel rows as they are (plus a halo for 3x3) and the
+// pass warps write BOTH x1 and x2, in the MN-major bf16 operand layout (64 columns x 8 channels atoms in the
+// 128-byte swizzle; LBO = next 64 columns, SBO = next 8 channels); a pipeline stage holds one or two chunks
+// (template parameter SUB). Thread roles, barriers, persistence, the two accumulators and the epilogue are those of
+// ubp_tc2.cu.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -33,7 +35,6 @@ constexpr int T3_XL_GROUPS = 2;                           // two groups of four 
 constexpr int T3_EPI_WARPS = 8;                           // warps 10..17
 constexpr int T3_THREADS = (2 + T3_XL_WARPS + T3_EPI_WARPS) * 32;
 constexpr int T3_MAX_STAGES = 8;
-constexpr int T3_MAX_SUB = 2;                             // 16-channel chunks per pipeline stage: 1 or 2 (chosen per launch)
 constexpr uint32_t T3_A_PART = 128 * TC_KC * 2;           // W1 or W2 chunk of this CTA's 128 rows: 4 KB
 constexpr uint32_t T3_ATOM = 64 * TC_KC * 2;              // x1 or x2 of 64 columns x 16 channels: 2 KB
 constexpr uint32_t T3_PIPE_BUDGET = 222 * 1024;
