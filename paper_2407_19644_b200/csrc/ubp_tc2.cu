@@ -353,7 +353,7 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             st += T2_XL_GROUPS;
             if (st >= S) { st -= S; ph ^= 1u; }
         }
-        // ---------------- the last tile has nothing to overlap with: take column blocks 2, 3, 6, 7 of its epilogue.
+        // ---------------- the last tile has nothing to overlap with: take the 16-column units 2, 3, 6, 7, ... of its epilogue.
         // Its own barrier (one phase) rather than the accumulator's, whose earlier phases these warps did not see.
         if (ok && nmy > 0) ok = mbar_wait_relaxed(smem_u32(&bar_last), 0, &abort_flag);
         if (ok && nmy > 0) {

@@ -355,7 +355,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             st += T3_XL_GROUPS;
             if (st >= S) { st -= S; ph ^= 1u; }
         }
-        // ---------------- the last tile has nothing to overlap with: take column blocks 2, 3, 6, 7 of its epilogue.
+        // ---------------- the last tile has nothing to overlap with: take the 16-column units 2, 3, 6, 7, ... of its epilogue.
         // Its own barrier (one phase) rather than the accumulator's, whose earlier phases these warps did not see.
         if (ok && nmy > 0) ok = mbar_wait_relaxed(smem_u32(&bar_last), 0, &abort_flag);
         if (ok && nmy > 0) {

@@ -189,46 +189,45 @@ __device__ __forceinline__ void mma2_commit_both(uint32_t bar)
         ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16])
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&r)[8])
 {
     asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        "tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
         : "r"(taddr) : "memory");
 }
 
-// Epilogue of 32 rows (tensor-memory lane quarter q of accumulator `acc`) x the 32-column blocks first, first + step,
+// Epilogue of 32 rows (tensor-memory lane quarter q of accumulator `acc`) x the 16-column units first, first + step,
 // ... of one CTA's 128 x N part of a tile, without shared memory (the MMA operands and the copies already use all
 // of its bandwidth). The accumulator is read in the 16 x 256-bit shape: lane t gets, per group j of 8 columns,
 // the column pair 8j + 2(t mod 4) of rows t/4 and t/4 + 8 of a 16-row half. Four lanes therefore hold 32
 // consecutive bytes of an output row, and every 8-byte store instruction of the warp writes eight whole 32-byte
-// sectors; bias and ReLU are applied in registers.
+// sectors; bias and ReLU are applied in registers. (Units of 16 columns rather than 32 so that the warps sharing a
+// lane quarter get equal shares of tile widths such as 192 or 224.)
 // `done_bar` != 0: once this warp's last tensor-memory read has completed, lane 0 arrives on that barrier of the
 // leader CTA (the accumulator may be overwritten from then on).
 __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, int q, int first, int step, int N,
                                                 int row0, int64_t col0, int lane, uint32_t done_bar, uint32_t rank)
 {
     const int rbase = row0 + q * 32 + (lane >> 2);          // this lane's rows: rbase + {0, 8, 16, 24}
-    const int nblk = N / 32;
+    const int nunit = N / 16;
     float bias[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) bias[i] = (a.bias && rbase + 8 * i < a.M) ? __ldg(a.bias + rbase + 8 * i) : 0.f;
 #pragma unroll 1
-    for (int cc = first; cc < nblk; cc += step) {
-        uint32_t r[2][16];
-        tmem_ld_16x256b_x4(acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), r[0]);
-        tmem_ld_16x256b_x4(acc + ((uint32_t)(q * 32 + 16) << 16) + (uint32_t)(cc * 32), r[1]);
+    for (int cc = first; cc < nunit; cc += step) {
+        uint32_t r[2][8];
+        tmem_ld_16x256b_x2(acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), r[0]);
+        tmem_ld_16x256b_x2(acc + ((uint32_t)(q * 32 + 16) << 16) + (uint32_t)(cc * 16), r[1]);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (done_bar && cc + step >= nblk) {
+        if (done_bar && cc + step >= nunit) {
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             if (lane == 0) {
                 if (rank == 0) mbar_arrive(done_bar);
                 else mbar_arrive_remote(done_bar, 0);
             }
         }
-        const int64_t cb = col0 + cc * 32 + 2 * (lane & 3);
+        const int64_t cb = col0 + cc * 16 + 2 * (lane & 3);
 #pragma unroll
         for (int half = 0; half < 2; ++half)
 #pragma unroll
@@ -238,7 +237,7 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
                 float *yrow = a.Y + (size_t)row * a.ldy;
                 const float b = bias[2 * half + h];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < 2; ++j) {
                     float2 o = make_float2(__uint_as_float(r[half][4 * j + 2 * h]) + b,
                                            __uint_as_float(r[half][4 * j + 2 * h + 1]) + b);
                     if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); }
@@ -248,8 +247,8 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
                 }
             }
     }
-    // a warp with no block of its own still owes its arrival
-    if (done_bar && first >= nblk) {
+    // a warp with no unit of its own still owes its arrival
+    if (done_bar && first >= nunit) {
         if (lane == 0) {
             if (rank == 0) mbar_arrive(done_bar);
             else mbar_arrive_remote(done_bar, 0);
