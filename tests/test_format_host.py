@@ -197,3 +197,28 @@ def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     got16 = W1[:, :C * R].astype(np.float64) + W2[:, :C * R]
     assert np.all(np.abs(got16 - Wm) <= np.abs(Wm) * 2.0 ** -16)
     assert not got16[Wm == 0].any()
+
+
+def test_bf16_three_term_product_error_bound():
+    """The arithmetic of the bf16-product tensor-core variants, emulated in numpy: with x1 = bf16(x), x2 = bf16(x - x1)
+    (round to nearest even, 8 significant bits) and likewise w, the three-term product w1 x1 + w2 x1 + w1 x2 is within
+    3 * 2^-16 of w x, relative to |w x|, for every pair - the bound the GPU tests assert and the 1e-4 gate contains."""
+    def bf16(v):
+        b = v.astype(np.float32).view(np.uint32).astype(np.uint64)
+        b = ((b + 0x7fff + ((b >> 16) & 1)) >> 16) << 16
+        return b.astype(np.uint32).view(np.float32)
+
+    rng = np.random.default_rng(12)
+    n = 1_000_000
+    cases = [(rng.standard_normal(n), rng.standard_normal(n) * 0.05), (rng.uniform(1, 2, n), rng.uniform(1, 2, n)),
+             (1 + 2.0 ** -8 - 2.0 ** -16 * rng.uniform(0.9, 1.1, n),) * 2,       # just below a rounding boundary
+             (rng.standard_normal(n) * 1e-20, rng.standard_normal(n) * 1e15)]    # far from 1: bf16 has fp32's range
+    for x, w in cases:
+        x, w = x.astype(np.float32), w.astype(np.float32)
+        x1, w1 = bf16(x), bf16(w)
+        x2, w2 = bf16(x - x1), bf16(w - w1)
+        assert np.all(np.abs((x - x1).astype(np.float64)) <= np.abs(x) * 2.0 ** -8)
+        assert np.all(np.abs(x.astype(np.float64) - x1 - x2) <= np.abs(x) * 2.0 ** -16)
+        approx = x1.astype(np.float64) * w1 + x1.astype(np.float64) * w2 + x2.astype(np.float64) * w1
+        exact = x.astype(np.float64) * w
+        assert np.all(np.abs(approx - exact) <= np.abs(exact) * 3 * 2.0 ** -16)

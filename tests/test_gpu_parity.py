@@ -274,6 +274,22 @@ def test_sweep_config_sampled(env, nb, sp, variant):
         assert scaled_error(Y[o], ys, as_) <= TOL
 
 
+def test_bf16_product_variant_few_terms_per_output(env):
+    """Where the split products' error cannot average out: 98 % sparsity (most outputs are one or two products) and
+    operands of magnitude >= 1 (no small values to hide behind). The bf16-product kernel must still be inside its worst-case
+    bound 3 * 2^-16 (+ accumulation), hence inside the 1e-4 gate; the TF32-product kernel inside 2^-18."""
+    torch, ubp = env
+    L = ubp_synth.make_layer("t", 256, 256, 4, 98, 4321, Nc=1024, w_dist="uniform", x_dist="normal", relu=False)
+    L.W[:] = np.abs(L.W) + 1.0
+    L.X[:] = np.abs(L.X) + 1.0
+    assert terms_per_output(L) <= 16
+    for variant in (36, 32):
+        Yh, Yref, A, plan = run_spmm(env, L, variant)
+        assert plan.variant == variant and plan.tile_choice(1024)[0] == 2
+        err = check(Yh, Yref, A, L, variant=variant)
+        assert err <= (3 * 2.0 ** -16 + 2.0 ** -20 if variant == 36 else 2.0 ** -18)
+
+
 def test_two_cta_kernel_padded_rows_and_repeated_launches(env):
     """The two-CTA tensor-core kernel with a leading dimension larger than the column count, and forty launches
     in a row on a layer with many column tiles and few chunks (several waves of CTA pairs; the copies of different
