@@ -33,6 +33,9 @@ struct KernelCfg {
 };
 const std::vector<KernelCfg> &kernel_cfgs();
 // tensor-core variants whose CTA-pair kernel uses three bf16 products per fp32 product instead of three TF32 products
+// Output rows per CTA of the bf16 CTA-pair kernel: 128, or for layers of at most 128 rows half of them (rounded up to
+// a multiple of 8) so that both CTAs of the pair have rows to store.
+inline int tc16_rows_per_cta(int M) { return M > 128 ? 128 : (((M + 1) / 2 + 7) & ~7); }
 inline bool cfg_bf16(const KernelCfg &c) { return (c.id >= 34 && c.id <= 37) || (c.id >= 44 && c.id <= 47); }
 const KernelCfg *find_cfg(int id);
 // pick a configuration for a layer (variant == 0)
@@ -56,8 +59,9 @@ struct PlanImage {
     size_t tc_off = 0;
     int tc_kp = 0;
     // and of the same weight as two bf16 pieces (W1 = the weight rounded to bf16, W2 = the remainder rounded to bf16),
-    // tiled: 8 KB blocks [row tile of 128][chunk of 16 channels] = [piece][128 rows][16 channels] in the 32-byte
-    // swizzle; tc16_kp = reduction length padded to whole chunks
+    // tiled: 8 KB blocks [row tile][chunk of 16 channels] = [piece][128 rows][16 channels] in the 32-byte swizzle;
+    // a row tile holds tc16_rows_per_cta(M) rows of the matrix (the rest of its 128 rows are zero);
+    // tc16_kp = reduction length padded to whole chunks
     size_t tc16_off = 0;
     int tc16_kp = 0;
 };

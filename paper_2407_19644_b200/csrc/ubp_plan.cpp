@@ -45,10 +45,10 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     (void)M; (void)C; (void)m;
     const int nbk = largest_pow2_divisor_le16(Nb);
     const double dens = (double)m * Nb / ((double)M * C);
-    // With more than 128 rows the tensor-core variants run on CTA pairs, and there the bf16-product form (ids + 4:
-    // half the tensor-core and shared-memory time, error <= 3 * 2^-16 |w||x|, inside the 1e-4 gate) is the default;
-    // the TF32-product ids stay selectable.
-    const int fast = M > 128 ? 4 : 0;
+    // The tensor-core variants run on CTA pairs, and there the bf16-product form (ids + 4: half the tensor-core and
+    // shared-memory time, error <= 3 * 2^-16 |w||x|, inside the 1e-4 gate) is the default; the TF32-product ids stay
+    // selectable (with at most 128 rows they run the one-CTA kernel).
+    const int fast = 4;
     if (R == 9 && dens >= 0.08 && M >= 128 && C >= 16) {    // implicit GEMM on tensor cores
         switch (nbk) {
             case 16: case 8: return find_cfg(40 + fast);
@@ -68,10 +68,10 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     if (R != 1) return nullptr;
     // Dense tensor-core variant when enough of the weight survives and the layer is large enough to amortise its
     // per-tile set-up: measured on B200 it takes the same time at every sparsity and beats the sparse kernel up to
-    // ~90 % sparsity on 2048 x 2048 x 8192. With more than 128 rows the CTA-pair kernel runs, which pays from 128
-    // input channels on; with exactly 128 rows (one CTA per tile) from 256 on; below that the sparse kernel is as
-    // fast or faster.
-    if (dens >= 0.08 && ((M > 128 && C >= 128) || (M >= 128 && C >= 256))) {
+    // ~90 % sparsity on 2048 x 2048 x 8192. It pays from 128 rows and 128 input channels on (measured on the
+    // MobileNet-shaped layers: 128 -> 128 channels 57 us against 66 us; 64 -> 128 channels 52 against 45); below
+    // that the sparse kernel is as fast or faster.
+    if (dens >= 0.08 && M >= 128 && C >= 128) {
         switch (nbk) {
             case 16: case 8: return find_cfg(33 + fast);
             case 4: return find_cfg(32 + fast);
@@ -162,7 +162,8 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         // The same matrix as two bf16 pieces, tiled for the CTA-pair kernel: one 8 KB block per (128-row tile,
         // 16-channel chunk) = [piece W1, W2][128 rows][16 channels] exactly as the kernel wants it in shared memory
         // (rows of 32 bytes whose two 16-byte halves are swapped on rows with bit 2 set: the 32-byte swizzle of a
-        // K-major operand), so that a chunk is ONE contiguous bulk copy instead of 256 row pieces.
+        // K-major operand), so that a chunk is ONE contiguous bulk copy instead of 256 row pieces. A layer of at most
+        // 128 rows puts half of them into each of the pair's two tiles (the rest of a tile stays zero).
         img.tc16_kp = (C * R + 15) & ~15;   // padded reduction length: whole chunks
         img.tc16_off = total;
         total += (size_t)((M + 255) / 256) * 2 * (img.tc16_kp / 16) * 8192;   // whole pairs of row tiles (zero rows pad)
@@ -240,9 +241,10 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         // and into two bf16 pieces: the weight rounded to nearest-even bf16, and the (exact) remainder rounded
         uint8_t *W16 = base + img.tc16_off;
         const size_t nchunk16 = (size_t)img.tc16_kp / 16;
+        const int rpc16 = tc16_rows_per_cta(M);            // matrix rows per 128-row tile (64 when M = 128, ...)
         auto w16_at = [&](int row, size_t k, int piece) -> uint16_t * {
-            const size_t blk = (size_t)(row / 128) * nchunk16 + k / 16;
-            const int i = row % 128, kk = (int)(k % 16);
+            const size_t blk = (size_t)(row / rpc16) * nchunk16 + k / 16;
+            const int i = row % rpc16, kk = (int)(k % 16);
             return reinterpret_cast<uint16_t *>(W16 + blk * 8192 + (size_t)piece * 4096 + (size_t)i * 32 +
                                                 (size_t)(((kk >> 3) ^ ((i >> 2) & 1)) * 16) + (size_t)(kk & 7) * 2);
         };

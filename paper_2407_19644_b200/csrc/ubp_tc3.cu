@@ -148,7 +148,8 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     // this pair's tiles: pair, pair + npairs, ...; tile t = (row pair t % nrp, column tile t / nrp)
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
     const int nmy = pair < ntiles ? (ntiles - pair + npairs - 1) / npairs : 0;
-    auto tile_row0 = [&](int i) { return ((pair + i * npairs) % nrp) * 256 + (int)rank * 128; };
+    const int rpc = a.rpc ? a.rpc : 128;                   // output rows per CTA (fewer than 128 only for layers of <= 128 rows)
+    auto tile_row0 = [&](int i) { return (((pair + i * npairs) % nrp) * 2 + (int)rank) * rpc; };
     auto tile_col0 = [&](int i) { return (int64_t)((pair + i * npairs) / nrp) * N; };
 
     // one stage's copies (stage sg of a tile = chunks sg * SUB ...): per chunk the W1 / W2 block of this CTA's 128
@@ -164,7 +165,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             if (u >= nsub) break;
             const int c = c0 + u;
             uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
-            bulk_load(smem_u32(chunk), W16 + ((size_t)(row0 >> 7) * nchunk + c) * (2 * T3_A_PART), 2 * T3_A_PART, bar);
+            bulk_load(smem_u32(chunk), W16 + ((size_t)(row0 / rpc) * nchunk + c) * (2 * T3_A_PART), 2 * T3_A_PART, bar);
             tma_load_2d(smem_u32(chunk + 2 * T3_A_PART + 2 * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
         }
     };

@@ -155,6 +155,8 @@ struct TcArgs {
     int ntile;               // columns per CTA: multiple of 32, <= 256
     int relu;
     int *status;             // plan status word
+    int rpc;                 // CTA-pair kernels: output rows per CTA (128; fewer when the layer has at most 128 rows
+                             // and the pair splits them evenly); 0 means 128
 };
 
 
@@ -209,11 +211,14 @@ __device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&r)
 __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, int q, int first, int step, int N,
                                                 int row0, int64_t col0, int lane, uint32_t done_bar, uint32_t rank)
 {
-    const int rbase = row0 + q * 32 + (lane >> 2);          // this lane's rows: rbase + {0, 8, 16, 24}
+    const int lbase = q * 32 + (lane >> 2);                 // this lane's rows inside the CTA's part: lbase + {0, 8, 16, 24}
+    const int rbase = row0 + lbase;
+    const int rpc = a.rpc ? a.rpc : 128;                    // rows of the CTA's part that exist
     const int nunit = N / 16;
     float bias[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) bias[i] = (a.bias && rbase + 8 * i < a.M) ? __ldg(a.bias + rbase + 8 * i) : 0.f;
+    for (int i = 0; i < 4; ++i)
+        bias[i] = (a.bias && lbase + 8 * i < rpc && rbase + 8 * i < a.M) ? __ldg(a.bias + rbase + 8 * i) : 0.f;
 #pragma unroll 1
     for (int cc = first; cc < nunit; cc += step) {
         uint32_t r[2][8];
@@ -233,7 +238,7 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int row = rbase + 16 * half + 8 * h;
-                if (row >= a.M) continue;
+                if (row >= a.M || lbase + 16 * half + 8 * h >= rpc) continue;
                 float *yrow = a.Y + (size_t)row * a.ldy;
                 const float b = bias[2 * half + h];
 #pragma unroll

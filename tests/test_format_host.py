@@ -188,7 +188,13 @@ def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     swap = ((rows >> 2) & 1).astype(bool)
     blocks = blocks.copy()
     blocks[:, :, :, swap] = blocks[:, :, :, swap][..., ::-1, :]
-    W12 = blocks.reshape(nrt, nch, 2, 128, 16).transpose(2, 0, 3, 1, 4).reshape(2, nrt * 128, kp16)
+    W12 = blocks.reshape(nrt, nch, 2, 128, 16).transpose(2, 0, 3, 1, 4)          # [piece][row tile][row in tile][k]
+    W12 = W12.reshape(2, nrt, 128, kp16)
+    # a row tile holds `rpc` rows of the matrix: 128, or half of them (rounded up to 8) for a layer of <= 128 rows,
+    # so that both CTAs of a pair have rows to store; the rest of the tile is zero
+    rpc = 128 if M > 128 else ((M + 1) // 2 + 7) // 8 * 8
+    assert not W12[:, :, rpc:].any()
+    W12 = W12[:, :, :rpc].reshape(2, nrt * rpc, kp16)
     assert not W12[:, M:].any()                                # padding rows
     W1 = (W12[0, :M].astype(np.uint32) << 16).view(np.float32)
     W2 = (W12[1, :M].astype(np.uint32) << 16).view(np.float32)

@@ -104,6 +104,8 @@ TC_CASES = [
     # more than 128 rows: the two-CTA kernel; whole 32-column groups (one 3-D copy of X per chunk) with and without
     # a ragged last column tile, more chunks than pipeline stages, a ragged last row pair
     (512, 96, 4, 60, 2048, 32), (300, 150, 4, 70, 544, 32), (256, 256, 4, 70, 4128, 32), (640, 40, 8, 50, 96, 33),
+    # at most 128 rows through the bf16-product CTA-pair kernel: each CTA of the pair takes half of the rows
+    (128, 128, 4, 60, 4100, 36), (100, 200, 4, 50, 8200, 36), (72, 144, 8, 50, 8196, 37), (128, 64, 2, 50, 16384, 35),
 ]
 
 
@@ -113,6 +115,8 @@ def test_spmm_tensor_core_variant(env, M, C, Nb, p, Nc, variant):
     Yh, Yref, A, plan = run_spmm(env, L, variant)
     assert plan.variant == variant
     check(Yh, Yref, A, L, variant=variant)
+    if (M, C) == (128, 128):
+        assert plan.tile_choice(Nc)[0] == 2          # the CTA pair splits the 128 rows 64 / 64
     if M > 128:                          # the same layer through the bf16-product form of the CTA-pair kernel
         Yh, Yref, A, plan = run_spmm(env, L, variant + 4)
         assert plan.variant == variant + 4 and plan.tile_choice(Nc)[0] in (1, 2)
