@@ -466,6 +466,7 @@ def main():
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
         "us_per_layer": step_ms * 1e3, "us_min": float(np.min(times)) * 1e3, "us_median": float(np.median(times)) * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "arithmetic": roof.get("arithmetic"),
         "config": {"workload": name, "M": L.M, "K": L.C * L.R, "Nc": L.Nc, "block": f"{L.Nb}x1x{L.R}",
                    "sparsity_pct": L.sparsity_pct, "blocks": L.m, "bias": L.bias is not None, "relu": bool(L.relu),
                    "variant": plan.variant, "l2": "warm" if args.no_flush else "flushed between steps (256 MiB write)",
