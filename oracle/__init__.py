@@ -37,6 +37,8 @@ def lib():
         L.orc_blob_size.restype = C.c_size_t
         L.orc_blob_size.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int64]
         L.orc_num_threads.restype = C.c_int
+        for f in (L.orc_bed_expand, L.orc_greedy_select, L.orc_optimal_select):
+            f.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -179,3 +181,74 @@ def wros_spmm(blob: bytes, X, bias=None, relu=False, tile_w: int = 4):
     _chk(lib().orc_wros_spmm(_p(b), C.c_size_t(b.size), _p(X), C.c_int64(Nc), C.c_int64(Nc),
                              _p(bias), int(bool(relu)), int(tile_w), _p(Y)), "wros_spmm")
     return Y
+
+
+# ---------------------------------------------------------------------------
+# Block selection (Section 3.1 Eq. 1, Section 3.2 Eq. 3 and Eq. 4, Section 4.1
+# Algorithms 1 and 2). Candidate index k = i + M*j (start row i, input channel j).
+# ---------------------------------------------------------------------------
+
+def block_scores(W: np.ndarray, Nb: int) -> np.ndarray:
+    """Eq. 1 scores as a float32 vector of length C*M (k = i + M*j); -inf where i + Nb > M."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    M, Cin = W.shape[:2]
+    W = W.reshape(M, Cin, -1)
+    S = np.empty(M * Cin, np.float32)
+    _chk(lib().orc_block_scores(_p(W), M, Cin, W.shape[2], Nb, _p(S)), "block_scores")
+    return S
+
+
+def bed_expand(S: np.ndarray, Nb: int, m: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Algorithm 1: the chosen original indices, in the order chosen, and their scores when chosen."""
+    S = np.ascontiguousarray(S, dtype=np.float32)
+    Ibar = np.zeros(max(m, 1), np.int64)
+    sc = np.zeros(max(m, 1), np.float32)
+    n = int(lib().orc_bed_expand(_p(S), C.c_int64(S.size), Nb, C.c_int64(m), _p(Ibar), _p(sc)))
+    if n < 0:
+        raise OracleError(n, "bed_expand")
+    return Ibar[:n].copy(), sc[:n].copy()
+
+
+def bed_divide(Ibar: np.ndarray, Nb: int) -> np.ndarray:
+    """Algorithm 2: final block start indices, ascending."""
+    Ibar = np.ascontiguousarray(Ibar, dtype=np.int64)
+    I = np.zeros(max(Ibar.size, 1), np.int64)
+    _chk(lib().orc_bed_divide(_p(Ibar), C.c_int64(Ibar.size), Nb, _p(I)), "bed_divide")
+    return I[:Ibar.size].copy()
+
+
+def greedy_select(S: np.ndarray, Nb: int, m: int) -> np.ndarray:
+    """Eq. 3: block start indices in the order chosen."""
+    S = np.ascontiguousarray(S, dtype=np.float32)
+    I = np.zeros(max(m, 1), np.int64)
+    n = int(lib().orc_greedy_select(_p(S), C.c_int64(S.size), Nb, C.c_int64(m), _p(I)))
+    if n < 0:
+        raise OracleError(n, "greedy_select")
+    return I[:n].copy()
+
+
+def optimal_select(S: np.ndarray, Nb: int, m: int) -> Tuple[Optional[np.ndarray], float]:
+    """Eq. 4: (ascending block start indices or None when m blocks do not fit, best total)."""
+    S = np.ascontiguousarray(S, dtype=np.float32)
+    I = np.zeros(max(m, 1), np.int64)
+    tot = C.c_double(0.0)
+    n = int(lib().orc_optimal_select(_p(S), C.c_int64(S.size), Nb, C.c_int64(m), _p(I), C.byref(tot)))
+    if n < -1:
+        raise OracleError(n, "optimal_select")
+    return (I[:m].copy() if n == m else None), float(tot.value)
+
+
+def starts_to_mask(I: np.ndarray, M: int, Cin: int, Nb: int) -> np.ndarray:
+    I = np.ascontiguousarray(I, dtype=np.int64)
+    mask = np.empty((M, Cin), np.uint8)
+    _chk(lib().orc_starts_to_mask(_p(I), C.c_int64(I.size), M, Cin, Nb, _p(mask)), "starts_to_mask")
+    return mask
+
+
+def bed_select(W: np.ndarray, Nb: int, m: int):
+    """Scores, expansion, division, mask: returns (mask [M][C] uint8, I ascending, Ibar in the order chosen)."""
+    M, Cin = W.shape[:2]
+    S = block_scores(W, Nb)
+    Ibar, _ = bed_expand(S, Nb, m)
+    I = bed_divide(Ibar, Nb)
+    return starts_to_mask(I, M, Cin, Nb), I, Ibar

@@ -18,7 +18,7 @@ import numpy as np
 
 __all__ = [
     "block_budget", "random_block_starts", "mask_from_starts", "random_mask",
-    "Layer", "make_layer", "CONFIGS", "MBV1_CHAIN", "config_layers",
+    "Layer", "make_layer", "CONFIGS", "MBV1_CHAIN", "config_layers", "selection_weights",
 ]
 
 
@@ -189,3 +189,24 @@ def config_layers(cfg: str, *, batch: Optional[int] = None, Nb: Optional[int] = 
                                   w_scale=0.05, bias=True, relu=True, make_x=make_x))
         return out
     raise KeyError(cfg)
+
+
+def selection_weights(M: int, C: int, R: int, seed: int, kind: str = "trained") -> np.ndarray:
+    """Dense weights [M][C][R] for block-selection experiments (stand-ins for
+    trained layers, which are not available). ``kind``:
+    'trained'  N(0, 0.05) scaled by a log-normal gain per output channel and per
+               input channel (sigma 0.5 each), so that important kernels cluster
+               along rows and columns the way trained layers do;
+    'normal'   plain N(0, 0.05);
+    'integer'  integers in [-3, 3]: many equal scores, every sum exact."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    if kind == "integer":
+        return rng.integers(-3, 4, size=(M, C, R)).astype(np.float32)
+    W = rng.standard_normal(size=(M, C, R), dtype=np.float32) * np.float32(0.05)
+    if kind == "trained":
+        go = np.exp(rng.standard_normal(M) * 0.5).astype(np.float32)
+        gc = np.exp(rng.standard_normal(C) * 0.5).astype(np.float32)
+        W = W * go[:, None, None] * gc[None, :, None]
+    elif kind != "normal":
+        raise ValueError(kind)
+    return np.ascontiguousarray(W, dtype=np.float32)
