@@ -225,6 +225,40 @@ size_t ubp_static_plan_capacity(void);
 int ubp_spmm_static(const void *blob, size_t len, const float *X, int64_t ldx, int64_t Nc,
                     const float *bias, int relu, float *Y, int64_t ldy, void *stream);
 
+/* --------------------------------------------------------- block selection
+ * Choosing which blocks to keep (Section 3.1 and Section 4.1): candidate block
+ * k = i + M*j starts at output row i of input channel j; its score is the l1
+ * norm of W[i..i+Nb-1][j][:] (Eq. 1), -inf when i + Nb > M. Block expansion
+ * (Algorithm 1) takes m times the best remaining candidate, re-scores the Nb-1
+ * candidates to its left as if the chosen block's kernels were gone (so a block
+ * may grow around an earlier choice instead of being excluded by it) and drops
+ * the Nb candidates starting inside the chosen block; block division
+ * (Algorithm 2) cuts the grown runs every Nb rows. The result is delivered as
+ * a mask[M][C] whose runs of ones are whole blocks -- what ubp_pack decodes.
+ * The device routines reproduce the sequential procedure bit for bit for this
+ * arithmetic: single precision; a kernel's norm = sum of |w| over its R taps in
+ * storage order; a block's score = sum of its Nb kernel norms in row order; a
+ * re-scored candidate = (S[k-n] + S[k-n+Nb]) - S[k]; ties in an arg max go to
+ * the lowest k.
+ * Limits: Nb <= M <= 16384, M*C < 2^31 (UBP_E_UNSUPPORTED beyond).
+ * All device work is enqueued on `stream`; nothing is synchronised. */
+
+/* bytes of device scratch ubp_block_scores / ubp_bed_select need (256-byte aligned buffer). */
+int ubp_bed_workspace_size(int M, int C, int Nb, size_t *dev_bytes);
+
+/* ubp_block_scores: W (device, [M][C][R] row-major) -> S (device, [C][M] floats,
+ * S[j*M + i] = score of candidate k = i + M*j). */
+int ubp_block_scores(const float *W, int M, int C, int R, int Nb, void *workspace, size_t workspace_bytes,
+                     float *S, void *stream);
+
+/* ubp_bed_select: W (device) -> mask (device, [M][C] bytes 0/1) keeping m blocks.
+ * n_selected (device, nullable) receives the number of blocks kept: m, or fewer
+ * when the columns cannot hold m blocks (each holds floor(M/Nb) at most).
+ * Errors: UBP_E_ARG (null, sizes, Nb > M, m < 0, workspace not 256-byte
+ * aligned), UBP_E_SPACE (workspace too small), UBP_E_UNSUPPORTED, UBP_E_CUDA. */
+int ubp_bed_select(const float *W, int M, int C, int R, int Nb, int64_t m, void *workspace, size_t workspace_bytes,
+                   uint8_t *mask, int64_t *n_selected, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -68,6 +68,9 @@ def load():
     L.ubp_selftest_bounded_wait.argtypes = [vp, C.c_uint, vp]
     L.ubp_static_plan_capacity.restype = sz
     L.ubp_spmm_static.argtypes = [vp, sz, vp, i64, i64, vp, i32, vp, i64, vp]
+    L.ubp_bed_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
+    L.ubp_block_scores.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, vp]
+    L.ubp_bed_select.argtypes = [vp, i32, i32, i32, i32, i64, vp, sz, vp, vp, vp]
     _lib = L
     return L
 
@@ -334,3 +337,79 @@ def ubp_spmm_static(blob: bytes, X, bias=None, relu: bool = False, out=None, str
 
 def static_plan_capacity() -> int:
     return int(load().ubp_static_plan_capacity())
+
+
+# ------------------------------------------------------------------ block selection (Section 4.1)
+class BedSelector:
+    """Device scratch for block selection on layers of one shape ([M][C][R] weights, block size Nb); the scratch
+    is a torch uint8 tensor owned by this object, so repeated calls allocate nothing but their outputs."""
+
+    def __init__(self, M: int, Cin: int, R: int, Nb: int, device="cuda"):
+        import torch
+        self._lib = load()
+        self.M, self.C, self.R, self.Nb = int(M), int(Cin), int(R), int(Nb)
+        n = C.c_size_t(0)
+        _chk(self._lib.ubp_bed_workspace_size(self.M, self.C, self.Nb, C.byref(n)), "ubp_bed_workspace_size")
+        self.bytes = n.value
+        self.buffer = torch.empty(n.value + 256, dtype=torch.uint8, device=device)
+        self._base = (self.buffer.data_ptr() + 255) // 256 * 256
+
+    def _w(self, W):
+        import torch
+        if not (isinstance(W, torch.Tensor) and W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
+                and W.numel() == self.M * self.C * self.R and W.shape[0] == self.M and W.shape[1] == self.C):
+            raise ValueError("W must be a contiguous float32 CUDA tensor [M][C][R] of this selector's shape")
+        if W.device != self.buffer.device:
+            raise ValueError("W is on another device than the selector")
+        return C.c_void_p(W.data_ptr())
+
+    def scores(self, W, out=None, stream=None):
+        """Eq. 1 scores of every candidate block: float32 CUDA tensor [C][M], -inf where the block would leave
+        the weights."""
+        import torch
+        if out is None:
+            out = torch.empty((self.C, self.M), dtype=torch.float32, device=W.device)
+        with torch.cuda.device(W.device):
+            _chk(self._lib.ubp_block_scores(self._w(W), self.M, self.C, self.R, self.Nb, C.c_void_p(self._base),
+                                            self.bytes, C.c_void_p(out.data_ptr()), _stream_ptr(stream)),
+                 "ubp_block_scores")
+        return out
+
+    def select(self, W, m: int, mask=None, n_selected=None, stream=None):
+        """Block expansion and division: (mask uint8 CUDA tensor [M][C], n_selected int64 CUDA tensor [1])."""
+        import torch
+        if mask is None:
+            mask = torch.empty((self.M, self.C), dtype=torch.uint8, device=W.device)
+        if n_selected is None:
+            n_selected = torch.zeros(1, dtype=torch.int64, device=W.device)
+        if mask.dtype != torch.uint8 or tuple(mask.shape) != (self.M, self.C) or not mask.is_contiguous():
+            raise ValueError("mask must be a contiguous uint8 CUDA tensor [M][C]")
+        with torch.cuda.device(W.device):
+            _chk(self._lib.ubp_bed_select(self._w(W), self.M, self.C, self.R, self.Nb, int(m), C.c_void_p(self._base),
+                                          self.bytes, C.c_void_p(mask.data_ptr()), C.c_void_p(n_selected.data_ptr()),
+                                          _stream_ptr(stream)), "ubp_bed_select")
+        return mask, n_selected
+
+
+def _selector_for(W, Nb: int) -> BedSelector:
+    if W.dim() not in (2, 3):
+        raise ValueError("W must be [M][C] or [M][C][R]")
+    return BedSelector(W.shape[0], W.shape[1], W.shape[2] if W.dim() == 3 else 1, Nb, device=W.device)
+
+
+def ubp_block_scores(W, Nb: int, stream=None):
+    """One-shot form of BedSelector.scores (allocates its scratch; synchronises before freeing it)."""
+    import torch
+    sel = _selector_for(W, Nb)
+    S = sel.scores(W, stream=stream)
+    torch.cuda.synchronize(W.device)
+    return S
+
+
+def ubp_bed_select(W, Nb: int, m: int, stream=None):
+    """One-shot form of BedSelector.select (allocates its scratch; synchronises before freeing it)."""
+    import torch
+    sel = _selector_for(W, Nb)
+    out = sel.select(W, m, stream=stream)
+    torch.cuda.synchronize(W.device)
+    return out

@@ -1,0 +1,421 @@
+// Block selection by expansion and division (Section 4.1, Algorithms 1 and 2) on the device.
+//
+// The paper's procedure is sequential over one score list of length b = c_out * c_in: m times take the arg max,
+// re-score the N-1 entries to its left, drop N entries. Two facts make it data-parallel without changing a bit of
+// its result:
+//   * a candidate's score is the l1 mass of the next N remaining kernels of ITS input channel (or -inf when fewer
+//     remain), so choosing a block only changes scores inside the same input channel: the columns evolve
+//     independently and meet only in the global arg max;
+//   * inside a column the chosen scores never increase (a re-scored entry is at most the maximum just removed,
+//     also in rounded arithmetic, because rounding is monotonic), so the global order of choices is the merge of
+//     the per-column sequences by (score descending, input channel ascending, position in the sequence ascending)
+//     -- lowest-index tie-breaking of the global arg max, restated.
+// So: every column runs the expansion to exhaustion (one warp per column, the score list in shared memory), the
+// m-th largest chosen score over all columns is found by a radix select, ties at that score are given to the
+// lowest input channels first, and the mask is the set of kernels a column removed before its cut. Cutting the
+// resulting runs of ones every N rows (Algorithm 2) is what ubp_pack does when it decodes the mask.
+//
+// Arithmetic (part of the result, because it decides an arg max): single precision throughout; a kernel's norm is
+// the sum of |w| over its taps in storage order, a block's score the sum of its N kernels' norms in row order
+// (Eq. 1), and a re-scored entry is (S[k-n] + S[k-n+N]) - S[k] in that order (Algorithm 1).
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "ubp_internal.h"
+
+namespace ubp {
+namespace bed {
+
+constexpr uint16_t NONE = 0xFFFFu;
+constexpr int MAX_M = 16384;
+
+struct SelState {
+    unsigned int hist[4][256];
+    unsigned int prefix;      // bits of the threshold score found so far
+    unsigned int none;        // 1 = nothing to select
+    unsigned long long rank;  // how many of the entries matching `prefix` are still to be taken
+    long long nsel;           // blocks selected in the end
+};
+
+struct Workspace {
+    float *aT;        // [C][M] l1 norm of kernel (i, j)
+    float *S;         // [C][M] Eq. 1 scores
+    float *ev;        // [T][C] score of the t-th block chosen in column j
+    uint16_t *order;  // [C][M] iteration at which kernel (i, j) left the list, NONE if it never did
+    int *nev;         // [C] blocks chosen in column j
+    int *cut;         // [C] how many of them are selected
+    SelState *sel;
+    size_t bytes;
+};
+
+static inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static Workspace carve(void *base, int M, int C, int Nb)
+{
+    Workspace w;
+    const size_t mc = (size_t)M * C, T = (size_t)(M / Nb);
+    size_t off = 0;
+    auto take = [&](size_t n) { size_t o = off; off += up256(n); return reinterpret_cast<char *>(reinterpret_cast<uintptr_t>(base) + o); };
+    w.aT = (float *)take(mc * 4);
+    w.S = (float *)take(mc * 4);
+    w.ev = (float *)take((T > 0 ? T : 1) * C * 4);
+    w.order = (uint16_t *)take(mc * 2);
+    w.nev = (int *)take((size_t)C * 4);
+    w.cut = (int *)take((size_t)C * 4);
+    w.sel = (SelState *)take(sizeof(SelState));
+    w.bytes = off;
+    return w;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Eq. 1, part one: aT[j][i] = sum over taps of |W[i][j][r]| (storage order), written transposed so that an input
+// channel's column is contiguous.
+__global__ void __launch_bounds__(256) bed_norm_kernel(const float *__restrict__ W, int M, int C, int R, float *__restrict__ aT)
+{
+    __shared__ float tile[32][33];
+    const int j0 = blockIdx.x * 32, i0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int ii = ty; ii < 32; ii += 8) {
+        const int i = i0 + ii, j = j0 + tx;
+        float a = 0.0f;
+        if (i < M && j < C) {
+            const float *w = W + ((size_t)i * C + j) * R;
+            for (int r = 0; r < R; ++r) a += fabsf(w[r]);
+        }
+        tile[ii][tx] = a;
+    }
+    __syncthreads();
+    for (int jj = ty; jj < 32; jj += 8) {
+        const int j = j0 + jj, i = i0 + tx;
+        if (i < M && j < C) aT[(size_t)j * M + i] = tile[tx][jj];
+    }
+}
+
+// Eq. 1, part two: S[j][i] = aT[j][i] + ... + aT[j][i+N-1] in that order, -inf when the block would leave the column.
+__global__ void __launch_bounds__(256) bed_window_kernel(const float *__restrict__ aT, int M, int C, int Nb, float *__restrict__ S)
+{
+    const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= (size_t)M * C) return;
+    const int i = (int)(idx % (size_t)M);
+    float s = __int_as_float(0xff800000);
+    if (i + Nb <= M) {
+        const float *a = aT + idx;
+        s = a[0];
+        for (int t = 1; t < Nb; ++t) s += a[t];
+    }
+    S[idx] = s;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Algorithm 1 for one input channel per warp. Shared memory per warp: the scores (padded with -inf to a multiple
+// of 128), a doubly linked list over the entries still in the list (entry M = end marker), and the positions met
+// while walking N steps to either side of the chosen entry.
+__global__ void __launch_bounds__(32) bed_expand_kernel(const float *__restrict__ S, int M, int C, int Nb, int Mpad,
+                                                        float *__restrict__ ev, uint16_t *__restrict__ order,
+                                                        int *__restrict__ nev)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    float *s = reinterpret_cast<float *>(smem);
+    uint16_t *nxt = reinterpret_cast<uint16_t *>(s + Mpad);
+    uint16_t *prv = nxt + (M + 1);
+    uint16_t *wk = prv + (M + 1);                  // [2][Nb + 1]: successors, predecessors
+    const int lane = threadIdx.x;
+    const int j = blockIdx.x;
+    const float NEG = __int_as_float(0xff800000);
+    const float *Sj = S + (size_t)j * M;
+    uint16_t *oj = order + (size_t)j * M;
+    for (int i = lane; i < Mpad; i += 32) s[i] = i < M ? Sj[i] : NEG;
+    for (int i = lane; i <= M; i += 32) {
+        nxt[i] = (uint16_t)(i < M ? i + 1 : M);
+        prv[i] = (uint16_t)(i > 0 ? i - 1 : NONE);
+    }
+    for (int i = lane; i < M; i += 32) oj[i] = NONE;
+    __syncwarp();
+
+    const float4 *s4 = reinterpret_cast<const float4 *>(s);
+    const int nq = Mpad >> 2;
+    const int T = M / Nb;
+    int it = 0;
+    for (; it < T; ++it) {
+        // arg max, lowest position among equals
+        float best = NEG;
+        int bidx = 0x7fffffff;
+        for (int q = lane; q < nq; q += 32) {
+            const float4 v = s4[q];
+            const int base = q << 2;
+            if (v.x > best) { best = v.x; bidx = base; }
+            if (v.y > best) { best = v.y; bidx = base + 1; }
+            if (v.z > best) { best = v.z; bidx = base + 2; }
+            if (v.w > best) { best = v.w; bidx = base + 3; }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, bidx, off);
+            if (ob > best || (ob == best && oi < bidx)) { best = ob; bidx = oi; }
+        }
+        if (!(best > NEG)) break;
+        const int k = bidx;
+        // the N entries after k (lane 0) and before it (lane 1) that are still in the list
+        if (lane < 2) {
+            const uint16_t *link = lane == 0 ? nxt : prv;
+            uint16_t *out = wk + lane * (Nb + 1);
+            unsigned cur = (unsigned)k;
+            for (int t = 1; t <= Nb; ++t) {
+                cur = cur == NONE ? NONE : link[cur];
+                out[t] = (uint16_t)cur;
+            }
+        }
+        __syncwarp();
+        // entry n to the left now spans n kernels before the block and N-n after it
+        for (int n = 1 + lane; n < Nb; n += 32) {
+            const unsigned p = wk[(Nb + 1) + n];
+            if (p != NONE) {
+                const unsigned r = wk[Nb - n];
+                s[p] = (s[p] + s[r]) - best;
+            }
+        }
+        __syncwarp();
+        for (int t = lane; t < Nb; t += 32) {
+            const unsigned idx = t == 0 ? (unsigned)k : wk[t];
+            s[idx] = NEG;
+            oj[idx] = (uint16_t)it;
+        }
+        if (lane == 0) {
+            const unsigned p1 = wk[(Nb + 1) + 1], sN = wk[Nb];
+            if (p1 != NONE) nxt[p1] = (uint16_t)sN;
+            prv[sN] = (uint16_t)p1;
+            ev[(size_t)it * C + j] = best;
+        }
+        __syncwarp();
+    }
+    if (lane == 0) nev[j] = it;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// The m-th largest chosen score over all columns: radix select over the bit patterns (scores are finite and >= 0,
+// so unsigned order of the bits is the order of the values), 8 bits per pass from the top.
+__global__ void __launch_bounds__(256) bed_hist_kernel(const float *__restrict__ ev, const int *__restrict__ nev, int T, int C,
+                                                       int pass, SelState *st)
+{
+    __shared__ unsigned int h[256];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const int shift = 24 - 8 * pass;
+    const unsigned int prefix = st->prefix;
+    const size_t total = (size_t)T * C;
+    for (size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x; idx < total; idx += (size_t)gridDim.x * 256) {
+        const int j = (int)(idx % (size_t)C), t = (int)(idx / (size_t)C);
+        if (t < nev[j]) {
+            const unsigned int key = __float_as_uint(ev[idx]);
+            if (pass == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&h[(key >> shift) & 255u], 1u);
+        }
+    }
+    __syncthreads();
+    if (h[threadIdx.x]) atomicAdd(&st->hist[pass][threadIdx.x], h[threadIdx.x]);
+}
+
+__global__ void bed_pick_kernel(int pass, long long m, SelState *st)
+{
+    if (threadIdx.x != 0) return;
+    unsigned long long rank = st->rank;
+    if (pass == 0) {
+        unsigned long long tot = 0;
+        for (int d = 0; d < 256; ++d) tot += st->hist[0][d];
+        rank = (unsigned long long)m < tot ? (unsigned long long)m : tot;
+        st->none = rank == 0 ? 1u : 0u;
+    }
+    if (st->none) { st->rank = 0; return; }
+    const int shift = 24 - 8 * pass;
+    unsigned long long cum = 0;
+    int d = 255;
+    for (; d > 0; --d) {
+        const unsigned long long hd = st->hist[pass][d];
+        if (cum + hd >= rank) break;
+        cum += hd;
+    }
+    st->prefix |= (unsigned int)d << shift;
+    st->rank = rank - cum;
+}
+
+// Per column: how many of its chosen blocks score above the threshold, how many exactly at it; ties are handed out
+// to the lowest input channels first. One CTA, columns in chunks of 1024 with a running carry.
+__global__ void __launch_bounds__(1024) bed_cut_kernel(const float *__restrict__ ev, const int *__restrict__ nev, int C,
+                                                        SelState *st, int *__restrict__ cut, long long *nsel_out)
+{
+    __shared__ unsigned long long warp_sum[32];
+    __shared__ unsigned long long carry_s;
+    __shared__ long long nsel_s;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (tid == 0) { carry_s = 0; nsel_s = 0; }
+    __syncthreads();
+    const unsigned int tau = st->prefix;
+    const unsigned long long r = st->rank;
+    const bool none = st->none != 0;
+    for (int j0 = 0; j0 < C; j0 += 1024) {
+        const int j = j0 + tid;
+        int gt = 0, eq = 0;
+        if (j < C && !none) {
+            const int n = nev[j];
+            int lo = 0, hi = n;                     // first position whose score is <= tau
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (__float_as_uint(ev[(size_t)mid * C + j]) > tau) lo = mid + 1; else hi = mid;
+            }
+            gt = lo;
+            hi = n;                                 // first position whose score is < tau
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (__float_as_uint(ev[(size_t)mid * C + j]) >= tau) lo = mid + 1; else hi = mid;
+            }
+            eq = lo - gt;
+        }
+        // exclusive prefix sum of eq over the chunk
+        unsigned long long incl = (unsigned long long)eq;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned long long o = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (lane == 31) warp_sum[wid] = incl;
+        __syncthreads();
+        if (wid == 0) {
+            unsigned long long w = warp_sum[lane];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned long long o = __shfl_up_sync(0xffffffffu, w, off);
+                if (lane >= off) w += o;
+            }
+            warp_sum[lane] = w;                     // inclusive over warps
+        }
+        __syncthreads();
+        const unsigned long long before = carry_s + (wid > 0 ? warp_sum[wid - 1] : 0ull) + incl - (unsigned long long)eq;
+        int c = 0;
+        if (j < C && !none) {
+            const unsigned long long left = r > before ? r - before : 0ull;
+            c = gt + (int)((unsigned long long)eq < left ? (unsigned long long)eq : left);
+            cut[j] = c;
+        } else if (j < C) {
+            cut[j] = 0;
+        }
+        // block sum of c
+        long long cs = c;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) cs += __shfl_xor_sync(0xffffffffu, cs, off);
+        __syncthreads();
+        if (lane == 0 && cs) atomicAdd((unsigned long long *)&nsel_s, (unsigned long long)cs);
+        if (tid == 0) carry_s += warp_sum[31];
+        __syncthreads();
+    }
+    if (tid == 0) {
+        st->nsel = nsel_s;
+        if (nsel_out) *nsel_out = nsel_s;
+    }
+}
+
+// mask[i][j] = 1 when kernel (i, j) left its column's list before the column's cut.
+__global__ void __launch_bounds__(256) bed_mask_kernel(const uint16_t *__restrict__ order, const int *__restrict__ cut, int M, int C,
+                                                       uint8_t *__restrict__ mask)
+{
+    __shared__ uint8_t tile[32][33];
+    const int i0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int jj = ty; jj < 32; jj += 8) {
+        const int j = j0 + jj, i = i0 + tx;
+        uint8_t v = 0;
+        if (i < M && j < C) v = (int)order[(size_t)j * M + i] < cut[j] ? 1 : 0;
+        tile[jj][tx] = v;
+    }
+    __syncthreads();
+    for (int ii = ty; ii < 32; ii += 8) {
+        const int i = i0 + ii, j = j0 + tx;
+        if (i < M && j < C) mask[(size_t)i * C + j] = tile[tx][ii];
+    }
+}
+
+static int check(cudaError_t e)
+{
+    if (e == cudaSuccess) return UBP_OK;
+    set_last_cuda_error((int)e);
+    return UBP_E_CUDA;
+}
+
+static int check_dims(int M, int C, int R, int Nb)
+{
+    if (M < 1 || C < 1 || R < 1 || Nb < 1 || Nb > M) return UBP_E_ARG;
+    if (M > MAX_M || (int64_t)M * C >= ((int64_t)1 << 31)) return UBP_E_UNSUPPORTED;
+    return UBP_OK;
+}
+
+static int launch_scores(const float *W, int M, int C, int R, int Nb, float *aT, float *S, cudaStream_t st)
+{
+    dim3 g1((unsigned)((C + 31) / 32), (unsigned)((M + 31) / 32));
+    bed_norm_kernel<<<g1, 256, 0, st>>>(W, M, C, R, aT);
+    const size_t mc = (size_t)M * C;
+    bed_window_kernel<<<(unsigned)((mc + 255) / 256), 256, 0, st>>>(aT, M, C, Nb, S);
+    return check(cudaGetLastError());
+}
+
+}  // namespace bed
+}  // namespace ubp
+
+using namespace ubp::bed;
+
+extern "C" {
+
+int ubp_bed_workspace_size(int M, int C, int Nb, size_t *dev_bytes)
+{
+    if (!dev_bytes) return UBP_E_ARG;
+    if (int rc = check_dims(M, C, 1, Nb)) return rc;
+    *dev_bytes = carve(nullptr, M, C, Nb).bytes;
+    return UBP_OK;
+}
+
+int ubp_block_scores(const float *W, int M, int C, int R, int Nb, void *workspace, size_t workspace_bytes,
+                     float *S, void *stream)
+{
+    if (!W || !workspace || !S) return UBP_E_ARG;
+    if (int rc = check_dims(M, C, R, Nb)) return rc;
+    if (((uintptr_t)workspace & 255u) != 0) return UBP_E_ARG;
+    Workspace w = carve(workspace, M, C, Nb);
+    if (workspace_bytes < w.bytes) return UBP_E_SPACE;
+    return launch_scores(W, M, C, R, Nb, w.aT, S, (cudaStream_t)stream);
+}
+
+int ubp_bed_select(const float *W, int M, int C, int R, int Nb, int64_t m, void *workspace, size_t workspace_bytes,
+                   uint8_t *mask, int64_t *n_selected, void *stream)
+{
+    if (!W || !workspace || !mask || m < 0) return UBP_E_ARG;
+    if (int rc = check_dims(M, C, R, Nb)) return rc;
+    if (((uintptr_t)workspace & 255u) != 0) return UBP_E_ARG;
+    Workspace w = carve(workspace, M, C, Nb);
+    if (workspace_bytes < w.bytes) return UBP_E_SPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = launch_scores(W, M, C, R, Nb, w.aT, w.S, st)) return rc;
+
+    const int Mpad = (M + 127) & ~127;
+    const size_t smem = (size_t)Mpad * 4 + (size_t)(M + 1) * 4 + (size_t)(Nb + 1) * 4;
+    if (smem > 48 * 1024)
+        if (int rc = check(cudaFuncSetAttribute(bed_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)))
+            return rc;
+    bed_expand_kernel<<<(unsigned)C, 32, smem, st>>>(w.S, M, C, Nb, Mpad, w.ev, w.order, w.nev);
+    if (int rc = check(cudaGetLastError())) return rc;
+
+    if (int rc = check(cudaMemsetAsync(w.sel, 0, sizeof(SelState), st))) return rc;
+    const int T = M / Nb;
+    const size_t total = (size_t)T * C;
+    unsigned hb = (unsigned)((total + 255) / 256);
+    if (hb > 1184) hb = 1184;
+    if (hb < 1) hb = 1;
+    for (int pass = 0; pass < 4; ++pass) {
+        bed_hist_kernel<<<hb, 256, 0, st>>>(w.ev, w.nev, T, C, pass, w.sel);
+        bed_pick_kernel<<<1, 32, 0, st>>>(pass, (long long)m, w.sel);
+    }
+    bed_cut_kernel<<<1, 1024, 0, st>>>(w.ev, w.nev, C, w.sel, w.cut, (long long *)n_selected);
+    dim3 gm((unsigned)((M + 31) / 32), (unsigned)((C + 31) / 32));
+    bed_mask_kernel<<<gm, 256, 0, st>>>(w.order, w.cut, M, C, mask);
+    return check(cudaGetLastError());
+}
+
+}  // extern "C"

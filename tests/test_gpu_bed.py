@@ -1,0 +1,129 @@
+"""Block selection on the device (block scores, expansion and division) against the sequential CPU oracle:
+scores and masks must be identical bit for bit, on layers with many equal scores too."""
+import numpy as np
+import pytest
+
+import oracle
+import ubp_synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(W):
+    import torch
+    return torch.from_numpy(W).cuda()
+
+
+CASES = [
+    # M, C, R, Nb, sparsity %, kind
+    (64, 48, 1, 4, 70, "trained"),
+    (96, 32, 9, 8, 80, "trained"),
+    (50, 40, 1, 2, 50, "normal"),          # rows not a multiple of the block size
+    (33, 20, 1, 16, 50, "trained"),
+    (128, 130, 1, 4, 90, "trained"),       # more columns than one chunk of warps in the tie pass needs
+    (200, 64, 9, 2, 50, "trained"),
+    (64, 64, 1, 1, 75, "trained"),         # element pruning
+    (48, 24, 1, 4, 60, "integer"),         # many ties, inside columns and across them
+    (40, 1100, 1, 4, 80, "integer"),       # ties spread over more than 1024 columns
+    (257, 16, 1, 32, 40, "integer"),
+    (130, 12, 1, 64, 50, "trained"),       # block longer than a warp
+    (8, 8, 1, 8, 0, "trained"),            # one block per column, all kept
+    (384, 96, 1, 4, 50, "trained"),
+]
+
+
+@pytest.mark.parametrize("M,C,R,Nb,p,kind", CASES)
+def test_scores_and_mask_match_the_sequential_oracle(M, C, R, Nb, p, kind):
+    import torch
+    import paper_2407_19644_b200 as ubp
+    W = ubp_synth.selection_weights(M, C, R, seed=7 * M + C + Nb, kind=kind)
+    m = oracle.block_budget(M, C, p, Nb)
+    S_ref = oracle.block_scores(W, Nb)
+    mask_ref, I, Ibar = oracle.bed_select(W, Nb, m)
+    sel = ubp.BedSelector(M, C, R, Nb)
+    Wd = _dev(W)
+    S = sel.scores(Wd).cpu().numpy().ravel()
+    assert np.array_equal(S.view(np.uint32), S_ref.view(np.uint32))
+    mask, nsel = sel.select(Wd, m)
+    torch.cuda.synchronize()
+    assert int(nsel.item()) == Ibar.size
+    assert np.array_equal(mask.cpu().numpy(), mask_ref)
+    # and the mask goes straight into the packer: the blocks it decodes are the oracle's
+    blob = ubp.pack_ubp(W, mask.cpu().numpy(), Nb)
+    v = ubp.blob_view(blob)
+    assert v["m"] == Ibar.size
+    starts = np.repeat(np.arange(M), np.diff(v["indptr"])) + M * v["indices"].astype(np.int64)
+    assert np.array_equal(np.sort(starts), I)
+
+
+@pytest.mark.parametrize("m", [0, 1, 5, 10**6])
+def test_budget_of_zero_one_and_more_than_fits(m):
+    import torch
+    import paper_2407_19644_b200 as ubp
+    M, C, Nb = 23, 9, 3                     # 7 blocks per column at most
+    W = ubp_synth.selection_weights(M, C, 1, seed=77, kind="integer")
+    W[W == 0] = 1.0
+    mask_ref, I, Ibar = oracle.bed_select(W, Nb, min(m, 10**4))
+    mask, nsel = ubp.ubp_bed_select(_dev(W), Nb, m)
+    assert int(nsel.item()) == Ibar.size == min(m, 7 * C)
+    assert np.array_equal(mask.cpu().numpy(), mask_ref)
+
+
+def test_repeated_calls_reuse_the_scratch_and_give_the_same_mask():
+    import torch
+    import paper_2407_19644_b200 as ubp
+    M, C, Nb = 256, 64, 4
+    sel = ubp.BedSelector(M, C, 1, Nb)
+    first = None
+    for rep in range(3):
+        for seed, p in ((1, 50), (2, 90)):
+            W = ubp_synth.selection_weights(M, C, 1, seed=seed, kind="trained")
+            mask, nsel = sel.select(_dev(W), oracle.block_budget(M, C, p, Nb))
+            torch.cuda.synchronize()
+            got = mask.cpu().numpy()
+            if rep == 0:
+                ref = oracle.bed_select(W, Nb, oracle.block_budget(M, C, p, Nb))[0]
+                assert np.array_equal(got, ref)
+                first = first or {}
+                first[(seed, p)] = got
+            else:
+                assert np.array_equal(got, first[(seed, p)])
+
+
+def test_full_size_layer_properties_and_sampled_columns():
+    """512 x 512 x 3x3 at 50 % with blocks of two (the selection the paper reports as its slowest: Section 5.2).
+    The sequential oracle is far too slow here, so: invariants that hold at any size, and a check that only
+    needs per-column work -- every column's kept kernels must be what the oracle keeps when it is run on that
+    column alone with the column's own number of blocks (the columns only meet in the global arg max)."""
+    import torch
+    import paper_2407_19644_b200 as ubp
+    M, C, R, Nb, p = 512, 512, 9, 2, 50
+    W = ubp_synth.selection_weights(M, C, R, seed=4242, kind="trained")
+    m = oracle.block_budget(M, C, p, Nb)
+    mask, nsel = ubp.ubp_bed_select(_dev(W), Nb, m)
+    mask = mask.cpu().numpy()
+    assert int(nsel.item()) == m and int(mask.sum()) == m * Nb
+    bi, bj = oracle.decode_mask(mask, Nb)                    # raises on a run that is not whole blocks
+    assert bi.size == m and (bi + Nb <= M).all()
+    a = np.abs(W.astype(np.float64)).sum(axis=2)
+    kept = a[mask == 1].sum()
+    al = a.reshape(M // Nb, Nb, C).sum(axis=1).ravel()
+    abp = np.sort(al)[::-1][:m].sum()
+    ep = np.sort(a.ravel())[::-1][:m * Nb].sum()
+    assert abp < kept < ep                                   # efficacy strictly between aligned and element pruning
+    rng = np.random.default_rng(5)
+    for j in rng.choice(C, 6, replace=False):
+        nj = int(mask[:, j].sum()) // Nb
+        ref = oracle.bed_select(W[:, j:j + 1, :], Nb, nj)[0]
+        assert np.array_equal(mask[:, j], ref[:, 0])
+    # the threshold is global: no column's next choice may score above another column's last kept choice
+    S = oracle.block_scores(W, Nb).reshape(C, M)
+    last_kept, next_left = [], []
+    for j in rng.choice(C, 12, replace=False):
+        nj = int(mask[:, j].sum()) // Nb
+        _, sc = oracle.bed_expand(S[j], Nb, nj + 1)
+        if nj > 0:
+            last_kept.append(sc[nj - 1])
+        if sc.size > nj:
+            next_left.append(sc[nj])
+    assert max(next_left) <= min(last_kept)
