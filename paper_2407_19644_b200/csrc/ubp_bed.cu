@@ -30,12 +30,16 @@ namespace bed {
 constexpr uint16_t NONE = 0xFFFFu;
 constexpr int MAX_M = 16384;
 
+constexpr int FINE_SHIFT = 19;      // fine histogram bin = score bits >> 19 (below 4096 for finite scores)
+constexpr int COARSE_SHIFT = 24;    // coarse histogram bin = score bits >> 24 = 32 fine bins
+
 struct SelState {
-    unsigned int hist[4][256];
-    unsigned int prefix;      // bits of the threshold score found so far
-    unsigned int none;        // 1 = nothing to select
-    unsigned long long rank;  // how many of the entries matching `prefix` are still to be taken
-    long long nsel;           // blocks selected in the end
+    unsigned int coarse[128];    // chosen scores so far, by sign and the top seven exponent bits
+    unsigned int fine[4096];     // and by sign, exponent and the top four mantissa bits
+    unsigned int hist[4][256];   // radix-select histograms, one per pass
+    unsigned int tau_lb;         // bits of a lower bound on the m-th largest chosen score (only ever rises)
+    unsigned int pad;
+    long long nsel;              // blocks selected in the end
 };
 
 struct Workspace {
@@ -108,10 +112,68 @@ __global__ void __launch_bounds__(256) bed_window_kernel(const float *__restrict
 }
 
 // ---------------------------------------------------------------------------------------------------------------
+// A lower bound on the m-th largest chosen score, shared by all columns while they run: every chosen score is
+// counted in two histograms of its bit pattern (128 bins by sign and the top seven exponent bits; 4096 bins by
+// sign, exponent and four mantissa bits), and the lower edge of the highest fine bin with at least m scores at or
+// above it can only rise. A column whose best remaining score is below the bound stops: nothing it could still
+// choose can be among the m best (its later scores are no larger).
+// Warp-collective: lane l holds coarse bins [4 l, 4 l + 4), then fine bin l of the coarse bin where the count crosses m.
+__device__ __forceinline__ void refresh_bound(SelState *st, unsigned long long m, int lane)
+{
+    const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(st->coarse) + lane);
+    const unsigned int c4[4] = {v.x, v.y, v.z, v.w};
+    const unsigned long long t = (unsigned long long)v.x + v.y + v.z + v.w;
+    unsigned long long incl = t;                 // sum over lanes >= lane
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long o = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += o;
+    }
+    unsigned long long above = incl - t;
+    const bool mine = above < m && incl >= m;
+    int cb = 0;
+    if (mine) {
+        bool found = false;
+#pragma unroll
+        for (int b = 3; b >= 0; --b)
+            if (!found) {
+                if (above + c4[b] >= m) { cb = lane * 4 + b; found = true; }
+                else above += c4[b];
+            }
+    }
+    const unsigned int who = __ballot_sync(0xffffffffu, mine);
+    if (who == 0u) return;                       // fewer than m scores so far
+    const int src = __ffs(who) - 1;
+    cb = __shfl_sync(0xffffffffu, cb, src);
+    above = __shfl_sync(0xffffffffu, above, src);    // scores in coarse bins above cb
+    const unsigned long long f = __ldcg(st->fine + cb * 32 + lane);
+    unsigned long long fin = f;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long o = __shfl_down_sync(0xffffffffu, fin, off);
+        if (lane + off < 32) fin += o;
+    }
+    // the highest fine bin with at least m scores at or above it (the counts may have grown since the first look,
+    // which only makes the bound found here lower than it could be)
+    const unsigned int ok = __ballot_sync(0xffffffffu, above + fin >= m);
+    if (ok != 0u && lane == 0) atomicMax(&st->tau_lb, (unsigned int)(cb * 32 + (31 - __clz(ok))) << FINE_SHIFT);
+}
+
+__device__ __forceinline__ void flush_counts(SelState *st, unsigned int bin, unsigned int cnt)
+{
+    if (cnt) {
+        atomicAdd(&st->fine[bin], cnt);
+        atomicAdd(&st->coarse[bin >> (COARSE_SHIFT - FINE_SHIFT)], cnt);
+    }
+}
+
 // Algorithm 1 for one input channel per warp. Shared memory per warp: the scores (padded with -inf to a multiple
 // of 128), a doubly linked list over the entries still in the list (entry M = end marker), and the positions met
-// while walking N steps to either side of the chosen entry.
-__global__ void __launch_bounds__(32) bed_expand_kernel(const float *__restrict__ S, int M, int C, int Nb, int Mpad,
+// while walking N steps to either side of the chosen entry. Lane l owns the entries of the float4 groups
+// l, l + 32, ... and keeps their maximum in registers; after a choice only the lanes that own a changed entry
+// look at their entries again.
+__global__ void __launch_bounds__(32) bed_expand_kernel(const float *__restrict__ S, int M, int C, int Nb, int Mpad, int T,
+                                                        unsigned long long m, SelState *st,
                                                         float *__restrict__ ev, uint16_t *__restrict__ order,
                                                         int *__restrict__ nev)
 {
@@ -134,28 +196,41 @@ __global__ void __launch_bounds__(32) bed_expand_kernel(const float *__restrict_
     __syncwarp();
 
     const float4 *s4 = reinterpret_cast<const float4 *>(s);
-    const int nq = Mpad >> 2;
-    const int T = M / Nb;
+    const int G = Mpad >> 7;                        // float4 groups per lane
+    float lbest;
+    int lidx;
+    // maximum of this lane's entries and the lowest position that holds it: the first float4 group that reaches the
+    // maximum, then the first component of that group
+    auto rescan = [&]() {
+        float mx = NEG;
+        int gb = 0;
+#pragma unroll 4
+        for (int g = 0; g < G; ++g) {
+            const float4 v = s4[lane + 32 * g];
+            const float m4 = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+            if (m4 > mx) { mx = m4; gb = g; }
+        }
+        const float4 v = s4[lane + 32 * gb];
+        const int base = (lane + 32 * gb) << 2;
+        lidx = v.x == mx ? base : v.y == mx ? base + 1 : v.z == mx ? base + 2 : base + 3;
+        lbest = mx;
+    };
+    rescan();
+
+    unsigned int tau_next = __ldcg(&st->tau_lb);
+    unsigned int pend_bin = 0, pend_cnt = 0;        // lane 0: chosen scores not yet added to the shared histograms
+    float *evp = ev + j;
     int it = 0;
     for (; it < T; ++it) {
-        // arg max, lowest position among equals
-        float best = NEG;
-        int bidx = 0x7fffffff;
-        for (int q = lane; q < nq; q += 32) {
-            const float4 v = s4[q];
-            const int base = q << 2;
-            if (v.x > best) { best = v.x; bidx = base; }
-            if (v.y > best) { best = v.y; bidx = base + 1; }
-            if (v.z > best) { best = v.z; bidx = base + 2; }
-            if (v.w > best) { best = v.w; bidx = base + 3; }
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ob = __shfl_xor_sync(0xffffffffu, best, off);
-            const int oi = __shfl_xor_sync(0xffffffffu, bidx, off);
-            if (ob > best || (ob == best && oi < bidx)) { best = ob; bidx = oi; }
-        }
-        if (!(best > NEG)) break;
+        // arg max, lowest position among equals. Scores are finite and >= 0 (or -inf), so their order is the
+        // order of their bit patterns; bits + 1 leaves 0 for -inf.
+        const unsigned int kb = lbest > NEG ? __float_as_uint(lbest) + 1u : 0u;
+        const unsigned int mk = __reduce_max_sync(0xffffffffu, kb);
+        if (mk == 0u) break;
+        const int bidx = (int)__reduce_min_sync(0xffffffffu, kb == mk ? (unsigned int)lidx : 0x7fffffffu);
+        const float best = __uint_as_float(mk - 1u);
+        if (__float_as_uint(best) < tau_next) break;        // below the m-th largest score of the whole layer
+        tau_next = __ldcg(&st->tau_lb);                      // looked at in the next round
         const int k = bidx;
         // the N entries after k (lane 0) and before it (lane 1) that are still in the list
         if (lane < 2) {
@@ -168,12 +243,14 @@ __global__ void __launch_bounds__(32) bed_expand_kernel(const float *__restrict_
             }
         }
         __syncwarp();
+        unsigned int dirty = 0;
         // entry n to the left now spans n kernels before the block and N-n after it
         for (int n = 1 + lane; n < Nb; n += 32) {
             const unsigned p = wk[(Nb + 1) + n];
             if (p != NONE) {
                 const unsigned r = wk[Nb - n];
                 s[p] = (s[p] + s[r]) - best;
+                dirty |= 1u << ((p >> 2) & 31u);
             }
         }
         __syncwarp();
@@ -181,29 +258,109 @@ __global__ void __launch_bounds__(32) bed_expand_kernel(const float *__restrict_
             const unsigned idx = t == 0 ? (unsigned)k : wk[t];
             s[idx] = NEG;
             oj[idx] = (uint16_t)it;
+            dirty |= 1u << ((idx >> 2) & 31u);
         }
         if (lane == 0) {
             const unsigned p1 = wk[(Nb + 1) + 1], sN = wk[Nb];
             if (p1 != NONE) nxt[p1] = (uint16_t)sN;
             prv[sN] = (uint16_t)p1;
-            ev[(size_t)it * C + j] = best;
+            *evp = best;
+            evp += C;
+            // count it; a column's scores fall, so equal bins come in runs: one update per run
+            const unsigned int bin = __float_as_uint(best) >> FINE_SHIFT;
+            if (bin != pend_bin) {
+                flush_counts(st, pend_bin, pend_cnt);
+                pend_bin = bin;
+                pend_cnt = 0;
+            }
+            ++pend_cnt;
         }
+        dirty = __reduce_or_sync(0xffffffffu, dirty);
         __syncwarp();
+        if ((dirty >> lane) & 1u) rescan();
+        if ((it & 15) == 15) {
+            if (lane == 0) { flush_counts(st, pend_bin, pend_cnt); pend_cnt = 0; }
+            refresh_bound(st, m, lane);
+        }
     }
-    if (lane == 0) nev[j] = it;
+    if (lane == 0) {
+        flush_counts(st, pend_bin, pend_cnt);
+        nev[j] = it;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------------------------
 // The m-th largest chosen score over all columns: radix select over the bit patterns (scores are finite and >= 0,
-// so unsigned order of the bits is the order of the values), 8 bits per pass from the top.
+// so unsigned order of the bits is the order of the values), 8 bits per pass from the top. The digit a pass settles
+// is read off its histogram by whoever needs it next (warp-collective; lane l holds bins [8 l, 8 l + 8)).
+__device__ __forceinline__ void settle_digit(const unsigned int *hist_row, int shift, unsigned int &prefix,
+                                             unsigned long long &rank, int lane)
+{
+    unsigned int v[8];
+    unsigned long long t = 0;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) { v[b] = __ldcg(hist_row + lane * 8 + b); t += v[b]; }
+    unsigned long long incl = t;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long o = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += o;
+    }
+    const unsigned long long above = incl - t;
+    const bool mine = above < rank && incl >= rank;
+    unsigned int d = 0;
+    unsigned long long nr = 0;
+    if (mine) {
+        unsigned long long cum = above;
+#pragma unroll
+        for (int b = 7; b >= 0; --b) {
+            if (nr == 0) {
+                if (cum + v[b] >= rank) { d = (unsigned)(lane * 8 + b); nr = rank - cum; }
+                else cum += v[b];
+            }
+        }
+    }
+    const unsigned int who = __ballot_sync(0xffffffffu, mine);
+    const int src = who ? __ffs(who) - 1 : 0;
+    d = __shfl_sync(0xffffffffu, d, src);
+    nr = __shfl_sync(0xffffffffu, nr, src);
+    prefix |= d << shift;
+    rank = nr;
+}
+
+// (prefix, rank) after `passes` settled digits; rank = 0 means there is nothing to select. Warp-collective.
+__device__ __forceinline__ void settled(const SelState *st, int passes, unsigned long long m, unsigned int &prefix,
+                                        unsigned long long &rank, int lane)
+{
+    prefix = 0;
+    rank = 0;
+    if (passes == 0) return;
+    unsigned long long t = 0;
+    for (int b = lane; b < 256; b += 32) t += __ldcg(&st->hist[0][b]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+    rank = m < t ? m : t;
+    if (rank == 0) return;
+    for (int p = 0; p < passes; ++p) settle_digit(st->hist[p], 24 - 8 * p, prefix, rank, lane);
+}
+
 __global__ void __launch_bounds__(256) bed_hist_kernel(const float *__restrict__ ev, const int *__restrict__ nev, int T, int C,
-                                                       int pass, SelState *st)
+                                                       int pass, unsigned long long m, SelState *st)
 {
     __shared__ unsigned int h[256];
+    __shared__ unsigned int prefix_s;
+    __shared__ unsigned long long rank_s;
     h[threadIdx.x] = 0;
+    if (threadIdx.x < 32) {
+        unsigned int prefix;
+        unsigned long long rank;
+        settled(st, pass, m, prefix, rank, threadIdx.x);
+        if (threadIdx.x == 0) { prefix_s = prefix; rank_s = rank; }
+    }
     __syncthreads();
+    if (pass > 0 && rank_s == 0) return;
     const int shift = 24 - 8 * pass;
-    const unsigned int prefix = st->prefix;
+    const unsigned int prefix = prefix_s;
     const size_t total = (size_t)T * C;
     for (size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x; idx < total; idx += (size_t)gridDim.x * 256) {
         const int j = (int)(idx % (size_t)C), t = (int)(idx / (size_t)C);
@@ -216,43 +373,29 @@ __global__ void __launch_bounds__(256) bed_hist_kernel(const float *__restrict__
     if (h[threadIdx.x]) atomicAdd(&st->hist[pass][threadIdx.x], h[threadIdx.x]);
 }
 
-__global__ void bed_pick_kernel(int pass, long long m, SelState *st)
-{
-    if (threadIdx.x != 0) return;
-    unsigned long long rank = st->rank;
-    if (pass == 0) {
-        unsigned long long tot = 0;
-        for (int d = 0; d < 256; ++d) tot += st->hist[0][d];
-        rank = (unsigned long long)m < tot ? (unsigned long long)m : tot;
-        st->none = rank == 0 ? 1u : 0u;
-    }
-    if (st->none) { st->rank = 0; return; }
-    const int shift = 24 - 8 * pass;
-    unsigned long long cum = 0;
-    int d = 255;
-    for (; d > 0; --d) {
-        const unsigned long long hd = st->hist[pass][d];
-        if (cum + hd >= rank) break;
-        cum += hd;
-    }
-    st->prefix |= (unsigned int)d << shift;
-    st->rank = rank - cum;
-}
-
 // Per column: how many of its chosen blocks score above the threshold, how many exactly at it; ties are handed out
 // to the lowest input channels first. One CTA, columns in chunks of 1024 with a running carry.
 __global__ void __launch_bounds__(1024) bed_cut_kernel(const float *__restrict__ ev, const int *__restrict__ nev, int C,
-                                                        SelState *st, int *__restrict__ cut, long long *nsel_out)
+                                                        unsigned long long m, SelState *st, int *__restrict__ cut,
+                                                        long long *nsel_out)
 {
     __shared__ unsigned long long warp_sum[32];
     __shared__ unsigned long long carry_s;
     __shared__ long long nsel_s;
+    __shared__ unsigned int tau_s;
+    __shared__ unsigned long long r_s;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     if (tid == 0) { carry_s = 0; nsel_s = 0; }
+    if (wid == 0) {
+        unsigned int prefix;
+        unsigned long long rank;
+        settled(st, 4, m, prefix, rank, lane);
+        if (lane == 0) { tau_s = prefix; r_s = rank; }
+    }
     __syncthreads();
-    const unsigned int tau = st->prefix;
-    const unsigned long long r = st->rank;
-    const bool none = st->none != 0;
+    const unsigned int tau = tau_s;
+    const unsigned long long r = r_s;
+    const bool none = r == 0;
     for (int j0 = 0; j0 < C; j0 += 1024) {
         const int j = j0 + tid;
         int gt = 0, eq = 0;
@@ -295,11 +438,8 @@ __global__ void __launch_bounds__(1024) bed_cut_kernel(const float *__restrict__
         if (j < C && !none) {
             const unsigned long long left = r > before ? r - before : 0ull;
             c = gt + (int)((unsigned long long)eq < left ? (unsigned long long)eq : left);
-            cut[j] = c;
-        } else if (j < C) {
-            cut[j] = 0;
         }
-        // block sum of c
+        if (j < C) cut[j] = c;
         long long cs = c;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) cs += __shfl_xor_sync(0xffffffffu, cs, off);
@@ -399,20 +539,18 @@ int ubp_bed_select(const float *W, int M, int C, int R, int Nb, int64_t m, void 
     if (smem > 48 * 1024)
         if (int rc = check(cudaFuncSetAttribute(bed_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)))
             return rc;
-    bed_expand_kernel<<<(unsigned)C, 32, smem, st>>>(w.S, M, C, Nb, Mpad, w.ev, w.order, w.nev);
-    if (int rc = check(cudaGetLastError())) return rc;
-
     if (int rc = check(cudaMemsetAsync(w.sel, 0, sizeof(SelState), st))) return rc;
     const int T = M / Nb;
+    bed_expand_kernel<<<(unsigned)C, 32, smem, st>>>(w.S, M, C, Nb, Mpad, m > 0 ? T : 0, (unsigned long long)m, w.sel,
+                                                     w.ev, w.order, w.nev);
+    if (int rc = check(cudaGetLastError())) return rc;
     const size_t total = (size_t)T * C;
     unsigned hb = (unsigned)((total + 255) / 256);
     if (hb > 1184) hb = 1184;
     if (hb < 1) hb = 1;
-    for (int pass = 0; pass < 4; ++pass) {
-        bed_hist_kernel<<<hb, 256, 0, st>>>(w.ev, w.nev, T, C, pass, w.sel);
-        bed_pick_kernel<<<1, 32, 0, st>>>(pass, (long long)m, w.sel);
-    }
-    bed_cut_kernel<<<1, 1024, 0, st>>>(w.ev, w.nev, C, w.sel, w.cut, (long long *)n_selected);
+    for (int pass = 0; pass < 4; ++pass)
+        bed_hist_kernel<<<hb, 256, 0, st>>>(w.ev, w.nev, T, C, pass, (unsigned long long)m, w.sel);
+    bed_cut_kernel<<<1, 1024, 0, st>>>(w.ev, w.nev, C, (unsigned long long)m, w.sel, w.cut, (long long *)n_selected);
     dim3 gm((unsigned)((M + 31) / 32), (unsigned)((C + 31) / 32));
     bed_mask_kernel<<<gm, 256, 0, st>>>(w.order, w.cut, M, C, mask);
     return check(cudaGetLastError());
