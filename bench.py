@@ -48,6 +48,18 @@ for _li in range(13):
     WORKLOADS[f"mbv1_L{_li + 1}"] = dict(cfg="mbv1_chain", kw={}, index=_li)
 
 
+# Block selection (expansion and division, Section 4.1) on dense weights: M x C x R, block size, sparsity %.
+# bed_r50_3x3 is the case Section 5.2 names as the slowest selection of its experiments (ResNet50's largest layers,
+# block size 2, 50 % sparsity); bed_mbv1_pw1024 is MobileNetV1's largest pointwise layer at the setting of the
+# Section 3.2 example (block size 4, 90 %).
+BED_WORKLOADS = {
+    "bed_r50_3x3": (512, 512, 9, 2, 50),
+    "bed_mbv1_pw1024": (1024, 1024, 1, 4, 90),
+    "bed_2048_nb2_p50": (2048, 2048, 1, 2, 50),
+    "bed_2048_nb4_p70": (2048, 2048, 1, 4, 70),
+}
+
+
 def get_layer(name: str, seed_index: int = 0):
     w = WORKLOADS[name]
     layers = ubp_synth.config_layers(w["cfg"], index=seed_index, **w["kw"])
@@ -345,6 +357,134 @@ def run_reference(args, L, name):
     print(json.dumps(line), flush=True)
 
 
+def cpu_bed_time(W, Nb: int, m: int, budget_s: float = 15.0):
+    """Time of the sequential oracle (scores, Algorithm 1, Algorithm 2) for this layer on the host. Algorithm 1 is run
+    for a bounded number of its m iterations (each costs the same arg max over the remaining score list) and scaled."""
+    import oracle
+    t0 = time.perf_counter()
+    S = oracle.block_scores(W, Nb)
+    t_scores = time.perf_counter() - t0
+    n = min(m, 64)
+    t0 = time.perf_counter()
+    oracle.bed_expand(S, Nb, n)
+    t_n = time.perf_counter() - t0
+    n2 = int(min(m, max(n, budget_s / max(t_n / max(n, 1), 1e-9))))
+    t0 = time.perf_counter()
+    Ibar, _ = oracle.bed_expand(S, Nb, n2)
+    t_exp = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    oracle.bed_divide(Ibar, Nb)
+    t_div = time.perf_counter() - t0
+    full = t_scores + (t_exp + t_div) * (m / max(n2, 1))
+    sample = (f"scores of the whole layer + first {n2} of {m} iterations of Algorithm 1 on the full score list "
+              f"(then Algorithm 2), scaled by {m / max(n2, 1):.2f}" if n2 < m else "the whole selection")
+    return full, 1, sample
+
+
+def run_bed(args, name, rank, local_rank, world):
+    """One step = one block selection (scores, expansion, threshold, mask) of the layer's dense weights resident in
+    HBM. Every rank selects for its own layer of the same shape (layers are independent: no collective)."""
+    M, C, R, Nb, p = BED_WORKLOADS[name]
+    W = ubp_synth.selection_weights(M, C, R, seed=9000 + rank, kind="trained")
+    m = ubp_synth.block_budget(M, C, p, Nb)
+    metric = "blocks selected per second by block expansion and division (m / time)"
+    cfg = {"workload": name, "M": M, "C": C, "R": R, "block": f"{Nb}x1x{R}", "sparsity_pct": p, "blocks": m,
+           "candidates": M * C}
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        import oracle
+        vals = []
+        for i in range(args.warmup + args.steps):
+            t, cores, sample = cpu_bed_time(W, Nb, m, budget_s=2.0)
+            if i >= args.warmup:
+                vals.append(t)
+            if i >= args.warmup + 2 and sum(vals) > 0 and (i + 1) * 3.0 > 120:
+                break
+        t = float(np.median(vals))
+        cfg["sample"] = sample
+        print(json.dumps({"metric": metric, "value": m / t, "unit": "blocks/s", "impl": "reference", "n_gpus": args.gpus,
+                          "steps": len(vals), "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg,
+                          "cpu_baseline": {"value": m / t, "unit": "blocks/s", "cores": cores, "kind": "oracle", "sample": sample},
+                          "e2e": {"value": m / t, "unit": "blocks/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}),
+              flush=True)
+        return
+    import torch
+    import paper_2407_19644_b200 as ubp
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    ubp.load()
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    sel = ubp.BedSelector(M, C, R, Nb)
+    Wd = torch.from_numpy(W).cuda()
+    mask = torch.empty((M, C), dtype=torch.uint8, device="cuda")
+    nsel = torch.zeros(1, dtype=torch.int64, device="cuda")
+    run = lambda: sel.select(Wd, m, mask, nsel)          # noqa: E731
+    if args.profile > 0:
+        for _ in range(args.profile):
+            run()
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_launches": args.profile, "workload": name, "selected": int(nsel.item())}), flush=True)
+        return
+    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    sampler = ClockSampler(local_rank)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    times = time_steps(torch, run, args.steps, args.warmup, flush)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if int(nsel.item()) != m:
+        raise SystemExit(f"selected {int(nsel.item())} blocks, wanted {m}")
+    step_ms = max_over_ranks(float(np.mean(times)), dist, torch, "cuda")
+    # end to end: weights from pinned host memory, mask back to pinned host memory
+    Wh = torch.from_numpy(W).pin_memory()
+    mh = torch.empty((M, C), dtype=torch.uint8).pin_memory()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    et = []
+    for i in range(3 + max(5, min(args.steps, 20))):
+        torch.cuda.synchronize()
+        e0.record()
+        Wd.copy_(Wh, non_blocking=True)
+        run()
+        mh.copy_(mask, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            et.append(e0.elapsed_time(e1))
+    e2e_ms = max_over_ranks(float(np.mean(et)), dist, torch, "cuda")
+    line = {
+        "metric": metric, "value": world * m / (step_ms * 1e-3), "unit": "blocks/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_ms, "us_min": float(np.min(times)) * 1e3,
+        "us_median": float(np.median(times)) * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": dict(cfg, l2="warm" if args.no_flush else "flushed between steps (256 MiB write)",
+                       parallelism=f"independent layers x{world}"),
+        "roofline": {"bound": "latency", "achieved": None, "peak": None, "unit": None, "frac": None, "traffic": None,
+                     "note": "a chain of dependent arg max / re-score rounds per input channel (at most M/Nb of them); "
+                             "neither memory traffic nor arithmetic is near a hardware limit",
+                     "candidates_per_second": M * C / (step_ms * 1e-3)},
+        "clocks": clocks, "gpu_launches": args.steps * 9,
+        "e2e": {"value": world * m / (e2e_ms * 1e-3), "unit": "blocks/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": W.nbytes, "d2h_bytes_per_step": M * C},
+    }
+    if rank == 0 and not args.no_cpu:
+        t, cores, sample = cpu_bed_time(W, Nb, m)
+        line["cpu_baseline"] = {"value": m / t, "unit": "blocks/s", "cores": cores, "kind": "oracle", "sample": sample,
+                                "seconds_for_the_layer": t}
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -382,6 +522,9 @@ def main():
         if dist is not None:
             dist.barrier()
             dist.destroy_process_group()
+        return
+    if name in BED_WORKLOADS:
+        run_bed(args, name, rank, local_rank, world)
         return
     L = get_layer(name, seed_index=rank)
 
