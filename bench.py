@@ -99,7 +99,7 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
 
 def compulsory_bytes(L) -> int:
     """Activations read once + outputs written once + packed weights/indices + bias."""
-    x = L.X.size * 4
+    x = L.C * L.Nc * 4
     y = L.M * L.Nc * 4
     w = L.m * L.Nb * L.R * 4 + L.m * 4 + (L.M + 1) * 4 + (L.M * 4 if L.bias is not None else 0)
     return x + y + w
@@ -266,15 +266,35 @@ def roofline_us(L, hbm_gbs):
     return (2.0 * L.surviving_macs / (FP32_PEAK_TFLOPS * 1e12) * 1e6, compulsory_bytes(L) / (hbm_gbs * 1e9) * 1e6)
 
 
-def run_chain(args, torch, ubp, rank, world, dist):
-    """The 13 pointwise layers of the MobileNetV1-shaped chain (batch 64, 1x4 blocks, 80 %, bias+ReLU, independent
-    seeded inputs per layer). One step = the 13 launches replayed from one CUDA graph."""
-    layers = ubp_synth.config_layers("mbv1_chain", index=rank)
+def build_chained(ubp, torch, layers, variant):
+    """Runners for layers that feed one another: layer i + 1 reads the output tensor of layer i."""
+    plans, runs, keep = [], [], []
+    x = torch.from_numpy(layers[0].X).cuda()
+    for L in layers:
+        plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb), variant)
+        bias = torch.from_numpy(L.bias).cuda() if L.bias is not None else None
+        y = torch.empty((L.M, L.B, L.H, L.Wd), dtype=torch.float32, device="cuda")
+        fn = ubp.ubp_conv3x3_implicit if L.R == 9 else ubp.ubp_conv1x1
+        runs.append(lambda fn=fn, plan=plan, x=x, bias=bias, relu=L.relu, y=y: fn(plan, x, bias, relu, out=y))
+        plans.append(plan); keep.append((x, y, bias))
+        x = y
+    return plans, runs, keep
+
+
+def run_chain(args, torch, ubp, rank, world, dist, cfg="mbv1_chain"):
+    """mbv1_chain: the 13 pointwise layers of the MobileNetV1-shaped network (batch 64, 1x4 blocks, 80 %, bias+ReLU,
+    independent seeded inputs per layer). r50_bottleneck: a ResNet-50-shaped bottleneck (1x1, 3x3, 1x1; batch 32,
+    blocks of 4, 80 %), each layer reading its predecessor's output. One step = all launches replayed from one
+    CUDA graph."""
+    layers = ubp_synth.config_layers(cfg, index=rank)
     hbm_gbs, peak_src = measured_peaks()
     runs, plans, keep = [], [], []
-    for L in layers:
-        plan, run, _, _, X, Y, bias = build_runner(ubp, torch, L, args.variant)
-        plans.append(plan); runs.append(run); keep.append((X, Y, bias))
+    if cfg == "r50_bottleneck":
+        plans, runs, keep = build_chained(ubp, torch, layers, args.variant)
+    else:
+        for L in layers:
+            plan, run, _, _, X, Y, bias = build_runner(ubp, torch, L, args.variant)
+            plans.append(plan); runs.append(run); keep.append((X, Y, bias))
     flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     for run in runs:            # warm every kernel outside the capture (first-launch attribute set-up)
         run()
@@ -299,20 +319,20 @@ def run_chain(args, torch, ubp, rank, world, dist):
     roofs = [roofline_us(L, hbm_gbs) for L in layers]
     roof_total_us = sum(max(r) for r in roofs)
     line = {
-        "metric": "effective GFLOP/s (2 x surviving MACs / time) of the 13-layer pointwise chain",
+        "metric": f"effective GFLOP/s (2 x surviving MACs / time) of the {len(layers)}-layer chain",
         "value": aggregate_gflops(flops, world, step_ms), "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "mbv1_chain", "layers": 13, "batch": 64, "block": "4x1x1", "sparsity_pct": 80,
-                   "launch": "13 kernels replayed from one CUDA graph",
+        "config": {"workload": cfg, "layers": len(layers), "batch": layers[0].B, "block": "4x1xR", "sparsity_pct": 80,
+                   "launch": f"{len(layers)} kernels replayed from one CUDA graph",
                    "l2": "warm" if args.no_flush else "flushed between steps (256 MiB write)"},
-        "roofline": {"bound": "mixed (layers 1-4 hbm, 5-13 alu)", "roofline_us": roof_total_us,
+        "roofline": {"bound": "mixed (per layer: see layers)", "roofline_us": roof_total_us,
                      "frac_of_roofline_time": roof_total_us / (step_ms * 1e3),
                      "peak_source": f"FP32 74.45 TFLOP/s derived; HBM {hbm_gbs} GB/s {peak_src}"},
-        "layers": [{"name": L.name, "M": L.M, "K": L.C, "Nc": L.Nc, "variant": p.variant, "us": us,
+        "layers": [{"name": L.name, "M": L.M, "K": L.C * L.R, "Nc": L.B * L.H * L.Wd, "variant": p.variant, "us": us,
                     "roofline_us": max(r), "bound": "alu" if r[0] >= r[1] else "hbm", "frac": max(r) / us}
                    for L, p, us, r in zip(layers, plans, per_layer, roofs)],
-        "clocks": clocks, "gpu_launches": 13 * args.steps,
+        "clocks": clocks, "gpu_launches": len(layers) * args.steps,
     }
     if rank == 0:
         print(json.dumps(line), flush=True)
@@ -505,7 +525,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     name = args.workload
-    if name == "mbv1_chain":
+    if name in ("mbv1_chain", "r50_bottleneck"):
         if args.impl == "reference":
             raise SystemExit("--impl reference times single layers; pick a layer workload")
         import torch
@@ -518,7 +538,7 @@ def main():
         if world > 1:
             import torch.distributed as dist
             dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-        run_chain(args, torch, ubp, rank, world, dist)
+        run_chain(args, torch, ubp, rank, world, dist, cfg=name)
         if dist is not None:
             dist.barrier()
             dist.destroy_process_group()

@@ -137,22 +137,41 @@ int orc_bed_divide(const int64_t *Ibar, int64_t cnt, int Nb, int64_t *I)
     return ORC_OK;
 }
 
-/* Eq. 3. Returns the number chosen (fewer than m when nothing finite is left); I in the order chosen. */
+/*
+ * Eq. 3, as the text describes it: candidates sorted by score (best first, lowest index among equals), walked in
+ * that order; a candidate is taken unless an earlier choice set it to -inf, and taking k sets k-N+1 .. k+N-1 to
+ * -inf. Returns the number chosen (fewer than m when nothing finite is left); I in the order chosen.
+ */
+static const float *g_sort_scores;
+static int cmp_score_desc(const void *a, const void *b)
+{
+    const int64_t x = *(const int64_t *)a, y = *(const int64_t *)b;
+    const float sx = g_sort_scores[x], sy = g_sort_scores[y];
+    if (sx > sy) return -1;
+    if (sx < sy) return 1;
+    return (x > y) - (x < y);
+}
+
 int64_t orc_greedy_select(const float *S_in, int64_t b, int Nb, int64_t m, int64_t *I)
 {
     if (!S_in || !I || b < 1 || Nb < 1 || m < 0) return ORC_E_ARG;
-    float *S = (float *)malloc((size_t)b * sizeof(float));
-    if (!S) return ORC_E_SPACE;
-    memcpy(S, S_in, (size_t)b * sizeof(float));
+    int64_t *ord = (int64_t *)malloc((size_t)b * sizeof(int64_t));
+    uint8_t *gone = (uint8_t *)calloc((size_t)b, 1);
+    if (!ord || !gone) { free(ord); free(gone); return ORC_E_SPACE; }
+    for (int64_t q = 0; q < b; ++q) ord[q] = q;
+    g_sort_scores = S_in;
+    qsort(ord, (size_t)b, sizeof(int64_t), cmp_score_desc);
     int64_t cnt = 0;
-    for (int64_t it = 0; it < m; ++it) {
-        const int64_t k = first_max(S, b);
-        if (!(S[k] > -INFINITY)) break;
+    for (int64_t q = 0; q < b && cnt < m; ++q) {
+        const int64_t k = ord[q];
+        if (!(S_in[k] > -INFINITY)) break;
+        if (gone[k]) continue;
         I[cnt++] = k;
         for (int64_t n = -(int64_t)Nb + 1; n < Nb; ++n)
-            if (k + n >= 0 && k + n < b) S[k + n] = -INFINITY;
+            if (k + n >= 0 && k + n < b) gone[k + n] = 1;
     }
-    free(S);
+    free(ord);
+    free(gone);
     return cnt;
 }
 

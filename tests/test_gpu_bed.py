@@ -127,3 +127,24 @@ def test_full_size_layer_properties_and_sampled_columns():
         if sc.size > nj:
             next_left.append(sc[nj])
     assert max(next_left) <= min(last_kept)
+
+
+@pytest.mark.parametrize("M,C,R,Nb,p", [(512, 512, 1, 4, 70), (256, 256, 9, 2, 50), (1024, 512, 1, 8, 90)])
+def test_efficacy_of_the_device_selection_is_above_greedy(M, C, R, Nb, p):
+    """The efficacy metric of Section 5.2 (kept l1 mass between aligned block pruning = 0 and element pruning = 1):
+    expansion and division on the device must keep more mass than greedy selection (Eq. 3, oracle) on layer-sized
+    inputs, as the paper's comparison reports."""
+    import paper_2407_19644_b200 as ubp
+    W = ubp_synth.selection_weights(M, C, R, seed=31 * Nb + p, kind="trained")
+    m = oracle.block_budget(M, C, p, Nb)
+    a = np.abs(W.astype(np.float64)).sum(axis=2)
+    ep = np.sort(a.ravel())[::-1][:m * Nb].sum()
+    abp = np.sort(a[:M // Nb * Nb].reshape(M // Nb, Nb, C).sum(axis=1).ravel())[::-1][:m].sum()
+    mask, nsel = ubp.ubp_bed_select(_dev(W), Nb, m)
+    assert int(nsel.item()) == m
+    kept = a[mask.cpu().numpy() == 1].sum()
+    g = oracle.greedy_select(oracle.block_scores(W, Nb), Nb, m)
+    kept_g = a[oracle.starts_to_mask(g, M, C, Nb) == 1].sum() if g.size == m else 0.0
+    eff, eff_g = (kept - abp) / (ep - abp), (kept_g - abp) / (ep - abp)
+    print(f"efficacy {M}x{C}x{R} N={Nb} {p}%: expansion+division {eff:.4f}, greedy {eff_g:.4f} ({g.size} of {m} blocks)")
+    assert 0.0 < eff < 1.0 and eff > eff_g

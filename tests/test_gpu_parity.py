@@ -464,3 +464,45 @@ def test_launches_can_be_captured_in_a_cuda_graph(env):
     Yref1, _ = oracle.masked_matmul(L1.W, L1.mask, L1.X, L1.bias, relu=True)
     Yref2, A2 = oracle.masked_matmul(L2.W, L2.mask, Yref1.astype(np.float32), L2.bias, relu=True)
     assert scaled_error(Y2.cpu().numpy(), Yref2, A2) <= TOL
+
+
+def test_bottleneck_trio_chained_through_fused_epilogues(env):
+    """A ResNet-50-shaped bottleneck (1x1 1024->256 + ReLU, 3x3 256->256 + ReLU, 1x1 256->1024), each layer reading
+    the previous layer's output tensor, eagerly and replayed from one CUDA graph. Every layer is checked against the
+    oracle evaluated on the activations that layer actually read."""
+    torch, ubp = env
+    layers = ubp_synth.config_layers("r50_bottleneck", batch=4)
+    x = torch.from_numpy(layers[0].X).cuda()
+    plans, outs, ins, runs = [], [], [], []
+    for L in layers:
+        plan = ubp.Plan(ubp.pack_ubp(L.W, L.mask, L.Nb))
+        bias = torch.from_numpy(L.bias).cuda()
+        y = torch.empty((L.M, L.B, L.H, L.Wd), dtype=torch.float32, device="cuda")
+        fn = ubp.ubp_conv3x3_implicit if L.R == 9 else ubp.ubp_conv1x1
+        runs.append(lambda fn=fn, plan=plan, x=x, bias=bias, relu=L.relu, y=y: fn(plan, x, bias, relu, out=y))
+        plans.append(plan); ins.append(x); outs.append(y)
+        x = y
+    for r in runs:
+        r()
+    torch.cuda.synchronize()
+    eager = [y.cpu().numpy().copy() for y in outs]
+    for L, plan, xin, y in zip(layers, plans, ins, eager):
+        plan.check()
+        xh = xin.cpu().numpy()
+        if L.R == 9:
+            Yref, A = oracle.masked_conv3x3(L.W, L.mask, xh, L.bias, relu=L.relu)
+        else:
+            Yref, A = oracle.masked_matmul(L.W, L.mask, xh.reshape(L.C, -1), L.bias, relu=L.relu)
+            Yref, A = Yref.reshape(y.shape), A.reshape(y.shape)
+        assert scaled_error(y, Yref, A) <= 1e-4
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    for y in outs:
+        y.zero_()
+    with torch.cuda.graph(g, stream=s):
+        for r in runs:
+            r()
+    g.replay()
+    torch.cuda.synchronize()
+    for y, e in zip(outs, eager):
+        assert np.array_equal(y.cpu().numpy(), e)

@@ -108,7 +108,9 @@ class Layer:
 
     @property
     def Nc(self) -> int:
-        return int(self.X.size // self.C)
+        if self.X.size:
+            return int(self.X.size // self.C)
+        return self.B * self.H * self.Wd        # made without activations: the conv view's column count
 
     @property
     def surviving_macs(self) -> int:
@@ -157,6 +159,7 @@ CONFIGS = {
     "r50_3x3": "3x3 conv 256->256 at 14x14, batch 64, pad 1, blocks 8x1x3x3, 80 %",
     "sweep": "M=K=2048, Nc=8192; Nb in {2,4,8,16} x sparsity in {50,70,80,90}",
     "mbv1_chain": "13 pointwise layers of MobileNetV1, batch 64, 1x4, 80 %, bias+ReLU",
+    "r50_bottleneck": "1x1 1024->256, 3x3 256->256, 1x1 256->1024 at 14x14, batch 32, blocks of 4, 80 %, chained",
 }
 
 
@@ -188,6 +191,14 @@ def config_layers(cfg: str, *, batch: Optional[int] = None, Nb: Optional[int] = 
             out.append(make_layer(f"mbv1_L{li + 1}", co, ci, 4, 80, 5000 + li, B=b, H=hw, Wd=hw,
                                   w_scale=0.05, bias=True, relu=True, make_x=make_x))
         return out
+    if cfg == "r50_bottleneck":
+        # a ResNet-50-shaped bottleneck of the 14x14 stage: 1x1 1024->256, 3x3 256->256, 1x1 256->1024;
+        # only the first layer's activations are an input, the other two read their predecessor's output
+        b = 32 if batch is None else batch
+        shapes = [(256, 1024, 1, True), (256, 256, 9, True), (1024, 256, 1, False)]
+        return [make_layer(f"r50_bn_{li + 1}", co, ci, 4, 80, 6000 + 10 * index + li, B=b, H=14, Wd=14, R=r,
+                           w_scale=0.03, bias=True, relu=relu, make_x=make_x and li == 0)
+                for li, (co, ci, r, relu) in enumerate(shapes)]
     raise KeyError(cfg)
 
 
