@@ -192,6 +192,24 @@ int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, 
                          const float *bias, int relu,
                          float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);
 
+/* Strided forms (the downsampling layers of ResNet-shaped networks). Output planes are Ho x Wo with
+ * Ho = (H-1)/stride + 1, Wo = (W-1)/stride + 1; strides of `out` are in elements of those planes.
+ * stride == 1 forwards to the call above.
+ * ubp_conv3x3_strided: 3x3, zero padding 1: out[b][o][yo][xo] = act(bias[o] + sum W[o][c][3r+s] *
+ *   in[b][c][yo*stride + r - 1][xo*stride + s - 1]). For stride > 1 every output pixel is computed by one lane that
+ *   reads its taps in place (correct for any layout, far from the roofline; the implicit-GEMM kernels are stride 1).
+ * ubp_conv1x1_strided: out[b][o][yo][xo] = act(bias[o] + sum W[o][c] * in[b][c][yo*stride][xo*stride]). For
+ *   stride > 1 the pixels read are first gathered into `scratch` (device, 16-byte aligned, at least
+ *   ubp_conv1x1_strided_scratch(C, B, H, W, stride) bytes, channel-major [C][B][Ho][Wo]) by one extra kernel, then the
+ *   stride-1 path runs on them. UBP_E_SPACE if the scratch is too small. */
+int ubp_conv3x3_strided(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
+                        int64_t in_stride_b, int64_t in_stride_c, const float *bias, int relu,
+                        float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);
+size_t ubp_conv1x1_strided_scratch(int C, int B, int H, int Wd, int stride);
+int ubp_conv1x1_strided(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
+                        int64_t in_stride_b, int64_t in_stride_c, void *scratch, size_t scratch_bytes,
+                        const float *bias, int relu, float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);
+
 /* ubp_spmm_static: same result as ubp_spmm, for callers that cannot allocate.
  * (The paper has no counterpart; this is a deployment convenience.)
  *

@@ -68,6 +68,10 @@ def load():
     L.ubp_selftest_bounded_wait.argtypes = [vp, C.c_uint, vp]
     L.ubp_static_plan_capacity.restype = sz
     L.ubp_spmm_static.argtypes = [vp, sz, vp, i64, i64, vp, i32, vp, i64, vp]
+    L.ubp_conv3x3_strided.argtypes = [vp, vp, i32, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
+    L.ubp_conv1x1_strided_scratch.restype = sz
+    L.ubp_conv1x1_strided_scratch.argtypes = [i32, i32, i32, i32, i32]
+    L.ubp_conv1x1_strided.argtypes = [vp, vp, i32, i32, i32, i32, i64, i64, vp, sz, vp, i32, vp, i64, i64, vp]
     L.ubp_bed_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
     L.ubp_block_scores.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, vp]
     L.ubp_bed_select.argtypes = [vp, i32, i32, i32, i32, i64, vp, sz, vp, vp, vp]
@@ -267,42 +271,66 @@ def ubp_spmm(plan: Plan, X, bias=None, relu: bool = False, out=None, stream=None
     return out
 
 
-def _conv_args(plan, x, out, layout):
+def _conv_args(plan, x, out, layout, stride=1):
     import torch
+    if stride < 1:
+        raise ValueError("stride must be >= 1")
     if layout == "CNHW":
         Cin, B, H, Wd = x.shape
         sb, sc = x.stride(1), x.stride(0)
-        oshape = (plan.M, B, H, Wd)
+        oshape = (plan.M, B, (H - 1) // stride + 1, (Wd - 1) // stride + 1)
     elif layout == "NCHW":
         B, Cin, H, Wd = x.shape
         sb, sc = x.stride(0), x.stride(1)
-        oshape = (B, plan.M, H, Wd)
+        oshape = (B, plan.M, (H - 1) // stride + 1, (Wd - 1) // stride + 1)
     else:
         raise ValueError("layout must be 'CNHW' or 'NCHW'")
     if Cin != plan.C or x.stride(3) != 1 or x.stride(2) != Wd:
         raise ValueError("input planes must be contiguous [H][W] and have plan.C channels")
     if out is None:
         out = torch.empty(oshape, dtype=torch.float32, device=x.device)
-    if tuple(out.shape) != oshape or out.stride(3) != 1 or out.stride(2) != Wd:
+    if tuple(out.shape) != oshape or out.stride(3) != 1 or out.stride(2) != oshape[3]:
         raise ValueError("bad output tensor")
     osb, osc = (out.stride(1), out.stride(0)) if layout == "CNHW" else (out.stride(0), out.stride(1))
     return B, H, Wd, sb, sc, out, osb, osc
 
 
-def ubp_conv1x1(plan: Plan, x, bias=None, relu: bool = False, out=None, layout: str = "CNHW", stream=None):
-    """1x1 stride-1 convolution. layout 'CNHW': x [C][B][H][W] -> out [M][B][H][W]; 'NCHW': x [B][C][H][W]."""
+def ubp_conv1x1(plan: Plan, x, bias=None, relu: bool = False, out=None, layout: str = "CNHW", stream=None,
+                stride: int = 1, scratch=None):
+    """1x1 convolution. layout 'CNHW': x [C][B][H][W] -> out [M][B][Ho][Wo]; 'NCHW': x [B][C][H][W]. With stride > 1
+    the pixels read are gathered into `scratch` first (a float32 CUDA tensor of at least C*B*Ho*Wo elements; allocated
+    here when not given)."""
     import torch
-    B, H, Wd, sb, sc, out, osb, osc = _conv_args(plan, x, out, layout)
+    B, H, Wd, sb, sc, out, osb, osc = _conv_args(plan, x, out, layout, stride)
+    if stride != 1:
+        need = plan._lib.ubp_conv1x1_strided_scratch(plan.C, B, H, Wd, stride)
+        if scratch is None:
+            scratch = torch.empty(need // 4, dtype=torch.float32, device=x.device)
+        with torch.cuda.device(x.device):
+            _chk(plan._lib.ubp_conv1x1_strided(plan.handle, _dev_ptr(x, "x"), B, H, Wd, stride, sb, sc,
+                                               _dev_ptr(scratch, "scratch"), scratch.numel() * 4,
+                                               _dev_ptr(bias, "bias", True), int(bool(relu)), _dev_ptr(out, "out"),
+                                               osb, osc, _stream_ptr(stream)), "ubp_conv1x1_strided")
+            scratch.record_stream(torch.cuda.current_stream() if stream is None else stream)
+        return out
     with torch.cuda.device(x.device):
         _chk(plan._lib.ubp_conv1x1(plan.handle, _dev_ptr(x, "x"), B, H, Wd, sb, sc, _dev_ptr(bias, "bias", True),
                                    int(bool(relu)), _dev_ptr(out, "out"), osb, osc, _stream_ptr(stream)), "ubp_conv1x1")
     return out
 
 
-def ubp_conv3x3_implicit(plan: Plan, x, bias=None, relu: bool = False, out=None, layout: str = "CNHW", stream=None):
-    """3x3 / stride 1 / pad 1 convolution on a plan built from an R = 9 blob."""
+def ubp_conv3x3_implicit(plan: Plan, x, bias=None, relu: bool = False, out=None, layout: str = "CNHW", stream=None,
+                         stride: int = 1):
+    """3x3 / pad 1 convolution on a plan built from an R = 9 blob (stride 1: the implicit-GEMM kernels; stride > 1:
+    one lane per output pixel)."""
     import torch
-    B, H, Wd, sb, sc, out, osb, osc = _conv_args(plan, x, out, layout)
+    B, H, Wd, sb, sc, out, osb, osc = _conv_args(plan, x, out, layout, stride)
+    if stride != 1:
+        with torch.cuda.device(x.device):
+            _chk(plan._lib.ubp_conv3x3_strided(plan.handle, _dev_ptr(x, "x"), B, H, Wd, stride, sb, sc,
+                                               _dev_ptr(bias, "bias", True), int(bool(relu)), _dev_ptr(out, "out"),
+                                               osb, osc, _stream_ptr(stream)), "ubp_conv3x3_strided")
+        return out
     with torch.cuda.device(x.device):
         _chk(plan._lib.ubp_conv3x3_implicit(plan.handle, _dev_ptr(x, "x"), B, H, Wd, sb, sc,
                                             _dev_ptr(bias, "bias", True), int(bool(relu)), _dev_ptr(out, "out"),

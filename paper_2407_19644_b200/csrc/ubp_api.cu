@@ -230,4 +230,51 @@ int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, 
                                out_stride_c, stream);
 }
 
+int ubp_conv3x3_strided(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
+                        int64_t in_stride_b, int64_t in_stride_c, const float *bias, int relu,
+                        float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream)
+{
+    if (stride == 1)
+        return ubp_conv3x3_implicit(plan, in, B, H, Wd, in_stride_b, in_stride_c, bias, relu, out, out_stride_b,
+                                    out_stride_c, stream);
+    if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
+    if (plan->dims.R != 9 || (plan->cfg.kind != 1 && plan->cfg.kind != 3)) return UBP_E_ARG;
+    if (stride < 1 || B < 0 || H <= 0 || Wd <= 0) return UBP_E_ARG;
+    if (B == 0) return UBP_OK;
+    if (!in || !out) return UBP_E_ARG;
+    const int64_t hw = (int64_t)H * Wd;
+    const int64_t ohw = (int64_t)((H - 1) / stride + 1) * ((Wd - 1) / stride + 1);
+    if (in_stride_c < hw || out_stride_c < ohw || in_stride_b < 0 || out_stride_b < 0) return UBP_E_ARG;
+    return ubp::launch_conv3x3(plan, in, B, H, Wd, in_stride_b, in_stride_c, bias, relu, out, out_stride_b,
+                               out_stride_c, stream, stride);
+}
+
+size_t ubp_conv1x1_strided_scratch(int C, int B, int H, int Wd, int stride)
+{
+    if (C <= 0 || B <= 0 || H <= 0 || Wd <= 0 || stride <= 1) return 0;
+    return (size_t)C * B * ((H - 1) / stride + 1) * ((Wd - 1) / stride + 1) * sizeof(float);
+}
+
+int ubp_conv1x1_strided(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
+                        int64_t in_stride_b, int64_t in_stride_c, void *scratch, size_t scratch_bytes,
+                        const float *bias, int relu, float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream)
+{
+    if (stride == 1)
+        return ubp_conv1x1(plan, in, B, H, Wd, in_stride_b, in_stride_c, bias, relu, out, out_stride_b, out_stride_c, stream);
+    if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
+    if (plan->dims.R != 1 || plan->cfg.kind == 1 || plan->cfg.kind == 3) return UBP_E_ARG;
+    if (stride < 1 || B < 0 || H <= 0 || Wd <= 0) return UBP_E_ARG;
+    if (B == 0) return UBP_OK;
+    if (!in || !out || !scratch || ((uintptr_t)scratch & 15u) != 0) return UBP_E_ARG;
+    const int64_t hw = (int64_t)H * Wd;
+    if (in_stride_c < hw || in_stride_b < 0) return UBP_E_ARG;
+    const int C = plan->dims.C;
+    if (scratch_bytes < ubp_conv1x1_strided_scratch(C, B, H, Wd, stride)) return UBP_E_SPACE;
+    const int Ho = (H - 1) / stride + 1, Wo = (Wd - 1) / stride + 1;
+    float *xs = static_cast<float *>(scratch);
+    if (int rc = ubp::launch_subsample(in, C, B, H, Wd, in_stride_b, in_stride_c, stride, xs, stream)) return rc;
+    return ubp_conv1x1(plan, xs, B, Ho, Wo, (int64_t)Ho * Wo, (int64_t)B * Ho * Wo, bias, relu, out, out_stride_b,
+                       out_stride_c, stream);
+}
+
 }  // extern "C"

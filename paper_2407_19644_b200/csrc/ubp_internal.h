@@ -89,8 +89,11 @@ int launch_spmm_tc(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc
                    float *Y, int64_t ldy, void *stream);
 int launch_conv3x3_tc(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
                       const float *bias, int relu, float *out, int64_t out_ld, void *stream);
+// stride 1: tensor-core implicit GEMM when the plan and the layouts allow it; stride > 1: one lane per output pixel
 int launch_conv3x3(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
-                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream);
+                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream, int stride = 1);
+int launch_subsample(const float *in, int C, int B, int H, int Wd, int64_t isb, int64_t isc, int stride, float *out,
+                     void *stream);
 void set_last_cuda_error(int e);
 }
 

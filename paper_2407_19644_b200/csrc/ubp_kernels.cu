@@ -474,18 +474,19 @@ template <int NBK, int P>
 __global__ void __launch_bounds__(128)
 ubp_conv3x3_simple_kernel(const uint8_t *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
                           const float *bias, int relu, float *out, int64_t osb, int64_t osc,
-                          int M, int NP, int nkt, int NG, int WR, int KT)
+                          int M, int NP, int nkt, int NG, int WR, int KT, int stride)
 {
     constexpr int F = P + NBK - 1;
     constexpr int FO_BYTES = ((F + 1) * 2 + 15) & ~15;
     const int panel = blockIdx.y;
     const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t total = (int64_t)B * H * Wd;
+    const int Ho = (H - 1) / stride + 1, Wo = (Wd - 1) / stride + 1;   // pad 1, 3x3: output pixel (yo, xo) is centred
+    const int64_t total = (int64_t)B * Ho * Wo;                         // on input pixel (yo * stride, xo * stride)
     const bool live = n < total;
     const int64_t nn = live ? n : 0;
-    const int b = (int)(nn / (H * Wd));
-    const int pix = (int)(nn % (H * Wd));
-    const int y = pix / Wd, x = pix % Wd;
+    const int b = (int)(nn / (Ho * Wo));
+    const int pix = (int)(nn % (Ho * Wo));
+    const int y = (pix / Wo) * stride, x = (pix % Wo) * stride;
     const int g = panel / WR, wr = panel % WR;
     const uint32_t *gtab = reinterpret_cast<const uint32_t *>(plan + 256);
     const float *inb = in + (size_t)b * isb;
@@ -622,14 +623,14 @@ struct CfgLaunch {
         else return UBP_E_UNSUPPORTED;
     }
     static int conv_kernel(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
-                           const float *bias, int relu, float *out, int64_t osb, int64_t osc, cudaStream_t s)
+                           const float *bias, int relu, float *out, int64_t osb, int64_t osc, cudaStream_t s, int stride)
     {
         if constexpr (KIND == 1 || KIND == 3) {
-            const int64_t total = (int64_t)B * H * Wd;
+            const int64_t total = (int64_t)B * ((H - 1) / stride + 1) * ((Wd - 1) / stride + 1);
             dim3 grid((unsigned)((total + 127) / 128), (unsigned)pl->img.NP);
             ubp_conv3x3_simple_kernel<NBK, P><<<grid, 128, 0, s>>>(
                 static_cast<const uint8_t *>(pl->dev), in, B, H, Wd, isb, isc, bias, relu, out, osb, osc, pl->dims.M,
-                pl->img.NP, pl->img.nkt, pl->img.NG, pl->cfg.WR, pl->cfg.KT);
+                pl->img.NP, pl->img.nkt, pl->img.NG, pl->cfg.WR, pl->cfg.KT, stride);
             return check(cudaGetLastError());
         } else {
             return UBP_E_UNSUPPORTED;
@@ -663,21 +664,51 @@ int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, con
 }
 
 int launch_conv3x3(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
-                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream_)
+                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream_, int stride)
 {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const KernelCfg &c = pl->cfg;
     const int64_t total = (int64_t)B * H * Wd;
     // tensor-core path: needs the output as one [M][B*H*W] matrix (batch stride = plane size) with 16-byte rows
-    if (c.kind == 3 && osb == (int64_t)H * Wd && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && osc % 4 == 0 &&
+    if (stride == 1 && c.kind == 3 && osb == (int64_t)H * Wd && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && osc % 4 == 0 &&
         osc >= total && total < (1ll << 31))
         return launch_conv3x3_tc(pl, in, B, H, Wd, isb, isc, bias, relu, out, osc, stream_);
 #define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP) \
     if (c.id == ID)                                        \
-        return CfgLaunch<KIND, NBK, P_, V_, WR_, WC_, KT_, (DUP != 0)>::conv_kernel(pl, in, B, H, Wd, isb, isc, bias, relu, out, osb, osc, stream);
+        return CfgLaunch<KIND, NBK, P_, V_, WR_, WC_, KT_, (DUP != 0)>::conv_kernel(pl, in, B, H, Wd, isb, isc, bias, relu, out, osb, osc, stream, stride);
 #include "ubp_cfgs.inc"
 #undef UBP_CFG
     return UBP_E_UNSUPPORTED;
+}
+
+// Every stride-th pixel of every stride-th row of each input plane, into a dense channel-major tensor
+// [C][B][Ho][Wo]: the activations a strided 1x1 convolution reads.
+__global__ void __launch_bounds__(256) ubp_subsample_kernel(const float *__restrict__ in, int C, int B, int H, int Wd,
+                                                             int64_t isb, int64_t isc, int stride, int Ho, int Wo,
+                                                             float *__restrict__ out)
+{
+    const int64_t total = (int64_t)C * B * Ho * Wo;
+    for (int64_t n = (int64_t)blockIdx.x * 256 + threadIdx.x; n < total; n += (int64_t)gridDim.x * 256) {
+        const int xo = (int)(n % Wo);
+        const int64_t r1 = n / Wo;
+        const int yo = (int)(r1 % Ho);
+        const int64_t r2 = r1 / Ho;
+        const int b = (int)(r2 % B), c = (int)(r2 / B);
+        out[n] = in[(size_t)b * isb + (size_t)c * isc + (size_t)(yo * stride) * Wd + (size_t)xo * stride];
+    }
+}
+
+int launch_subsample(const float *in, int C, int B, int H, int Wd, int64_t isb, int64_t isc, int stride, float *out,
+                     void *stream_)
+{
+    const int Ho = (H - 1) / stride + 1, Wo = (Wd - 1) / stride + 1;
+    const int64_t total = (int64_t)C * B * Ho * Wo;
+    if (total == 0) return UBP_OK;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    ubp_subsample_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream_)>>>(in, C, B, H, Wd, isb, isc,
+                                                                                              stride, Ho, Wo, out);
+    return check(cudaGetLastError());
 }
 
 }  // namespace ubp

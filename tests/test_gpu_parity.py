@@ -506,3 +506,36 @@ def test_bottleneck_trio_chained_through_fused_epilogues(env):
     torch.cuda.synchronize()
     for y, e in zip(outs, eager):
         assert np.array_equal(y.cpu().numpy(), e)
+
+
+@pytest.mark.parametrize("layout", ["CNHW", "NCHW"])
+@pytest.mark.parametrize("H,Wd", [(14, 14), (7, 9)])
+def test_stride_two_convolutions(env, layout, H, Wd):
+    """Downsampling layers: 1x1 stride 2 reads every other pixel of every other row; 3x3 stride 2 / pad 1 is the
+    stride-1 result at those pixels. Both against the oracle's stride-1 definitions, subsampled."""
+    torch, ubp = env
+    B = 3
+    L1 = ubp_synth.make_layer("s2_pw", 96, 64, 4, 70, 801, B=B, H=H, Wd=Wd)
+    L3 = ubp_synth.make_layer("s2_3x3", 64, 32, 8, 75, 802, B=B, H=H, Wd=Wd, R=9)
+    for L in (L1, L3):
+        plan = ubp.Plan(ubp.pack_ubp(L.W, L.mask, L.Nb))
+        x = torch.from_numpy(L.X).cuda()                       # [C][B][H][W]
+        if layout == "NCHW":
+            x = x.permute(1, 0, 2, 3).contiguous()
+        bias = torch.from_numpy(L.bias).cuda()
+        fn = ubp.ubp_conv3x3_implicit if L.R == 9 else ubp.ubp_conv1x1
+        y = fn(plan, x, bias, True, layout=layout, stride=2)
+        torch.cuda.synchronize()
+        plan.check()
+        y = y.cpu().numpy()
+        if layout == "NCHW":
+            y = y.transpose(1, 0, 2, 3)
+        if L.R == 9:
+            Yref, A = oracle.masked_conv3x3(L.W, L.mask, L.X, L.bias, relu=True)
+            Yref, A = Yref[:, :, ::2, ::2], A[:, :, ::2, ::2]
+        else:
+            xs = np.ascontiguousarray(L.X[:, :, ::2, ::2])
+            Yref, A = oracle.masked_matmul(L.W, L.mask, xs.reshape(L.C, -1), L.bias, relu=True)
+            Yref, A = Yref.reshape(L.M, B, *xs.shape[2:]), A.reshape(L.M, B, *xs.shape[2:])
+        assert y.shape == Yref.shape
+        assert scaled_error(y, Yref, A) <= 1e-4
