@@ -60,7 +60,16 @@ BED_WORKLOADS = {
 }
 
 
+KMAJOR_B = 4     # kmajor_pw512: the headline layer's shape with blocks of 4 consecutive INPUT channels in one output row
+
+
 def get_layer(name: str, seed_index: int = 0):
+    if name == "kmajor_pw512":
+        # generated as the transposed layer (blocks run down the rows of [C][M]) and turned round; to the kernels it is
+        # a layer of M*C*(1-p) single-channel blocks
+        t = ubp_synth.make_layer(name, 512, 512, KMAJOR_B, 70, 7000 + seed_index, B=32, H=14, Wd=14, w_scale=0.05)
+        return ubp_synth.Layer(name, t.C, t.M, 1, 1, 70, t.m * KMAJOR_B, np.ascontiguousarray(t.W.transpose(1, 0, 2)),
+                               np.ascontiguousarray(t.mask.T), t.X, t.bias, True, t.B, t.H, t.Wd)
     w = WORKLOADS[name]
     layers = ubp_synth.config_layers(w["cfg"], index=seed_index, **w["kw"])
     return layers[w.get("index", 0)]
@@ -155,7 +164,10 @@ class ClockSampler:
 def build_runner(ubp, torch, L, variant):
     """Returns (plan, run(stream-less call), pack_ms, plan_ms, device tensors)."""
     t0 = time.perf_counter()
-    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    if L.name == "kmajor_pw512":
+        blob = ubp.ubp_kmajor_to_plan_blob(ubp.ubp_pack_kmajor(L.W[:, :, 0], L.mask, KMAJOR_B))
+    else:
+        blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
     t1 = time.perf_counter()
     plan = ubp.Plan(blob, variant)
     torch.cuda.synchronize()

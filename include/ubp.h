@@ -80,6 +80,21 @@ typedef struct {
 /* ubp_blob_view (host): validate a blob and expose its arrays (no copy). */
 int ubp_blob_view(const void *blob, size_t len, ubp_view_t *view);
 
+/* The other block orientation: B consecutive INPUT channels of ONE output row (runs along K inside a row of W),
+ * starting at any input channel <= C-B. It is the same format with the two channel roles exchanged, and R = 1.
+ * ubp_pack_kmajor (host): W[M][C], mask[M][C] whose runs of ones along each row are whole multiples of B
+ *   -> the canonical blob of the transposed layer (its header reads M' = C, C' = M, Nb = B; indptr runs over the
+ *   input channel a block starts at, indices hold the output row). Same size-query and error rules as ubp_pack
+ *   (UBP_E_RAGGED for a run that is not a whole number of blocks).
+ * ubp_kmajor_to_plan_blob (host): that blob -> a blob ubp_plan_size / ubp_plan_build accept: the same kept weights
+ *   in the layer's own orientation as blocks of ONE output channel (any mask is a valid set of such blocks). The
+ *   tensor-core kernels work on the densified weight and do not care about the orientation; below their density
+ *   threshold the layer runs on the sparse kernel's element-wise configuration, one index per kept weight (a
+ *   kernel that walks K-runs with one index per B weights is not built). */
+int ubp_pack_kmajor(const float *W, const uint8_t *mask, int M, int C, int B,
+                    void *blob, size_t blob_cap, size_t *blob_len);
+int ubp_kmajor_to_plan_blob(const void *kblob, size_t klen, void *blob, size_t blob_cap, size_t *blob_len);
+
 /* ------------------------------------------------------------------ plan
  * The kernels do not walk the canonical arrays directly: a plan is the same
  * blocks re-bucketed for the GPU (by row panel, input-channel tile and start

@@ -8,8 +8,10 @@ is missing or a call fails, an exception is raised.
 """
 from .binding import (UbpError, Plan, pack_ubp, unpack_ubp, blob_view, plan_size, plan_image, variants,
                       ubp_pack, ubp_unpack, ubp_spmm, ubp_conv1x1, ubp_conv3x3_implicit, ubp_spmm_static,
-                      static_plan_capacity, lib_path, load, BedSelector, ubp_block_scores, ubp_bed_select)
+                      static_plan_capacity, lib_path, load, BedSelector, ubp_block_scores, ubp_bed_select,
+                      ubp_pack_kmajor, ubp_kmajor_to_plan_blob)
 
 __all__ = ["UbpError", "Plan", "pack_ubp", "unpack_ubp", "blob_view", "plan_size", "plan_image", "variants",
            "ubp_pack", "ubp_unpack", "ubp_spmm", "ubp_conv1x1", "ubp_conv3x3_implicit", "ubp_spmm_static",
-           "static_plan_capacity", "lib_path", "load", "BedSelector", "ubp_block_scores", "ubp_bed_select"]
+           "static_plan_capacity", "lib_path", "load", "BedSelector", "ubp_block_scores", "ubp_bed_select",
+           "ubp_pack_kmajor", "ubp_kmajor_to_plan_blob"]

@@ -72,6 +72,8 @@ def load():
     L.ubp_conv1x1_strided_scratch.restype = sz
     L.ubp_conv1x1_strided_scratch.argtypes = [i32, i32, i32, i32, i32]
     L.ubp_conv1x1_strided.argtypes = [vp, vp, i32, i32, i32, i32, i64, i64, vp, sz, vp, i32, vp, i64, i64, vp]
+    L.ubp_pack_kmajor.argtypes = [vp, vp, i32, i32, i32, vp, sz, C.POINTER(sz)]
+    L.ubp_kmajor_to_plan_blob.argtypes = [vp, sz, vp, sz, C.POINTER(sz)]
     L.ubp_bed_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
     L.ubp_block_scores.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, vp]
     L.ubp_bed_select.argtypes = [vp, i32, i32, i32, i32, i64, vp, sz, vp, vp, vp]
@@ -137,6 +139,31 @@ def ubp_unpack(blob: bytes) -> Tuple[np.ndarray, np.ndarray]:
 
 pack_ubp = ubp_pack
 unpack_ubp = ubp_unpack
+
+
+def ubp_pack_kmajor(W: np.ndarray, mask: np.ndarray, B: int) -> bytes:
+    """Blocks of B consecutive input channels inside one output row: mask [M][C] + W [M][C] -> the canonical blob of
+    the transposed layer."""
+    L = load()
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    M, Cin = mask.shape
+    W = np.ascontiguousarray(W, dtype=np.float32).reshape(M, Cin)
+    n = C.c_size_t(0)
+    _chk(L.ubp_pack_kmajor(_np_ptr(W), _np_ptr(mask), M, Cin, B, None, 0, C.byref(n)), "ubp_pack_kmajor")
+    buf = np.empty(n.value, np.uint8)
+    _chk(L.ubp_pack_kmajor(_np_ptr(W), _np_ptr(mask), M, Cin, B, _np_ptr(buf), n.value, C.byref(n)), "ubp_pack_kmajor")
+    return buf.tobytes()
+
+
+def ubp_kmajor_to_plan_blob(kblob: bytes) -> bytes:
+    """Blob of ubp_pack_kmajor -> a blob Plan() accepts (the layer's own orientation, blocks of one output channel)."""
+    L = load()
+    b = np.frombuffer(kblob, np.uint8)
+    n = C.c_size_t(0)
+    _chk(L.ubp_kmajor_to_plan_blob(_np_ptr(b), b.size, None, 0, C.byref(n)), "ubp_kmajor_to_plan_blob")
+    buf = np.empty(n.value, np.uint8)
+    _chk(L.ubp_kmajor_to_plan_blob(_np_ptr(b), b.size, _np_ptr(buf), n.value, C.byref(n)), "ubp_kmajor_to_plan_blob")
+    return buf.tobytes()
 
 
 def variants():

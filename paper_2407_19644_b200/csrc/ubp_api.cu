@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "ubp_internal.h"
 
@@ -50,6 +51,44 @@ int ubp_unpack(const void *blob, size_t len, float *W_out, uint8_t *mask_out)
 }
 
 int ubp_blob_view(const void *blob, size_t len, ubp_view_t *view) { return ubp::blob_view(blob, len, view); }
+
+int ubp_pack_kmajor(const float *W, const uint8_t *mask, int M, int C, int B,
+                    void *blob, size_t blob_cap, size_t *blob_len)
+{
+    if (!W || !mask || !blob_len || M < 1 || C < 1 || B < 1 || B > C) return UBP_E_ARG;
+    try {
+        // the same layer seen from the other side: rows <-> columns, so runs along the input channels of one output
+        // row become runs along the rows of one column, which is what the packer cuts into blocks
+        std::vector<float> Wt((size_t)M * C);
+        std::vector<uint8_t> mt((size_t)M * C);
+        for (int i = 0; i < M; ++i)
+            for (int j = 0; j < C; ++j) {
+                Wt[(size_t)j * M + i] = W[(size_t)i * C + j];
+                mt[(size_t)j * M + i] = mask[(size_t)i * C + j];
+            }
+        return ubp::pack(Wt.data(), mt.data(), C, M, 1, B, blob, blob_cap, blob_len);
+    } catch (const std::bad_alloc &) { return UBP_E_SPACE; }
+}
+
+int ubp_kmajor_to_plan_blob(const void *kblob, size_t klen, void *blob, size_t blob_cap, size_t *blob_len)
+{
+    if (!kblob || !blob_len) return UBP_E_ARG;
+    ubp_view_t v;
+    if (int rc = ubp::blob_view(kblob, klen, &v)) return rc;
+    if (v.R != 1) return UBP_E_UNSUPPORTED;
+    try {
+        const int M = v.C, C = v.M;            // the layer's own output / input channel counts
+        std::vector<float> Wt((size_t)M * C), W((size_t)M * C);
+        std::vector<uint8_t> mt((size_t)M * C), mask((size_t)M * C);
+        if (int rc = ubp::unpack(kblob, klen, Wt.data(), mt.data())) return rc;
+        for (int j = 0; j < C; ++j)
+            for (int i = 0; i < M; ++i) {
+                W[(size_t)i * C + j] = Wt[(size_t)j * M + i];
+                mask[(size_t)i * C + j] = mt[(size_t)j * M + i];
+            }
+        return ubp::pack(W.data(), mask.data(), M, C, 1, 1, blob, blob_cap, blob_len);
+    } catch (const std::bad_alloc &) { return UBP_E_SPACE; }
+}
 
 int ubp_variant_count(void) { return (int)ubp::kernel_cfgs().size(); }
 

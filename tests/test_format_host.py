@@ -228,3 +228,28 @@ def test_bf16_three_term_product_error_bound():
         approx = x1.astype(np.float64) * w1 + x1.astype(np.float64) * w2 + x2.astype(np.float64) * w1
         exact = x.astype(np.float64) * w
         assert np.all(np.abs(approx - exact) <= np.abs(exact) * 3 * 2.0 ** -16)
+
+
+def test_kmajor_blocks_pack_as_the_transposed_layer_and_convert_to_a_plan_blob():
+    """Blocks of B consecutive input channels inside one output row (the other orientation): the blob is the oracle's
+    blob of the transposed layer, bit for bit; a run that is not a whole number of blocks is refused; the conversion
+    for the plan builder keeps exactly the same weights as blocks of one output channel."""
+    import paper_2407_19644_b200 as ubp
+    M, Cin, B = 24, 40, 4
+    Lt = ubp_synth.make_layer("kmajor", Cin, M, B, 70, 4242, Nc=8, make_x=False)      # transposed roles: [C][M]
+    W = np.ascontiguousarray(Lt.W[:, :, 0].T)                                         # [M][C]
+    mask = np.ascontiguousarray(Lt.mask.T)
+    kblob = ubp.ubp_pack_kmajor(W, mask, B)
+    assert kblob == oracle.pack(np.ascontiguousarray(W.T), np.ascontiguousarray(mask.T), B)
+    v = ubp.blob_view(kblob)
+    assert (v["M"], v["C"], v["Nb"], v["m"]) == (Cin, M, B, Lt.m)
+    pblob = ubp.ubp_kmajor_to_plan_blob(kblob)
+    assert pblob == oracle.pack(W, mask, 1)
+    W2, m2 = ubp.unpack_ubp(pblob)
+    assert np.array_equal(m2, mask) and np.array_equal(W2[:, :, 0].view(np.uint32), np.where(mask == 1, W, np.float32(0)).view(np.uint32))
+    bad = mask.copy()
+    i, j = np.argwhere(bad == 1)[0]
+    bad[i, j] = 0                                      # shortens one run by one element
+    with pytest.raises(ubp.UbpError) as e:
+        ubp.ubp_pack_kmajor(W, bad, B)
+    assert e.value.code == -2

@@ -539,3 +539,23 @@ def test_stride_two_convolutions(env, layout, H, Wd):
             Yref, A = Yref.reshape(L.M, B, *xs.shape[2:]), A.reshape(L.M, B, *xs.shape[2:])
         assert y.shape == Yref.shape
         assert scaled_error(y, Yref, A) <= 1e-4
+
+
+@pytest.mark.parametrize("M,Cin,B,p,Nc", [(256, 256, 4, 70, 1000), (192, 320, 8, 95, 520), (64, 96, 2, 50, 260)])
+def test_kmajor_orientation_through_the_plan(env, M, Cin, B, p, Nc):
+    """Blocks that run along the input channels of one output row: packed as the transposed layer, converted for
+    the plan builder, run through ubp_spmm (tensor-core kernel at 70 %, sparse element-wise kernel at 95 %)."""
+    torch, ubp = env
+    Lt = ubp_synth.make_layer("kmajor", Cin, M, B, p, 900 + B, Nc=8, make_x=False)    # roles exchanged: [C][M]
+    W = np.ascontiguousarray(Lt.W[:, :, 0].T)
+    mask = np.ascontiguousarray(Lt.mask.T)
+    rng = np.random.default_rng(5)
+    X = rng.standard_normal((Cin, Nc)).astype(np.float32)
+    bias = rng.standard_normal(M).astype(np.float32)
+    plan = ubp.Plan(ubp.ubp_kmajor_to_plan_blob(ubp.ubp_pack_kmajor(W, mask, B)))
+    assert plan.m == Lt.m * B and plan.Nb == 1
+    Y = ubp.ubp_spmm(plan, torch.from_numpy(X).cuda(), torch.from_numpy(bias).cuda(), True)
+    torch.cuda.synchronize()
+    plan.check()
+    Yref, A = oracle.masked_matmul(W, mask, X, bias, relu=True)
+    assert scaled_error(Y.cpu().numpy(), Yref, A) <= 1e-4
