@@ -262,7 +262,11 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         constexpr int GT = (T3_XL_WARPS / T3_XL_GROUPS) * 32;
         const int grp = (warp - 2) / (T3_XL_WARPS / T3_XL_GROUPS);
         const int gt = (int)threadIdx.x - 64 - grp * GT;
-        const int cg = gt & 15, kq = gt >> 4;
+        // Up to 64 columns per CTA: 8 column groups x 16 channels, one channel per thread; wider: 16 column groups x 8
+        // channel pairs, two channels per thread.
+        const bool narrow = NH <= 64;
+        const int cg = narrow ? (gt & 7) : (gt & 15), kq = narrow ? (gt >> 3) : (gt >> 4);
+        const int nk = narrow ? 1 : 2;
         const bool mine = cg * 8 < NH;
         const int total = nmy * nstage;
         const uint32_t dst = (uint32_t)(cg >> 3) * T3_ATOM;   // 64-column atom; inside it row k is 128 bytes whose
@@ -315,6 +319,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                     const int o = 8 * cg + sh, ob = o & ~3, r = o & 3;      // r is the same for every lane
 #pragma unroll
                     for (int i = 0; i < 2; ++i) {
+                        if (i >= nk) break;
                         const int k = kq + 8 * i;
                         const float4 q0 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4);
                         const float4 q1 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 16);
