@@ -57,3 +57,27 @@ def test_single_process_helpers():
     assert (L.M, L.C, L.Nc, L.m) == (512, 512, 6272, 19660)
     assert bench.compulsory_bytes(L) == 512 * 6272 * 4 * 2 + 19660 * 4 * 4 + 19660 * 4 + 513 * 4 + 512 * 4
     assert abs(bench.FP32_PEAK_TFLOPS - 74.44992) < 1e-6
+
+
+def test_added_workloads_are_well_formed():
+    sys.path.insert(0, ROOT)
+    import bench
+    import ubp_synth
+    # the other block orientation: every row's runs of ones are whole blocks of KMAJOR_B input channels
+    L = bench.get_layer("kmajor_pw512")
+    assert (L.M, L.C, L.Nb, L.Nc) == (512, 512, 1, 6272) and L.m == int(L.mask.sum())
+    assert L.m == ubp_synth.block_budget(512, 512, 70, bench.KMAJOR_B) * bench.KMAJOR_B
+    padded = np.pad(L.mask, ((0, 0), (1, 1))).astype(np.int8)
+    d = np.diff(padded, axis=1)
+    starts, ends = np.argwhere(d == 1), np.argwhere(d == -1)
+    assert ((ends[:, 1] - starts[:, 1]) % bench.KMAJOR_B == 0).all()
+    # the chained bottleneck: shapes agree along the chain and only the first layer carries activations
+    layers = ubp_synth.config_layers("r50_bottleneck", batch=2)
+    assert [(l.M, l.C, l.R) for l in layers] == [(256, 1024, 1), (256, 256, 9), (1024, 256, 1)]
+    assert layers[0].X.size and not layers[1].X.size and layers[1].Nc == layers[0].Nc == 2 * 14 * 14
+    assert all(a.M == b.C for a, b in zip(layers, layers[1:]))
+    # block-selection workloads: the oracle timing extrapolates from a bounded number of rounds
+    t, cores, sample = bench.cpu_bed_time(ubp_synth.selection_weights(64, 32, 1, 1), 4, 100, budget_s=0.05)
+    assert t > 0 and cores == 1 and ("iterations" in sample or "whole" in sample)
+    for name, (M, C, R, Nb, p) in bench.BED_WORKLOADS.items():
+        assert name.startswith("bed_") and M % Nb == 0 and 0 < p < 100
