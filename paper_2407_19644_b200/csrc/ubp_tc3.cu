@@ -286,17 +286,25 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             if (CONV && ti != mask_tile) {                 // new tile: which taps of my eight columns are inside the image
                 mask_tile = ti;
                 const int64_t n0 = tile_col0(ti) + (int64_t)rank * NH + 8 * cg;
-                const int hw = a.H * a.W;
+                const uint32_t hw = (uint32_t)(a.H * a.W);
                 tap_lo = 0; tap_hi = 0;
-                for (int e = 0; e < 8; ++e) {
-                    const int64_t n = n0 + e;
-                    if (!mine || n >= a.Nc) continue;
-                    const int pix = (int)(n % hw), y = pix / a.W, x = pix - y * a.W;
-                    for (int t9 = 0; t9 < 9; ++t9) {
-                        const int yy = y + t9 / 3 - 1, xx = x + t9 % 3 - 1;
-                        if (yy >= 0 && yy < a.H && xx >= 0 && xx < a.W) {
-                            if (t9 < 8) tap_lo |= 1ull << (t9 * 8 + e); else tap_hi |= 1u << e;
+                if (mine && n0 < a.Nc) {
+                    // pixel of the first column by two 32-bit divisions (column numbers are below 2^31), the other
+                    // seven by stepping; a tap is inside the image when its row and its column are
+                    uint32_t pix = (uint32_t)n0 % hw;
+                    int y = (int)(pix / (uint32_t)a.W), x = (int)(pix - (uint32_t)y * (uint32_t)a.W);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        if (n0 + e < a.Nc) {
+                            const uint32_t rows = (y > 0 ? 1u : 0u) | 2u | (y < a.H - 1 ? 4u : 0u);
+                            const uint32_t cols = (x > 0 ? 1u : 0u) | 2u | (x < a.W - 1 ? 4u : 0u);
+#pragma unroll
+                            for (int t9 = 0; t9 < 9; ++t9)
+                                if (((rows >> (t9 / 3)) & (cols >> (t9 % 3)) & 1u) != 0u) {
+                                    if (t9 < 8) tap_lo |= 1ull << (t9 * 8 + e); else tap_hi |= 1u << e;
+                                }
                         }
+                        if (++x == a.W) { x = 0; if (++y == a.H) y = 0; }
                     }
                 }
             }
