@@ -253,3 +253,23 @@ def test_kmajor_blocks_pack_as_the_transposed_layer_and_convert_to_a_plan_blob()
     with pytest.raises(ubp.UbpError) as e:
         ubp.ubp_pack_kmajor(W, bad, B)
     assert e.value.code == -2
+
+
+def test_block_selection_argument_checks_need_no_device():
+    """Size query and limits of the block-selection entry points (no kernel runs): bad sizes are refused, layers
+    beyond the supported row count are reported as unsupported, the scratch grows with the layer."""
+    import ctypes as C
+    import paper_2407_19644_b200 as ubp
+    L = ubp.load()
+    n = C.c_size_t(0)
+    assert L.ubp_bed_workspace_size(64, 32, 4, C.byref(n)) == 0 and n.value > 64 * 32 * 10
+    small = n.value
+    assert L.ubp_bed_workspace_size(512, 512, 2, C.byref(n)) == 0 and n.value > small
+    assert L.ubp_bed_workspace_size(64, 32, 0, C.byref(n)) == -1          # block size < 1
+    assert L.ubp_bed_workspace_size(3, 32, 4, C.byref(n)) == -1           # block longer than the column
+    assert L.ubp_bed_workspace_size(64, 32, 4, None) == -1
+    assert L.ubp_bed_workspace_size(16385, 8, 4, C.byref(n)) == -6        # more rows than the kernel's lists hold
+    assert L.ubp_bed_workspace_size(16384, 1 << 17, 4, C.byref(n)) == -6  # M * C >= 2^31
+    # null pointers are refused before anything is launched
+    assert L.ubp_bed_select(None, 64, 32, 1, 4, 10, None, 0, None, None, None) == -1
+    assert L.ubp_block_scores(None, 64, 32, 1, 4, None, 0, None, None) == -1

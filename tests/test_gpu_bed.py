@@ -29,6 +29,9 @@ CASES = [
     (130, 12, 1, 64, 50, "trained"),       # block longer than a warp
     (8, 8, 1, 8, 0, "trained"),            # one block per column, all kept
     (384, 96, 1, 4, 50, "trained"),
+    (77, 1, 1, 3, 30, "trained"),          # a single input channel
+    (1, 5, 1, 1, 40, "trained"),           # a single output channel, blocks of one
+    (1030, 6, 1, 2, 20, "normal"),         # more rows than 1024: several float4 groups per lane, low sparsity
 ]
 
 
