@@ -172,6 +172,10 @@ __device__ __forceinline__ void flush_counts(SelState *st, unsigned int bin, uns
 // while walking N steps to either side of the chosen entry. Lane l owns the entries of the float4 groups
 // l, l + 32, ... and keeps their maximum in registers; after a choice only the lanes that own a changed entry
 // look at their entries again.
+// NS > 0: the block size, known at compile time and small: lane 0 alone walks the list, re-scores and drops (its
+// loops unroll and their operands stay in registers); NS = 0: any block size, the lanes share that work through a
+// scratch array.
+template <int NS>
 __global__ void __launch_bounds__(32) bed_expand_kernel(const float *__restrict__ S, int M, int C, int Nb, int Mpad, int T,
                                                         unsigned long long m, SelState *st,
                                                         float *__restrict__ ev, uint16_t *__restrict__ order,
@@ -232,51 +236,97 @@ __global__ void __launch_bounds__(32) bed_expand_kernel(const float *__restrict_
         if (__float_as_uint(best) < tau_next) break;        // below the m-th largest score of the whole layer
         tau_next = __ldcg(&st->tau_lb);                      // looked at in the next round
         const int k = bidx;
-        // the N entries after k (lane 0) and before it (lane 1) that are still in the list
-        if (lane < 2) {
-            const uint16_t *link = lane == 0 ? nxt : prv;
-            uint16_t *out = wk + lane * (Nb + 1);
-            unsigned cur = (unsigned)k;
-            for (int t = 1; t <= Nb; ++t) {
-                cur = cur == NONE ? NONE : link[cur];
-                out[t] = (uint16_t)cur;
-            }
-        }
-        __syncwarp();
         unsigned int dirty = 0;
-        // entry n to the left now spans n kernels before the block and N-n after it
-        for (int n = 1 + lane; n < Nb; n += 32) {
-            const unsigned p = wk[(Nb + 1) + n];
-            if (p != NONE) {
-                const unsigned r = wk[Nb - n];
-                s[p] = (s[p] + s[r]) - best;
-                dirty |= 1u << ((p >> 2) & 31u);
+        if constexpr (NS > 0) {
+            if (lane == 0) {
+                unsigned succ[NS + 1], pred[NS];
+                unsigned cur = (unsigned)k;
+#pragma unroll
+                for (int t = 1; t <= NS; ++t) { cur = nxt[cur]; succ[t] = cur; }       // succ[NS] may be the end marker
+                cur = (unsigned)k;
+#pragma unroll
+                for (int n = 1; n < NS; ++n) { cur = cur == NONE ? NONE : prv[cur]; pred[n] = cur; }
+                const unsigned p1 = NS > 1 ? pred[NS > 1 ? 1 : 0] : (unsigned)prv[k];
+                float sv[NS];
+#pragma unroll
+                for (int t = 1; t < NS; ++t) sv[t] = s[succ[t]];
+                // entry n to the left now spans n kernels before the block and N-n after it
+#pragma unroll
+                for (int n = 1; n < NS; ++n)
+                    if (pred[n] != NONE) {
+                        s[pred[n]] = (s[pred[n]] + sv[NS - n]) - best;
+                        dirty |= 1u << ((pred[n] >> 2) & 31u);
+                    }
+                s[k] = NEG;
+                oj[k] = (uint16_t)it;
+                dirty |= 1u << (((unsigned)k >> 2) & 31u);
+#pragma unroll
+                for (int t = 1; t < NS; ++t) {
+                    s[succ[t]] = NEG;
+                    oj[succ[t]] = (uint16_t)it;
+                    dirty |= 1u << ((succ[t] >> 2) & 31u);
+                }
+                if (p1 != NONE) nxt[p1] = (uint16_t)succ[NS];
+                prv[succ[NS]] = (uint16_t)p1;
+                *evp = best;
+                evp += C;
+                // count it; a column's scores fall, so equal bins come in runs: one update per run
+                const unsigned int bin = __float_as_uint(best) >> FINE_SHIFT;
+                if (bin != pend_bin) {
+                    flush_counts(st, pend_bin, pend_cnt);
+                    pend_bin = bin;
+                    pend_cnt = 0;
+                }
+                ++pend_cnt;
             }
-        }
-        __syncwarp();
-        for (int t = lane; t < Nb; t += 32) {
-            const unsigned idx = t == 0 ? (unsigned)k : wk[t];
-            s[idx] = NEG;
-            oj[idx] = (uint16_t)it;
-            dirty |= 1u << ((idx >> 2) & 31u);
-        }
-        if (lane == 0) {
-            const unsigned p1 = wk[(Nb + 1) + 1], sN = wk[Nb];
-            if (p1 != NONE) nxt[p1] = (uint16_t)sN;
-            prv[sN] = (uint16_t)p1;
-            *evp = best;
-            evp += C;
-            // count it; a column's scores fall, so equal bins come in runs: one update per run
-            const unsigned int bin = __float_as_uint(best) >> FINE_SHIFT;
-            if (bin != pend_bin) {
-                flush_counts(st, pend_bin, pend_cnt);
-                pend_bin = bin;
-                pend_cnt = 0;
+            dirty = __shfl_sync(0xffffffffu, dirty, 0);
+            __syncwarp();
+        } else {
+            // the N entries after k (lane 0) and before it (lane 1) that are still in the list
+            if (lane < 2) {
+                const uint16_t *link = lane == 0 ? nxt : prv;
+                uint16_t *out = wk + lane * (Nb + 1);
+                unsigned cur = (unsigned)k;
+                for (int t = 1; t <= Nb; ++t) {
+                    cur = cur == NONE ? NONE : link[cur];
+                    out[t] = (uint16_t)cur;
+                }
             }
-            ++pend_cnt;
+            __syncwarp();
+            // entry n to the left now spans n kernels before the block and N-n after it
+            for (int n = 1 + lane; n < Nb; n += 32) {
+                const unsigned p = wk[(Nb + 1) + n];
+                if (p != NONE) {
+                    const unsigned r = wk[Nb - n];
+                    s[p] = (s[p] + s[r]) - best;
+                    dirty |= 1u << ((p >> 2) & 31u);
+                }
+            }
+            __syncwarp();
+            for (int t = lane; t < Nb; t += 32) {
+                const unsigned idx = t == 0 ? (unsigned)k : wk[t];
+                s[idx] = NEG;
+                oj[idx] = (uint16_t)it;
+                dirty |= 1u << ((idx >> 2) & 31u);
+            }
+            if (lane == 0) {
+                const unsigned p1 = wk[(Nb + 1) + 1], sN = wk[Nb];
+                if (p1 != NONE) nxt[p1] = (uint16_t)sN;
+                prv[sN] = (uint16_t)p1;
+                *evp = best;
+                evp += C;
+                // count it; a column's scores fall, so equal bins come in runs: one update per run
+                const unsigned int bin = __float_as_uint(best) >> FINE_SHIFT;
+                if (bin != pend_bin) {
+                    flush_counts(st, pend_bin, pend_cnt);
+                    pend_bin = bin;
+                    pend_cnt = 0;
+                }
+                ++pend_cnt;
+            }
+            dirty = __reduce_or_sync(0xffffffffu, dirty);
+            __syncwarp();
         }
-        dirty = __reduce_or_sync(0xffffffffu, dirty);
-        __syncwarp();
         if ((dirty >> lane) & 1u) rescan();
         if ((it & 15) == 15) {
             if (lane == 0) { flush_counts(st, pend_bin, pend_cnt); pend_cnt = 0; }
@@ -536,12 +586,15 @@ int ubp_bed_select(const float *W, int M, int C, int R, int Nb, int64_t m, void 
 
     const int Mpad = (M + 127) & ~127;
     const size_t smem = (size_t)Mpad * 4 + (size_t)(M + 1) * 4 + (size_t)(Nb + 1) * 4;
+    using ExpandFn = void (*)(const float *, int, int, int, int, int, unsigned long long, SelState *, float *, uint16_t *, int *);
+    const ExpandFn expand = Nb == 1 ? bed_expand_kernel<1> : Nb == 2 ? bed_expand_kernel<2> : Nb == 4 ? bed_expand_kernel<4>
+                            : Nb == 8 ? bed_expand_kernel<8> : bed_expand_kernel<0>;
     if (smem > 48 * 1024)
-        if (int rc = check(cudaFuncSetAttribute(bed_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)))
+        if (int rc = check(cudaFuncSetAttribute(expand, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)))
             return rc;
     if (int rc = check(cudaMemsetAsync(w.sel, 0, sizeof(SelState), st))) return rc;
     const int T = M / Nb;
-    bed_expand_kernel<<<(unsigned)C, 32, smem, st>>>(w.S, M, C, Nb, Mpad, m > 0 ? T : 0, (unsigned long long)m, w.sel,
+    expand<<<(unsigned)C, 32, smem, st>>>(w.S, M, C, Nb, Mpad, m > 0 ? T : 0, (unsigned long long)m, w.sel,
                                                      w.ev, w.order, w.nev);
     if (int rc = check(cudaGetLastError())) return rc;
     const size_t total = (size_t)T * C;
