@@ -170,6 +170,10 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         }
     };
 
+    // Launched with programmatic stream serialisation, the grid may become resident while the kernel before it in
+    // the stream is still running: let the kernel after this one do the same, set up everything that reads no global
+    // data, and only then wait for the earlier kernel's results (a plain launch passes both instructions at once).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) {
         prefetch_tensormap(&tmX);
         abort_flag = 0;
@@ -187,6 +191,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         // the first copy lands in this CTA's own memory and signals its own barrier: start it before the
         // tensor-memory allocation and the cluster barrier
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if (nmy > 0) issue_stage(0, 0, tile_row0(0), (int)(tile_col0(0) + (int64_t)rank * NH));
     }
     if (warp == 1) {   // tensor memory of the pair: the same warp of both CTAs allocates
@@ -194,6 +199,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // every thread: nothing below may overtake the earlier kernel
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     cluster_sync();                                        // both CTAs' barriers exist before anyone signals them
@@ -435,9 +441,18 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     if (ntiles <= 0) return UBP_OK;
     if (ntiles > 0x7fffffffll) return UBP_E_UNSUPPORTED;
     const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
-    kern<<<dim3((unsigned)(2 * pairs)), T3_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint8_t *>(W16), *tmX, a, halo, nrp, (int)ntiles);
-    cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3(T3_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, static_cast<const uint8_t *>(W16), *tmX, a, halo, nrp, (int)ntiles);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
     return UBP_OK;
 }
