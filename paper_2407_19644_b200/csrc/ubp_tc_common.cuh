@@ -202,9 +202,10 @@ __device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&r)
 // Epilogue of 32 rows (tensor-memory lane quarter q of accumulator `acc`) x the 16-column units first, first + step,
 // ... of one CTA's 128 x N part of a tile, without shared memory (the MMA operands and the copies already use all
 // of its bandwidth). The accumulator is read in the 16 x 256-bit shape: lane t gets, per group j of 8 columns,
-// the column pair 8j + 2(t mod 4) of rows t/4 and t/4 + 8 of a 16-row half. Four lanes therefore hold 32
-// consecutive bytes of an output row, and every 8-byte store instruction of the warp writes eight whole 32-byte
-// sectors; bias and ReLU are applied in registers. (Units of 16 columns rather than 32 so that the warps sharing a
+// the column pair 8j + 2(t mod 4) of rows t/4 and t/4 + 8 of a 16-row half. Neighbouring lanes exchange one pair
+// each, after which a lane holds 16 consecutive bytes of a row and the four lanes of a row its 64 bytes of the unit:
+// every 16-byte store instruction of the warp writes two whole sectors in each of eight rows; bias and ReLU are
+// applied in registers. (Units of 16 columns rather than 32 so that the warps sharing a
 // lane quarter get equal shares of tile widths such as 192 or 224.)
 // `done_bar` != 0: once this warp's last tensor-memory read has completed, lane 0 arrives on that barrier of the
 // leader CTA (the accumulator may be overwritten from then on).
@@ -232,25 +233,59 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
                 else mbar_arrive_remote(done_bar, 0);
             }
         }
-        const int64_t cb = col0 + cc * 16 + 2 * (lane & 3);
+        if (rpc < 128) {
+            // Layers of at most 128 rows: only the warps of two lane quarters have rows to store and they are what the
+            // tile waits for; they store the column pairs as they come (8 bytes per lane, eight 32-byte sectors per
+            // instruction) rather than spend shuffles on wider stores.
+            const int64_t cb = col0 + cc * 16 + 2 * (lane & 3);
 #pragma unroll
-        for (int half = 0; half < 2; ++half)
+            for (int half = 0; half < 2; ++half)
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int row = rbase + 16 * half + 8 * h;
-                if (row >= a.M || lbase + 16 * half + 8 * h >= rpc) continue;
-                float *yrow = a.Y + (size_t)row * a.ldy;
-                const float b = bias[2 * half + h];
+                for (int h = 0; h < 2; ++h) {
+                    const int row = rbase + 16 * half + 8 * h;
+                    if (row >= a.M || lbase + 16 * half + 8 * h >= rpc) continue;
+                    float *yrow = a.Y + (size_t)row * a.ldy;
+                    const float b = bias[2 * half + h];
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    float2 o = make_float2(__uint_as_float(r[half][4 * j + 2 * h]) + b,
-                                           __uint_as_float(r[half][4 * j + 2 * h + 1]) + b);
-                    if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); }
-                    const int64_t col = cb + 8 * j;
-                    if (col + 1 < a.Nc) *reinterpret_cast<float2 *>(yrow + col) = o;
-                    else if (col < a.Nc) yrow[col] = o.x;
+                    for (int j = 0; j < 2; ++j) {
+                        float2 o = make_float2(__uint_as_float(r[half][4 * j + 2 * h]) + b,
+                                               __uint_as_float(r[half][4 * j + 2 * h + 1]) + b);
+                        if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); }
+                        const int64_t col = cb + 8 * j;
+                        if (col + 1 < a.Nc) *reinterpret_cast<float2 *>(yrow + col) = o;
+                        else if (col < a.Nc) yrow[col] = o.x;
+                    }
                 }
-            }
+        } else {
+            // Lanes 2i and 2i + 1 swap a column pair, so that every lane holds four consecutive columns of each of its rows
+            // (even lanes: columns 4i .. 4i + 3 of the unit, odd lanes: 8 + 4i ..) and the warp's 16-byte stores write the
+            // unit's 64 bytes of a row as two whole sectors.
+            const bool odd = (lane & 1) != 0;
+            const int64_t cb = col0 + cc * 16 + (odd ? 8 + 2 * ((lane & 3) - 1) : 2 * (lane & 3));
+#pragma unroll
+            for (int half = 0; half < 2; ++half)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t p0x = r[half][2 * h], p0y = r[half][2 * h + 1];           // columns 2 (t mod 4) + {0, 1}
+                    const uint32_t p1x = r[half][4 + 2 * h], p1y = r[half][4 + 2 * h + 1];   // columns 8 + 2 (t mod 4) + {0, 1}
+                    const uint32_t gx = __shfl_xor_sync(0xffffffffu, odd ? p0x : p1x, 1);
+                    const uint32_t gy = __shfl_xor_sync(0xffffffffu, odd ? p0y : p1y, 1);
+                    const int row = rbase + 16 * half + 8 * h;
+                    if (row >= a.M || lbase + 16 * half + 8 * h >= rpc) continue;
+                    float *yrow = a.Y + (size_t)row * a.ldy;
+                    const float b = bias[2 * half + h];
+                    float4 o = odd ? make_float4(__uint_as_float(gx), __uint_as_float(gy), __uint_as_float(p1x), __uint_as_float(p1y))
+                                   : make_float4(__uint_as_float(p0x), __uint_as_float(p0y), __uint_as_float(gx), __uint_as_float(gy));
+                    o.x += b; o.y += b; o.z += b; o.w += b;
+                    if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                    if (cb + 3 < a.Nc) *reinterpret_cast<float4 *>(yrow + cb) = o;
+                    else {
+                        if (cb < a.Nc) yrow[cb] = o.x;
+                        if (cb + 1 < a.Nc) yrow[cb + 1] = o.y;
+                        if (cb + 2 < a.Nc) yrow[cb + 2] = o.z;
+                    }
+                }
+        }
     }
     // a warp with no unit of its own still owes its arrival
     if (done_bar && first >= nunit) {
