@@ -212,19 +212,28 @@ __device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&r)
 __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, int q, int first, int step, int N,
                                                 int row0, int64_t col0, int lane, uint32_t done_bar, uint32_t rank)
 {
-    const int lbase = q * 32 + (lane >> 2);                 // this lane's rows inside the CTA's part: lbase + {0, 8, 16, 24}
-    const int rbase = row0 + lbase;
     const int rpc = a.rpc ? a.rpc : 128;                    // rows of the CTA's part that exist
     const int nunit = N / 16;
+    // Matrix row of this lane's four accumulator rows (tensor-memory lanes 32 q + t/4 + {0, 8, 16, 24}), -1 where there
+    // is none. A CTA with 128 rows has them in lane order. One with fewer (layers of at most 128 rows) has a quarter of
+    // them at the start of each lane quarter, so that the warps of all four quarters have rows to store: rows
+    // q * rpc/4 ... are lanes 32 q + 0 ..., which is how the plan laid the weight rows out.
+    int rows[4];
     float bias[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-        bias[i] = (a.bias && lbase + 8 * i < rpc && rbase + 8 * i < a.M) ? __ldg(a.bias + rbase + 8 * i) : 0.f;
+    for (int i = 0; i < 4; ++i) {
+        int r = -1;
+        if (rpc == 128) r = row0 + q * 32 + (lane >> 2) + 8 * i;
+        else if ((lane >> 2) + 8 * i < (rpc >> 2)) r = row0 + q * (rpc >> 2) + (lane >> 2) + 8 * i;
+        rows[i] = r < a.M ? r : -1;
+        bias[i] = (a.bias && rows[i] >= 0) ? __ldg(a.bias + rows[i]) : 0.f;
+    }
+    const bool second_half = rpc == 128 || (rpc >> 2) > 16;   // lanes 16 .. 31 of the quarter hold rows at all
 #pragma unroll 1
     for (int cc = first; cc < nunit; cc += step) {
         uint32_t r[2][8];
         tmem_ld_16x256b_x2(acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), r[0]);
-        tmem_ld_16x256b_x2(acc + ((uint32_t)(q * 32 + 16) << 16) + (uint32_t)(cc * 16), r[1]);
+        if (second_half) tmem_ld_16x256b_x2(acc + ((uint32_t)(q * 32 + 16) << 16) + (uint32_t)(cc * 16), r[1]);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (done_bar && cc + step >= nunit) {
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -242,8 +251,8 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
             for (int half = 0; half < 2; ++half)
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const int row = rbase + 16 * half + 8 * h;
-                    if (row >= a.M || lbase + 16 * half + 8 * h >= rpc) continue;
+                    const int row = rows[2 * half + h];
+                    if (row < 0) continue;
                     float *yrow = a.Y + (size_t)row * a.ldy;
                     const float b = bias[2 * half + h];
 #pragma unroll
@@ -270,8 +279,8 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
                     const uint32_t p1x = r[half][4 + 2 * h], p1y = r[half][4 + 2 * h + 1];   // columns 8 + 2 (t mod 4) + {0, 1}
                     const uint32_t gx = __shfl_xor_sync(0xffffffffu, odd ? p0x : p1x, 1);
                     const uint32_t gy = __shfl_xor_sync(0xffffffffu, odd ? p0y : p1y, 1);
-                    const int row = rbase + 16 * half + 8 * h;
-                    if (row >= a.M || lbase + 16 * half + 8 * h >= rpc) continue;
+                    const int row = rows[2 * half + h];
+                    if (row < 0) continue;
                     float *yrow = a.Y + (size_t)row * a.ldy;
                     const float b = bias[2 * half + h];
                     float4 o = odd ? make_float4(__uint_as_float(gx), __uint_as_float(gy), __uint_as_float(p1x), __uint_as_float(p1y))
