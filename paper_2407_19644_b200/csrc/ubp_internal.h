@@ -60,7 +60,9 @@ struct PlanImage {
     int tc_kp = 0;
     // and of the same weight as two bf16 pieces (W1 = the weight rounded to bf16, W2 = the remainder rounded to bf16),
     // tiled: 8 KB blocks [row tile][chunk of 16 channels] = [piece][128 rows][16 channels] in the 32-byte swizzle;
-    // a row tile holds tc16_rows_per_cta(M) rows of the matrix (the rest of its 128 rows are zero);
+    // a row tile holds tc16_rows_per_cta(M) rows of the matrix (the rest of its 128 rows are zero), in order when that
+    // is 128, else a quarter of them at the start of each 32-row quarter of the tile (row positions = tensor-memory
+    // lanes of the accumulator; each epilogue warp reads one lane quarter);
     // tc16_kp = reduction length padded to whole chunks
     size_t tc16_off = 0;
     int tc16_kp = 0;
