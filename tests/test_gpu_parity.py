@@ -106,6 +106,10 @@ TC_CASES = [
     (512, 96, 4, 60, 2048, 32), (300, 150, 4, 70, 544, 32), (256, 256, 4, 70, 4128, 32), (640, 40, 8, 50, 96, 33),
     # at most 128 rows through the bf16-product CTA-pair kernel: each CTA of the pair takes half of the rows
     (128, 128, 4, 60, 4100, 36), (100, 200, 4, 50, 8200, 36), (72, 144, 8, 50, 8196, 37), (128, 64, 2, 50, 16384, 35),
+    # ... and a quarter of those in each tensor-memory lane quarter: 2, 6, 10 and 14 rows per quarter, with row
+    # counts that leave the last quarters partly or wholly empty
+    (8, 128, 4, 50, 8192, 36), (40, 160, 4, 60, 4160, 36), (66, 128, 2, 50, 8200, 35), (120, 256, 8, 70, 4096, 37),
+    (9, 64, 1, 50, 4100, 34),
 ]
 
 
