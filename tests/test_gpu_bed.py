@@ -151,3 +151,30 @@ def test_efficacy_of_the_device_selection_is_above_greedy(M, C, R, Nb, p):
     eff, eff_g = (kept - abp) / (ep - abp), (kept_g - abp) / (ep - abp)
     print(f"efficacy {M}x{C}x{R} N={Nb} {p}%: expansion+division {eff:.4f}, greedy {eff_g:.4f} ({g.size} of {m} blocks)")
     assert 0.0 < eff < 1.0 and eff > eff_g
+
+
+def test_selection_can_be_captured_into_a_cuda_graph():
+    """The selection only enqueues work on the caller's stream (nine kernels and one memset), so it can be captured
+    and replayed; a replay on new weights in the same buffer gives that layer's mask."""
+    import torch
+    import paper_2407_19644_b200 as ubp
+    M, C, R, Nb = 192, 80, 9, 4
+    m = oracle.block_budget(M, C, 75, Nb)
+    sel = ubp.BedSelector(M, C, R, Nb)
+    Wa = ubp_synth.selection_weights(M, C, R, seed=51, kind="trained")
+    Wb = ubp_synth.selection_weights(M, C, R, seed=52, kind="integer")
+    Wd = _dev(Wa)
+    mask = torch.empty((M, C), dtype=torch.uint8, device="cuda")
+    nsel = torch.zeros(1, dtype=torch.int64, device="cuda")
+    sel.select(Wd, m, mask, nsel)                          # once outside the capture (first-launch set-up)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=torch.cuda.Stream()):
+        sel.select(Wd, m, mask, nsel)
+    for W in (Wa, Wb, Wa):
+        Wd.copy_(torch.from_numpy(W))
+        mask.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert int(nsel.item()) == m
+        assert np.array_equal(mask.cpu().numpy(), oracle.bed_select(W, Nb, m)[0])
