@@ -166,7 +166,7 @@ int ubp_plan_check(const ubp_plan_t *plan, void *stream);
 int ubp_plan_clear_status(const ubp_plan_t *plan, void *stream);
 
 /* ubp_selftest_bounded_wait: enqueue a one-warp kernel that waits on an mbarrier nobody ever completes, with
- * the same bounded-wait code the product kernels use but a limit of `limit_us` microseconds (1 .. 1 000 000).
+ * the bounded-wait routine of the tensor-core kernels but a limit of `limit_us` microseconds (1 .. 1 000 000).
  * When the limit runs out the kernel sets the plan's status word and returns, so a following ubp_plan_check
  * reports UBP_E_DEVICE and the context stays usable. Exists so that the "a wait that runs out is reported, not
  * hung" path can be exercised without any fault; not part of the paper's method. */
@@ -181,13 +181,25 @@ int ubp_selftest_bounded_wait(const ubp_plan_t *plan, unsigned limit_us, void *s
  *   bias device [M] or NULL;  relu != 0 applies max(.,0)
  *   Y    device, row o at Y + o*ldy (ldy >= Nc)
  * Fast path needs X, Y 16-byte aligned and ldx, ldy multiples of 4; otherwise a
- * slower kernel is used (same result). Nc == 0 is a no-op.
- * fp32 multiply-add, fp32 accumulation, fixed summation order (bitwise
- * reproducible run to run). */
+ * slower kernel is used (same arithmetic as the sparse kernel). Nc == 0 is a no-op.
+ * Arithmetic, by the kernel the plan's variant selects (ubp_plan_tile_choice names it):
+ *   sparse kernel (variants 1..17, 50..57, and every fallback): fp32 fused
+ *     multiply-add, fp32 accumulation: |Y - exact| <= (L + 2) 2^-24 (|Wm||X| + |bias|),
+ *     L = kept weights of the output row;
+ *   tensor-core kernels, TF32 products (30..33): every fp32 product w x is replaced by
+ *     three products of the operands' TF32 heads and remainders, accumulated in fp32 in
+ *     tensor memory: error <= 2^-18 |w||x| per product plus the accumulation;
+ *   tensor-core kernels, bf16 products (34..37, the choice of variant 0 for layers with
+ *     at least 8 % of the weights kept, 128 output and 128 input channels): three products
+ *     of bf16 heads and remainders, fp32 accumulation: error <= 3 * 2^-16 |w||x| per
+ *     product in the worst case (about 2 * 10^-6 of |Wm||X| on random data).
+ * Every kernel sums in a fixed order: results are bitwise reproducible run to run. */
 int ubp_spmm(const ubp_plan_t *plan, const float *X, int64_t ldx, int64_t Nc,
              const float *bias, int relu, float *Y, int64_t ldy, void *stream);
 
-/* ubp_conv1x1: 1x1 stride-1 convolution = ubp_spmm over columns n = (b, y, x).
+/* ubp_conv1x1: 1x1 stride-1 convolution = ubp_spmm over columns n = (b, y, x)
+ * (Section 4.2: the pointwise convolution is the sparse matrix product the
+ * weight-rotating kernel is written for; Section 3.1 for the block shape).
  * Element strides: in[b][c][y][x] at in + b*in_stride_b + c*in_stride_c + y*Wd + x
  * (NCHW: (C*H*W, H*W); channel-major "CNHW": (H*W, B*H*W)); same for out.
  * If both batch strides equal H*W all images form one product with
@@ -200,8 +212,14 @@ int ubp_conv1x1(const ubp_plan_t *plan, const float *in, int B, int H, int Wd,
 /* ubp_conv3x3_implicit: 3x3, stride 1, zero padding 1, cross-correlation; the
  * plan must come from a blob with R == 9 (a block = Nb output channels x one
  * input channel x all nine taps, Section 3.1). The K = 9*C lowered matrix is
- * never formed: input planes are staged once with their halo and every tap
- * reads them in place. Same strides as ubp_conv1x1. */
+ * never formed in memory. Tensor-core plans (variants 40..47; input and output
+ * each one [channel][batch, y, x] matrix with 16-byte aligned rows) run an
+ * implicit GEMM whose reduction index is tap * C + channel: the input rows of a
+ * 16-channel chunk are copied into shared memory once with a halo of columns
+ * and the nine shifted, border-masked operand tiles are cut from that copy.
+ * Other plans and layouts run a kernel with one lane per output pixel that
+ * reads its taps in place. Arithmetic per kernel as for ubp_spmm.
+ * Same strides as ubp_conv1x1. */
 int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, int Wd,
                          int64_t in_stride_b, int64_t in_stride_c,
                          const float *bias, int relu,
@@ -246,8 +264,11 @@ int ubp_conv1x1_strided(const ubp_plan_t *plan, const float *in, int B, int H, i
  * `stream` -- then the same kernel as ubp_spmm is launched. The function calls
  * no cudaMalloc / cudaFree and no other device-allocating routine.
  * First call on a device: resolves the array's device address
- * (cudaGetSymbolAddress) with that device current; make that first call
- * outside any stream capture.
+ * (cudaGetSymbolAddress) with that device current.
+ * The call cannot be recorded by a stream capture: the upload's source is a
+ * host buffer that lives only for the call, so a replay would read freed
+ * memory. A capturing `stream` is refused with UBP_E_UNSUPPORTED before
+ * anything is enqueued or the array is touched.
  * All calls on a device share the one array: two calls whose GPU work overlaps
  * (different streams, or threads) race on it -- serialise them. The array
  * keeps the previous call's plan until the next upload overwrites it; the

@@ -114,7 +114,13 @@ static int cmp_i64(const void *a, const void *b)
     return (x > y) - (x < y);
 }
 
-/* Algorithm 2. Ibar (cnt indices, any order) -> I (cnt block start indices, ascending). */
+/*
+ * Block division (Algorithm 2). Ibar (cnt chosen indices of the expansion, any order) -> I (cnt block start
+ * indices, ascending). Seen on the original index axis, the kernels the expansion removed form runs: a chosen index
+ * that lies at or beyond everything placed so far opens a run at its own position, and every further chosen index that
+ * falls inside what the run already covers lengthens the run by one block. Division places the t-th block of a run at
+ * run start + t * Nb, i.e. cuts each run every Nb positions from its first one.
+ */
 int orc_bed_divide(const int64_t *Ibar, int64_t cnt, int Nb, int64_t *I)
 {
     if (cnt < 0 || Nb < 1 || (cnt > 0 && (!Ibar || !I))) return ORC_E_ARG;
@@ -122,16 +128,15 @@ int orc_bed_divide(const int64_t *Ibar, int64_t cnt, int Nb, int64_t *I)
     if (!sorted) return ORC_E_SPACE;
     memcpy(sorted, Ibar, (size_t)cnt * sizeof(int64_t));
     qsort(sorted, (size_t)cnt, sizeof(int64_t), cmp_i64);
-    int64_t next_idx = 0;
-    for (int64_t q = 0; q < cnt; ++q) {
-        const int64_t k = sorted[q];
-        if (next_idx > k) {
-            I[q] = next_idx;
-            next_idx += Nb;
-        } else {
-            I[q] = k;
-            next_idx = k + Nb;
-        }
+    int64_t q = 0;
+    while (q < cnt) {
+        const int64_t run_start = sorted[q];
+        int64_t blocks = 0;                           /* blocks of this run placed so far */
+        do {
+            I[q] = run_start + blocks * Nb;
+            ++blocks;
+            ++q;
+        } while (q < cnt && sorted[q] < run_start + blocks * Nb);
     }
     free(sorted);
     return ORC_OK;

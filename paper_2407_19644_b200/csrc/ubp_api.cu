@@ -15,8 +15,6 @@ static thread_local int g_last_cuda = 0;
 void set_last_cuda_error(int e) { g_last_cuda = e; }
 }  // namespace ubp
 
-static const uint32_t kPlanMagic = 0x50504255u;   // "UBPP"
-
 extern "C" {
 
 const char *ubp_strerror(int status)
@@ -103,9 +101,13 @@ int ubp_variant_describe(int variant, char *buf, size_t cap)
 {
     const ubp::KernelCfg *c = ubp::find_cfg(variant);
     if (!c || !buf || cap == 0) return UBP_E_ARG;
-    std::snprintf(buf, cap, "%s nbk=%d panel=%d cols/warp=%d warps=%dx%d ktile=%d%s",
-                  c->kind == 0 ? "spmm" : (c->kind == 1 ? "conv3x3" : (c->kind == 2 ? "spmm-tensorcore(3xTF32) fallback" : "conv3x3-tensorcore(3xTF32) fallback")), c->nbk, c->P, 128 * c->V, c->WR, c->WC, c->KT,
-                  c->dupw ? " dupw" : "");
+    const char *prod = ubp::cfg_bf16(*c) ? "3xBF16" : "3xTF32";
+    char kind[64];
+    if (c->kind == 0) std::snprintf(kind, sizeof kind, "spmm");
+    else if (c->kind == 1) std::snprintf(kind, sizeof kind, "conv3x3");
+    else std::snprintf(kind, sizeof kind, "%s-tensorcore(%s) fallback", c->kind == 2 ? "spmm" : "conv3x3", prod);
+    std::snprintf(buf, cap, "%s nbk=%d panel=%d cols/warp=%d warps=%dx%d ktile=%d%s", kind, c->nbk, c->P, 128 * c->V,
+                  c->WR, c->WC, c->KT, c->dupw ? " dupw" : "");
     return UBP_OK;
 }
 

@@ -127,8 +127,12 @@ int blob_view(const void *blob, size_t len, ubp_view_t *v)
     v->indices = reinterpret_cast<const int32_t *>(base + l.off_indices);
     v->values = reinterpret_cast<const float *>(base + l.off_values);
     // structural checks: monotone indptr ending at m, no start below M - Nb,
-    // channels in range and ascending inside a start row
+    // channels in range and ascending inside a start row, and no two blocks of
+    // one input channel overlapping (Eq. 2): walking the start rows upwards,
+    // next_free[j] is the first row of channel j not covered by a block so far
     if (v->indptr[0] != 0 || v->indptr[h.M] != h.m) return UBP_E_FORMAT;
+    std::vector<int32_t> next_free;
+    try { next_free.assign((size_t)h.C, 0); } catch (const std::bad_alloc &) { return UBP_E_SPACE; }
     for (int i = 0; i < h.M; ++i) {
         const int32_t b0 = v->indptr[i], b1 = v->indptr[i + 1];
         if (b1 < b0 || b1 > h.m) return UBP_E_FORMAT;
@@ -137,6 +141,8 @@ int blob_view(const void *blob, size_t len, ubp_view_t *v)
             const int32_t j = v->indices[b];
             if (j < 0 || j >= h.C) return UBP_E_FORMAT;
             if (b > b0 && v->indices[b - 1] >= j) return UBP_E_FORMAT;
+            if (next_free[(size_t)j] > i) return UBP_E_FORMAT;
+            next_free[(size_t)j] = i + h.Nb;
         }
     }
     return UBP_OK;

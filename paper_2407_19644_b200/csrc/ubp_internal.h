@@ -71,6 +71,8 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
 
 }  // namespace ubp
 
+constexpr uint32_t kPlanMagic = 0x50504255u;   // "UBPP": first word of a live plan handle
+
 struct ubp_plan {
     uint32_t magic;                 // 'UBPP'
     ubp_view_t dims;                // M, C, R, Nb, m (pointers unused)

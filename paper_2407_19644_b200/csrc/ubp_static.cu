@@ -7,6 +7,7 @@
 #include <new>
 
 #include "ubp_internal.h"
+#include "ubp_tc_common.cuh"
 
 #define UBP_STATIC_PLAN_BYTES (2u * 1024u * 1024u)
 
@@ -42,29 +43,17 @@ int static_plan_ptr(void **out)
 
 // ---- bounded-wait self test -------------------------------------------------------------------------------
 namespace {
+// One thread waits on a barrier nobody ever completes, through the wait routine of the tensor-core kernels
+// (tc::mbar_wait) with the caller's limit; when it gives up the plan's status word is set.
 __global__ void ubp_wait_selftest_kernel(int *status, unsigned long long limit_ns)
 {
     __shared__ __align__(8) unsigned long long bar;
-    const unsigned addr = (unsigned)__cvta_generic_to_shared(&bar);
+    __shared__ int abort_flag;
     if (threadIdx.x == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(addr));
+        abort_flag = 0;
+        ubp::tc::mbar_init(ubp::tc::smem_u32(&bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncwarp();
-    if (threadIdx.x == 0) {
-        unsigned long long t0, t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-        bool done = false;
-        for (unsigned it = 0; !done; ++it) {          // nobody arrives: only the clock ends this loop
-            unsigned ok;
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                         "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(addr), "r"(0u) : "memory");
-            if (ok) break;
-            if ((it & 63u) == 0u) {
-                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-                if (t - t0 > limit_ns) { atomicExch(status, 1); done = true; }
-            }
-        }
+        if (!ubp::tc::mbar_wait(ubp::tc::smem_u32(&bar), 0, &abort_flag, limit_ns)) atomicExch(status, 1);
     }
 }
 }  // namespace
@@ -73,7 +62,7 @@ extern "C" {
 
 int ubp_plan_clear_status(const ubp_plan_t *plan, void *stream)
 {
-    if (!plan || !plan->dev) return UBP_E_ARG;
+    if (!plan || plan->magic != kPlanMagic || !plan->dev) return UBP_E_ARG;
     cudaError_t e = cudaMemsetAsync(plan->dev, 0, sizeof(int), static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { ubp::set_last_cuda_error((int)e); return UBP_E_CUDA; }
     return UBP_OK;
@@ -81,7 +70,7 @@ int ubp_plan_clear_status(const ubp_plan_t *plan, void *stream)
 
 int ubp_selftest_bounded_wait(const ubp_plan_t *plan, unsigned limit_us, void *stream)
 {
-    if (!plan || !plan->dev || limit_us == 0 || limit_us > 1000000u) return UBP_E_ARG;
+    if (!plan || plan->magic != kPlanMagic || !plan->dev || limit_us == 0 || limit_us > 1000000u) return UBP_E_ARG;
     ubp_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<int *>(plan->dev),
                                                                              (unsigned long long)limit_us * 1000ull);
     cudaError_t e = cudaGetLastError();
@@ -100,6 +89,15 @@ int ubp_spmm_static(const void *blob, size_t len, const float *X, int64_t ldx, i
     if (v.R != 1 || Nc < 0) return UBP_E_ARG;
     if (Nc == 0) return UBP_OK;
     if (!X || !Y || ldx < Nc || ldy < Nc) return UBP_E_ARG;
+    {
+        // The plan is uploaded from a host buffer that dies with this call. Outside capture the runtime stages the
+        // bytes before cudaMemcpyAsync returns; a captured copy would keep the host pointer and every replay would
+        // read freed memory. So a capturing stream is refused before anything is touched.
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        cudaError_t ce = cudaStreamIsCapturing(static_cast<cudaStream_t>(stream), &cs);
+        if (ce != cudaSuccess) { ubp::set_last_cuda_error((int)ce); return UBP_E_CUDA; }
+        if (cs != cudaStreamCaptureStatusNone) return UBP_E_UNSUPPORTED;
+    }
     const ubp::KernelCfg *cfg = ubp::auto_cfg(v.M, v.C, v.R, v.Nb, v.m);
     if (!cfg) return UBP_E_UNSUPPORTED;
     try {

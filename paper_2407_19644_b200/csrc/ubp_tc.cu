@@ -440,12 +440,6 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
                               (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && a.isc >= Nc;
     const int bf16 = cfg_bf16(pl->cfg) ? 1 : 0;            // variants 34..37 / 44..47
     tc_choose(M, K, Nc, a.conv ? (conv_pair_ok ? a.W : -1) : 0, bf16, sms, &kernel, &rows, &best_n);
-#ifdef UBP_TC_TUNE   // calibration builds only (-DUBP_TC_TUNE): UBP_TC_FORCE=<kernel>,<columns> overrides the choice
-    if (const char *e = getenv("UBP_TC_FORCE")) {
-        int k = 0, n = 0;
-        if (sscanf(e, "%d,%d", &k, &n) == 2) { kernel = k == 12 ? 1 : k; best_n = n; rows = (k == 2 || k == 12) ? 256 : 128; }
-    }
-#endif
     if (kernel == 2 && bf16) {
         CUtensorMap tmX;
         // the input as (column, channel): 16 channel rows of the CTA's columns per chunk, plus the halo for 3x3

@@ -402,7 +402,8 @@ int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d
     TcArgs a = *static_cast<const TcArgs *>(args_);
     a.ntile = ntile;
     const int ngrp = ntile / 64;
-    const size_t smem = (size_t)t2_stages(ngrp, halo) * t2_stage_bytes(ngrp, halo) + 1024;
+    size_t smem = (size_t)t2_stages(ngrp, halo) * t2_stage_bytes(ngrp, halo) + 1024;
+    if (smem < TC_PAIR_MIN_SMEM) smem = TC_PAIR_MIN_SMEM;   // one CTA per SM, whatever the tile width (see the constant)
     static bool done[2][64] = {};
     int devid = 0;
     if (cudaGetDevice(&devid) != cudaSuccess) devid = -1;
@@ -413,6 +414,12 @@ int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d
                              : cudaFuncSetAttribute(ubp_tc2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                     (int)(T2_PIPE_BUDGET + 1024));
         if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+        // the smallest launch this function ever makes must already fill an SM (a query, nothing is launched)
+        int per_sm = 0;
+        e = halo ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ubp_tc2_kernel<true>, T2_THREADS, TC_PAIR_MIN_SMEM)
+                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ubp_tc2_kernel<false>, T2_THREADS, TC_PAIR_MIN_SMEM);
+        if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+        if (per_sm != 1) return UBP_E_UNSUPPORTED;
         if (devid >= 0 && devid < 64) done[which][devid] = true;
     }
     const int nrp = (M + 255) / 256;

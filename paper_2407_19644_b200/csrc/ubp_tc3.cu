@@ -423,7 +423,8 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     const int nh = ntile / 2;
     // chunks per stage: two on long reductions (48 chunks and more), else one
     const int sub = (a.K + TC_KC - 1) / TC_KC >= 48 && t3_stages(nh, halo, 2) >= 4 ? 2 : 1;
-    const size_t smem = (size_t)t3_stages(nh, halo, sub) * t3_stage_bytes(nh, halo, sub) + 1024;
+    size_t smem = (size_t)t3_stages(nh, halo, sub) * t3_stage_bytes(nh, halo, sub) + 1024;
+    if (smem < TC_PAIR_MIN_SMEM) smem = TC_PAIR_MIN_SMEM;   // one CTA per SM, whatever the tile width (see the constant)
     static bool done[4][64] = {};
     int devid = 0;
     if (cudaGetDevice(&devid) != cudaSuccess) devid = -1;
@@ -434,6 +435,11 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     if (devid < 0 || devid >= 64 || !done[which][devid]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(T3_PIPE_BUDGET + 1024));
         if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+        // the smallest launch this function ever makes must already fill an SM (a query, nothing is launched)
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, T3_THREADS, TC_PAIR_MIN_SMEM);
+        if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+        if (per_sm != 1) return UBP_E_UNSUPPORTED;
         if (devid >= 0 && devid < 64) done[which][devid] = true;
     }
     const int nrp = (M + 255) / 256;

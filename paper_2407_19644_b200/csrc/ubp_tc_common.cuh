@@ -43,8 +43,10 @@ __device__ __forceinline__ uint64_t global_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// bounded wait (one second); false if it ran out or another thread of the CTA already gave up
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+// bounded wait (one second unless the caller gives another limit); false if it ran out or another thread of the
+// CTA already gave up
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          uint64_t limit_ns = 1000000000ull)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
@@ -52,7 +54,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > 1000000000ull) break;
+            if (global_ns() - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;
@@ -140,6 +142,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
+
+// The CTA-pair kernels allocate all 512 tensor-memory columns of their SM and then meet the other CTA of the pair at
+// a cluster barrier. Two such CTAs resident on one SM could therefore block each other for good (each pair holding
+// one SM's tensor memory and waiting for the other's). The launchers rule that out by never asking for less dynamic
+// shared memory than this: more than half of what an SM has (228 KB), so a second CTA of any of these kernels never
+// fits beside the first.
+constexpr size_t TC_PAIR_MIN_SMEM = 118 * 1024;
 
 struct TcArgs {
     const float *X;          // 1x1: [K][ldx]; 3x3: input tensor, element (b, c, y, x) at b*isb + c*isc + y*W + x

@@ -118,6 +118,33 @@ def test_blob_view_rejects_corruption():
         assert e.value.code == -4
 
 
+def test_blob_with_overlapping_blocks_is_refused_everywhere():
+    """Two blocks of one input channel that share rows violate Eq. 2. Such a blob must be refused by the validation
+    every consumer runs (view, unpack, plan size, plan image), so that no plan is ever built from it: the sparse and
+    the dense part of a plan would otherwise disagree about the doubly covered rows."""
+    M, C, Nb = 12, 3, 4
+    mask = np.zeros((M, C), np.uint8)
+    mask[0:4, 1] = 1; mask[6:10, 1] = 1; mask[2:6, 2] = 1
+    W = np.arange(M * C, dtype=np.float32).reshape(M, C) + 1
+    blob = bytearray(ubp.ubp_pack(W, mask, Nb))
+    d = ubp.blob_view(bytes(blob))
+    assert d["m"] == 3 and list(d["indptr"][:8]) == [0, 1, 1, 2, 2, 2, 2, 3]
+    # move the block that starts at row 6 of channel 1 up to row 2: rows 2 and 3 of channel 1 are now covered twice.
+    # New start rows: 0 (channel 1), 2 (channels 1 and 2) -> indptr 0,1,1,3,...; indices 1,1,2; channels ascending
+    indptr = [0, 1, 1] + [3] * (M - 2)
+    struct.pack_into(f"<{M + 1}i", blob, 64, *indptr)
+    off_idx = 64 + (4 * (M + 1) + 63) // 64 * 64
+    struct.pack_into("<3i", blob, off_idx, 1, 1, 2)
+    for call in (lambda b: ubp.blob_view(b), lambda b: ubp.ubp_unpack(b), lambda b: ubp.plan_size(b),
+                 lambda b: ubp.plan_image(b), lambda b: ubp.plan_size(b, 32)):
+        with pytest.raises(ubp.UbpError) as e:
+            call(bytes(blob))
+        assert e.value.code == -4
+    # adjacent blocks (a run of two blocks) are fine
+    mask2 = np.zeros((M, C), np.uint8); mask2[0:8, 0] = 1
+    assert ubp.blob_view(ubp.ubp_pack(W, mask2, Nb))["m"] == 2
+
+
 @pytest.mark.parametrize("M,C,Nb,p,R,variant", [
     (64, 64, 4, 50, 1, 0), (100, 70, 4, 60, 1, 1), (100, 70, 4, 60, 1, 3), (100, 70, 4, 60, 1, 4), (100, 70, 4, 60, 1, 5), (100, 70, 4, 60, 1, 7),
     (37, 45, 3, 40, 1, 0), (50, 33, 2, 50, 1, 0), (72, 40, 8, 50, 1, 0), (72, 40, 8, 50, 1, 9),
@@ -236,6 +263,16 @@ def test_bf16_three_term_product_error_bound():
         approx = x1.astype(np.float64) * w1 + x1.astype(np.float64) * w2 + x2.astype(np.float64) * w1
         exact = x.astype(np.float64) * w
         assert np.all(np.abs(approx - exact) <= np.abs(exact) * 3 * 2.0 ** -16)
+    # The bound cannot be tightened to 3 * 2^-18: bf16 keeps 8 significant bits, so rounding to nearest leaves up to
+    # 2^-8 |x| (not 2^-9), the second piece up to 2^-16 |x|, and the dropped terms w1 x3, w3 x1 and w2 x2 reach
+    # 2^-16 |w x| each. One witness pair (both operands a little above 1):
+    x = np.array([float.fromhex("0x1.0aea86p+0")], np.float32)
+    w = np.array([float.fromhex("0x1.031c8ap+0")], np.float32)
+    x1, w1 = bf16(x), bf16(w)
+    x2, w2 = bf16(x - x1), bf16(w - w1)
+    approx = x1.astype(np.float64) * w1 + x1.astype(np.float64) * w2 + x2.astype(np.float64) * w1
+    rel = float(np.abs(approx - x.astype(np.float64) * w)[0] / (float(x[0]) * float(w[0])))
+    assert 3 * 2.0 ** -18 < rel <= 3 * 2.0 ** -16
 
 
 def test_kmajor_blocks_pack_as_the_transposed_layer_and_convert_to_a_plan_blob():

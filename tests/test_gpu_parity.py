@@ -96,6 +96,18 @@ def test_spmm_small(env, M, C, Nb, p, Nc, variant):
     check(Yh, Yref, A, L, variant=plan.variant)
 
 
+@pytest.mark.parametrize("M,C,Nb,p,Nc,variant", [c for c in SMALL if c[2] > 1 and c[3] > 0] +
+                         [c for c in [(128, 64, 4, 50, 256, 32), (300, 150, 4, 70, 520, 32), (520, 200, 8, 50, 1028, 33),
+                                      (256, 256, 4, 70, 4128, 36), (100, 200, 4, 50, 8200, 36), (260, 40, 16, 50, 516, 37)]])
+def test_spmm_aligned_blocks(env, M, C, Nb, p, Nc, variant):
+    """The aligned pattern (every block starts at a multiple of its size: Section 3.1's remark that aligned pruning is
+    the special case of the unaligned one) through the same kernels: sparse configurations and tensor-core variants."""
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 20 * M + C, Nc=Nc, x_dist="normal", relu=(M % 2 == 0), aligned=True)
+    assert all((s % Nb == 0).all() for s in L.starts)
+    Yh, Yref, A, plan = run_spmm(env, L, variant)
+    check(Yh, Yref, A, L, variant=plan.variant)
+
+
 TC_CASES = [
     # M, C, Nb, p, Nc, variant  (30..33 = tensor-core variants for 1 / 2 / 4 / 8-row entries)
     (128, 64, 4, 50, 256, 32), (128, 16, 4, 50, 256, 32), (100, 70, 4, 60, 300, 32), (300, 150, 4, 70, 520, 32),

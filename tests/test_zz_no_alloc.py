@@ -1,9 +1,10 @@
 """ubp_spmm_static: the entry point for callers that cannot allocate device memory (its plan lives in a fixed
-array inside the library). Checked against ubp_spmm on two calls in a row -- the second call finds the
-first call's plan still in the array and must replace it. Collected last on purpose."""
+array inside the library). Checked against ubp_spmm and against the CPU oracle on two calls in a row -- the
+second call finds the first call's plan still in the array and must replace it. Collected last on purpose."""
 import numpy as np
 import pytest
 
+import oracle
 import ubp_synth
 
 pytestmark = pytest.mark.gpu
@@ -30,6 +31,9 @@ def test_static_entry_matches_planned_entry_twice():
         err = np.max(np.abs(got.cpu().numpy().astype(np.float64) - want.cpu().numpy()) / scale)
         assert err <= 1e-4
         assert torch.equal(got, want)
+        # and against the definition itself (the oracle), at the same gate
+        Yref, A = oracle.masked_matmul(L.W, L.mask, L.X, L.bias, relu=L.relu)
+        assert float(np.max(np.abs(got.cpu().numpy() - Yref) / A)) <= 1e-4
     # and the first layer again: the array now holds layer b's plan
     L = layers[0]
     blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
@@ -61,3 +65,30 @@ def test_static_entry_rejects_oversized_layer():
     with pytest.raises(ubp.UbpError) as e:
         ubp.ubp_spmm_static(blob, X)
     assert e.value.code == -8 and "fixed device scratch" in str(e.value)
+
+
+def test_static_entry_refuses_a_capturing_stream():
+    """The upload inside ubp_spmm_static reads a host buffer that lives only for the call, so a captured call would
+    replay from freed memory. A capturing stream is refused (UBP_E_UNSUPPORTED) before anything is enqueued: the
+    capture ends empty and valid, nothing was launched, and an ordinary call afterwards still works."""
+    import torch
+    import paper_2407_19644_b200 as ubp
+    L = ubp_synth.make_layer("cap", 64, 48, 4, 60, 505, Nc=260, x_dist="normal")
+    blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
+    X = torch.from_numpy(L.X).cuda(); bias = torch.from_numpy(L.bias).cuda()
+    out = torch.full((L.M, L.Nc), float("nan"), dtype=torch.float32, device="cuda")
+    want = ubp.ubp_spmm_static(blob, X, bias, L.relu).clone()        # first call on the device, outside capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    marker = torch.zeros(4, device="cuda")
+    with torch.cuda.graph(g, stream=s):
+        marker.fill_(1.0)                                            # so that the graph is not empty
+        with pytest.raises(ubp.UbpError) as e:
+            ubp.ubp_spmm_static(blob, X, bias, L.relu, out=out, stream=s)
+        assert e.value.code == -6
+    g.replay()
+    torch.cuda.synchronize()
+    assert bool((marker == 1).all())                                 # the capture stayed valid
+    assert torch.isnan(out).all()                                    # the refused call recorded nothing
+    assert torch.equal(ubp.ubp_spmm_static(blob, X, bias, L.relu, out=out), want)
