@@ -33,6 +33,7 @@ sys.path.insert(0, ROOT)
 
 import ubp_synth  # noqa: E402
 
+METRIC = "effective GFLOP/s (2 x surviving MACs / time) of one UBP layer"
 SM_COUNT, FP32_LANES, SM_MAX_GHZ = 148, 128, 1.965
 FP32_PEAK_TFLOPS = SM_COUNT * FP32_LANES * 2 * SM_MAX_GHZ / 1e3     # 74.45: plain FP32 FMA pipes at max clock
 
@@ -93,16 +94,17 @@ def tf32_peak_tflops():
     return 1590.0 / 2, "fallback bf16 x 0.5"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (key: workload, plan variant)
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the layer's kernel, from an ncu capture of exactly
+# this launch (`--profile N` runs the bench's kernel on the bench's tensors); key: workload, plan variant. DRAM counters
+# cannot be read outside a profiler, so the line carries these captured figures (null where none was taken).
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("mbv1_pw512", 36): 13936896 + 0,          # profiles/ncu_ubp_tc3_kernel_mbv1_pw512.md (the output is still in L2)
-    ("sweep_nb4_p70", 36): 84903936 + 40135680,  # profiles/ncu_ubp_tc3_kernel_sweep_nb4_p70.md
-    ("r50_3x3", 44): 15257344 + 1280,            # profiles/ncu_ubp_tc3_kernel_r50_3x3.md
-    ("mbv1_pw512", 32): 14984448 + 256,          # profiles/ncu_ubp_tc2_kernel_mbv1_pw512.md
-    ("sweep_nb4_p70", 32): 124626432 + 48126208, # profiles/ncu_ubp_tc2_kernel_sweep_nb4_p70.md
-    ("r50_3x3", 40): 17614080 + 0,               # profiles/ncu_ubp_tc2_kernel_r50_3x3.md
-    ("sweep_nb4_p90", 14): 70554368 + 23536640,  # profiles/ncu_ubp_spmm_kernel_sweep_nb4_p90.md
+    ("mbv1_pw512", 36): 13936896 + 0,            # the 12.8 MB output is still in L2 when the kernel ends
+    ("sweep_nb4_p70", 36): 84903936 + 40135680,
+    ("r50_3x3", 44): 15257344 + 1280,
+    ("mbv1_pw512", 32): 14984448 + 256,
+    ("sweep_nb4_p70", 32): 124626432 + 48126208,
+    ("r50_3x3", 40): 17614080 + 0,
+    ("sweep_nb4_p90", 14): 70554368 + 23536640,
 }
 
 
@@ -246,36 +248,117 @@ def time_e2e(torch, ubp, plan, L, steps, warmup):
     return a.elapsed_time(b) / steps, lanes[0]["Xh"].numel() * 4, lanes[0]["Yh"].numel() * 4
 
 
-def cpu_oracle_time(L, budget_s=20.0):
-    """The oracle as it stands on the host cores, on a bounded sample of the workload's columns."""
+def oracle_sample(L):
+    """The bounded sample of the workload the oracle is run on: (activations of the sample, columns, description,
+    callable that evaluates the oracle on it and returns (Yref, A) as [M][columns] arrays)."""
     import oracle
     dense_macs_per_col = L.M * L.C * L.R
-    # aim at ~1 GMAC per timed call, at least 64 columns (3x3: whole images)
+    # aim at ~1 GMAC per call, at least 64 columns (3x3: whole images)
     if L.R == 9:
         nb = max(1, min(L.B, int(1.0e9 // (dense_macs_per_col * L.H * L.Wd * 0.2 + 1))))
         Xs = np.ascontiguousarray(L.X[:, :nb])
         cols = nb * L.H * L.Wd
-        fn = lambda: oracle.masked_conv3x3(L.W, L.mask, Xs, L.bias, relu=L.relu)
-        sample = f"first {nb} of {L.B} images"
-    else:
-        X2 = L.X.reshape(L.C, -1)
-        cols = int(max(64, min(X2.shape[1], 1.5e9 // dense_macs_per_col)))
-        Xs = np.ascontiguousarray(X2[:, :cols])
-        fn = lambda: oracle.masked_matmul(L.W, L.mask, Xs, L.bias, relu=L.relu)
-        sample = f"first {cols} of {X2.shape[1]} columns"
-    fn()
+
+        def fn():
+            y, a = oracle.masked_conv3x3(L.W, L.mask, Xs, L.bias, relu=L.relu)
+            return y.reshape(L.M, -1), a.reshape(L.M, -1)
+        return Xs, cols, f"first {nb} of {L.B} images", fn
+    X2 = L.X.reshape(L.C, -1)
+    cols = int(max(64, min(X2.shape[1], 1.5e9 // dense_macs_per_col)))
+    Xs = np.ascontiguousarray(X2[:, :cols])
+    return Xs, cols, f"first {cols} of {X2.shape[1]} columns", lambda: oracle.masked_matmul(L.W, L.mask, Xs, L.bias, relu=L.relu)
+
+
+def cpu_oracle_time(L, budget_s=20.0):
+    """The oracle as it stands on the host cores, on a bounded sample of the workload's columns. Returns (effective
+    GFLOP/s, threads, sample description, seconds per call, (Yref, A) of the sample)."""
+    import oracle
+    _, cols, sample, fn = oracle_sample(L)
+    ref = fn()
     ts = []
     t_start = time.perf_counter()
     while len(ts) < 3 and time.perf_counter() - t_start < budget_s:
         t0 = time.perf_counter(); fn(); ts.append(time.perf_counter() - t0)
     t = float(np.median(ts))
     flops = 2.0 * L.m * L.Nb * L.R * cols
-    return flops / t / 1e9, oracle.num_threads(), sample, t
+    return flops / t / 1e9, oracle.num_threads(), sample, t, ref
+
+
+def error_figures(Y, Yref, A):
+    """The three error figures of a result against the oracle's double-precision result on the same columns:
+    scaled      max |Y - Yref| / (|Wm||X| + |bias|)           -- the gate (<= 1e-4)
+    normwise    max |Y - Yref| / max |Yref|
+    elementwise max |Y - Yref| / |Yref| over the outputs with |Yref| >= 1e-3 * rms(Yref)"""
+    Y = np.asarray(Y, dtype=np.float64)
+    d = np.abs(Y - Yref)
+    scale = np.where(A > 0, A, 1.0)
+    rms = float(np.sqrt(np.mean(Yref * Yref)))
+    big = np.abs(Yref) >= 1e-3 * rms
+    return {"scaled": float(np.max(d / scale)), "normwise": float(d.max() / max(float(np.abs(Yref).max()), 1e-300)),
+            "elementwise": float(np.max(d[big] / np.abs(Yref[big]))) if big.any() else 0.0,
+            "outputs_compared": int(Y.size)}
 
 
 def roofline_us(L, hbm_gbs):
     """(time at the FP32 peak, time at the HBM copy bandwidth) of one layer, in microseconds."""
     return (2.0 * L.surviving_macs / (FP32_PEAK_TFLOPS * 1e12) * 1e6, compulsory_bytes(L) / (hbm_gbs * 1e9) * 1e6)
+
+
+KERNEL_NAMES = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF32 on tcgen05, one CTA per tile)",
+                "ubp_tc2_kernel (dense 3xTF32 on tcgen05, CTA pair per tile)",
+                "ubp_tc3_kernel (dense 3xBF16 on tcgen05, CTA pair per tile)")
+ARITHMETIC = ("fp32 FMA, fp32 accumulate",
+              "3 TF32 products per fp32 product, fp32 accumulate (error <= 2^-18 |w||x|)",
+              "3 TF32 products per fp32 product, fp32 accumulate (error <= 2^-18 |w||x|)",
+              "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)")
+
+
+def kernel_info(plan, L):
+    """(index into KERNEL_NAMES / ARITHMETIC, [tile rows, tile columns]) of a fast-path launch of this plan."""
+    kern, tile_rows, tile_cols = plan.tile_choice(L.Nc, L.Wd if L.R == 9 else 0)
+    bf16 = 34 <= plan.variant <= 37 or 44 <= plan.variant <= 47
+    if L.R == 9 and plan.variant < 40:
+        return 0, [tile_rows, tile_cols]
+    return (3 if (kern == 2 and bf16) else kern), [tile_rows, tile_cols]
+
+
+def layer_roofline(L, us, hbm_gbs):
+    """Roofline of one layer at `us` microseconds per launch: the slower of kept FLOPs at the FP32 peak and compulsory
+    bytes at the measured copy bandwidth."""
+    t_alu, t_hbm = roofline_us(L, hbm_gbs)
+    return {"bound": "alu" if t_alu >= t_hbm else "hbm", "roofline_us": max(t_alu, t_hbm), "frac": max(t_alu, t_hbm) / us}
+
+
+def measure_layer(ubp, torch, L, variant, steps, warmup, flush, hbm_gbs, name=None):
+    """Plan + timed launches of one layer (same protocol as the headline: CUDA events per step, L2 flushed). Returns
+    (record, plan, Y): record = {workload, variant, kernel, arithmetic, tile, us (mean), us_median, us_min, bound,
+    roofline_us, frac (from the mean)}."""
+    plan, run, pack_ms, plan_ms, X, Y, bias = build_runner(ubp, torch, L, variant)
+    times = time_steps(torch, run, steps, warmup, flush)
+    plan.check()
+    us = float(np.mean(times)) * 1e3
+    k, tile = kernel_info(plan, L)
+    rec = {"workload": name or L.name, "M": L.M, "K": L.C * L.R, "Nc": L.Nc, "block": f"{L.Nb}x1x{L.R}",
+           "sparsity_pct": L.sparsity_pct, "variant": plan.variant, "kernel": KERNEL_NAMES[k].split(" ")[0],
+           "arithmetic": ARITHMETIC[k].split(",")[0], "tile": tile, "us": us, "us_median": float(np.median(times)) * 1e3,
+           "us_min": float(np.min(times)) * 1e3, "eff_tflops": 2.0 * L.surviving_macs / us / 1e6}
+    rec.update(layer_roofline(L, us, hbm_gbs))
+    return rec, plan, Y
+
+
+def workload_config(L, name, world, no_flush):
+    """The `config` object of the JSON line: the workload and the measurement protocol (the same in both arms)."""
+    return {"workload": name, "M": L.M, "K": L.C * L.R, "Nc": L.Nc, "block": f"{L.Nb}x1x{L.R}",
+            "sparsity_pct": L.sparsity_pct, "blocks": L.m, "bias": L.bias is not None, "relu": bool(L.relu),
+            "l2": "warm" if no_flush else "flushed between steps (256 MiB write)",
+            "parallelism": f"replicated weights, columns sharded x{world}"}
+
+
+# The other BASELINE configurations the default run measures beside the headline (every frac from the mean time)
+EXTRA_CONFIGS = ["r50_3x3", "sweep_nb2_p50", "sweep_nb16_p50", "sweep_nb4_p70", "sweep_nb2_p90", "sweep_nb16_p90"] + \
+                [f"mbv1_L{i + 1}" for i in range(13)]
+# The headline layer through the other two arithmetics: TF32 products on tensor cores, fp32 FMA on the CUDA cores
+HEADLINE_VARIANTS = [32, 14]
 
 
 def build_chained(ubp, torch, layers, variant):
@@ -373,17 +456,17 @@ def run_reference(args, L, name):
     vals = []
     sample = ""
     for i in range(args.warmup + args.steps):
-        g, cores, sample, t = cpu_oracle_time(L, budget_s=1.0)
+        g, cores, sample, t, _ = cpu_oracle_time(L, budget_s=1.0)
         if i >= args.warmup:
             vals.append((g, t))
         if i >= args.warmup + 2 and sum(t for _, t in vals) > 90:
             break
     g = float(np.median([v for v, _ in vals]))
     t = float(np.median([t for _, t in vals]))
-    line = {"metric": "effective GFLOP/s (2 x surviving MACs / time) of one UBP layer", "value": g, "unit": "GFLOP/s",
+    line = {"metric": METRIC, "value": g, "unit": "GFLOP/s",
             "impl": "reference", "n_gpus": args.gpus, "steps": len(vals), "warmup": args.warmup,
             "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": name, "sample": sample},
+            "data": "synthetic", "config": workload_config(L, name, args.gpus, args.no_flush),
             "cpu_baseline": {"value": g, "unit": "GFLOP/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": g, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -534,15 +617,22 @@ def main():
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     ap.add_argument("--no-flush", action="store_true", help="do not flush L2 between steps (warm-L2 figure)")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="default workload only: skip the other arithmetics and the other configurations")
     ap.add_argument("--profile", type=int, default=0, metavar="N",
                     help="build the plan, launch the layer N times and exit (a small target for ncu captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s): start bench.py with "
+                         f"torch.distributed.run --nproc-per-node {args.gpus}, or with no launcher at all")
     name = args.workload
     if name in ("mbv1_chain", "r50_bottleneck"):
         if args.impl == "reference":
@@ -601,6 +691,7 @@ def main():
     torch.cuda.synchronize()
     clocks = sampler.stop()
     plan.check()
+    launches = args.steps
     step_ms = max_over_ranks(float(np.mean(times)), dist, torch, "cuda")
     e2e_ms, h2d, d2h = time_e2e(torch, ubp, plan, L, max(5, min(args.steps, 30)), 3)
     e2e_ms = max_over_ranks(e2e_ms, dist, torch, "cuda")
@@ -622,51 +713,91 @@ def main():
     roof["roofline_us"] = max(t_alu, t_hbm) * 1e6
     roof["frac_of_roofline_time"] = max(t_alu, t_hbm) / (step_ms * 1e-3)
     roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((name, plan.variant))
-    kern, tile_rows, tile_cols = plan.tile_choice(L.Nc, L.Wd if L.R == 9 else 0)
-    bf16 = 34 <= plan.variant <= 37 or 44 <= plan.variant <= 47
-    roof["kernel"] = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF32 on tcgen05, one CTA per tile)",
-                      "ubp_tc3_kernel (dense 3xBF16 on tcgen05, CTA pair per tile)" if bf16 else
-                      "ubp_tc2_kernel (dense 3xTF32 on tcgen05, CTA pair per tile)")[kern]
-    roof["arithmetic"] = ("fp32 FMA, fp32 accumulate", "3 TF32 products per fp32 product, fp32 accumulate (error ~2^-20 |w||x|)",
-                          "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)" if bf16 else
-                          "3 TF32 products per fp32 product, fp32 accumulate (error ~2^-20 |w||x|)")[kern]
-    roof["tile"] = [tile_rows, tile_cols]
-    if plan.variant >= 30:
+    roof["algorithmic_bytes"] = compulsory_bytes(L)
+    k, tile = kernel_info(plan, L)
+    roof["kernel"] = KERNEL_NAMES[k]
+    roof["arithmetic"] = ARITHMETIC[k]
+    roof["tile"] = tile
+    if plan.variant >= 30 and k > 0:
         # the tensor-core variants do 3 x the DENSE multiply-adds; report that rate against the tensor peak of the
         # operand type too (bf16: the measured cuBLAS figure; TF32: half of it, the nominal ratio)
         dense_tf = 3 * 2.0 * L.M * L.C * L.R * L.Nc / (step_ms * 1e-3) / 1e12
         tf32_peak = tf32_peak_tflops()
-        if bf16 and kern == 2:
+        if k == 3:
             roof["tensor"] = {"dense_bf16_tflops": dense_tf, "peak": tf32_peak[0] * 2,
                               "peak_source": tf32_peak[1].replace(" x 0.5", ""), "frac": dense_tf / (tf32_peak[0] * 2)}
         else:
             roof["tensor"] = {"dense_tf32_tflops": dense_tf, "peak": tf32_peak[0], "peak_source": tf32_peak[1],
                               "frac": dense_tf / tf32_peak[0]}
 
+    dtype = "f32" if k == 0 else ("f32 in/out/accumulate; bf16x3 products" if k == 3 else "f32 in/out/accumulate; tf32x3 products")
     line = {
-        "metric": "effective GFLOP/s (2 x surviving MACs / time) of one UBP layer", "value": gflops, "unit": "GFLOP/s",
+        "metric": METRIC, "value": gflops, "unit": "GFLOP/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
         "us_per_layer": step_ms * 1e3, "us_min": float(np.min(times)) * 1e3, "us_median": float(np.median(times)) * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
         "arithmetic": roof.get("arithmetic"),
-        "config": {"workload": name, "M": L.M, "K": L.C * L.R, "Nc": L.Nc, "block": f"{L.Nb}x1x{L.R}",
-                   "sparsity_pct": L.sparsity_pct, "blocks": L.m, "bias": L.bias is not None, "relu": bool(L.relu),
-                   "variant": plan.variant, "l2": "warm" if args.no_flush else "flushed between steps (256 MiB write)",
-                   "parallelism": f"replicated weights, columns sharded x{world}"},
-        "roofline": roof, "clocks": clocks, "gpu_launches": args.steps,
+        "config": workload_config(L, name, world, args.no_flush),
+        "variant": plan.variant,
+        "roofline": roof, "clocks": clocks,
         "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e9, "unit": "GFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "overlap": "steps alternate between two streams with their own buffers"},
         "offline": {"pack_ms": pack_ms, "plan_ms": plan_ms, "plan_bytes": plan.dev_bytes},
     }
+    ref = None
     if rank == 0 and not args.no_cpu:
-        g, cores, sample, _ = cpu_oracle_time(L)
+        g, cores, sample, _, ref = cpu_oracle_time(L)
         line["cpu_baseline"] = {"value": g, "unit": "GFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}
+        # the oracle's outputs on that sample also give the error figures of what the timed kernel wrote
+        run()
+        torch.cuda.synchronize()
+        ncol = ref[0].shape[1]
+        line["errors"] = dict(error_figures(Y.reshape(L.M, -1)[:, :ncol].cpu().numpy(), *ref), sample=sample)
+        launches += 1
+    extras = rank == 0 and not args.headline_only and name == "mbv1_pw512" and args.variant == 0
+    if extras:
+        # the same layer, same protocol, through the other two arithmetics; error figures on the oracle's sample
+        esteps = max(10, min(args.steps, 30))
+        line["variants"] = []
+        for v in HEADLINE_VARIANTS:
+            rec, pv, Yv = measure_layer(ubp, torch, L, v, esteps, 3, flush, hbm_gbs, name=name)
+            launches += esteps + 3
+            if ref is not None:
+                rec["errors"] = error_figures(Yv.reshape(L.M, -1)[:, :ref[0].shape[1]].cpu().numpy(), *ref)
+            line["variants"].append(rec)
+            del pv, Yv
+        # the other BASELINE configurations (automatic variant), each timed like the headline
+        del X, Y, plan, run
+        line["configs"] = []
+        for cname in EXTRA_CONFIGS:
+            Lc = get_layer(cname, seed_index=rank)
+            rec, pc, Yc = measure_layer(ubp, torch, Lc, 0, esteps, 3, flush, hbm_gbs, name=cname)
+            launches += esteps + 3
+            line["configs"].append(rec)
+            del pc, Yc, Lc
+            torch.cuda.empty_cache()
+        chain = [r for r in line["configs"] if r["workload"].startswith("mbv1_L")]
+        line["configs_summary"] = {"min_frac": min(r["frac"] for r in line["configs"]),
+                                   "chain_us_sum": sum(r["us"] for r in chain),
+                                   "chain_roofline_us_sum": sum(r["roofline_us"] for r in chain),
+                                   "steps_each": esteps, "frac_from": "mean"}
+    line["gpu_launches"] = launches
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line), flush=True)
+
+
+def spawn_ranks(n: int, argv) -> int:
+    """`python bench.py --gpus N` without a launcher: start N local ranks of this script under torch.distributed.run
+    (one per GPU, rendezvous on 127.0.0.1) and return their exit code. Rank 0 prints the line."""
+    import socket
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
 
 
 if __name__ == "__main__":

@@ -81,3 +81,46 @@ def test_added_workloads_are_well_formed():
     assert t > 0 and cores == 1 and ("iterations" in sample or "whole" in sample)
     for name, (M, C, R, Nb, p) in bench.BED_WORKLOADS.items():
         assert name.startswith("bed_") and M % Nb == 0 and 0 < p < 100
+
+
+def test_gpus_flag_without_a_launcher_spawns_the_ranks():
+    """`python bench.py --gpus 2` started by hand must not silently measure one rank: it starts two local ranks under
+    torch.distributed.run itself. Exercised on CPU through the reference arm (rank 0 times the oracle and prints the
+    line, the other rank exits 0 without work)."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--workload",
+                        "fc64", "--steps", "1", "--warmup", "3"], capture_output=True, text=True, timeout=600, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(ln) for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                        # rank 0 alone prints
+    assert lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2 and lines[0]["config"]["workload"] == "fc64"
+    # a launcher that started another number of ranks than --gpus says is an error, not a silent one-GPU run
+    env2 = dict(env, WORLD_SIZE="3", RANK="0", LOCAL_RANK="0")
+    r2 = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--workload",
+                         "fc64", "--steps", "1"], capture_output=True, text=True, timeout=600, env=env2)
+    assert r2.returncode != 0 and "rank" in (r2.stderr + r2.stdout)
+
+
+def test_both_arms_describe_the_same_config():
+    sys.path.insert(0, ROOT)
+    import bench
+    L = bench.get_layer("mbv1_pw512")
+    c = bench.workload_config(L, "mbv1_pw512", 1, False)
+    assert c["workload"] == "mbv1_pw512" and c["M"] == 512 and c["Nc"] == 6272 and c["blocks"] == 19660
+    assert set(bench.EXTRA_CONFIGS) >= {"r50_3x3", "sweep_nb2_p50", "sweep_nb16_p90", "mbv1_L1", "mbv1_L13"}
+    assert all(n in bench.WORKLOADS for n in bench.EXTRA_CONFIGS)
+
+
+def test_error_figures_on_known_values():
+    sys.path.insert(0, ROOT)
+    import bench
+    Yref = np.array([[1.0, -2.0, 0.0], [4.0, 1e-9, 2.0]])
+    A = np.array([[2.0, 4.0, 1.0], [8.0, 1.0, 4.0]])
+    Y = Yref + np.array([[1e-3, 0.0, 1e-3], [0.0, 1e-3, -2e-3]])
+    e = bench.error_figures(Y.astype(np.float64), Yref, A)
+    assert abs(e["scaled"] - 1e-3) < 1e-12                       # |d|/A: 5e-4, 0, 1e-3, 0, 1e-3, 5e-4
+    assert abs(e["normwise"] - 2e-3 / 4.0) < 1e-12
+    assert abs(e["elementwise"] - 1e-3) < 1e-9                   # zeros and the 1e-9 entry are below 1e-3 rms: left out
+    assert e["outputs_compared"] == 6
