@@ -206,6 +206,62 @@ def time_steps(torch, run, steps, warmup, flush_buf):
     return [a.elapsed_time(b) for a, b in evs]
 
 
+L2_BYTES = 126 * 1024 * 1024
+
+
+def rotating_sets(torch, ubp, plan, L, X, bias, min_bytes=int(2.5 * L2_BYTES), max_sets=24):
+    """Independent copies of the layer's activations, each with its own output tensor: as many as it takes for the
+    set of all of them to exceed the L2 cache 2.5 times over (at least two), so that a step that walks through them
+    in turn never finds its inputs or its output lines in L2. Returns (runs, tensors): runs[i]() launches the layer
+    on copy i."""
+    per_set = X.numel() * 4 + L.M * L.Nc * 4
+    nsets = int(max(2, min(max_sets, -(-min_bytes // per_set))))
+    runs, keep = [], []
+    for i in range(nsets):
+        Xi = X if i == 0 else X.clone()
+        if L.R == 9:
+            Yi = torch.empty((L.M, L.B, L.H, L.Wd), dtype=torch.float32, device="cuda")
+            runs.append(lambda Xi=Xi, Yi=Yi: ubp.ubp_conv3x3_implicit(plan, Xi, bias, L.relu, out=Yi))
+        elif L.X.ndim == 4:
+            Yi = torch.empty((L.M, L.B, L.H, L.Wd), dtype=torch.float32, device="cuda")
+            runs.append(lambda Xi=Xi, Yi=Yi: ubp.ubp_conv1x1(plan, Xi, bias, L.relu, out=Yi))
+        else:
+            Yi = torch.empty((L.M, L.Nc), dtype=torch.float32, device="cuda")
+            runs.append(lambda Xi=Xi, Yi=Yi: ubp.ubp_spmm(plan, Xi, bias, L.relu, out=Yi))
+        keep.append((Xi, Yi))
+    return runs, keep
+
+
+def time_region(torch, runs, steps, warmup, extra_regions=0, hold_s=0.0):
+    """EXACTLY `steps` steps timed as ONE region: step i launches runs[i % len(runs)] (independent batches whose
+    tensors together exceed L2, so every step starts cold), all of them enqueued from one CUDA graph on one stream
+    and bracketed by one pair of CUDA events with a synchronize on both sides. Returns [ms of the region, ms of
+    `extra_regions` repetitions...]; afterwards the same graph keeps replaying for `hold_s` seconds (untimed) so
+    that a clock sampler sees the load. A pair of events around a single launch reads about 6 us even for an empty
+    kernel on this hardware; bracketing the whole region, as a serving loop would run it, leaves that out and lets
+    a launch start while its predecessor drains."""
+    for i in range(warmup):
+        runs[i % len(runs)]()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=torch.cuda.Stream()):
+        for i in range(steps):
+            runs[i % len(runs)]()
+    graph.replay()                       # untimed: uploads the graph and counts as further warm-up
+    torch.cuda.synchronize()
+    out = []
+    for _ in range(1 + extra_regions):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); graph.replay(); b.record()
+        torch.cuda.synchronize()
+        out.append(a.elapsed_time(b))
+    t_end = time.perf_counter() + hold_s
+    while time.perf_counter() < t_end:
+        graph.replay()
+        torch.cuda.synchronize()
+    return out
+
+
 def time_e2e(torch, ubp, plan, L, steps, warmup):
     """Same step through the public call with HOST buffers: pinned X -> device, kernel, Y -> pinned host, every
     step. Steps alternate between two streams with their own device and host buffers, so that the upload of step
@@ -330,19 +386,27 @@ def layer_roofline(L, us, hbm_gbs):
 
 
 def measure_layer(ubp, torch, L, variant, steps, warmup, flush, hbm_gbs, name=None):
-    """Plan + timed launches of one layer (same protocol as the headline: CUDA events per step, L2 flushed). Returns
-    (record, plan, Y): record = {workload, variant, kernel, arithmetic, tile, us (mean), us_median, us_min, bound,
-    roofline_us, frac (from the mean)}."""
+    """Plan + timed launches of one layer, same protocol as the headline: one region of `steps` launches over rotating
+    batches (time_region); beside it the older per-step figure (a pair of events around every launch, L2 flushed by a
+    256 MiB write before it). Returns (record, plan, Y): record = {workload, variant, kernel, arithmetic, tile, us
+    (region time / steps), bound, roofline_us, frac, us_flushed (mean), frac_flushed}."""
     plan, run, pack_ms, plan_ms, X, Y, bias = build_runner(ubp, torch, L, variant)
-    times = time_steps(torch, run, steps, warmup, flush)
+    runs, keep = rotating_sets(torch, ubp, plan, L, X, bias)
+    regions = time_region(torch, runs, steps, warmup, extra_regions=2)
+    times = time_steps(torch, run, max(5, steps // 3), 3, flush)
     plan.check()
-    us = float(np.mean(times)) * 1e3
+    us = regions[0] / steps * 1e3
+    usf = float(np.mean(times)) * 1e3
     k, tile = kernel_info(plan, L)
     rec = {"workload": name or L.name, "M": L.M, "K": L.C * L.R, "Nc": L.Nc, "block": f"{L.Nb}x1x{L.R}",
            "sparsity_pct": L.sparsity_pct, "variant": plan.variant, "kernel": KERNEL_NAMES[k].split(" ")[0],
-           "arithmetic": ARITHMETIC[k].split(",")[0], "tile": tile, "us": us, "us_median": float(np.median(times)) * 1e3,
-           "us_min": float(np.min(times)) * 1e3, "eff_tflops": 2.0 * L.surviving_macs / us / 1e6}
+           "arithmetic": ARITHMETIC[k].split(",")[0], "tile": tile, "us": us,
+           "us_regions": [r / steps * 1e3 for r in regions], "batches": len(runs),
+           "eff_tflops": 2.0 * L.surviving_macs / us / 1e6}
     rec.update(layer_roofline(L, us, hbm_gbs))
+    rec["us_flushed"] = usf
+    rec["frac_flushed"] = rec["roofline_us"] / usf
+    del runs, keep
     return rec, plan, Y
 
 
@@ -350,7 +414,9 @@ def workload_config(L, name, world, no_flush):
     """The `config` object of the JSON line: the workload and the measurement protocol (the same in both arms)."""
     return {"workload": name, "M": L.M, "K": L.C * L.R, "Nc": L.Nc, "block": f"{L.Nb}x1x{L.R}",
             "sparsity_pct": L.sparsity_pct, "blocks": L.m, "bias": L.bias is not None, "relu": bool(L.relu),
-            "l2": "warm" if no_flush else "flushed between steps (256 MiB write)",
+            "l2": "warm: one batch reused" if no_flush else
+                  "cold: steps walk through independent batches whose tensors exceed L2 2.5 times over",
+            "timed_region": "all steps enqueued from one CUDA graph, one event pair around them",
             "parallelism": f"replicated weights, columns sharded x{world}"}
 
 
@@ -390,23 +456,28 @@ def run_chain(args, torch, ubp, rank, world, dist, cfg="mbv1_chain"):
         for L in layers:
             plan, run, _, _, X, Y, bias = build_runner(ubp, torch, L, args.variant)
             plans.append(plan); runs.append(run); keep.append((X, Y, bias))
-    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
-    for run in runs:            # warm every kernel outside the capture (first-launch attribute set-up)
-        run()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+
+    def one_pass():
+        for run in runs:
+            run()
+    one_pass()                  # warm every kernel outside the capture (first-launch attribute set-up)
     torch.cuda.synchronize()
     graph = torch.cuda.CUDAGraph()
     cap_stream = torch.cuda.Stream()
     with torch.cuda.graph(graph, stream=cap_stream):
-        for run in runs:
-            run()
+        one_pass()
     per_layer = []
     for L, run in zip(layers, runs):
         ts = time_steps(torch, run, max(5, args.steps // 5), 3, flush)
         per_layer.append(float(np.median(ts)) * 1e3)
+    flushed = time_steps(torch, graph.replay, max(5, args.steps // 3), 3, flush)
     sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
     sampler.start()
-    times = time_steps(torch, graph.replay, args.steps, args.warmup, flush)
+    # the timed region: `steps` passes over the chain, all launches from one CUDA graph, one event pair around them
+    regions = time_region(torch, [one_pass], args.steps, args.warmup, extra_regions=1, hold_s=0.4)
     clocks = sampler.stop()
+    times = [regions[0] / args.steps]
     for p in plans:
         p.check()
     step_ms = max_over_ranks(float(np.mean(times)), dist, torch, "cuda")
@@ -417,15 +488,19 @@ def run_chain(args, torch, ubp, rank, world, dist, cfg="mbv1_chain"):
         "metric": f"effective GFLOP/s (2 x surviving MACs / time) of the {len(layers)}-layer chain",
         "value": aggregate_gflops(flops, world, step_ms), "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32 in/out/accumulate; per layer fp32 FMA or bf16x3 products (layers[].variant)",
+        "data": "synthetic",
         "config": {"workload": cfg, "layers": len(layers), "batch": layers[0].B, "block": "4x1xR", "sparsity_pct": 80,
-                   "launch": f"{len(layers)} kernels replayed from one CUDA graph",
-                   "l2": "warm" if args.no_flush else "flushed between steps (256 MiB write)"},
+                   "launch": f"{len(layers)} kernels per step; all steps replayed from one CUDA graph, one event pair around them",
+                   "l2": "not flushed: the chain's tensors (about 1.5 GB) exceed L2 many times over" if cfg == "mbv1_chain"
+                         else "not flushed: the three layers' tensors (about 70 MB) partly stay in L2 from step to step"},
+        "per_step_flushed": {"us_mean": float(np.mean(flushed)) * 1e3, "frac": roof_total_us / (float(np.mean(flushed)) * 1e3),
+                             "protocol": "one graph replay of the chain per event pair, L2 flushed by a 256 MiB write before it"},
         "roofline": {"bound": "mixed (per layer: see layers)", "roofline_us": roof_total_us,
                      "frac_of_roofline_time": roof_total_us / (step_ms * 1e3),
                      "peak_source": f"FP32 74.45 TFLOP/s derived; HBM {hbm_gbs} GB/s {peak_src}"},
-        "layers": [{"name": L.name, "M": L.M, "K": L.C * L.R, "Nc": L.B * L.H * L.Wd, "variant": p.variant, "us": us,
-                    "roofline_us": max(r), "bound": "alu" if r[0] >= r[1] else "hbm", "frac": max(r) / us}
+        "layers": [{"name": L.name, "M": L.M, "K": L.C * L.R, "Nc": L.B * L.H * L.Wd, "variant": p.variant, "us_flushed": us,
+                    "roofline_us": max(r), "bound": "alu" if r[0] >= r[1] else "hbm", "frac_flushed": max(r) / us}
                    for L, p, us, r in zip(layers, plans, per_layer, roofs)],
         "clocks": clocks, "gpu_launches": len(layers) * args.steps,
     }
@@ -680,19 +755,25 @@ def main():
         plan.check()
         print(json.dumps({"profile_launches": args.profile, "workload": name, "variant": plan.variant}), flush=True)
         return
-    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    runs, keep = ([run], []) if args.no_flush else rotating_sets(torch, ubp, plan, L, X, bias)
 
     sampler = ClockSampler(local_rank)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
-    times = time_steps(torch, run, args.steps, args.warmup, flush)
+    regions = time_region(torch, runs, args.steps, args.warmup, extra_regions=2, hold_s=0.4)
     torch.cuda.synchronize()
     clocks = sampler.stop()
+    clocks["sampled"] = "from the timed region on, while the same graph kept replaying for 0.4 s"
     plan.check()
     launches = args.steps
-    step_ms = max_over_ranks(float(np.mean(times)), dist, torch, "cuda")
+    step_ms = max_over_ranks(regions[0] / args.steps, dist, torch, "cuda")
+    # the older per-step protocol beside it: a pair of events around every launch, L2 flushed by a 256 MiB write
+    times = time_steps(torch, run, max(10, min(args.steps, 50)), 3, flush)
+    plan.check()
+    del runs, keep
     e2e_ms, h2d, d2h = time_e2e(torch, ubp, plan, L, max(5, min(args.steps, 30)), 3)
     e2e_ms = max_over_ranks(e2e_ms, dist, torch, "cuda")
 
@@ -734,7 +815,12 @@ def main():
     line = {
         "metric": METRIC, "value": gflops, "unit": "GFLOP/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
-        "us_per_layer": step_ms * 1e3, "us_min": float(np.min(times)) * 1e3, "us_median": float(np.median(times)) * 1e3,
+        "us_per_layer": step_ms * 1e3, "us_per_layer_regions": [r / args.steps * 1e3 for r in regions],
+        "per_step_flushed": {"us_mean": float(np.mean(times)) * 1e3, "us_median": float(np.median(times)) * 1e3,
+                             "us_min": float(np.min(times)) * 1e3, "steps": len(times),
+                             "frac": max(t_alu, t_hbm) / (float(np.mean(times)) * 1e-3),
+                             "protocol": "a pair of CUDA events around every launch, L2 flushed by a 256 MiB write before "
+                                         "it; two events around an empty kernel read about 6 us here"},
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
         "arithmetic": roof.get("arithmetic"),
         "config": workload_config(L, name, world, args.no_flush),
@@ -782,7 +868,9 @@ def main():
                                    "chain_us_sum": sum(r["us"] for r in chain),
                                    "chain_roofline_us_sum": sum(r["roofline_us"] for r in chain),
                                    "steps_each": esteps, "frac_from": "mean"}
-    line["gpu_launches"] = launches
+    line["gpu_launches"] = args.steps                 # inside the timed region: one kernel per step
+    line["gpu_launches_beside"] = launches - args.steps + len(times) + 3 * args.steps   # warm-up replay, two more regions,
+                                                                                      # flushed steps, variants and configs
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
