@@ -362,11 +362,14 @@ def roofline_us(L, hbm_gbs):
 
 KERNEL_NAMES = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF32 on tcgen05, one CTA per tile)",
                 "ubp_tc2_kernel (dense 3xTF32 on tcgen05, CTA pair per tile)",
-                "ubp_tc3_kernel (dense 3xBF16 on tcgen05, CTA pair per tile)")
+                "ubp_tc3_kernel (dense 3xBF16 on tcgen05, CTA pair per tile)",
+                "ubp_wros_kernel (the paper's loop over the canonical arrays, weight rotation, FP32 FMA)",
+                "ubp_wros_kernel (the paper's loop over the canonical arrays, naive shift, FP32 FMA)")
 ARITHMETIC = ("fp32 FMA, fp32 accumulate",
               "3 TF32 products per fp32 product, fp32 accumulate (error <= 2^-18 |w||x|)",
               "3 TF32 products per fp32 product, fp32 accumulate (error <= 2^-18 |w||x|)",
-              "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)")
+              "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)",
+              "fp32 FMA, fp32 accumulate", "fp32 FMA, fp32 accumulate")
 
 
 def kernel_info(plan, L):
@@ -375,6 +378,8 @@ def kernel_info(plan, L):
     bf16 = 34 <= plan.variant <= 37 or 44 <= plan.variant <= 47
     if L.R == 9 and plan.variant < 40:
         return 0, [tile_rows, tile_cols]
+    if plan.variant in (60, 61):
+        return plan.variant - 56, [tile_rows, tile_cols]
     return (3 if (kern == 2 and bf16) else kern), [tile_rows, tile_cols]
 
 
@@ -504,6 +509,77 @@ def run_chain(args, torch, ubp, rank, world, dist, cfg="mbv1_chain"):
                    for L, p, us, r in zip(layers, plans, per_layer, roofs)],
         "clocks": clocks, "gpu_launches": len(layers) * args.steps,
     }
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+# Per-layer comparison of pruning patterns and dataflows (the paper's Section 5.4 on B200): layer shape, sparsity
+CMP_WORKLOADS = {
+    "cmp_pw512_p80": dict(M=512, C=512, B=64, H=14, Wd=14, p=80, w_scale=0.05),
+    "cmp_pw512_p90": dict(M=512, C=512, B=64, H=14, Wd=14, p=90, w_scale=0.05),
+    "cmp_2048_p80": dict(M=2048, C=2048, Nc=8192, p=80, w_scale=0.02),
+    "cmp_2048_p90": dict(M=2048, C=2048, Nc=8192, p=90, w_scale=0.02),
+}
+CMP_PATTERNS = [("EP", 1, False), ("ABP 1x2", 2, True), ("UBP 1x2", 2, False), ("ABP 1x4", 4, True), ("UBP 1x4", 4, False)]
+CMP_KERNELS = [("plan, sparse FP32 kernel", {1: 17, 2: 15, 4: 14}), ("paper loop, weight rotation (60)", 60),
+               ("paper loop, naive shift (61)", 61), ("plan, tensor-core bf16x3 kernel", {1: 34, 2: 35, 4: 36})]
+
+
+def cmp_layer(name, pattern_index, seed_index=0):
+    w = CMP_WORKLOADS[name]
+    label, nb, aligned = CMP_PATTERNS[pattern_index]
+    kw = dict(Nc=w["Nc"], x_dist="normal") if "Nc" in w else dict(B=w["B"], H=w["H"], Wd=w["Wd"])
+    return ubp_synth.make_layer(f"{name}:{label}", w["M"], w["C"], nb, w["p"], 8000 + 10 * seed_index + pattern_index,
+                                w_scale=w["w_scale"], aligned=aligned, **kw)
+
+
+def run_cmp(args, name, rank, local_rank, world):
+    """Element-wise, aligned and unaligned pruning of one layer at one sparsity through (a) the plan-based sparse
+    kernel, (b) the two kernels that keep the paper's own loop over the canonical arrays, with weight rotation and
+    naive, (c) the tensor-core kernel. One JSON line; `comparison` holds the table (us per launch, region protocol)
+    and the ratios Section 5.4 discusses: unaligned / aligned and naive / weight-rotating."""
+    import torch
+    import paper_2407_19644_b200 as ubp
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    ubp.load()
+    torch.cuda.set_device(local_rank)
+    hbm_gbs, _ = measured_peaks()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    steps = max(10, min(args.steps, 40))
+    table = {}
+    head = None
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for pi, (label, nb, aligned) in enumerate(CMP_PATTERNS):
+        L = cmp_layer(name, pi, seed_index=rank)
+        row = {}
+        for kname, v in CMP_KERNELS:
+            variant = v[nb] if isinstance(v, dict) else v
+            rec, plan, Y = measure_layer(ubp, torch, L, variant, steps, 3, flush, hbm_gbs, name=f"{name}:{label}")
+            row[kname] = {"us": rec["us"], "us_flushed": rec["us_flushed"], "variant": rec["variant"], "frac": rec["frac"]}
+            if label == "UBP 1x4" and variant == 14:
+                head = (L, rec)
+            del plan, Y
+            torch.cuda.empty_cache()
+        table[label] = row
+    clocks = sampler.stop()
+    ratios = {}
+    for kname, _ in CMP_KERNELS[:3]:
+        ratios[kname] = {f"UBP/ABP 1x{nb}": table[f"UBP 1x{nb}"][kname]["us"] / table[f"ABP 1x{nb}"][kname]["us"] for nb in (2, 4)}
+        ratios[kname].update({f"EP/UBP 1x{nb}": table["EP"][kname]["us"] / table[f"UBP 1x{nb}"][kname]["us"] for nb in (2, 4)})
+    ratios["naive/weight-rotating"] = {lab: table[lab][CMP_KERNELS[2][0]]["us"] / table[lab][CMP_KERNELS[1][0]]["us"]
+                                       for lab in ("UBP 1x2", "UBP 1x4", "ABP 1x2", "ABP 1x4")}
+    L, rec = head
+    line = {"metric": METRIC, "value": 2.0 * L.surviving_macs / rec["us"] / 1e3, "unit": "GFLOP/s", "n_gpus": 1,
+            "steps": steps, "warmup": 3, "ms_per_step": rec["us"] / 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": dict(workload_config(L, name, 1, False), headline_cell="UBP 1x4 through the plan-based sparse kernel"),
+            "roofline": {"bound": rec["bound"], "frac": rec["frac"], "roofline_us": rec["roofline_us"]},
+            "comparison": {"us_per_launch": table, "ratios": ratios,
+                           "paper": "Section 5.4 (phone CPU): unaligned with weight rotation about equal to aligned, the "
+                                    "naive unaligned kernel clearly slower, larger blocks faster than element-wise"},
+            "clocks": clocks, "gpu_launches": steps}
     if rank == 0:
         print(json.dumps(line), flush=True)
 
@@ -729,6 +805,11 @@ def main():
         return
     if name in BED_WORKLOADS:
         run_bed(args, name, rank, local_rank, world)
+        return
+    if name in CMP_WORKLOADS:
+        if args.impl == "reference":
+            raise SystemExit("--impl reference times single layers; pick a layer workload")
+        run_cmp(args, name, rank, local_rank, world)
         return
     L = get_layer(name, seed_index=rank)
 

@@ -106,6 +106,12 @@ int ubp_kmajor_to_plan_blob(const void *kblob, size_t klen, void *blob, size_t b
  * variant: 0 = choose from the layer shape; > 0 = a specific kernel
  * configuration (ubp_variant_count / ubp_variant_describe list them), meant
  * for measuring configurations against each other.
+ * Variants 60 and 61 (R == 1, Nb in {1, 2, 4, 8, 16}) are comparison kernels that keep the paper's own dataflow:
+ * their plan is the canonical arrays themselves, a thread walks the start rows with row step 1 and keeps Nb
+ * stationary accumulators; 60 uses the stored rotation (Section 4.2: the finished row sits in slot i mod Nb, no
+ * accumulator ever moves), 61 is the naive form of Section 3.3 (row order, store the first accumulator and move
+ * the others down after every start row). With aligned masks they are the aligned kernel, with Nb = 1 the
+ * element-wise one (Section 5.4's comparison).
  */
 typedef struct ubp_plan ubp_plan_t;
 
@@ -152,7 +158,8 @@ int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info);
  * operands qualify for the fast path (for 3x3: input and output as one [channel][batch, y, x] matrix each), and
  * its output tile. `image_width` is the width of the input planes for a 3x3 plan (Nc = batch * height * width),
  * ignored for 1x1. *kernel: 0 = sparse FP32 kernel (Section 4.2's output-stationary product on the CUDA cores),
- * 1 = tensor-core kernel with one CTA per tile, 2 = tensor-core kernel with a CTA pair per tile. Host only;
+ * 1 = tensor-core kernel with one CTA per tile, 2 = tensor-core kernel with a CTA pair per tile, 3 = the comparison
+ * kernels that walk the canonical arrays in the paper's own dataflow (variants 60 and 61; tile_rows is 0). Host only;
  * enqueues nothing. Not part of the paper's method: it exists so that measurements and tests can name what ran. */
 int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, int *kernel, int *tile_rows,
                          int *tile_cols);

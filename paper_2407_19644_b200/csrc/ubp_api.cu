@@ -103,6 +103,11 @@ int ubp_variant_describe(int variant, char *buf, size_t cap)
     if (!c || !buf || cap == 0) return UBP_E_ARG;
     const char *prod = ubp::cfg_bf16(*c) ? "3xBF16" : "3xTF32";
     char kind[64];
+    if (c->kind == 4) {
+        std::snprintf(buf, cap, "spmm-from-canonical-arrays %s", c->id == 61 ? "naive(outputs shifted per start row)"
+                                                                            : "weight-rotating output-stationary");
+        return UBP_OK;
+    }
     if (c->kind == 0) std::snprintf(kind, sizeof kind, "spmm");
     else if (c->kind == 1) std::snprintf(kind, sizeof kind, "conv3x3");
     else std::snprintf(kind, sizeof kind, "%s-tensorcore(%s) fallback", c->kind == 2 ? "spmm" : "conv3x3", prod);
@@ -206,6 +211,8 @@ int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, in
         if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
         ubp::tc_choose(plan->dims.M, plan->dims.C * plan->dims.R, Nc, c.kind == 3 ? image_width : 0, ubp::cfg_bf16(c) ? 1 : 0, sms, kernel, tile_rows,
                        tile_cols);
+    } else if (c.kind == 4) {
+        *kernel = 3; *tile_rows = 0; *tile_cols = 512;       // row ranges are chosen per launch; 128 threads x 4 columns
     } else {
         *kernel = 0; *tile_rows = c.P * c.WR; *tile_cols = 128 * c.V * c.WC;
     }

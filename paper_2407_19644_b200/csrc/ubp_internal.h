@@ -21,7 +21,8 @@ int blob_view(const void *blob, size_t len, ubp_view_t *v);
 // kernel instantiation consumes them.
 struct KernelCfg {
     int id;        // 1-based variant id
-    int kind;      // 0 = 1x1 product (R == 1), 1 = implicit 3x3 (R == 9), 2 = 1x1 on tensor cores (densified
+    int kind;      // 4 = 1x1 product walked from the canonical arrays in the paper's own dataflow (ubp_wros.cu);
+                   // 0 = 1x1 product (R == 1), 1 = implicit 3x3 (R == 9), 2 = 1x1 on tensor cores (densified
                    //     panels, 3 x TF32) with the kind-0 plan of the same geometry embedded as its fallback,
                    // 3 = 3x3 as an implicit GEMM on tensor cores with the kind-1 plan embedded
     int nbk;       // rows per plan entry; divides the layer's Nb
@@ -66,6 +67,8 @@ struct PlanImage {
     // tc16_kp = reduction length padded to whole chunks
     size_t tc16_off = 0;
     int tc16_kp = 0;
+    // kind 4 only: byte offsets of the canonical arrays indptr [M+1], indices [m], values [m][Nb] in the image
+    size_t wros_off[3] = {0, 0, 0};
 };
 int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only, PlanImage &img, size_t *bytes);
 
@@ -98,6 +101,9 @@ int launch_conv3x3(const ubp_plan *plan, const float *in, int B, int H, int Wd, 
                    const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream, int stride = 1);
 int launch_subsample(const float *in, int C, int B, int H, int Wd, int64_t isb, int64_t isc, int stride, float *out,
                      void *stream);
+// the paper's dataflow on the canonical arrays (ubp_wros.cu): variants 60 (weight rotation) and 61 (naive shift)
+int launch_wros(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu, float *Y,
+                int64_t ldy, void *stream);
 void set_last_cuda_error(int e);
 }
 

@@ -647,6 +647,7 @@ int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, con
                       (ldx % 4 == 0) && (ldy % 4 == 0) && (int64_t)ldx * 4 < (1ll << 40) &&
                       pl->dims.C < (1 << 30) && Nc < (1ll << 31);
     int rc = UBP_E_UNSUPPORTED;
+    if (c.kind == 4) return launch_wros(pl, X, ldx, Nc, bias, relu, Y, ldy, stream_);
     if (fast && c.kind == 2) return launch_spmm_tc(pl, X, ldx, Nc, bias, relu, Y, ldy, stream);
 #define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP)                                                \
     if (fast && c.id == ID)                                                                               \

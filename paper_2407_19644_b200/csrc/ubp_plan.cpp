@@ -98,6 +98,23 @@ static inline size_t pad16(size_t x) { return (x + 15) & ~(size_t)15; }
 int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only, PlanImage &img, size_t *bytes)
 {
     const int M = v.M, C = v.C, R = v.R, Nb = v.Nb;
+    if (cfg.kind == 4) {
+        // the canonical arrays as they are, behind the 256-byte header with the status word
+        if (R != 1 || (Nb != 1 && Nb != 2 && Nb != 4 && Nb != 8 && Nb != 16)) return UBP_E_UNSUPPORTED;
+        const size_t o0 = 256, o1 = pad16(o0 + sizeof(int32_t) * ((size_t)M + 1));
+        const size_t o2 = pad16(o1 + sizeof(int32_t) * (size_t)v.m);
+        const size_t total = (o2 + sizeof(float) * (size_t)v.m * Nb + 255) & ~(size_t)255;
+        img = PlanImage();
+        img.wros_off[0] = o0; img.wros_off[1] = o1; img.wros_off[2] = o2;
+        img.entries = v.m;
+        if (bytes) *bytes = total;
+        if (count_only) return UBP_OK;
+        img.bytes.assign(total, 0);
+        std::memcpy(img.bytes.data() + o0, v.indptr, sizeof(int32_t) * ((size_t)M + 1));
+        std::memcpy(img.bytes.data() + o1, v.indices, sizeof(int32_t) * (size_t)v.m);
+        std::memcpy(img.bytes.data() + o2, v.values, sizeof(float) * (size_t)v.m * Nb);
+        return UBP_OK;
+    }
     const int nbk = cfg.nbk, P = cfg.P, KT = cfg.KT, WR = cfg.WR;
     if (Nb % nbk != 0) return UBP_E_UNSUPPORTED;
     const bool conv = (cfg.kind == 1 || cfg.kind == 3);

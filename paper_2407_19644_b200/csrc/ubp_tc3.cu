@@ -35,6 +35,9 @@ constexpr int T3_XL_GROUPS = 2;                           // two groups of four 
 constexpr int T3_EPI_WARPS = 8;                           // warps 10..17
 constexpr int T3_THREADS = (2 + T3_XL_WARPS + T3_EPI_WARPS) * 32;
 constexpr int T3_MAX_STAGES = 8;
+#ifndef T3_PRE
+#define T3_PRE 1
+#endif
 constexpr uint32_t T3_A_PART = 128 * TC_KC * 2;           // W1 or W2 chunk of this CTA's 128 rows: 4 KB
 constexpr uint32_t T3_ATOM = 64 * TC_KC * 2;              // x1 or x2 of 64 columns x 16 channels: 2 KB
 constexpr uint32_t T3_PIPE_BUDGET = 222 * 1024;
@@ -155,20 +158,32 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     // one stage's copies (stage sg of a tile = chunks sg * SUB ...): per chunk the W1 / W2 block of this CTA's 128
     // rows (8 KB, stored in the plan exactly as it must lie in shared memory: one contiguous bulk copy) and 16
     // channel rows of the input for this CTA's columns (3x3: the channels of the chunk's tap, and a halo of columns
-    // either side)
-    auto issue_stage = [&](int sg, int st, int row0, int xcol) {
+    // either side). The weight copies come first and announce the bytes of both; the activation copies may follow
+    // later (the kernel's first stages start their weight copies before the previous kernel in the stream is done).
+    auto issue_w = [&](int sg, int st, int row0) {
         const uint32_t bar = smem_u32(&bar_full[st]);
         const int c0 = sg * SUB, nsub = nchunk - c0 < SUB ? nchunk - c0 : SUB;
         mbar_expect_tx(bar, (uint32_t)nsub * tx);
 #pragma unroll
         for (int u = 0; u < SUB; ++u) {
             if (u >= nsub) break;
+            uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
+            bulk_load(smem_u32(chunk), W16 + ((size_t)(row0 / rpc) * nchunk + c0 + u) * (2 * T3_A_PART), 2 * T3_A_PART, bar);
+        }
+    };
+    auto issue_x = [&](int sg, int st, int xcol) {
+        const uint32_t bar = smem_u32(&bar_full[st]);
+        const int c0 = sg * SUB, nsub = nchunk - c0 < SUB ? nchunk - c0 : SUB;
+#pragma unroll
+        for (int u = 0; u < SUB; ++u) {
+            if (u >= nsub) break;
             const int c = c0 + u;
             uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
-            bulk_load(smem_u32(chunk), W16 + ((size_t)(row0 / rpc) * nchunk + c) * (2 * T3_A_PART), 2 * T3_A_PART, bar);
             tma_load_2d(smem_u32(chunk + 2 * T3_A_PART + 2 * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
         }
     };
+    // stages whose weight copies start before the wait for the previous kernel
+    const int npre = nmy * nstage < T3_PRE ? nmy * nstage : T3_PRE;
 
     // Launched with programmatic stream serialisation, the grid may become resident while the kernel before it in
     // the stream is still running: let the kernel after this one do the same, set up everything that reads no global
@@ -189,10 +204,12 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         mbar_init(smem_u32(&bar_last), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        // the first copy lands in this CTA's own memory and signals its own barrier: start it before the
-        // tensor-memory allocation and the cluster barrier
+        // The first copies land in this CTA's own memory and signal its own barriers: start them before the
+        // tensor-memory allocation and the cluster barrier. The weights are constants of the layer, so the copies of
+        // the ring's first stages do not wait for the kernel before this one; the activations may be its output.
+        for (int f = 0; f < npre; ++f) issue_w(f % nstage, f, tile_row0(f / nstage));
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (nmy > 0) issue_stage(0, 0, tile_row0(0), (int)(tile_col0(0) + (int64_t)rank * NH));
+        for (int f = 0; f < npre; ++f) issue_x(f % nstage, f, (int)(tile_col0(f / nstage) + (int64_t)rank * NH));
     }
     if (warp == 1) {   // tensor memory of the pair: the same warp of both CTAs allocates
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -210,15 +227,18 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     if (warp == 0) {
         // ---------------- TMA producer: one ring of S stages straight through all of this pair's tiles
         if (lane == 0) {
-            int st = 1 % S, round = 1 / S;                 // stage 0 of the first tile was started above
+            int st = npre % S, round = npre / S;           // the first npre stages were started above
+            int f = 0;                                     // stages counted through all tiles
             for (int i = 0; i < nmy && ok; ++i) {
                 const int row0 = tile_row0(i), xcol = (int)(tile_col0(i) + (int64_t)rank * NH);
-                for (int sg = (i == 0 ? 1 : 0); sg < nstage; ++sg) {
+                for (int sg = 0; sg < nstage; ++sg, ++f) {
+                    if (f < npre) continue;
                     if (round > 0) {                       // the stage's previous contents must have been consumed
                         ok = mbar_wait_relaxed(smem_u32(&bar_empty[st]), (uint32_t)(round - 1) & 1u, &abort_flag);
                         if (!ok) break;
                     }
-                    issue_stage(sg, st, row0, xcol);
+                    issue_w(sg, st, row0);
+                    issue_x(sg, st, xcol);
                     if (++st == S) { st = 0; ++round; }
                 }
             }

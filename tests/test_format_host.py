@@ -169,6 +169,28 @@ def test_plan_image_replays_to_masked_weight(M, C, Nb, p, R, variant):
     assert n_entries == len(sub) + crossing
 
 
+def test_plan_of_the_paper_dataflow_variants_is_the_canonical_arrays():
+    """Variants 60 / 61 walk the packed format itself: their plan image is a 256-byte header followed by indptr,
+    indices and the rotated values, each on a 16-byte boundary, bit for bit as in the blob."""
+    L = ubp_synth.make_layer("t", 50, 30, 4, 60, 77, Nc=4)
+    blob = ubp.ubp_pack(L.W, L.mask, 4)
+    d = ubp.blob_view(blob)
+    for variant in (60, 61):
+        img, _ = ubp.plan_image(blob, variant)
+        assert len(img) % 256 == 0 and not img[:256].any()
+        o1 = (256 + 4 * 51 + 15) // 16 * 16
+        o2 = (o1 + 4 * d["m"] + 15) // 16 * 16
+        assert np.array_equal(np.frombuffer(img, "<i4", 51, 256), d["indptr"])
+        assert np.array_equal(np.frombuffer(img, "<i4", d["m"], o1), d["indices"])
+        assert np.array_equal(np.frombuffer(img, "<u4", d["m"] * 4, o2), d["values"].view(np.uint32).ravel())
+    L3 = ubp_synth.make_layer("t", 24, 12, 3, 50, 78, Nc=4)
+    with pytest.raises(ubp.UbpError):
+        ubp.plan_size(ubp.ubp_pack(L3.W, L3.mask, 3), 60)         # block sizes 1, 2, 4, 8, 16 only
+    L9 = ubp_synth.make_layer("t", 16, 8, 4, 50, 79, R=9, B=1, H=2, Wd=2)
+    with pytest.raises(ubp.UbpError):
+        ubp.plan_size(ubp.ubp_pack(L9.W, L9.mask, 4), 61)         # 1x1 only
+
+
 def test_plan_rejects_wrong_kind():
     L = ubp_synth.make_layer("t", 16, 8, 4, 50, 3, Nc=4)
     blob = ubp.ubp_pack(L.W, L.mask, 4)

@@ -108,6 +108,37 @@ def test_spmm_aligned_blocks(env, M, C, Nb, p, Nc, variant):
     check(Yh, Yref, A, L, variant=plan.variant)
 
 
+@pytest.mark.parametrize("variant", [60, 61])
+@pytest.mark.parametrize("M,C,Nb,p,Nc,aligned,pad,misalign", [
+    (64, 64, 4, 50, 256, False, 0, 0), (100, 70, 4, 60, 300, False, 0, 0), (300, 150, 2, 70, 516, False, 0, 0),
+    (33, 20, 1, 50, 260, False, 0, 0), (72, 40, 8, 50, 264, False, 0, 0), (80, 40, 16, 50, 260, False, 0, 0),
+    (130, 257, 4, 80, 1028, False, 0, 0), (16, 8, 4, 50, 4, False, 0, 0), (8, 40, 8, 50, 128, False, 0, 0),
+    (100, 70, 4, 60, 300, True, 0, 0), (72, 40, 8, 50, 264, True, 0, 0), (96, 64, 2, 70, 520, True, 0, 0),
+    (70, 50, 4, 60, 130, False, 2, 0), (70, 50, 4, 60, 131, False, 1, 0), (70, 50, 4, 60, 255, False, 0, 0),
+    (70, 50, 4, 60, 256, False, 0, 1), (70, 50, 2, 60, 1, False, 3, 0), (512, 96, 4, 80, 2048, False, 0, 0),
+])
+def test_paper_dataflow_variants(env, variant, M, C, Nb, p, Nc, aligned, pad, misalign):
+    """The comparison kernels that keep the paper's own loop (row step 1 over the canonical arrays; Section 3.3 and
+    Section 4.2): weight-rotating output-stationary (60) and naive with shifted outputs (61), on unaligned and aligned
+    masks, element-wise pruning (Nb = 1), ragged and misaligned operands. fp32 FMA: the fp32 summation bound holds."""
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 30 * M + C, Nc=Nc, x_dist="normal", relu=(M % 2 == 0), aligned=aligned)
+    Yh, Yref, A, plan = run_spmm(env, L, variant, pad=pad, misalign=misalign)
+    assert plan.variant == variant and plan.tile_choice(Nc)[0] == 3
+    check(Yh, Yref, A, L, variant=0)
+
+
+def test_paper_dataflow_variants_agree_bitwise_where_the_order_is_the_same(env):
+    """Both forms add a row's products in the same order (tiles ascending, channels ascending inside a tile), so the
+    rotation changes where an accumulator lives, not what it holds: identical bits."""
+    torch, ubp = env
+    L = ubp_synth.make_layer("t", 200, 120, 4, 70, 4711, Nc=1024, x_dist="normal")
+    blob = ubp.ubp_pack(L.W, L.mask, 4)
+    X = torch.from_numpy(L.X).cuda(); b = torch.from_numpy(L.bias).cuda()
+    Y60 = ubp.ubp_spmm(ubp.Plan(blob, 60), X, b, True)
+    Y61 = ubp.ubp_spmm(ubp.Plan(blob, 61), X, b, True)
+    assert torch.equal(Y60, Y61)
+
+
 TC_CASES = [
     # M, C, Nb, p, Nc, variant  (30..33 = tensor-core variants for 1 / 2 / 4 / 8-row entries)
     (128, 64, 4, 50, 256, 32), (128, 16, 4, 50, 256, 32), (100, 70, 4, 60, 300, 32), (300, 150, 4, 70, 520, 32),
