@@ -64,12 +64,17 @@ BED_WORKLOADS = {
 KMAJOR_B = 4     # kmajor_pw512: the headline layer's shape with blocks of 4 consecutive INPUT channels in one output row
 
 
+KMAJOR_WORKLOADS = {"kmajor_pw512": 70, "kmajor_pw512_p80": 80, "kmajor_pw512_p90": 90, "kmajor_pw512_p95": 95}
+
+
 def get_layer(name: str, seed_index: int = 0):
-    if name == "kmajor_pw512":
-        # generated as the transposed layer (blocks run down the rows of [C][M]) and turned round; to the kernels it is
-        # a layer of M*C*(1-p) single-channel blocks
-        t = ubp_synth.make_layer(name, 512, 512, KMAJOR_B, 70, 7000 + seed_index, B=32, H=14, Wd=14, w_scale=0.05)
-        return ubp_synth.Layer(name, t.C, t.M, 1, 1, 70, t.m * KMAJOR_B, np.ascontiguousarray(t.W.transpose(1, 0, 2)),
+    if name in KMAJOR_WORKLOADS:
+        # 512 -> 512 channels at 14 x 14, batch 32, blocks of KMAJOR_B consecutive INPUT channels inside one output row:
+        # generated as the transposed layer (blocks run down the rows of [C][M]) and turned round. The Layer object
+        # describes it as M*C*(1-p) single weights (Nb = 1); the packed form keeps the runs (build_runner).
+        sp = KMAJOR_WORKLOADS[name]
+        t = ubp_synth.make_layer(name, 512, 512, KMAJOR_B, sp, 7000 + seed_index, B=32, H=14, Wd=14, w_scale=0.05)
+        return ubp_synth.Layer(name, t.C, t.M, 1, 1, sp, t.m * KMAJOR_B, np.ascontiguousarray(t.W.transpose(1, 0, 2)),
                                np.ascontiguousarray(t.mask.T), t.X, t.bias, True, t.B, t.H, t.Wd)
     w = WORKLOADS[name]
     layers = ubp_synth.config_layers(w["cfg"], index=seed_index, **w["kw"])
@@ -166,12 +171,13 @@ class ClockSampler:
 def build_runner(ubp, torch, L, variant):
     """Returns (plan, run(stream-less call), pack_ms, plan_ms, device tensors)."""
     t0 = time.perf_counter()
-    if L.name == "kmajor_pw512":
-        blob = ubp.ubp_kmajor_to_plan_blob(ubp.ubp_pack_kmajor(L.W[:, :, 0], L.mask, KMAJOR_B))
+    kmajor = L.name in KMAJOR_WORKLOADS
+    if kmajor:
+        blob = ubp.ubp_pack_kmajor(L.W[:, :, 0], L.mask, KMAJOR_B)
     else:
         blob = ubp.ubp_pack(L.W, L.mask, L.Nb)
     t1 = time.perf_counter()
-    plan = ubp.Plan(blob, variant)
+    plan = ubp.Plan(blob, variant, kmajor=kmajor)
     torch.cuda.synchronize()
     t2 = time.perf_counter()
     X = torch.from_numpy(L.X).cuda()
@@ -380,6 +386,8 @@ def kernel_info(plan, L):
         return 0, [tile_rows, tile_cols]
     if plan.variant in (60, 61):
         return plan.variant - 56, [tile_rows, tile_cols]
+    if 70 <= plan.variant <= 73:
+        return 0, [tile_rows, tile_cols]
     return (3 if (kern == 2 and bf16) else kern), [tile_rows, tile_cols]
 
 

@@ -88,9 +88,8 @@ int ubp_blob_view(const void *blob, size_t len, ubp_view_t *view);
  *   (UBP_E_RAGGED for a run that is not a whole number of blocks).
  * ubp_kmajor_to_plan_blob (host): that blob -> a blob ubp_plan_size / ubp_plan_build accept: the same kept weights
  *   in the layer's own orientation as blocks of ONE output channel (any mask is a valid set of such blocks). The
- *   tensor-core kernels work on the densified weight and do not care about the orientation; below their density
- *   threshold the layer runs on the sparse kernel's element-wise configuration, one index per kept weight (a
- *   kernel that walks K-runs with one index per B weights is not built). */
+ *   tensor-core kernels work on the densified weight and do not care about the orientation; on the sparse kernel
+ *   this form costs one index per kept weight (ubp_plan_build_kmajor below keeps one index per run instead). */
 int ubp_pack_kmajor(const float *W, const uint8_t *mask, int M, int C, int B,
                     void *blob, size_t blob_cap, size_t *blob_len);
 int ubp_kmajor_to_plan_blob(const void *kblob, size_t klen, void *blob, size_t blob_cap, size_t *blob_len);
@@ -145,6 +144,20 @@ int ubp_plan_build(const void *blob, size_t len, int variant, void *dev_buf, siz
                    void *stream, ubp_plan_t **plan);
 void ubp_plan_free(ubp_plan_t *plan);
 
+/* Plans straight from a K-major blob (the forms of ubp_plan_size / ubp_plan_image / ubp_plan_build for the other
+ * orientation; the handle reports the layer's own M and C, and ubp_spmm / ubp_conv1x1 take it like any other).
+ * variant 0 chooses: the tensor-core kernel where it pays (at least 8 % of the weights kept, 128 output and input
+ * channels; the weight is densified, the orientation does not matter there), else the K-run sparse kernel
+ * (variants 70..73 for B = 2, 4, 8, 16): fp32 FMA, output rows stationary in registers, a plan entry = one run
+ * (row, first channel, B weights), i.e. ONE channel index per B weights and B consecutive rows of the staged
+ * activation tile per entry; a run that crosses a channel-tile boundary is cut there. Other run lengths fall back
+ * to the element-wise configuration (one index per weight). A variant > 0 that is not 70..73 is applied to the
+ * re-expressed layer (ubp_kmajor_to_plan_blob). */
+int ubp_plan_size_kmajor(const void *kblob, size_t klen, int variant, size_t *dev_bytes);
+int ubp_plan_image_kmajor(const void *kblob, size_t klen, int variant, void *host_buf, size_t cap, int32_t geom[8]);
+int ubp_plan_build_kmajor(const void *kblob, size_t klen, int variant, void *dev_buf, size_t dev_bytes, void *stream,
+                          ubp_plan_t **plan);
+
 typedef struct {
     int32_t M, C, R, Nb, m;      /* layer                                         */
     int32_t variant;             /* configuration actually chosen                 */
@@ -190,7 +203,7 @@ int ubp_selftest_bounded_wait(const ubp_plan_t *plan, unsigned limit_us, void *s
  * Fast path needs X, Y 16-byte aligned and ldx, ldy multiples of 4; otherwise a
  * slower kernel is used (same arithmetic as the sparse kernel). Nc == 0 is a no-op.
  * Arithmetic, by the kernel the plan's variant selects (ubp_plan_tile_choice names it):
- *   sparse kernel (variants 1..17, 50..57, and every fallback): fp32 fused
+ *   sparse kernel (variants 1..17, 50..57, 70..73, and every fallback) and the comparison kernels 60, 61: fp32 fused
  *     multiply-add, fp32 accumulation: |Y - exact| <= (L + 2) 2^-24 (|Wm||X| + |bias|),
  *     L = kept weights of the output row;
  *   tensor-core kernels, TF32 products (30..33): every fp32 product w x is replaced by

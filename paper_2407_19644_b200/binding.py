@@ -74,6 +74,9 @@ def load():
     L.ubp_conv1x1_strided.argtypes = [vp, vp, i32, i32, i32, i32, i64, i64, vp, sz, vp, i32, vp, i64, i64, vp]
     L.ubp_pack_kmajor.argtypes = [vp, vp, i32, i32, i32, vp, sz, C.POINTER(sz)]
     L.ubp_kmajor_to_plan_blob.argtypes = [vp, sz, vp, sz, C.POINTER(sz)]
+    L.ubp_plan_size_kmajor.argtypes = [vp, sz, i32, C.POINTER(sz)]
+    L.ubp_plan_image_kmajor.argtypes = [vp, sz, i32, vp, sz, C.POINTER(C.c_int32)]
+    L.ubp_plan_build_kmajor.argtypes = [vp, sz, i32, vp, sz, vp, C.POINTER(vp)]
     L.ubp_bed_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
     L.ubp_block_scores.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, vp]
     L.ubp_bed_select.argtypes = [vp, i32, i32, i32, i32, i64, vp, sz, vp, vp, vp]
@@ -177,22 +180,26 @@ def variants():
     return out
 
 
-def plan_size(blob: bytes, variant: int = 0) -> int:
+def plan_size(blob: bytes, variant: int = 0, kmajor: bool = False) -> int:
+    """Bytes of device memory the plan needs. kmajor: `blob` comes from ubp_pack_kmajor (blocks along the input
+    channels)."""
     L = load()
     b = np.frombuffer(blob, np.uint8)
     n = C.c_size_t(0)
-    _chk(L.ubp_plan_size(_np_ptr(b), b.size, variant, C.byref(n)), "ubp_plan_size")
+    fn = L.ubp_plan_size_kmajor if kmajor else L.ubp_plan_size
+    _chk(fn(_np_ptr(b), b.size, variant, C.byref(n)), "ubp_plan_size")
     return n.value
 
 
-def plan_image(blob: bytes, variant: int = 0):
+def plan_image(blob: bytes, variant: int = 0, kmajor: bool = False):
     """Host copy of the device plan image and its geometry (no GPU needed)."""
     L = load()
     b = np.frombuffer(blob, np.uint8)
-    n = plan_size(blob, variant)
+    n = plan_size(blob, variant, kmajor)
     buf = np.zeros(n, np.uint8)
     geom = (C.c_int32 * 8)()
-    _chk(L.ubp_plan_image(_np_ptr(b), b.size, variant, _np_ptr(buf), n, geom), "ubp_plan_image")
+    fn = L.ubp_plan_image_kmajor if kmajor else L.ubp_plan_image
+    _chk(fn(_np_ptr(b), b.size, variant, _np_ptr(buf), n, geom), "ubp_plan_image")
     keys = ["nbk", "panel_rows", "k_tile", "WR", "dupw", "nkt", "NP", "NG"]
     return buf, dict(zip(keys, [int(g) for g in geom]))
 
@@ -219,20 +226,22 @@ class Plan:
     """Device plan of one packed layer. The device buffer is a torch uint8
     tensor owned by this object; the library holds only a small host handle."""
 
-    def __init__(self, blob: bytes, variant: int = 0, device="cuda", stream=None):
+    def __init__(self, blob: bytes, variant: int = 0, device="cuda", stream=None, kmajor: bool = False):
+        """kmajor: `blob` comes from ubp_pack_kmajor (blocks of consecutive input channels inside one output row)."""
         import torch
         L = load()
         self._lib = L
         self._handle = None
         b = np.frombuffer(blob, np.uint8)
-        n = plan_size(blob, variant)
+        n = plan_size(blob, variant, kmajor)
         self.buffer = torch.empty(n + 256, dtype=torch.uint8, device=device)
         base = self.buffer.data_ptr()
         self._dev = (base + 255) // 256 * 256
         h = C.c_void_p()
         with torch.cuda.device(self.buffer.device):
-            _chk(L.ubp_plan_build(_np_ptr(b), b.size, variant, C.c_void_p(self._dev), n, _stream_ptr(stream),
-                                  C.byref(h)), "ubp_plan_build")
+            build = L.ubp_plan_build_kmajor if kmajor else L.ubp_plan_build
+            _chk(build(_np_ptr(b), b.size, variant, C.c_void_p(self._dev), n, _stream_ptr(stream), C.byref(h)),
+                 "ubp_plan_build")
         self._handle = h
         info = _PlanInfo()
         _chk(L.ubp_plan_info(h, C.byref(info)), "ubp_plan_info")

@@ -109,6 +109,7 @@ int ubp_variant_describe(int variant, char *buf, size_t cap)
         return UBP_OK;
     }
     if (c->kind == 0) std::snprintf(kind, sizeof kind, "spmm");
+    else if (c->kind == 5) std::snprintf(kind, sizeof kind, "spmm-k-runs(blocks along the input channels)");
     else if (c->kind == 1) std::snprintf(kind, sizeof kind, "conv3x3");
     else std::snprintf(kind, sizeof kind, "%s-tensorcore(%s) fallback", c->kind == 2 ? "spmm" : "conv3x3", prod);
     std::snprintf(buf, cap, "%s nbk=%d panel=%d cols/warp=%d warps=%dx%d ktile=%d%s", kind, c->nbk, c->P, 128 * c->V,
@@ -120,6 +121,7 @@ static int resolve_cfg(const ubp_view_t &v, int variant, const ubp::KernelCfg **
 {
     const ubp::KernelCfg *c = variant == 0 ? ubp::auto_cfg(v.M, v.C, v.R, v.Nb, v.m) : ubp::find_cfg(variant);
     if (!c) return variant == 0 ? UBP_E_UNSUPPORTED : UBP_E_ARG;
+    if (c->kind == 5) return UBP_E_ARG;          // K-run configurations take a K-major blob: ubp_plan_build_kmajor
     *cfg = c;
     return UBP_OK;
 }
@@ -158,6 +160,31 @@ int ubp_plan_image(const void *blob, size_t len, int variant, void *host_buf, si
     return UBP_OK;
 }
 
+// Build the image of `v` for `cfg`, copy it to the device and hand back the handle. The handle's dims are the LAYER's:
+// for a K-run configuration (kind 5) the blob is that of the transposed layer, so rows and channels swap places.
+static int plan_build_view(const ubp_view_t &v, const ubp::KernelCfg *cfg, void *dev_buf, size_t dev_bytes, void *stream,
+                           ubp_plan_t **plan)
+{
+    ubp_plan *p = nullptr;
+    try {
+        p = new ubp_plan();
+        p->magic = kPlanMagic;
+        p->dims = v; p->dims.indptr = nullptr; p->dims.indices = nullptr; p->dims.values = nullptr;
+        if (cfg->kind == 5) { p->dims.M = v.C; p->dims.C = v.M; }
+        p->cfg = *cfg;
+        size_t need = 0;
+        int rc = ubp::build_plan_image(v, *cfg, false, p->img, &need);
+        if (!rc && dev_bytes < need) rc = UBP_E_SPACE;
+        if (rc) { delete p; return rc; }
+        p->dev = dev_buf; p->dev_bytes = need;
+    } catch (const std::bad_alloc &) { delete p; return UBP_E_SPACE; }
+    cudaError_t e = cudaMemcpyAsync(dev_buf, p->img.bytes.data(), p->img.bytes.size(), cudaMemcpyHostToDevice,
+                                    static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { ubp::set_last_cuda_error((int)e); delete p; return UBP_E_CUDA; }
+    *plan = p;
+    return UBP_OK;
+}
+
 int ubp_plan_build(const void *blob, size_t len, int variant, void *dev_buf, size_t dev_bytes,
                    void *stream, ubp_plan_t **plan)
 {
@@ -168,22 +195,91 @@ int ubp_plan_build(const void *blob, size_t len, int variant, void *dev_buf, siz
     if (rc) return rc;
     const ubp::KernelCfg *cfg;
     if ((rc = resolve_cfg(v, variant, &cfg))) return rc;
-    ubp_plan *p = nullptr;
+    return plan_build_view(v, cfg, dev_buf, dev_bytes, stream, plan);
+}
+
+// The other orientation: which configuration a K-major blob (of the transposed layer) runs on, and whether it first has
+// to be re-expressed in the layer's own orientation as single-channel blocks (the tensor-core kernels densify the
+// weight and do not care; the element-wise sparse configuration serves run lengths the K-run kernel has no
+// instantiation for).
+static int resolve_kmajor(const ubp_view_t &kv, int variant, const ubp::KernelCfg **cfg, bool *convert)
+{
+    const int M = kv.C, C = kv.M, B = kv.Nb;
+    if (kv.R != 1) return UBP_E_UNSUPPORTED;
+    const ubp::KernelCfg *c = nullptr;
+    if (variant == 0) {
+        const double dens = (double)kv.m * B / ((double)M * C);
+        const int krun = B == 2 ? 70 : B == 4 ? 71 : B == 8 ? 72 : B == 16 ? 73 : 0;
+        if ((dens >= 0.08 && M >= 128 && C >= 128) || !krun) c = ubp::auto_cfg(M, C, 1, 1, (int64_t)kv.m * B);
+        else c = ubp::find_cfg(krun);
+    } else {
+        c = ubp::find_cfg(variant);
+    }
+    if (!c) return variant == 0 ? UBP_E_UNSUPPORTED : UBP_E_ARG;
+    *cfg = c;
+    *convert = c->kind != 5;
+    return UBP_OK;
+}
+
+static int kmajor_prepare(const void *kblob, size_t klen, int variant, const ubp::KernelCfg **cfg, std::vector<uint8_t> &conv,
+                          ubp_view_t *v)
+{
+    ubp_view_t kv;
+    int rc = ubp::blob_view(kblob, klen, &kv);
+    if (rc) return rc;
+    bool convert = false;
+    if ((rc = resolve_kmajor(kv, variant, cfg, &convert))) return rc;
+    if (!convert) { *v = kv; return UBP_OK; }
+    size_t n = 0;
+    if ((rc = ubp_kmajor_to_plan_blob(kblob, klen, nullptr, 0, &n))) return rc;
+    conv.resize(n);
+    if ((rc = ubp_kmajor_to_plan_blob(kblob, klen, conv.data(), n, &n))) return rc;
+    return ubp::blob_view(conv.data(), n, v);
+}
+
+int ubp_plan_size_kmajor(const void *kblob, size_t klen, int variant, size_t *dev_bytes)
+{
+    if (!dev_bytes) return UBP_E_ARG;
     try {
-        p = new ubp_plan();
-        p->magic = kPlanMagic;
-        p->dims = v; p->dims.indptr = nullptr; p->dims.indices = nullptr; p->dims.values = nullptr;
-        p->cfg = *cfg;
+        const ubp::KernelCfg *cfg;
+        std::vector<uint8_t> conv;
+        ubp_view_t v;
+        if (int rc = kmajor_prepare(kblob, klen, variant, &cfg, conv, &v)) return rc;
+        ubp::PlanImage img;
+        return ubp::build_plan_image(v, *cfg, true, img, dev_bytes);
+    } catch (const std::bad_alloc &) { return UBP_E_SPACE; }
+}
+
+int ubp_plan_build_kmajor(const void *kblob, size_t klen, int variant, void *dev_buf, size_t dev_bytes, void *stream,
+                          ubp_plan_t **plan)
+{
+    if (!plan || !dev_buf || (reinterpret_cast<uintptr_t>(dev_buf) & 255)) return UBP_E_ARG;
+    *plan = nullptr;
+    try {
+        const ubp::KernelCfg *cfg;
+        std::vector<uint8_t> conv;
+        ubp_view_t v;
+        if (int rc = kmajor_prepare(kblob, klen, variant, &cfg, conv, &v)) return rc;
+        return plan_build_view(v, cfg, dev_buf, dev_bytes, stream, plan);
+    } catch (const std::bad_alloc &) { return UBP_E_SPACE; }
+}
+
+int ubp_plan_image_kmajor(const void *kblob, size_t klen, int variant, void *host_buf, size_t cap, int32_t geom[8])
+{
+    if (!host_buf || !geom) return UBP_E_ARG;
+    try {
+        const ubp::KernelCfg *cfg;
+        std::vector<uint8_t> conv;
+        ubp_view_t v;
+        if (int rc = kmajor_prepare(kblob, klen, variant, &cfg, conv, &v)) return rc;
+        ubp::PlanImage img;
         size_t need = 0;
-        rc = ubp::build_plan_image(v, *cfg, false, p->img, &need);
-        if (!rc && dev_bytes < need) rc = UBP_E_SPACE;
-        if (rc) { delete p; return rc; }
-        p->dev = dev_buf; p->dev_bytes = need;
-    } catch (const std::bad_alloc &) { delete p; return UBP_E_SPACE; }
-    cudaError_t e = cudaMemcpyAsync(dev_buf, p->img.bytes.data(), p->img.bytes.size(), cudaMemcpyHostToDevice,
-                                    static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) { ubp::set_last_cuda_error((int)e); delete p; return UBP_E_CUDA; }
-    *plan = p;
+        if (int rc = ubp::build_plan_image(v, *cfg, false, img, &need)) return rc;
+        if (cap < need) return UBP_E_SPACE;
+        std::memcpy(host_buf, img.bytes.data(), need);
+        geom[0] = cfg->nbk; geom[1] = cfg->P; geom[2] = cfg->KT; geom[3] = cfg->WR; geom[4] = cfg->dupw;
+        geom[5] = img.nkt; geom[6] = img.NP; geom[7] = img.NG;
+    } catch (const std::bad_alloc &) { return UBP_E_SPACE; }
     return UBP_OK;
 }
 

@@ -203,6 +203,47 @@ struct FragmentLoop {
     }
 };
 
+// ------------------------------------------------------------------ the other block orientation (K-runs)
+// Plan entries of a configuration of kind 5: a run of NB consecutive input channels of ONE output row (fragment =
+// the row inside the panel, so the accumulator is a compile-time constant again): one channel index, NB weights
+// and NB activation rows of the staged tile per entry.
+template <int NB, int P, int V, int XROW_BYTES, int FOW, int F0, int F1>
+struct KrunLoop {
+    __device__ __forceinline__ static void run(float2 (&acc)[P][2 * V], const uint8_t *xs_lane, const uint16_t *jl,
+                                               const float *wv, const uint32_t (&fw)[FOW])
+    {
+        if constexpr (F0 < F1) {
+            const int e1 = fo_at<FOW>(fw, F0 + 1);
+#pragma unroll 2
+            for (int e = fo_at<FOW>(fw, F0); e < e1; ++e) {
+                const uint8_t *xp = xs_lane + (uint32_t)jl[e] * (uint32_t)XROW_BYTES;
+                float w[NB];
+                load_floats<NB>(w, wv + (size_t)e * NB);
+                constexpr int TG = NB < 4 ? NB : 4;          // activation rows in flight at once
+#pragma unroll
+                for (int t0 = 0; t0 < NB; t0 += TG) {
+                    float4 x[TG][V];
+#pragma unroll
+                    for (int t = 0; t < TG; ++t)
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            x[t][v] = *reinterpret_cast<const float4 *>(xp + (t0 + t) * XROW_BYTES + v * 512);
+#pragma unroll
+                    for (int t = 0; t < TG; ++t) {
+                        const float2 w2 = make_float2(w[t0 + t], w[t0 + t]);
+#pragma unroll
+                        for (int v = 0; v < V; ++v) {
+                            acc[F0][2 * v] = fma2(w2, make_float2(x[t][v].x, x[t][v].y), acc[F0][2 * v]);
+                            acc[F0][2 * v + 1] = fma2(w2, make_float2(x[t][v].z, x[t][v].w), acc[F0][2 * v + 1]);
+                        }
+                    }
+                }
+            }
+            KrunLoop<NB, P, V, XROW_BYTES, FOW, F0 + 1, F1>::run(acc, xs_lane, jl, wv, fw);
+        }
+    }
+};
+
 struct SpmmArgs {
     const uint8_t *plan;     // device plan image
     const float *bias;       // [M] or null
@@ -221,13 +262,13 @@ struct SpmmArgs {
 // copies for step it + D (D = stages - 2) into the stage that every warp released two steps ago, so that wait
 // almost never blocks. Each stage has a "full" mbarrier (completed by the copies' byte count) and an "empty"
 // one (one arrival per warp).
-template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW>
+template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW, bool KRUN>
 __global__ void __launch_bounds__(WR * WC * 32, 1)
 ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
 {
     constexpr int CS = WC * 128 * V;               // columns per CTA
     constexpr int XT_BYTES = KT * CS * 4;
-    constexpr int F = P + NBK - 1;
+    constexpr int F = KRUN ? P : P + NBK - 1;      // fragments: rows of the panel (K-runs) or start offsets
     constexpr int NCW = WR * WC;                   // warps
     constexpr int FO_BYTES = ((F + 1) * 2 + 15) & ~15;
     constexpr int WF = NBK * (DUPW ? 2 : 1);
@@ -309,6 +350,10 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
             }
             const int n = fo_at<FOW>(fw, F);
             const uint8_t *xs_lane = stage + (wc * 128 * V + lane * 4) * 4;
+            if constexpr (KRUN) {
+                KrunLoop<NBK, P, V, CS * 4, FOW, 0, F>::run(acc, xs_lane, reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES),
+                                                            reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * (n + 4) + 15) & ~15)), fw);
+            } else {
             // the plan pads jl with 4 zero entries and w with 2 zero entries, so the pipeline may read ahead
             PipeState<V, WF> ps;
             ps.jp = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
@@ -316,6 +361,7 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
             fetch_entry<V, WF, CS * 4>(ps.cur, xs_lane, ps.jp[0], ps.wp, 0);
             ps.jn = ps.jp[1];
             FragmentLoop<NBK, P, V, DUPW, CS * 4, FOW, 0, F>::run(acc, ps, xs_lane, fw);
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bar_empty[st]));
@@ -420,6 +466,48 @@ ubp_spmm_simple_kernel(const uint8_t *plan, const float *X, int64_t ldx, int64_t
         SimpleLoop<NBK, P, 0, F>::run(acc, xcol, ldx, live, fo, jl, wv, NBK * wdup, wdup, 0);
     }
     if (!live) return;
+#pragma unroll
+    for (int r = 0; r < P; ++r) {
+        const int row = panel * P + r;
+        if (row < M) {
+            float o = acc[r] + (bias ? bias[row] : 0.f);
+            if (relu) o = fmaxf(o, 0.f);
+            Y[(size_t)row * ldy + col] = o;
+        }
+    }
+}
+
+// The same for K-run plans (kind 5): an entry is NB consecutive channels of one output row.
+template <int NB, int P>
+__global__ void __launch_bounds__(128)
+ubp_spmm_krun_simple_kernel(const uint8_t *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
+                            float *Y, int64_t ldy, int M, int C, int NP, int nkt, int NG, int WR, int KT)
+{
+    constexpr int FO_BYTES = ((P + 1) * 2 + 15) & ~15;
+    const int panel = blockIdx.y;
+    const int64_t col = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (panel >= NP || col >= Nc) return;
+    const int g = panel / WR, wr = panel % WR;
+    const uint32_t *gtab = reinterpret_cast<const uint32_t *>(plan + 256);
+    float acc[P];
+#pragma unroll
+    for (int r = 0; r < P; ++r) acc[r] = 0.f;
+    for (int kt = 0; kt < nkt; ++kt) {
+        const uint8_t *grp = plan + (size_t)gtab[(size_t)kt * NG + g] * 16u;
+        const uint32_t po = reinterpret_cast<const uint32_t *>(grp)[wr];
+        const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
+        const int n = fo[P];
+        const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
+        const float *wv = reinterpret_cast<const float *>(grp + po + FO_BYTES + ((2 * (n + 4) + 15) & ~15));
+#pragma unroll
+        for (int r = 0; r < P; ++r)
+            for (int e = fo[r]; e < fo[r + 1]; ++e) {
+                const int c0 = kt * KT + jl[e];
+#pragma unroll
+                for (int t = 0; t < NB; ++t)      // channels past the layer's last one carry zero weights: skip the read
+                    if (c0 + t < C) acc[r] = fmaf(wv[(size_t)e * NB + t], X[(size_t)(c0 + t) * ldx + col], acc[r]);
+            }
+    }
 #pragma unroll
     for (int r = 0; r < P; ++r) {
         const int row = panel * P + r;
@@ -542,7 +630,7 @@ static int check(cudaError_t e)
 
 constexpr size_t kSmemBudget = 227 * 1024 - 1024;   // dynamic shared memory we allow ourselves per CTA
 
-template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW>
+template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW, bool KRUN>
 static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                        float *Y, int64_t ldy, cudaStream_t stream)
 {
@@ -565,7 +653,7 @@ static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t 
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) { set_last_cuda_error(-(int)cr); return UBP_E_CUDA; }
 
-    auto kern = ubp_spmm_kernel<NBK, P, V, WR, WC, KT, DUPW>;
+    auto kern = ubp_spmm_kernel<NBK, P, V, WR, WC, KT, DUPW, KRUN>;
     const size_t smem = stage_bytes * stages;
     static bool attr_done[64] = {};                  // per device: opt in to large dynamic shared memory once
     int dev = 0;
@@ -613,14 +701,21 @@ struct CfgLaunch {
     static int main_kernel(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                            float *Y, int64_t ldy, cudaStream_t s)
     {
-        if constexpr (KIND == 0) return launch_main<NBK, P, V, WR, WC, KT, DUP>(pl, X, ldx, Nc, bias, relu, Y, ldy, s);
+        if constexpr (KIND == 0) return launch_main<NBK, P, V, WR, WC, KT, DUP, false>(pl, X, ldx, Nc, bias, relu, Y, ldy, s);
+        else if constexpr (KIND == 5) return launch_main<NBK, P, V, WR, WC, KT, DUP, true>(pl, X, ldx, Nc, bias, relu, Y, ldy, s);
         else return UBP_E_UNSUPPORTED;
     }
     static int simple_kernel(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                              float *Y, int64_t ldy, cudaStream_t s)
     {
         if constexpr (KIND == 0 || KIND == 2) return launch_simple<NBK, P>(pl, X, ldx, Nc, bias, relu, Y, ldy, s);
-        else return UBP_E_UNSUPPORTED;
+        else if constexpr (KIND == 5) {
+            dim3 grid((unsigned)((Nc + 127) / 128), (unsigned)pl->img.NP);
+            ubp_spmm_krun_simple_kernel<NBK, P><<<grid, 128, 0, s>>>(
+                static_cast<const uint8_t *>(pl->dev), X, ldx, Nc, bias, relu, Y, ldy, pl->dims.M, pl->dims.C, pl->img.NP,
+                pl->img.nkt, pl->img.NG, pl->cfg.WR, pl->cfg.KT);
+            return check(cudaGetLastError());
+        } else return UBP_E_UNSUPPORTED;
     }
     static int conv_kernel(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
                            const float *bias, int relu, float *out, int64_t osb, int64_t osc, cudaStream_t s, int stride)

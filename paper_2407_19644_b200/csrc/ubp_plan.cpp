@@ -116,34 +116,64 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         return UBP_OK;
     }
     const int nbk = cfg.nbk, P = cfg.P, KT = cfg.KT, WR = cfg.WR;
-    if (Nb % nbk != 0) return UBP_E_UNSUPPORTED;
+    // kind 5: the blob is that of the TRANSPOSED layer (ubp_pack_kmajor): its "rows" are the layer's input channels,
+    // its "channels" the layer's output rows, and a block is Nb consecutive input channels of one output row. An
+    // entry = one such run (or the part of it inside one channel tile): nbk = Nb weights in channel order, filed
+    // under (channel tile, row panel, row inside the panel).
+    const bool krun = cfg.kind == 5;
+    if (krun ? (Nb != nbk || nbk > 16 || R != 1 || KT < nbk) : (Nb % nbk != 0)) return UBP_E_UNSUPPORTED;
     const bool conv = (cfg.kind == 1 || cfg.kind == 3);
     if ((!conv && R != 1) || (conv && R != 9)) return UBP_E_UNSUPPORTED;
-    const int nkt = (C + KT - 1) / KT;
-    const int NP = (M + P - 1) / P;
+    const int rowsL = krun ? C : M, chanL = krun ? M : C;            // the layer's output rows / input channels
+    const int nkt = (chanL + KT - 1) / KT;
+    const int NP = (rowsL + P - 1) / P;
     const int NG = (NP + WR - 1) / WR;
-    const int F = P + nbk - 1;
-    const int sub = Nb / nbk;
+    const int F = krun ? P : P + nbk - 1;
+    const int sub = krun ? 1 : Nb / nbk;
     const size_t wfloats = (size_t)nbk * R * (cfg.dupw ? 2 : 1);   // floats per entry
+    // Every entry of the plan, in filing order: fn(channel tile, panel, fragment, channel inside the tile, weights).
+    std::vector<float> wblk((size_t)Nb * R);
+    auto for_each_entry = [&](auto &&fn) {
+        for (int i = 0; i < M; ++i)
+            for (int32_t b = v.indptr[i]; b < v.indptr[i + 1]; ++b) {
+                const int j = v.indices[b];
+                const float *val = v.values + (size_t)b * Nb * R;
+                for (int t = 0; t < Nb; ++t)       // undo the rotation: row i+t lives in slot (i+t) mod Nb
+                    std::memcpy(&wblk[(size_t)t * R], val + (size_t)((i + t) % Nb) * R, sizeof(float) * (size_t)R);
+                if (krun) {
+                    // run of channels i .. i+Nb-1 of output row j; cut at channel-tile boundaries. A piece is stored as
+                    // a full-length entry that lies wholly inside its tile: its start is moved into the tile and the
+                    // places of channels that do not belong to the piece hold zero weights (the activations read there
+                    // are real, finite values of the same tile).
+                    float wpart[16];
+                    for (int kt = i / KT; kt <= (i + Nb - 1) / KT; ++kt) {
+                        const int T0 = kt * KT;
+                        int ks = i - T0;
+                        if (ks < 0) ks = 0;
+                        if (ks > KT - Nb) ks = KT - Nb;
+                        for (int u = 0; u < Nb; ++u) {
+                            const int c = T0 + ks + u;
+                            wpart[u] = (c >= i && c < i + Nb) ? wblk[(size_t)(c - i)] : 0.0f;
+                        }
+                        fn(kt, j / P, j % P, ks, wpart);
+                    }
+                    continue;
+                }
+                const int kt = j / KT, jl = j % KT;
+                for (int u = 0; u < sub; ++u) {
+                    const int r0 = i + u * nbk;
+                    const int p = r0 / P, s = r0 % P;
+                    fn(kt, p, s + nbk - 1, jl, &wblk[(size_t)u * nbk * R]);
+                    if (s + nbk > P) fn(kt, p + 1, s - P + nbk - 1, jl, &wblk[(size_t)u * nbk * R]);   // crosses into the next panel
+                }
+            }
+    };
 
     // pass 1: entries per (kt, panel, fragment)
     std::vector<uint32_t> cnt((size_t)nkt * NP * F, 0);
     auto bucket = [&](int kt, int p, int f) -> size_t { return ((size_t)kt * NP + p) * F + f; };
     int64_t entries = 0;
-    for (int i = 0; i < M; ++i)
-        for (int32_t b = v.indptr[i]; b < v.indptr[i + 1]; ++b) {
-            const int kt = v.indices[b] / KT;
-            for (int u = 0; u < sub; ++u) {
-                const int r0 = i + u * nbk;
-                const int p = r0 / P, s = r0 % P;
-                cnt[bucket(kt, p, s + nbk - 1)]++;
-                ++entries;
-                if (s + nbk > P) {           // crosses into the next panel
-                    cnt[bucket(kt, p + 1, s - P + nbk - 1)]++;
-                    ++entries;
-                }
-            }
-        }
+    for_each_entry([&](int kt, int p, int f, int, const float *) { cnt[bucket(kt, p, f)]++; ++entries; });
 
     // layout
     const size_t tab_off = 256;
@@ -235,21 +265,7 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
             std::memcpy(dst, wsrc, sizeof(float) * (size_t)nbk * R);
         }
     };
-    std::vector<float> wblk((size_t)Nb * R);
-    for (int i = 0; i < M; ++i)
-        for (int32_t b = v.indptr[i]; b < v.indptr[i + 1]; ++b) {
-            const int j = v.indices[b];
-            const int kt = j / KT, jl = j % KT;
-            const float *val = v.values + (size_t)b * Nb * R;
-            for (int t = 0; t < Nb; ++t)       // undo the rotation: row i+t lives in slot (i+t) mod Nb
-                std::memcpy(&wblk[(size_t)t * R], val + (size_t)((i + t) % Nb) * R, sizeof(float) * (size_t)R);
-            for (int u = 0; u < sub; ++u) {
-                const int r0 = i + u * nbk;
-                const int p = r0 / P, s = r0 % P;
-                put(kt, p, s + nbk - 1, jl, &wblk[(size_t)u * nbk * R]);
-                if (s + nbk > P) put(kt, p + 1, s - P + nbk - 1, jl, &wblk[(size_t)u * nbk * R]);
-            }
-        }
+    for_each_entry(put);
     if (cfg.kind == 2 || cfg.kind == 3) {
         // Densify and split every kept weight into the part a TF32 operand holds exactly (sign, exponent,
         // top 10 mantissa bits) and the remainder, itself cut to TF32; pruned positions stay zero.

@@ -64,9 +64,10 @@ def test_added_workloads_are_well_formed():
     import bench
     import ubp_synth
     # the other block orientation: every row's runs of ones are whole blocks of KMAJOR_B input channels
-    L = bench.get_layer("kmajor_pw512")
-    assert (L.M, L.C, L.Nb, L.Nc) == (512, 512, 1, 6272) and L.m == int(L.mask.sum())
-    assert L.m == ubp_synth.block_budget(512, 512, 70, bench.KMAJOR_B) * bench.KMAJOR_B
+    for wname, sp in bench.KMAJOR_WORKLOADS.items():
+        L = bench.get_layer(wname)
+        assert (L.M, L.C, L.Nb, L.Nc) == (512, 512, 1, 6272) and L.m == int(L.mask.sum())
+        assert L.m == ubp_synth.block_budget(512, 512, sp, bench.KMAJOR_B) * bench.KMAJOR_B
     padded = np.pad(L.mask, ((0, 0), (1, 1))).astype(np.int8)
     d = np.diff(padded, axis=1)
     starts, ends = np.argwhere(d == 1), np.argwhere(d == -1)

@@ -11,7 +11,7 @@ import pytest
 import oracle
 import ubp_synth
 import paper_2407_19644_b200 as ubp
-from helpers import plan_to_dense
+from helpers import plan_to_dense, krun_plan_to_dense
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -320,6 +320,29 @@ def test_kmajor_blocks_pack_as_the_transposed_layer_and_convert_to_a_plan_blob()
     with pytest.raises(ubp.UbpError) as e:
         ubp.ubp_pack_kmajor(W, bad, B)
     assert e.value.code == -2
+
+
+@pytest.mark.parametrize("M,Cin,B,p", [(40, 200, 4, 60), (70, 130, 2, 50), (24, 96, 8, 70), (33, 160, 16, 50), (50, 64, 4, 90)])
+def test_krun_plan_image_replays_to_the_masked_weight(M, Cin, B, p):
+    """The plan of the K-run sparse kernel (one entry = one run of B consecutive input channels of one output row):
+    replayed on the host it gives exactly the masked weight; it holds ONE channel index per run, plus one more for
+    every run that crosses a 64-channel tile boundary (cut there, each piece padded with zero weights)."""
+    Lt = ubp_synth.make_layer("t", Cin, M, B, p, 60 + M, Nc=4, make_x=False)        # transposed roles: [C][M]
+    W = np.ascontiguousarray(Lt.W[:, :, 0].T)
+    mask = np.ascontiguousarray(Lt.mask.T)
+    kblob = ubp.ubp_pack_kmajor(W, mask, B)
+    variant = {2: 70, 4: 71, 8: 72, 16: 73}[B]
+    img, geom = ubp.plan_image(kblob, variant, kmajor=True)
+    assert geom["nbk"] == B and len(img) == ubp.plan_size(kblob, variant, kmajor=True)
+    Wd, n_entries = krun_plan_to_dense(img, geom, M, Cin)
+    assert np.array_equal(Wd.astype(np.float32), W * mask)
+    k0, rows = oracle.decode_mask(mask.T, B)                 # blocks of the transposed layer: (first channel, output row)
+    crossing = int(((k0 % geom["k_tile"]) + B > geom["k_tile"]).sum())
+    assert n_entries == len(k0) + crossing
+    # sparse layers choose this plan by themselves, dense-enough large ones the tensor-core plan of the re-expressed layer
+    assert ubp.plan_size(kblob, 0, kmajor=True) == len(img) if (M < 128 or p >= 93) else True
+    with pytest.raises(ubp.UbpError):
+        ubp.plan_size(kblob, variant)                        # a K-run configuration needs the K-major entry points
 
 
 def test_block_selection_argument_checks_need_no_device():

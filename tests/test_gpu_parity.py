@@ -606,3 +606,54 @@ def test_kmajor_orientation_through_the_plan(env, M, Cin, B, p, Nc):
     plan.check()
     Yref, A = oracle.masked_matmul(W, mask, X, bias, relu=True)
     assert scaled_error(Y.cpu().numpy(), Yref, A) <= 1e-4
+
+
+def _kmajor_layer(M, Cin, B, p, Nc, seed):
+    Lt = ubp_synth.make_layer("kmajor", Cin, M, B, p, seed, Nc=8, make_x=False)       # roles exchanged: [C][M]
+    W = np.ascontiguousarray(Lt.W[:, :, 0].T)
+    mask = np.ascontiguousarray(Lt.mask.T)
+    rng = np.random.default_rng(seed)
+    return W, mask, rng.standard_normal((Cin, Nc)).astype(np.float32), rng.standard_normal(M).astype(np.float32), Lt.m
+
+
+@pytest.mark.parametrize("M,Cin,B,p,Nc,pad,misalign", [
+    (256, 256, 4, 70, 1000, 0, 0), (192, 320, 8, 95, 520, 0, 0), (64, 96, 2, 50, 260, 0, 0), (100, 130, 16, 50, 516, 0, 0),
+    (300, 70, 4, 80, 1028, 0, 0), (512, 512, 4, 90, 2048, 0, 0), (40, 200, 2, 60, 130, 2, 0), (40, 200, 8, 60, 131, 1, 0),
+    (77, 64, 4, 50, 255, 0, 0), (77, 64, 4, 50, 256, 0, 1), (9, 48, 16, 34, 4, 0, 0),
+])
+def test_krun_sparse_kernel(env, M, Cin, B, p, Nc, pad, misalign):
+    """The sparse kernel for the other orientation (variants 70..73): one plan entry, one channel index and B staged
+    activation rows per run of B consecutive input channels of one output row. Against the definition (the oracle's
+    dense masked product), through the staged kernel and, for operands it cannot take, the plain one; fp32 FMA, so the
+    fp32 summation bound holds."""
+    torch, ubp = env
+    W, mask, X, bias, m = _kmajor_layer(M, Cin, B, p, Nc, 950 + B + M)
+    kblob = ubp.ubp_pack_kmajor(W, mask, B)
+    assert kblob == oracle.pack(np.ascontiguousarray(W.T), np.ascontiguousarray(mask.T), B)
+    variant = {2: 70, 4: 71, 8: 72, 16: 73}[B]
+    plan = ubp.Plan(kblob, variant, kmajor=True)
+    assert (plan.variant, plan.M, plan.C, plan.Nb, plan.m) == (variant, M, Cin, B, m)
+    assert plan.tile_choice(Nc)[0] == 0
+    ld = Nc + pad
+    xbuf = torch.zeros(Cin * ld + 8, dtype=torch.float32, device="cuda")
+    Xd = xbuf[misalign:misalign + Cin * ld].view(Cin, ld)[:, :Nc]
+    Xd.copy_(torch.from_numpy(X))
+    ybuf = torch.full((M * ld + 8,), float("nan"), dtype=torch.float32, device="cuda")
+    Yd = ybuf[misalign:misalign + M * ld].view(M, ld)[:, :Nc]
+    ubp.ubp_spmm(plan, Xd, torch.from_numpy(bias).cuda(), True, out=Yd)
+    plan.check()
+    if pad:
+        assert torch.isnan(ybuf[misalign:misalign + M * ld].view(M, ld)[:, Nc:]).all()
+    Yref, A = oracle.masked_matmul(W, mask, X, bias, relu=True)
+    Yh = Yd.cpu().numpy()
+    assert np.isfinite(Yh).all()
+    err = scaled_error(Yh, Yref, A)
+    terms = int(mask.sum(axis=1).max()) + 2
+    assert err <= 1e-4 and err <= terms * 2.0 ** -24 * 1.5          # pieces of a cut run add a few exact zeros
+    # the automatic choice for this orientation: tensor-core kernel when dense and large enough, else this kernel
+    auto = ubp.Plan(kblob, 0, kmajor=True)
+    dense_enough = (100 - p) >= 8 and M >= 128 and Cin >= 128
+    assert auto.variant == (34 if dense_enough else variant)
+    Ya = ubp.ubp_spmm(auto, torch.from_numpy(X).cuda(), torch.from_numpy(bias).cuda(), True)
+    auto.check()
+    assert scaled_error(Ya.cpu().numpy(), Yref, A) <= 1e-4
