@@ -115,8 +115,8 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
 
 def compulsory_bytes(L) -> int:
     """Activations read once + outputs written once + packed weights/indices + bias."""
-    x = L.C * L.Nc * 4
-    y = L.M * L.Nc * 4
+    x = L.C * (L.Nc_out if L.R == 1 else L.Nc) * 4       # a strided 1x1 reads only the pixels it keeps
+    y = L.M * L.Nc_out * 4
     w = L.m * L.Nb * L.R * 4 + L.m * 4 + (L.M + 1) * 4 + (L.M * 4 if L.bias is not None else 0)
     return x + y + w
 
@@ -441,17 +441,25 @@ HEADLINE_VARIANTS = [32, 14]
 
 
 def build_chained(ubp, torch, layers, variant):
-    """Runners for layers that feed one another: layer i + 1 reads the output tensor of layer i."""
-    plans, runs, keep = [], [], []
-    x = torch.from_numpy(layers[0].X).cuda()
-    for L in layers:
+    """Runners for layers that feed one another: a layer reads the output tensor of layer L.src (the block input for
+    -1; by default its predecessor); strided layers produce the smaller planes."""
+    plans, runs, keep, outs = [], [], [], []
+    x0 = torch.from_numpy(layers[0].X).cuda()
+    for li, L in enumerate(layers):
+        src = li - 1 if L.src is None else L.src
+        x = x0 if src < 0 else outs[src]
         plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb), variant)
         bias = torch.from_numpy(L.bias).cuda() if L.bias is not None else None
-        y = torch.empty((L.M, L.B, L.H, L.Wd), dtype=torch.float32, device="cuda")
+        Ho, Wo = (L.H - 1) // L.stride + 1, (L.Wd - 1) // L.stride + 1
+        y = torch.empty((L.M, L.B, Ho, Wo), dtype=torch.float32, device="cuda")
         fn = ubp.ubp_conv3x3_implicit if L.R == 9 else ubp.ubp_conv1x1
-        runs.append(lambda fn=fn, plan=plan, x=x, bias=bias, relu=L.relu, y=y: fn(plan, x, bias, relu, out=y))
-        plans.append(plan); keep.append((x, y, bias))
-        x = y
+        kw = {}
+        if L.stride != 1:
+            kw["stride"] = L.stride
+            if L.R == 1:
+                kw["scratch"] = torch.empty(L.C * L.B * Ho * Wo, dtype=torch.float32, device="cuda")
+        runs.append(lambda fn=fn, plan=plan, x=x, bias=bias, relu=L.relu, y=y, kw=kw: fn(plan, x, bias, relu, out=y, **kw))
+        plans.append(plan); keep.append((x, y, bias, kw)); outs.append(y)
     return plans, runs, keep
 
 
@@ -463,7 +471,7 @@ def run_chain(args, torch, ubp, rank, world, dist, cfg="mbv1_chain"):
     layers = ubp_synth.config_layers(cfg, index=rank)
     hbm_gbs, peak_src = measured_peaks()
     runs, plans, keep = [], [], []
-    if cfg == "r50_bottleneck":
+    if cfg in ("r50_bottleneck", "r50_downsample"):
         plans, runs, keep = build_chained(ubp, torch, layers, args.variant)
     else:
         for L in layers:
@@ -512,7 +520,7 @@ def run_chain(args, torch, ubp, rank, world, dist, cfg="mbv1_chain"):
         "roofline": {"bound": "mixed (per layer: see layers)", "roofline_us": roof_total_us,
                      "frac_of_roofline_time": roof_total_us / (step_ms * 1e3),
                      "peak_source": f"FP32 74.45 TFLOP/s derived; HBM {hbm_gbs} GB/s {peak_src}"},
-        "layers": [{"name": L.name, "M": L.M, "K": L.C * L.R, "Nc": L.B * L.H * L.Wd, "variant": p.variant, "us_flushed": us,
+        "layers": [{"name": L.name, "M": L.M, "K": L.C * L.R, "Nc": L.Nc_out, "stride": L.stride, "variant": p.variant, "us_flushed": us,
                     "roofline_us": max(r), "bound": "alu" if r[0] >= r[1] else "hbm", "frac_flushed": max(r) / us}
                    for L, p, us, r in zip(layers, plans, per_layer, roofs)],
         "clocks": clocks, "gpu_launches": len(layers) * args.steps,
@@ -793,7 +801,7 @@ def main():
         raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s): start bench.py with "
                          f"torch.distributed.run --nproc-per-node {args.gpus}, or with no launcher at all")
     name = args.workload
-    if name in ("mbv1_chain", "r50_bottleneck"):
+    if name in ("mbv1_chain", "r50_bottleneck", "r50_downsample"):
         if args.impl == "reference":
             raise SystemExit("--impl reference times single layers; pick a layer workload")
         import torch

@@ -170,7 +170,8 @@ int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info);
 /* ubp_plan_tile_choice: which kernel a launch of this plan over `Nc` columns uses on the current device when the
  * operands qualify for the fast path (for 3x3: input and output as one [channel][batch, y, x] matrix each), and
  * its output tile. `image_width` is the width of the input planes for a 3x3 plan (Nc = batch * height * width),
- * ignored for 1x1. *kernel: 0 = sparse FP32 kernel (Section 4.2's output-stationary product on the CUDA cores),
+ * ignored for 1x1; a negative value asks about a strided 3x3 launch (Nc = batch * Ho * Wo), which the one-CTA kernel
+ * serves. *kernel: 0 = sparse FP32 kernel (Section 4.2's output-stationary product on the CUDA cores),
  * 1 = tensor-core kernel with one CTA per tile, 2 = tensor-core kernel with a CTA pair per tile, 3 = the comparison
  * kernels that walk the canonical arrays in the paper's own dataflow (variants 60 and 61; tile_rows is 0). Host only;
  * enqueues nothing. Not part of the paper's method: it exists so that measurements and tests can name what ran. */
@@ -249,8 +250,11 @@ int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, 
  * Ho = (H-1)/stride + 1, Wo = (W-1)/stride + 1; strides of `out` are in elements of those planes.
  * stride == 1 forwards to the call above.
  * ubp_conv3x3_strided: 3x3, zero padding 1: out[b][o][yo][xo] = act(bias[o] + sum W[o][c][3r+s] *
- *   in[b][c][yo*stride + r - 1][xo*stride + s - 1]). For stride > 1 every output pixel is computed by one lane that
- *   reads its taps in place (correct for any layout, far from the roofline; the implicit-GEMM kernels are stride 1).
+ *   in[b][c][yo*stride + r - 1][xo*stride + s - 1]). For stride > 1 a tensor-core plan whose output is one
+ *   [channel][batch, yo, xo] matrix with 16-byte aligned rows runs the one-CTA implicit-GEMM kernel (its loader warps
+ *   gather every tap pixel by pixel, so the stride is only a change of the column -> pixel map); other plans and
+ *   layouts are computed by one lane per output pixel that reads its taps in place (correct for any layout, far from
+ *   the roofline).
  * ubp_conv1x1_strided: out[b][o][yo][xo] = act(bias[o] + sum W[o][c] * in[b][c][yo*stride][xo*stride]). For
  *   stride > 1 the pixels read are first gathered into `scratch` (device, 16-byte aligned, at least
  *   ubp_conv1x1_strided_scratch(C, B, H, W, stride) bytes, channel-major [C][B][Ho][Wo]) by one extra kernel, then the

@@ -261,8 +261,9 @@ class Plan:
 
     def tile_choice(self, Nc: int, image_width: int = 0):
         """(kernel, tile_rows, tile_cols) of a fast-path launch over Nc columns on the plan's device (3x3 plans:
-        Nc = batch * height * width and image_width = width): kernel 0 = sparse FP32, 1 = tensor core / one CTA
-        per tile, 2 = tensor core / CTA pair per tile."""
+        Nc = batch * height * width and image_width = width; strided 3x3: Nc = batch * Ho * Wo and image_width = -width):
+        kernel 0 = sparse FP32, 1 = tensor core / one CTA per tile, 2 = tensor core / CTA pair per tile, 3 = the
+        comparison kernels that walk the canonical arrays."""
         k, r, c = C.c_int32(), C.c_int32(), C.c_int32()
         import torch
         with torch.cuda.device(self.buffer.device):

@@ -300,12 +300,12 @@ int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info)
 int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, int *kernel, int *tile_rows, int *tile_cols)
 {
     if (!plan || plan->magic != kPlanMagic || Nc < 0 || !kernel || !tile_rows || !tile_cols) return UBP_E_ARG;
-    if (plan->dims.R == 9 && image_width <= 0) return UBP_E_ARG;
+    if (plan->dims.R == 9 && image_width == 0) return UBP_E_ARG;
     const ubp::KernelCfg &c = plan->cfg;
     if (c.kind == 2 || c.kind == 3) {
         int sms = 148, devid = 0;
         if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
-        ubp::tc_choose(plan->dims.M, plan->dims.C * plan->dims.R, Nc, c.kind == 3 ? image_width : 0, ubp::cfg_bf16(c) ? 1 : 0, sms, kernel, tile_rows,
+        ubp::tc_choose(plan->dims.M, plan->dims.C * plan->dims.R, Nc, c.kind == 3 ? (image_width > 0 ? image_width : -1) : 0, ubp::cfg_bf16(c) ? 1 : 0, sms, kernel, tile_rows,
                        tile_cols);
     } else if (c.kind == 4) {
         *kernel = 3; *tile_rows = 0; *tile_cols = 512;       // row ranges are chosen per launch; 128 threads x 4 columns

@@ -95,8 +95,9 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
 int launch_spmm_tc(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                    float *Y, int64_t ldy, void *stream);
 int launch_conv3x3_tc(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
-                      const float *bias, int relu, float *out, int64_t out_ld, void *stream);
-// stride 1: tensor-core implicit GEMM when the plan and the layouts allow it; stride > 1: one lane per output pixel
+                      const float *bias, int relu, float *out, int64_t out_ld, void *stream, int stride = 1);
+// tensor-core implicit GEMM when the plan and the layouts allow it (stride 1: CTA pairs where the operands qualify;
+// stride > 1: the one-CTA kernel, whose loaders gather the taps pixel by pixel); else one lane per output pixel
 int launch_conv3x3(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
                    const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream, int stride = 1);
 int launch_subsample(const float *in, int C, int B, int H, int Wd, int64_t isb, int64_t isc, int stride, float *out,

@@ -764,11 +764,12 @@ int launch_conv3x3(const ubp_plan *pl, const float *in, int B, int H, int Wd, in
 {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const KernelCfg &c = pl->cfg;
-    const int64_t total = (int64_t)B * H * Wd;
-    // tensor-core path: needs the output as one [M][B*H*W] matrix (batch stride = plane size) with 16-byte rows
-    if (stride == 1 && c.kind == 3 && osb == (int64_t)H * Wd && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && osc % 4 == 0 &&
-        osc >= total && total < (1ll << 31))
-        return launch_conv3x3_tc(pl, in, B, H, Wd, isb, isc, bias, relu, out, osc, stream_);
+    const int64_t ohw = (int64_t)((H - 1) / stride + 1) * ((Wd - 1) / stride + 1);
+    const int64_t total = (int64_t)B * ohw;
+    // tensor-core path: needs the output as one [M][B*Ho*Wo] matrix (batch stride = plane size) with 16-byte rows
+    if (c.kind == 3 && osb == ohw && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && osc % 4 == 0 &&
+        osc >= total && total < (1ll << 31) && (int64_t)B * H * Wd < (1ll << 31))
+        return launch_conv3x3_tc(pl, in, B, H, Wd, isb, isc, bias, relu, out, osc, stream_, stride);
 #define UBP_CFG(ID, KIND, NBK, P_, V_, WR_, WC_, KT_, DUP) \
     if (c.id == ID)                                        \
         return CfgLaunch<KIND, NBK, P_, V_, WR_, WC_, KT_, (DUP != 0)>::conv_kernel(pl, in, B, H, Wd, isb, isc, bias, relu, out, osb, osc, stream, stride);

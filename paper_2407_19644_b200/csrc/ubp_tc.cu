@@ -153,9 +153,11 @@ ubp_tc_kernel(const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ 
         uint32_t tap_ok = 0;
         if (a.conv && col_live) {
             const int64_t n = col0 + t;
-            const int hw = a.H * a.W;
+            const int sd = a.stride > 1 ? a.stride : 1;
+            const int Ho = (a.H - 1) / sd + 1, Wo = (a.W - 1) / sd + 1;
+            const int hw = Ho * Wo;
             const int b = (int)(n / hw), pix = (int)(n - (int64_t)b * hw);
-            const int y = pix / a.W, x = pix - y * a.W;
+            const int y = (pix / Wo) * sd, x = (pix % Wo) * sd;       // the input pixel under the centre tap
             pix_base = a.X + (size_t)b * a.isb + (size_t)y * a.W + x;
 #pragma unroll
             for (int tp = 0; tp < 9; ++tp) {
@@ -439,7 +441,7 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
     const bool conv_pair_ok = a.conv && a.isb == (int64_t)a.H * a.W && a.isc % 4 == 0 &&
                               (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && a.isc >= Nc;
     const int bf16 = cfg_bf16(pl->cfg) ? 1 : 0;            // variants 34..37 / 44..47
-    tc_choose(M, K, Nc, a.conv ? (conv_pair_ok ? a.W : -1) : 0, bf16, sms, &kernel, &rows, &best_n);
+    tc_choose(M, K, Nc, a.conv ? (conv_pair_ok && a.stride <= 1 ? a.W : -1) : 0, bf16, sms, &kernel, &rows, &best_n);
     if (kernel == 2 && bf16) {
         CUtensorMap tmX;
         // the input as (column, channel): 16 channel rows of the CTA's columns per chunk, plus the halo for 3x3
@@ -508,11 +510,12 @@ int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, 
 }
 
 int launch_conv3x3_tc(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
-                      const float *bias, int relu, float *out, int64_t out_ld, void *stream_)
+                      const float *bias, int relu, float *out, int64_t out_ld, void *stream_, int stride)
 {
     TcArgs a{};
-    a.X = in; a.ldx = 0; a.conv = 1; a.H = H; a.W = Wd; a.isb = isb; a.isc = isc;
-    a.bias = bias; a.Y = out; a.ldy = out_ld; a.Nc = (int64_t)B * H * Wd; a.K = pl->dims.C * 9; a.relu = relu;
+    a.X = in; a.ldx = 0; a.conv = 1; a.H = H; a.W = Wd; a.isb = isb; a.isc = isc; a.stride = stride;
+    a.bias = bias; a.Y = out; a.ldy = out_ld; a.K = pl->dims.C * 9; a.relu = relu;
+    a.Nc = (int64_t)B * ((H - 1) / stride + 1) * ((Wd - 1) / stride + 1);
     return launch_tc_common(pl, a, static_cast<cudaStream_t>(stream_));
 }
 

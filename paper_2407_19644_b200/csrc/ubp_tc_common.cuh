@@ -154,7 +154,9 @@ struct TcArgs {
     const float *X;          // 1x1: [K][ldx]; 3x3: input tensor, element (b, c, y, x) at b*isb + c*isc + y*W + x
     int64_t ldx;
     int conv;                // 0 = 1x1 product, 1 = 3x3 / stride 1 / pad 1 implicit GEMM (k = tap * C + channel)
-    int H, W;                // 3x3 only: plane size; column n = b*H*W + y*W + x
+    int H, W;                // 3x3 only: input plane size; output column n = b*Ho*Wo + yo*Wo + xo
+    int stride;              // 3x3 only: 1, or > 1 (one-CTA kernel only): output pixel (yo, xo) is centred on input
+                             // pixel (yo*stride, xo*stride), Ho = (H-1)/stride + 1, Wo = (W-1)/stride + 1
     int64_t isb, isc;        // 3x3 only: input batch / channel strides (elements)
     const float *bias;
     float *Y;

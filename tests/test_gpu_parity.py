@@ -588,6 +588,34 @@ def test_stride_two_convolutions(env, layout, H, Wd):
         assert scaled_error(y, Yref, A) <= 1e-4
 
 
+@pytest.mark.parametrize("M,C,Nb,p,B,H,Wd,stride", [(128, 32, 4, 60, 3, 14, 14, 2), (256, 48, 8, 70, 2, 28, 28, 2),
+                                                      (200, 20, 4, 50, 2, 7, 9, 2), (130, 16, 2, 50, 1, 13, 12, 3),
+                                                      (256, 64, 4, 80, 4, 8, 8, 2)])
+def test_strided_conv3x3_on_tensor_cores(env, M, C, Nb, p, B, H, Wd, stride):
+    """A downsampling 3x3 with a tensor-core plan runs the one-CTA implicit-GEMM kernel (the loaders gather the taps of
+    output pixel (yo, xo) around input pixel (yo*stride, xo*stride)); against the oracle's stride-1 definition at
+    those pixels."""
+    torch, ubp = env
+    L = ubp_synth.make_layer("s3", M, C, Nb, p, 13 * M + C, B=B, H=H, Wd=Wd, R=9, x_dist="normal")
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb))
+    assert plan.variant >= 44
+    Ho, Wo = (H - 1) // stride + 1, (Wd - 1) // stride + 1
+    assert plan.tile_choice(B * Ho * Wo, -Wd)[0] == 1
+    bias = torch.from_numpy(L.bias).cuda()
+    y = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda(), bias, True, stride=stride)
+    plan.check()
+    Yref, A = oracle.masked_conv3x3(L.W, L.mask, L.X, L.bias, relu=True)
+    Yref, A = Yref[:, :, ::stride, ::stride], A[:, :, ::stride, ::stride]
+    yh = y.cpu().numpy()
+    assert yh.shape == Yref.shape == (M, B, Ho, Wo)
+    err = scaled_error(yh, Yref, A)
+    assert err <= 1e-4 and err <= arith_bound(L, 40)                 # three TF32 products per product
+    # the plain kernel on the same layer agrees to fp32 accuracy
+    ys = ubp.ubp_conv3x3_implicit(ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb), 20 if Nb % 8 == 0 else (21 if Nb % 4 == 0 else 22)),
+                                  torch.from_numpy(L.X).cuda(), bias, True, stride=stride)
+    assert scaled_error(ys.cpu().numpy(), Yref, A) <= (terms_per_output(L) + 2) * 2.0 ** -24
+
+
 @pytest.mark.parametrize("M,Cin,B,p,Nc", [(256, 256, 4, 70, 1000), (192, 320, 8, 95, 520), (64, 96, 2, 50, 260)])
 def test_kmajor_orientation_through_the_plan(env, M, Cin, B, p, Nc):
     """Blocks that run along the input channels of one output row: packed as the transposed layer, converted for

@@ -105,6 +105,9 @@ class Layer:
     H: int = 1
     Wd: int = 1
     starts: List[np.ndarray] = field(default_factory=list, repr=False)
+    stride: int = 1          # convolution stride (the strided workloads only)
+    src: Optional[int] = None   # chained workloads: index of the layer whose output this one reads (-1 = the block
+                                # input, None = the layer before it)
 
     @property
     def Nc(self) -> int:
@@ -113,8 +116,15 @@ class Layer:
         return self.B * self.H * self.Wd        # made without activations: the conv view's column count
 
     @property
+    def Nc_out(self) -> int:
+        """Output columns: Nc, or batch x the strided output plane for a strided layer."""
+        if self.stride == 1:
+            return self.Nc
+        return self.B * ((self.H - 1) // self.stride + 1) * ((self.Wd - 1) // self.stride + 1)
+
+    @property
     def surviving_macs(self) -> int:
-        return self.m * self.Nb * self.R * self.Nc
+        return self.m * self.Nb * self.R * self.Nc_out
 
 
 def make_layer(name: str, M: int, C: int, Nb: int, sparsity_pct: int, seed: int, *,
@@ -160,7 +170,14 @@ CONFIGS = {
     "sweep": "M=K=2048, Nc=8192; Nb in {2,4,8,16} x sparsity in {50,70,80,90}",
     "mbv1_chain": "13 pointwise layers of MobileNetV1, batch 64, 1x4, 80 %, bias+ReLU",
     "r50_bottleneck": "1x1 1024->256, 3x3 256->256, 1x1 256->1024 at 14x14, batch 32, blocks of 4, 80 %, chained",
+    "r50_downsample": "downsampling bottleneck 28x28 -> 14x14: 1x1 512->256, 3x3 256->256 stride 2, 1x1 256->1024, and "
+                      "the shortcut 1x1 512->1024 stride 2 on the block input; batch 32, blocks of 4, 80 %",
 }
+
+# r50_downsample: (output channels, input channels, taps, stride, relu, index of the layer whose output it reads;
+# -1 = the block input)
+R50_DOWNSAMPLE = [(256, 512, 1, 1, True, -1), (256, 256, 9, 2, True, 0), (1024, 256, 1, 1, False, 1),
+                  (1024, 512, 1, 2, False, -1)]
 
 
 def config_layers(cfg: str, *, batch: Optional[int] = None, Nb: Optional[int] = None,
@@ -199,6 +216,16 @@ def config_layers(cfg: str, *, batch: Optional[int] = None, Nb: Optional[int] = 
         return [make_layer(f"r50_bn_{li + 1}", co, ci, 4, 80, 6000 + 10 * index + li, B=b, H=14, Wd=14, R=r,
                            w_scale=0.03, bias=True, relu=relu, make_x=make_x and li == 0)
                 for li, (co, ci, r, relu) in enumerate(shapes)]
+    if cfg == "r50_downsample":
+        b = 32 if batch is None else batch
+        out = []
+        for li, (co, ci, r, stride, relu, src) in enumerate(R50_DOWNSAMPLE):
+            hw = 28 if src == -1 or li == 1 else 14          # spatial size of the tensor the layer READS
+            L = make_layer(f"r50_ds_{li + 1}", co, ci, 4, 80, 6500 + 10 * index + li, B=b, H=hw, Wd=hw, R=r, w_scale=0.03,
+                           bias=True, relu=relu, make_x=make_x and li == 0)
+            L.stride, L.src = stride, src
+            out.append(L)
+        return out
     raise KeyError(cfg)
 
 
