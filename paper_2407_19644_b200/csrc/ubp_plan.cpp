@@ -68,10 +68,10 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     if (R != 1) return nullptr;
     // Dense tensor-core variant when enough of the weight survives and the layer is large enough to amortise its
     // per-tile set-up: measured on B200 it takes the same time at every sparsity and beats the sparse kernel up to
-    // ~90 % sparsity on 2048 x 2048 x 8192. It pays from 128 rows and 128 input channels on (measured on the
-    // MobileNet-shaped layers: 128 -> 128 channels 57 us against 66 us; 64 -> 128 channels 52 against 45); below
-    // that the sparse kernel is as fast or faster.
-    if (dens >= 0.08 && M >= 128 && C >= 128) {
+    // ~90 % sparsity on 2048 x 2048 x 8192. It pays from 128 rows and 64 input channels on (measured on the
+    // MobileNet-shaped layers, launches back to back: 128 -> 128 channels 42 us against 60 us; 64 -> 128 channels 35
+    // against 39; 32 -> 64 channels 95 against 68, so below that the sparse kernel stays).
+    if (dens >= 0.08 && M >= 128 && C >= 64) {
         switch (nbk) {
             case 16: case 8: return find_cfg(33 + fast);
             case 4: return find_cfg(32 + fast);
