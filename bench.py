@@ -105,7 +105,7 @@ def tf32_peak_tflops():
 NCU_DRAM_BYTES_PER_LAUNCH = {
     ("mbv1_pw512", 36): 13936896 + 0,            # the 12.8 MB output is still in L2 when the kernel ends
     ("sweep_nb4_p70", 36): 84903936 + 40135680,
-    ("r50_3x3", 44): 15257344 + 1280,
+    ("r50_3x3", 44): 15257344 + 1280,            # the per-tap kernel
     ("mbv1_pw512", 32): 14984448 + 256,
     ("sweep_nb4_p70", 32): 124626432 + 48126208,
     ("r50_3x3", 40): 17614080 + 0,
@@ -370,18 +370,25 @@ KERNEL_NAMES = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF
                 "ubp_tc2_kernel (dense 3xTF32 on tcgen05, CTA pair per tile)",
                 "ubp_tc3_kernel (dense 3xBF16 on tcgen05, CTA pair per tile)",
                 "ubp_wros_kernel (the paper's loop over the canonical arrays, weight rotation, FP32 FMA)",
-                "ubp_wros_kernel (the paper's loop over the canonical arrays, naive shift, FP32 FMA)")
+                "ubp_wros_kernel (the paper's loop over the canonical arrays, naive shift, FP32 FMA)",
+                "ubp_conv3_kernel (3x3 on the padded pixel grid, taps as operand shifts, dense 3xBF16 on tcgen05, CTA pair per tile)")
 ARITHMETIC = ("fp32 FMA, fp32 accumulate",
               "3 TF32 products per fp32 product, fp32 accumulate (error <= 2^-18 |w||x|)",
               "3 TF32 products per fp32 product, fp32 accumulate (error <= 2^-18 |w||x|)",
               "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)",
-              "fp32 FMA, fp32 accumulate", "fp32 FMA, fp32 accumulate")
+              "fp32 FMA, fp32 accumulate", "fp32 FMA, fp32 accumulate",
+              "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)")
 
 
 def kernel_info(plan, L):
     """(index into KERNEL_NAMES / ARITHMETIC, [tile rows, tile columns]) of a fast-path launch of this plan."""
-    kern, tile_rows, tile_cols = plan.tile_choice(L.Nc, L.Wd if L.R == 9 else 0)
-    bf16 = 34 <= plan.variant <= 37 or 44 <= plan.variant <= 47
+    if L.R == 9:
+        kern, tile_rows, tile_cols = plan.tile_choice_conv(L.B, L.H, L.Wd, L.stride)
+        if kern == 4:
+            return 6, [tile_rows, tile_cols]
+    else:
+        kern, tile_rows, tile_cols = plan.tile_choice(L.Nc, 0)
+    bf16 = 34 <= plan.variant <= 37 or 44 <= plan.variant <= 47 or 64 <= plan.variant <= 67
     if L.R == 9 and plan.variant < 40:
         return 0, [tile_rows, tile_cols]
     if plan.variant in (60, 61):

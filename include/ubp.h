@@ -178,6 +178,14 @@ int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info);
 int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, int *kernel, int *tile_rows,
                          int *tile_cols);
 
+/* ubp_plan_tile_choice_conv: the same question for a 3x3 plan and a batch of B images of H x Wd pixels in the layout
+ * the fast paths take (input and output each one [channel][batch, y, x] matrix): *kernel as above, or 4 = the CTA-pair
+ * kernel that computes on the zero-padded pixel grid and takes the nine taps as shifts of one staged operand
+ * (variants 64..67, stride 1, more than 128 output channels, input channels a multiple of 16); tile_cols then counts
+ * padded positions. */
+int ubp_plan_tile_choice_conv(const ubp_plan_t *plan, int B, int H, int Wd, int stride, int *kernel, int *tile_rows,
+                              int *tile_cols);
+
 /* Read the plan's device status word: blocks until `stream` has finished
  * (cudaStreamSynchronize), then returns UBP_OK or UBP_E_DEVICE if a kernel
  * launched with this plan gave up on a bounded wait. */
@@ -233,11 +241,16 @@ int ubp_conv1x1(const ubp_plan_t *plan, const float *in, int B, int H, int Wd,
 /* ubp_conv3x3_implicit: 3x3, stride 1, zero padding 1, cross-correlation; the
  * plan must come from a blob with R == 9 (a block = Nb output channels x one
  * input channel x all nine taps, Section 3.1). The K = 9*C lowered matrix is
- * never formed in memory. Tensor-core plans (variants 40..47; input and output
- * each one [channel][batch, y, x] matrix with 16-byte aligned rows) run an
- * implicit GEMM whose reduction index is tap * C + channel: the input rows of a
- * 16-channel chunk are copied into shared memory once with a halo of columns
- * and the nine shifted, border-masked operand tiles are cut from that copy.
+ * never formed in memory. Tensor-core plans (input and output each one
+ * [channel][batch, y, x] matrix with 16-byte aligned rows) run an implicit GEMM.
+ * Variants 64..67 (the choice of variant 0; more than 128 output channels, input
+ * channels a multiple of 16): the outputs are computed on the zero-padded pixel
+ * grid, where a tap is a pure shift; per 16 input channels the real pixels a
+ * tile touches are copied into shared memory once, split once into the bf16
+ * operand pair, and the nine taps read that one operand at nine start offsets.
+ * Variants 40..47 (and 64..67 on layers that kernel does not take): reduction
+ * index tap * C + channel; per tap and 16-channel chunk the input rows are copied
+ * with a halo of columns and a shifted, border-masked operand tile is cut out.
  * Other plans and layouts run a kernel with one lane per output pixel that
  * reads its taps in place. Arithmetic per kernel as for ubp_spmm.
  * Same strides as ubp_conv1x1. */

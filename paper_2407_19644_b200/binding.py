@@ -61,6 +61,7 @@ def load():
     L.ubp_plan_info.argtypes = [vp, C.POINTER(_PlanInfo)]
     L.ubp_plan_check.argtypes = [vp, vp]
     L.ubp_plan_tile_choice.argtypes = [vp, i64, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+    L.ubp_plan_tile_choice_conv.argtypes = [vp, i32, i32, i32, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
     L.ubp_spmm.argtypes = [vp, vp, i64, i64, vp, i32, vp, i64, vp]
     L.ubp_conv1x1.argtypes = [vp, vp, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
     L.ubp_conv3x3_implicit.argtypes = [vp, vp, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
@@ -269,6 +270,16 @@ class Plan:
         with torch.cuda.device(self.buffer.device):
             _chk(self._lib.ubp_plan_tile_choice(self.handle, int(Nc), int(image_width), C.byref(k), C.byref(r), C.byref(c)),
                  "ubp_plan_tile_choice")
+        return k.value, r.value, c.value
+
+    def tile_choice_conv(self, B: int, H: int, Wd: int, stride: int = 1):
+        """(kernel, tile_rows, tile_cols) of a fast-path 3x3 launch on B images of H x Wd pixels; kernel 4 = the CTA-pair
+        kernel on the padded pixel grid (tile_cols in padded positions), else as tile_choice."""
+        k, r, c = C.c_int32(), C.c_int32(), C.c_int32()
+        import torch
+        with torch.cuda.device(self.buffer.device):
+            _chk(self._lib.ubp_plan_tile_choice_conv(self.handle, int(B), int(H), int(Wd), int(stride), C.byref(k), C.byref(r),
+                                                     C.byref(c)), "ubp_plan_tile_choice_conv")
         return k.value, r.value, c.value
 
     def clear_status(self, stream=None):

@@ -315,6 +315,23 @@ int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, in
     return UBP_OK;
 }
 
+int ubp_plan_tile_choice_conv(const ubp_plan_t *plan, int B, int H, int Wd, int stride, int *kernel, int *tile_rows,
+                              int *tile_cols)
+{
+    if (!plan || plan->magic != kPlanMagic || !kernel || !tile_rows || !tile_cols) return UBP_E_ARG;
+    if (plan->dims.R != 9 || B < 1 || H < 1 || Wd < 1 || stride < 1) return UBP_E_ARG;
+    const ubp::KernelCfg &c = plan->cfg;
+    int sms = 148, devid = 0;
+    if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
+    int n = 0;
+    if (stride == 1 && ubp::cfg_conv3_shift(c) && ubp::conv3_pair_tile(plan->dims.M, plan->dims.C, B, H, Wd, sms, &n)) {
+        *kernel = 4; *tile_rows = 256; *tile_cols = n;
+        return UBP_OK;
+    }
+    const int64_t Nc = (int64_t)B * ((H - 1) / stride + 1) * ((Wd - 1) / stride + 1);
+    return ubp_plan_tile_choice(plan, Nc, stride == 1 ? Wd : -Wd, kernel, tile_rows, tile_cols);
+}
+
 int ubp_plan_check(const ubp_plan_t *plan, void *stream)
 {
     if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;

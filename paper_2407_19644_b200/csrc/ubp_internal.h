@@ -37,7 +37,9 @@ const std::vector<KernelCfg> &kernel_cfgs();
 // Output rows per CTA of the bf16 CTA-pair kernel: 128, or for layers of at most 128 rows half of them (rounded up to
 // a multiple of 8) so that both CTAs of the pair have rows to store.
 inline int tc16_rows_per_cta(int M) { return M > 128 ? 128 : (((M + 1) / 2 + 7) & ~7); }
-inline bool cfg_bf16(const KernelCfg &c) { return (c.id >= 34 && c.id <= 37) || (c.id >= 44 && c.id <= 47); }
+// 64..67: 3x3 with the taps as shifts of one staged operand on the padded pixel grid (ubp_conv3.cu; bf16 products too)
+inline bool cfg_conv3_shift(const KernelCfg &c) { return c.id >= 64 && c.id <= 67; }
+inline bool cfg_bf16(const KernelCfg &c) { return (c.id >= 34 && c.id <= 37) || (c.id >= 44 && c.id <= 47) || cfg_conv3_shift(c); }
 const KernelCfg *find_cfg(int id);
 // pick a configuration for a layer (variant == 0)
 const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m);
@@ -105,6 +107,10 @@ int launch_subsample(const float *in, int C, int B, int H, int Wd, int64_t isb, 
 // the paper's dataflow on the canonical arrays (ubp_wros.cu): variants 60 (weight rotation) and 61 (naive shift)
 int launch_wros(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu, float *Y,
                 int64_t ldy, void *stream);
+// 3x3 on the padded pixel grid, taps as descriptor shifts (ubp_conv3.cu); UBP_E_UNSUPPORTED when the layer does not fit
+int launch_conv3_pair(const void *W16, const float *X, int64_t isc, const void *args, int M, int C, int B, int H, int W,
+                      int sms, void *stream);
+bool conv3_pair_tile(int M, int C, int B, int H, int W, int sms, int *tile_cols);
 void set_last_cuda_error(int e);
 }
 

@@ -49,12 +49,12 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     // shared-memory time, error <= 3 * 2^-16 |w||x|, inside the 1e-4 gate) is the default; the TF32-product ids stay
     // selectable (with at most 128 rows they run the one-CTA kernel).
     const int fast = 4;
-    if (R == 9 && dens >= 0.08 && M >= 128 && C >= 16) {    // implicit GEMM on tensor cores
+    if (R == 9 && dens >= 0.08 && M >= 128 && C >= 16) {    // implicit GEMM on tensor cores, taps as operand shifts
         switch (nbk) {
-            case 16: case 8: return find_cfg(40 + fast);
-            case 4: return find_cfg(41 + fast);
-            case 2: return find_cfg(42 + fast);
-            default: return find_cfg(43 + fast);
+            case 16: case 8: return find_cfg(64);
+            case 4: return find_cfg(65);
+            case 2: return find_cfg(66);
+            default: return find_cfg(67);
         }
     }
     if (R == 9) {

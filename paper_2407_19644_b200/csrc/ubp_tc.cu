@@ -442,6 +442,12 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
                               (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && a.isc >= Nc;
     const int bf16 = cfg_bf16(pl->cfg) ? 1 : 0;            // variants 34..37 / 44..47
     tc_choose(M, K, Nc, a.conv ? (conv_pair_ok && a.stride <= 1 ? a.W : -1) : 0, bf16, sms, &kernel, &rows, &best_n);
+    if (a.conv && conv_pair_ok && a.stride <= 1 && cfg_conv3_shift(pl->cfg)) {
+        // the padded-grid kernel where it takes the layer; otherwise on through the per-tap kernels below
+        a.rpc = 128;
+        rc = launch_conv3_pair(dev + pl->img.tc16_off, a.X, a.isc, &a, M, K / 9, (int)(Nc / ((int64_t)a.H * a.W)), a.H, a.W, sms, stream);
+        if (rc != UBP_E_UNSUPPORTED) return rc;
+    }
     if (kernel == 2 && bf16) {
         CUtensorMap tmX;
         // the input as (column, channel): 16 channel rows of the CTA's columns per chunk, plus the halo for 3x3

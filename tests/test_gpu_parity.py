@@ -52,7 +52,7 @@ def run_spmm(env, L, variant=0, pad=0, misalign=0, relu=None, use_bias=True):
 
 def is_bf16(variant):
     """Tensor-core variants whose CTA-pair kernel multiplies with three bf16 products instead of three TF32 ones."""
-    return 34 <= variant <= 37 or 44 <= variant <= 47
+    return 34 <= variant <= 37 or 44 <= variant <= 47 or 64 <= variant <= 67
 
 
 def arith_bound(L, variant):
@@ -435,7 +435,7 @@ def test_conv3x3_tensor_core_variant(env, M, C, Nb, p, B, H, Wd, variant):
     plan.check()
     Yref, A = oracle.masked_conv3x3(L.W, L.mask, L.X, L.bias, relu=True)
     check(Y.cpu().numpy(), Yref, A, L, variant=plan.variant)
-    if plan.variant < 44 and M > 128:    # the same layer through the TF32 / the bf16 form explicitly
+    if plan.variant < 44 and M > 128:    # the same layer through the TF32 / the bf16 form explicitly (per-tap kernels)
         for v in (plan.variant, plan.variant + 4):
             pv = ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb), v)
             Yv = ubp.ubp_conv3x3_implicit(pv, torch.from_numpy(L.X).cuda(), b, True, layout="CNHW")
@@ -444,6 +444,35 @@ def test_conv3x3_tensor_core_variant(env, M, C, Nb, p, B, H, Wd, variant):
     # NCHW output is not one [M][B*H*W] matrix: served by the plain kernel on the embedded sparse plan
     Yn = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda().permute(1, 0, 2, 3).contiguous(), b, True, layout="NCHW")
     check(Yn.permute(1, 0, 2, 3).contiguous().cpu().numpy(), Yref, A, L)
+
+
+@pytest.mark.parametrize("M,C,Nb,p,B,H,Wd", [(256, 32, 4, 60, 3, 7, 9), (300, 48, 4, 60, 2, 14, 14), (256, 16, 8, 50, 1, 28, 28),
+                                              (260, 32, 2, 50, 3, 13, 11), (512, 64, 4, 70, 7, 14, 14), (256, 32, 4, 60, 1, 9, 60),
+                                              (256, 32, 4, 60, 2, 5, 80), (384, 160, 8, 80, 40, 14, 14), (256, 16, 1, 50, 150, 3, 3),
+                                              (256, 32, 4, 100, 2, 6, 6)])
+def test_conv3x3_taps_as_operand_shifts(env, M, C, Nb, p, B, H, Wd):
+    """The 3x3 kernel that computes on the zero-padded pixel grid and takes the nine taps as shifts of one staged
+    operand (variants 64..67, the automatic choice): small and wide images (up to 80 pixels: the halo grows with the
+    width), image sizes that put tile boundaries anywhere in a row, batches that give a pair several tiles, a layer
+    with no block kept. Against the oracle's direct convolution, at the bound of the bf16-product arithmetic."""
+    torch, ubp = env
+    L = ubp_synth.make_layer("c", M, C, Nb, p, 17 * M + C + Wd, B=B, H=H, Wd=Wd, R=9, x_dist="normal")
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb), 65 if p == 100 else 0)       # nothing kept: not the automatic choice
+    assert 64 <= plan.variant <= 67
+    kern, rows, cols = plan.tile_choice_conv(B, H, Wd)
+    assert kern == 4 and rows == 256 and cols % 16 == 0 and cols // 2 + 2 * (Wd + 3) <= 256
+    b = torch.from_numpy(L.bias).cuda()
+    ybuf = torch.full((M, B, H, Wd), float("nan"), dtype=torch.float32, device="cuda")
+    Y = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda(), b, True, out=ybuf)
+    plan.check()
+    Yref, A = oracle.masked_conv3x3(L.W, L.mask, L.X, L.bias, relu=True)
+    check(Y.cpu().numpy(), Yref, A, L, variant=plan.variant)
+    # the per-tap kernel on the same layer gives the same result to the same bound; and twice the same bits
+    Y2 = ubp.ubp_conv3x3_implicit(plan, torch.from_numpy(L.X).cuda(), b, True)
+    assert torch.equal(Y, Y2)
+    pold = ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb), plan.variant - 20)
+    assert pold.tile_choice_conv(B, H, Wd)[0] in (1, 2)
+    check(ubp.ubp_conv3x3_implicit(pold, torch.from_numpy(L.X).cuda(), b, True).cpu().numpy(), Yref, A, L, variant=pold.variant)
 
 
 def test_r50_3x3_config_sampled(env):
