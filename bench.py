@@ -371,13 +371,15 @@ KERNEL_NAMES = ("ubp_spmm_kernel (sparse, FP32 FMA)", "ubp_tc_kernel (dense 3xTF
                 "ubp_tc3_kernel (dense 3xBF16 on tcgen05, CTA pair per tile)",
                 "ubp_wros_kernel (the paper's loop over the canonical arrays, weight rotation, FP32 FMA)",
                 "ubp_wros_kernel (the paper's loop over the canonical arrays, naive shift, FP32 FMA)",
-                "ubp_conv3_kernel (3x3 on the padded pixel grid, taps as operand shifts, dense 3xBF16 on tcgen05, CTA pair per tile)")
+                "ubp_conv3_kernel (3x3 on the padded pixel grid, taps as operand shifts, dense 3xBF16 on tcgen05, CTA pair per tile)",
+                "ubp_tc3_kernel (dense 6xBF16 in three pieces on tcgen05, CTA pair per tile)")
 ARITHMETIC = ("fp32 FMA, fp32 accumulate",
               "3 TF32 products per fp32 product, fp32 accumulate (error <= 2^-18 |w||x|)",
               "3 TF32 products per fp32 product, fp32 accumulate (error <= 2^-18 |w||x|)",
               "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)",
               "fp32 FMA, fp32 accumulate", "fp32 FMA, fp32 accumulate",
-              "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)")
+              "3 bf16 products per fp32 product, fp32 accumulate (error <= 3 * 2^-16 |w||x|)",
+              "6 bf16 products of three exact pieces per fp32 product, fp32 accumulate (product error < 2^-23 |w||x|)")
 
 
 def kernel_info(plan, L):
@@ -389,6 +391,8 @@ def kernel_info(plan, L):
     else:
         kern, tile_rows, tile_cols = plan.tile_choice(L.Nc, 0)
     bf16 = 34 <= plan.variant <= 37 or 44 <= plan.variant <= 47 or 64 <= plan.variant <= 67
+    if 84 <= plan.variant <= 87:
+        return 7, [tile_rows, tile_cols]
     if L.R == 9 and plan.variant < 40:
         return 0, [tile_rows, tile_cols]
     if plan.variant in (60, 61):
@@ -443,8 +447,8 @@ def workload_config(L, name, world, no_flush):
 # The other BASELINE configurations the default run measures beside the headline (every frac from the mean time)
 EXTRA_CONFIGS = ["r50_3x3", "sweep_nb2_p50", "sweep_nb16_p50", "sweep_nb4_p70", "sweep_nb2_p90", "sweep_nb16_p90"] + \
                 [f"mbv1_L{i + 1}" for i in range(13)]
-# The headline layer through the other two arithmetics: TF32 products on tensor cores, fp32 FMA on the CUDA cores
-HEADLINE_VARIANTS = [32, 14]
+# The headline layer through the other arithmetics: three bf16 pieces (six products), TF32 products, fp32 FMA on the CUDA cores
+HEADLINE_VARIANTS = [86, 32, 14]
 
 
 def build_chained(ubp, torch, layers, variant):

@@ -101,7 +101,7 @@ int ubp_variant_describe(int variant, char *buf, size_t cap)
 {
     const ubp::KernelCfg *c = ubp::find_cfg(variant);
     if (!c || !buf || cap == 0) return UBP_E_ARG;
-    const char *prod = ubp::cfg_bf16(*c) ? "3xBF16" : "3xTF32";
+    const char *prod = ubp::cfg_pieces(*c) == 3 ? "6xBF16, three pieces" : (ubp::cfg_bf16(*c) ? "3xBF16" : "3xTF32");
     char kind[64];
     if (c->kind == 4) {
         std::snprintf(buf, cap, "spmm-from-canonical-arrays %s", c->id == 61 ? "naive(outputs shifted per start row)"
@@ -305,7 +305,7 @@ int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, in
     if (c.kind == 2 || c.kind == 3) {
         int sms = 148, devid = 0;
         if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
-        ubp::tc_choose(plan->dims.M, plan->dims.C * plan->dims.R, Nc, c.kind == 3 ? (image_width > 0 ? image_width : -1) : 0, ubp::cfg_bf16(c) ? 1 : 0, sms, kernel, tile_rows,
+        ubp::tc_choose(plan->dims.M, plan->dims.C * plan->dims.R, Nc, c.kind == 3 ? (image_width > 0 ? image_width : -1) : 0, ubp::cfg_bf16(c) ? (ubp::cfg_pieces(c) == 3 ? 2 : 1) : 0, sms, kernel, tile_rows,
                        tile_cols);
     } else if (c.kind == 4) {
         *kernel = 3; *tile_rows = 0; *tile_cols = 512;       // row ranges are chosen per launch; 128 threads x 4 columns

@@ -39,7 +39,12 @@ const std::vector<KernelCfg> &kernel_cfgs();
 inline int tc16_rows_per_cta(int M) { return M > 128 ? 128 : (((M + 1) / 2 + 7) & ~7); }
 // 64..67: 3x3 with the taps as shifts of one staged operand on the padded pixel grid (ubp_conv3.cu; bf16 products too)
 inline bool cfg_conv3_shift(const KernelCfg &c) { return c.id >= 64 && c.id <= 67; }
-inline bool cfg_bf16(const KernelCfg &c) { return (c.id >= 34 && c.id <= 37) || (c.id >= 44 && c.id <= 47) || cfg_conv3_shift(c); }
+// 84..87: the bf16 CTA-pair kernel with every operand in THREE bf16 pieces (exact) and six products per fp32 product
+inline int cfg_pieces(const KernelCfg &c) { return (c.id >= 84 && c.id <= 87) ? 3 : 2; }
+inline bool cfg_bf16(const KernelCfg &c)
+{
+    return (c.id >= 34 && c.id <= 37) || (c.id >= 44 && c.id <= 47) || cfg_conv3_shift(c) || cfg_pieces(c) == 3;
+}
 const KernelCfg *find_cfg(int id);
 // pick a configuration for a layer (variant == 0)
 const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m);
@@ -69,6 +74,7 @@ struct PlanImage {
     // tc16_kp = reduction length padded to whole chunks
     size_t tc16_off = 0;
     int tc16_kp = 0;
+    int tc16_pieces = 2;     // bf16 pieces per weight in that part (3: W3 = the remainder after W1 + W2, blocks of 12 KB)
     // kind 4 only: byte offsets of the canonical arrays indptr [M+1], indices [m], values [m][Nb] in the image
     size_t wros_off[3] = {0, 0, 0};
 };

@@ -213,7 +213,8 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         // 128 rows puts half of them into each of the pair's two tiles (the rest of a tile stays zero).
         img.tc16_kp = (C * R + 15) & ~15;   // padded reduction length: whole chunks
         img.tc16_off = total;
-        total += (size_t)((M + 255) / 256) * 2 * (img.tc16_kp / 16) * 8192;   // whole pairs of row tiles (zero rows pad)
+        img.tc16_pieces = cfg_pieces(cfg);  // 2 pieces: 8 KB blocks; 3 pieces (W3 = what W1 + W2 leave): 12 KB blocks
+        total += (size_t)((M + 255) / 256) * 2 * (img.tc16_kp / 16) * 4096 * img.tc16_pieces;   // whole pairs of row tiles
     }
     if (bytes) *bytes = total;
     img.nkt = nkt; img.NP = NP; img.NG = NG; img.F = F; img.entries = entries; img.max_group_bytes = max_group;
@@ -283,7 +284,7 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
             int i = row % rpc16;
             if (rpc16 < 128) i = (i / (rpc16 / 4)) * 32 + i % (rpc16 / 4);
             const int kk = (int)(k % 16);
-            return reinterpret_cast<uint16_t *>(W16 + blk * 8192 + (size_t)piece * 4096 + (size_t)i * 32 +
+            return reinterpret_cast<uint16_t *>(W16 + blk * (4096 * (size_t)img.tc16_pieces) + (size_t)piece * 4096 + (size_t)i * 32 +
                                                 (size_t)(((kk >> 3) ^ ((i >> 2) & 1)) * 16) + (size_t)(kk & 7) * 2);
         };
         auto bf16_rn = [](float f) -> uint16_t {
@@ -318,8 +319,10 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
                     Wh[(size_t)(i + t) * img.tc_kp + (size_t)r * C + j] = hi;
                     Wl[(size_t)(i + t) * img.tc_kp + (size_t)r * C + j] = lo;
                     const uint16_t w1 = bf16_rn(w);
+                    const uint16_t w2 = bf16_rn(w - bf16_f(w1));
                     *w16_at(i + t, (size_t)r * C + j, 0) = w1;
-                    *w16_at(i + t, (size_t)r * C + j, 1) = bf16_rn(w - bf16_f(w1));
+                    *w16_at(i + t, (size_t)r * C + j, 1) = w2;
+                    if (img.tc16_pieces == 3) *w16_at(i + t, (size_t)r * C + j, 2) = bf16_rn((w - bf16_f(w1)) - bf16_f(w2));
                   }
             }
     }

@@ -351,7 +351,7 @@ int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d
 int tc_pair_stages(int ntile, int halo);
 // same pipeline with three bf16 products per fp32 product (ubp_tc3.cu)
 int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, int halo, const void *args,
-                        int M, int64_t Nc, int ntile, int sms, void *stream);
+                        int M, int64_t Nc, int ntile, int sms, void *stream, int pieces);
 int tc_pair_bf16_stages(int ntile, int halo);
 
 // Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
@@ -410,7 +410,7 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
             // fp32 rows) arrive at ~32 B/cycle/SM, the rate of the L2-to-SM path; 3x3: the shifted-tile pass
             // (~700 + 0.6 n). A tile costs its chunks or its epilogue (~50 cycles per column) plus ~2500 cycles of
             // hand-over between tiles.
-            double per_chunk = bf16 ? 1.65 * n : 3.3 * n;
+            double per_chunk = bf16 == 2 ? 3.3 * n : (bf16 ? 1.65 * n : 3.3 * n);     // bf16 == 2: three pieces, six MMAs
             const double smem_chunk = bf16 ? (conv ? 700.0 + 0.6 * n : 470.0 + 0.33 * n) : (conv ? 560.0 + 1.0 * n : 500.0 + 0.5 * n);
             if (per_chunk < smem_chunk) per_chunk = smem_chunk;
             double per_tile = nchunk * per_chunk;
@@ -420,7 +420,8 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
             const double t = 4400.0 + (double)per_pair * per_tile + 4500.0 + 30.0 * n;
             if (t < best2) { best2 = t; best2_n = n; }
         }
-        if (best2_n && best2 < best) { *kernel = 2; *rows = 256; *cols = best2_n; }
+        // (three pieces exist on the pair kernel only: never weigh it against the one-CTA TF32 kernel)
+        if (best2_n && (best2 < best || bf16 == 2)) { *kernel = 2; *rows = 256; *cols = best2_n; }
     }
 }
 
@@ -440,7 +441,7 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
     // 3x3 on CTA pairs needs the input as one [channel][b, y, x] matrix with 16-byte aligned rows
     const bool conv_pair_ok = a.conv && a.isb == (int64_t)a.H * a.W && a.isc % 4 == 0 &&
                               (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && a.isc >= Nc;
-    const int bf16 = cfg_bf16(pl->cfg) ? 1 : 0;            // variants 34..37 / 44..47
+    const int bf16 = cfg_bf16(pl->cfg) ? (cfg_pieces(pl->cfg) == 3 ? 2 : 1) : 0;   // 1: two bf16 pieces, 2: three
     tc_choose(M, K, Nc, a.conv ? (conv_pair_ok && a.stride <= 1 ? a.W : -1) : 0, bf16, sms, &kernel, &rows, &best_n);
     if (a.conv && conv_pair_ok && a.stride <= 1 && cfg_conv3_shift(pl->cfg)) {
         // the padded-grid kernel where it takes the layer; otherwise on through the per-tap kernels below
@@ -455,7 +456,7 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
         if ((rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)(a.conv ? K / 9 : K), (uint64_t)(a.conv ? a.isc : a.ldx) * 4,
                             (uint32_t)(best_n / 2 + 2 * halo), TC_KC, CU_TENSOR_MAP_SWIZZLE_NONE))) return rc;
         a.rpc = tc16_rows_per_cta(M);
-        return launch_tc_pair_bf16(dev + pl->img.tc16_off, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream);
+        return launch_tc_pair_bf16(dev + pl->img.tc16_off, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream, cfg_pieces(pl->cfg));
     }
     if (kernel == 2) {
         // Wh and Wl as one 3-D tensor (channel, row, part): one copy per chunk brings both

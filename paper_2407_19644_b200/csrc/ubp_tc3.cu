@@ -53,18 +53,19 @@ __host__ __device__ constexpr uint32_t t3_raw_bytes(int nh, int halo)
     return ((uint32_t)(nh + 2 * halo) * TC_KC * 4 + 1023u) & ~1023u;
 }
 // one chunk's part of a stage
-__host__ __device__ constexpr uint32_t t3_chunk_bytes(int nh, int halo)
+// (np = pieces per operand: 2, or 3 for the variant whose products are exact to fp32's last bits)
+__host__ __device__ constexpr uint32_t t3_chunk_bytes(int nh, int halo, int np)
 {
-    return 2 * T3_A_PART + 2 * t3_x_bytes(nh) + t3_raw_bytes(nh, halo);
+    return (uint32_t)np * T3_A_PART + (uint32_t)np * t3_x_bytes(nh) + t3_raw_bytes(nh, halo);
 }
 // A stage holds `sub` chunks. With two, every barrier round trip (copies landed -> split pass -> MMA issue -> stage
 // free) serves 32 channels: fewer waits per channel, which pays on long reductions (3x3: 144 chunks; 1024 channels)
 // where the pass or the issue thread is the bound; with one, the pipeline fills and drains in finer steps, which
 // pays on short reductions (512 channels: 32 chunks).
-__host__ __device__ constexpr uint32_t t3_stage_bytes(int nh, int halo, int sub) { return (uint32_t)sub * t3_chunk_bytes(nh, halo); }
-__host__ __device__ constexpr int t3_stages(int nh, int halo, int sub)
+__host__ __device__ constexpr uint32_t t3_stage_bytes(int nh, int halo, int sub, int np) { return (uint32_t)sub * t3_chunk_bytes(nh, halo, np); }
+__host__ __device__ constexpr int t3_stages(int nh, int halo, int sub, int np)
 {
-    const int s = (int)(T3_PIPE_BUDGET / t3_stage_bytes(nh, halo, sub));
+    const int s = (int)(T3_PIPE_BUDGET / t3_stage_bytes(nh, halo, sub, np));
     return (s > T3_MAX_STAGES ? T3_MAX_STAGES : s) / T3_XL_GROUPS * T3_XL_GROUPS;
 }
 
@@ -105,6 +106,59 @@ __device__ __forceinline__ bool mma3_chunk(uint32_t d_tmem, uint64_t dW1, uint64
     return ready != 0;
 }
 
+// The same for operands in THREE bf16 pieces (w = w1 + w2 + w3 exactly, likewise x): the six products whose pieces'
+// orders add up to at most four, w1 x1, w2 x1, w1 x2, w3 x1, w2 x2, w1 x3; what is dropped is below 2^-23 |w x|.
+__device__ __forceinline__ bool mma6_chunk(uint32_t d_tmem, uint64_t dW1, uint64_t dX1, uint32_t w_step, uint32_t x_step,
+                                           uint32_t idesc, uint32_t acc_first, uint32_t next_bar, uint32_t next_parity,
+                                           uint32_t empty_bar, uint32_t last)
+{
+    uint32_t ready;
+    asm volatile(
+        "{\n\t.reg .pred pn, pa, pt, pe, pc;\n\t.reg .b64 w2, w3, x2, x3, ws, xs;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 pn, [%8], %9;\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "setp.ne.b32 pc, %13, 0;\n\t"
+        "and.pred pc, pc, pe;\n\t"
+        "setp.ne.b32 pa, %7, 0;\n\t"
+        "setp.eq.b32 pt, %10, 0;\n\t"
+        "cvt.u64.u32 ws, %4;\n\tadd.s64 w2, ws, %2;\n\tadd.s64 w3, w2, ws;\n\t"
+        "cvt.u64.u32 xs, %5;\n\tadd.s64 x2, xs, %3;\n\tadd.s64 x3, x2, xs;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %6, pa;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w2, %3, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, x2, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w3, %3, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w2, x2, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, x3, %6, pt;\n\t"
+        "@pc tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%11], %12;\n\t"
+        "selp.u32 %0, 1, 0, pn;\n\t}"
+        : "=r"(ready)
+        : "r"(d_tmem), "l"(dW1), "l"(dX1), "r"(w_step), "r"(x_step), "r"(idesc), "r"(acc_first), "r"(next_bar),
+          "r"(next_parity), "r"(0u), "r"(empty_bar), "h"((uint16_t)3), "r"(last)
+        : "memory");
+    return ready != 0;
+}
+
+// eight fp32 -> three bf16 pieces each (x = x1 + x2 + x3 exactly: 8 + 8 + 8 significant bits), packed two per word
+__device__ __forceinline__ void split8x3(const float (&v)[8], uint4 &p1, uint4 &p2, uint4 &p3)
+{
+    uint32_t a1[4], a2[4], a3[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        const float2 af = __bfloat1622float2(a);
+        const float r0 = v[2 * i] - af.x, r1 = v[2 * i + 1] - af.y;
+        const __nv_bfloat162 b = __floats2bfloat162_rn(r0, r1);
+        const float2 bf = __bfloat1622float2(b);
+        const __nv_bfloat162 c = __floats2bfloat162_rn(r0 - bf.x, r1 - bf.y);
+        a1[i] = *reinterpret_cast<const uint32_t *>(&a);
+        a2[i] = *reinterpret_cast<const uint32_t *>(&b);
+        a3[i] = *reinterpret_cast<const uint32_t *>(&c);
+    }
+    p1 = make_uint4(a1[0], a1[1], a1[2], a1[3]);
+    p2 = make_uint4(a2[0], a2[1], a2[2], a2[3]);
+    p3 = make_uint4(a3[0], a3[1], a3[2], a3[3]);
+}
+
 // eight fp32 -> their bf16 heads (x1) and the bf16 of the remainders (x2), packed two per word
 __device__ __forceinline__ void split8(const float (&v)[8], uint4 &h, uint4 &l)
 {
@@ -121,7 +175,7 @@ __device__ __forceinline__ void split8(const float (&v)[8], uint4 &h, uint4 &l)
     l = make_uint4(ll[0], ll[1], ll[2], ll[3]);
 }
 
-template <bool CONV, int SUB>
+template <bool CONV, int SUB, int NP>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T3_THREADS, 1)
 ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensorMap tmX, const TcArgs a,
                const int halo, const int nrp, const int ntiles)
@@ -141,12 +195,12 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     const uint32_t rank = cluster_rank();
     const int N = a.ntile, NH = N / 2;                     // tile columns; columns whose X this CTA holds
     const uint32_t xb = t3_x_bytes(NH);                    // x1 (and x2) bytes per chunk
-    const uint32_t chunk_bytes = t3_chunk_bytes(NH, halo), stage_bytes = (uint32_t)SUB * chunk_bytes;
+    const uint32_t chunk_bytes = t3_chunk_bytes(NH, halo, NP), stage_bytes = (uint32_t)SUB * chunk_bytes;
     const uint32_t raw_row = (uint32_t)(NH + 2 * halo) * 4;   // bytes per channel row of the raw copy
-    const int S = t3_stages(NH, halo, SUB);
+    const int S = t3_stages(NH, halo, SUB, NP);
     const int nchunk = (a.K + TC_KC - 1) / TC_KC;
     const int nstage = (nchunk + SUB - 1) / SUB;     // stages per tile; the last one may hold a single chunk
-    const uint32_t tx = 2 * T3_A_PART + raw_row * TC_KC;   // bytes copied per chunk
+    const uint32_t tx = NP * T3_A_PART + raw_row * TC_KC;  // bytes copied per chunk
     const int Cin = CONV ? a.K / 9 : a.K;                  // 3x3: reduction index k = tap * Cin + channel, Cin % 16 == 0
     // this pair's tiles: pair, pair + npairs, ...; tile t = (row pair t % nrp, column tile t / nrp)
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
@@ -168,7 +222,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         for (int u = 0; u < SUB; ++u) {
             if (u >= nsub) break;
             uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
-            bulk_load(smem_u32(chunk), W16 + ((size_t)(row0 / rpc) * nchunk + c0 + u) * (2 * T3_A_PART), 2 * T3_A_PART, bar);
+            bulk_load(smem_u32(chunk), W16 + ((size_t)(row0 / rpc) * nchunk + c0 + u) * (NP * T3_A_PART), NP * T3_A_PART, bar);
         }
     };
     auto issue_x = [&](int sg, int st, int xcol) {
@@ -179,7 +233,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             if (u >= nsub) break;
             const int c = c0 + u;
             uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
-            tma_load_2d(smem_u32(chunk + 2 * T3_A_PART + 2 * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
+            tma_load_2d(smem_u32(chunk + NP * T3_A_PART + NP * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
         }
     };
     // stages whose weight copies start before the wait for the previous kernel
@@ -248,7 +302,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             // ---------------- leader: MMA issuer for the pair (whole warp converged, one elected lane issues)
             const uint32_t idesc = make_idesc3(N);
             const uint64_t dW0 = make_desc(smem_u32(smem), 16, 256, SWZ_32B);
-            const uint64_t dX0 = make_desc(smem_u32(smem) + 2 * T3_A_PART, 2048, 1024, SWZ_128B);
+            const uint64_t dX0 = make_desc(smem_u32(smem) + NP * T3_A_PART, 2048, 1024, SWZ_128B);
             const uint32_t stage_u = stage_bytes >> 4, chunk_u = chunk_bytes >> 4;
             int st = 0;
             uint32_t ph = 0;
@@ -271,9 +325,16 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                     const int nsub = nchunk - sg * SUB < SUB ? nchunk - sg * SUB : SUB;
 #pragma unroll
                     for (int u = 0; u < SUB; ++u)
-                        if (u < nsub) ready = mma3_chunk(acc, dW0 + soff + (uint64_t)(u * chunk_u), dX0 + soff + (uint64_t)(u * chunk_u),
-                                           T3_A_PART >> 4, xb >> 4, idesc, (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
-                                           smem_u32(&bar_empty[st]), u == nsub - 1 ? 1u : 0u);
+                        if (u < nsub) {
+                            if constexpr (NP == 3)
+                                ready = mma6_chunk(acc, dW0 + soff + (uint64_t)(u * chunk_u), dX0 + soff + (uint64_t)(u * chunk_u),
+                                                   T3_A_PART >> 4, xb >> 4, idesc, (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
+                                                   smem_u32(&bar_empty[st]), u == nsub - 1 ? 1u : 0u);
+                            else
+                                ready = mma3_chunk(acc, dW0 + soff + (uint64_t)(u * chunk_u), dX0 + soff + (uint64_t)(u * chunk_u),
+                                                   T3_A_PART >> 4, xb >> 4, idesc, (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
+                                                   smem_u32(&bar_empty[st]), u == nsub - 1 ? 1u : 0u);
+                        }
                     st = nst; ph = nph;
                 }
                 if (!ok) break;
@@ -339,8 +400,8 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 #pragma unroll
             for (int u = 0; u < SUB; ++u) {
                 if (u >= nsub) break;
-                uint8_t *x1 = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes + 2 * T3_A_PART;
-                const uint8_t *raw = x1 + 2 * xb;
+                uint8_t *x1 = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes + NP * T3_A_PART;
+                const uint8_t *raw = x1 + NP * xb;
                 int sh = 0;
                 uint32_t ok8 = 0xffu;
                 if (CONV) {
@@ -371,11 +432,19 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 #pragma unroll
                             for (int e = 0; e < 8; ++e) if (!((ok8 >> e) & 1u)) v[e] = 0.f;
                         }
-                        uint4 h, l;
-                        split8(v, h, l);
                         const uint32_t off = dst + (uint32_t)k * 128u + ((c16 ^ ((uint32_t)k & 7u)) << 4);
-                        *reinterpret_cast<uint4 *>(x1 + off) = h;
-                        *reinterpret_cast<uint4 *>(x1 + xb + off) = l;
+                        if constexpr (NP == 3) {
+                            uint4 p1, p2, p3;
+                            split8x3(v, p1, p2, p3);
+                            *reinterpret_cast<uint4 *>(x1 + off) = p1;
+                            *reinterpret_cast<uint4 *>(x1 + xb + off) = p2;
+                            *reinterpret_cast<uint4 *>(x1 + 2 * xb + off) = p3;
+                        } else {
+                            uint4 h, l;
+                            split8(v, h, l);
+                            *reinterpret_cast<uint4 *>(x1 + off) = h;
+                            *reinterpret_cast<uint4 *>(x1 + xb + off) = l;
+                        }
                     }
                 }
             }
@@ -436,21 +505,24 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 // tmX: plain 2-D fp32 map (column, channel), box (ntile/2 + 2 halo) x 16; halo = 0 for 1x1, image width + 1
 // rounded up to a multiple of 4 for 3x3 (columns = the flattened (b, y, x) axis).
 int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, int halo, const void *args_,
-                        int M, int64_t Nc, int ntile, int sms, void *stream)
+                        int M, int64_t Nc, int ntile, int sms, void *stream, int pieces)
 {
     TcArgs a = *static_cast<const TcArgs *>(args_);
     a.ntile = ntile;
     const int nh = ntile / 2;
+    if (pieces != 2 && !(pieces == 3 && !conv)) return UBP_E_UNSUPPORTED;
     // chunks per stage: two on long reductions (48 chunks and more), else one
-    const int sub = (a.K + TC_KC - 1) / TC_KC >= 48 && t3_stages(nh, halo, 2) >= 4 ? 2 : 1;
-    size_t smem = (size_t)t3_stages(nh, halo, sub) * t3_stage_bytes(nh, halo, sub) + 1024;
+    const int sub = pieces == 2 && (a.K + TC_KC - 1) / TC_KC >= 48 && t3_stages(nh, halo, 2, pieces) >= 4 ? 2 : 1;
+    if (t3_stages(nh, halo, sub, pieces) < 4) return UBP_E_UNSUPPORTED;
+    size_t smem = (size_t)t3_stages(nh, halo, sub, pieces) * t3_stage_bytes(nh, halo, sub, pieces) + 1024;
     if (smem < TC_PAIR_MIN_SMEM) smem = TC_PAIR_MIN_SMEM;   // one CTA per SM, whatever the tile width (see the constant)
-    static bool done[4][64] = {};
+    static bool done[5][64] = {};
     int devid = 0;
     if (cudaGetDevice(&devid) != cudaSuccess) devid = -1;
-    const int which = (conv ? 2 : 0) + (sub == 2 ? 1 : 0);
+    const int which = pieces == 3 ? 4 : (conv ? 2 : 0) + (sub == 2 ? 1 : 0);
     using KernelFn = void (*)(const uint8_t *, const CUtensorMap, const TcArgs, const int, const int, const int);
-    const KernelFn kernels[4] = {ubp_tc3_kernel<false, 1>, ubp_tc3_kernel<false, 2>, ubp_tc3_kernel<true, 1>, ubp_tc3_kernel<true, 2>};
+    const KernelFn kernels[5] = {ubp_tc3_kernel<false, 1, 2>, ubp_tc3_kernel<false, 2, 2>, ubp_tc3_kernel<true, 1, 2>,
+                                 ubp_tc3_kernel<true, 2, 2>, ubp_tc3_kernel<false, 1, 3>};
     const KernelFn kern = kernels[which];
     if (devid < 0 || devid >= 64 || !done[which][devid]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(T3_PIPE_BUDGET + 1024));
@@ -484,6 +556,6 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
 }
 
 // how many pipeline stages the bf16 pair kernel gets for a tile width and halo
-int tc_pair_bf16_stages(int ntile, int halo) { return t3_stages(ntile / 2, halo, 1); }
+int tc_pair_bf16_stages(int ntile, int halo) { return t3_stages(ntile / 2, halo, 1, 2); }
 
 }  // namespace ubp

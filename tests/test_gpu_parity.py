@@ -171,6 +171,25 @@ def test_spmm_tensor_core_variant(env, M, C, Nb, p, Nc, variant):
         assert err <= 2e-5               # far inside its worst-case bound on random data
 
 
+@pytest.mark.parametrize("M,C,Nb,p,Nc,variant", [(256, 256, 4, 70, 4128, 86), (300, 150, 4, 70, 544, 86), (520, 200, 8, 50, 1028, 87),
+                                                  (128, 128, 4, 60, 4100, 86), (72, 144, 8, 50, 8196, 87), (257, 33, 1, 60, 260, 84),
+                                                  (512, 512, 2, 80, 6272, 85)])
+def test_spmm_three_piece_variant(env, M, C, Nb, p, Nc, variant):
+    """The bf16 CTA-pair kernel with every operand in three bf16 pieces and six products per fp32 product (variants
+    84..87): the dropped terms are below 2^-23 |w||x|, so what is left is the tensor core's fp32 accumulation (it
+    truncates): inside 2^-22 + (L + 2) 2^-23, about 1-2 * 10^-6 of |Wm||X| on random data -- closer to the oracle than
+    the two-piece form, not as close as the fp32 FMA kernel (3 * 10^-7), whose roundings are to nearest."""
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 10 * M + C, Nc=Nc, x_dist="normal", relu=(M % 2 == 0))
+    Yh, Yref, A, plan = run_spmm(env, L, variant)
+    assert plan.variant == variant and plan.tile_choice(Nc)[0] == 2
+    assert np.isfinite(Yh).all()
+    err = scaled_error(Yh, Yref, A)
+    n = terms_per_output(L) + 2
+    assert err <= 2.0 ** -22 + n * 2.0 ** -23 and err <= 3e-6
+    Y2, _, _, _ = run_spmm(env, L, variant - 50)                 # the two-piece form of the same layer
+    assert scaled_error(Y2, Yref, A) > err
+
+
 def test_tensor_core_variant_ragged_unaligned_and_auto(env):
     torch, ubp = env
     # ragged last strip on the fast path, then operands the fast path cannot take (falls back to the embedded
