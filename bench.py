@@ -105,6 +105,7 @@ def tf32_peak_tflops():
 NCU_DRAM_BYTES_PER_LAUNCH = {
     ("mbv1_pw512", 36): 13936896 + 0,            # the 12.8 MB output is still in L2 when the kernel ends
     ("sweep_nb4_p70", 36): 84903936 + 40135680,
+    ("r50_3x3", 64): 15389696 + 131840,
     ("r50_3x3", 44): 15257344 + 1280,            # the per-tap kernel
     ("mbv1_pw512", 32): 14984448 + 256,
     ("sweep_nb4_p70", 32): 124626432 + 48126208,
