@@ -192,6 +192,42 @@ __device__ __forceinline__ void c3_epilogue(const TcArgs &a, const C3Geom &g, ui
     }
 }
 
+// The same for the LAST tile of a pair, where nothing runs beside the epilogue and the weight ring is free to stage
+// in: units of 32 positions, a row of the unit per store instruction (up to 128 contiguous bytes).
+constexpr uint32_t C3_EPI32_PITCH = 144;                     // bytes per staged row of 32 floats (conflict-free 16-byte writes)
+constexpr uint32_t C3_EPI32_STAGE = 32 * C3_EPI32_PITCH;     // per warp
+__device__ __forceinline__ void c3_epilogue32(const TcArgs &a, const C3Geom &g, uint32_t acc, int q, int first, int step,
+                                              int row0, int p0, int lane, uint8_t *stage)
+{
+    const int nunit = (g.N + 31) / 32;
+    const int total_real = (int)a.Nc;
+#pragma unroll 1
+    for (int cc = first; cc < nunit; cc += step) {
+        uint32_t r[32];
+        tmem_ld32(acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 32), r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        int before; bool real;
+        c3_pad_map(p0 + cc * 32 + lane, a.H, a.W, g.Pn, total_real, before, real);
+        const int col = (real && cc * 32 + lane < g.N) ? before : -1;
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+            *reinterpret_cast<uint4 *>(stage + lane * C3_EPI32_PITCH + v * 16) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+        __syncwarp();
+        if (col >= 0) {
+#pragma unroll 4
+            for (int rr = 0; rr < 32; ++rr) {
+                const int row = row0 + q * 32 + rr;
+                if (row < a.M) {
+                    float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI32_PITCH + lane * 4) + (a.bias ? __ldg(a.bias + row) : 0.f);
+                    if (a.relu) o = fmaxf(o, 0.f);
+                    a.Y[(size_t)row * a.ldy + col] = o;
+                }
+            }
+        }
+        __syncwarp();
+    }
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(C3_THREADS, 1)
 ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensorMap tmX, const TcArgs a, const C3Geom g)
 {
@@ -381,8 +417,8 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
         if (ok && nmy > 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int i = nmy - 1;
-            c3_epilogue(a, g, tmem_base + (uint32_t)(i & 1) * C3_ACC_COLS, warp & 3, 2 + ((warp - C3_FIRST_PASS) >> 2), 4,
-                        tile_row0(i), tile_p0(i), lane, 0u, rank, smem + (size_t)(warp - C3_FIRST_PASS) * C3_EPI_STAGE);
+            c3_epilogue32(a, g, tmem_base + (uint32_t)(i & 1) * C3_ACC_COLS, warp & 3, 2 + ((warp - C3_FIRST_PASS) >> 2), 4,
+                          tile_row0(i), tile_p0(i), lane, smem + (size_t)(8 + warp - C3_FIRST_PASS) * C3_EPI32_STAGE);
         }
     } else {
         // ---------------- epilogue warps: tile i's accumulator while the main loop works on tile i + 1
@@ -392,9 +428,12 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
             ok = mbar_wait_relaxed(smem_u32(&acc_full[b]), (uint32_t)(i >> 1) & 1u, &abort_flag);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const bool last = i == nmy - 1;
-            c3_epilogue(a, g, tmem_base + (uint32_t)b * C3_ACC_COLS, warp & 3, part, last ? 4 : 2, tile_row0(i), tile_p0(i), lane,
-                        last ? 0u : smem_u32(&acc_empty[b]), rank, smem + c3_off_epi(g) + (size_t)(warp - C3_FIRST_EPI) * C3_EPI_STAGE);
+            if (i == nmy - 1)       // the weight ring is free by now (every MMA has completed): stage the last tile there
+                c3_epilogue32(a, g, tmem_base + (uint32_t)b * C3_ACC_COLS, warp & 3, part, 4, tile_row0(i), tile_p0(i), lane,
+                              smem + (size_t)(warp - C3_FIRST_EPI) * C3_EPI32_STAGE);
+            else
+                c3_epilogue(a, g, tmem_base + (uint32_t)b * C3_ACC_COLS, warp & 3, part, 2, tile_row0(i), tile_p0(i), lane,
+                            smem_u32(&acc_empty[b]), rank, smem + c3_off_epi(g) + (size_t)(warp - C3_FIRST_EPI) * C3_EPI_STAGE);
         }
     }
     if (!ok && lane == 0) atomicExch(a.status, 1);
