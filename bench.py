@@ -470,6 +470,10 @@ def build_chained(ubp, torch, layers, variant):
             kw["stride"] = L.stride
             if L.R == 1:
                 kw["scratch"] = torch.empty(L.C * L.B * Ho * Wo, dtype=torch.float32, device="cuda")
+            else:       # stride-2 3x3: the phase planes (allocated here so that the launches can be captured in a graph)
+                need = ubp.load().ubp_conv3x3_strided_scratch(L.C, L.B, L.H, L.Wd, L.stride)
+                if need:
+                    kw["scratch"] = torch.empty(need // 4, dtype=torch.float32, device="cuda")
         runs.append(lambda fn=fn, plan=plan, x=x, bias=bias, relu=L.relu, y=y, kw=kw: fn(plan, x, bias, relu, out=y, **kw))
         plans.append(plan); keep.append((x, y, bias, kw)); outs.append(y)
     return plans, runs, keep

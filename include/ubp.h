@@ -280,6 +280,18 @@ int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, 
 int ubp_conv3x3_strided(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
                         int64_t in_stride_b, int64_t in_stride_c, const float *bias, int relu,
                         float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);
+/* ubp_conv3x3_strided_ws: ubp_conv3x3_strided with caller-provided scratch (device, 16-byte aligned, at least
+ *   ubp_conv3x3_strided_scratch(C, B, H, W, stride) bytes; that is 0 unless stride == 2). With it, a stride-2 layer
+ *   whose plan is a variant 64..67 and whose output is one [channel][batch, yo, xo] matrix runs the padded-grid CTA-pair
+ *   kernel: one extra kernel first writes the four phase planes of the input (even/odd rows x even/odd columns,
+ *   [4*C][B*Ho*Wo]) into the scratch, on which output (yo, xo) reads tap (dy, dx) at plane (dy != 1, dx != 1), position
+ *   (yo - [dy == 0], xo - [dx == 0]): every tap is a shift of 0 or -1 of one plane. scratch == NULL or other cases:
+ *   exactly ubp_conv3x3_strided. UBP_E_SPACE if the scratch is too small. (ubp_plan_tile_choice_conv with stride 2
+ *   answers for this call.) */
+size_t ubp_conv3x3_strided_scratch(int C, int B, int H, int Wd, int stride);
+int ubp_conv3x3_strided_ws(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
+                           int64_t in_stride_b, int64_t in_stride_c, void *scratch, size_t scratch_bytes,
+                           const float *bias, int relu, float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);
 size_t ubp_conv1x1_strided_scratch(int C, int B, int H, int Wd, int stride);
 int ubp_conv1x1_strided(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
                         int64_t in_stride_b, int64_t in_stride_c, void *scratch, size_t scratch_bytes,

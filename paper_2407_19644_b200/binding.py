@@ -70,6 +70,9 @@ def load():
     L.ubp_static_plan_capacity.restype = sz
     L.ubp_spmm_static.argtypes = [vp, sz, vp, i64, i64, vp, i32, vp, i64, vp]
     L.ubp_conv3x3_strided.argtypes = [vp, vp, i32, i32, i32, i32, i64, i64, vp, i32, vp, i64, i64, vp]
+    L.ubp_conv3x3_strided_scratch.restype = sz
+    L.ubp_conv3x3_strided_scratch.argtypes = [i32, i32, i32, i32, i32]
+    L.ubp_conv3x3_strided_ws.argtypes = [vp, vp, i32, i32, i32, i32, i64, i64, vp, sz, vp, i32, vp, i64, i64, vp]
     L.ubp_conv1x1_strided_scratch.restype = sz
     L.ubp_conv1x1_strided_scratch.argtypes = [i32, i32, i32, i32, i32]
     L.ubp_conv1x1_strided.argtypes = [vp, vp, i32, i32, i32, i32, i64, i64, vp, sz, vp, i32, vp, i64, i64, vp]
@@ -368,16 +371,24 @@ def ubp_conv1x1(plan: Plan, x, bias=None, relu: bool = False, out=None, layout: 
 
 
 def ubp_conv3x3_implicit(plan: Plan, x, bias=None, relu: bool = False, out=None, layout: str = "CNHW", stream=None,
-                         stride: int = 1):
-    """3x3 / pad 1 convolution on a plan built from an R = 9 blob (stride 1: the implicit-GEMM kernels; stride > 1:
-    one lane per output pixel)."""
+                         stride: int = 1, scratch=None):
+    """3x3 / pad 1 convolution on a plan built from an R = 9 blob. stride 2: the four phase planes of the input go to
+    `scratch` first (a float32 CUDA tensor of at least 4*C*B*Ho*Wo (+ row padding) elements; allocated here when not
+    given), then the padded-grid kernel runs on them where the plan and layout allow; other strides > 1: the one-CTA
+    tensor-core kernel or one lane per output pixel."""
     import torch
     B, H, Wd, sb, sc, out, osb, osc = _conv_args(plan, x, out, layout, stride)
     if stride != 1:
+        need = plan._lib.ubp_conv3x3_strided_scratch(plan.C, B, H, Wd, stride)
+        if scratch is None and need:
+            scratch = torch.empty(need // 4, dtype=torch.float32, device=x.device)
         with torch.cuda.device(x.device):
-            _chk(plan._lib.ubp_conv3x3_strided(plan.handle, _dev_ptr(x, "x"), B, H, Wd, stride, sb, sc,
-                                               _dev_ptr(bias, "bias", True), int(bool(relu)), _dev_ptr(out, "out"),
-                                               osb, osc, _stream_ptr(stream)), "ubp_conv3x3_strided")
+            _chk(plan._lib.ubp_conv3x3_strided_ws(plan.handle, _dev_ptr(x, "x"), B, H, Wd, stride, sb, sc,
+                                                  _dev_ptr(scratch, "scratch", True), scratch.numel() * 4 if scratch is not None else 0,
+                                                  _dev_ptr(bias, "bias", True), int(bool(relu)), _dev_ptr(out, "out"),
+                                                  osb, osc, _stream_ptr(stream)), "ubp_conv3x3_strided_ws")
+            if scratch is not None:
+                scratch.record_stream(torch.cuda.current_stream() if stream is None else stream)
         return out
     with torch.cuda.device(x.device):
         _chk(plan._lib.ubp_conv3x3_implicit(plan.handle, _dev_ptr(x, "x"), B, H, Wd, sb, sc,

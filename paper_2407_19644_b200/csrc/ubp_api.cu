@@ -324,7 +324,8 @@ int ubp_plan_tile_choice_conv(const ubp_plan_t *plan, int B, int H, int Wd, int 
     int sms = 148, devid = 0;
     if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
     int n = 0;
-    if (stride == 1 && ubp::cfg_conv3_shift(c) && ubp::conv3_pair_tile(plan->dims.M, plan->dims.C, B, H, Wd, sms, &n)) {
+    const int Hq = stride == 2 ? (H - 1) / 2 + 1 : H, Wq = stride == 2 ? (Wd - 1) / 2 + 1 : Wd;      // stride 2: phase planes
+    if ((stride == 1 || stride == 2) && ubp::cfg_conv3_shift(c) && ubp::conv3_pair_tile(plan->dims.M, plan->dims.C, B, Hq, Wq, sms, &n)) {
         *kernel = 4; *tile_rows = 256; *tile_cols = n;
         return UBP_OK;
     }
@@ -408,6 +409,31 @@ int ubp_conv3x3_strided(const ubp_plan_t *plan, const float *in, int B, int H, i
     if (in_stride_c < hw || out_stride_c < ohw || in_stride_b < 0 || out_stride_b < 0) return UBP_E_ARG;
     return ubp::launch_conv3x3(plan, in, B, H, Wd, in_stride_b, in_stride_c, bias, relu, out, out_stride_b,
                                out_stride_c, stream, stride);
+}
+
+size_t ubp_conv3x3_strided_scratch(int C, int B, int H, int Wd, int stride)
+{
+    return ubp::conv3x3_strided_scratch_bytes(C, B, H, Wd, stride);
+}
+
+int ubp_conv3x3_strided_ws(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
+                           int64_t in_stride_b, int64_t in_stride_c, void *scratch, size_t scratch_bytes,
+                           const float *bias, int relu, float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream)
+{
+    if (stride == 1 || !scratch)
+        return ubp_conv3x3_strided(plan, in, B, H, Wd, stride, in_stride_b, in_stride_c, bias, relu, out, out_stride_b,
+                                   out_stride_c, stream);
+    if (!plan || plan->magic != kPlanMagic) return UBP_E_ARG;
+    if (plan->dims.R != 9 || (plan->cfg.kind != 1 && plan->cfg.kind != 3)) return UBP_E_ARG;
+    if (stride < 1 || B < 0 || H <= 0 || Wd <= 0) return UBP_E_ARG;
+    if (B == 0) return UBP_OK;
+    if (!in || !out || ((uintptr_t)scratch & 15u) != 0) return UBP_E_ARG;
+    const int64_t hw = (int64_t)H * Wd;
+    const int64_t ohw = (int64_t)((H - 1) / stride + 1) * ((Wd - 1) / stride + 1);
+    if (in_stride_c < hw || out_stride_c < ohw || in_stride_b < 0 || out_stride_b < 0) return UBP_E_ARG;
+    if (scratch_bytes < ubp_conv3x3_strided_scratch(plan->dims.C, B, H, Wd, stride)) return UBP_E_SPACE;
+    return ubp::launch_conv3x3(plan, in, B, H, Wd, in_stride_b, in_stride_c, bias, relu, out, out_stride_b, out_stride_c,
+                               stream, stride, scratch, scratch_bytes);
 }
 
 size_t ubp_conv1x1_strided_scratch(int C, int B, int H, int Wd, int stride)

@@ -15,7 +15,8 @@
 //     descriptor may start at ANY position: the MMAs of tap (dy, dx) use start + 16 bytes x (halo + shift);
 //   * the weights of a channel group (nine taps x 8 KB per CTA, the plan's bf16 tiling indexed as chunk = tap * C/16 +
 //     group) come as one barrier phase of a two-stage ring; the leader issues the group's 27 MMAs back to back.
-// Roles per CTA (608 threads): warp 0 producer (TMA / bulk copies), warp 1 MMA issuer (leader CTA only), warp 2 spare,
+// Roles per CTA (608 threads): warp 0 weight producer (bulk copies), warp 1 MMA issuer (leader CTA only), warp 2 raw-row
+// producer (TMA),
 // warps 3-10 operand pass (they also tell the leader that this CTA's weights of the group have landed), warps 11-18
 // epilogue (tile i while the main loop works on tile i + 1; two accumulators). All waits are bounded; no load is
 // multicast.
@@ -37,10 +38,11 @@ using namespace tc;
 constexpr int C3_PASS_WARPS = 8, C3_EPI_WARPS = 8;
 constexpr int C3_FIRST_PASS = 3, C3_FIRST_EPI = C3_FIRST_PASS + C3_PASS_WARPS;
 constexpr int C3_THREADS = (C3_FIRST_EPI + C3_EPI_WARPS) * 32;          // 608
-constexpr int C3_MAX_XS = 3;                   // stages of raw rows and of built operands (one channel group each): 2 or 3
-constexpr int C3_WG = 2;                       // stages of the weight ring; a stage holds the nine taps of a channel group
+constexpr int C3_MAX_XS = 6;                   // stages of raw rows and of built operands (one group step each): 2 .. 6
+constexpr int C3_MAX_WG = 4;                   // stages of the weight ring; a stage holds the taps of one group step:
 constexpr uint32_t C3_W_BYTES = 2 * 128 * TC_KC * 2;                      // W1 + W2 of one (tap, group): 8 KB
-constexpr uint32_t C3_WG_BYTES = 9 * C3_W_BYTES;                          // 72 KB
+constexpr uint32_t C3_WRING_BYTES = 2 * 9 * C3_W_BYTES;                   // two stages of nine taps (stride 1) or four
+                                                                          // of at most four taps (stride 2): 144 KB
 constexpr uint32_t C3_ACC_COLS = 256;
 constexpr uint32_t C3_SWZ_32B = 6;
 
@@ -54,11 +56,31 @@ struct C3Geom {
     int ntiles;       // nrp x column tiles
     int Pn;           // padded positions in all: B (H+2) (W+2)
     int cg;           // channel groups: C / 16
+    int wg;           // weight stages: 2 (nine taps each) or, for stride 2, 4 (at most four taps each)
+    int s2;           // 1: stride 2 -- X holds the four phase planes (rows phase * C + channel), a tile's group steps are
+                      // (channel group, phase) and each phase has its own taps, all of them shifts of 0 or -1
 };
+// The taps of a group step and their shifts on the padded grid (row pitch Wp). Stride 1: all nine, shift (dy-1) Wp +
+// (dx-1). Stride 2: output (yo, xo) reads input (2 yo + dy - 1, 2 xo + dx - 1) = plane (dy != 1, dx != 1) at
+// (yo - [dy == 0], xo - [dx == 0]).
+__device__ __forceinline__ int c3_ntaps(int s2, int ph) { return !s2 ? 9 : (ph == 0 ? 1 : (ph == 3 ? 4 : 2)); }
+__device__ __forceinline__ void c3_tap(int s2, int ph, int t, int Wp, int &tap, int &shift)
+{
+    if (!s2) { tap = t; shift = (t / 3 - 1) * Wp + (t % 3 - 1); return; }
+    // phase = 2 * (dy != 1) + (dx != 1); taps of a phase in ascending order
+    int dy, dx;
+    if (ph == 0) { dy = 1; dx = 1; }
+    else if (ph == 1) { dy = 1; dx = t == 0 ? 0 : 2; }
+    else if (ph == 2) { dy = t == 0 ? 0 : 2; dx = 1; }
+    else { dy = t < 2 ? 0 : 2; dx = (t & 1) ? 2 : 0; }
+    tap = 3 * dy + dx;
+    shift = (dy == 0 ? -Wp : 0) + (dx == 0 ? -1 : 0);
+}
 __host__ __device__ inline uint32_t c3_raw_bytes(const C3Geom &g) { return (uint32_t)g.rawn * TC_KC * 4; }
 __host__ __device__ inline uint32_t c3_kg_bytes(const C3Geom &g) { return (uint32_t)g.E * 16; }                 // one k-group of x1 or x2
 __host__ __device__ inline uint32_t c3_op_bytes(const C3Geom &g) { return 4 * c3_kg_bytes(g); }                  // x1, x2 x two k-groups
-__host__ __device__ inline uint32_t c3_off_op(const C3Geom &) { return (uint32_t)C3_WG * C3_WG_BYTES; }
+__host__ __device__ inline uint32_t c3_wg_bytes(const C3Geom &g) { return C3_WRING_BYTES / (uint32_t)g.wg; }      // 72 or 36 KB
+__host__ __device__ inline uint32_t c3_off_op(const C3Geom &) { return C3_WRING_BYTES; }
 __host__ __device__ inline uint32_t c3_off_raw(const C3Geom &g) { return c3_off_op(g) + (uint32_t)g.xs * ((c3_op_bytes(g) + 127u) & ~127u); }
 __host__ __device__ inline uint32_t c3_off_epi(const C3Geom &g) { return c3_off_raw(g) + (uint32_t)g.xs * ((c3_raw_bytes(g) + 127u) & ~127u); }
 __host__ __device__ inline uint32_t c3_smem_bytes(const C3Geom &g) { return c3_off_epi(g) + 8u * 2560u; }          // 8 epilogue warps x 2.5 KB
@@ -236,20 +258,23 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     // identical layout in both CTAs: the multicast commits and the remote arrives address barriers by offset
     __shared__ __align__(8) uint64_t raw_full[C3_MAX_XS], raw_empty[C3_MAX_XS], g_full[C3_MAX_XS], g_empty[C3_MAX_XS],
-        wg_full[C3_WG], wg_empty[C3_WG], acc_full[2], acc_empty[2], bar_last;
+        wg_full[C3_MAX_WG], wg_empty[C3_MAX_WG], acc_full[2], acc_empty[2], bar_last;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();
-    const int N = g.N, NH = N / 2, Wp = a.W + 2, XS = g.xs;
+    const int N = g.N, NH = N / 2, Wp = a.W + 2, XS = g.xs, WG = g.wg;
+    const uint32_t wg_bytes = c3_wg_bytes(g);
     const int total_real = (int)a.Nc;
     const uint32_t kgb = c3_kg_bytes(g), op_stride = (c3_op_bytes(g) + 127u) & ~127u, raw_stride = (c3_raw_bytes(g) + 127u) & ~127u;
     const uint32_t off_op = c3_off_op(g), off_raw = c3_off_raw(g);
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
     const int nmy = pair < g.ntiles ? (g.ntiles - pair + npairs - 1) / npairs : 0;
     const int nchunk = 9 * g.cg;
-    const int G = nmy * g.cg;                              // channel-group steps of this pair
+    const int GT = g.s2 ? 4 * g.cg : g.cg;                 // group steps per tile: channel groups (x four phases)
+    const int G = nmy * GT;                                // group steps of this pair
+    const int Cin = g.cg * TC_KC;
     auto tile_row0 = [&](int i) { return (((pair + i * npairs) % g.nrp) * 2 + (int)rank) * 128; };
     auto tile_p0 = [&](int i) { return ((pair + i * npairs) / g.nrp) * N; };
     // first staged padded position of this CTA for tile i, and the (4-aligned) first real pixel its raw copy holds
@@ -270,7 +295,7 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
             mbar_init(smem_u32(&g_full[s]), 2 * C3_PASS_WARPS);          // used in the leader CTA only
             mbar_init(smem_u32(&g_empty[s]), 1);
         }
-        for (int s = 0; s < C3_WG; ++s) {
+        for (int s = 0; s < g.wg; ++s) {
             mbar_init(smem_u32(&wg_full[s]), 1);
             mbar_init(smem_u32(&wg_empty[s]), 1);
         }
@@ -296,32 +321,25 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
 
     bool ok = true;
     if (warp == 0) {
-        // ---------------- producer: raw rows of a channel group (one TMA copy, up to XS groups ahead) and the nine
-        // weight blocks of a group as ONE barrier phase (nine bulk copies), one group ahead
+        // ---------------- weight producer: the taps of a group step as ONE barrier phase (up to nine bulk copies), as far
+        // ahead as the ring has stages. (The raw rows have a producer of their own, warp 2: a single thread that
+        // served both rings issued a step's weights only after the previous step's had landed.)
         if (lane == 0) {
-            int raw_issued = 0;
             for (int gs = 0; gs < G && ok; ++gs) {
-                const int lim = gs + XS < G ? gs + XS : G;
-                for (; raw_issued < lim && ok; ++raw_issued) {
-                    const int xs = raw_issued % XS, use = raw_issued / XS;
-                    if (use > 0) ok = mbar_wait_relaxed(smem_u32(&raw_empty[xs]), (uint32_t)(use - 1) & 1u, &abort_flag);
-                    if (!ok) break;
-                    const uint32_t bar = smem_u32(&raw_full[xs]);
-                    mbar_expect_tx(bar, c3_raw_bytes(g));
-                    tma_load_2d(smem_u32(smem + off_raw + (size_t)xs * raw_stride), &tmX, tile_ra(raw_issued / g.cg),
-                                (raw_issued % g.cg) * TC_KC, bar);
-                }
-                if (!ok) break;
-                const int i = gs / g.cg, chg = gs % g.cg;
+                const int i = gs / GT, gl = gs % GT;
+                const int chg = g.s2 ? gl >> 2 : gl, ph = g.s2 ? gl & 3 : 0, nt = c3_ntaps(g.s2, ph);
                 const uint8_t *wrow = W16 + (size_t)(tile_row0(i) / 128) * nchunk * C3_W_BYTES;
-                const int s = gs % C3_WG, use = gs / C3_WG;
+                const int s = gs % WG, use = gs / WG;
                 if (use > 0) ok = mbar_wait_relaxed(smem_u32(&wg_empty[s]), (uint32_t)(use - 1) & 1u, &abort_flag);
                 if (!ok) break;
                 const uint32_t bar = smem_u32(&wg_full[s]);
-                mbar_expect_tx(bar, C3_WG_BYTES);
-                for (int tap = 0; tap < 9; ++tap)
-                    bulk_load(smem_u32(smem + (size_t)s * C3_WG_BYTES + (size_t)tap * C3_W_BYTES),
+                mbar_expect_tx(bar, (uint32_t)nt * C3_W_BYTES);
+                for (int t = 0; t < nt; ++t) {
+                    int tap, shift;
+                    c3_tap(g.s2, ph, t, Wp, tap, shift);
+                    bulk_load(smem_u32(smem + (size_t)s * wg_bytes + (size_t)t * C3_W_BYTES),
                               wrow + (size_t)(tap * g.cg + chg) * C3_W_BYTES, C3_W_BYTES, bar);
+                }
             }
         }
     } else if (warp == 1) {
@@ -336,21 +354,23 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
                     ok = mbar_wait(smem_u32(&acc_empty[b]), (uint32_t)((i >> 1) - 1) & 1u, &abort_flag);
                     if (!ok) break;
                 }
-                for (int chg = 0; chg < g.cg && ok; ++chg, ++gs) {
+                for (int gl = 0; gl < GT && ok; ++gl, ++gs) {
                     // the operand of the group is built in both CTAs and both have the group's weights
-                    const int xs = gs % XS, wgs = gs % C3_WG;
+                    const int xs = gs % XS, wgs = gs % WG;
                     ok = mbar_wait(smem_u32(&g_full[xs]), (uint32_t)(gs / XS) & 1u, &abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t op = smem_u32(smem + off_op + (size_t)xs * op_stride);
-                    const uint32_t wb = smem_u32(smem + (size_t)wgs * C3_WG_BYTES);
-#pragma unroll
-                    for (int tap = 0; tap < 9; ++tap) {
-                        const int shift = (tap / 3 - 1) * Wp + (tap % 3 - 1);
-                        const uint64_t dW = make_desc(wb + (uint32_t)tap * C3_W_BYTES, 16, 256, C3_SWZ_32B);
+                    const uint32_t wb = smem_u32(smem + (size_t)wgs * wg_bytes);
+                    const int ph = g.s2 ? gl & 3 : 0, nt = c3_ntaps(g.s2, ph);
+#pragma unroll 3
+                    for (int t = 0; t < nt; ++t) {
+                        int tap, shift;
+                        c3_tap(g.s2, ph, t, Wp, tap, shift);
+                        const uint64_t dW = make_desc(wb + (uint32_t)t * C3_W_BYTES, 16, 256, C3_SWZ_32B);
                         const uint64_t dX = make_desc(op + (uint32_t)(g.halo + shift) * 16u, kgb, 128, SWZ_NONE);
-                        c3_mma_step(acc, dW, dX, (C3_W_BYTES / 2) >> 4, (2 * kgb) >> 4, idesc, (chg | tap) ? 1u : 0u,
-                                    smem_u32(&wg_empty[wgs]), smem_u32(&g_empty[xs]), tap == 8 ? 1u : 0u);
+                        c3_mma_step(acc, dW, dX, (C3_W_BYTES / 2) >> 4, (2 * kgb) >> 4, idesc, (gl | t) ? 1u : 0u,
+                                    smem_u32(&wg_empty[wgs]), smem_u32(&g_empty[xs]), t == nt - 1 ? 1u : 0u);
                     }
                 }
                 if (!ok) break;
@@ -359,7 +379,20 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
             }
         }
     } else if (warp == 2) {
-        // (spare warp)
+        // ---------------- raw-row producer: one TMA copy per group step (16 channel rows of the real pixels the CTA's
+        // staged positions cover), XS steps ahead
+        if (lane == 0) {
+            for (int r = 0; r < G && ok; ++r) {
+                const int xs = r % XS, use = r / XS;
+                if (use > 0) ok = mbar_wait_relaxed(smem_u32(&raw_empty[xs]), (uint32_t)(use - 1) & 1u, &abort_flag);
+                if (!ok) break;
+                const uint32_t bar = smem_u32(&raw_full[xs]);
+                mbar_expect_tx(bar, c3_raw_bytes(g));
+                const int rl = r % GT;                     // group step inside its tile
+                tma_load_2d(smem_u32(smem + off_raw + (size_t)xs * raw_stride), &tmX, tile_ra(r / GT),
+                            g.s2 ? (rl & 3) * Cin + (rl >> 2) * TC_KC : rl * TC_KC, bar);
+            }
+        }
     } else if (warp < C3_FIRST_EPI) {
         // ---------------- operand pass: once per channel group, raw fp32 rows of the real pixels -> x1, x2 (bf16) for
         // every staged padded position, K-major without swizzle: [x1 k-group 0][x1 k-group 1][x2 0][x2 1], position e of
@@ -369,7 +402,7 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
         int src[2] = {-1, -1};
         int cur_tile = -1;
         for (int gs = 0; gs < G && ok; ++gs) {
-            const int i = gs / g.cg;
+            const int i = gs / GT;
             if (i != cur_tile) {                           // new tile: where in the raw copy each of my positions comes from
                 cur_tile = i;
                 const int qa = tile_qa(i), ra = tile_ra(i);
@@ -401,7 +434,7 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the writes visible to the MMA unit
             // this CTA's weights of the group must have landed too before the leader may issue the group's MMAs
-            ok = mbar_wait_relaxed(smem_u32(&wg_full[gs % C3_WG]), (uint32_t)(gs / C3_WG) & 1u, &abort_flag);
+            ok = mbar_wait_relaxed(smem_u32(&wg_full[gs % WG]), (uint32_t)(gs / WG) & 1u, &abort_flag);
             if (!ok) break;
             __syncwarp();
             if (lane == 0) {
@@ -451,9 +484,9 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
 }  // namespace
 
 // Tile width for a launch: the padded positions per tile (a multiple of 16) that gives the pairs the fewest, cheapest
-// rounds. A step (tap, channel group) costs its three MMAs (1.5 cycles per position) or, for narrow tiles, what the
-// weight copy and the operand reads of shared memory need (about 380 cycles); a tile adds its epilogue.
-static bool c3_geometry(int M, int C, int B, int H, int W, int sms, C3Geom *out)
+// rounds. A step (tap, channel group) costs its three MMAs (about 1.6 cycles per position) or, for narrow tiles, what
+// the copy of its 8 KB of weights needs at the L2 -> SM rate (about 260 cycles); a tile adds its epilogue.
+static bool c3_geometry(int M, int C, int B, int H, int W, int sms, int s2, C3Geom *out)
 {
     if (C % TC_KC != 0 || M <= 128) return false;
     const long long Pn = (long long)B * (H + 2) * (W + 2);
@@ -463,7 +496,7 @@ static bool c3_geometry(int M, int C, int B, int H, int W, int sms, C3Geom *out)
     const int pairs_max = sms / 2;
     for (int n = 256; n >= 64; n -= 16) {
         C3Geom g{};
-        g.N = n; g.halo = W + 3; g.cg = C / TC_KC; g.Pn = (int)Pn; g.nrp = (M + 255) / 256;
+        g.N = n; g.halo = W + 3; g.cg = C / TC_KC; g.Pn = (int)Pn; g.nrp = (M + 255) / 256; g.s2 = s2;
         g.E = (n / 2 + 2 * g.halo + 7) & ~7;
         if (g.E > 256) continue;
         g.rawn = (g.E + 4 + 3) & ~3;
@@ -471,12 +504,14 @@ static bool c3_geometry(int M, int C, int B, int H, int W, int sms, C3Geom *out)
         const long long tiles = (long long)g.nrp * ((Pn + n - 1) / n);
         if (tiles > 0x7fffffffll) continue;
         g.ntiles = (int)tiles;
-        g.xs = C3_MAX_XS;
-        if (c3_smem_bytes(g) > 224u * 1024u) g.xs = 2;
+        // stride 2 has four times the group steps with a quarter of the MMAs each: deeper rings hide the hand-offs
+        g.wg = s2 ? 4 : 2;
+        g.xs = s2 ? C3_MAX_XS : 3;
+        while (g.xs > 2 && c3_smem_bytes(g) > 224u * 1024u) --g.xs;
         if (c3_smem_bytes(g) > 224u * 1024u) continue;
         const long long pairs = tiles < pairs_max ? tiles : pairs_max;
         const long long rounds = (tiles + pairs - 1) / pairs;
-        const double step = 1.5 * n > 380.0 ? 1.5 * n : 380.0;
+        const double step = 1.6 * n > 260.0 ? 1.6 * n : 260.0;      // three MMAs, or the 8 KB of weights at the L2 -> SM rate
         const double cost = (double)rounds * (9.0 * g.cg * step + 25.0 * n + 2500.0);
         if (cost < best_cost) { best_cost = cost; best = g; }
     }
@@ -489,19 +524,20 @@ static bool c3_geometry(int M, int C, int B, int H, int W, int sms, C3Geom *out)
 bool conv3_pair_tile(int M, int C, int B, int H, int W, int sms, int *tile_cols)
 {
     C3Geom g;
-    if (!c3_geometry(M, C, B, H, W, sms, &g)) return false;
+    if (!c3_geometry(M, C, B, H, W, sms, 0, &g)) return false;
     if (tile_cols) *tile_cols = g.N;
     return true;
 }
 
 // Launch on tiles of 256 rows x N padded positions. X: the input as one [C][B*H*W] matrix (rows 16-byte aligned, row
-// stride isc floats); W16: the plan's bf16 part (8 KB blocks [128-row tile][chunk = tap * C/16 + group]).
+// stride isc floats); s2: X is instead the four phase planes of a stride-2 layer, [4*C][B*H*W] with H x W the OUTPUT
+// plane (launch_phase_planes below writes them), and a.H, a.W, a.Nc describe that plane; W16: the plan's bf16 part (8 KB blocks [128-row tile][chunk = tap * C/16 + group]).
 // Returns UBP_E_UNSUPPORTED when the layer does not fit this kernel (the caller then uses the per-tap kernel).
 int launch_conv3_pair(const void *W16, const float *X, int64_t isc, const void *args_, int M, int C, int B, int H, int W,
-                      int sms, void *stream)
+                      int sms, void *stream, int s2)
 {
     C3Geom g;
-    if (!c3_geometry(M, C, B, H, W, sms, &g)) return UBP_E_UNSUPPORTED;
+    if (!c3_geometry(M, C, B, H, W, sms, s2, &g)) return UBP_E_UNSUPPORTED;
     TcArgs a = *static_cast<const TcArgs *>(args_);
     a.ntile = g.N;
     typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -516,7 +552,7 @@ int launch_conv3_pair(const void *W16, const float *X, int64_t isc, const void *
         enc = reinterpret_cast<EncodeTiledFn>(p);
     }
     CUtensorMap tmX;
-    const cuuint64_t dims[2] = {(cuuint64_t)a.Nc, (cuuint64_t)C};
+    const cuuint64_t dims[2] = {(cuuint64_t)a.Nc, (cuuint64_t)(s2 ? 4 * C : C)};
     const cuuint64_t strides[1] = {(cuuint64_t)isc * 4};
     const cuuint32_t box[2] = {(cuuint32_t)g.rawn, TC_KC};
     const cuuint32_t estr[2] = {1, 1};
@@ -551,6 +587,49 @@ int launch_conv3_pair(const void *W16, const float *X, int64_t isc, const void *
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, ubp_conv3_kernel, static_cast<const uint8_t *>(W16), tmX, a, g);
     if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+    return UBP_OK;
+}
+
+// Stride 2: the four phase planes of the input, P[2 py + px][c][b][yo][xo] = in[b][c][2 yo + py][2 xo + px] (zero
+// outside the image), as a matrix of 4*C rows of `ld` floats: on them every tap of the strided 3x3 is a shift of 0 or
+// -1 of one plane.
+// One CTA per (channel, image): the plane comes in by rows (coalesced), goes out as four contiguous pieces of
+// Ho x Wo floats, one per phase.
+__global__ void __launch_bounds__(256) ubp_phase_planes_kernel(const float *__restrict__ in, int C, int B, int H, int Wd,
+                                                                int64_t isb, int64_t isc, int Ho, int Wo, int64_t ld,
+                                                                float *__restrict__ out)
+{
+    extern __shared__ float plane[];                          // [H][Wd]
+    const int c = blockIdx.x, b = blockIdx.y;
+    const float *src = in + (size_t)b * isb + (size_t)c * isc;
+    const int hw = H * Wd, ohw = Ho * Wo;
+    for (int i = threadIdx.x; i < hw; i += 256) plane[i] = __ldg(src + i);
+    __syncthreads();
+    for (int ph = 0; ph < 4; ++ph) {
+        float *dst = out + ((size_t)ph * C + c) * ld + (size_t)b * ohw;
+        for (int i = threadIdx.x; i < ohw; i += 256) {
+            const int yo = i / Wo, xo = i - yo * Wo;
+            const int y = 2 * yo + (ph >> 1), x = 2 * xo + (ph & 1);
+            dst[i] = (y < H && x < Wd) ? plane[y * Wd + x] : 0.f;
+        }
+    }
+}
+
+int launch_phase_planes(const float *in, int C, int B, int H, int Wd, int64_t isb, int64_t isc, float *out, int64_t ld,
+                        void *stream)
+{
+    const int Ho = (H - 1) / 2 + 1, Wo = (Wd - 1) / 2 + 1;
+    if (B == 0 || C == 0) return UBP_OK;
+    const size_t smem = (size_t)H * Wd * sizeof(float);
+    if (B > 65535 || smem > 200 * 1024) return UBP_E_UNSUPPORTED;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(ubp_phase_planes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
+    }
+    ubp_phase_planes_kernel<<<dim3((unsigned)C, (unsigned)B), 256, smem, static_cast<cudaStream_t>(stream)>>>(
+        in, C, B, H, Wd, isb, isc, Ho, Wo, ld, out);
+    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
     return UBP_OK;
 }

@@ -107,7 +107,10 @@ int launch_conv3x3_tc(const ubp_plan *plan, const float *in, int B, int H, int W
 // tensor-core implicit GEMM when the plan and the layouts allow it (stride 1: CTA pairs where the operands qualify;
 // stride > 1: the one-CTA kernel, whose loaders gather the taps pixel by pixel); else one lane per output pixel
 int launch_conv3x3(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
-                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream, int stride = 1);
+                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream, int stride = 1,
+                   void *scratch = nullptr, size_t scratch_bytes = 0);
+// bytes of scratch the stride-2 3x3 fast path needs (phase planes), 0 for other strides
+size_t conv3x3_strided_scratch_bytes(int C, int B, int H, int Wd, int stride);
 int launch_subsample(const float *in, int C, int B, int H, int Wd, int64_t isb, int64_t isc, int stride, float *out,
                      void *stream);
 // the paper's dataflow on the canonical arrays (ubp_wros.cu): variants 60 (weight rotation) and 61 (naive shift)
@@ -115,7 +118,10 @@ int launch_wros(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, c
                 int64_t ldy, void *stream);
 // 3x3 on the padded pixel grid, taps as descriptor shifts (ubp_conv3.cu); UBP_E_UNSUPPORTED when the layer does not fit
 int launch_conv3_pair(const void *W16, const float *X, int64_t isc, const void *args, int M, int C, int B, int H, int W,
-                      int sms, void *stream);
+                      int sms, void *stream, int s2 = 0);
+// stride 2: the four phase planes of the input as a [4*C][ld] matrix (ubp_conv3.cu)
+int launch_phase_planes(const float *in, int C, int B, int H, int Wd, int64_t isb, int64_t isc, float *out, int64_t ld,
+                        void *stream);
 bool conv3_pair_tile(int M, int C, int B, int H, int W, int sms, int *tile_cols);
 void set_last_cuda_error(int e);
 }

@@ -23,6 +23,7 @@
 #include <mutex>
 
 #include "ubp_internal.h"
+#include "ubp_tc_common.cuh"
 
 namespace ubp {
 
@@ -759,13 +760,42 @@ int launch_spmm(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, con
     return UBP_E_UNSUPPORTED;
 }
 
+size_t conv3x3_strided_scratch_bytes(int C, int B, int H, int Wd, int stride)
+{
+    if (stride != 2 || C <= 0 || B <= 0 || H <= 0 || Wd <= 0) return 0;
+    const int64_t cols = (int64_t)B * ((H - 1) / 2 + 1) * ((Wd - 1) / 2 + 1);
+    return (size_t)4 * C * ((cols + 3) & ~(int64_t)3) * sizeof(float);
+}
+
 int launch_conv3x3(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
-                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream_, int stride)
+                   const float *bias, int relu, float *out, int64_t osb, int64_t osc, void *stream_, int stride,
+                   void *scratch, size_t scratch_bytes)
 {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const KernelCfg &c = pl->cfg;
     const int64_t ohw = (int64_t)((H - 1) / stride + 1) * ((Wd - 1) / stride + 1);
     const int64_t total = (int64_t)B * ohw;
+    // stride 2 with scratch: gather the four phase planes, then the padded-grid kernel with every tap a shift of one plane
+    if (stride == 2 && scratch && cfg_conv3_shift(c) && osb == ohw && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && osc % 4 == 0 &&
+        osc >= total && total < (1ll << 30) && (reinterpret_cast<uintptr_t>(scratch) & 15) == 0 &&
+        scratch_bytes >= conv3x3_strided_scratch_bytes(pl->dims.C, B, H, Wd, 2)) {
+        const int Ho = (H - 1) / 2 + 1, Wo = (Wd - 1) / 2 + 1, C = pl->dims.C;
+        const int64_t ld = (total + 3) & ~(int64_t)3;
+        int sms = 148, devid = 0;
+        if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
+        int ncols = 0;
+        if (conv3_pair_tile(pl->dims.M, C, B, Ho, Wo, sms, &ncols)) {
+            float *planes = static_cast<float *>(scratch);
+            if (int rc = launch_phase_planes(in, C, B, H, Wd, isb, isc, planes, ld, stream_)) return rc;
+            tc::TcArgs a{};
+            a.X = planes; a.conv = 1; a.H = Ho; a.W = Wo; a.isb = ohw; a.isc = ld; a.stride = 1;
+            a.bias = bias; a.Y = out; a.ldy = osc; a.Nc = total; a.M = pl->dims.M; a.K = C * 9; a.relu = relu;
+            a.status = reinterpret_cast<int *>(pl->dev); a.rpc = 128;
+            const uint8_t *dev = static_cast<const uint8_t *>(pl->dev);
+            const int rc = launch_conv3_pair(dev + pl->img.tc16_off, planes, ld, &a, pl->dims.M, C, B, Ho, Wo, sms, stream_, 1);
+            if (rc != UBP_E_UNSUPPORTED) return rc;
+        }
+    }
     // tensor-core path: needs the output as one [M][B*Ho*Wo] matrix (batch stride = plane size) with 16-byte rows
     if (c.kind == 3 && osb == ohw && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && osc % 4 == 0 &&
         osc >= total && total < (1ll << 31) && (int64_t)B * H * Wd < (1ll << 31))
