@@ -351,8 +351,8 @@ int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d
 int tc_pair_stages(int ntile, int halo);
 // same pipeline with three bf16 products per fp32 product (ubp_tc3.cu)
 int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, int halo, const void *args,
-                        int M, int64_t Nc, int ntile, int sms, void *stream, int pieces);
-int tc_pair_bf16_stages(int ntile, int halo);
+                        int M, int64_t Nc, int ntile, int sms, void *stream, int pieces, int mt);
+int tc_pair_bf16_stages(int ntile, int halo, int mt = 1);
 
 // Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
 // Each candidate's time is estimated as (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost)
@@ -420,8 +420,23 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
             const double t = 4400.0 + (double)per_pair * per_tile + 4500.0 + 30.0 * n;
             if (t < best2) { best2 = t; best2_n = n; }
         }
+        int best2_rows = 256;
+        // bf16 1x1, rows in whole 512-row tiles, few enough tiles for one per pair: a pair may stack two 256-row MMA
+        // tiles on one staged activation tile (one copy and one split pass serve both; a chunk then brings two weight
+        // blocks and its six MMAs: measured ~585-605 cycles per chunk at 96 and 192 columns) instead of making two
+        // rounds; narrow stacked tiles lose against one round of wide plain ones, which the estimate reproduces
+        if (bf16 == 1 && !conv && ((M + 255) / 256) % 2 == 0) {
+            for (int n = 64; n <= 256; n += 32) {
+                const long long ntiles = (long long)((M + 511) / 512) * ((Nc + n - 1) / n);
+                if (ntiles > sms / 2 || tc_pair_bf16_stages(n, 0, 2) < 4) continue;
+                double per_chunk = 3.3 * n;
+                if (per_chunk < 600.0 + 0.33 * n) per_chunk = 600.0 + 0.33 * n;
+                const double t = 4400.0 + nchunk * per_chunk + 2500.0 + 4500.0 + 60.0 * n;
+                if (t < best2) { best2 = t; best2_n = n; best2_rows = 512; }
+            }
+        }
         // (three pieces exist on the pair kernel only: never weigh it against the one-CTA TF32 kernel)
-        if (best2_n && (best2 < best || bf16 == 2)) { *kernel = 2; *rows = 256; *cols = best2_n; }
+        if (best2_n && (best2 < best || bf16 == 2)) { *kernel = 2; *rows = best2_rows; *cols = best2_n; }
     }
 }
 
@@ -456,7 +471,8 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
         if ((rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)(a.conv ? K / 9 : K), (uint64_t)(a.conv ? a.isc : a.ldx) * 4,
                             (uint32_t)(best_n / 2 + 2 * halo), TC_KC, CU_TENSOR_MAP_SWIZZLE_NONE))) return rc;
         a.rpc = tc16_rows_per_cta(M);
-        return launch_tc_pair_bf16(dev + pl->img.tc16_off, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream, cfg_pieces(pl->cfg));
+        return launch_tc_pair_bf16(dev + pl->img.tc16_off, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream, cfg_pieces(pl->cfg),
+                                   rows / 256);
     }
     if (kernel == 2) {
         // Wh and Wl as one 3-D tensor (channel, row, part): one copy per chunk brings both

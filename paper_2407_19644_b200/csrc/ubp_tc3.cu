@@ -54,18 +54,22 @@ __host__ __device__ constexpr uint32_t t3_raw_bytes(int nh, int halo)
 }
 // one chunk's part of a stage
 // (np = pieces per operand: 2, or 3 for the variant whose products are exact to fp32's last bits)
-__host__ __device__ constexpr uint32_t t3_chunk_bytes(int nh, int halo, int np)
+// (mt = 256-row MMA tiles stacked on the same activation tile: each brings its own weight block)
+__host__ __device__ constexpr uint32_t t3_chunk_bytes(int nh, int halo, int np, int mt = 1)
 {
-    return (uint32_t)np * T3_A_PART + (uint32_t)np * t3_x_bytes(nh) + t3_raw_bytes(nh, halo);
+    return (uint32_t)(mt * np) * T3_A_PART + (uint32_t)np * t3_x_bytes(nh) + t3_raw_bytes(nh, halo);
 }
 // A stage holds `sub` chunks. With two, every barrier round trip (copies landed -> split pass -> MMA issue -> stage
 // free) serves 32 channels: fewer waits per channel, which pays on long reductions (3x3: 144 chunks; 1024 channels)
 // where the pass or the issue thread is the bound; with one, the pipeline fills and drains in finer steps, which
 // pays on short reductions (512 channels: 32 chunks).
-__host__ __device__ constexpr uint32_t t3_stage_bytes(int nh, int halo, int sub, int np) { return (uint32_t)sub * t3_chunk_bytes(nh, halo, np); }
-__host__ __device__ constexpr int t3_stages(int nh, int halo, int sub, int np)
+__host__ __device__ constexpr uint32_t t3_stage_bytes(int nh, int halo, int sub, int np, int mt = 1)
 {
-    const int s = (int)(T3_PIPE_BUDGET / t3_stage_bytes(nh, halo, sub, np));
+    return (uint32_t)sub * t3_chunk_bytes(nh, halo, np, mt);
+}
+__host__ __device__ constexpr int t3_stages(int nh, int halo, int sub, int np, int mt = 1)
+{
+    const int s = (int)(T3_PIPE_BUDGET / t3_stage_bytes(nh, halo, sub, np, mt));
     return (s > T3_MAX_STAGES ? T3_MAX_STAGES : s) / T3_XL_GROUPS * T3_XL_GROUPS;
 }
 
@@ -195,18 +199,23 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     const uint32_t rank = cluster_rank();
     const int N = a.ntile, NH = N / 2;                     // tile columns; columns whose X this CTA holds
     const uint32_t xb = t3_x_bytes(NH);                    // x1 (and x2) bytes per chunk
-    const uint32_t chunk_bytes = t3_chunk_bytes(NH, halo, NP), stage_bytes = (uint32_t)SUB * chunk_bytes;
+    // MT 256-row MMA tiles share the staged activations (MT = 2: the pair owns a tile of 512 rows, at most one per
+    // pair, its two accumulators side by side in tensor memory; the split pass then runs once for both)
+    const int MT = a.mt > 1 ? 2 : 1;
+    const uint32_t wbytes = (uint32_t)(MT * NP) * T3_A_PART;   // weight blocks at the head of a chunk
+    const uint32_t chunk_bytes = t3_chunk_bytes(NH, halo, NP, MT), stage_bytes = (uint32_t)SUB * chunk_bytes;
     const uint32_t raw_row = (uint32_t)(NH + 2 * halo) * 4;   // bytes per channel row of the raw copy
-    const int S = t3_stages(NH, halo, SUB, NP);
+    const int S = t3_stages(NH, halo, SUB, NP, MT);
     const int nchunk = (a.K + TC_KC - 1) / TC_KC;
     const int nstage = (nchunk + SUB - 1) / SUB;     // stages per tile; the last one may hold a single chunk
-    const uint32_t tx = NP * T3_A_PART + raw_row * TC_KC;  // bytes copied per chunk
+    const uint32_t tx = wbytes + raw_row * TC_KC;          // bytes copied per chunk
     const int Cin = CONV ? a.K / 9 : a.K;                  // 3x3: reduction index k = tap * Cin + channel, Cin % 16 == 0
     // this pair's tiles: pair, pair + npairs, ...; tile t = (row pair t % nrp, column tile t / nrp)
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
     const int nmy = pair < ntiles ? (ntiles - pair + npairs - 1) / npairs : 0;
     const int rpc = a.rpc ? a.rpc : 128;                   // output rows per CTA (fewer than 128 only for layers of <= 128 rows)
-    auto tile_row0 = [&](int i) { return (((pair + i * npairs) % nrp) * 2 + (int)rank) * rpc; };
+    // first row of this CTA in the tile's first MMA tile; MMA tile m of the tile starts 2 m rpc rows further on
+    auto tile_row0 = [&](int i) { return (((pair + i * npairs) % nrp) * 2 * MT + (int)rank) * rpc; };
     auto tile_col0 = [&](int i) { return (int64_t)((pair + i * npairs) / nrp) * N; };
 
     // one stage's copies (stage sg of a tile = chunks sg * SUB ...): per chunk the W1 / W2 block of this CTA's 128
@@ -222,7 +231,9 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         for (int u = 0; u < SUB; ++u) {
             if (u >= nsub) break;
             uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
-            bulk_load(smem_u32(chunk), W16 + ((size_t)(row0 / rpc) * nchunk + c0 + u) * (NP * T3_A_PART), NP * T3_A_PART, bar);
+            for (int m = 0; m < MT; ++m)
+                bulk_load(smem_u32(chunk + (uint32_t)m * (NP * T3_A_PART)),
+                          W16 + ((size_t)(row0 / rpc + 2 * m) * nchunk + c0 + u) * (NP * T3_A_PART), NP * T3_A_PART, bar);
         }
     };
     auto issue_x = [&](int sg, int st, int xcol) {
@@ -233,7 +244,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             if (u >= nsub) break;
             const int c = c0 + u;
             uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
-            tma_load_2d(smem_u32(chunk + NP * T3_A_PART + NP * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
+            tma_load_2d(smem_u32(chunk + wbytes + NP * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
         }
     };
     // stages whose weight copies start before the wait for the previous kernel
@@ -302,7 +313,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             // ---------------- leader: MMA issuer for the pair (whole warp converged, one elected lane issues)
             const uint32_t idesc = make_idesc3(N);
             const uint64_t dW0 = make_desc(smem_u32(smem), 16, 256, SWZ_32B);
-            const uint64_t dX0 = make_desc(smem_u32(smem) + NP * T3_A_PART, 2048, 1024, SWZ_128B);
+            const uint64_t dX0 = make_desc(smem_u32(smem) + wbytes, 2048, 1024, SWZ_128B);
             const uint32_t stage_u = stage_bytes >> 4, chunk_u = chunk_bytes >> 4;
             int st = 0;
             uint32_t ph = 0;
@@ -326,14 +337,19 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 #pragma unroll
                     for (int u = 0; u < SUB; ++u)
                         if (u < nsub) {
-                            if constexpr (NP == 3)
+                            if constexpr (NP == 3) {
                                 ready = mma6_chunk(acc, dW0 + soff + (uint64_t)(u * chunk_u), dX0 + soff + (uint64_t)(u * chunk_u),
                                                    T3_A_PART >> 4, xb >> 4, idesc, (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
                                                    smem_u32(&bar_empty[st]), u == nsub - 1 ? 1u : 0u);
-                            else
-                                ready = mma3_chunk(acc, dW0 + soff + (uint64_t)(u * chunk_u), dX0 + soff + (uint64_t)(u * chunk_u),
-                                                   T3_A_PART >> 4, xb >> 4, idesc, (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
-                                                   smem_u32(&bar_empty[st]), u == nsub - 1 ? 1u : 0u);
+                            } else {
+                                // every MMA tile of the stack on the same x1 / x2; the stage goes back after the last one
+                                for (int m = 0; m < MT; ++m)
+                                    ready = mma3_chunk(acc + (uint32_t)m * T3_ACC_COLS,
+                                                       dW0 + soff + (uint64_t)(u * chunk_u) + (uint64_t)((uint32_t)m * (NP * T3_A_PART) >> 4),
+                                                       dX0 + soff + (uint64_t)(u * chunk_u), T3_A_PART >> 4, xb >> 4, idesc,
+                                                       (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
+                                                       smem_u32(&bar_empty[st]), (u == nsub - 1 && m == MT - 1) ? 1u : 0u);
+                            }
                         }
                     st = nst; ph = nph;
                 }
@@ -400,7 +416,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 #pragma unroll
             for (int u = 0; u < SUB; ++u) {
                 if (u >= nsub) break;
-                uint8_t *x1 = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes + NP * T3_A_PART;
+                uint8_t *x1 = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes + wbytes;
                 const uint8_t *raw = x1 + NP * xb;
                 int sh = 0;
                 uint32_t ok8 = 0xffu;
@@ -470,8 +486,9 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         if (ok && nmy > 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int i = nmy - 1;
-            epilogue_blocks(a, tmem_base + (uint32_t)(i & 1) * T3_ACC_COLS, warp & 3, 2 + ((warp - 2) >> 2), 4, N,
-                            tile_row0(i), tile_col0(i), lane, 0u, rank);
+            for (int m = 0; m < MT; ++m)
+                epilogue_blocks(a, tmem_base + (uint32_t)((i & 1) + m) * T3_ACC_COLS, warp & 3, 2 + ((warp - 2) >> 2), 4, N,
+                                tile_row0(i) + 2 * m * rpc, tile_col0(i), lane, 0u, rank);
         }
     } else {
         // ---------------- epilogue warps: tile i's accumulator while the main loop works on tile i + 1
@@ -482,8 +499,9 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const bool last = i == nmy - 1;
-            epilogue_blocks(a, tmem_base + (uint32_t)b * T3_ACC_COLS, warp & 3, part, last ? 4 : 2, N, tile_row0(i),
-                            tile_col0(i), lane, last ? 0u : smem_u32(&bar_acc_empty[b]), rank);
+            for (int m = 0; m < MT; ++m)     // (a stack of two is always the pair's only, hence last, tile)
+                epilogue_blocks(a, tmem_base + (uint32_t)(b + m) * T3_ACC_COLS, warp & 3, part, last ? 4 : 2, N,
+                                tile_row0(i) + 2 * m * rpc, tile_col0(i), lane, last ? 0u : smem_u32(&bar_acc_empty[b]), rank);
         }
     }
     if (!ok && lane == 0) atomicExch(a.status, 1);
@@ -505,16 +523,20 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 // tmX: plain 2-D fp32 map (column, channel), box (ntile/2 + 2 halo) x 16; halo = 0 for 1x1, image width + 1
 // rounded up to a multiple of 4 for 3x3 (columns = the flattened (b, y, x) axis).
 int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, int halo, const void *args_,
-                        int M, int64_t Nc, int ntile, int sms, void *stream, int pieces)
+                        int M, int64_t Nc, int ntile, int sms, void *stream, int pieces, int mt)
 {
     TcArgs a = *static_cast<const TcArgs *>(args_);
     a.ntile = ntile;
+    a.mt = mt;
     const int nh = ntile / 2;
     if (pieces != 2 && !(pieces == 3 && !conv)) return UBP_E_UNSUPPORTED;
+    // tiles of 512 rows: two-piece 1x1 products of layers whose rows fill whole 512-row tiles, one tile per pair
+    if (mt != 1 && !(mt == 2 && pieces == 2 && !conv && ((M + 255) / 256) % 2 == 0 &&
+                     (long long)((M + 511) / 512) * ((Nc + ntile - 1) / ntile) <= sms / 2)) return UBP_E_UNSUPPORTED;
     // chunks per stage: two on long reductions (48 chunks and more), else one
-    const int sub = pieces == 2 && (a.K + TC_KC - 1) / TC_KC >= 48 && t3_stages(nh, halo, 2, pieces) >= 4 ? 2 : 1;
-    if (t3_stages(nh, halo, sub, pieces) < 4) return UBP_E_UNSUPPORTED;
-    size_t smem = (size_t)t3_stages(nh, halo, sub, pieces) * t3_stage_bytes(nh, halo, sub, pieces) + 1024;
+    const int sub = pieces == 2 && (a.K + TC_KC - 1) / TC_KC >= 48 && t3_stages(nh, halo, 2, pieces, mt) >= 4 ? 2 : 1;
+    if (t3_stages(nh, halo, sub, pieces, mt) < 4) return UBP_E_UNSUPPORTED;
+    size_t smem = (size_t)t3_stages(nh, halo, sub, pieces, mt) * t3_stage_bytes(nh, halo, sub, pieces, mt) + 1024;
     if (smem < TC_PAIR_MIN_SMEM) smem = TC_PAIR_MIN_SMEM;   // one CTA per SM, whatever the tile width (see the constant)
     static bool done[5][64] = {};
     int devid = 0;
@@ -534,7 +556,7 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
         if (per_sm != 1) return UBP_E_UNSUPPORTED;
         if (devid >= 0 && devid < 64) done[which][devid] = true;
     }
-    const int nrp = (M + 255) / 256;
+    const int nrp = (M + 256 * mt - 1) / (256 * mt);
     const long long ntiles = (long long)nrp * ((Nc + ntile - 1) / ntile);
     if (ntiles <= 0) return UBP_OK;
     if (ntiles > 0x7fffffffll) return UBP_E_UNSUPPORTED;
@@ -556,6 +578,6 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
 }
 
 // how many pipeline stages the bf16 pair kernel gets for a tile width and halo
-int tc_pair_bf16_stages(int ntile, int halo) { return t3_stages(ntile / 2, halo, 1, 2); }
+int tc_pair_bf16_stages(int ntile, int halo, int mt) { return t3_stages(ntile / 2, halo, 1, 2, mt); }
 
 }  // namespace ubp

@@ -168,6 +168,8 @@ struct TcArgs {
     int *status;             // plan status word
     int rpc;                 // CTA-pair kernels: output rows per CTA (128; fewer when the layer has at most 128 rows
                              // and the pair splits them evenly); 0 means 128
+    int mt;                  // bf16 CTA-pair kernel: 256-row MMA tiles a pair stacks on ONE staged activation tile
+                             // (1, or 2 = tiles of 512 rows, one per pair); 0 means 1
 };
 
 
