@@ -188,7 +188,12 @@ int ubp_plan_tile_choice_conv(const ubp_plan_t *plan, int B, int H, int Wd, int 
 
 /* Read the plan's device status word: blocks until `stream` has finished
  * (cudaStreamSynchronize), then returns UBP_OK or UBP_E_DEVICE if a kernel
- * launched with this plan gave up on a bounded wait. */
+ * launched with this plan gave up on a bounded wait (word = 1).
+ * The checked build of the library (compiled with -DUBP_DEBUG: libubp_b200_debug.so, same entry points) also
+ * compares every index its kernels take from the plan or compute for shared or global memory with the extent
+ * it has to stay in; a failing check sets the word (2: shared memory or plan contents, 3: global memory), the
+ * access is skipped, the kernel runs to its end and this call reports UBP_E_DEVICE. Nothing traps in either
+ * build. */
 int ubp_plan_check(const ubp_plan_t *plan, void *stream);
 
 /* ubp_plan_clear_status: reset the plan's device status word to 0 (one 4-byte cudaMemsetAsync on `stream`). */

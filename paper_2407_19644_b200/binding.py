@@ -8,7 +8,8 @@ from typing import Optional, Tuple
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libubp_b200.so")
+# UBP_B200_LIBRARY names another build of the same library to load instead (the checked build, libubp_b200_debug.so)
+_LIB_PATH = os.environ.get("UBP_B200_LIBRARY") or os.path.join(_HERE, "libubp_b200.so")
 _lib = None
 
 

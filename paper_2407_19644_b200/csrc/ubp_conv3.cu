@@ -200,7 +200,7 @@ __device__ __forceinline__ void c3_epilogue(const TcArgs &a, const C3Geom &g, ui
                 if (row < a.M) {
                     float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI_PITCH + jpos * 4) + (a.bias ? __ldg(a.bias + row) : 0.f);
                     if (a.relu) o = fmaxf(o, 0.f);
-                    a.Y[(size_t)row * a.ldy + col] = o;
+                    if (UBP_CHK_GMEM(col < total_real, a.status)) a.Y[(size_t)row * a.ldy + col] = o;
                 }
             }
         }
@@ -242,7 +242,7 @@ __device__ __forceinline__ void c3_epilogue32(const TcArgs &a, const C3Geom &g, 
                 if (row < a.M) {
                     float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI32_PITCH + lane * 4) + (a.bias ? __ldg(a.bias + row) : 0.f);
                     if (a.relu) o = fmaxf(o, 0.f);
-                    a.Y[(size_t)row * a.ldy + col] = o;
+                    if (UBP_CHK_GMEM(col < total_real, a.status)) a.Y[(size_t)row * a.ldy + col] = o;
                 }
             }
         }
@@ -424,6 +424,9 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
             for (int u = 0; u < 2; ++u) {
                 const int e = l + 128 * u;
                 if (e >= g.E) break;
+                // (checked build: the source column lies in the raw copy, the stage inside the CTA's shared memory)
+                if (!UBP_CHK_SMEM(src[u] < g.rawn && (size_t)(smem - smem_raw) + off_op + (size_t)(xs + 1) * op_stride <= tc::dbg_dynamic_smem() &&
+                                  (size_t)(smem - smem_raw) + off_raw + (size_t)xs * raw_stride + c3_raw_bytes(g) <= tc::dbg_dynamic_smem(), a.status)) break;
                 float v[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) v[c] = src[u] >= 0 ? raw[(size_t)c * g.rawn + src[u]] : 0.f;
@@ -495,6 +498,9 @@ static bool c3_geometry(int M, int C, int B, int H, int W, int sms, int s2, C3Ge
     double best_cost = 1e300;
     const int pairs_max = sms / 2;
     for (int n = 256; n >= 64; n -= 16) {
+#ifdef C3_S2_FORCE_N
+        if (s2 && n != C3_S2_FORCE_N) continue;
+#endif
         C3Geom g{};
         g.N = n; g.halo = W + 3; g.cg = C / TC_KC; g.Pn = (int)Pn; g.nrp = (M + 255) / 256; g.s2 = s2;
         g.E = (n / 2 + 2 * g.halo + 7) & ~7;

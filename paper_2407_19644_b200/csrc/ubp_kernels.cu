@@ -340,7 +340,27 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
         const uint8_t *stage = smem + (size_t)st * a.stage_bytes;
         const uint8_t *grp = stage + XT_BYTES;
         const uint32_t po = reinterpret_cast<const uint32_t *>(grp)[wr];
-        const uint32_t pn = reinterpret_cast<const uint32_t *>(grp)[wr + 1];
+        uint32_t pn = reinterpret_cast<const uint32_t *>(grp)[wr + 1];
+#ifdef UBP_DEBUG
+        {
+            // checked build: the stage lies inside the CTA's shared memory; the panel's lists lie inside the stage, have
+            // exactly the length their entry count implies and ascending fragment offsets; every entry names a channel
+            // (K-runs: NBK channels) of the staged tile. A panel that fails is skipped.
+            int *status = reinterpret_cast<int *>(const_cast<uint8_t *>(a.plan));
+            bool good = UBP_CHK_SMEM((uint64_t)(st + 1) * a.stage_bytes <= tc::dbg_dynamic_smem() && po <= pn &&
+                                     pn <= a.stage_bytes - (uint32_t)XT_BYTES, status);
+            if (good && pn > po) {
+                const uint16_t *fo = reinterpret_cast<const uint16_t *>(grp + po);
+                const uint32_t n = fo[F];
+                good = UBP_CHK_SMEM(pn - po == (uint32_t)FO_BYTES + ((2u * (n + 4) + 15u) & ~15u) + ((4u * (n + 2) * WF + 15u) & ~15u), status);
+                for (int f = 0; good && f < F; ++f) good = UBP_CHK_SMEM(fo[f] <= fo[f + 1], status);
+                const uint16_t *jl = reinterpret_cast<const uint16_t *>(grp + po + FO_BYTES);
+                for (uint32_t e = lane; good && e < n; e += 32) good = UBP_CHK_SMEM((int)jl[e] + (KRUN ? NBK : 1) <= KT, status);
+                good = __all_sync(0xffffffffu, good);
+            }
+            if (!good) pn = po;
+        }
+#endif
         if (pn > po) {                               // panel exists in this group
             constexpr int FOW = FO_BYTES / 4;
             uint32_t fw[FOW];
@@ -382,6 +402,8 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
                     float4 o = make_float4(acc[r][2 * v].x + b, acc[r][2 * v].y + b,
                                            acc[r][2 * v + 1].x + b, acc[r][2 * v + 1].y + b);
                     if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                    if (!UBP_CHK_GMEM(col >= 0 && (col >= a.Nc || (size_t)row * a.ldy + col < (size_t)(a.M - 1) * a.ldy + a.Nc),
+                                      reinterpret_cast<int *>(const_cast<uint8_t *>(a.plan)))) continue;
                     if (col + 3 < a.Nc) {
                         *reinterpret_cast<float4 *>(yrow + col) = o;
                     } else {

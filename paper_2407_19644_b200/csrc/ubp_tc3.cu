@@ -426,7 +426,11 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                     chu += TC_KC;
                     if (chu >= Cin) { chu = 0; ++tpu; }
                 }
-                if (mine) {
+                // (checked build: the columns this thread needs lie inside the raw rows, everything it reads inside the
+                // CTA's shared memory, its writes inside the x1 / x2 tiles)
+                if (mine && UBP_CHK_SMEM(sh >= 0 && (uint32_t)(8 * cg + sh + 8) * 4u <= raw_row &&
+                                         (size_t)(raw - smem_raw) + 15u * raw_row + (uint32_t)((8 * cg + sh) & ~3) * 4u + 48u <= tc::dbg_dynamic_smem() &&
+                                         dst + 16u * 128u <= xb, a.status)) {
                     const int o = 8 * cg + sh, ob = o & ~3, r = o & 3;      // r is the same for every lane
 #pragma unroll
                     for (int i = 0; i < 2; ++i) {

@@ -150,6 +150,30 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 // fits beside the first.
 constexpr size_t TC_PAIR_MIN_SMEM = 118 * 1024;
 
+// ---------------------------------------------------------------- the checked build (-DUBP_DEBUG)
+// Every index that a kernel takes from the plan or computes for shared or global memory is compared with the extent it
+// has to stay in before it is used. A failing check sets the plan's status word (2: shared memory or plan contents,
+// 3: global memory; the first failure wins) and the access is skipped: nothing traps, the kernel runs to its end and
+// ubp_plan_check reports UBP_E_DEVICE. The ordinary build compiles the checks away.
+#ifdef UBP_DEBUG
+__device__ __forceinline__ bool dbg_check(bool ok, int *status, int code)
+{
+    if (!ok && status) atomicCAS(status, 0, code);
+    return ok;
+}
+__device__ __forceinline__ uint32_t dbg_dynamic_smem()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(r));
+    return r;
+}
+#define UBP_CHK_SMEM(ok, status) (::ubp::tc::dbg_check((ok), (status), 2))
+#define UBP_CHK_GMEM(ok, status) (::ubp::tc::dbg_check((ok), (status), 3))
+#else
+#define UBP_CHK_SMEM(ok, status) (true)
+#define UBP_CHK_GMEM(ok, status) (true)
+#endif
+
 struct TcArgs {
     const float *X;          // 1x1: [K][ldx]; 3x3: input tensor, element (b, c, y, x) at b*isb + c*isc + y*W + x
     int64_t ldx;
@@ -222,6 +246,9 @@ __device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&r)
 // lane quarter get equal shares of tile widths such as 192 or 224.)
 // `done_bar` != 0: once this warp's last tensor-memory read has completed, lane 0 arrives on that barrier of the
 // leader CTA (the accumulator may be overwritten from then on).
+// (checked build) last column a tile that starts at col0 may touch
+__device__ __forceinline__ int64_t tile_cols_end(int64_t col0, int N) { return col0 + N - 1; }
+
 __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, int q, int first, int step, int N,
                                                 int row0, int64_t col0, int lane, uint32_t done_bar, uint32_t rank)
 {
@@ -275,6 +302,7 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
                                                __uint_as_float(r[half][4 * j + 2 * h + 1]) + b);
                         if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); }
                         const int64_t col = cb + 8 * j;
+                        if (!UBP_CHK_GMEM(col >= 0 && row < a.M && (tile_cols_end(col0, N) >= col), a.status)) continue;
                         if (col + 1 < a.Nc) *reinterpret_cast<float2 *>(yrow + col) = o;
                         else if (col < a.Nc) yrow[col] = o.x;
                     }
@@ -301,6 +329,7 @@ __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, i
                                    : make_float4(__uint_as_float(p0x), __uint_as_float(p0y), __uint_as_float(gx), __uint_as_float(gy));
                     o.x += b; o.y += b; o.z += b; o.w += b;
                     if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                    if (!UBP_CHK_GMEM(cb >= 0 && row < a.M && (tile_cols_end(col0, N) >= cb + 3), a.status)) continue;
                     if (cb + 3 < a.Nc) *reinterpret_cast<float4 *>(yrow + cb) = o;
                     else {
                         if (cb < a.Nc) yrow[cb] = o.x;

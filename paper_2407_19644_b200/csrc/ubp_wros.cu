@@ -19,6 +19,7 @@
 #include <cstdint>
 
 #include "ubp_internal.h"
+#include "ubp_tc_common.cuh"
 
 namespace ubp {
 
@@ -33,6 +34,8 @@ struct WrosArgs {
     float *Y;
     int64_t ldy;
     int M, relu, rows_per_cta;
+    int C, m;                // input channels and blocks of the layer (what the checked build compares indices with)
+    int *status;             // plan status word
 };
 
 constexpr int WROS_THREADS = 128;
@@ -90,6 +93,7 @@ ubp_wros_kernel(const WrosArgs a)
                 if (tile < t_first || tile >= r1) continue;
                 const int b1 = __ldg(a.indptr + tile + 1);
                 for (int b = __ldg(a.indptr + tile); b < b1; ++b) {
+                    if (!UBP_CHK_GMEM(b >= 0 && b < a.m && (unsigned)__ldg(a.indices + b) < (unsigned)a.C, a.status)) break;
                     const float4 x = load_x<VEC>(a.X + (size_t)__ldg(a.indices + b) * a.ldx, col, a.Nc);
                     const float *v = a.values + (size_t)b * NB;
 #pragma unroll
@@ -104,6 +108,7 @@ ubp_wros_kernel(const WrosArgs a)
         for (int tile = t_first; tile < r1; ++tile) {
             const int b1 = __ldg(a.indptr + tile + 1);
             for (int b = __ldg(a.indptr + tile); b < b1; ++b) {
+                if (!UBP_CHK_GMEM(b >= 0 && b < a.m && (unsigned)__ldg(a.indices + b) < (unsigned)a.C, a.status)) break;
                 const float4 x = load_x<VEC>(a.X + (size_t)__ldg(a.indices + b) * a.ldx, col, a.Nc);
                 const float *v = a.values + (size_t)b * NB;
 #pragma unroll
@@ -146,6 +151,7 @@ int launch_wros(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, con
     a.indices = reinterpret_cast<const int32_t *>(dev + pl->img.wros_off[1]);
     a.values = reinterpret_cast<const float *>(dev + pl->img.wros_off[2]);
     a.X = X; a.ldx = ldx; a.Nc = Nc; a.bias = bias; a.Y = Y; a.ldy = ldy; a.M = pl->dims.M; a.relu = relu;
+    a.C = pl->dims.C; a.m = (int)pl->img.entries; a.status = static_cast<int *>(pl->dev);
     const int Nb = pl->dims.Nb;
     const int64_t strips = (Nc + 4 * WROS_THREADS - 1) / (4 * WROS_THREADS);
     if (strips > 0x7fffffffll) return UBP_E_UNSUPPORTED;
