@@ -600,24 +600,37 @@ int launch_conv3_pair(const void *W16, const float *X, int64_t isc, const void *
 // Stride 2: the four phase planes of the input, P[2 py + px][c][b][yo][xo] = in[b][c][2 yo + py][2 xo + px] (zero
 // outside the image), as a matrix of 4*C rows of `ld` floats: on them every tap of the strided 3x3 is a shift of 0 or
 // -1 of one plane.
-// One CTA per (channel, image): the plane comes in by rows (coalesced), goes out as four contiguous pieces of
-// Ho x Wo floats, one per phase.
+// One CTA per (four channels, image), no shared memory: a thread takes the pixel pair (y, 2 xo), (y, 2 xo + 1) of
+// each of the four planes (eight independent loads in flight) and writes them to phases 2 (y & 1) and 2 (y & 1) + 1 at
+// (y / 2, xo): reads and writes run along the image rows. (A CTA per plane that went through shared memory spent its
+// time on the load -> barrier -> store latency of 8192 tiny CTAs: 28 us for 51 MB.)
+constexpr int PP_CH = 4;
 __global__ void __launch_bounds__(256) ubp_phase_planes_kernel(const float *__restrict__ in, int C, int B, int H, int Wd,
                                                                 int64_t isb, int64_t isc, int Ho, int Wo, int64_t ld,
                                                                 float *__restrict__ out)
 {
-    extern __shared__ float plane[];                          // [H][Wd]
-    const int c = blockIdx.x, b = blockIdx.y;
-    const float *src = in + (size_t)b * isb + (size_t)c * isc;
-    const int hw = H * Wd, ohw = Ho * Wo;
-    for (int i = threadIdx.x; i < hw; i += 256) plane[i] = __ldg(src + i);
-    __syncthreads();
-    for (int ph = 0; ph < 4; ++ph) {
-        float *dst = out + ((size_t)ph * C + c) * ld + (size_t)b * ohw;
-        for (int i = threadIdx.x; i < ohw; i += 256) {
-            const int yo = i / Wo, xo = i - yo * Wo;
-            const int y = 2 * yo + (ph >> 1), x = 2 * xo + (ph & 1);
-            dst[i] = (y < H && x < Wd) ? plane[y * Wd + x] : 0.f;
+    const int c0 = (int)blockIdx.x * PP_CH, b = blockIdx.y;
+    const int items = 2 * Ho * Wo, ohw = Ho * Wo;
+    const float *src = in + (size_t)b * isb + (size_t)c0 * isc;
+    for (int i = threadIdx.x; i < items; i += 256) {
+        const int y = i / Wo, xo = i - y * Wo;
+        const int x = 2 * xo;
+        const bool in0 = y < H, in1 = in0 && x + 1 < Wd;
+        float v0[PP_CH], v1[PP_CH];
+#pragma unroll
+        for (int k = 0; k < PP_CH; ++k) {
+            const bool ch = c0 + k < C;
+            const float *p = src + (size_t)k * isc + (size_t)y * Wd + x;
+            v0[k] = (ch && in0) ? __ldg(p) : 0.f;
+            v1[k] = (ch && in1) ? __ldg(p + 1) : 0.f;
+        }
+        const int ph = (y & 1) * 2;
+        const size_t o = (size_t)b * ohw + (size_t)(y >> 1) * Wo + xo;
+#pragma unroll
+        for (int k = 0; k < PP_CH; ++k) {
+            if (c0 + k >= C) break;
+            out[((size_t)ph * C + c0 + k) * ld + o] = v0[k];
+            out[((size_t)(ph + 1) * C + c0 + k) * ld + o] = v1[k];
         }
     }
 }
@@ -627,13 +640,8 @@ int launch_phase_planes(const float *in, int C, int B, int H, int Wd, int64_t is
 {
     const int Ho = (H - 1) / 2 + 1, Wo = (Wd - 1) / 2 + 1;
     if (B == 0 || C == 0) return UBP_OK;
-    const size_t smem = (size_t)H * Wd * sizeof(float);
-    if (B > 65535 || smem > 200 * 1024) return UBP_E_UNSUPPORTED;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(ubp_phase_planes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
-    }
-    ubp_phase_planes_kernel<<<dim3((unsigned)C, (unsigned)B), 256, smem, static_cast<cudaStream_t>(stream)>>>(
+    if (B > 65535 || (int64_t)2 * Ho * Wo >= (1ll << 30)) return UBP_E_UNSUPPORTED;
+    ubp_phase_planes_kernel<<<dim3((unsigned)((C + PP_CH - 1) / PP_CH), (unsigned)B), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         in, C, B, H, Wd, isb, isc, Ho, Wo, ld, out);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }

@@ -264,7 +264,7 @@ struct SpmmArgs {
 // almost never blocks. Each stage has a "full" mbarrier (completed by the copies' byte count) and an "empty"
 // one (one arrival per warp).
 template <int NBK, int P, int V, int WR, int WC, int KT, bool DUPW, bool KRUN>
-__global__ void __launch_bounds__(WR * WC * 32, 1)
+__global__ void __launch_bounds__(WR * WC * 32, WR * WC <= 8 ? 2 : 1)
 ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
 {
     constexpr int CS = WC * 128 * V;               // columns per CTA
@@ -663,6 +663,10 @@ static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t 
     int stages = (int)(kSmemBudget / stage_bytes);
     if (stages < 2) return UBP_E_UNSUPPORTED;
     if (stages > 5) stages = 5;
+    // Eight-warp configurations (layers of at most 64 rows): two CTAs per SM with three stages each hide the latency of
+    // the entry loop and of the stores better than one CTA with five.
+    constexpr bool kTwoPerSm = WR * WC <= 8;
+    if (kTwoPerSm && stages >= 3 && 3 * stage_bytes <= 110 * 1024) stages = 3;
 
     EncodeTiledFn enc = encode_fn();
     if (!enc) return UBP_E_CUDA;
@@ -695,7 +699,7 @@ static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t 
     const int nstrips = (int)((Nc + CS - 1) / CS);
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    int gy = sms / pl->img.NG;
+    int gy = (kTwoPerSm && stages == 3 ? 2 * sms : sms) / pl->img.NG;
     if (gy < 1) gy = 1;
     if (gy > nstrips) gy = nstrips;
     // even out the strips per CTA: with k strips each at most, do not launch more CTAs than needed for that k
@@ -831,19 +835,25 @@ int launch_conv3x3(const ubp_plan *pl, const float *in, int B, int H, int Wd, in
 }
 
 // Every stride-th pixel of every stride-th row of each input plane, into a dense channel-major tensor
-// [C][B][Ho][Wo]: the activations a strided 1x1 convolution reads.
+// [C][B][Ho][Wo]: the activations a strided 1x1 convolution reads. One CTA per (four channels, image); a thread takes
+// output pixels (yo, xo) of the four planes: four independent loads in flight, one 32-bit division per pixel.
+constexpr int SUBS_CH = 4;
 __global__ void __launch_bounds__(256) ubp_subsample_kernel(const float *__restrict__ in, int C, int B, int H, int Wd,
                                                              int64_t isb, int64_t isc, int stride, int Ho, int Wo,
                                                              float *__restrict__ out)
 {
-    const int64_t total = (int64_t)C * B * Ho * Wo;
-    for (int64_t n = (int64_t)blockIdx.x * 256 + threadIdx.x; n < total; n += (int64_t)gridDim.x * 256) {
-        const int xo = (int)(n % Wo);
-        const int64_t r1 = n / Wo;
-        const int yo = (int)(r1 % Ho);
-        const int64_t r2 = r1 / Ho;
-        const int b = (int)(r2 % B), c = (int)(r2 / B);
-        out[n] = in[(size_t)b * isb + (size_t)c * isc + (size_t)(yo * stride) * Wd + (size_t)xo * stride];
+    const int c0 = (int)blockIdx.x * SUBS_CH, b = blockIdx.y;
+    const int ohw = Ho * Wo;
+    const float *src = in + (size_t)b * isb + (size_t)c0 * isc;
+    for (int i = threadIdx.x; i < ohw; i += 256) {
+        const int yo = i / Wo, xo = i - yo * Wo;
+        const size_t off = (size_t)(yo * stride) * Wd + (size_t)xo * stride;
+        float v[SUBS_CH];
+#pragma unroll
+        for (int k = 0; k < SUBS_CH; ++k) v[k] = c0 + k < C ? __ldg(src + (size_t)k * isc + off) : 0.f;
+#pragma unroll
+        for (int k = 0; k < SUBS_CH; ++k)
+            if (c0 + k < C) out[((size_t)(c0 + k) * B + b) * ohw + i] = v[k];
     }
 }
 
@@ -853,10 +863,9 @@ int launch_subsample(const float *in, int C, int B, int H, int Wd, int64_t isb, 
     const int Ho = (H - 1) / stride + 1, Wo = (Wd - 1) / stride + 1;
     const int64_t total = (int64_t)C * B * Ho * Wo;
     if (total == 0) return UBP_OK;
-    int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    ubp_subsample_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream_)>>>(in, C, B, H, Wd, isb, isc,
-                                                                                              stride, Ho, Wo, out);
+    if (B > 65535 || (int64_t)Ho * Wo >= (1ll << 30)) return UBP_E_UNSUPPORTED;
+    ubp_subsample_kernel<<<dim3((unsigned)((C + SUBS_CH - 1) / SUBS_CH), (unsigned)B), 256, 0, static_cast<cudaStream_t>(stream_)>>>(
+        in, C, B, H, Wd, isb, isc, stride, Ho, Wo, out);
     return check(cudaGetLastError());
 }
 
