@@ -39,10 +39,9 @@ constexpr int C3_PASS_WARPS = 8, C3_EPI_WARPS = 8;
 constexpr int C3_FIRST_PASS = 3, C3_FIRST_EPI = C3_FIRST_PASS + C3_PASS_WARPS;
 constexpr int C3_THREADS = (C3_FIRST_EPI + C3_EPI_WARPS) * 32;          // 608
 constexpr int C3_MAX_XS = 6;                   // stages of raw rows and of built operands (one group step each): 2 .. 6
-constexpr int C3_MAX_WG = 4;                   // stages of the weight ring; a stage holds the taps of one group step:
+constexpr int C3_MAX_WG = 4;                   // stages of the weight ring; a stage holds the taps of one group step
+                                               // (nine, 72 KB; stride 2: at most six, 48 KB)
 constexpr uint32_t C3_W_BYTES = 2 * 128 * TC_KC * 2;                      // W1 + W2 of one (tap, group): 8 KB
-constexpr uint32_t C3_WRING_BYTES = 2 * 9 * C3_W_BYTES;                   // two stages of nine taps (stride 1) or four
-                                                                          // of at most four taps (stride 2): 144 KB
 constexpr uint32_t C3_ACC_COLS = 256;
 constexpr uint32_t C3_SWZ_32B = 6;
 
@@ -56,31 +55,39 @@ struct C3Geom {
     int ntiles;       // nrp x column tiles
     int Pn;           // padded positions in all: B (H+2) (W+2)
     int cg;           // channel groups: C / 16
-    int wg;           // weight stages: 2 (nine taps each) or, for stride 2, 4 (at most four taps each)
+    int wg;           // weight stages: 2 (nine taps each; stride 2: at most six taps each)
     int s2;           // 1: stride 2 -- X holds the four phase planes (rows phase * C + channel), a tile's group steps are
-                      // (channel group, phase) and each phase has its own taps, all of them shifts of 0 or -1
+                      // (channel group, phase pair {0, 1} or {2, 3}): a stage holds the raw rows and the operands of both
+                      // phases of the pair, and each phase has its own taps, all of them shifts of 0 or -1
 };
 // The taps of a group step and their shifts on the padded grid (row pitch Wp). Stride 1: all nine, shift (dy-1) Wp +
 // (dx-1). Stride 2: output (yo, xo) reads input (2 yo + dy - 1, 2 xo + dx - 1) = plane (dy != 1, dx != 1) at
 // (yo - [dy == 0], xo - [dx == 0]).
-__device__ __forceinline__ int c3_ntaps(int s2, int ph) { return !s2 ? 9 : (ph == 0 ? 1 : (ph == 3 ? 4 : 2)); }
-__device__ __forceinline__ void c3_tap(int s2, int ph, int t, int Wp, int &tap, int &shift)
+// (stride 2: `hf` = which phase pair; taps of phase 2 hf first, then those of phase 2 hf + 1; `sub` = which of the
+// stage's two operands the tap reads)
+__device__ __forceinline__ int c3_ntaps(int s2, int hf) { return !s2 ? 9 : (hf == 0 ? 3 : 6); }
+__device__ __forceinline__ void c3_tap(int s2, int hf, int t, int Wp, int &tap, int &shift, int &sub)
 {
-    if (!s2) { tap = t; shift = (t / 3 - 1) * Wp + (t % 3 - 1); return; }
+    if (!s2) { tap = t; shift = (t / 3 - 1) * Wp + (t % 3 - 1); sub = 0; return; }
     // phase = 2 * (dy != 1) + (dx != 1); taps of a phase in ascending order
     int dy, dx;
-    if (ph == 0) { dy = 1; dx = 1; }
-    else if (ph == 1) { dy = 1; dx = t == 0 ? 0 : 2; }
-    else if (ph == 2) { dy = t == 0 ? 0 : 2; dx = 1; }
-    else { dy = t < 2 ? 0 : 2; dx = (t & 1) ? 2 : 0; }
+    if (hf == 0) {
+        if (t == 0) { dy = 1; dx = 1; sub = 0; }                               // phase 0
+        else { dy = 1; dx = t == 1 ? 0 : 2; sub = 1; }                         // phase 1
+    } else {
+        if (t < 2) { dy = t == 0 ? 0 : 2; dx = 1; sub = 0; }                   // phase 2
+        else { dy = t < 4 ? 0 : 2; dx = (t & 1) ? 2 : 0; sub = 1; }            // phase 3
+    }
     tap = 3 * dy + dx;
     shift = (dy == 0 ? -Wp : 0) + (dx == 0 ? -1 : 0);
 }
-__host__ __device__ inline uint32_t c3_raw_bytes(const C3Geom &g) { return (uint32_t)g.rawn * TC_KC * 4; }
+__host__ __device__ inline uint32_t c3_raw1_bytes(const C3Geom &g) { return (uint32_t)g.rawn * TC_KC * 4; }      // one phase's raw rows
+__host__ __device__ inline uint32_t c3_raw_bytes(const C3Geom &g) { return (g.s2 ? 2u : 1u) * c3_raw1_bytes(g); }
 __host__ __device__ inline uint32_t c3_kg_bytes(const C3Geom &g) { return (uint32_t)g.E * 16; }                 // one k-group of x1 or x2
-__host__ __device__ inline uint32_t c3_op_bytes(const C3Geom &g) { return 4 * c3_kg_bytes(g); }                  // x1, x2 x two k-groups
-__host__ __device__ inline uint32_t c3_wg_bytes(const C3Geom &g) { return C3_WRING_BYTES / (uint32_t)g.wg; }      // 72 or 36 KB
-__host__ __device__ inline uint32_t c3_off_op(const C3Geom &) { return C3_WRING_BYTES; }
+__host__ __device__ inline uint32_t c3_op1_bytes(const C3Geom &g) { return 4 * c3_kg_bytes(g); }                 // x1, x2 x two k-groups
+__host__ __device__ inline uint32_t c3_op_bytes(const C3Geom &g) { return (g.s2 ? 2u : 1u) * c3_op1_bytes(g); }
+__host__ __device__ inline uint32_t c3_wg_bytes(const C3Geom &g) { return (g.s2 ? 6u : 9u) * C3_W_BYTES; }        // 72 or 48 KB
+__host__ __device__ inline uint32_t c3_off_op(const C3Geom &g) { return (uint32_t)g.wg * c3_wg_bytes(g); }
 __host__ __device__ inline uint32_t c3_off_raw(const C3Geom &g) { return c3_off_op(g) + (uint32_t)g.xs * ((c3_op_bytes(g) + 127u) & ~127u); }
 __host__ __device__ inline uint32_t c3_off_epi(const C3Geom &g) { return c3_off_raw(g) + (uint32_t)g.xs * ((c3_raw_bytes(g) + 127u) & ~127u); }
 __host__ __device__ inline uint32_t c3_smem_bytes(const C3Geom &g) { return c3_off_epi(g) + 8u * 2560u; }          // 8 epilogue warps x 2.5 KB
@@ -272,7 +279,9 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
     const int nmy = pair < g.ntiles ? (g.ntiles - pair + npairs - 1) / npairs : 0;
     const int nchunk = 9 * g.cg;
-    const int GT = g.s2 ? 4 * g.cg : g.cg;                 // group steps per tile: channel groups (x four phases)
+    const int GT = g.s2 ? 2 * g.cg : g.cg;                 // group steps per tile: channel groups (x two phase pairs)
+    const int NSUB = g.s2 ? 2 : 1;                         // phases (raw blocks, operands) per stage
+    const uint32_t raw1 = c3_raw1_bytes(g), op1 = c3_op1_bytes(g);
     const int G = nmy * GT;                                // group steps of this pair
     const int Cin = g.cg * TC_KC;
     auto tile_row0 = [&](int i) { return (((pair + i * npairs) % g.nrp) * 2 + (int)rank) * 128; };
@@ -327,7 +336,7 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
         if (lane == 0) {
             for (int gs = 0; gs < G && ok; ++gs) {
                 const int i = gs / GT, gl = gs % GT;
-                const int chg = g.s2 ? gl >> 2 : gl, ph = g.s2 ? gl & 3 : 0, nt = c3_ntaps(g.s2, ph);
+                const int chg = g.s2 ? gl >> 1 : gl, ph = g.s2 ? gl & 1 : 0, nt = c3_ntaps(g.s2, ph);
                 const uint8_t *wrow = W16 + (size_t)(tile_row0(i) / 128) * nchunk * C3_W_BYTES;
                 const int s = gs % WG, use = gs / WG;
                 if (use > 0) ok = mbar_wait_relaxed(smem_u32(&wg_empty[s]), (uint32_t)(use - 1) & 1u, &abort_flag);
@@ -335,8 +344,8 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
                 const uint32_t bar = smem_u32(&wg_full[s]);
                 mbar_expect_tx(bar, (uint32_t)nt * C3_W_BYTES);
                 for (int t = 0; t < nt; ++t) {
-                    int tap, shift;
-                    c3_tap(g.s2, ph, t, Wp, tap, shift);
+                    int tap, shift, sub;
+                    c3_tap(g.s2, ph, t, Wp, tap, shift, sub);
                     bulk_load(smem_u32(smem + (size_t)s * wg_bytes + (size_t)t * C3_W_BYTES),
                               wrow + (size_t)(tap * g.cg + chg) * C3_W_BYTES, C3_W_BYTES, bar);
                 }
@@ -362,13 +371,13 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t op = smem_u32(smem + off_op + (size_t)xs * op_stride);
                     const uint32_t wb = smem_u32(smem + (size_t)wgs * wg_bytes);
-                    const int ph = g.s2 ? gl & 3 : 0, nt = c3_ntaps(g.s2, ph);
+                    const int ph = g.s2 ? gl & 1 : 0, nt = c3_ntaps(g.s2, ph);
 #pragma unroll 3
                     for (int t = 0; t < nt; ++t) {
-                        int tap, shift;
-                        c3_tap(g.s2, ph, t, Wp, tap, shift);
+                        int tap, shift, sub;
+                        c3_tap(g.s2, ph, t, Wp, tap, shift, sub);
                         const uint64_t dW = make_desc(wb + (uint32_t)t * C3_W_BYTES, 16, 256, C3_SWZ_32B);
-                        const uint64_t dX = make_desc(op + (uint32_t)(g.halo + shift) * 16u, kgb, 128, SWZ_NONE);
+                        const uint64_t dX = make_desc(op + (uint32_t)sub * op1 + (uint32_t)(g.halo + shift) * 16u, kgb, 128, SWZ_NONE);
                         c3_mma_step(acc, dW, dX, (C3_W_BYTES / 2) >> 4, (2 * kgb) >> 4, idesc, (gl | t) ? 1u : 0u,
                                     smem_u32(&wg_empty[wgs]), smem_u32(&g_empty[xs]), t == nt - 1 ? 1u : 0u);
                     }
@@ -389,8 +398,9 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
                 const uint32_t bar = smem_u32(&raw_full[xs]);
                 mbar_expect_tx(bar, c3_raw_bytes(g));
                 const int rl = r % GT;                     // group step inside its tile
-                tma_load_2d(smem_u32(smem + off_raw + (size_t)xs * raw_stride), &tmX, tile_ra(r / GT),
-                            g.s2 ? (rl & 3) * Cin + (rl >> 2) * TC_KC : rl * TC_KC, bar);
+                for (int sub = 0; sub < NSUB; ++sub)       // stride 2: rows of phase 2 (rl & 1) + sub, channel group rl >> 1
+                    tma_load_2d(smem_u32(smem + off_raw + (size_t)xs * raw_stride + (size_t)sub * raw1), &tmX, tile_ra(r / GT),
+                                g.s2 ? (2 * (rl & 1) + sub) * Cin + (rl >> 1) * TC_KC : rl * TC_KC, bar);
             }
         }
     } else if (warp < C3_FIRST_EPI) {
@@ -418,8 +428,9 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
             ok = mbar_wait_relaxed(smem_u32(&raw_full[xs]), (uint32_t)use & 1u, &abort_flag);
             if (ok && use > 0) ok = mbar_wait_relaxed(smem_u32(&g_empty[xs]), (uint32_t)(use - 1) & 1u, &abort_flag);
             if (!ok) break;
-            const float *raw = reinterpret_cast<const float *>(smem + off_raw + (size_t)xs * raw_stride) + (size_t)(kg * 8) * g.rawn;
-            uint8_t *x1 = smem + off_op + (size_t)xs * op_stride + (size_t)kg * kgb;
+            for (int sub = 0; sub < NSUB; ++sub) {
+            const float *raw = reinterpret_cast<const float *>(smem + off_raw + (size_t)xs * raw_stride + (size_t)sub * raw1) + (size_t)(kg * 8) * g.rawn;
+            uint8_t *x1 = smem + off_op + (size_t)xs * op_stride + (size_t)sub * op1 + (size_t)kg * kgb;
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
                 const int e = l + 128 * u;
@@ -434,6 +445,7 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
                 c3_split8(v, h, lo);
                 *reinterpret_cast<uint4 *>(x1 + (size_t)e * 16) = h;
                 *reinterpret_cast<uint4 *>(x1 + 2 * kgb + (size_t)e * 16) = lo;
+            }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the writes visible to the MMA unit
             // this CTA's weights of the group must have landed too before the leader may issue the group's MMAs
@@ -498,9 +510,6 @@ static bool c3_geometry(int M, int C, int B, int H, int W, int sms, int s2, C3Ge
     double best_cost = 1e300;
     const int pairs_max = sms / 2;
     for (int n = 256; n >= 64; n -= 16) {
-#ifdef C3_S2_FORCE_N
-        if (s2 && n != C3_S2_FORCE_N) continue;
-#endif
         C3Geom g{};
         g.N = n; g.halo = W + 3; g.cg = C / TC_KC; g.Pn = (int)Pn; g.nrp = (M + 255) / 256; g.s2 = s2;
         g.E = (n / 2 + 2 * g.halo + 7) & ~7;
@@ -510,9 +519,9 @@ static bool c3_geometry(int M, int C, int B, int H, int W, int sms, int s2, C3Ge
         const long long tiles = (long long)g.nrp * ((Pn + n - 1) / n);
         if (tiles > 0x7fffffffll) continue;
         g.ntiles = (int)tiles;
-        // stride 2 has four times the group steps with a quarter of the MMAs each: deeper rings hide the hand-offs
-        g.wg = s2 ? 4 : 2;
-        g.xs = s2 ? C3_MAX_XS : 3;
+        // stride 2 has twice the group steps with half the MMAs each: deeper rings hide the hand-offs
+        g.wg = 2;
+        g.xs = s2 ? 4 : 3;
         while (g.xs > 2 && c3_smem_bytes(g) > 224u * 1024u) --g.xs;
         if (c3_smem_bytes(g) > 224u * 1024u) continue;
         const long long pairs = tiles < pairs_max ? tiles : pairs_max;
