@@ -43,7 +43,7 @@ WORKLOADS = {
     "r50_3x3": dict(cfg="r50_3x3", kw={}),
 }
 for _nb in (2, 4, 8, 16):
-    for _sp in (50, 70, 80, 90):
+    for _sp in (50, 70, 80, 90, 95):
         WORKLOADS[f"sweep_nb{_nb}_p{_sp}"] = dict(cfg="sweep", kw=dict(Nb=_nb, sparsity_pct=_sp))
 for _li in range(13):
     WORKLOADS[f"mbv1_L{_li + 1}"] = dict(cfg="mbv1_chain", kw={}, index=_li)
@@ -446,7 +446,8 @@ def workload_config(L, name, world, no_flush):
 
 
 # The other BASELINE configurations the default run measures beside the headline (every frac from the mean time)
-EXTRA_CONFIGS = ["r50_3x3", "sweep_nb2_p50", "sweep_nb16_p50", "sweep_nb4_p70", "sweep_nb2_p90", "sweep_nb16_p90"] + \
+EXTRA_CONFIGS = ["r50_3x3", "sweep_nb2_p50", "sweep_nb16_p50", "sweep_nb4_p70", "sweep_nb2_p90", "sweep_nb16_p90",
+                 "sweep_nb4_p95"] + \
                 [f"mbv1_L{i + 1}" for i in range(13)]
 # The headline layer through the other arithmetics: three bf16 pieces (six products), TF32 products, fp32 FMA on the CUDA cores
 HEADLINE_VARIANTS = [86, 32, 14]

@@ -146,8 +146,8 @@ void ubp_plan_free(ubp_plan_t *plan);
 
 /* Plans straight from a K-major blob (the forms of ubp_plan_size / ubp_plan_image / ubp_plan_build for the other
  * orientation; the handle reports the layer's own M and C, and ubp_spmm / ubp_conv1x1 take it like any other).
- * variant 0 chooses: the tensor-core kernel where it pays (at least 8 % of the weights kept, 128 output and 64 input
- * channels; the weight is densified, the orientation does not matter there), else the K-run sparse kernel
+ * variant 0 chooses: the tensor-core kernel where it pays (at least 3 % of the weights kept -- 0.5 % for layers of a
+ * million weights or more --, 128 output and 64 input channels; the weight is densified, the orientation does not matter there), else the K-run sparse kernel
  * (variants 70..73 for B = 2, 4, 8, 16): fp32 FMA, output rows stationary in registers, a plan entry = one run
  * (row, first channel, B weights), i.e. ONE channel index per B weights and B consecutive rows of the staged
  * activation tile per entry; a run that crosses a channel-tile boundary is cut there. Other run lengths fall back
@@ -224,7 +224,8 @@ int ubp_selftest_bounded_wait(const ubp_plan_t *plan, unsigned limit_us, void *s
  *     three products of the operands' TF32 heads and remainders, accumulated in fp32 in
  *     tensor memory: error <= 2^-18 |w||x| per product plus the accumulation;
  *   tensor-core kernels, bf16 products (34..37, the choice of variant 0 for layers with
- *     at least 8 % of the weights kept, 128 output and 64 input channels): three products
+ *     at least 3 % of the weights kept (0.5 % from a million weights on), 128 output and 64 input
+ *     channels): three products
  *     of bf16 heads and remainders, fp32 accumulation: error <= 3 * 2^-16 |w||x| per
  *     product in the worst case (about 2 * 10^-6 of |Wm||X| on random data).
  *   tensor-core kernel, three bf16 pieces (84..87): w = w1 + w2 + w3 and x = x1 + x2 + x3 exactly (8 + 8 + 8

@@ -210,7 +210,7 @@ static int resolve_kmajor(const ubp_view_t &kv, int variant, const ubp::KernelCf
     if (variant == 0) {
         const double dens = (double)kv.m * B / ((double)M * C);
         const int krun = B == 2 ? 70 : B == 4 ? 71 : B == 8 ? 72 : B == 16 ? 73 : 0;
-        if ((dens >= 0.08 && M >= 128 && C >= 64) || !krun) c = ubp::auto_cfg(M, C, 1, 1, (int64_t)kv.m * B);
+        if ((ubp::tensor_core_pays(M, C, dens) && M >= 128 && C >= 64) || !krun) c = ubp::auto_cfg(M, C, 1, 1, (int64_t)kv.m * B);
         else c = ubp::find_cfg(krun);
     } else {
         c = ubp::find_cfg(variant);

@@ -46,6 +46,16 @@ inline bool cfg_bf16(const KernelCfg &c)
     return (c.id >= 34 && c.id <= 37) || (c.id >= 44 && c.id <= 47) || cfg_conv3_shift(c) || cfg_pieces(c) == 3;
 }
 const KernelCfg *find_cfg(int id);
+// Whether the dense tensor-core form beats the sparse kernel for a layer with `dens` of its weights kept. Measured on
+// B200, launches back to back, blocks of 4: the tensor-core kernel takes the same time at every sparsity; the sparse
+// kernel re-stages the activations once per 128 output rows and pays a fixed cost per (panel, channel tile, start offset),
+// so it shrinks slowly: 512x512x6272 at 92 / 95 / 97 % sparsity 19.4 / 16.8 / 15.4 us against 16.7; 1024x1024x3136
+// 36.3 / 31.3 / 28.4 against 22.4; 2048x2048x8192 286 / 234 / 210 against 152; 256x256x50176 31.9 / 28.1 / 26.7 against
+// 25.7. Hence: from 3 % kept on, and for layers of a million weights or more from 0.5 % on.
+inline bool tensor_core_pays(int M, int C, double dens)
+{
+    return dens >= 0.03 || ((int64_t)M * C >= (1ll << 20) && dens >= 0.005);
+}
 // pick a configuration for a layer (variant == 0)
 const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m);
 

@@ -49,7 +49,7 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
     // shared-memory time, error <= 3 * 2^-16 |w||x|, inside the 1e-4 gate) is the default; the TF32-product ids stay
     // selectable (with at most 128 rows they run the one-CTA kernel).
     const int fast = 4;
-    if (R == 9 && dens >= 0.08 && M >= 128 && C >= 16) {    // implicit GEMM on tensor cores, taps as operand shifts
+    if (R == 9 && tensor_core_pays(M, C, dens) && M >= 128 && C >= 16) {    // implicit GEMM on tensor cores, taps as operand shifts
         switch (nbk) {
             case 16: case 8: return find_cfg(64);
             case 4: return find_cfg(65);
@@ -66,12 +66,11 @@ const KernelCfg *auto_cfg(int M, int C, int R, int Nb, int64_t m)
         }
     }
     if (R != 1) return nullptr;
-    // Dense tensor-core variant when enough of the weight survives and the layer is large enough to amortise its
-    // per-tile set-up: measured on B200 it takes the same time at every sparsity and beats the sparse kernel up to
-    // ~90 % sparsity on 2048 x 2048 x 8192. It pays from 128 rows and 64 input channels on (measured on the
+    // Dense tensor-core variant when enough of the weight survives (tensor_core_pays) and the layer is large enough
+    // to amortise its per-tile set-up: it pays from 128 rows and 64 input channels on (measured on the
     // MobileNet-shaped layers, launches back to back: 128 -> 128 channels 42 us against 60 us; 64 -> 128 channels 35
-    // against 39; 32 -> 64 channels 95 against 68, so below that the sparse kernel stays).
-    if (dens >= 0.08 && M >= 128 && C >= 64) {
+    // against 39; 32 -> 64 channels 95 against 54, so below that the sparse kernel stays).
+    if (tensor_core_pays(M, C, dens) && M >= 128 && C >= 64) {
         switch (nbk) {
             case 16: case 8: return find_cfg(33 + fast);
             case 4: return find_cfg(32 + fast);

@@ -167,7 +167,7 @@ CONFIGS = {
     "fc64": "FC 64x64, 1x4 blocks, 50 % sparsity, X 64x256 ~ N(0,1), bias, no ReLU",
     "mbv1_pw512": "pointwise 512->512 at 14x14, batch 32 (M=K=512, Nc=6272), 1x4, 70 %, bias+ReLU",
     "r50_3x3": "3x3 conv 256->256 at 14x14, batch 64, pad 1, blocks 8x1x3x3, 80 %",
-    "sweep": "M=K=2048, Nc=8192; Nb in {2,4,8,16} x sparsity in {50,70,80,90}",
+    "sweep": "M=K=2048, Nc=8192; Nb in {2,4,8,16} x sparsity in {50,70,80,90} (and 95: where the sparse kernel takes over)",
     "mbv1_chain": "13 pointwise layers of MobileNetV1, batch 64, 1x4, 80 %, bias+ReLU",
     "r50_bottleneck": "1x1 1024->256, 3x3 256->256, 1x1 256->1024 at 14x14, batch 32, blocks of 4, 80 %, chained",
     "r50_downsample": "downsampling bottleneck 28x28 -> 14x14: 1x1 512->256, 3x3 256->256 stride 2, 1x1 256->1024, and "
@@ -198,7 +198,8 @@ def config_layers(cfg: str, *, batch: Optional[int] = None, Nb: Optional[int] = 
     if cfg == "sweep":
         nb = 4 if Nb is None else Nb
         sp = 70 if sparsity_pct is None else sparsity_pct
-        idx = [2, 4, 8, 16].index(nb) * 4 + [50, 70, 80, 90].index(sp)
+        # (the 95 % points were added after the 4 x 4 grid: their seeds follow it)
+        idx = [2, 4, 8, 16].index(nb) * 4 + [50, 70, 80, 90].index(sp) if sp != 95 else 16 + [2, 4, 8, 16].index(nb)
         return [make_layer(f"sweep_nb{nb}_p{sp}", 2048, 2048, nb, sp, 4000 + idx, Nc=8192,
                            w_scale=0.02, x_dist="normal", bias=False, relu=False, make_x=make_x)]
     if cfg == "mbv1_chain":
