@@ -978,7 +978,10 @@ def main():
             del pc, Yc, Lc
             torch.cuda.empty_cache()
         chain = [r for r in line["configs"] if r["workload"].startswith("mbv1_L")]
-        line["configs_summary"] = {"min_frac": min(r["frac"] for r in line["configs"]),
+        worst = min(line["configs"], key=lambda r: r["frac"])
+        upto90 = [r for r in line["configs"] if r["sparsity_pct"] <= 90]
+        line["configs_summary"] = {"min_frac": worst["frac"], "min_frac_workload": worst["workload"],
+                                   "min_frac_up_to_90pct_sparsity": min(r["frac"] for r in upto90),
                                    "chain_us_sum": sum(r["us"] for r in chain),
                                    "chain_roofline_us_sum": sum(r["roofline_us"] for r in chain),
                                    "steps_each": esteps, "frac_from": "mean"}
