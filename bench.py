@@ -269,21 +269,21 @@ def time_region(torch, runs, steps, warmup, extra_regions=0, hold_s=0.0):
     return out
 
 
-def time_e2e(torch, ubp, plan, L, steps, warmup):
+def time_e2e(torch, ubp, plan, L, steps, warmup, nlanes=2):
     """Same step through the public call with HOST buffers: pinned X -> device, kernel, Y -> pinned host, every
     step. Steps alternate between two streams with their own device and host buffers, so that the upload of step
     i + 1 runs under the download of step i (PCIe is full duplex); the value is the steady-state rate."""
     bias = torch.from_numpy(L.bias).cuda() if L.bias is not None else None
     shape = (L.M, L.B, L.H, L.Wd) if L.X.ndim == 4 else (L.M, L.Nc)
     lanes = []
-    for _ in range(2):
+    for _ in range(nlanes):
         Xh = torch.from_numpy(L.X).pin_memory()
         lanes.append(dict(stream=torch.cuda.Stream(), Xh=Xh, Xd=torch.empty_like(Xh, device="cuda"),
                           Yd=torch.empty(shape, dtype=torch.float32, device="cuda"),
                           Yh=torch.empty(shape, dtype=torch.float32).pin_memory()))
 
     def step(i):
-        ln = lanes[i & 1]
+        ln = lanes[i % nlanes]
         with torch.cuda.stream(ln["stream"]):
             ln["Xd"].copy_(ln["Xh"], non_blocking=True)
             if L.R == 9:
@@ -294,7 +294,7 @@ def time_e2e(torch, ubp, plan, L, steps, warmup):
                 ubp.ubp_spmm(plan, ln["Xd"], bias, L.relu, out=ln["Yd"])
             ln["Yh"].copy_(ln["Yd"], non_blocking=True)
 
-    for i in range(max(warmup, 2)):
+    for i in range(max(warmup, nlanes)):
         step(i)
     torch.cuda.synchronize()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
