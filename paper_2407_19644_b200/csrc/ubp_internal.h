@@ -34,9 +34,6 @@ struct KernelCfg {
 };
 const std::vector<KernelCfg> &kernel_cfgs();
 // tensor-core variants whose CTA-pair kernel uses three bf16 products per fp32 product instead of three TF32 products
-// Output rows per CTA of the bf16 CTA-pair kernel: 128, or for layers of at most 128 rows half of them (rounded up to
-// a multiple of 8) so that both CTAs of the pair have rows to store.
-inline int tc16_rows_per_cta(int M) { return M > 128 ? 128 : (((M + 1) / 2 + 7) & ~7); }
 // 64..67: 3x3 with the taps as shifts of one staged operand on the padded pixel grid (ubp_conv3.cu; bf16 products too)
 inline bool cfg_conv3_shift(const KernelCfg &c) { return c.id >= 64 && c.id <= 67; }
 // 84..87: the bf16 CTA-pair kernel with every operand in THREE bf16 pieces (exact) and six products per fp32 product
@@ -78,9 +75,7 @@ struct PlanImage {
     int tc_kp = 0;
     // and of the same weight as two bf16 pieces (W1 = the weight rounded to bf16, W2 = the remainder rounded to bf16),
     // tiled: 8 KB blocks [row tile][chunk of 16 channels] = [piece][128 rows][16 channels] in the 32-byte swizzle;
-    // a row tile holds tc16_rows_per_cta(M) rows of the matrix (the rest of its 128 rows are zero), in order when that
-    // is 128, else a quarter of them at the start of each 32-row quarter of the tile (row positions = tensor-memory
-    // lanes of the accumulator; each epilogue warp reads one lane quarter);
+    // row tile t holds rows 128 t .. 128 t + 127 of the matrix in order (rows beyond M are zero; whole pairs of tiles);
     // tc16_kp = reduction length padded to whole chunks
     size_t tc16_off = 0;
     int tc16_kp = 0;

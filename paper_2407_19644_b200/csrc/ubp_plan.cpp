@@ -274,14 +274,9 @@ int build_plan_image(const ubp_view_t &v, const KernelCfg &cfg, bool count_only,
         // and into two bf16 pieces: the weight rounded to nearest-even bf16, and the (exact) remainder rounded
         uint8_t *W16 = base + img.tc16_off;
         const size_t nchunk16 = (size_t)img.tc16_kp / 16;
-        const int rpc16 = tc16_rows_per_cta(M);            // matrix rows per 128-row tile (64 when M = 128, ...)
         auto w16_at = [&](int row, size_t k, int piece) -> uint16_t * {
-            const size_t blk = (size_t)(row / rpc16) * nchunk16 + k / 16;
-            // position in the 128-row tile = tensor-memory lane of the output row: in order when the CTA has 128 rows;
-            // a quarter of the rows at the start of each 32-lane quarter when it has fewer, so that every epilogue warp
-            // (each reads one lane quarter) has rows to store
-            int i = row % rpc16;
-            if (rpc16 < 128) i = (i / (rpc16 / 4)) * 32 + i % (rpc16 / 4);
+            const size_t blk = (size_t)(row / 128) * nchunk16 + k / 16;
+            const int i = row % 128;           // position in the 128-row tile = tensor-memory lane of the output row
             const int kk = (int)(k % 16);
             return reinterpret_cast<uint16_t *>(W16 + blk * (4096 * (size_t)img.tc16_pieces) + (size_t)piece * 4096 + (size_t)i * 32 +
                                                 (size_t)(((kk >> 3) ^ ((i >> 2) & 1)) * 16) + (size_t)(kk & 7) * 2);

@@ -394,7 +394,7 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
     // adds shared-memory traffic (raw copy in, two reads of it, Xh and Xl out: ~560 + n cycles per chunk, measured
     // ~740 at n = 192) and leaves fewer stages.
     const int halo = conv_w > 0 ? (conv_w + 1 + 3) & ~3 : 0;
-    // (layers of at most 128 rows: only the bf16 kernel, which then gives each CTA of the pair half of the rows)
+    // (layers of at most 128 rows: only the bf16 kernel, whose two CTAs then both take the one row tile and split the columns)
     if ((M > 128 || bf16) && conv_w >= 0 && (!conv || ((K / 9) % TC_KC == 0 && halo <= 64))) {
         double best2 = 1e300;
         int best2_n = 0;
@@ -414,7 +414,7 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
             const double smem_chunk = bf16 ? (conv ? 700.0 + 0.6 * n : 470.0 + 0.33 * n) : (conv ? 560.0 + 1.0 * n : 500.0 + 0.5 * n);
             if (per_chunk < smem_chunk) per_chunk = smem_chunk;
             double per_tile = nchunk * per_chunk;
-            const double epi = (bf16 ? 50.0 * n : 45.0 * n) * (M > 128 ? 1.0 : tc16_rows_per_cta(M) / 128.0);
+            const double epi = (bf16 ? 50.0 * n : 45.0 * n) * (M > 128 ? 1.0 : 0.5);   // <= 128 rows: half the columns per CTA
             if (per_tile < epi) per_tile = epi;
             if (bf16) per_tile += 2500.0;
             const double t = 4400.0 + (double)per_pair * per_tile + 4500.0 + 30.0 * n;
@@ -470,7 +470,8 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
         const int halo = a.conv ? (a.W + 1 + 3) & ~3 : 0;
         if ((rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)(a.conv ? K / 9 : K), (uint64_t)(a.conv ? a.isc : a.ldx) * 4,
                             (uint32_t)(best_n / 2 + 2 * halo), TC_KC, CU_TENSOR_MAP_SWIZZLE_NONE))) return rc;
-        a.rpc = tc16_rows_per_cta(M);
+        a.rpc = 128;
+        a.dup = M <= 128 ? 1 : 0;          // one row tile: both CTAs of a pair take it and split the columns between them
         return launch_tc_pair_bf16(dev + pl->img.tc16_off, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream, cfg_pieces(pl->cfg),
                                    rows / 256);
     }

@@ -213,9 +213,10 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     // this pair's tiles: pair, pair + npairs, ...; tile t = (row pair t % nrp, column tile t / nrp)
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
     const int nmy = pair < ntiles ? (ntiles - pair + npairs - 1) / npairs : 0;
-    const int rpc = a.rpc ? a.rpc : 128;                   // output rows per CTA (fewer than 128 only for layers of <= 128 rows)
+    const int rpc = 128;                                   // output rows per CTA
     // first row of this CTA in the tile's first MMA tile; MMA tile m of the tile starts 2 m rpc rows further on
-    auto tile_row0 = [&](int i) { return (((pair + i * npairs) % nrp) * 2 * MT + (int)rank) * rpc; };
+    // (layers of at most 128 rows: both CTAs take the layer's only row tile, see TcArgs::dup)
+    auto tile_row0 = [&](int i) { return (((pair + i * npairs) % nrp) * 2 * MT + (a.dup ? 0 : (int)rank)) * rpc; };
     auto tile_col0 = [&](int i) { return (int64_t)((pair + i * npairs) / nrp) * N; };
 
     // one stage's copies (stage sg of a tile = chunks sg * SUB ...): per chunk the W1 / W2 block of this CTA's 128

@@ -190,8 +190,10 @@ struct TcArgs {
     int ntile;               // columns per CTA: multiple of 32, <= 256
     int relu;
     int *status;             // plan status word
-    int rpc;                 // CTA-pair kernels: output rows per CTA (128; fewer when the layer has at most 128 rows
-                             // and the pair splits them evenly); 0 means 128
+    int rpc;                 // CTA-pair kernels: output rows per CTA: 128 (0 means 128)
+    int dup;                 // bf16 CTA-pair kernel, layers of at most 128 rows: both CTAs of a pair multiply the SAME
+                             // 128-row weight tile (the pair's MMA needs 256 rows; the second half repeats the first) and
+                             // each stores the whole rows of its own half of the tile's columns
     int mt;                  // bf16 CTA-pair kernel: 256-row MMA tiles a pair stacks on ONE staged activation tile
                              // (1, or 2 = tiles of 512 rows, one per pair); 0 means 1
 };
@@ -252,95 +254,64 @@ __device__ __forceinline__ int64_t tile_cols_end(int64_t col0, int N) { return c
 __device__ __forceinline__ void epilogue_blocks(const TcArgs &a, uint32_t acc, int q, int first, int step, int N,
                                                 int row0, int64_t col0, int lane, uint32_t done_bar, uint32_t rank)
 {
-    const int rpc = a.rpc ? a.rpc : 128;                    // rows of the CTA's part that exist
-    const int nunit = N / 16;
-    // Matrix row of this lane's four accumulator rows (tensor-memory lanes 32 q + t/4 + {0, 8, 16, 24}), -1 where there
-    // is none. A CTA with 128 rows has them in lane order. One with fewer (layers of at most 128 rows) has a quarter of
-    // them at the start of each lane quarter, so that the warps of all four quarters have rows to store: rows
-    // q * rpc/4 ... are lanes 32 q + 0 ..., which is how the plan laid the weight rows out.
+    // this CTA's units of the tile: all of them, or -- layers of at most 128 rows, where both CTAs of the pair hold
+    // the whole product (TcArgs::dup) -- the half of the columns that belongs to its rank
+    const int nall = N / 16;
+    const int u0 = a.dup ? (int)rank * (nall / 2) : 0, u1 = a.dup ? u0 + nall / 2 : nall;
+    // matrix row of this lane's four accumulator rows (tensor-memory lanes 32 q + t/4 + {0, 8, 16, 24}), -1 beyond the matrix
     int rows[4];
     float bias[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        int r = -1;
-        if (rpc == 128) r = row0 + q * 32 + (lane >> 2) + 8 * i;
-        else if ((lane >> 2) + 8 * i < (rpc >> 2)) r = row0 + q * (rpc >> 2) + (lane >> 2) + 8 * i;
+        const int r = row0 + q * 32 + (lane >> 2) + 8 * i;
         rows[i] = r < a.M ? r : -1;
         bias[i] = (a.bias && rows[i] >= 0) ? __ldg(a.bias + rows[i]) : 0.f;
     }
-    const bool second_half = rpc == 128 || (rpc >> 2) > 16;   // lanes 16 .. 31 of the quarter hold rows at all
 #pragma unroll 1
-    for (int cc = first; cc < nunit; cc += step) {
+    for (int cc = u0 + first; cc < u1; cc += step) {
         uint32_t r[2][8];
         tmem_ld_16x256b_x2(acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(cc * 16), r[0]);
-        if (second_half) tmem_ld_16x256b_x2(acc + ((uint32_t)(q * 32 + 16) << 16) + (uint32_t)(cc * 16), r[1]);
+        tmem_ld_16x256b_x2(acc + ((uint32_t)(q * 32 + 16) << 16) + (uint32_t)(cc * 16), r[1]);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (done_bar && cc + step >= nunit) {
+        if (done_bar && cc + step >= u1) {
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             if (lane == 0) {
                 if (rank == 0) mbar_arrive(done_bar);
                 else mbar_arrive_remote(done_bar, 0);
             }
         }
-        if (rpc < 128) {
-            // Layers of at most 128 rows: every warp has at most 16 rows, in the first half of its lane quarter, and the
-            // epilogue is what the tile waits for; the column pairs are stored as they come (8 bytes per lane, eight
-            // 32-byte sectors per instruction), which measures slightly faster here than spending shuffles on wider
-            // stores.
-            const int64_t cb = col0 + cc * 16 + 2 * (lane & 3);
+        // Lanes 2i and 2i + 1 swap a column pair, so that every lane holds four consecutive columns of each of its rows
+        // (even lanes: columns 4i .. 4i + 3 of the unit, odd lanes: 8 + 4i ..) and the warp's 16-byte stores write the
+        // unit's 64 bytes of a row as two whole sectors.
+        const bool odd = (lane & 1) != 0;
+        const int64_t cb = col0 + cc * 16 + (odd ? 8 + 2 * ((lane & 3) - 1) : 2 * (lane & 3));
 #pragma unroll
-            for (int half = 0; half < 2; ++half)
+        for (int half = 0; half < 2; ++half)
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int row = rows[2 * half + h];
-                    if (row < 0) continue;
-                    float *yrow = a.Y + (size_t)row * a.ldy;
-                    const float b = bias[2 * half + h];
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        float2 o = make_float2(__uint_as_float(r[half][4 * j + 2 * h]) + b,
-                                               __uint_as_float(r[half][4 * j + 2 * h + 1]) + b);
-                        if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); }
-                        const int64_t col = cb + 8 * j;
-                        if (!UBP_CHK_GMEM(col >= 0 && row < a.M && (tile_cols_end(col0, N) >= col), a.status)) continue;
-                        if (col + 1 < a.Nc) *reinterpret_cast<float2 *>(yrow + col) = o;
-                        else if (col < a.Nc) yrow[col] = o.x;
-                    }
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t p0x = r[half][2 * h], p0y = r[half][2 * h + 1];           // columns 2 (t mod 4) + {0, 1}
+                const uint32_t p1x = r[half][4 + 2 * h], p1y = r[half][4 + 2 * h + 1];   // columns 8 + 2 (t mod 4) + {0, 1}
+                const uint32_t gx = __shfl_xor_sync(0xffffffffu, odd ? p0x : p1x, 1);
+                const uint32_t gy = __shfl_xor_sync(0xffffffffu, odd ? p0y : p1y, 1);
+                const int row = rows[2 * half + h];
+                if (row < 0) continue;
+                float *yrow = a.Y + (size_t)row * a.ldy;
+                const float b = bias[2 * half + h];
+                float4 o = odd ? make_float4(__uint_as_float(gx), __uint_as_float(gy), __uint_as_float(p1x), __uint_as_float(p1y))
+                               : make_float4(__uint_as_float(p0x), __uint_as_float(p0y), __uint_as_float(gx), __uint_as_float(gy));
+                o.x += b; o.y += b; o.z += b; o.w += b;
+                if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+                if (!UBP_CHK_GMEM(cb >= 0 && row < a.M && (tile_cols_end(col0, N) >= cb + 3), a.status)) continue;
+                if (cb + 3 < a.Nc) *reinterpret_cast<float4 *>(yrow + cb) = o;
+                else {
+                    if (cb < a.Nc) yrow[cb] = o.x;
+                    if (cb + 1 < a.Nc) yrow[cb + 1] = o.y;
+                    if (cb + 2 < a.Nc) yrow[cb + 2] = o.z;
                 }
-        } else {
-            // Lanes 2i and 2i + 1 swap a column pair, so that every lane holds four consecutive columns of each of its rows
-            // (even lanes: columns 4i .. 4i + 3 of the unit, odd lanes: 8 + 4i ..) and the warp's 16-byte stores write the
-            // unit's 64 bytes of a row as two whole sectors.
-            const bool odd = (lane & 1) != 0;
-            const int64_t cb = col0 + cc * 16 + (odd ? 8 + 2 * ((lane & 3) - 1) : 2 * (lane & 3));
-#pragma unroll
-            for (int half = 0; half < 2; ++half)
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t p0x = r[half][2 * h], p0y = r[half][2 * h + 1];           // columns 2 (t mod 4) + {0, 1}
-                    const uint32_t p1x = r[half][4 + 2 * h], p1y = r[half][4 + 2 * h + 1];   // columns 8 + 2 (t mod 4) + {0, 1}
-                    const uint32_t gx = __shfl_xor_sync(0xffffffffu, odd ? p0x : p1x, 1);
-                    const uint32_t gy = __shfl_xor_sync(0xffffffffu, odd ? p0y : p1y, 1);
-                    const int row = rows[2 * half + h];
-                    if (row < 0) continue;
-                    float *yrow = a.Y + (size_t)row * a.ldy;
-                    const float b = bias[2 * half + h];
-                    float4 o = odd ? make_float4(__uint_as_float(gx), __uint_as_float(gy), __uint_as_float(p1x), __uint_as_float(p1y))
-                                   : make_float4(__uint_as_float(p0x), __uint_as_float(p0y), __uint_as_float(gx), __uint_as_float(gy));
-                    o.x += b; o.y += b; o.z += b; o.w += b;
-                    if (a.relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
-                    if (!UBP_CHK_GMEM(cb >= 0 && row < a.M && (tile_cols_end(col0, N) >= cb + 3), a.status)) continue;
-                    if (cb + 3 < a.Nc) *reinterpret_cast<float4 *>(yrow + cb) = o;
-                    else {
-                        if (cb < a.Nc) yrow[cb] = o.x;
-                        if (cb + 1 < a.Nc) yrow[cb + 1] = o.y;
-                        if (cb + 2 < a.Nc) yrow[cb + 2] = o.z;
-                    }
-                }
-        }
+            }
     }
     // a warp with no unit of its own still owes its arrival
-    if (done_bar && first >= nunit) {
+    if (done_bar && u0 + first >= u1) {
         if (lane == 0) {
             if (rank == 0) mbar_arrive(done_bar);
             else mbar_arrive_remote(done_bar, 0);

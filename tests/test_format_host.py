@@ -239,19 +239,9 @@ def test_tensor_core_plan_dense_part(M, C, Nb, p, R, variant, sparse_variant):
     blocks[:, :, :, swap] = blocks[:, :, :, swap][..., ::-1, :]
     W12 = blocks.reshape(nrt, nch, 2, 128, 16).transpose(2, 0, 3, 1, 4)          # [piece][row tile][row in tile][k]
     W12 = W12.reshape(2, nrt, 128, kp16)
-    # a row tile holds `rpc` rows of the matrix: 128, or half of them (rounded up to 8) for a layer of <= 128 rows,
-    # so that both CTAs of a pair have rows to store; the rest of the tile is zero
-    rpc = 128 if M > 128 else ((M + 1) // 2 + 7) // 8 * 8
-    if rpc < 128:
-        # ... and those rows sit a quarter each at the start of the four 32-row quarters of the tile (every epilogue
-        # warp reads one quarter of the accumulator's rows and so has rows to store)
-        q4 = rpc // 4
-        pos = (np.arange(rpc) // q4) * 32 + np.arange(rpc) % q4
-        rest = np.setdiff1d(np.arange(128), pos)
-        assert not W12[:, :, rest].any()
-        W12 = W12[:, :, pos]
-    assert not W12[:, :, rpc:].any()
-    W12 = W12[:, :, :rpc].reshape(2, nrt * rpc, kp16)
+    # row tile t holds rows 128 t .. 128 t + 127 of the matrix in order (a layer of at most 128 rows: tile 0 holds it,
+    # tile 1 is zero: both CTAs of a pair multiply tile 0 and split the columns)
+    W12 = W12.reshape(2, nrt * 128, kp16)
     assert not W12[:, M:].any()                                # padding rows
     W1 = (W12[0, :M].astype(np.uint32) << 16).view(np.float32)
     W2 = (W12[1, :M].astype(np.uint32) << 16).view(np.float32)
