@@ -316,6 +316,10 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // Cluster barrier, first half: every thread arrives once its CTA's barriers exist (thread 0: after it has
+    // initialised them); the wait comes after the wait for the earlier kernel, when the other CTA has normally arrived
+    // long ago, so the barrier's round trip is off the path.
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
     if (warp == 1) {   // tensor memory of the pair: the same warp of both CTAs allocates
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
@@ -324,7 +328,7 @@ ubp_conv3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtens
     asm volatile("griddepcontrol.wait;" ::: "memory");     // every thread: nothing below may overtake the earlier kernel
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    cluster_sync();                                        // both CTAs' barriers exist before anyone signals them
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");   // both CTAs' barriers exist before anyone signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
 

@@ -274,18 +274,22 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         // tensor-memory allocation and the cluster barrier. The weights are constants of the layer, so the copies of
         // the ring's first stages do not wait for the kernel before this one; the activations may be its output.
         for (int f = 0; f < npre; ++f) issue_w(f % nstage, f, tile_row0(f / nstage));
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        for (int f = 0; f < npre; ++f) issue_x(f % nstage, f, (int)(tile_col0(f / nstage) + (int64_t)rank * NH));
     }
+    // Cluster barrier, first half: every thread arrives once its CTA's barriers exist (thread 0: after it has
+    // initialised them). The wait comes after the wait for the earlier kernel, by when the other CTA has normally
+    // arrived long ago: the barrier's round trip is off the path.
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
     if (warp == 1) {   // tensor memory of the pair: the same warp of both CTAs allocates
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");     // every thread: nothing below may overtake the earlier kernel
+    if (threadIdx.x == 0)
+        for (int f = 0; f < npre; ++f) issue_x(f % nstage, f, (int)(tile_col0(f / nstage) + (int64_t)rank * NH));
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    cluster_sync();                                        // both CTAs' barriers exist before anyone signals them
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");   // both CTAs' barriers exist before anyone signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
 
