@@ -249,7 +249,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         }
     };
     // stages whose weight copies start before the wait for the previous kernel
-    const int npre = nmy * nstage < T3_PRE ? nmy * nstage : T3_PRE;
+    const int npre = nmy * nstage < (T3_PRE < S ? T3_PRE : S) ? nmy * nstage : (T3_PRE < S ? T3_PRE : S);   // never beyond the ring
 
     // Launched with programmatic stream serialisation, the grid may become resident while the kernel before it in
     // the stream is still running: let the kernel after this one do the same, set up everything that reads no global
