@@ -353,3 +353,25 @@ def test_block_selection_argument_checks_need_no_device():
     # null pointers are refused before anything is launched
     assert L.ubp_bed_select(None, 64, 32, 1, 4, 10, None, 0, None, None, None) == -1
     assert L.ubp_block_scores(None, 64, 32, 1, 4, None, 0, None, None) == -1
+
+
+@pytest.mark.parametrize("M,C,p,tensor", [(256, 256, 90, True), (256, 256, 95, True), (256, 256, 98, False),
+                                          (1024, 1024, 99, True), (1024, 1024, 99.7, False), (64, 256, 70, False),
+                                          (256, 32, 70, False)])
+def test_automatic_variant_by_density_and_size(M, C, p, tensor):
+    """Variant 0: the dense tensor-core form from 128 rows x 64 channels on whenever at least 3 % of the weights are
+    kept (0.5 % for layers of a million weights or more), else the sparse kernel. Seen on the host through the plan's
+    size: a tensor-core plan carries the dense weight beside the sparse plan."""
+    rng = np.random.default_rng(int(M + C + 10 * p))
+    Nb = 4
+    m = int(M * C * (100 - p) / 100) // Nb
+    mask = np.zeros((M, C), np.uint8)
+    # m blocks at aligned, distinct places (the rule only looks at their number)
+    for q in rng.choice((M // Nb) * C, m, replace=False):
+        mask[(q % (M // Nb)) * Nb:(q % (M // Nb)) * Nb + Nb, q // (M // Nb)] = 1
+    W = rng.standard_normal((M, C, 1)).astype(np.float32)
+    blob = ubp.ubp_pack(W, mask, Nb)
+    sparse_id = 14 if M > 64 else 51
+    auto, dense, sparse = ubp.plan_size(blob, 0), ubp.plan_size(blob, 36), ubp.plan_size(blob, sparse_id)
+    assert dense > sparse
+    assert auto == (dense if tensor else sparse)
