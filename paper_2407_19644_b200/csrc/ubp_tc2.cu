@@ -176,6 +176,9 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
     };
 
+    // Launched with programmatic stream serialisation (as ubp_tc3.cu): let the next kernel become resident early, set
+    // up everything that reads no global data, then wait for the earlier kernel before the first copy.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) {
         prefetch_tensormap(&tmW);
         prefetch_tensormap(&tmX);
@@ -192,18 +195,22 @@ ubp_tc2_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         mbar_init(smem_u32(&bar_last), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        // the first copy lands in this CTA's own memory and signals its own barrier: start it before the
-        // tensor-memory allocation and the cluster barrier, so that the first data is on its way meanwhile
-        if (nmy > 0) issue_chunk(0, 0, tile_row0(0), (int)(tile_col0(0) + (int64_t)rank * NH));
     }
+    // cluster barrier, first half: arrive once this CTA's barriers exist; the wait follows the wait for the earlier
+    // kernel, when the other CTA has normally arrived long ago
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
     if (warp == 1) {   // tensor memory of the pair: the same warp of both CTAs allocates
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // every thread: nothing below may overtake the earlier kernel
+    // the first copy lands in this CTA's own memory and signals its own barrier: start it before the rest of the
+    // set-up completes, so that the first data is on its way meanwhile
+    if (threadIdx.x == 0 && nmy > 0) issue_chunk(0, 0, tile_row0(0), (int)(tile_col0(0) + (int64_t)rank * NH));
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    cluster_sync();                                        // both CTAs' barriers exist before anyone signals them
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");   // both CTAs' barriers exist before anyone signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
 
@@ -427,12 +434,19 @@ int launch_tc_pair(const CUtensorMap_st *tmW, const CUtensorMap_st *tmX, int x3d
     if (ntiles <= 0) return UBP_OK;
     if (ntiles > 0x7fffffffll) return UBP_E_UNSUPPORTED;
     const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
-    const dim3 grid((unsigned)(2 * pairs));
-    if (halo)
-        ubp_tc2_kernel<true><<<grid, T2_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(*tmW, *tmX, a, halo, nrp, (int)ntiles);
-    else
-        ubp_tc2_kernel<false><<<grid, T2_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(*tmW, *tmX, a, x3d, nrp, (int)ntiles);
-    cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3(T2_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = halo ? cudaLaunchKernelEx(&cfg, ubp_tc2_kernel<true>, *tmW, *tmX, a, halo, nrp, (int)ntiles)
+                         : cudaLaunchKernelEx(&cfg, ubp_tc2_kernel<false>, *tmW, *tmX, a, x3d, nrp, (int)ntiles);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return UBP_E_CUDA; }
     return UBP_OK;
 }
