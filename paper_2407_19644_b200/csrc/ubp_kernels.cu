@@ -290,6 +290,9 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
     const int D = S > 2 ? S - 2 : 1;               // steps in flight ahead of the one being computed
     const uint32_t *gtab = reinterpret_cast<const uint32_t *>(a.plan + 256);
 
+    // Launched with programmatic stream serialisation: the next kernel in the stream may become resident while this one
+    // drains, and this one sets its barriers up while its predecessor drains; nothing global is touched before the wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < S; ++s) {
@@ -299,6 +302,7 @@ ubp_spmm_kernel(const __grid_constant__ CUtensorMap tmX, const SpmmArgs a)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
 
     int issued = 0;                                // steps whose copies thread 0 has issued
@@ -706,9 +710,19 @@ static int launch_main(const ubp_plan *pl, const float *X, int64_t ldx, int64_t 
     const int per = (nstrips + gy - 1) / gy;
     gy = (nstrips + per - 1) / per;
     a.nstrips = nstrips;
-    dim3 grid((unsigned)pl->img.NG, (unsigned)gy);
-    kern<<<grid, WR * WC * 32, smem, stream>>>(tm, a);
-    return check(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)pl->img.NG, (unsigned)gy);
+    cfg.blockDim = dim3(WR * WC * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm, a);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    return check(e);
 }
 
 template <int NBK, int P>
