@@ -421,17 +421,21 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
             if (t < best2) { best2 = t; best2_n = n; }
         }
         int best2_rows = 256;
-        // bf16 1x1, rows in whole 512-row tiles, few enough tiles for one per pair: a pair may stack two 256-row MMA
+        // bf16 1x1, rows in whole 512-row tiles: a pair may stack two 256-row MMA
         // tiles on one staged activation tile (one copy and one split pass serve both; a chunk then brings two weight
         // blocks and its six MMAs: measured ~585-605 cycles per chunk at 96 and 192 columns) instead of making two
         // rounds; narrow stacked tiles lose against one round of wide plain ones, which the estimate reproduces
         if (bf16 == 1 && !conv && ((M + 255) / 256) % 2 == 0) {
             for (int n = 64; n <= 256; n += 32) {
                 const long long ntiles = (long long)((M + 511) / 512) * ((Nc + n - 1) / n);
-                if (ntiles > sms / 2 || tc_pair_bf16_stages(n, 0, 2) < 4) continue;
+                if (tc_pair_bf16_stages(n, 0, 2) < 4) continue;
+                const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
+                const long long per_pair = (ntiles + pairs - 1) / pairs;
                 double per_chunk = 3.3 * n;
                 if (per_chunk < 600.0 + 0.33 * n) per_chunk = 600.0 + 0.33 * n;
-                const double t = 4400.0 + nchunk * per_chunk + 2500.0 + 4500.0 + 60.0 * n;
+                // (both accumulators belong to one tile: every tile's epilogue, ~100 cycles per column, is exposed)
+                const double t = 4400.0 + (double)per_pair * (nchunk * per_chunk + 2500.0) + (double)(per_pair - 1) * 100.0 * n +
+                                 4500.0 + 60.0 * n;
                 if (t < best2) { best2 = t; best2_n = n; best2_rows = 512; }
             }
         }

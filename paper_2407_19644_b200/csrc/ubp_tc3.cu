@@ -199,8 +199,9 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     const uint32_t rank = cluster_rank();
     const int N = a.ntile, NH = N / 2;                     // tile columns; columns whose X this CTA holds
     const uint32_t xb = t3_x_bytes(NH);                    // x1 (and x2) bytes per chunk
-    // MT 256-row MMA tiles share the staged activations (MT = 2: the pair owns a tile of 512 rows, at most one per
-    // pair, its two accumulators side by side in tensor memory; the split pass then runs once for both)
+    // MT 256-row MMA tiles share the staged activations (MT = 2: the pair owns tiles of 512 rows, their two
+    // accumulators side by side in tensor memory, so a tile's epilogue is not hidden under the next tile's main loop;
+    // the split pass then runs once for both)
     const int MT = a.mt > 1 ? 2 : 1;
     const uint32_t wbytes = (uint32_t)(MT * NP) * T3_A_PART;   // weight blocks at the head of a chunk
     const uint32_t chunk_bytes = t3_chunk_bytes(NH, halo, NP, MT), stage_bytes = (uint32_t)SUB * chunk_bytes;
@@ -324,10 +325,12 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             uint32_t ph = 0;
             bool ready = nmy > 0 && mbar_try_wait(smem_u32(&bar_go[0]), 0);
             for (int i = 0; i < nmy && ok; ++i) {
-                const int b = i & 1;
+                // two accumulators take turns -- or, with stacked tiles, one tile owns both and the next tile waits
+                // for this one's epilogue
+                const int b = MT == 2 ? 0 : (i & 1);
                 const uint32_t acc = tmem_base + (uint32_t)b * T3_ACC_COLS;
-                if (i >= 2) {                              // the epilogue of tile i - 2 must have read this accumulator
-                    ok = mbar_wait(smem_u32(&bar_acc_empty[b]), (uint32_t)((i >> 1) - 1) & 1u, &abort_flag);
+                if (MT == 2 ? i >= 1 : i >= 2) {           // the epilogue of the tile that used it must have read this accumulator
+                    ok = mbar_wait(smem_u32(&bar_acc_empty[b]), (uint32_t)(MT == 2 ? i - 1 : (i >> 1) - 1) & 1u, &abort_flag);
                     if (!ok) break;
                 }
                 for (int sg = 0; sg < nstage; ++sg) {
@@ -496,21 +499,22 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int i = nmy - 1;
             for (int m = 0; m < MT; ++m)
-                epilogue_blocks(a, tmem_base + (uint32_t)((i & 1) + m) * T3_ACC_COLS, warp & 3, 2 + ((warp - 2) >> 2), 4, N,
+                epilogue_blocks(a, tmem_base + (uint32_t)(MT == 2 ? m : (i & 1)) * T3_ACC_COLS, warp & 3, 2 + ((warp - 2) >> 2), 4, N,
                                 tile_row0(i) + 2 * m * rpc, tile_col0(i), lane, 0u, rank);
         }
     } else {
         // ---------------- epilogue warps: tile i's accumulator while the main loop works on tile i + 1
         const int part = (warp - 2 - T3_XL_WARPS) >> 2;       // two warps share a lane quarter and split the columns
         for (int i = 0; i < nmy && ok; ++i) {
-            const int b = i & 1;
-            ok = mbar_wait_relaxed(smem_u32(&bar_acc_full[b]), (uint32_t)(i >> 1) & 1u, &abort_flag);
+            const int b = MT == 2 ? 0 : (i & 1);
+            ok = mbar_wait_relaxed(smem_u32(&bar_acc_full[b]), (uint32_t)(MT == 2 ? i : (i >> 1)) & 1u, &abort_flag);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const bool last = i == nmy - 1;
-            for (int m = 0; m < MT; ++m)     // (a stack of two is always the pair's only, hence last, tile)
+            for (int m = 0; m < MT; ++m)     // (stacked: the accumulators go back once the second one has been read)
                 epilogue_blocks(a, tmem_base + (uint32_t)(b + m) * T3_ACC_COLS, warp & 3, part, last ? 4 : 2, N,
-                                tile_row0(i) + 2 * m * rpc, tile_col0(i), lane, last ? 0u : smem_u32(&bar_acc_empty[b]), rank);
+                                tile_row0(i) + 2 * m * rpc, tile_col0(i), lane,
+                                (last || m != MT - 1) ? 0u : smem_u32(&bar_acc_empty[b]), rank);
         }
     }
     if (!ok && lane == 0) atomicExch(a.status, 1);
@@ -539,9 +543,8 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     a.mt = mt;
     const int nh = ntile / 2;
     if (pieces != 2 && !(pieces == 3 && !conv)) return UBP_E_UNSUPPORTED;
-    // tiles of 512 rows: two-piece 1x1 products of layers whose rows fill whole 512-row tiles, one tile per pair
-    if (mt != 1 && !(mt == 2 && pieces == 2 && !conv && ((M + 255) / 256) % 2 == 0 &&
-                     (long long)((M + 511) / 512) * ((Nc + ntile - 1) / ntile) <= sms / 2)) return UBP_E_UNSUPPORTED;
+    // tiles of 512 rows: two-piece 1x1 products of layers whose rows fill whole 512-row tiles
+    if (mt != 1 && !(mt == 2 && pieces == 2 && !conv && ((M + 255) / 256) % 2 == 0)) return UBP_E_UNSUPPORTED;
     // chunks per stage: two on long reductions (48 chunks and more), else one
     const int sub = pieces == 2 && (a.K + TC_KC - 1) / TC_KC >= 48 && t3_stages(nh, halo, 2, pieces, mt) >= 4 ? 2 : 1;
     if (t3_stages(nh, halo, sub, pieces, mt) < 4) return UBP_E_UNSUPPORTED;

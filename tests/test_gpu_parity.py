@@ -192,11 +192,12 @@ def test_spmm_three_piece_variant(env, M, C, Nb, p, Nc, variant):
 
 @pytest.mark.parametrize("M,C,Nb,p,Nc,rows", [(512, 256, 4, 80, 12544, 512), (1024, 96, 8, 50, 6001, 512),
                                               (1000, 160, 2, 70, 4099, 512), (768, 128, 4, 70, 6272, 256),
-                                              (512, 64, 4, 60, 14208, 512), (512, 64, 4, 60, 19201, 256)])
+                                              (512, 64, 4, 60, 14208, 512), (512, 64, 4, 60, 19201, 512),
+                                              (512, 48, 4, 60, 45001, 512), (1024, 32, 2, 50, 30003, 512)])
 def test_spmm_stacked_row_tiles(env, M, C, Nb, p, Nc, rows):
-    """Layers whose rows fill whole 512-row tiles and whose tiles number at most one per CTA pair run two 256-row MMA
-    tiles on one staged activation tile (one copy and one split pass for both); an odd number of 256-row tiles, or one
-    column too many for a single round (75 tiles of 256 columns), keeps the plain tiles. Same arithmetic either way."""
+    """Layers whose rows fill whole 512-row tiles may run two 256-row MMA tiles on one staged activation tile (one copy
+    and one split pass for both), with one tile per CTA pair or several (then a tile's epilogue is not hidden: both
+    accumulators belong to it); an odd number of 256-row tiles keeps the plain tiles. Same arithmetic either way."""
     L = ubp_synth.make_layer("t", M, C, Nb, p, 3 * M + C, Nc=Nc, x_dist="normal", relu=(Nc % 2 == 0))
     Yh, Yref, A, plan = run_spmm(env, L, 34 + {2: 1, 4: 2, 8: 3}[Nb])
     assert (plan.tile_choice(Nc)[:2] == (2, 512)) == (rows == 512)
