@@ -104,7 +104,9 @@ def tf32_peak_tflops():
 # cannot be read outside a profiler, so the line carries these captured figures (null where none was taken).
 NCU_DRAM_BYTES_PER_LAUNCH = {
     ("mbv1_pw512", 36): 13936896 + 0,            # the 12.8 MB output is still in L2 when the kernel ends
-    ("sweep_nb4_p70", 36): 84903936 + 40135680,
+    ("sweep_nb4_p70", 36): 99645440 + 35270656,  # stacked tiles of 512 rows
+    ("mbv1_L1", 50): 102844672 + 148400128,
+    ("mbv1_L7", 36): 26784768 + 63488,
     ("r50_3x3", 64): 15389696 + 131840,
     ("r50_3x3", 44): 15257344 + 1280,            # the per-tap kernel
     ("mbv1_pw512", 32): 14984448 + 256,
