@@ -179,6 +179,10 @@ __device__ __forceinline__ void c3_epilogue(const TcArgs &a, const C3Geom &g, ui
     const int nunit = g.N / 16;
     const int total_real = (int)a.Nc;
     const int jpos = lane & 15, rsub = lane >> 4;
+    // the bias of the quarter's 32 rows, one per lane, fetched once (a load per row inside the store loop made every
+    // iteration wait for it)
+    const int brow = row0 + q * 32 + lane;
+    const float bias_l = (a.bias && brow < a.M) ? __ldg(a.bias + brow) : 0.f;
 #pragma unroll 1
     for (int cc = first; cc < nunit; cc += step) {
         uint32_t r[16];
@@ -199,16 +203,15 @@ __device__ __forceinline__ void c3_epilogue(const TcArgs &a, const C3Geom &g, ui
         for (int v = 0; v < 4; ++v)
             *reinterpret_cast<uint4 *>(stage + lane * C3_EPI_PITCH + v * 16) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
         __syncwarp();
-        if (col >= 0) {
 #pragma unroll 4
-            for (int k = 0; k < 16; ++k) {
-                const int rr = 2 * k + rsub;
-                const int row = row0 + q * 32 + rr;
-                if (row < a.M) {
-                    float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI_PITCH + jpos * 4) + (a.bias ? __ldg(a.bias + row) : 0.f);
-                    if (a.relu) o = fmaxf(o, 0.f);
-                    if (UBP_CHK_GMEM(col < total_real, a.status)) a.Y[(size_t)row * a.ldy + col] = o;
-                }
+        for (int k = 0; k < 16; ++k) {                     // (every lane takes part in the shuffle)
+            const int rr = 2 * k + rsub;
+            const int row = row0 + q * 32 + rr;
+            const float bv = __shfl_sync(0xffffffffu, bias_l, rr);
+            if (col >= 0 && row < a.M) {
+                float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI_PITCH + jpos * 4) + bv;
+                if (a.relu) o = fmaxf(o, 0.f);
+                if (UBP_CHK_GMEM(col < total_real, a.status)) a.Y[(size_t)row * a.ldy + col] = o;
             }
         }
         __syncwarp();
@@ -230,6 +233,8 @@ __device__ __forceinline__ void c3_epilogue32(const TcArgs &a, const C3Geom &g, 
 {
     const int nunit = (g.N + 31) / 32;
     const int total_real = (int)a.Nc;
+    const int brow = row0 + q * 32 + lane;                  // (bias once per lane, as above)
+    const float bias_l = (a.bias && brow < a.M) ? __ldg(a.bias + brow) : 0.f;
 #pragma unroll 1
     for (int cc = first; cc < nunit; cc += step) {
         uint32_t r[32];
@@ -242,15 +247,14 @@ __device__ __forceinline__ void c3_epilogue32(const TcArgs &a, const C3Geom &g, 
         for (int v = 0; v < 8; ++v)
             *reinterpret_cast<uint4 *>(stage + lane * C3_EPI32_PITCH + v * 16) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
         __syncwarp();
-        if (col >= 0) {
 #pragma unroll 4
-            for (int rr = 0; rr < 32; ++rr) {
-                const int row = row0 + q * 32 + rr;
-                if (row < a.M) {
-                    float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI32_PITCH + lane * 4) + (a.bias ? __ldg(a.bias + row) : 0.f);
-                    if (a.relu) o = fmaxf(o, 0.f);
-                    if (UBP_CHK_GMEM(col < total_real, a.status)) a.Y[(size_t)row * a.ldy + col] = o;
-                }
+        for (int rr = 0; rr < 32; ++rr) {                  // (every lane takes part in the shuffle)
+            const int row = row0 + q * 32 + rr;
+            const float bv = __shfl_sync(0xffffffffu, bias_l, rr);
+            if (col >= 0 && row < a.M) {
+                float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI32_PITCH + lane * 4) + bv;
+                if (a.relu) o = fmaxf(o, 0.f);
+                if (UBP_CHK_GMEM(col < total_real, a.status)) a.Y[(size_t)row * a.ldy + col] = o;
             }
         }
         __syncwarp();
