@@ -247,14 +247,42 @@ __device__ __forceinline__ void c3_epilogue32(const TcArgs &a, const C3Geom &g, 
         for (int v = 0; v < 8; ++v)
             *reinterpret_cast<uint4 *>(stage + lane * C3_EPI32_PITCH + v * 16) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
         __syncwarp();
+        // The unit's real positions are consecutive output columns. Where that run starts at an even column (always so
+        // for even image widths whose padded rows divide the unit: 14 x 14), a lane takes a PAIR of columns of one of
+        // two rows and writes 8 bytes: half as many store instructions, each of which the memory system makes wait.
+        const uint32_t mask = __ballot_sync(0xffffffffu, col >= 0);
+        const int nreal = __popc(mask);
+        const int c0 = __shfl_sync(0xffffffffu, col, mask ? __ffs(mask) - 1 : 0);
+        if (mask != 0u && (c0 & 1) == 0 && (a.ldy & 1) == 0) {
+            const int rs = lane >> 4, m = lane & 15;
+            const int s0 = 2 * m < nreal ? (int)__fns(mask, 0, 2 * m + 1) : -1;          // lanes (positions) of my two columns
+            const int s1 = 2 * m + 1 < nreal ? (int)__fns(mask, 0, 2 * m + 2) : -1;
 #pragma unroll 4
-        for (int rr = 0; rr < 32; ++rr) {                  // (every lane takes part in the shuffle)
-            const int row = row0 + q * 32 + rr;
-            const float bv = __shfl_sync(0xffffffffu, bias_l, rr);
-            if (col >= 0 && row < a.M) {
-                float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI32_PITCH + lane * 4) + bv;
-                if (a.relu) o = fmaxf(o, 0.f);
-                if (UBP_CHK_GMEM(col < total_real, a.status)) a.Y[(size_t)row * a.ldy + col] = o;
+            for (int k = 0; k < 16; ++k) {
+                const int rr = 2 * k + rs;
+                const int row = row0 + q * 32 + rr;
+                const float bv = __shfl_sync(0xffffffffu, bias_l, rr);
+                if (s0 >= 0 && row < a.M) {
+                    float o0 = *reinterpret_cast<const float *>(stage + rr * C3_EPI32_PITCH + s0 * 4) + bv;
+                    float o1 = s1 >= 0 ? *reinterpret_cast<const float *>(stage + rr * C3_EPI32_PITCH + s1 * 4) + bv : 0.f;
+                    if (a.relu) { o0 = fmaxf(o0, 0.f); o1 = fmaxf(o1, 0.f); }
+                    float *dst = a.Y + (size_t)row * a.ldy + c0 + 2 * m;
+                    if (UBP_CHK_GMEM(c0 + 2 * m < total_real, a.status)) {
+                        if (s1 >= 0) *reinterpret_cast<float2 *>(dst) = make_float2(o0, o1);
+                        else *dst = o0;
+                    }
+                }
+            }
+        } else {
+#pragma unroll 4
+            for (int rr = 0; rr < 32; ++rr) {              // (every lane takes part in the shuffle)
+                const int row = row0 + q * 32 + rr;
+                const float bv = __shfl_sync(0xffffffffu, bias_l, rr);
+                if (col >= 0 && row < a.M) {
+                    float o = *reinterpret_cast<const float *>(stage + rr * C3_EPI32_PITCH + lane * 4) + bv;
+                    if (a.relu) o = fmaxf(o, 0.f);
+                    if (UBP_CHK_GMEM(col < total_real, a.status)) a.Y[(size_t)row * a.ldy + col] = o;
+                }
             }
         }
         __syncwarp();
