@@ -353,6 +353,7 @@ int tc_pair_stages(int ntile, int halo);
 int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, int halo, const void *args,
                         int M, int64_t Nc, int ntile, int sms, void *stream, int pieces, int mt);
 int tc_pair_bf16_stages(int ntile, int halo, int mt = 1);
+int tc_pair_bf16_sub(int K, int ntile, int halo, int pieces, int mt);
 
 // Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
 // Each candidate's time is estimated as (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost)
@@ -470,10 +471,12 @@ static int launch_tc_common(const ubp_plan *pl, TcArgs a, cudaStream_t stream)
     }
     if (kernel == 2 && bf16) {
         CUtensorMap tmX;
-        // the input as (column, channel): 16 channel rows of the CTA's columns per chunk, plus the halo for 3x3
+        // the input as (column, channel): 16 channel rows of the CTA's columns per chunk, plus the halo for 3x3; 1x1: the
+        // rows of all the chunks of a pipeline stage in one box
         const int halo = a.conv ? (a.W + 1 + 3) & ~3 : 0;
+        const int box_rows = a.conv ? TC_KC : TC_KC * tc_pair_bf16_sub(K, best_n, halo, cfg_pieces(pl->cfg), rows / 256);
         if ((rc = encode_2d(&tmX, a.X, (uint64_t)Nc, (uint64_t)(a.conv ? K / 9 : K), (uint64_t)(a.conv ? a.isc : a.ldx) * 4,
-                            (uint32_t)(best_n / 2 + 2 * halo), TC_KC, CU_TENSOR_MAP_SWIZZLE_NONE))) return rc;
+                            (uint32_t)(best_n / 2 + 2 * halo), (uint32_t)box_rows, CU_TENSOR_MAP_SWIZZLE_NONE))) return rc;
         a.rpc = 128;
         a.dup = M <= 128 ? 1 : 0;          // one row tile: both CTAs of a pair take it and split the columns between them
         return launch_tc_pair_bf16(dev + pl->img.tc16_off, &tmX, a.conv, halo, &a, M, Nc, best_n, sms, stream, cfg_pieces(pl->cfg),

@@ -38,6 +38,9 @@ constexpr int T3_MAX_STAGES = 8;
 #ifndef T3_PRE
 #define T3_PRE 1
 #endif
+#ifndef T3_SUB2_FROM
+#define T3_SUB2_FROM 32                                   // chunks in the reduction from which a stage holds two
+#endif
 constexpr uint32_t T3_A_PART = 128 * TC_KC * 2;           // W1 or W2 chunk of this CTA's 128 rows: 4 KB
 constexpr uint32_t T3_ATOM = 64 * TC_KC * 2;              // x1 or x2 of 64 columns x 16 channels: 2 KB
 constexpr uint32_t T3_PIPE_BUDGET = 222 * 1024;
@@ -59,7 +62,9 @@ __host__ __device__ constexpr uint32_t t3_chunk_bytes(int nh, int halo, int np, 
 {
     return (uint32_t)(mt * np) * T3_A_PART + (uint32_t)np * t3_x_bytes(nh) + t3_raw_bytes(nh, halo);
 }
-// A stage holds `sub` chunks. With two, every barrier round trip (copies landed -> split pass -> MMA issue -> stage
+// A stage holds `sub` chunks, part by part: the weight blocks of all its chunks (per MMA tile of a stack the chunks one
+// after the other, as they lie in the plan: ONE bulk copy per MMA tile and stage), then each chunk's x1 / x2 tiles,
+// then the raw rows of all chunks (1x1: consecutive channels, ONE tensor copy per stage). With two, every barrier round trip (copies landed -> split pass -> MMA issue -> stage
 // free) serves 32 channels: fewer waits per channel, which pays on long reductions (3x3: 144 chunks; 1024 channels)
 // where the pass or the issue thread is the bound; with one, the pipeline fills and drains in finer steps, which
 // pays on short reductions (512 channels: 32 chunks).
@@ -204,12 +209,15 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     // the split pass then runs once for both)
     const int MT = a.mt > 1 ? 2 : 1;
     const uint32_t wbytes = (uint32_t)(MT * NP) * T3_A_PART;   // weight blocks at the head of a chunk
-    const uint32_t chunk_bytes = t3_chunk_bytes(NH, halo, NP, MT), stage_bytes = (uint32_t)SUB * chunk_bytes;
+    const uint32_t stage_bytes = (uint32_t)SUB * t3_chunk_bytes(NH, halo, NP, MT);
+    // inside a stage: weight blocks [MMA tile][chunk], x tiles [chunk][piece], raw rows [chunk]
+    const uint32_t xoff = (uint32_t)SUB * wbytes, xchunk = (uint32_t)NP * xb, roff = xoff + (uint32_t)SUB * xchunk;
     const uint32_t raw_row = (uint32_t)(NH + 2 * halo) * 4;   // bytes per channel row of the raw copy
     const int S = t3_stages(NH, halo, SUB, NP, MT);
     const int nchunk = (a.K + TC_KC - 1) / TC_KC;
     const int nstage = (nchunk + SUB - 1) / SUB;     // stages per tile; the last one may hold a single chunk
-    const uint32_t tx = wbytes + raw_row * TC_KC;          // bytes copied per chunk
+    const uint32_t raw_chunk = raw_row * TC_KC;            // raw bytes per chunk
+    constexpr bool XMERGED = !CONV && SUB > 1;             // one tensor copy brings the rows of all the stage's chunks
     const int Cin = CONV ? a.K / 9 : a.K;                  // 3x3: reduction index k = tap * Cin + channel, Cin % 16 == 0
     // this pair's tiles: pair, pair + npairs, ...; tile t = (row pair t % nrp, column tile t / nrp)
     const int npairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
@@ -228,25 +236,26 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     auto issue_w = [&](int sg, int st, int row0) {
         const uint32_t bar = smem_u32(&bar_full[st]);
         const int c0 = sg * SUB, nsub = nchunk - c0 < SUB ? nchunk - c0 : SUB;
-        mbar_expect_tx(bar, (uint32_t)nsub * tx);
-#pragma unroll
-        for (int u = 0; u < SUB; ++u) {
-            if (u >= nsub) break;
-            uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
-            for (int m = 0; m < MT; ++m)
-                bulk_load(smem_u32(chunk + (uint32_t)m * (NP * T3_A_PART)),
-                          W16 + ((size_t)(row0 / rpc + 2 * m) * nchunk + c0 + u) * (NP * T3_A_PART), NP * T3_A_PART, bar);
-        }
+        // (a merged activation copy always brings the whole box: rows past the last channel arrive as zeros)
+        mbar_expect_tx(bar, (uint32_t)nsub * wbytes + (uint32_t)(XMERGED ? SUB : nsub) * raw_chunk);
+        uint8_t *stage = smem + (size_t)st * stage_bytes;
+        for (int m = 0; m < MT; ++m)
+            bulk_load(smem_u32(stage + (uint32_t)(m * SUB) * (NP * T3_A_PART)),
+                      W16 + ((size_t)(row0 / rpc + 2 * m) * nchunk + c0) * (NP * T3_A_PART), (uint32_t)nsub * (NP * T3_A_PART), bar);
     };
     auto issue_x = [&](int sg, int st, int xcol) {
         const uint32_t bar = smem_u32(&bar_full[st]);
         const int c0 = sg * SUB, nsub = nchunk - c0 < SUB ? nchunk - c0 : SUB;
+        uint8_t *raw = smem + (size_t)st * stage_bytes + roff;
+        if constexpr (XMERGED) {
+            tma_load_2d(smem_u32(raw), &tmX, xcol - halo, c0 * TC_KC, bar);
+        } else {
 #pragma unroll
-        for (int u = 0; u < SUB; ++u) {
-            if (u >= nsub) break;
-            const int c = c0 + u;
-            uint8_t *chunk = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes;
-            tma_load_2d(smem_u32(chunk + wbytes + NP * xb), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
+            for (int u = 0; u < SUB; ++u) {
+                if (u >= nsub) break;
+                const int c = c0 + u;
+                tma_load_2d(smem_u32(raw + (uint32_t)u * raw_chunk), &tmX, xcol - halo, CONV ? (c * TC_KC) % Cin : c * TC_KC, bar);
+            }
         }
     };
     // stages whose weight copies start before the wait for the previous kernel
@@ -319,8 +328,8 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
             // ---------------- leader: MMA issuer for the pair (whole warp converged, one elected lane issues)
             const uint32_t idesc = make_idesc3(N);
             const uint64_t dW0 = make_desc(smem_u32(smem), 16, 256, SWZ_32B);
-            const uint64_t dX0 = make_desc(smem_u32(smem) + wbytes, 2048, 1024, SWZ_128B);
-            const uint32_t stage_u = stage_bytes >> 4, chunk_u = chunk_bytes >> 4;
+            const uint64_t dX0 = make_desc(smem_u32(smem) + xoff, 2048, 1024, SWZ_128B);
+            const uint32_t stage_u = stage_bytes >> 4, wchunk_u = (NP * T3_A_PART) >> 4, xchunk_u = xchunk >> 4;
             int st = 0;
             uint32_t ph = 0;
             bool ready = nmy > 0 && mbar_try_wait(smem_u32(&bar_go[0]), 0);
@@ -346,15 +355,15 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                     for (int u = 0; u < SUB; ++u)
                         if (u < nsub) {
                             if constexpr (NP == 3) {
-                                ready = mma6_chunk(acc, dW0 + soff + (uint64_t)(u * chunk_u), dX0 + soff + (uint64_t)(u * chunk_u),
+                                ready = mma6_chunk(acc, dW0 + soff + (uint64_t)(u * wchunk_u), dX0 + soff + (uint64_t)(u * xchunk_u),
                                                    T3_A_PART >> 4, xb >> 4, idesc, (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
                                                    smem_u32(&bar_empty[st]), u == nsub - 1 ? 1u : 0u);
                             } else {
                                 // every MMA tile of the stack on the same x1 / x2; the stage goes back after the last one
                                 for (int m = 0; m < MT; ++m)
                                     ready = mma3_chunk(acc + (uint32_t)m * T3_ACC_COLS,
-                                                       dW0 + soff + (uint64_t)(u * chunk_u) + (uint64_t)((uint32_t)m * (NP * T3_A_PART) >> 4),
-                                                       dX0 + soff + (uint64_t)(u * chunk_u), T3_A_PART >> 4, xb >> 4, idesc,
+                                                       dW0 + soff + (uint64_t)((uint32_t)(m * SUB + u) * wchunk_u),
+                                                       dX0 + soff + (uint64_t)(u * xchunk_u), T3_A_PART >> 4, xb >> 4, idesc,
                                                        (sg > 0 || u > 0) ? 1u : 0u, smem_u32(&bar_go[nst]), nph,
                                                        smem_u32(&bar_empty[st]), (u == nsub - 1 && m == MT - 1) ? 1u : 0u);
                             }
@@ -424,8 +433,8 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 #pragma unroll
             for (int u = 0; u < SUB; ++u) {
                 if (u >= nsub) break;
-                uint8_t *x1 = smem + (size_t)st * stage_bytes + (size_t)u * chunk_bytes + wbytes;
-                const uint8_t *raw = x1 + NP * xb;
+                uint8_t *x1 = smem + (size_t)st * stage_bytes + xoff + (uint32_t)u * xchunk;
+                const uint8_t *raw = smem + (size_t)st * stage_bytes + roff + (uint32_t)u * raw_chunk;
                 int sh = 0;
                 uint32_t ok8 = 0xffu;
                 if (CONV) {
@@ -533,8 +542,15 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 
 // Launch the bf16 pair kernel on tiles of 256 rows x `ntile` columns (a multiple of 64).
 // W16: the plan's bf16 part: 8 KB blocks [row tile of 128][chunk] = [W1, W2][128 rows][16 channels], pre-swizzled.
-// tmX: plain 2-D fp32 map (column, channel), box (ntile/2 + 2 halo) x 16; halo = 0 for 1x1, image width + 1
-// rounded up to a multiple of 4 for 3x3 (columns = the flattened (b, y, x) axis).
+// chunks per pipeline stage: two on reductions of 32 chunks and more (where the ring still gets four stages), else one
+int tc_pair_bf16_sub(int K, int ntile, int halo, int pieces, int mt)
+{
+    return pieces == 2 && (K + TC_KC - 1) / TC_KC >= T3_SUB2_FROM && t3_stages(ntile / 2, halo, 2, pieces, mt) >= 4 ? 2 : 1;
+}
+
+// tmX: plain 2-D fp32 map (column, channel), box (ntile/2 + 2 halo) x 16 -- 1x1: x 16 tc_pair_bf16_sub(...), one copy
+// per stage; halo = 0 for 1x1, image width + 1 rounded up to a multiple of 4 for 3x3 (columns = the flattened
+// (b, y, x) axis).
 int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, int halo, const void *args_,
                         int M, int64_t Nc, int ntile, int sms, void *stream, int pieces, int mt)
 {
@@ -545,8 +561,7 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     if (pieces != 2 && !(pieces == 3 && !conv)) return UBP_E_UNSUPPORTED;
     // tiles of 512 rows: two-piece 1x1 products of layers whose rows fill whole 512-row tiles
     if (mt != 1 && !(mt == 2 && pieces == 2 && !conv && ((M + 255) / 256) % 2 == 0)) return UBP_E_UNSUPPORTED;
-    // chunks per stage: two on long reductions (48 chunks and more), else one
-    const int sub = pieces == 2 && (a.K + TC_KC - 1) / TC_KC >= 48 && t3_stages(nh, halo, 2, pieces, mt) >= 4 ? 2 : 1;
+    const int sub = tc_pair_bf16_sub(a.K, ntile, halo, pieces, mt);
     if (t3_stages(nh, halo, sub, pieces, mt) < 4) return UBP_E_UNSUPPORTED;
     size_t smem = (size_t)t3_stages(nh, halo, sub, pieces, mt) * t3_stage_bytes(nh, halo, sub, pieces, mt) + 1024;
     if (smem < TC_PAIR_MIN_SMEM) smem = TC_PAIR_MIN_SMEM;   // one CTA per SM, whatever the tile width (see the constant)
