@@ -33,7 +33,12 @@ using namespace tc;
 constexpr int T3_XL_WARPS = 8;                            // warps 2..9: the split pass
 constexpr int T3_XL_GROUPS = 2;                           // two groups of four warps take turns on the chunks
 constexpr int T3_EPI_WARPS = 8;                           // warps 10..17
-constexpr int T3_THREADS = (2 + T3_XL_WARPS + T3_EPI_WARPS) * 32;
+// Copies are issued by three threads (lane 0 of warp 0 and of the last two warps): one for the weight copies of the first
+// MMA tile, one for the activation copies, one for the weight copies of a stacked second MMA tile. With a single
+// producer thread the ISSUE of a stage's copies was what a chunk waited for (each copy instruction holds its thread for
+// the order of 100 cycles).
+constexpr int T3_PROD2_WARP = 2 + T3_XL_WARPS + T3_EPI_WARPS;   // first of the two extra producer warps
+constexpr int T3_THREADS = (T3_PROD2_WARP + 2) * 32;
 constexpr int T3_MAX_STAGES = 8;
 #ifndef T3_PRE
 #define T3_PRE 1
@@ -233,15 +238,16 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     // channel rows of the input for this CTA's columns (3x3: the channels of the chunk's tap, and a halo of columns
     // either side). The weight copies come first and announce the bytes of both; the activation copies may follow
     // later (the kernel's first stages start their weight copies before the previous kernel in the stream is done).
-    auto issue_w = [&](int sg, int st, int row0) {
+    // (the thread that issues MMA tile 0's weights also announces the stage's bytes; the other copies may complete
+    // before that: the phase cannot end until the announcing arrival has come)
+    auto issue_w = [&](int sg, int st, int row0, int m) {
         const uint32_t bar = smem_u32(&bar_full[st]);
         const int c0 = sg * SUB, nsub = nchunk - c0 < SUB ? nchunk - c0 : SUB;
         // (a merged activation copy always brings the whole box: rows past the last channel arrive as zeros)
-        mbar_expect_tx(bar, (uint32_t)nsub * wbytes + (uint32_t)(XMERGED ? SUB : nsub) * raw_chunk);
+        if (m == 0) mbar_expect_tx(bar, (uint32_t)nsub * wbytes + (uint32_t)(XMERGED ? SUB : nsub) * raw_chunk);
         uint8_t *stage = smem + (size_t)st * stage_bytes;
-        for (int m = 0; m < MT; ++m)
-            bulk_load(smem_u32(stage + (uint32_t)(m * SUB) * (NP * T3_A_PART)),
-                      W16 + ((size_t)(row0 / rpc + 2 * m) * nchunk + c0) * (NP * T3_A_PART), (uint32_t)nsub * (NP * T3_A_PART), bar);
+        bulk_load(smem_u32(stage + (uint32_t)(m * SUB) * (NP * T3_A_PART)),
+                  W16 + ((size_t)(row0 / rpc + 2 * m) * nchunk + c0) * (NP * T3_A_PART), (uint32_t)nsub * (NP * T3_A_PART), bar);
     };
     auto issue_x = [&](int sg, int st, int xcol) {
         const uint32_t bar = smem_u32(&bar_full[st]);
@@ -283,7 +289,8 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         // The first copies land in this CTA's own memory and signal its own barriers: start them before the
         // tensor-memory allocation and the cluster barrier. The weights are constants of the layer, so the copies of
         // the ring's first stages do not wait for the kernel before this one; the activations may be its output.
-        for (int f = 0; f < npre; ++f) issue_w(f % nstage, f, tile_row0(f / nstage));
+        for (int f = 0; f < npre; ++f)
+            for (int m = 0; m < MT; ++m) issue_w(f % nstage, f, tile_row0(f / nstage), m);
     }
     // Cluster barrier, first half: every thread arrives once its CTA's barriers exist (thread 0: after it has
     // initialised them). The wait comes after the wait for the earlier kernel, by when the other CTA has normally
@@ -304,9 +311,12 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
     const uint32_t tmem_base = tmem_base_slot;
 
     bool ok = true;
-    if (warp == 0) {
-        // ---------------- TMA producer: one ring of S stages straight through all of this pair's tiles
-        if (lane == 0) {
+    if (warp == 0 || warp >= T3_PROD2_WARP) {
+        // ---------------- TMA producers: one ring of S stages straight through all of this pair's tiles; each of the
+        // three threads issues its own kind of copy for every stage (what: 0 = weights of MMA tile 0, 1 = activations,
+        // 2 = weights of a stacked second MMA tile) and waits for the stage itself
+        const int what = warp == 0 ? 0 : warp - T3_PROD2_WARP + 1;
+        if (lane == 0 && (what < 2 || MT == 2)) {
             int st = npre % S, round = npre / S;           // the first npre stages were started above
             int f = 0;                                     // stages counted through all tiles
             for (int i = 0; i < nmy && ok; ++i) {
@@ -317,8 +327,8 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                         ok = mbar_wait_relaxed(smem_u32(&bar_empty[st]), (uint32_t)(round - 1) & 1u, &abort_flag);
                         if (!ok) break;
                     }
-                    issue_w(sg, st, row0);
-                    issue_x(sg, st, xcol);
+                    if (what == 1) issue_x(sg, st, xcol);
+                    else issue_w(sg, st, row0, what >> 1);
                     if (++st == S) { st = 0; ++round; }
                 }
             }
