@@ -960,7 +960,7 @@ def main():
     extras = rank == 0 and not args.headline_only and name == "mbv1_pw512" and args.variant == 0
     if extras:
         # the same layer, same protocol, through the other two arithmetics; error figures on the oracle's sample
-        esteps = max(10, min(args.steps, 30))
+        esteps = max(10, min(args.steps, 100))           # the headline's region length by default
         line["variants"] = []
         for v in HEADLINE_VARIANTS:
             rec, pv, Yv = measure_layer(ubp, torch, L, v, esteps, 3, flush, hbm_gbs, name=name)
