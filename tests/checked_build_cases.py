@@ -105,6 +105,8 @@ def main():
         ("pair kernel bf16 ragged", lambda: spmm_case(200, 150, 4, 60, 130, 36, pad=2)),
         ("pair kernel bf16, <= 128 rows", lambda: spmm_case(72, 144, 8, 50, 1028, 37)),
         ("pair kernel bf16, stacked tiles", lambda: spmm_case(512, 64, 4, 60, 2000, 36)),
+        ("pair kernel bf16, two chunks per stage, odd chunk count", lambda: spmm_case(256, 520, 4, 70, 1000, 36)),
+        ("pair kernel bf16, two chunks per stage, <= 128 rows", lambda: spmm_case(100, 1000, 4, 80, 516, 36, pad=4)),
         ("pair kernel, three pieces", lambda: spmm_case(300, 150, 4, 70, 544, 86)),
         ("pair kernel TF32", lambda: spmm_case(300, 150, 4, 70, 516, 32)),
         ("one-CTA TF32", lambda: spmm_case(128, 128, 4, 60, 388, 32)),

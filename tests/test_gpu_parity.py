@@ -204,6 +204,20 @@ def test_spmm_stacked_row_tiles(env, M, C, Nb, p, Nc, rows):
     check(Yh, Yref, A, L, variant=36)
 
 
+@pytest.mark.parametrize("M,C,Nb,p,Nc,pad", [(256, 520, 4, 70, 2100, 0), (300, 1000, 2, 80, 1531, 4), (128, 777, 1, 60, 2050, 0),
+                                             (512, 512, 4, 70, 1030, 8), (1024, 528, 8, 80, 900, 0), (260, 2048, 4, 90, 777, 0),
+                                             (768, 1037, 4, 75, 4100, 0)])
+def test_spmm_long_reductions(env, M, C, Nb, p, Nc, pad):
+    """Reductions of 32 sixteen-channel chunks and more: a pipeline stage of the bf16 pair kernel holds two chunks, their
+    weight blocks arrive in one copy and their 32 channel rows in one box. Odd chunk counts (the last stage holds a single
+    chunk and the box reaches past the last channel), channel counts that are no multiple of 16, every tile kind
+    (plain, both CTAs on one row tile, several tiles per pair), padded leading dimensions."""
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 5 * M + C, Nc=Nc, x_dist="normal", relu=(C % 2 == 0))
+    Yh, Yref, A, plan = run_spmm(env, L, 34 + {1: 0, 2: 1, 4: 2, 8: 3}[Nb], pad=pad)
+    assert plan.tile_choice(Nc)[0] == 2 and (C + 15) // 16 >= 32
+    check(Yh, Yref, A, L, variant=36)
+
+
 def test_tensor_core_variant_ragged_unaligned_and_auto(env):
     torch, ubp = env
     # ragged last strip on the fast path, then operands the fast path cannot take (falls back to the embedded
