@@ -550,7 +550,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
 
 }  // namespace
 
-// Launch the bf16 pair kernel on tiles of 256 rows x `ntile` columns (a multiple of 64).
+// Launch the bf16 pair kernel on tiles of 256 rows x `ntile` columns (a multiple of 16; of 32 where both CTAs take the one row tile).
 // W16: the plan's bf16 part: 8 KB blocks [row tile of 128][chunk] = [W1, W2][128 rows][16 channels], pre-swizzled.
 // chunks per pipeline stage: two on reductions of 32 chunks and more (where the ring still gets four stages), else one
 int tc_pair_bf16_sub(int K, int ntile, int halo, int pieces, int mt)
@@ -568,6 +568,7 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     a.ntile = ntile;
     a.mt = mt;
     const int nh = ntile / 2;
+    if (ntile % 16 != 0 || (a.dup && ntile % 32 != 0) || ntile < 32 || ntile > 256) return UBP_E_UNSUPPORTED;
     if (pieces != 2 && !(pieces == 3 && !conv)) return UBP_E_UNSUPPORTED;
     // tiles of 512 rows: two-piece 1x1 products of layers whose rows fill whole 512-row tiles
     if (mt != 1 && !(mt == 2 && pieces == 2 && !conv && ((M + 255) / 256) % 2 == 0)) return UBP_E_UNSUPPORTED;

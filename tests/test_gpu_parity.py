@@ -218,6 +218,22 @@ def test_spmm_long_reductions(env, M, C, Nb, p, Nc, pad):
     check(Yh, Yref, A, L, variant=36)
 
 
+@pytest.mark.parametrize("M,C,Nb,p,Nc", [(512, 64, 4, 60, 13000), (256, 256, 4, 70, 12900), (1024, 48, 2, 50, 6500)])
+def test_spmm_tile_widths_in_steps_of_16(env, M, C, Nb, p, Nc):
+    """Where every CTA pair gets one tile, the narrowest width that still fits one round is taken, in steps of 16 columns
+    (the MMA's step): each CTA then holds a number of columns that is no multiple of 16, its last 64-column atom is
+    partly used, and the epilogue's 16-column units no longer pair up."""
+    torch, ubp = env
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 7 * M + C, Nc=Nc, x_dist="normal", relu=True)
+    Yh, Yref, A, plan = run_spmm(env, L, 34 + {2: 1, 4: 2}[Nb])
+    kernel, rows, cols = plan.tile_choice(Nc)
+    assert kernel == 2
+    if sms == 148:
+        assert cols % 32 == 16, (rows, cols)
+    check(Yh, Yref, A, L, variant=36)
+
+
 def test_tensor_core_variant_ragged_unaligned_and_auto(env):
     torch, ubp = env
     # ragged last strip on the fast path, then operands the fast path cannot take (falls back to the embedded
