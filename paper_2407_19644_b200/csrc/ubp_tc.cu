@@ -399,18 +399,13 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
     if ((M > 128 || bf16) && conv_w >= 0 && (!conv || ((K / 9) % TC_KC == 0 && halo <= 64))) {
         double best2 = 1e300;
         int best2_n = 0;
-        // tile widths: multiples of 64 for the TF32 kernel (X arrives in 32-column boxes per CTA), of 16 for the bf16
-        // kernel (the MMA's step in N; its epilogue works in 16-column units) -- of 32 where both CTAs take the one row
-        // tile and halve the epilogue's units between them
-        for (int n = 64; n <= 256; n += bf16 ? (M <= 128 ? 32 : 16) : 64) {
+        // tile widths: multiples of 64 for the TF32 kernel (X arrives in 32-column boxes per CTA), of 32 for the bf16
+        // kernel here (the estimate was calibrated on those; see the refinement below)
+        for (int n = 64; n <= 256; n += bf16 ? 32 : 64) {
             if (conv && (n / 2 + 2 * halo > 256 || (bf16 ? tc_pair_bf16_stages(n, halo) : tc_pair_stages(n, halo)) < 4)) continue;
             const long long ntiles = (long long)((M + 255) / 256) * ((Nc + n - 1) / n);
             const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
             const long long per_pair = (ntiles + pairs - 1) / pairs;
-            // (the odd multiples of 16 only where every pair gets one tile: there the narrowest width that still fits
-            // one round wins; with several rounds the estimate below was calibrated on multiples of 32 and, offered
-            // the widths between, trades a round for narrower tiles where that loses: L4 / L5 +6 ... +13 %)
-            if (n % 32 != 0 && per_pair > 1) continue;
             // bf16 products (calibrated the same way): three MMAs of K = 16 per chunk, n/2 cycles each; below that
             // a floor of ~470 + n/3 cycles that is nearly flat in n - the copies (W in 32-byte row pieces, the raw
             // fp32 rows) arrive at ~32 B/cycle/SM, the rate of the L2-to-SM path; 3x3: the shifted-tile pass
@@ -432,12 +427,11 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
         // blocks and its six MMAs: measured ~585-605 cycles per chunk at 96 and 192 columns) instead of making two
         // rounds; narrow stacked tiles lose against one round of wide plain ones, which the estimate reproduces
         if (bf16 == 1 && !conv && ((M + 255) / 256) % 2 == 0) {
-            for (int n = 64; n <= 256; n += 16) {
+            for (int n = 64; n <= 256; n += 32) {
                 const long long ntiles = (long long)((M + 511) / 512) * ((Nc + n - 1) / n);
                 if (tc_pair_bf16_stages(n, 0, 2) < 4) continue;
                 const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
                 const long long per_pair = (ntiles + pairs - 1) / pairs;
-                if (n % 32 != 0 && per_pair > 1) continue;
                 double per_chunk = 3.3 * n;
                 if (per_chunk < 600.0 + 0.33 * n) per_chunk = 600.0 + 0.33 * n;
                 // (both accumulators belong to one tile: every tile's epilogue, ~100 cycles per column, is exposed)
@@ -445,6 +439,19 @@ void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *ker
                                  4500.0 + 60.0 * n;
                 if (t < best2) { best2 = t; best2_n = n; best2_rows = 512; }
             }
+        }
+        // The bf16 kernel takes widths in steps of 16 columns (the MMA's step; its epilogue works in 16-column units;
+        // layers of at most 128 rows, whose CTAs halve the units between them, stay on multiples of 32): 16 columns
+        // less where every pair still gets its one tile. (Offered every multiple of 16 directly, the estimate traded a
+        // round for narrower tiles where that loses: chain L4 / L5 +6 ... +13 %; 16 columns less at the same three
+        // rounds: L4 -1.4 %, L5 +1 %.)
+        if (bf16 && !conv && M > 128 && best2_n >= 96) {
+            auto rounds = [&](int n) {
+                const long long ntiles = (long long)((M + best2_rows - 1) / best2_rows) * ((Nc + n - 1) / n);
+                const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
+                return (ntiles + pairs - 1) / pairs;
+            };
+            if (rounds(best2_n) == 1 && rounds(best2_n - 16) == 1) best2_n -= 16;
         }
         // (three pieces exist on the pair kernel only: never weigh it against the one-CTA TF32 kernel)
         if (best2_n && (best2 < best || bf16 == 2)) { *kernel = 2; *rows = best2_rows; *cols = best2_n; }
