@@ -458,6 +458,12 @@ int ubp_conv1x1_strided(const ubp_plan_t *plan, const float *in, int B, int H, i
     const int C = plan->dims.C;
     if (scratch_bytes < ubp_conv1x1_strided_scratch(C, B, H, Wd, stride)) return UBP_E_SPACE;
     const int Ho = (H - 1) / stride + 1, Wo = (Wd - 1) / stride + 1;
+    // stride 2, one channel-major product over all images, on the bf16 CTA-pair kernel: straight from the
+    // full-resolution input (its copies bring the even rows, its split pass takes every other pixel); no gather
+    if (stride == 2 && in_stride_b == hw && out_stride_b == (int64_t)Ho * Wo && out_stride_c >= (int64_t)B * Ho * Wo) {
+        const int rc = ubp::launch_spmm_tc_s2(plan, in, B, H, Wd, in_stride_c, bias, relu, out, out_stride_c, stream);
+        if (rc != UBP_E_UNSUPPORTED) return rc;
+    }
     float *xs = static_cast<float *>(scratch);
     if (int rc = ubp::launch_subsample(in, C, B, H, Wd, in_stride_b, in_stride_c, stride, xs, stream)) return rc;
     return ubp_conv1x1(plan, xs, B, Ho, Wo, (int64_t)Ho * Wo, (int64_t)B * Ho * Wo, bias, relu, out, out_stride_b,

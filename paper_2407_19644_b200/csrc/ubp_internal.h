@@ -107,6 +107,9 @@ int launch_spmm(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, c
 void tc_choose(int M, int K, int64_t Nc, int conv_w, int bf16, int sms, int *kernel, int *rows, int *cols);
 int launch_spmm_tc(const ubp_plan *plan, const float *X, int64_t ldx, int64_t Nc, const float *bias, int relu,
                    float *Y, int64_t ldy, void *stream);
+// 1x1, stride 2, straight from the full-resolution input (bf16 CTA-pair kernel); UBP_E_UNSUPPORTED if not applicable
+int launch_spmm_tc_s2(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isc, const float *bias, int relu,
+                      float *out, int64_t ldy, void *stream);
 int launch_conv3x3_tc(const ubp_plan *plan, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,
                       const float *bias, int relu, float *out, int64_t out_ld, void *stream, int stride = 1);
 // tensor-core implicit GEMM when the plan and the layouts allow it (stride 1: CTA pairs where the operands qualify;

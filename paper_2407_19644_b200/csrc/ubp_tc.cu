@@ -354,6 +354,7 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
                         int M, int64_t Nc, int ntile, int sms, void *stream, int pieces, int mt);
 int tc_pair_bf16_stages(int ntile, int halo, int mt = 1);
 int tc_pair_bf16_sub(int K, int ntile, int halo, int pieces, int mt);
+int tc_pair_bf16_stages_sub(int ntile, int halo, int sub, int mt);
 
 // Tile choice for one launch: which kernel (1 = one CTA per tile, 2 = CTA pair per tile), tile rows and columns.
 // Each candidate's time is estimated as (waves over the SMs) x (chunks x cycles per chunk + a fixed per-tile cost)
@@ -551,6 +552,72 @@ int launch_spmm_tc(const ubp_plan *pl, const float *X, int64_t ldx, int64_t Nc, 
     TcArgs a{};
     a.X = X; a.ldx = ldx; a.conv = 0; a.bias = bias; a.Y = Y; a.ldy = ldy; a.Nc = Nc; a.K = pl->dims.C; a.relu = relu;
     return launch_tc_common(pl, a, static_cast<cudaStream_t>(stream_));
+}
+
+// 1x1 with stride 2 on the bf16 CTA-pair kernel WITHOUT a gathered copy of the input: the tensor map shows the input
+// [C][B][H][W] (rows contiguous over the images, H and W even) as (2 W floats of a row pair, B H / 2 row pairs, C); a box
+// of W floats x (tile columns / Wo) row pairs x the stage's channels brings the even rows, and the split pass takes
+// every other float. A CTA's half tile is whole output rows: NH a multiple of Wo (and of 8), N = 2 NH a multiple of 16.
+// UBP_E_UNSUPPORTED where the plan, the shapes or the alignment do not allow it (the caller then gathers first).
+int launch_spmm_tc_s2(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isc, const float *bias, int relu,
+                      float *out, int64_t ldy, void *stream_)
+{
+    const int M = pl->dims.M, K = pl->dims.C;
+    if (pl->cfg.kind != 2 || !cfg_bf16(pl->cfg) || cfg_pieces(pl->cfg) != 2 || pl->img.tc16_off == 0) return UBP_E_UNSUPPORTED;
+    if ((H & 1) || (Wd & 3) || Wd > 256 || isc % 4 != 0 || isc < (int64_t)B * H * Wd || ldy % 4 != 0) return UBP_E_UNSUPPORTED;
+    if (((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15) != 0) return UBP_E_UNSUPPORTED;
+    const int Ho = H / 2, Wo = Wd / 2;
+    const int64_t Nc = (int64_t)B * Ho * Wo;
+    if (Nc >= (1ll << 31) || (int64_t)B * H / 2 >= (1ll << 31)) return UBP_E_UNSUPPORTED;
+    int sms = 148, devid = 0;
+    if (cudaGetDevice(&devid) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, devid);
+    // half-tile widths: the multiples of lcm(Wo, 8) from 32 up to 128 columns
+    int unit = Wo;
+    while (unit % 8 != 0) unit += Wo;
+    if (unit > 128) return UBP_E_UNSUPPORTED;
+    const int nchunk = (K + TC_KC - 1) / TC_KC;
+    double best = 1e300;
+    int best_nh = 0, best_mt = 1;
+    for (int mt = 1; mt <= 2; ++mt) {
+        if (mt == 2 && (M <= 128 || ((M + 255) / 256) % 2 != 0)) continue;
+        for (int nh = unit; nh <= 128; nh += unit) {
+            if (nh < 32 || (M <= 128 && (2 * nh) % 32 != 0)) continue;      // tiles of 64 columns and more, as tc_choose
+            // (the raw rows are twice as long as the tile: `halo` = nh / 2 sizes them)
+            const int sub = tc_pair_bf16_sub(K, 2 * nh, nh / 2, 2, mt);
+            const int stages = tc_pair_bf16_stages_sub(2 * nh, nh / 2, sub, mt);
+            if (stages < 4) continue;
+            const int n = 2 * nh;
+            const long long ntiles = (long long)((M + 256 * mt - 1) / (256 * mt)) * ((Nc + n - 1) / n);
+            const long long pairs = ntiles < sms / 2 ? ntiles : sms / 2;
+            const long long per_pair = (ntiles + pairs - 1) / pairs;
+            // the estimate of tc_choose for plain and stacked tiles
+            double per_chunk = mt == 2 ? 3.3 * n : 1.65 * n;
+            const double floor_chunk = mt == 2 ? 600.0 + 0.33 * n : 470.0 + 0.33 * n;
+            if (per_chunk < floor_chunk) per_chunk = floor_chunk;
+            const double t = mt == 2 ? 4400.0 + (double)per_pair * (nchunk * per_chunk + 2500.0) + (double)(per_pair - 1) * 100.0 * n + 4500.0 + 60.0 * n
+                                     : 4400.0 + (double)per_pair * ((nchunk * per_chunk > 50.0 * n ? nchunk * per_chunk : 50.0 * n) + 2500.0) + 4500.0 + 30.0 * n;
+            if (t < best) { best = t; best_nh = nh; best_mt = mt; }
+        }
+    }
+    if (!best_nh) return UBP_E_UNSUPPORTED;
+#ifdef S2_FORCE_MT
+    best_mt = S2_FORCE_MT; best_nh = S2_FORCE_NH;
+#endif
+    const int sub = tc_pair_bf16_sub(K, 2 * best_nh, best_nh / 2, 2, best_mt);
+    CUtensorMap tmX;
+    const uint64_t dims[3] = {(uint64_t)(2 * Wd), (uint64_t)((int64_t)B * H / 2), (uint64_t)K};
+    const uint32_t box[3] = {(uint32_t)Wd, (uint32_t)(best_nh / Wo), (uint32_t)(TC_KC * sub)};
+    int rc;
+    if ((rc = encode_3d(&tmX, in, dims, (uint64_t)(2 * Wd) * 4, (uint64_t)isc * 4, box, CU_TENSOR_MAP_SWIZZLE_NONE))) return rc;
+    TcArgs a{};
+    a.X = in; a.ldx = isc; a.conv = 0; a.bias = bias; a.Y = out; a.ldy = ldy; a.Nc = Nc; a.K = K; a.relu = relu;
+    a.M = M;
+    a.status = reinterpret_cast<int *>(pl->dev);
+    a.rpc = 128;
+    a.dup = M <= 128 ? 1 : 0;
+    a.s2 = Wo;
+    const uint8_t *dev = static_cast<const uint8_t *>(pl->dev);
+    return launch_tc_pair_bf16(dev + pl->img.tc16_off, &tmX, 0, best_nh / 2, &a, M, Nc, 2 * best_nh, sms, stream_, 2, best_mt);
 }
 
 int launch_conv3x3_tc(const ubp_plan *pl, const float *in, int B, int H, int Wd, int64_t isb, int64_t isc,

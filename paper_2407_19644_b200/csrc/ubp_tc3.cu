@@ -253,7 +253,11 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         const uint32_t bar = smem_u32(&bar_full[st]);
         const int c0 = sg * SUB, nsub = nchunk - c0 < SUB ? nchunk - c0 : SUB;
         uint8_t *raw = smem + (size_t)st * stage_bytes + roff;
-        if constexpr (XMERGED) {
+        if (!CONV && a.s2) {
+            // stride 2: the even input rows of this CTA's NH / Wo output rows, all the stage's channels in one box
+            // (`halo` = NH / 2 here: it only sizes the raw rows, 2 NH floats per channel)
+            tma_load_3d(smem_u32(raw), &tmX, 0, xcol / a.s2, c0 * TC_KC, bar);
+        } else if constexpr (XMERGED) {
             tma_load_2d(smem_u32(raw), &tmX, xcol - halo, c0 * TC_KC, bar);
         } else {
 #pragma unroll
@@ -455,10 +459,11 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                 }
                 // (checked build: the columns this thread needs lie inside the raw rows, everything it reads inside the
                 // CTA's shared memory, its writes inside the x1 / x2 tiles)
-                if (mine && UBP_CHK_SMEM(sh >= 0 && (uint32_t)(8 * cg + sh + 8) * 4u <= raw_row &&
+                if (mine && UBP_CHK_SMEM(sh >= 0 && (uint32_t)((!CONV && a.s2 ? 16 * cg + 8 : 8 * cg + sh) + 8) * 4u <= raw_row &&
                                          (size_t)(raw - smem_raw) + 15u * raw_row + (uint32_t)((8 * cg + sh) & ~3) * 4u + 48u <= tc::dbg_dynamic_smem() &&
                                          dst + 16u * 128u <= xb, a.status)) {
-                    const int o = 8 * cg + sh, ob = o & ~3, r = o & 3;      // r is the same for every lane
+                    const bool s2 = !CONV && a.s2 != 0;
+                    const int o = s2 ? 16 * cg : 8 * cg + sh, ob = o & ~3, r = o & 3;      // r is the same for every lane
 #pragma unroll
                     for (int i = 0; i < 2; ++i) {
                         if (i >= nk) break;
@@ -466,7 +471,11 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                         const float4 q0 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4);
                         const float4 q1 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 16);
                         float v[8];
-                        if (!CONV || r == 0) {
+                        if (s2) {              // every other pixel of the even rows: floats 2 j of the copy
+                            const float4 q2 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 32);
+                            const float4 q3 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 48);
+                            v[0] = q0.x; v[1] = q0.z; v[2] = q1.x; v[3] = q1.z; v[4] = q2.x; v[5] = q2.z; v[6] = q3.x; v[7] = q3.z;
+                        } else if (!CONV || r == 0) {
                             v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w; v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
                         } else {
                             const float4 q2 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 32);
@@ -615,6 +624,7 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     return UBP_OK;
 }
 
+int tc_pair_bf16_stages_sub(int ntile, int halo, int sub, int mt) { return t3_stages(ntile / 2, halo, sub, 2, mt); }
 // how many pipeline stages the bf16 pair kernel gets for a tile width and halo
 int tc_pair_bf16_stages(int ntile, int halo, int mt) { return t3_stages(ntile / 2, halo, 1, 2, mt); }
 

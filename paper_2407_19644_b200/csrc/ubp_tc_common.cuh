@@ -196,6 +196,10 @@ struct TcArgs {
                              // each stores the whole rows of its own half of the tile's columns
     int mt;                  // bf16 CTA-pair kernel: 256-row MMA tiles a pair stacks on ONE staged activation tile
                              // (1, or 2 = tiles of 512 rows, one per pair); 0 means 1
+    int s2;                  // bf16 CTA-pair kernel, 1x1 with stride 2: output row length Wo (0 = ordinary product). The
+                             // tensor map then shows the input as (2 W floats of a row pair, row pair, channel) and a
+                             // box brings the EVEN rows of whole output rows: per channel, output column j of the tile
+                             // is float 2 j of the copy (W = 2 Wo); a CTA's columns are whole output rows
 };
 
 

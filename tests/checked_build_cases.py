@@ -63,6 +63,17 @@ def conv_case(M, C, Nb, p, B, H, Wd, variant, stride=1):
     return scaled_error(Y.cpu().numpy(), Yref, A), plan.variant
 
 
+def s2_case(M, C, Nb, p, B, H, Wd):
+    """1x1 with stride 2 read straight from the full-resolution input by the bf16 pair kernel."""
+    L = ubp_synth.make_layer("t", M, C, Nb, p, 3 * M + C, B=B, H=H, Wd=Wd, x_dist="normal")
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb), 36)
+    Y = ubp.ubp_conv1x1(plan, torch.from_numpy(L.X).cuda(), torch.from_numpy(L.bias).cuda(), True, stride=2)
+    plan.check()
+    xs = np.ascontiguousarray(L.X[:, :, ::2, ::2])
+    Yref, A = oracle.masked_matmul(L.W, L.mask, xs.reshape(C, -1), L.bias, relu=True)
+    return scaled_error(Y.cpu().numpy().reshape(M, -1), Yref, A), plan.variant
+
+
 def damaged_plan_is_reported():
     """Sparse kernel, one entry's channel index moved one past the staged tile: the checked build skips that panel's
     list and sets the status word; nothing else happens."""
@@ -110,6 +121,8 @@ def main():
         ("pair kernel, three pieces", lambda: spmm_case(300, 150, 4, 70, 544, 86)),
         ("pair kernel TF32", lambda: spmm_case(300, 150, 4, 70, 516, 32)),
         ("one-CTA TF32", lambda: spmm_case(128, 128, 4, 60, 388, 32)),
+        ("1x1 stride 2, straight from the input", lambda: s2_case(256, 64, 4, 70, 5, 28, 28)),
+        ("1x1 stride 2, stacked tiles, two chunks per stage", lambda: s2_case(512, 520, 4, 80, 3, 12, 20)),
         ("3x3 plain", lambda: conv_case(32, 32, 8, 80, 2, 14, 14, 0)),
         ("3x3 padded grid", lambda: conv_case(256, 32, 8, 60, 3, 14, 14, 64)),
         ("3x3 padded grid, odd image", lambda: conv_case(260, 32, 4, 70, 2, 9, 13, 65)),

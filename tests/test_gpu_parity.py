@@ -680,6 +680,33 @@ def test_stride_two_convolutions(env, layout, H, Wd):
         assert scaled_error(y, Yref, A) <= 1e-4
 
 
+@pytest.mark.parametrize("M,C,Nb,p,B,H,Wd", [(256, 64, 4, 70, 5, 28, 28), (1024, 512, 4, 80, 6, 28, 28), (512, 96, 2, 60, 9, 56, 56),
+                                             (128, 80, 4, 50, 4, 28, 28), (300, 40, 8, 60, 3, 8, 16), (256, 520, 4, 75, 7, 12, 20),
+                                             (260, 64, 4, 70, 2, 14, 14), (256, 64, 4, 70, 3, 28, 26)])
+def test_stride_two_1x1_without_gather(env, M, C, Nb, p, B, H, Wd):
+    """1x1 with stride 2 under a bf16 tensor-core plan, channel-major input with even H and W a multiple of 4: the
+    CTA-pair kernel reads the full-resolution input itself (boxes of the even rows, every other pixel in the split pass),
+    tiles of whole output rows; plain, stacked and duplicated-row tiles, one or two chunks per stage, a ragged last tile.
+    The last two shapes (W no multiple of 4) take the gathered copy instead. Against the oracle on the subsampled input;
+    the scratch buffer must stay untouched on the direct path."""
+    torch, ubp = env
+    L = ubp_synth.make_layer("s2", M, C, Nb, p, 9 * M + C + Wd, B=B, H=H, Wd=Wd, x_dist="normal")
+    plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, L.Nb), 34 + {2: 1, 4: 2, 8: 3}[Nb])
+    x = torch.from_numpy(L.X).cuda()                           # [C][B][H][W]
+    Ho, Wo = H // 2, Wd // 2
+    scratch = torch.full((C * B * Ho * Wo,), float("nan"), dtype=torch.float32, device="cuda")
+    y = ubp.ubp_conv1x1(plan, x, torch.from_numpy(L.bias).cuda(), True, stride=2, scratch=scratch)
+    torch.cuda.synchronize()
+    plan.check()
+    direct = Wd % 4 == 0
+    assert bool(torch.isnan(scratch).all()) == direct
+    xs = np.ascontiguousarray(L.X[:, :, ::2, ::2])
+    Yref, A = oracle.masked_matmul(L.W, L.mask, xs.reshape(C, -1), L.bias, relu=True)
+    yh = y.cpu().numpy().reshape(M, -1)
+    assert yh.shape == Yref.shape and np.isfinite(yh).all()
+    assert scaled_error(yh, Yref, A) <= 1e-4
+
+
 @pytest.mark.parametrize("M,C,Nb,p,B,H,Wd,stride", [(128, 32, 4, 60, 3, 14, 14, 2), (256, 48, 8, 70, 2, 28, 28, 2),
                                                       (200, 20, 4, 50, 2, 7, 9, 2), (130, 16, 2, 50, 1, 13, 12, 3),
                                                       (256, 64, 4, 80, 4, 8, 8, 2), (300, 32, 4, 60, 5, 7, 7, 2),
