@@ -284,7 +284,11 @@ int ubp_conv3x3_implicit(const ubp_plan_t *plan, const float *in, int B, int H, 
  * ubp_conv1x1_strided: out[b][o][yo][xo] = act(bias[o] + sum W[o][c] * in[b][c][yo*stride][xo*stride]). For
  *   stride > 1 the pixels read are first gathered into `scratch` (device, 16-byte aligned, at least
  *   ubp_conv1x1_strided_scratch(C, B, H, W, stride) bytes, channel-major [C][B][Ho][Wo]) by one extra kernel, then the
- *   stride-1 path runs on them. UBP_E_SPACE if the scratch is too small. */
+ *   stride-1 path runs on them. UBP_E_SPACE if the scratch is too small. Exception: stride 2 under a bf16 tensor-core
+ *   plan (variants 34..37), channel-major tensors (both batch strides equal to their plane size), H even, W a multiple
+ *   of 4, 16-byte aligned pointers and channel strides that are multiples of 4: the CTA-pair kernel reads the
+ *   full-resolution input itself (its copies bring the even rows, its split pass takes every other pixel) and
+ *   `scratch` is not touched (it must still be given: which path runs is the library's choice). */
 int ubp_conv3x3_strided(const ubp_plan_t *plan, const float *in, int B, int H, int Wd, int stride,
                         int64_t in_stride_b, int64_t in_stride_c, const float *bias, int relu,
                         float *out, int64_t out_stride_b, int64_t out_stride_c, void *stream);

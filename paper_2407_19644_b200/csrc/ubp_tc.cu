@@ -600,9 +600,6 @@ int launch_spmm_tc_s2(const ubp_plan *pl, const float *in, int B, int H, int Wd,
         }
     }
     if (!best_nh) return UBP_E_UNSUPPORTED;
-#ifdef S2_FORCE_MT
-    best_mt = S2_FORCE_MT; best_nh = S2_FORCE_NH;
-#endif
     const int sub = tc_pair_bf16_sub(K, 2 * best_nh, best_nh / 2, 2, best_mt);
     CUtensorMap tmX;
     const uint64_t dims[3] = {(uint64_t)(2 * Wd), (uint64_t)((int64_t)B * H / 2), (uint64_t)K};
