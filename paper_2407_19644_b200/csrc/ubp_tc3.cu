@@ -189,7 +189,9 @@ __device__ __forceinline__ void split8(const float (&v)[8], uint4 &h, uint4 &l)
     l = make_uint4(ll[0], ll[1], ll[2], ll[3]);
 }
 
-template <bool CONV, int SUB, int NP>
+// (S2: the 1x1 product with stride 2 read straight from the full-resolution input, see TcArgs::s2 -- an instance of its
+// own: as a run-time branch it cost the ordinary kernel's split pass 1.5 - 4 %)
+template <bool CONV, int SUB, int NP, bool S2 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T3_THREADS, 1)
 ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensorMap tmX, const TcArgs a,
                const int halo, const int nrp, const int ntiles)
@@ -253,7 +255,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
         const uint32_t bar = smem_u32(&bar_full[st]);
         const int c0 = sg * SUB, nsub = nchunk - c0 < SUB ? nchunk - c0 : SUB;
         uint8_t *raw = smem + (size_t)st * stage_bytes + roff;
-        if (!CONV && a.s2) {
+        if constexpr (S2) {
             // stride 2: the even input rows of this CTA's NH / Wo output rows, all the stage's channels in one box
             // (`halo` = NH / 2 here: it only sizes the raw rows, 2 NH floats per channel)
             tma_load_3d(smem_u32(raw), &tmX, 0, xcol / a.s2, c0 * TC_KC, bar);
@@ -459,10 +461,10 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                 }
                 // (checked build: the columns this thread needs lie inside the raw rows, everything it reads inside the
                 // CTA's shared memory, its writes inside the x1 / x2 tiles)
-                if (mine && UBP_CHK_SMEM(sh >= 0 && (uint32_t)((!CONV && a.s2 ? 16 * cg + 8 : 8 * cg + sh) + 8) * 4u <= raw_row &&
+                if (mine && UBP_CHK_SMEM(sh >= 0 && (uint32_t)((S2 ? 16 * cg + 8 : 8 * cg + sh) + 8) * 4u <= raw_row &&
                                          (size_t)(raw - smem_raw) + 15u * raw_row + (uint32_t)((8 * cg + sh) & ~3) * 4u + 48u <= tc::dbg_dynamic_smem() &&
                                          dst + 16u * 128u <= xb, a.status)) {
-                    const bool s2 = !CONV && a.s2 != 0;
+                    constexpr bool s2 = S2;
                     const int o = s2 ? 16 * cg : 8 * cg + sh, ob = o & ~3, r = o & 3;      // r is the same for every lane
 #pragma unroll
                     for (int i = 0; i < 2; ++i) {
@@ -471,7 +473,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                         const float4 q0 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4);
                         const float4 q1 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 16);
                         float v[8];
-                        if (s2) {              // every other pixel of the even rows: floats 2 j of the copy
+                        if constexpr (s2) {    // every other pixel of the even rows: floats 2 j of the copy
                             const float4 q2 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 32);
                             const float4 q3 = *reinterpret_cast<const float4 *>(raw + k * raw_row + ob * 4 + 48);
                             v[0] = q0.x; v[1] = q0.z; v[2] = q1.x; v[3] = q1.z; v[4] = q2.x; v[5] = q2.z; v[6] = q3.x; v[7] = q3.z;
@@ -585,13 +587,15 @@ int launch_tc_pair_bf16(const void *W16, const CUtensorMap_st *tmX, int conv, in
     if (t3_stages(nh, halo, sub, pieces, mt) < 4) return UBP_E_UNSUPPORTED;
     size_t smem = (size_t)t3_stages(nh, halo, sub, pieces, mt) * t3_stage_bytes(nh, halo, sub, pieces, mt) + 1024;
     if (smem < TC_PAIR_MIN_SMEM) smem = TC_PAIR_MIN_SMEM;   // one CTA per SM, whatever the tile width (see the constant)
-    static bool done[5][64] = {};
+    static bool done[7][64] = {};
     int devid = 0;
     if (cudaGetDevice(&devid) != cudaSuccess) devid = -1;
-    const int which = pieces == 3 ? 4 : (conv ? 2 : 0) + (sub == 2 ? 1 : 0);
+    if (a.s2 && (conv || pieces != 2)) return UBP_E_UNSUPPORTED;
+    const int which = a.s2 ? 5 + (sub == 2 ? 1 : 0) : pieces == 3 ? 4 : (conv ? 2 : 0) + (sub == 2 ? 1 : 0);
     using KernelFn = void (*)(const uint8_t *, const CUtensorMap, const TcArgs, const int, const int, const int);
-    const KernelFn kernels[5] = {ubp_tc3_kernel<false, 1, 2>, ubp_tc3_kernel<false, 2, 2>, ubp_tc3_kernel<true, 1, 2>,
-                                 ubp_tc3_kernel<true, 2, 2>, ubp_tc3_kernel<false, 1, 3>};
+    const KernelFn kernels[7] = {ubp_tc3_kernel<false, 1, 2>, ubp_tc3_kernel<false, 2, 2>, ubp_tc3_kernel<true, 1, 2>,
+                                 ubp_tc3_kernel<true, 2, 2>, ubp_tc3_kernel<false, 1, 3>,
+                                 ubp_tc3_kernel<false, 1, 2, true>, ubp_tc3_kernel<false, 2, 2, true>};
     const KernelFn kern = kernels[which];
     if (devid < 0 || devid >= 64 || !done[which][devid]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(T3_PIPE_BUDGET + 1024));
