@@ -330,7 +330,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                 for (int sg = 0; sg < nstage; ++sg, ++f) {
                     if (f < npre) continue;
                     if (round > 0) {                       // the stage's previous contents must have been consumed
-                        ok = mbar_wait_relaxed(smem_u32(&bar_empty[st]), (uint32_t)(round - 1) & 1u, &abort_flag);
+                        ok = mbar_wait(smem_u32(&bar_empty[st]), (uint32_t)(round - 1) & 1u, &abort_flag);   // polling: one lane per warp
                         if (!ok) break;
                     }
                     if (what == 1) issue_x(sg, st, xcol);
