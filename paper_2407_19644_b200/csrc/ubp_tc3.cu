@@ -13,8 +13,12 @@
 // fp32 activations any more, so TMA copies the chunk's 16 channel rows as they are (plus a halo for 3x3) and the
 // pass warps write BOTH x1 and x2, in the MN-major bf16 operand layout (64 columns x 8 channels atoms in the
 // 128-byte swizzle; LBO = next 64 columns, SBO = next 8 channels); a pipeline stage holds one or two chunks
-// (template parameter SUB). Thread roles, barriers, persistence, the two accumulators and the epilogue are those of
-// ubp_tc2.cu.
+// (template parameter SUB), laid out by kind so that the weight blocks of its chunks arrive in one bulk copy and
+// (1x1) their channel rows in one box; three threads issue the copies (lane 0 of warp 0 and of two extra warps after
+// the epilogue warps); a pair may stack two 256-row MMA tiles on one staged activation tile (TcArgs::mt); layers of
+// at most 128 rows run both CTAs on the one row tile (TcArgs::dup); a 1x1 with stride 2 reads the full-resolution
+// input itself (template parameter S2, TcArgs::s2). Barriers, persistence, the two accumulators and the epilogue
+// are those of ubp_tc2.cu.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
