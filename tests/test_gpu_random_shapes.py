@@ -81,3 +81,45 @@ def test_random_3x3_layers(env, seed):
         assert scaled_error(Yh, Yref, A) <= TOL, what
         kernels.add(plan.tile_choice_conv(B, H, Wd, stride)[0])
     assert len(kernels) >= 3
+
+
+@pytest.mark.parametrize("seed", [31])
+def test_random_stride_two_1x1_layers(env, seed):
+    """1x1 with stride 2 on random shapes and both layouts: whichever path the library takes (the CTA-pair kernel reading
+    the full-resolution input itself, or the gathered copy first), against the oracle on the subsampled input."""
+    torch, ubp = env
+    rng = np.random.default_rng(seed)
+    paths = set()
+    for it in range(40):
+        Nb = int(rng.choice([2, 4, 8]))
+        M = max(Nb, int(rng.choice([rng.integers(16, 130), rng.integers(129, 600), rng.choice([256, 512, 1024, 768])])))
+        C = int(rng.choice([rng.integers(16, 100), rng.integers(64, 300), rng.choice([512, 520, 64, 128])]))
+        H = int(rng.choice([4, 8, 12, 14, 16, 28, 56, 7]))
+        Wd = int(rng.choice([4, 8, 12, 16, 20, 28, 56, 14, 6]))
+        B = int(rng.integers(1, 9))
+        if M * C * B * H * Wd // 4 > 1.5e9:
+            B = 1
+        p = int(rng.integers(30, 95))
+        relu = bool(it & 1)
+        L = ubp_synth.make_layer("f", M, C, Nb, p, 100 * seed + it, B=B, H=H, Wd=Wd, x_dist="normal")
+        plan = ubp.Plan(ubp.ubp_pack(L.W, L.mask, Nb), int(rng.choice([0, 34 + {2: 1, 4: 2, 8: 3}[Nb]])))
+        layout = str(rng.choice(["CNHW", "NCHW"]))
+        x = torch.from_numpy(L.X).cuda()
+        if layout == "NCHW":
+            x = x.permute(1, 0, 2, 3).contiguous()
+        Ho, Wo = (H - 1) // 2 + 1, (Wd - 1) // 2 + 1
+        scratch = torch.full((C * B * Ho * Wo,), float("nan"), dtype=torch.float32, device="cuda")
+        y = ubp.ubp_conv1x1(plan, x, torch.from_numpy(L.bias).cuda(), relu, stride=2, scratch=scratch, layout=layout)
+        torch.cuda.synchronize()
+        plan.check()
+        paths.add(bool(torch.isnan(scratch).all()))
+        y = y.cpu().numpy()
+        if layout == "NCHW":
+            y = y.transpose(1, 0, 2, 3)
+        xs = np.ascontiguousarray(L.X[:, :, ::2, ::2])
+        Yref, A = oracle.masked_matmul(L.W, L.mask, xs.reshape(C, -1), L.bias, relu=relu)
+        yh = y.reshape(M, -1)
+        what = (M, C, Nb, p, B, H, Wd, layout, plan.variant)
+        assert yh.shape == Yref.shape and np.isfinite(yh).all(), what
+        assert scaled_error(yh, Yref, A) <= TOL, what
+    assert paths == {True, False}                 # both the direct and the gathered path came up
