@@ -193,6 +193,16 @@ __device__ __forceinline__ void split8(const float (&v)[8], uint4 &h, uint4 &l)
     l = make_uint4(ll[0], ll[1], ll[2], ll[3]);
 }
 
+// four fp32 -> bf16 heads and bf16 remainders, packed two per word
+__device__ __forceinline__ void split4(const float4 &v, uint2 &h, uint2 &l)
+{
+    const __nv_bfloat162 a0 = __floats2bfloat162_rn(v.x, v.y), a1 = __floats2bfloat162_rn(v.z, v.w);
+    const float2 f0 = __bfloat1622float2(a0), f1 = __bfloat1622float2(a1);
+    const __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x - f0.x, v.y - f0.y), b1 = __floats2bfloat162_rn(v.z - f1.x, v.w - f1.y);
+    h = make_uint2(*reinterpret_cast<const uint32_t *>(&a0), *reinterpret_cast<const uint32_t *>(&a1));
+    l = make_uint2(*reinterpret_cast<const uint32_t *>(&b0), *reinterpret_cast<const uint32_t *>(&b1));
+}
+
 // (S2: the 1x1 product with stride 2 read straight from the full-resolution input, see TcArgs::s2 -- an instance of its
 // own: as a run-time branch it cost the ordinary kernel's split pass 1.5 - 4 %)
 template <bool CONV, int SUB, int NP, bool S2 = false>
@@ -463,6 +473,38 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                     chu += TC_KC;
                     if (chu >= Cin) { chu = 0; ++tpu; }
                 }
+                if (!CONV && !S2 && NP == 2 && !narrow) {
+                    // 1x1, more than 64 columns per CTA: thread (j, kq) takes the 16-byte pieces j and 16 + j of its
+                    // rows -- columns 4 j .. 4 j + 3 of both 64-column atoms -- so that eight neighbouring threads read
+                    // 128 contiguous bytes (eight columns per thread = 32-byte steps cost every 128-bit load two
+                    // wavefronts: 37 % of the kernel's shared-memory wavefronts were such conflicts) and a half warp's
+                    // 8-byte stores fill one 128-byte row of an atom
+                    const uint32_t j = (uint32_t)cg;
+                    const bool has2 = 64 + 4 * (int)j < NH;
+                    // (checked build: the last byte this thread reads lies inside its raw rows and the CTA's shared memory,
+                    // its writes inside the two atoms of the x1 / x2 tiles)
+                    const uint32_t rd_end = (has2 ? 256u : 0u) + j * 16u + 16u;
+                    if (UBP_CHK_SMEM(rd_end <= raw_row && (size_t)(raw - smem_raw) + 15u * raw_row + rd_end <= tc::dbg_dynamic_smem() &&
+                                     2u * T3_ATOM <= xb, a.status)) {
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            const int k = kq + 8 * i;
+                            const uint8_t *rowp = raw + k * raw_row;
+                            const float4 qa = *reinterpret_cast<const float4 *>(rowp + j * 16u);
+                            uint2 h, l;
+                            split4(qa, h, l);
+                            const uint32_t off = (uint32_t)k * 128u + (((j >> 1) ^ ((uint32_t)k & 7u)) << 4) + (j & 1u) * 8u;
+                            *reinterpret_cast<uint2 *>(x1 + off) = h;
+                            *reinterpret_cast<uint2 *>(x1 + xb + off) = l;
+                            if (has2) {
+                                const float4 qb = *reinterpret_cast<const float4 *>(rowp + 256u + j * 16u);
+                                split4(qb, h, l);
+                                *reinterpret_cast<uint2 *>(x1 + T3_ATOM + off) = h;
+                                *reinterpret_cast<uint2 *>(x1 + xb + T3_ATOM + off) = l;
+                            }
+                        }
+                    }
+                } else
                 // (checked build: the columns this thread needs lie inside the raw rows, everything it reads inside the
                 // CTA's shared memory, its writes inside the x1 / x2 tiles)
                 if (mine && UBP_CHK_SMEM(sh >= 0 && (uint32_t)((S2 ? 16 * cg + 8 : 8 * cg + sh) + 8) * 4u <= raw_row &&
