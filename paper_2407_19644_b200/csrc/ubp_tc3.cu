@@ -93,7 +93,8 @@ __device__ __forceinline__ uint32_t make_idesc3(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
-// One chunk's three MMAs (K = 16 each: w1 x1, w2 x1, w1 x2) and, after a stage's last chunk (`last`), the commit that
+// One chunk's three MMAs (K = 16 each: w1 x1, w1 x2, w2 x1; the second takes w1 from the tensor core's operand collector,
+// where the first left it, instead of reading it from shared memory again -- shared memory is this kernel's wall) and, after a stage's last chunk (`last`), the commit that
 // hands the stage back to both CTAs, in a single statement, with a non-blocking test of the NEXT stage's barrier
 // issued first and its result read last. Executed by a whole converged warp: one elected lane issues. Returns
 // whether the next stage is ready.
@@ -112,9 +113,9 @@ __device__ __forceinline__ bool mma3_chunk(uint32_t d_tmem, uint64_t dW1, uint64
         "setp.eq.b32 pt, %10, 0;\n\t"
         "cvt.u64.u32 w2, %4;\n\tadd.s64 w2, w2, %2;\n\t"
         "cvt.u64.u32 x2, %5;\n\tadd.s64 x2, x2, %3;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %6, pa;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16.collector::a::fill [%1], %2, %3, %6, pa;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16.collector::a::lastuse [%1], %2, x2, %6, pt;\n\t"
         "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w2, %3, %6, pt;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, x2, %6, pt;\n\t"
         "@pc tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%11], %12;\n\t"
         "selp.u32 %0, 1, 0, pn;\n\t}"
         : "=r"(ready)
@@ -141,12 +142,12 @@ __device__ __forceinline__ bool mma6_chunk(uint32_t d_tmem, uint64_t dW1, uint64
         "setp.eq.b32 pt, %10, 0;\n\t"
         "cvt.u64.u32 ws, %4;\n\tadd.s64 w2, ws, %2;\n\tadd.s64 w3, w2, ws;\n\t"
         "cvt.u64.u32 xs, %5;\n\tadd.s64 x2, xs, %3;\n\tadd.s64 x3, x2, xs;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %6, pa;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w2, %3, %6, pt;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, x2, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16.collector::a::fill [%1], %2, %3, %6, pa;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16.collector::a::use [%1], %2, x2, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16.collector::a::lastuse [%1], %2, x3, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16.collector::a::fill [%1], w2, %3, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16.collector::a::lastuse [%1], w2, x2, %6, pt;\n\t"
         "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w3, %3, %6, pt;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], w2, x2, %6, pt;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::f16 [%1], %2, x3, %6, pt;\n\t"
         "@pc tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%11], %12;\n\t"
         "selp.u32 %0, 1, 0, pn;\n\t}"
         : "=r"(ready)
