@@ -105,13 +105,14 @@ __device__ __forceinline__ bool mma2_chunk(uint32_t d_tmem, uint64_t dWh, uint64
         "setp.eq.b32 pt, %10, 0;\n\t"
         "cvt.u64.u32 wl, %4;\n\tadd.s64 wl, wl, %2;\n\t"
         "cvt.u64.u32 xl, %5;\n\tadd.s64 xl, xl, %3;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::tf32 [%1], %2, %3, %6, pa;\n\t"
+        // (Wh is used twice per 8 channels: the second product takes it from the tensor core's operand collector)
+        "@pe tcgen05.mma.cta_group::2.kind::tf32.collector::a::fill [%1], %2, %3, %6, pa;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::tf32.collector::a::lastuse [%1], %2, xl, %6, pt;\n\t"
         "@pe tcgen05.mma.cta_group::2.kind::tf32 [%1], wl, %3, %6, pt;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::tf32 [%1], %2, xl, %6, pt;\n\t"
         "add.s64 wh, %2, 2;\n\tadd.s64 wl, wl, 2;\n\tadd.s64 xh, %3, 64;\n\tadd.s64 xl, xl, 64;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::tf32 [%1], wh, xh, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::tf32.collector::a::fill [%1], wh, xh, %6, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::tf32.collector::a::lastuse [%1], wh, xl, %6, pt;\n\t"
         "@pe tcgen05.mma.cta_group::2.kind::tf32 [%1], wl, xh, %6, pt;\n\t"
-        "@pe tcgen05.mma.cta_group::2.kind::tf32 [%1], wh, xl, %6, pt;\n\t"
         "@pe tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%11], %12;\n\t"
         "selp.u32 %0, 1, 0, pn;\n\t}"
         : "=r"(ready)
