@@ -484,7 +484,7 @@ ubp_tc3_kernel(const uint8_t *__restrict__ W16, const __grid_constant__ CUtensor
                     const bool has2 = 64 + 4 * (int)j < NH;
                     // (checked build: the last byte this thread reads lies inside its raw rows and the CTA's shared memory,
                     // its writes inside the two atoms of the x1 / x2 tiles)
-                    const uint32_t rd_end = (has2 ? 256u : 0u) + j * 16u + 16u;
+                    [[maybe_unused]] const uint32_t rd_end = (has2 ? 256u : 0u) + j * 16u + 16u;
                     if (UBP_CHK_SMEM(rd_end <= raw_row && (size_t)(raw - smem_raw) + 15u * raw_row + rd_end <= tc::dbg_dynamic_smem() &&
                                      2u * T3_ATOM <= xb, a.status)) {
 #pragma unroll
