@@ -175,7 +175,8 @@ int ubp_plan_info(const ubp_plan_t *plan, ubp_plan_info_t *info);
  * 1 = tensor-core kernel with one CTA per tile, 2 = tensor-core kernel with a CTA pair per tile, 3 = the comparison
  * kernels that walk the canonical arrays in the paper's own dataflow (variants 60 and 61; tile_rows is 0).
  * tile_rows is 256 for the CTA-pair kernel, or 512 where a pair stacks two 256-row MMA tiles on one staged activation
- * tile (layers whose rows fill whole 512-row tiles and whose tiles then number at most one per pair). Host only;
+ * tile (layers whose rows fill whole 512-row tiles, where the tile estimate prefers that); tile_cols of the CTA-pair
+ * kernels is a multiple of 16 (bf16 products) or 64 (TF32 products), at most 256. Host only;
  * enqueues nothing. Not part of the paper's method: it exists so that measurements and tests can name what ran. */
 int ubp_plan_tile_choice(const ubp_plan_t *plan, int64_t Nc, int image_width, int *kernel, int *tile_rows,
                          int *tile_cols);
